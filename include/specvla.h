@@ -1,0 +1,207 @@
+/*
+ * specvla.h - C ABI of the B200 (sm_100a) tree-verification path of Spec-VLA.
+ *
+ * The library runs the hot path of Spec-VLA decoding (Algorithm 1, Appendix B) for an
+ * OpenVLA-style Llama decoder: prefill, the Eagle-style one-layer draft model M_D (Eq. 2,
+ * Eq. 5), one verification forward of M_V over all draft-tree rows under a tree mask
+ * (Section 3.2 / 4.1), greedy argmax (Eq. 1), relaxed acceptance (Eq. 4, Section 4.3),
+ * longest-accepted-path selection and KV-cache compaction.
+ *
+ * Conventions
+ *  - Every function returns 0 on success or a negative SPECVLA_ERR_* code; nothing throws.
+ *  - "device" pointers are CUDA device memory of the current device; "host" pointers are
+ *    ordinary host memory. The caller owns every buffer it passes in; the library owns
+ *    only the host-side context object and a few KB of pinned staging memory.
+ *  - All weights are bfloat16, row-major [out_features, in_features]; RMSNorm gains are
+ *    float32. The workspace (KV caches, activations, split-K scratch) is one device buffer
+ *    allocated by the caller, at least specvla_workspace_bytes() long, 1024-byte aligned;
+ *    it must outlive the context and must not be touched while a call is in flight.
+ *  - Work is enqueued on `stream` (a cudaStream_t passed as void*). Calls that return
+ *    values through host pointers synchronise that stream before returning.
+ *  - One context per host thread; calls on one context must not overlap.
+ *  - There is no CPU fallback: creation fails with SPECVLA_ERR_UNSUPPORTED_ARCH unless the
+ *    current device is compute capability 10.x.
+ */
+#ifndef SPECVLA_H
+#define SPECVLA_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SPECVLA_OK                     0
+#define SPECVLA_ERR_INVALID_ARG       -1   /* NULL pointer, size out of range */
+#define SPECVLA_ERR_CAPACITY          -2   /* rows / slots / episodes exceed the context's capacity */
+#define SPECVLA_ERR_BAD_TREE          -3   /* parent[i] >= i, wrong depth, parent[0] != -1 ... */
+#define SPECVLA_ERR_BAD_STATE         -4   /* episode not prefilled, nothing pending ... */
+#define SPECVLA_ERR_CUDA              -5   /* a CUDA call failed; see specvla_last_cuda_error */
+#define SPECVLA_ERR_TIMEOUT           -6   /* a bounded device-side wait gave up */
+#define SPECVLA_ERR_UNSUPPORTED_ARCH  -7   /* not an sm_100 device */
+
+#define SPECVLA_MAX_TREE_ROWS   128        /* rows of one verification tree, root included */
+#define SPECVLA_MAX_DEPTH       8          /* deepest draft level */
+#define SPECVLA_MAX_BRANCH      8          /* children per expanded node */
+
+typedef struct specvla_ctx specvla_ctx;
+
+/* Model and capacity description (Section 4.1: Llama decoder; Section 4.3: 256 action bins). */
+typedef struct {
+  int n_layers, d_model, n_heads, head_dim, d_ffn, vocab;
+  int action_base;      /* token id of action bin 0; bins are ids action_base .. action_base+n_bins-1 */
+  int n_bins;           /* 256 */
+  float rms_eps;        /* 1e-6 */
+  float rope_theta;     /* 1e4 */
+  int max_seq;          /* KV slots per episode: committed positions + rows of the tree in flight */
+  int max_episodes;     /* episodes with their own KV caches */
+  int max_rows;         /* rows of one forward call summed over its episodes (prefill sets this) */
+  int action_only;      /* 1: greedy argmax and draft top-k range over the action ids only */
+} specvla_model_desc;
+
+/* Target (verification) model weights. Per-layer members are HOST arrays of n_layers DEVICE
+ * pointers. wqkv = [Wq; Wk; Wv] stacked [3*H*dh, d]; wgu = [Wgate; Wup] stacked [2F, d]. */
+typedef struct {
+  const void *embed;              /* bf16 [vocab, d] */
+  const void *lm_head;            /* bf16 [vocab, d] */
+  const float *final_norm;        /* f32 [d] */
+  const void *const *wqkv;        /* bf16 [3*H*dh, d] */
+  const void *const *wo;          /* bf16 [d, H*dh] */
+  const void *const *wgu;         /* bf16 [2F, d] */
+  const void *const *wd;          /* bf16 [d, F] */
+  const float *const *norm1;      /* f32 [d] */
+  const float *const *norm2;      /* f32 [d] */
+} specvla_weights;
+
+/* Draft model M_D (Eq. 2): fc over [feature ; token embedding] + one decoder layer. It shares
+ * the target's embedding and LM head. May be NULL at creation when only caller-supplied
+ * trees are verified. */
+typedef struct {
+  const void *fc;                 /* bf16 [d, 2d] */
+  const void *wqkv, *wo, *wgu, *wd;
+  const float *norm1, *norm2;
+} specvla_draft_weights;
+
+/* Static-size draft tree (Section 4.1, Eagle-2 style): level l (0-based) expands the
+ * expand[l] best nodes of level l-1 (expand[0] must be 1: the root) into branch[l] children
+ * each. depth = 0 means no drafting: every iteration is one plain autoregressive step. */
+typedef struct {
+  int depth;
+  int branch[SPECVLA_MAX_DEPTH];
+  int expand[SPECVLA_MAX_DEPTH];
+} specvla_tree_shape;
+
+/* One draft tree in HOST memory. Row 0 is the root (the last emitted token, not yet in the
+ * target's cache): parent[0] = -1, depth[0] = 0, parent[i] < i, depth[i] = depth[parent[i]]+1.
+ * tokens[0] may be -1 to take the root token from the episode's state. score may be NULL. */
+typedef struct {
+  int n_rows;
+  int *tokens;
+  int *parent;
+  int *depth;
+  float *score;
+} specvla_tree;
+
+typedef struct {
+  int iterations;                 /* draft+verify iterations run (max over episodes) */
+  int tokens_emitted;             /* before clipping, first episode */
+  int accept_len[16];             /* accepted draft tokens m of the first 16 iterations, first episode */
+  float ms_prefill, ms_draft, ms_verify;   /* device time, CUDA events */
+} specvla_stats;
+
+/* Bytes of device workspace a context of this description needs. 0 on invalid description. */
+size_t specvla_workspace_bytes(const specvla_model_desc *desc);
+
+/* Creates a context. `workspace` (device) is carved into KV caches and activations and
+ * zero-initialised where needed on `stream`-0. draft may be NULL. */
+int specvla_create(const specvla_model_desc *desc, const specvla_weights *target,
+                   const specvla_draft_weights *draft, void *workspace, size_t workspace_bytes,
+                   specvla_ctx **out);
+int specvla_destroy(specvla_ctx *ctx);
+
+/* Forgets an episode's state (its caches are simply overwritten by the next prefill). */
+int specvla_reset(specvla_ctx *ctx, int episode);
+
+/* Prefill (Section 4.1): causal forward of M_V over each episode's prefix, the first token
+ * a_1 = greedy token of the last row (Eq. 1), and M_D over the shifted (feature_i, input_{i+1})
+ * pairs to fill the draft cache.
+ *   episodes   host [n_ep]        distinct episode ids in [0, max_episodes)
+ *   embeds     device bf16 [sum(lens), d]  row used where token_ids[row] < 0
+ *   token_ids  host [sum(lens)]   >= 0: the row is that id's embedding
+ *   lens       host [n_ep]        prefix length of each episode, >= 1
+ *   first_token_out  host [n_ep], may be NULL
+ *   logits_out device f32 [n_ep, vocab] logits of each episode's last row, may be NULL */
+int specvla_prefill(specvla_ctx *ctx, int n_ep, const int *episodes, const void *embeds,
+                    const int *token_ids, const int *lens, int *first_token_out,
+                    float *logits_out, void *stream);
+
+/* Draft phase (Algorithm 1, inner loop; Eq. 2): runs M_D on the rows pending since the last
+ * commit, then grows the static-size tree level by level from M_D's top-k tokens. The tree
+ * stays on the device for the next specvla_verify_tree(trees = NULL).
+ *   trees_out  host [n_ep], may be NULL; each entry's arrays must hold 1 + sum(branch*expand)
+ *              rows; n_rows is written. */
+int specvla_draft_tree(specvla_ctx *ctx, int n_ep, const int *episodes,
+                       const specvla_tree_shape *shape, specvla_tree *trees_out, void *stream);
+
+/* Verification (Algorithm 1; Eq. 3 / Eq. 4): one forward of M_V over all tree rows (row i at
+ * position P + depth[i], attending the committed cache, its ancestors and itself), greedy
+ * token per row, acceptance of node i when |bin(tokens[i]) - bin(g[parent[i]])| <= r and its
+ * parent is accepted (ids outside the action bins must match exactly), choice of the deepest
+ * accepted node (ties: lowest row), compaction of the accepted rows' K/V next to the root,
+ * and set-up of the next iteration's state.
+ *   trees          host [n_ep] caller-supplied trees, or NULL to verify the trees left by
+ *                  specvla_draft_tree
+ *   r              relaxation threshold >= 0 (0 = strict matching)
+ *   accept_len_out host [n_ep]: m, the number of accepted draft tokens
+ *   tokens_out     host [n_ep][SPECVLA_MAX_DEPTH+1]: the m accepted draft tokens, then the
+ *                  target's token after them (m + 1 valid entries per episode)
+ *   logits_out     device f32 [total rows, vocab], may be NULL (debug / parity) */
+int specvla_verify_tree(specvla_ctx *ctx, int n_ep, const int *episodes,
+                        const specvla_tree *trees, int r, int *accept_len_out, int *tokens_out,
+                        float *logits_out, void *stream);
+
+/* Whole chunk (Algorithm 1): prefill, then draft -> verify -> accept until every episode has
+ * n_tokens tokens; the result is clipped to n_tokens. One stream synchronisation per
+ * iteration (the accepted length decides termination).
+ *   tokens_out   host [n_ep][n_tokens]
+ *   actions_out  host [n_ep][n_tokens] bin centres in [-1, 1] (256 uniform bins), may be NULL
+ *   stats        may be NULL */
+int specvla_generate_action(specvla_ctx *ctx, int n_ep, const int *episodes, const void *embeds,
+                            const int *token_ids, const int *lens,
+                            const specvla_tree_shape *shape, int r, int n_tokens,
+                            int *tokens_out, float *actions_out, specvla_stats *stats,
+                            void *stream);
+
+/* Inspection (tests, parity): copies internal results of the last call to HOST memory and
+ * synchronises. `what`: */
+#define SPECVLA_BUF_GREEDY      1   /* int   [rows]      greedy token per row of the last verify */
+#define SPECVLA_BUF_MARGIN      2   /* float [rows]      top-1 minus top-2 logit per row */
+#define SPECVLA_BUF_FEATURES    3   /* float [rows, d]   final-norm outputs of the last target forward */
+#define SPECVLA_BUF_PATH        4   /* int   [n_ep][SPECVLA_MAX_DEPTH+1] accepted path rows */
+#define SPECVLA_BUF_STATE       5   /* int   [max_episodes][4]: P, Pd, root, n_pending */
+#define SPECVLA_BUF_DRAFT_TOPK_TOK 6 /* int   [rows][8]   top tokens of the last draft level */
+#define SPECVLA_BUF_DRAFT_TOPK_LP  7 /* float [rows][8]   their log-probabilities */
+int specvla_read_buffer(specvla_ctx *ctx, int what, void *host_dst, size_t bytes, void *stream);
+
+/* Copies KV-cache rows [slot0, slot0+n_slots) of one layer to host as bf16 [n_slots, H*dh].
+ * which: 0 = K, 1 = V; draft: 0 = target cache, 1 = draft cache (layer must be 0). */
+int specvla_read_kv(specvla_ctx *ctx, int draft, int episode, int layer, int which, int slot0,
+                    int n_slots, void *host_dst, void *stream);
+
+/* Y[T, N] (f32, device) = X[T, K] (bf16, device) * W[N, K]^T (bf16, device): the library's
+ * weight-streaming GEMM exposed for kernel-level parity tests and roofline measurement.
+ * scratch: device f32, at least specvla_gemm_scratch_bytes(T, N, K) bytes. */
+size_t specvla_gemm_scratch_bytes(int T, int N, int K);
+int specvla_gemm_bf16(const void *X, const void *W, float *Y, int T, int N, int K,
+                      void *scratch, size_t scratch_bytes, void *stream);
+
+const char *specvla_strerror(int code);
+/* Text of the last CUDA error seen by this context (empty string if none). */
+const char *specvla_last_cuda_error(const specvla_ctx *ctx);
+/* Number of kernels launched by this context since creation (for launch accounting). */
+long long specvla_kernel_launches(const specvla_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPECVLA_H */

@@ -1,0 +1,264 @@
+"""ctypes binding of libspecvla.so: argument marshalling only.
+
+PyTorch is used for device memory (weights, workspace, inputs) and the current stream;
+all computation happens inside the library. Method names follow the C entry points.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+from .build import LIB_PATH
+
+MAX_DEPTH = 8
+MAX_TREE_ROWS = 128
+
+BUF_GREEDY, BUF_MARGIN, BUF_FEATURES, BUF_PATH, BUF_STATE, BUF_TOPK_TOK, BUF_TOPK_LP = 1, 2, 3, 4, 5, 6, 7
+
+
+class ModelDesc(C.Structure):
+    _fields_ = [(n, C.c_int) for n in ("n_layers", "d_model", "n_heads", "head_dim", "d_ffn", "vocab",
+                                       "action_base", "n_bins")] + \
+               [("rms_eps", C.c_float), ("rope_theta", C.c_float)] + \
+               [(n, C.c_int) for n in ("max_seq", "max_episodes", "max_rows", "action_only")]
+
+
+class Weights(C.Structure):
+    _fields_ = [("embed", C.c_void_p), ("lm_head", C.c_void_p), ("final_norm", C.c_void_p)] + \
+               [(n, C.POINTER(C.c_void_p)) for n in ("wqkv", "wo", "wgu", "wd", "norm1", "norm2")]
+
+
+class DraftWeights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("fc", "wqkv", "wo", "wgu", "wd", "norm1", "norm2")]
+
+
+class TreeShape(C.Structure):
+    _fields_ = [("depth", C.c_int), ("branch", C.c_int * MAX_DEPTH), ("expand", C.c_int * MAX_DEPTH)]
+
+
+class Tree(C.Structure):
+    _fields_ = [("n_rows", C.c_int), ("tokens", C.POINTER(C.c_int)), ("parent", C.POINTER(C.c_int)),
+                ("depth", C.POINTER(C.c_int)), ("score", C.POINTER(C.c_float))]
+
+
+class Stats(C.Structure):
+    _fields_ = [("iterations", C.c_int), ("tokens_emitted", C.c_int), ("accept_len", C.c_int * 16),
+                ("ms_prefill", C.c_float), ("ms_draft", C.c_float), ("ms_verify", C.c_float)]
+
+
+EXPORTS = {
+    "specvla_workspace_bytes": (C.c_size_t, [C.POINTER(ModelDesc)]),
+    "specvla_create": (C.c_int, [C.POINTER(ModelDesc), C.POINTER(Weights), C.POINTER(DraftWeights),
+                                 C.c_void_p, C.c_size_t, C.POINTER(C.c_void_p)]),
+    "specvla_destroy": (C.c_int, [C.c_void_p]),
+    "specvla_reset": (C.c_int, [C.c_void_p, C.c_int]),
+    "specvla_prefill": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_int), C.c_void_p, C.POINTER(C.c_int),
+                                  C.POINTER(C.c_int), C.POINTER(C.c_int), C.c_void_p, C.c_void_p]),
+    "specvla_draft_tree": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_int), C.POINTER(TreeShape),
+                                     C.POINTER(Tree), C.c_void_p]),
+    "specvla_verify_tree": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_int), C.POINTER(Tree), C.c_int,
+                                      C.POINTER(C.c_int), C.POINTER(C.c_int), C.c_void_p, C.c_void_p]),
+    "specvla_generate_action": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_int), C.c_void_p,
+                                          C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(TreeShape),
+                                          C.c_int, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_float),
+                                          C.POINTER(Stats), C.c_void_p]),
+    "specvla_read_buffer": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "specvla_read_kv": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
+                                  C.c_void_p, C.c_void_p]),
+    "specvla_gemm_scratch_bytes": (C.c_size_t, [C.c_int, C.c_int, C.c_int]),
+    "specvla_gemm_bf16": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
+                                    C.c_void_p, C.c_size_t, C.c_void_p]),
+    "specvla_strerror": (C.c_char_p, [C.c_int]),
+    "specvla_last_cuda_error": (C.c_char_p, [C.c_void_p]),
+    "specvla_kernel_launches": (C.c_longlong, [C.c_void_p]),
+}
+
+
+def load_library(path: str = LIB_PATH) -> C.CDLL:
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} is missing: build it with `python -m paper_2507_22424_b200.build` "
+                           "(there is no fallback implementation)")
+    lib = C.CDLL(path)
+    for name, (res, args) in EXPORTS.items():
+        fn = getattr(lib, name)
+        fn.restype, fn.argtypes = res, args
+    return lib
+
+
+lib = load_library()
+
+
+class SpecVLAError(RuntimeError):
+    def __init__(self, code, detail=""):
+        self.code = code
+        super().__init__(f"specvla error {code}: {lib.specvla_strerror(code).decode()} {detail}")
+
+
+def _ints(values):
+    return (C.c_int * len(values))(*[int(v) for v in values])
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def make_shape(branch, expand) -> TreeShape:
+    s = TreeShape()
+    s.depth = len(branch)
+    for i, (b, e) in enumerate(zip(branch, expand)):
+        s.branch[i], s.expand[i] = int(b), int(e)
+    return s
+
+
+class SpecVLA:
+    """One library context over weights held in torch CUDA tensors (kept alive here)."""
+
+    def __init__(self, desc, weights: dict, max_seq=512, max_episodes=1, max_rows=512, action_only=True):
+        self.model = desc
+        self.md = ModelDesc(desc.n_layers, desc.d_model, desc.n_heads, desc.head_dim, desc.d_ffn, desc.vocab,
+                            desc.action_base, desc.n_bins, desc.rms_eps, desc.rope_theta,
+                            max_seq, max_episodes, max_rows, int(action_only))
+        self.w = weights
+        L = desc.n_layers
+
+        def per_layer(name):
+            return (C.c_void_p * L)(*[weights[f"layers.{l}.{name}"].data_ptr() for l in range(L)])
+
+        self._arrays = {n: per_layer(n) for n in ("wqkv", "wo", "wgu", "wd", "norm1", "norm2")}
+        tw = Weights(weights["embed"].data_ptr(), weights["lm_head"].data_ptr(),
+                     weights["final_norm"].data_ptr(), *[self._arrays[n] for n in
+                                                         ("wqkv", "wo", "wgu", "wd", "norm1", "norm2")])
+        dw = None
+        if "draft.fc" in weights:
+            dw = DraftWeights(weights["draft.fc"].data_ptr(),
+                              *[weights[f"draft.layer.{n}"].data_ptr()
+                                for n in ("wqkv", "wo", "wgu", "wd", "norm1", "norm2")])
+        nbytes = lib.specvla_workspace_bytes(C.byref(self.md))
+        if nbytes == 0:
+            raise SpecVLAError(-1, "(model description rejected)")
+        self.workspace = torch.empty(nbytes + 1024, dtype=torch.uint8, device="cuda")
+        base = (self.workspace.data_ptr() + 1023) // 1024 * 1024
+        self.workspace_bytes = nbytes
+        handle = C.c_void_p()
+        rc = lib.specvla_create(C.byref(self.md), C.byref(tw), C.byref(dw) if dw else None,
+                                C.c_void_p(base), nbytes, C.byref(handle))
+        if rc != 0:
+            raise SpecVLAError(rc)
+        self.h = handle
+
+    def close(self):
+        if getattr(self, "h", None):
+            lib.specvla_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, rc):
+        if rc != 0:
+            raise SpecVLAError(rc, lib.specvla_last_cuda_error(self.h).decode())
+
+    # ------------------------------------------------------------------ entry points
+    def prefill(self, episodes, embeds, token_ids, lens, want_logits=False):
+        """embeds: CUDA bf16 [sum(lens), d]; token_ids: host ints; returns first tokens."""
+        n = len(episodes)
+        first = (C.c_int * n)()
+        logits = torch.empty(n, self.model.vocab, dtype=torch.float32, device="cuda") if want_logits else None
+        self._check(lib.specvla_prefill(self.h, n, _ints(episodes), C.c_void_p(embeds.data_ptr()),
+                                        _ints(token_ids), _ints(lens), first,
+                                        C.c_void_p(logits.data_ptr()) if want_logits else None, _stream()))
+        return (list(first), logits) if want_logits else list(first)
+
+    def draft_tree(self, episodes, shape: TreeShape, want_trees=True):
+        n = len(episodes)
+        if not want_trees:
+            self._check(lib.specvla_draft_tree(self.h, n, _ints(episodes), C.byref(shape), None, _stream()))
+            return None
+        trees = (Tree * n)()
+        bufs = []
+        for i in range(n):
+            b = [(C.c_int * MAX_TREE_ROWS)() for _ in range(3)] + [(C.c_float * MAX_TREE_ROWS)()]
+            bufs.append(b)
+            trees[i].tokens, trees[i].parent, trees[i].depth = b[0], b[1], b[2]
+            trees[i].score = b[3]
+        self._check(lib.specvla_draft_tree(self.h, n, _ints(episodes), C.byref(shape), trees, _stream()))
+        out = []
+        for i in range(n):
+            k = trees[i].n_rows
+            out.append(dict(tokens=list(bufs[i][0][:k]), parent=list(bufs[i][1][:k]),
+                            depth=list(bufs[i][2][:k]), score=list(bufs[i][3][:k])))
+        return out
+
+    def verify_tree(self, episodes, trees, r, want_logits=False):
+        """trees: list of dicts (tokens, parent, depth) or None for the device-resident trees.
+        Returns (accept lengths, emitted tokens per episode[, logits [rows, V]])."""
+        n = len(episodes)
+        ctrees, keep, rows = None, [], 0
+        if trees is not None:
+            ctrees = (Tree * n)()
+            for i, t in enumerate(trees):
+                a, b, c = _ints(t["tokens"]), _ints(t["parent"]), _ints(t["depth"])
+                keep += [a, b, c]
+                ctrees[i].n_rows = len(t["tokens"])
+                ctrees[i].tokens, ctrees[i].parent, ctrees[i].depth = a, b, c
+                ctrees[i].score = None
+                rows += len(t["tokens"])
+        logits = None
+        if want_logits:
+            if trees is None:
+                raise ValueError("want_logits needs caller-supplied trees (row count)")
+            logits = torch.empty(rows, self.model.vocab, dtype=torch.float32, device="cuda")
+        m = (C.c_int * n)()
+        toks = (C.c_int * (n * (MAX_DEPTH + 1)))()
+        self._check(lib.specvla_verify_tree(self.h, n, _ints(episodes), ctrees, int(r), m, toks,
+                                            C.c_void_p(logits.data_ptr()) if want_logits else None, _stream()))
+        emitted = [list(toks[i * (MAX_DEPTH + 1): i * (MAX_DEPTH + 1) + m[i] + 1]) for i in range(n)]
+        return (list(m), emitted, logits) if want_logits else (list(m), emitted)
+
+    def generate_action(self, episodes, embeds, token_ids, lens, shape: TreeShape, r, n_tokens=7):
+        n = len(episodes)
+        toks = (C.c_int * (n * n_tokens))()
+        acts = (C.c_float * (n * n_tokens))()
+        stats = Stats()
+        self._check(lib.specvla_generate_action(self.h, n, _ints(episodes), C.c_void_p(embeds.data_ptr()),
+                                                _ints(token_ids), _ints(lens), C.byref(shape), int(r),
+                                                int(n_tokens), toks, acts, C.byref(stats), _stream()))
+        tokens = [list(toks[i * n_tokens:(i + 1) * n_tokens]) for i in range(n)]
+        actions = [list(acts[i * n_tokens:(i + 1) * n_tokens]) for i in range(n)]
+        return tokens, actions, stats
+
+    # ------------------------------------------------------------------ inspection
+    def read_buffer(self, what, count, dtype):
+        out = torch.empty(count, dtype=dtype)
+        self._check(lib.specvla_read_buffer(self.h, what, C.c_void_p(out.data_ptr()),
+                                            out.numel() * out.element_size(), _stream()))
+        return out
+
+    def read_kv(self, episode, layer, which, slot0, n_slots, draft=False):
+        hd = self.model.n_heads * self.model.head_dim
+        out = torch.empty(n_slots, hd, dtype=torch.bfloat16)
+        self._check(lib.specvla_read_kv(self.h, int(draft), episode, layer, which, slot0, n_slots,
+                                        C.c_void_p(out.data_ptr()), _stream()))
+        return out
+
+    def kernel_launches(self):
+        return int(lib.specvla_kernel_launches(self.h))
+
+
+def gemm_bf16(x: torch.Tensor, w: torch.Tensor) -> torch.Tensor:
+    """Y[T, N] = X[T, K] @ W[N, K]^T through the library's weight-streaming GEMM."""
+    T, K = x.shape
+    N = w.shape[0]
+    y = torch.empty(T, N, dtype=torch.float32, device="cuda")
+    nb = lib.specvla_gemm_scratch_bytes(T, N, K)
+    scratch = torch.empty(nb, dtype=torch.uint8, device="cuda")
+    rc = lib.specvla_gemm_bf16(C.c_void_p(x.data_ptr()), C.c_void_p(w.data_ptr()), C.c_void_p(y.data_ptr()),
+                               T, N, K, C.c_void_p(scratch.data_ptr()), nb, _stream())
+    if rc != 0:
+        raise SpecVLAError(rc)
+    return y

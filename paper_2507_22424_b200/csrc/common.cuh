@@ -1,0 +1,71 @@
+// Shared device/host declarations of the Spec-VLA verification path (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+typedef __nv_bfloat16 bf16;
+
+#define SV_MAX_TREE 128          // rows of one tree, root included
+#define SV_MAX_DEPTH 8
+#define SV_MAX_BRANCH 8
+#define SV_MAX_PENDING (SV_MAX_DEPTH + 1)
+#define SV_TOPK 8
+
+// Per-row description of one forward call (structure of arrays, all on the device).
+struct RowTable {
+  int *tok;       // token id, or -1: the row's input comes from the embeds buffer
+  int *src;       // row index into the embeds buffer (prefill) when tok < 0
+  int *ep;        // episode id (selects the KV cache)
+  int *pos;       // RoPE position
+  int *slot;      // cache slot the row's K/V are written to
+  int *nvis;      // cache slots [0, nvis) are visible to the row
+  int *tbase;     // slot of bit 0 of the mask
+  uint32_t *mask; // [rows][4] bit b set: slot tbase + b is visible
+};
+
+// Episode list of one call, passed to kernels by value.
+#define SV_MAX_EP 64
+struct EpArgs {
+  int n_ep;
+  int eps[SV_MAX_EP];     // episode ids
+  int row0[SV_MAX_EP];    // first row of each episode in the call's row table
+  int nrows[SV_MAX_EP];   // its number of rows
+  int aux[SV_MAX_EP];     // call-specific
+};
+
+// Per-episode decoding state on the device.
+struct EpState {
+  int P;                          // committed target positions
+  int Pd;                         // committed draft positions
+  int root;                       // last emitted token (not yet in the target cache)
+  int n_pending;                  // draft rows waiting: (feature_j, token_j) at position Pd + j
+  int pending_tok[SV_MAX_PENDING];
+  int pad[3];
+};
+
+// Per-episode draft tree on the device.
+struct DevTree {
+  int n_rows;
+  int n_drows;                    // draft rows used so far (row 0 = the root's catch-up row)
+  int level_begin, level_end;     // nodes of the level built last
+  int sel_count;                  // nodes selected for expansion at the next level
+  int sel[16];                    // ... in rank order
+  int tok[SV_MAX_TREE], parent[SV_MAX_TREE], depth[SV_MAX_TREE];
+  float score[SV_MAX_TREE];
+  int drow[SV_MAX_TREE];          // draft row that scored the node's children (-1: none)
+  uint32_t vmask[SV_MAX_TREE][4]; // ancestors-and-self over tree rows (verification mask)
+  uint32_t dmask[SV_MAX_TREE][4]; // ancestors-and-self over draft rows (draft mask), by draft row
+};
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}

@@ -1,0 +1,907 @@
+// Host side of the Spec-VLA verification library: context, workspace layout, and the
+// kernel sequences behind each C-ABI entry point (see include/specvla.h).
+#include "../../include/specvla.h"
+
+#include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "attention.cuh"
+#include "common.cuh"
+#include "epilogue.cuh"
+#include "gemm_mma.cuh"
+#include "tree.cuh"
+
+namespace {
+
+struct LayerW {
+  const bf16 *wqkv, *wo, *wgu, *wd;
+  const float *norm1, *norm2;
+};
+
+constexpr int MAX_SPLITS = 8;
+constexpr size_t ALIGN = 1024;
+
+struct Carver {
+  char *base;
+  size_t off;
+  template <typename T> T *take(size_t n) {
+    off = (off + ALIGN - 1) / ALIGN * ALIGN;
+    T *p = base ? reinterpret_cast<T *>(base + off) : nullptr;
+    off += n * sizeof(T);
+    return p;
+  }
+};
+
+}  // namespace
+
+struct specvla_ctx {
+  specvla_model_desc desc;
+  int hd;                       // n_heads * head_dim
+  int max_lm_rows;              // rows the LM head may see in one call
+  int max_draft_rows;           // rows of one draft-tree level summed over episodes
+  std::vector<LayerW> layers;
+  LayerW dlayer;
+  const bf16 *embed, *lm_head, *draft_fc;
+  const float *final_norm;
+  bool has_draft;
+
+  // workspace carve-up (device)
+  bf16 *kv_t, *kv_d;            // target [ep][layer][2][max_seq][hd], draft [ep][2][max_seq][hd]
+  size_t kv_t_ep_stride, kv_t_layer_stride, kv_d_ep_stride;
+  float2 *rope_tab;
+  float *x, *feat, *part, *lgs, *pend_feat, *dout, *margin, *top_lp;
+  size_t part_floats;
+  bf16 *xn, *xin, *q, *ao, *hid, *lm_in;
+  RowTable rt;
+  int *feat_src, *dst_row, *lm_rows, *greedy, *top_tok, *out_m, *out_tok, *out_path;
+  EpState *st;
+  DevTree *trees;
+
+  // host side
+  void *pinned;                 // pinned staging: [small results | tree staging | row tables]
+  size_t pinned_bytes;
+  int *pin_small;               // 4096 ints of results read back
+  DevTree *pin_trees;           // max_episodes trees
+  int *pin_rows;                // 8 * max_rows ints
+  std::vector<int> hP, hPending;  // host mirror of P and n_pending; -1 = not prefilled
+  std::vector<int> hTreeRows;     // rows of the device-resident tree left by the last draft call
+  int last_rows;                // rows of the last target forward
+  long long launches;
+  char cuda_err[256];
+  cudaEvent_t ev[4];
+};
+
+namespace {
+
+#define CU(call)                                                                        \
+  do {                                                                                  \
+    cudaError_t _e = (call);                                                            \
+    if (_e != cudaSuccess) {                                                            \
+      snprintf(ctx->cuda_err, sizeof(ctx->cuda_err), "%s at %s:%d", cudaGetErrorString(_e), \
+               __FILE__, __LINE__);                                                     \
+      return SPECVLA_ERR_CUDA;                                                          \
+    }                                                                                   \
+  } while (0)
+#define LAUNCHED()            \
+  do {                        \
+    ctx->launches++;          \
+    CU(cudaGetLastError());   \
+  } while (0)
+#define TRY(expr)             \
+  do {                        \
+    int _r = (expr);          \
+    if (_r != SPECVLA_OK) return _r; \
+  } while (0)
+
+bool desc_ok(const specvla_model_desc *d) {
+  if (!d) return false;
+  if (d->n_layers < 1 || d->d_model < 64 || d->n_heads < 1 || d->d_ffn < 8 || d->vocab < 16) return false;
+  if (d->head_dim != 64 && d->head_dim != 128) return false;
+  if (d->d_model % 8 || d->d_ffn % 8 || (d->n_heads * d->head_dim) % 8) return false;
+  if (d->n_bins < 1 || d->action_base < 0 || d->action_base + d->n_bins > d->vocab) return false;
+  if (d->max_seq < 2 || d->max_episodes < 1 || d->max_episodes > SV_MAX_EP || d->max_rows < 1) return false;
+  if (!(d->rms_eps > 0.f) || !(d->rope_theta > 1.f)) return false;
+  return true;
+}
+
+// Lays the workspace out; with base == NULL only measures it.
+size_t carve(specvla_ctx *c, char *base) {
+  const specvla_model_desc &d = c->desc;
+  const int hd = d.n_heads * d.head_dim;
+  const size_t R = d.max_rows, E = d.max_episodes;
+  const size_t lm_rows = c->max_lm_rows, dr = c->max_draft_rows;
+  Carver cv{base, 0};
+  c->kv_t_layer_stride = (size_t)2 * d.max_seq * hd;
+  c->kv_t_ep_stride = c->kv_t_layer_stride * d.n_layers;
+  c->kv_d_ep_stride = (size_t)2 * d.max_seq * hd;
+  c->kv_t = cv.take<bf16>(E * c->kv_t_ep_stride);
+  c->kv_d = cv.take<bf16>(E * c->kv_d_ep_stride);
+  c->rope_tab = cv.take<float2>((size_t)d.max_seq * (d.head_dim / 2));
+  c->x = cv.take<float>(R * d.d_model);
+  c->feat = cv.take<float>(R * d.d_model);
+  c->xn = cv.take<bf16>(R * d.d_model);
+  c->xin = cv.take<bf16>(R * 2 * d.d_model);
+  c->q = cv.take<bf16>(R * hd);
+  c->ao = cv.take<bf16>(R * hd);
+  c->hid = cv.take<bf16>(R * d.d_ffn);
+  c->lm_in = cv.take<bf16>(lm_rows * d.d_model);
+  size_t widest = (size_t)3 * hd;
+  if ((size_t)2 * d.d_ffn > widest) widest = (size_t)2 * d.d_ffn;
+  size_t pf = R * widest;                                  // one split over all rows
+  const size_t small_rows = lm_rows < R ? lm_rows : R;
+  if ((size_t)MAX_SPLITS * small_rows * widest > pf) pf = (size_t)MAX_SPLITS * small_rows * widest;
+  if (lm_rows * d.vocab > pf) pf = lm_rows * (size_t)d.vocab;
+  c->part_floats = pf;
+  c->part = cv.take<float>(pf);
+  c->lgs = cv.take<float>(dr * d.vocab);
+  c->pend_feat = cv.take<float>(E * SV_MAX_PENDING * d.d_model);
+  c->dout = cv.take<float>(E * SV_MAX_TREE * d.d_model);
+  c->margin = cv.take<float>(R);
+  c->top_lp = cv.take<float>(dr * SV_TOPK);
+  c->rt.tok = cv.take<int>(R);
+  c->rt.src = cv.take<int>(R);
+  c->rt.ep = cv.take<int>(R);
+  c->rt.pos = cv.take<int>(R);
+  c->rt.slot = cv.take<int>(R);
+  c->rt.nvis = cv.take<int>(R);
+  c->rt.tbase = cv.take<int>(R);
+  c->rt.mask = cv.take<uint32_t>(R * 4);
+  c->feat_src = cv.take<int>(R);
+  c->dst_row = cv.take<int>(R);
+  c->lm_rows = cv.take<int>(R);
+  c->greedy = cv.take<int>(R);
+  c->top_tok = cv.take<int>(dr * SV_TOPK);
+  c->out_m = cv.take<int>(E);
+  c->out_tok = cv.take<int>(E * (SV_MAX_DEPTH + 1));
+  c->out_path = cv.take<int>(E * (SV_MAX_DEPTH + 1));
+  c->st = cv.take<EpState>(E);
+  c->trees = cv.take<DevTree>(E);
+  return (cv.off + ALIGN - 1) / ALIGN * ALIGN;
+}
+
+void derive_caps(specvla_ctx *c) {
+  const specvla_model_desc &d = c->desc;
+  c->hd = d.n_heads * d.head_dim;
+  size_t lm = (size_t)d.max_episodes * SV_MAX_TREE;
+  if (lm > (size_t)d.max_rows) lm = d.max_rows;
+  c->max_lm_rows = (int)lm;
+  size_t dr = (size_t)d.max_episodes * 16;
+  if (dr > (size_t)d.max_rows) dr = d.max_rows;
+  c->max_draft_rows = (int)dr;
+}
+
+// part <- A[R, K] * W[N, K]^T split over K; returns the number of splits to sum.
+int gemm(specvla_ctx *ctx, const bf16 *A, const bf16 *W, int R, int N, int K, cudaStream_t st,
+         int *splits_out) {
+  int cap = (int)(ctx->part_floats / ((size_t)R * N));
+  if (cap < 1) return SPECVLA_ERR_CAPACITY;
+  if (cap > MAX_SPLITS) cap = MAX_SPLITS;
+  const int splits = gemm_mma::plan_splits(R, N, K, cap);
+  CU(gemm_mma::launch(A, W, ctx->part, R, N, K, splits, st));
+  ctx->launches++;
+  *splits_out = splits;
+  return SPECVLA_OK;
+}
+
+int attention(specvla_ctx *ctx, int R, const bf16 *cache, size_t ep_stride, cudaStream_t st) {
+  const specvla_model_desc &d = ctx->desc;
+  const float scale = 1.f / sqrtf((float)d.head_dim);
+  dim3 grid(d.n_heads, R);
+  if (d.head_dim == 128)
+    attn::tree_attention_kernel<128><<<grid, attn::WARPS * 32, 0, st>>>(
+        ctx->q, cache, ep_stride, d.max_seq, d.n_heads, ctx->rt, scale, ctx->ao);
+  else
+    attn::tree_attention_kernel<64><<<grid, attn::WARPS * 32, 0, st>>>(
+        ctx->q, cache, ep_stride, d.max_seq, d.n_heads, ctx->rt, scale, ctx->ao);
+  LAUNCHED();
+  return SPECVLA_OK;
+}
+
+// One pre-norm decoder layer over R rows. In: x (residual, fp32) and xn = bf16(norm1(x)).
+// Out: x updated; xn = bf16(rmsnorm(x) * next_gain) (or bf16(x) when next_gain is NULL);
+// feat_out (optional) receives the normalised rows in fp32.
+int run_layer(specvla_ctx *ctx, const LayerW &w, int R, bf16 *cache, size_t ep_stride,
+              const float *next_gain, float *feat_out, cudaStream_t st) {
+  const specvla_model_desc &d = ctx->desc;
+  const int hd = ctx->hd, D = d.d_model, F = d.d_ffn;
+  int s;
+  TRY(gemm(ctx, ctx->xn, w.wqkv, R, 3 * hd, D, st, &s));
+  epi::qkv_rope_append_kernel<<<R, epi::THREADS, 0, st>>>(ctx->part, s, R, d.n_heads, d.head_dim, ctx->rt,
+                                                          ctx->rope_tab, ctx->q, cache, ep_stride,
+                                                          d.max_seq);
+  LAUNCHED();
+  TRY(attention(ctx, R, cache, ep_stride, st));
+  TRY(gemm(ctx, ctx->ao, w.wo, R, D, hd, st, &s));
+  epi::residual_norm_kernel<<<R, epi::THREADS, 0, st>>>(ctx->part, s, R, D, 1, w.norm2, d.rms_eps, ctx->x,
+                                                        ctx->xn, nullptr);
+  LAUNCHED();
+  TRY(gemm(ctx, ctx->xn, w.wgu, R, 2 * F, D, st, &s));
+  epi::swiglu_kernel<<<dim3((F + epi::THREADS - 1) / epi::THREADS, R), epi::THREADS, 0, st>>>(
+      ctx->part, s, R, F, ctx->hid);
+  LAUNCHED();
+  TRY(gemm(ctx, ctx->hid, w.wd, R, D, F, st, &s));
+  epi::residual_norm_kernel<<<R, epi::THREADS, 0, st>>>(ctx->part, s, R, D, 1, next_gain, d.rms_eps,
+                                                        ctx->x, ctx->xn, feat_out);
+  LAUNCHED();
+  return SPECVLA_OK;
+}
+
+// Target model over the R rows described by ctx->rt: embedding, all layers, final norm.
+// Leaves features in ctx->feat (fp32) and ctx->xn (bf16).
+int target_forward(specvla_ctx *ctx, int R, const bf16 *embeds, cudaStream_t st) {
+  const specvla_model_desc &d = ctx->desc;
+  epi::embed_norm_kernel<<<R, epi::THREADS, 0, st>>>(ctx->rt, embeds, ctx->embed, ctx->layers[0].norm1,
+                                                     d.rms_eps, d.d_model, ctx->x, ctx->xn);
+  LAUNCHED();
+  for (int l = 0; l < d.n_layers; l++) {
+    const bool last = (l + 1 == d.n_layers);
+    TRY(run_layer(ctx, ctx->layers[l], R, ctx->kv_t + (size_t)l * ctx->kv_t_layer_stride,
+                  ctx->kv_t_ep_stride, last ? ctx->final_norm : ctx->layers[l + 1].norm1,
+                  last ? ctx->feat : nullptr, st));
+  }
+  ctx->last_rows = R;
+  return SPECVLA_OK;
+}
+
+// Draft model over R rows: ctx->xin = [feature ; embedding] rows are already built.
+// Leaves the layer outputs in ctx->x (fp32) and ctx->xn (bf16, un-normalised).
+int draft_forward(specvla_ctx *ctx, int R, cudaStream_t st) {
+  const specvla_model_desc &d = ctx->desc;
+  int s;
+  TRY(gemm(ctx, ctx->xin, ctx->draft_fc, R, d.d_model, 2 * d.d_model, st, &s));
+  epi::residual_norm_kernel<<<R, epi::THREADS, 0, st>>>(ctx->part, s, R, d.d_model, 0, ctx->dlayer.norm1,
+                                                        d.rms_eps, ctx->x, ctx->xn, nullptr);
+  LAUNCHED();
+  return run_layer(ctx, ctx->dlayer, R, ctx->kv_d, ctx->kv_d_ep_stride, nullptr, nullptr, st);
+}
+
+// LM head over `rows` bf16 rows of A: partial logits land in ctx->part; returns splits.
+int lm_head(specvla_ctx *ctx, const bf16 *A, int rows, cudaStream_t st, int *splits) {
+  if (rows > ctx->max_lm_rows) return SPECVLA_ERR_CAPACITY;
+  return gemm(ctx, A, ctx->lm_head, rows, ctx->desc.vocab, ctx->desc.d_model, st, splits);
+}
+
+void argmax_range(const specvla_ctx *ctx, int *lo, int *hi) {
+  if (ctx->desc.action_only) {
+    *lo = ctx->desc.action_base;
+    *hi = ctx->desc.action_base + ctx->desc.n_bins;
+  } else {
+    *lo = 0;
+    *hi = ctx->desc.vocab;
+  }
+}
+
+int check_episodes(const specvla_ctx *ctx, int n_ep, const int *episodes) {
+  if (!ctx || !episodes || n_ep < 1) return SPECVLA_ERR_INVALID_ARG;
+  if (n_ep > ctx->desc.max_episodes) return SPECVLA_ERR_CAPACITY;
+  for (int i = 0; i < n_ep; i++) {
+    if (episodes[i] < 0 || episodes[i] >= ctx->desc.max_episodes) return SPECVLA_ERR_INVALID_ARG;
+    for (int j = 0; j < i; j++)
+      if (episodes[j] == episodes[i]) return SPECVLA_ERR_INVALID_ARG;
+  }
+  return SPECVLA_OK;
+}
+
+int validate_tree(const specvla_tree &t) {
+  if (t.n_rows < 1 || t.n_rows > SV_MAX_TREE) return SPECVLA_ERR_BAD_TREE;
+  if (!t.tokens || !t.parent || !t.depth) return SPECVLA_ERR_INVALID_ARG;
+  if (t.parent[0] != -1 || t.depth[0] != 0) return SPECVLA_ERR_BAD_TREE;
+  for (int i = 1; i < t.n_rows; i++) {
+    const int p = t.parent[i];
+    if (p < 0 || p >= i) return SPECVLA_ERR_BAD_TREE;
+    if (t.depth[i] != t.depth[p] + 1 || t.depth[i] > SV_MAX_DEPTH) return SPECVLA_ERR_BAD_TREE;
+  }
+  return SPECVLA_OK;
+}
+
+int validate_shape(const specvla_tree_shape *s, int *n_nodes) {
+  if (!s || s->depth < 0 || s->depth > SV_MAX_DEPTH) return SPECVLA_ERR_INVALID_ARG;
+  int prev = 1, total = 0;
+  for (int l = 0; l < s->depth; l++) {
+    if (s->branch[l] < 1 || s->branch[l] > SV_MAX_BRANCH) return SPECVLA_ERR_INVALID_ARG;
+    if (s->expand[l] < 1 || s->expand[l] > 16 || s->expand[l] > prev) return SPECVLA_ERR_INVALID_ARG;
+    if (l == 0 && s->expand[0] != 1) return SPECVLA_ERR_INVALID_ARG;
+    prev = s->branch[l] * s->expand[l];
+    if (prev > 16) return SPECVLA_ERR_INVALID_ARG;   // one level: at most 16 nodes
+    total += prev;
+  }
+  if (1 + total > SV_MAX_TREE) return SPECVLA_ERR_INVALID_ARG;
+  *n_nodes = total;
+  return SPECVLA_OK;
+}
+
+}  // namespace
+
+// =====================================================================================
+extern "C" {
+
+size_t specvla_workspace_bytes(const specvla_model_desc *desc) {
+  if (!desc_ok(desc)) return 0;
+  specvla_ctx tmp{};
+  tmp.desc = *desc;
+  derive_caps(&tmp);
+  return carve(&tmp, nullptr);
+}
+
+int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
+                   const specvla_draft_weights *dw, void *workspace, size_t workspace_bytes,
+                   specvla_ctx **out) {
+  if (!out) return SPECVLA_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!desc_ok(desc) || !tw || !workspace) return SPECVLA_ERR_INVALID_ARG;
+  if (!tw->embed || !tw->lm_head || !tw->final_norm || !tw->wqkv || !tw->wo || !tw->wgu || !tw->wd ||
+      !tw->norm1 || !tw->norm2)
+    return SPECVLA_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(workspace) % ALIGN) != 0) return SPECVLA_ERR_INVALID_ARG;
+  int dev = 0;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess)
+    return SPECVLA_ERR_CUDA;
+  if (prop.major != 10) return SPECVLA_ERR_UNSUPPORTED_ARCH;
+
+  specvla_ctx *ctx = new (std::nothrow) specvla_ctx();
+  if (!ctx) return SPECVLA_ERR_INVALID_ARG;
+  ctx->desc = *desc;
+  derive_caps(ctx);
+  const size_t need = carve(ctx, nullptr);
+  if (workspace_bytes < need) {
+    delete ctx;
+    return SPECVLA_ERR_CAPACITY;
+  }
+  carve(ctx, static_cast<char *>(workspace));
+  ctx->embed = static_cast<const bf16 *>(tw->embed);
+  ctx->lm_head = static_cast<const bf16 *>(tw->lm_head);
+  ctx->final_norm = tw->final_norm;
+  ctx->layers.resize(desc->n_layers);
+  for (int l = 0; l < desc->n_layers; l++) {
+    ctx->layers[l] = LayerW{static_cast<const bf16 *>(tw->wqkv[l]), static_cast<const bf16 *>(tw->wo[l]),
+                            static_cast<const bf16 *>(tw->wgu[l]), static_cast<const bf16 *>(tw->wd[l]),
+                            tw->norm1[l], tw->norm2[l]};
+    if (!tw->wqkv[l] || !tw->wo[l] || !tw->wgu[l] || !tw->wd[l] || !tw->norm1[l] || !tw->norm2[l]) {
+      delete ctx;
+      return SPECVLA_ERR_INVALID_ARG;
+    }
+  }
+  ctx->has_draft = dw && dw->fc && dw->wqkv && dw->wo && dw->wgu && dw->wd && dw->norm1 && dw->norm2;
+  if (ctx->has_draft) {
+    ctx->draft_fc = static_cast<const bf16 *>(dw->fc);
+    ctx->dlayer = LayerW{static_cast<const bf16 *>(dw->wqkv), static_cast<const bf16 *>(dw->wo),
+                         static_cast<const bf16 *>(dw->wgu), static_cast<const bf16 *>(dw->wd),
+                         dw->norm1, dw->norm2};
+  }
+  ctx->hP.assign(desc->max_episodes, -1);
+  ctx->hPending.assign(desc->max_episodes, 0);
+  ctx->hTreeRows.assign(desc->max_episodes, 0);
+  const size_t small_b = 4096 * sizeof(int);
+  const size_t trees_b = (sizeof(DevTree) * desc->max_episodes + 255) / 256 * 256;
+  ctx->pinned_bytes = small_b + trees_b + ((size_t)desc->max_rows * 8 + 256) * sizeof(int);
+  ctx->cuda_err[0] = 0;
+  if (cudaHostAlloc(&ctx->pinned, ctx->pinned_bytes, cudaHostAllocDefault) != cudaSuccess) {
+    delete ctx;
+    return SPECVLA_ERR_CUDA;
+  }
+  ctx->pin_small = static_cast<int *>(ctx->pinned);
+  ctx->pin_trees = reinterpret_cast<DevTree *>(static_cast<char *>(ctx->pinned) + small_b);
+  ctx->pin_rows = reinterpret_cast<int *>(static_cast<char *>(ctx->pinned) + small_b + trees_b);
+  for (int i = 0; i < 4; i++) cudaEventCreate(&ctx->ev[i]);
+  // device-side initialisation: RoPE table, zeroed state
+  const int half = desc->head_dim / 2, n = desc->max_seq * half;
+  epi::rope_table_kernel<<<(n + 255) / 256, 256>>>(ctx->rope_tab, desc->max_seq, half, (double)desc->rope_theta);
+  cudaMemsetAsync(ctx->st, 0, sizeof(EpState) * desc->max_episodes);
+  cudaMemsetAsync(ctx->trees, 0, sizeof(DevTree) * desc->max_episodes);
+  if (cudaDeviceSynchronize() != cudaSuccess) {
+    cudaFreeHost(ctx->pinned);
+    delete ctx;
+    return SPECVLA_ERR_CUDA;
+  }
+  *out = ctx;
+  return SPECVLA_OK;
+}
+
+int specvla_destroy(specvla_ctx *ctx) {
+  if (!ctx) return SPECVLA_ERR_INVALID_ARG;
+  cudaDeviceSynchronize();
+  for (int i = 0; i < 4; i++) cudaEventDestroy(ctx->ev[i]);
+  cudaFreeHost(ctx->pinned);
+  delete ctx;
+  return SPECVLA_OK;
+}
+
+int specvla_reset(specvla_ctx *ctx, int episode) {
+  if (!ctx || episode < 0 || episode >= ctx->desc.max_episodes) return SPECVLA_ERR_INVALID_ARG;
+  ctx->hP[episode] = -1;
+  ctx->hPending[episode] = 0;
+  return SPECVLA_OK;
+}
+
+int specvla_prefill(specvla_ctx *ctx, int n_ep, const int *episodes, const void *embeds,
+                    const int *token_ids, const int *lens, int *first_token_out, float *logits_out,
+                    void *stream) {
+  TRY(check_episodes(ctx, n_ep, episodes));
+  if (!token_ids || !lens) return SPECVLA_ERR_INVALID_ARG;
+  const specvla_model_desc &d = ctx->desc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  EpArgs ea{};
+  ea.n_ep = n_ep;
+  int R = 0;
+  for (int i = 0; i < n_ep; i++) {
+    if (lens[i] < 1) return SPECVLA_ERR_INVALID_ARG;
+    if (lens[i] + 1 > d.max_seq) return SPECVLA_ERR_CAPACITY;
+    ea.eps[i] = episodes[i];
+    ea.row0[i] = R;
+    ea.nrows[i] = lens[i];
+    R += lens[i];
+    ea.aux[i] = R - 1;
+  }
+  if (R > d.max_rows) return SPECVLA_ERR_CAPACITY;
+  for (int r = 0; r < R; r++) {
+    if (token_ids[r] >= d.vocab) return SPECVLA_ERR_INVALID_ARG;
+    if (token_ids[r] < 0 && !embeds) return SPECVLA_ERR_INVALID_ARG;
+  }
+  // row table on the host: causal rows, slot = position = index within the episode
+  int *h = ctx->pin_rows;
+  int *h_tok = h, *h_src = h + R, *h_ep = h + 2 * R, *h_pos = h + 3 * R, *h_nvis = h + 4 * R;
+  for (int i = 0; i < n_ep; i++)
+    for (int j = 0; j < lens[i]; j++) {
+      const int r = ea.row0[i] + j;
+      h_tok[r] = token_ids[r];
+      h_src[r] = r;
+      h_ep[r] = episodes[i];
+      h_pos[r] = j;
+      h_nvis[r] = j + 1;
+    }
+  const size_t rb = (size_t)R * sizeof(int);
+  CU(cudaMemcpyAsync(ctx->rt.tok, h_tok, rb, cudaMemcpyHostToDevice, st));
+  CU(cudaMemcpyAsync(ctx->rt.src, h_src, rb, cudaMemcpyHostToDevice, st));
+  CU(cudaMemcpyAsync(ctx->rt.ep, h_ep, rb, cudaMemcpyHostToDevice, st));
+  CU(cudaMemcpyAsync(ctx->rt.pos, h_pos, rb, cudaMemcpyHostToDevice, st));
+  CU(cudaMemcpyAsync(ctx->rt.slot, h_pos, rb, cudaMemcpyHostToDevice, st));
+  CU(cudaMemcpyAsync(ctx->rt.nvis, h_nvis, rb, cudaMemcpyHostToDevice, st));
+  CU(cudaMemsetAsync(ctx->rt.tbase, 0, rb, st));
+  CU(cudaMemsetAsync(ctx->rt.mask, 0, rb * 4, st));
+
+  const bf16 *emb = static_cast<const bf16 *>(embeds);
+  TRY(target_forward(ctx, R, emb, st));
+
+  // first token: LM head on each episode's last row
+  int *h_last = h + 5 * R;
+  for (int i = 0; i < n_ep; i++) h_last[i] = ea.aux[i];
+  CU(cudaMemcpyAsync(ctx->lm_rows, h_last, n_ep * sizeof(int), cudaMemcpyHostToDevice, st));
+  epi::gather_rows_kernel<<<n_ep, 256, 0, st>>>(ctx->xn, ctx->lm_rows, d.d_model, ctx->lm_in);
+  LAUNCHED();
+  int s, lo, hi;
+  argmax_range(ctx, &lo, &hi);
+  TRY(lm_head(ctx, ctx->lm_in, n_ep, st, &s));
+  epi::argmax_kernel<<<n_ep, epi::THREADS, 0, st>>>(ctx->part, s, n_ep, d.vocab, lo, hi, ctx->greedy,
+                                                    ctx->margin, logits_out);
+  LAUNCHED();
+  tree::prefill_commit_kernel<<<n_ep, 256, 0, st>>>(ea, ctx->st, ctx->greedy, ctx->feat, d.d_model,
+                                                    ctx->pend_feat);
+  LAUNCHED();
+
+  // draft model over the shifted pairs (feature_i, input_{i+1}), i = 0 .. len-2
+  if (ctx->has_draft) {
+    int Rd = 0;
+    int *h_fs = h + 5 * R + n_ep;          // feature source rows
+    for (int i = 0; i < n_ep; i++)
+      for (int j = 0; j + 1 < lens[i]; j++) {
+        const int r = Rd++;
+        const int tr = ea.row0[i] + j;     // target row of f_j; the embedding comes from row tr+1
+        h_tok[r] = token_ids[tr + 1];
+        h_src[r] = tr + 1;
+        h_ep[r] = episodes[i];
+        h_pos[r] = j;
+        h_nvis[r] = j + 1;
+        h_fs[r] = tr;
+      }
+    if (Rd > 0) {
+      const size_t db = (size_t)Rd * sizeof(int);
+      // the uploads above are ordered before these on the same stream, but the pinned rows
+      // are being rewritten: wait until the first batch has been consumed
+      CU(cudaStreamSynchronize(st));
+      CU(cudaMemcpyAsync(ctx->rt.tok, h_tok, db, cudaMemcpyHostToDevice, st));
+      CU(cudaMemcpyAsync(ctx->rt.src, h_src, db, cudaMemcpyHostToDevice, st));
+      CU(cudaMemcpyAsync(ctx->rt.ep, h_ep, db, cudaMemcpyHostToDevice, st));
+      CU(cudaMemcpyAsync(ctx->rt.pos, h_pos, db, cudaMemcpyHostToDevice, st));
+      CU(cudaMemcpyAsync(ctx->rt.slot, h_pos, db, cudaMemcpyHostToDevice, st));
+      CU(cudaMemcpyAsync(ctx->rt.nvis, h_nvis, db, cudaMemcpyHostToDevice, st));
+      CU(cudaMemcpyAsync(ctx->feat_src, h_fs, db, cudaMemcpyHostToDevice, st));
+      tree::draft_input_kernel<<<Rd, 256, 0, st>>>(ctx->rt, ctx->feat_src, ctx->feat, emb, ctx->embed,
+                                                   d.d_model, ctx->xin);
+      LAUNCHED();
+      TRY(draft_forward(ctx, Rd, st));
+    }
+  }
+  int *h_g = ctx->pin_small;
+  CU(cudaMemcpyAsync(h_g, ctx->greedy, n_ep * sizeof(int), cudaMemcpyDeviceToHost, st));
+  CU(cudaStreamSynchronize(st));
+  for (int i = 0; i < n_ep; i++) {
+    ctx->hP[episodes[i]] = lens[i];
+    ctx->hPending[episodes[i]] = 1;
+    ctx->hTreeRows[episodes[i]] = 0;
+    if (first_token_out) first_token_out[i] = h_g[i];
+  }
+  return SPECVLA_OK;
+}
+
+int specvla_draft_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const specvla_tree_shape *shape,
+                       specvla_tree *trees_out, void *stream) {
+  TRY(check_episodes(ctx, n_ep, episodes));
+  if (!ctx->has_draft) return SPECVLA_ERR_BAD_STATE;
+  int n_nodes = 0;
+  TRY(validate_shape(shape, &n_nodes));
+  const specvla_model_desc &d = ctx->desc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  EpArgs ea{};
+  ea.n_ep = n_ep;
+  int R = 0;
+  for (int i = 0; i < n_ep; i++) {
+    const int e = episodes[i];
+    if (ctx->hP[e] < 0 || ctx->hPending[e] < 1) return SPECVLA_ERR_BAD_STATE;
+    if (ctx->hP[e] + 1 + n_nodes > d.max_seq) return SPECVLA_ERR_CAPACITY;
+    ea.eps[i] = e;
+    ea.row0[i] = R;
+    ea.nrows[i] = ctx->hPending[e];
+    R += ctx->hPending[e];
+  }
+  if (R > d.max_rows || n_ep * 16 > ctx->max_draft_rows) return SPECVLA_ERR_CAPACITY;
+  int lo, hi, s;
+  argmax_range(ctx, &lo, &hi);
+
+  // catch-up over the pending rows; the last row of each episode scores the root's children
+  tree::build_catchup_rows_kernel<<<(n_ep + 63) / 64, 64, 0, st>>>(ea, ctx->st, ctx->trees, ctx->rt,
+                                                                   ctx->feat_src);
+  LAUNCHED();
+  tree::catchup_dst_kernel<<<(n_ep + 63) / 64, 64, 0, st>>>(ea, ctx->dst_row, ctx->lm_rows);
+  LAUNCHED();
+  tree::draft_input_kernel<<<R, 256, 0, st>>>(ctx->rt, ctx->feat_src, ctx->pend_feat, nullptr, ctx->embed,
+                                              d.d_model, ctx->xin);
+  LAUNCHED();
+  TRY(draft_forward(ctx, R, st));
+  tree::save_draft_out_kernel<<<R, 256, 0, st>>>(ctx->x, ctx->dst_row, d.d_model, ctx->dout);
+  LAUNCHED();
+  for (int i = 0; i < n_ep; i++) {
+    ctx->hPending[episodes[i]] = 0;
+    ctx->hTreeRows[episodes[i]] = 1 + n_nodes;
+  }
+
+  int scored_rows = n_ep;            // rows scored by the LM head in the current round
+  bool gathered = true;              // round 0 scores the gathered last rows
+  for (int l = 0; l < shape->depth; l++) {
+    const bf16 *A = ctx->xn;
+    if (gathered) {
+      epi::gather_rows_kernel<<<n_ep, 256, 0, st>>>(ctx->xn, ctx->lm_rows, d.d_model, ctx->lm_in);
+      LAUNCHED();
+      A = ctx->lm_in;
+    }
+    TRY(lm_head(ctx, A, scored_rows, st, &s));
+    epi::logsoftmax_topk_kernel<<<scored_rows, epi::THREADS, 0, st>>>(
+        ctx->part, s, scored_rows, d.vocab, lo, hi, ctx->lgs, ctx->top_tok, ctx->top_lp);
+    LAUNCHED();
+    const int cur = (l == 0) ? 1 : shape->expand[l];            // parents scored per episode
+    const int next = (l + 1 < shape->depth) ? shape->expand[l + 1] : 0;
+    EpArgs la = ea;
+    for (int i = 0; i < n_ep; i++) {
+      la.row0[i] = i * cur;
+      la.aux[i] = i * next;
+    }
+    tree::expand_level_kernel<<<(n_ep + 63) / 64, 64, 0, st>>>(la, l, shape->branch[l], next, ctx->top_tok,
+                                                               ctx->top_lp, ctx->trees, ctx->st, ctx->rt,
+                                                               ctx->feat_src, ctx->dst_row);
+    LAUNCHED();
+    if (next == 0) break;
+    const int Rn = n_ep * next;
+    tree::draft_input_kernel<<<Rn, 256, 0, st>>>(ctx->rt, ctx->feat_src, ctx->dout, nullptr, ctx->embed,
+                                                 d.d_model, ctx->xin);
+    LAUNCHED();
+    TRY(draft_forward(ctx, Rn, st));
+    tree::save_draft_out_kernel<<<Rn, 256, 0, st>>>(ctx->x, ctx->dst_row, d.d_model, ctx->dout);
+    LAUNCHED();
+    scored_rows = Rn;
+    gathered = false;
+  }
+
+  if (trees_out) {
+    DevTree *h = ctx->pin_trees;
+    for (int i = 0; i < n_ep; i++)
+      CU(cudaMemcpyAsync(&h[i], &ctx->trees[episodes[i]], sizeof(DevTree), cudaMemcpyDeviceToHost, st));
+    CU(cudaStreamSynchronize(st));
+    for (int i = 0; i < n_ep; i++) {
+      specvla_tree &t = trees_out[i];
+      if (!t.tokens || !t.parent || !t.depth) return SPECVLA_ERR_INVALID_ARG;
+      t.n_rows = h[i].n_rows;
+      for (int k = 0; k < h[i].n_rows; k++) {
+        t.tokens[k] = h[i].tok[k];
+        t.parent[k] = h[i].parent[k];
+        t.depth[k] = h[i].depth[k];
+        if (t.score) t.score[k] = h[i].score[k];
+      }
+    }
+  }
+  return SPECVLA_OK;
+}
+
+// Verification of the device-resident trees of the episodes in `ea` (rows already counted):
+// forward, greedy tokens, acceptance, path selection, compaction, state update. Results stay
+// on the device (out_m / out_tok / out_path); the caller reads them back.
+static int verify_device_trees(specvla_ctx *ctx, const EpArgs &ea, int R, int r, float *logits_out,
+                               cudaStream_t st) {
+  const specvla_model_desc &d = ctx->desc;
+  const int n_ep = ea.n_ep;
+  tree::build_verify_rows_kernel<<<n_ep, 128, 0, st>>>(ea, ctx->trees, ctx->st, ctx->rt);
+  LAUNCHED();
+  TRY(target_forward(ctx, R, nullptr, st));
+  int s, lo, hi;
+  argmax_range(ctx, &lo, &hi);
+  TRY(lm_head(ctx, ctx->xn, R, st, &s));
+  epi::argmax_kernel<<<R, epi::THREADS, 0, st>>>(ctx->part, s, R, d.vocab, lo, hi, ctx->greedy, ctx->margin,
+                                                 logits_out);
+  LAUNCHED();
+  tree::accept_select_kernel<<<n_ep, 128, 0, st>>>(ea, ctx->trees, ctx->st, ctx->greedy, r, d.action_base,
+                                                   d.n_bins, ctx->feat, d.d_model, ctx->pend_feat,
+                                                   ctx->out_m, ctx->out_tok, ctx->out_path);
+  LAUNCHED();
+  tree::kv_compact_kernel<<<dim3(d.n_layers * 2, n_ep), 256, 0, st>>>(
+      ea, ctx->st, ctx->out_m, ctx->out_path, ctx->kv_t, ctx->kv_t_ep_stride, ctx->kv_t_layer_stride,
+      d.max_seq, ctx->hd);
+  LAUNCHED();
+  tree::advance_state_kernel<<<(n_ep + 63) / 64, 64, 0, st>>>(ea, ctx->st, ctx->out_m);
+  LAUNCHED();
+  return SPECVLA_OK;
+}
+
+// Reads m and the emitted tokens back, synchronises, and updates the host mirror.
+static int finish_verify(specvla_ctx *ctx, const EpArgs &ea, int *accept_len_out, int *tokens_out,
+                         cudaStream_t st) {
+  const int n_ep = ea.n_ep, W = SV_MAX_DEPTH + 1;
+  int *h = ctx->pin_small;
+  CU(cudaMemcpyAsync(h, ctx->out_m, n_ep * sizeof(int), cudaMemcpyDeviceToHost, st));
+  CU(cudaMemcpyAsync(h + SV_MAX_EP, ctx->out_tok, n_ep * W * sizeof(int), cudaMemcpyDeviceToHost, st));
+  CU(cudaStreamSynchronize(st));
+  for (int i = 0; i < n_ep; i++) {
+    const int e = ea.eps[i], m = h[i];
+    if (m < 0 || m > SV_MAX_DEPTH) return SPECVLA_ERR_BAD_STATE;
+    ctx->hP[e] += 1 + m;
+    ctx->hPending[e] = m + 1;
+    ctx->hTreeRows[e] = 0;
+    if (accept_len_out) accept_len_out[i] = m;
+    if (tokens_out)
+      for (int k = 0; k < W; k++) tokens_out[i * W + k] = h[SV_MAX_EP + i * W + k];
+  }
+  return SPECVLA_OK;
+}
+
+int specvla_verify_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const specvla_tree *trees, int r,
+                        int *accept_len_out, int *tokens_out, float *logits_out, void *stream) {
+  TRY(check_episodes(ctx, n_ep, episodes));
+  if (r < 0 || !accept_len_out || !tokens_out) return SPECVLA_ERR_INVALID_ARG;
+  const specvla_model_desc &d = ctx->desc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  EpArgs ea{};
+  ea.n_ep = n_ep;
+  int R = 0;
+  for (int i = 0; i < n_ep; i++) {
+    const int e = episodes[i];
+    if (ctx->hP[e] < 0) return SPECVLA_ERR_BAD_STATE;
+    int rows;
+    if (trees) {
+      TRY(validate_tree(trees[i]));
+      rows = trees[i].n_rows;
+      for (int k = 0; k < rows; k++)
+        if (trees[i].tokens[k] >= d.vocab || (k > 0 && trees[i].tokens[k] < 0)) return SPECVLA_ERR_BAD_TREE;
+    } else {
+      rows = ctx->hTreeRows[e];
+      if (rows < 1) return SPECVLA_ERR_BAD_STATE;
+    }
+    if (ctx->hP[e] + rows > d.max_seq) return SPECVLA_ERR_CAPACITY;
+    ea.eps[i] = e;
+    ea.row0[i] = R;
+    ea.nrows[i] = rows;
+    R += rows;
+  }
+  if (R > d.max_rows || R > ctx->max_lm_rows) return SPECVLA_ERR_CAPACITY;
+  if (trees) {
+    DevTree *h = ctx->pin_trees;
+    for (int i = 0; i < n_ep; i++) {
+      memset(&h[i], 0, sizeof(DevTree));
+      h[i].n_rows = trees[i].n_rows;
+      for (int k = 0; k < trees[i].n_rows; k++) {
+        h[i].tok[k] = trees[i].tokens[k];
+        h[i].parent[k] = trees[i].parent[k];
+        h[i].depth[k] = trees[i].depth[k];
+        h[i].score[k] = trees[i].score ? trees[i].score[k] : 0.f;
+        h[i].drow[k] = -1;
+      }
+      CU(cudaMemcpyAsync(&ctx->trees[episodes[i]], &h[i], sizeof(DevTree), cudaMemcpyHostToDevice, st));
+    }
+  }
+  TRY(verify_device_trees(ctx, ea, R, r, logits_out, st));
+  return finish_verify(ctx, ea, accept_len_out, tokens_out, st);
+}
+
+int specvla_generate_action(specvla_ctx *ctx, int n_ep, const int *episodes, const void *embeds,
+                            const int *token_ids, const int *lens, const specvla_tree_shape *shape, int r,
+                            int n_tokens, int *tokens_out, float *actions_out, specvla_stats *stats,
+                            void *stream) {
+  TRY(check_episodes(ctx, n_ep, episodes));
+  int n_nodes = 0;
+  TRY(validate_shape(shape, &n_nodes));
+  if (r < 0 || n_tokens < 1 || n_tokens > 64 || !tokens_out) return SPECVLA_ERR_INVALID_ARG;
+  if (shape->depth > 0 && !ctx->has_draft) return SPECVLA_ERR_BAD_STATE;
+  const specvla_model_desc &d = ctx->desc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int W = SV_MAX_DEPTH + 1;
+  std::vector<int> first(n_ep), count(n_ep, 0), m_out(n_ep), tok_out((size_t)n_ep * W);
+  if (stats) memset(stats, 0, sizeof(*stats));
+  float ms = 0.f;
+
+  CU(cudaEventRecord(ctx->ev[0], st));
+  TRY(specvla_prefill(ctx, n_ep, episodes, embeds, token_ids, lens, first.data(), nullptr, stream));
+  CU(cudaEventRecord(ctx->ev[1], st));
+  CU(cudaEventSynchronize(ctx->ev[1]));
+  CU(cudaEventElapsedTime(&ms, ctx->ev[0], ctx->ev[1]));
+  if (stats) stats->ms_prefill = ms;
+  for (int i = 0; i < n_ep; i++) {
+    tokens_out[(size_t)i * n_tokens] = first[i];
+    count[i] = 1;
+  }
+  int iterations = 0;
+  for (;;) {
+    bool done = true;
+    for (int i = 0; i < n_ep; i++) done &= (count[i] >= n_tokens);
+    if (done) break;
+    EpArgs ea{};
+    ea.n_ep = n_ep;
+    int R = 0;
+    CU(cudaEventRecord(ctx->ev[0], st));
+    if (shape->depth > 0) {
+      TRY(specvla_draft_tree(ctx, n_ep, episodes, shape, nullptr, stream));
+    } else {
+      // no drafting: a one-row tree (the root) per episode = one autoregressive step
+      DevTree *h = ctx->pin_trees;
+      for (int i = 0; i < n_ep; i++) {
+        memset(&h[i], 0, sizeof(DevTree));
+        h[i].n_rows = 1;
+        h[i].tok[0] = -1;
+        h[i].parent[0] = -1;
+        CU(cudaMemcpyAsync(&ctx->trees[episodes[i]], &h[i], sizeof(DevTree), cudaMemcpyHostToDevice, st));
+        ctx->hTreeRows[episodes[i]] = 1;
+      }
+    }
+    CU(cudaEventRecord(ctx->ev[1], st));
+    for (int i = 0; i < n_ep; i++) {
+      const int e = episodes[i];
+      if (ctx->hP[e] + ctx->hTreeRows[e] > d.max_seq) return SPECVLA_ERR_CAPACITY;
+      ea.eps[i] = e;
+      ea.row0[i] = R;
+      ea.nrows[i] = ctx->hTreeRows[e];
+      R += ctx->hTreeRows[e];
+    }
+    if (R > d.max_rows || R > ctx->max_lm_rows) return SPECVLA_ERR_CAPACITY;
+    TRY(verify_device_trees(ctx, ea, R, r, nullptr, st));
+    CU(cudaEventRecord(ctx->ev[2], st));
+    TRY(finish_verify(ctx, ea, m_out.data(), tok_out.data(), st));
+    if (stats) {
+      CU(cudaEventElapsedTime(&ms, ctx->ev[0], ctx->ev[1]));
+      stats->ms_draft += ms;
+      CU(cudaEventElapsedTime(&ms, ctx->ev[1], ctx->ev[2]));
+      stats->ms_verify += ms;
+      if (iterations < 16) stats->accept_len[iterations] = m_out[0];
+    }
+    for (int i = 0; i < n_ep; i++)
+      for (int k = 0; k <= m_out[i]; k++) {
+        if (count[i] < n_tokens) tokens_out[(size_t)i * n_tokens + count[i]] = tok_out[(size_t)i * W + k];
+        count[i]++;
+      }
+    iterations++;
+    if (iterations > 4 * n_tokens) return SPECVLA_ERR_BAD_STATE;
+  }
+  if (stats) {
+    stats->iterations = iterations;
+    stats->tokens_emitted = count[0];
+  }
+  if (actions_out)
+    for (int i = 0; i < n_ep * n_tokens; i++) {
+      const int b = tokens_out[i] - d.action_base;
+      actions_out[i] = (b >= 0 && b < d.n_bins) ? (-1.f + (2.f * b + 1.f) / d.n_bins) : NAN;
+    }
+  return SPECVLA_OK;
+}
+
+int specvla_read_buffer(specvla_ctx *ctx, int what, void *host_dst, size_t bytes, void *stream) {
+  if (!ctx || !host_dst) return SPECVLA_ERR_INVALID_ARG;
+  const specvla_model_desc &d = ctx->desc;
+  const void *src = nullptr;
+  size_t avail = 0;
+  switch (what) {
+    case SPECVLA_BUF_GREEDY: src = ctx->greedy; avail = (size_t)d.max_rows * sizeof(int); break;
+    case SPECVLA_BUF_MARGIN: src = ctx->margin; avail = (size_t)d.max_rows * sizeof(float); break;
+    case SPECVLA_BUF_FEATURES: src = ctx->feat; avail = (size_t)d.max_rows * d.d_model * sizeof(float); break;
+    case SPECVLA_BUF_PATH: src = ctx->out_path; avail = (size_t)d.max_episodes * (SV_MAX_DEPTH + 1) * sizeof(int); break;
+    case SPECVLA_BUF_DRAFT_TOPK_TOK: src = ctx->top_tok; avail = (size_t)ctx->max_draft_rows * SV_TOPK * sizeof(int); break;
+    case SPECVLA_BUF_DRAFT_TOPK_LP: src = ctx->top_lp; avail = (size_t)ctx->max_draft_rows * SV_TOPK * sizeof(float); break;
+    case SPECVLA_BUF_STATE: {
+      if (bytes > (size_t)d.max_episodes * 4 * sizeof(int)) return SPECVLA_ERR_INVALID_ARG;
+      cudaStream_t st = static_cast<cudaStream_t>(stream);
+      CU(cudaMemcpy2DAsync(host_dst, 4 * sizeof(int), ctx->st, sizeof(EpState), 4 * sizeof(int),
+                           bytes / (4 * sizeof(int)), cudaMemcpyDeviceToHost, st));
+      CU(cudaStreamSynchronize(st));
+      return SPECVLA_OK;
+    }
+    default: return SPECVLA_ERR_INVALID_ARG;
+  }
+  if (bytes > avail) return SPECVLA_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  CU(cudaMemcpyAsync(host_dst, src, bytes, cudaMemcpyDeviceToHost, st));
+  CU(cudaStreamSynchronize(st));
+  return SPECVLA_OK;
+}
+
+int specvla_read_kv(specvla_ctx *ctx, int draft, int episode, int layer, int which, int slot0, int n_slots,
+                    void *host_dst, void *stream) {
+  if (!ctx || !host_dst) return SPECVLA_ERR_INVALID_ARG;
+  const specvla_model_desc &d = ctx->desc;
+  if (episode < 0 || episode >= d.max_episodes || which < 0 || which > 1 || slot0 < 0 || n_slots < 1 ||
+      slot0 + n_slots > d.max_seq)
+    return SPECVLA_ERR_INVALID_ARG;
+  if (draft ? (layer != 0) : (layer < 0 || layer >= d.n_layers)) return SPECVLA_ERR_INVALID_ARG;
+  const bf16 *base = draft ? ctx->kv_d + (size_t)episode * ctx->kv_d_ep_stride
+                           : ctx->kv_t + (size_t)episode * ctx->kv_t_ep_stride + (size_t)layer * ctx->kv_t_layer_stride;
+  base += ((size_t)which * d.max_seq + slot0) * ctx->hd;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  CU(cudaMemcpyAsync(host_dst, base, (size_t)n_slots * ctx->hd * sizeof(bf16), cudaMemcpyDeviceToHost, st));
+  CU(cudaStreamSynchronize(st));
+  return SPECVLA_OK;
+}
+
+// ------------------------------------------------------------------ stand-alone GEMM
+__global__ void sum_splits_kernel(const float *__restrict__ part, int splits, size_t n, float *__restrict__ y) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  float v = 0.f;
+  for (int s = 0; s < splits; s++) v += part[(size_t)s * n + i];
+  y[i] = v;
+}
+
+size_t specvla_gemm_scratch_bytes(int T, int N, int K) {
+  if (T < 1 || N < 1 || K < 8) return 0;
+  return (size_t)gemm_mma::plan_splits(T, N, K, MAX_SPLITS) * T * N * sizeof(float);
+}
+
+int specvla_gemm_bf16(const void *X, const void *W, float *Y, int T, int N, int K, void *scratch,
+                      size_t scratch_bytes, void *stream) {
+  if (!X || !W || !Y || !scratch || T < 1 || N < 1 || K < 8 || (K % 8)) return SPECVLA_ERR_INVALID_ARG;
+  const int splits = gemm_mma::plan_splits(T, N, K, MAX_SPLITS);
+  if (scratch_bytes < (size_t)splits * T * N * sizeof(float)) return SPECVLA_ERR_CAPACITY;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (gemm_mma::launch(static_cast<const bf16 *>(X), static_cast<const bf16 *>(W), static_cast<float *>(scratch),
+                       T, N, K, splits, st) != cudaSuccess)
+    return SPECVLA_ERR_CUDA;
+  const size_t n = (size_t)T * N;
+  sum_splits_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(static_cast<const float *>(scratch), splits, n, Y);
+  return cudaGetLastError() == cudaSuccess ? SPECVLA_OK : SPECVLA_ERR_CUDA;
+}
+
+const char *specvla_strerror(int code) {
+  switch (code) {
+    case SPECVLA_OK: return "ok";
+    case SPECVLA_ERR_INVALID_ARG: return "invalid argument";
+    case SPECVLA_ERR_CAPACITY: return "capacity exceeded (rows, slots, episodes or workspace)";
+    case SPECVLA_ERR_BAD_TREE: return "malformed draft tree";
+    case SPECVLA_ERR_BAD_STATE: return "episode state does not allow this call";
+    case SPECVLA_ERR_CUDA: return "CUDA error";
+    case SPECVLA_ERR_TIMEOUT: return "device-side wait timed out";
+    case SPECVLA_ERR_UNSUPPORTED_ARCH: return "device is not sm_100";
+    default: return "unknown error";
+  }
+}
+
+const char *specvla_last_cuda_error(const specvla_ctx *ctx) { return ctx ? ctx->cuda_err : ""; }
+long long specvla_kernel_launches(const specvla_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+}  // extern "C"

@@ -1,0 +1,304 @@
+// Integer bookkeeping of Spec-VLA decoding on the device: row tables, the static-size draft
+// tree (Section 4.1), relaxed acceptance and longest-accepted-path selection (Eq. 4,
+// Algorithm 1), KV-cache compaction and the per-episode state that links iterations.
+#pragma once
+#include "common.cuh"
+
+namespace tree {
+
+// ---------------------------------------------------------------------------------------
+// Verification rows of each episode's tree: row i sits at position P + depth[i], slot P + i,
+// sees the P committed slots, its ancestors and itself. Also (re)computes vmask so that
+// caller-supplied trees need only tok / parent / depth. One CTA per episode.
+__global__ void build_verify_rows_kernel(EpArgs a, DevTree *trees, const EpState *__restrict__ st,
+                                         RowTable rt) {
+  const int e = a.eps[blockIdx.x];
+  DevTree &tr = trees[e];
+  const int P = st[e].P;
+  for (int i = threadIdx.x; i < tr.n_rows; i += blockDim.x) {
+    uint32_t m[4] = {0, 0, 0, 0};
+    for (int j = i; j >= 0; j = tr.parent[j]) m[j >> 5] |= 1u << (j & 31);
+    const int r = a.row0[blockIdx.x] + i;
+    rt.tok[r] = (i == 0 && tr.tok[0] < 0) ? st[e].root : tr.tok[i];
+    rt.src[r] = 0;
+    rt.ep[r] = e;
+    rt.pos[r] = P + tr.depth[i];
+    rt.slot[r] = P + i;
+    rt.nvis[r] = P;
+    rt.tbase[r] = P;
+#pragma unroll
+    for (int w = 0; w < 4; w++) { rt.mask[r * 4 + w] = m[w]; tr.vmask[i][w] = m[w]; }
+  }
+  if (threadIdx.x == 0 && tr.tok[0] < 0) tr.tok[0] = st[e].root;
+}
+
+// ---------------------------------------------------------------------------------------
+// Draft catch-up rows: the (feature_j, token_j) pairs pending since the last commit run at
+// draft positions Pd + j, causal among themselves. Advances Pd and opens a new tree whose
+// root is the episode's last emitted token. One thread per episode.
+__global__ void build_catchup_rows_kernel(EpArgs a, EpState *st, DevTree *trees, RowTable rt,
+                                          int *__restrict__ feat_src) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= a.n_ep) return;
+  const int e = a.eps[i];
+  EpState &s = st[e];
+  for (int j = 0; j < s.n_pending; j++) {
+    const int r = a.row0[i] + j;
+    rt.tok[r] = s.pending_tok[j];
+    rt.src[r] = 0;
+    rt.ep[r] = e;
+    rt.pos[r] = s.Pd + j;
+    rt.slot[r] = s.Pd + j;
+    rt.nvis[r] = s.Pd + j + 1;
+    rt.tbase[r] = 0;
+    for (int w = 0; w < 4; w++) rt.mask[r * 4 + w] = 0;
+    feat_src[r] = e * SV_MAX_PENDING + j;          // row of the pending-feature buffer
+  }
+  s.Pd += s.n_pending;
+  DevTree &tr = trees[e];
+  tr.n_rows = 1;
+  tr.n_drows = 1;
+  tr.tok[0] = s.root;
+  tr.parent[0] = -1;
+  tr.depth[0] = 0;
+  tr.score[0] = 0.f;
+  tr.drow[0] = 0;
+  for (int w = 0; w < 4; w++) { tr.vmask[0][w] = (w == 0); tr.dmask[0][w] = 0; }
+  tr.level_begin = 0;
+  tr.level_end = 1;
+  tr.sel_count = 1;
+  tr.sel[0] = 0;
+}
+
+// Draft-model input rows: xin[r] = bf16([feature ; embedding]) with the feature taken from
+// row feat_src[r] of `feat` and the embedding from E[tok] (or embeds[src] when tok < 0).
+__global__ void draft_input_kernel(RowTable rt, const int *__restrict__ feat_src,
+                                   const float *__restrict__ feat, const bf16 *__restrict__ embeds,
+                                   const bf16 *__restrict__ E, int d, bf16 *__restrict__ xin) {
+  const int r = blockIdx.x;
+  const float *f = feat + (size_t)feat_src[r] * d;
+  const int tok = rt.tok[r];
+  const bf16 *e = tok >= 0 ? E + (size_t)tok * d : embeds + (size_t)rt.src[r] * d;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) {
+    xin[(size_t)r * 2 * d + i] = __float2bfloat16(f[i]);
+    xin[(size_t)r * 2 * d + d + i] = e[i];
+  }
+}
+
+// Saves the draft outputs of the rows just run: dout[e][drow] = x[row]. For the catch-up
+// call only each episode's last row is kept, as draft row 0.
+__global__ void save_draft_out_kernel(const float *__restrict__ x, const int *__restrict__ dst_row,
+                                      int d, float *__restrict__ dout) {
+  const int r = blockIdx.x;
+  const int dst = dst_row[r];
+  if (dst < 0) return;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) dout[(size_t)dst * d + i] = x[(size_t)r * d + i];
+}
+
+// dst_row for the catch-up call: last pending row of episode i -> dout row e * SV_MAX_TREE.
+__global__ void catchup_dst_kernel(EpArgs a, int *__restrict__ dst_row, int *__restrict__ lm_rows) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= a.n_ep) return;
+  for (int j = 0; j < a.nrows[i]; j++) dst_row[a.row0[i] + j] = -1;
+  const int last = a.row0[i] + a.nrows[i] - 1;
+  dst_row[last] = a.eps[i] * SV_MAX_TREE;
+  lm_rows[i] = last;
+}
+
+// One level of tree growth. The rows scored last (one per selected parent, in rank order)
+// come with their top-K tokens and log-probabilities; parent sel[j] gets `branch` children
+// (score = parent score + log-prob). Then the `expand_next` best new nodes (by score, ties
+// to the lower node index) are selected, in rank order, and their draft rows are laid out
+// for the next level: input feature = output of the row that scored them, token = their own.
+// One thread per episode (at most 128 nodes, 16 per level).
+// a.row0 = first scored row of each episode, a.aux = first row of its next level.
+__global__ void expand_level_kernel(EpArgs a, int level, int branch, int expand_next,
+                                    const int *__restrict__ top_tok, const float *__restrict__ top_lp,
+                                    DevTree *trees, const EpState *__restrict__ st, RowTable rt,
+                                    int *__restrict__ feat_src, int *__restrict__ dst_row) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= a.n_ep) return;
+  const int e = a.eps[i];
+  DevTree &tr = trees[e];
+  const int begin = tr.n_rows;
+  for (int j = 0; j < tr.sel_count; j++) {
+    const int p = tr.sel[j];
+    const int srow = a.row0[i] + j;
+    for (int b = 0; b < branch; b++) {
+      const int n = tr.n_rows++;
+      tr.tok[n] = top_tok[srow * SV_TOPK + b];
+      tr.parent[n] = p;
+      tr.depth[n] = level + 1;
+      tr.score[n] = tr.score[p] + top_lp[srow * SV_TOPK + b];
+      tr.drow[n] = -1;
+      for (int w = 0; w < 4; w++) tr.vmask[n][w] = tr.vmask[p][w];
+      tr.vmask[n][n >> 5] |= 1u << (n & 31);
+    }
+  }
+  tr.level_begin = begin;
+  tr.level_end = tr.n_rows;
+  // selection of the next level's parents: repeated arg-best (<= 16 x 16 comparisons)
+  int cnt = 0;
+  uint32_t used = 0;
+  for (; cnt < expand_next && cnt < tr.level_end - begin; cnt++) {
+    int best = -1;
+    for (int n = begin; n < tr.level_end; n++) {
+      if (used & (1u << (n - begin))) continue;
+      if (best < 0 || tr.score[n] > tr.score[best]) best = n;
+    }
+    used |= 1u << (best - begin);
+    tr.sel[cnt] = best;
+  }
+  tr.sel_count = cnt;
+  const int Pd = st[e].Pd;
+  for (int j = 0; j < cnt; j++) {
+    const int n = tr.sel[j];
+    const int dr = tr.n_drows++;
+    const int pdr = tr.drow[tr.parent[n]];
+    tr.drow[n] = dr;
+    for (int w = 0; w < 4; w++) tr.dmask[dr][w] = tr.dmask[pdr][w];
+    tr.dmask[dr][dr >> 5] |= 1u << (dr & 31);
+    const int r = a.aux[i] + j;
+    rt.tok[r] = tr.tok[n];
+    rt.src[r] = 0;
+    rt.ep[r] = e;
+    rt.pos[r] = Pd - 1 + level + 1;
+    rt.slot[r] = Pd - 1 + dr;              // draft row dr >= 1 -> slot Pd + (dr - 1)
+    rt.nvis[r] = Pd;
+    rt.tbase[r] = Pd - 1;                  // bit dr of dmask <-> slot Pd - 1 + dr
+    for (int w = 0; w < 4; w++) rt.mask[r * 4 + w] = tr.dmask[dr][w];
+    feat_src[r] = e * SV_MAX_TREE + pdr;   // row of dout
+    dst_row[r] = e * SV_MAX_TREE + dr;
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Relaxed acceptance (Eq. 4) and longest-accepted-path selection, one warp per episode.
+// Node i is accepted iff its parent is accepted and |bin(tok[i]) - bin(g[parent[i]])| <= r
+// (ids outside [a0, a0 + nb) must be equal). The deepest accepted node wins, ties to the
+// lowest row. Lanes own rows i, i+32, ...; acceptance spreads one tree level per round
+// through ballots of the per-lane flags. Emits the m accepted draft tokens plus g[n*],
+// commits the state for the next iteration and gathers the features on the path.
+__global__ void __launch_bounds__(128)
+accept_select_kernel(EpArgs ea, DevTree *trees, EpState *st, const int *__restrict__ greedy, int r, int a0, int nb,
+                     const float *__restrict__ feat, int d, float *__restrict__ pend_feat,
+                     int *__restrict__ out_m, int *__restrict__ out_tok, int *__restrict__ out_path) {
+  __shared__ int s_path[SV_MAX_DEPTH + 1], s_m;
+  const int e = ea.eps[blockIdx.x];
+  const int base = ea.row0[blockIdx.x];
+  DevTree &tr = trees[e];
+  const int n = tr.n_rows;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (warp == 0) {
+    bool ok[4], a[4];
+#pragma unroll
+    for (int k = 0; k < 4; k++) {
+      const int i = lane + 32 * k;
+      ok[k] = false;
+      a[k] = (i == 0);
+      if (i > 0 && i < n) {
+        const int dt = tr.tok[i], gt = greedy[base + tr.parent[i]];
+        const bool da = dt >= a0 && dt < a0 + nb, ga = gt >= a0 && gt < a0 + nb;
+        ok[k] = (da && ga) ? (abs(dt - gt) <= r) : (dt == gt);
+      }
+    }
+    for (int round = 0; round < SV_MAX_DEPTH; round++) {
+      uint32_t words[4];
+#pragma unroll
+      for (int k = 0; k < 4; k++) words[k] = __ballot_sync(0xffffffffu, a[k]);
+#pragma unroll
+      for (int k = 0; k < 4; k++) {
+        const int i = lane + 32 * k;
+        if (i > 0 && i < n && ok[k]) {
+          const int p = tr.parent[i];
+          a[k] = (words[p >> 5] >> (p & 31)) & 1u;
+        }
+      }
+    }
+    // deepest accepted node, ties to the lowest row: maximise depth * 128 + (127 - row)
+    int key = -1;
+#pragma unroll
+    for (int k = 0; k < 4; k++) {
+      const int i = lane + 32 * k;
+      if (i < n && a[k]) key = max(key, tr.depth[i] * SV_MAX_TREE + (SV_MAX_TREE - 1 - i));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) key = max(key, __shfl_xor_sync(0xffffffffu, key, o));
+    if (lane == 0) {
+      const int best = SV_MAX_TREE - 1 - (key % SV_MAX_TREE);
+      const int m = tr.depth[best];
+      int j = best;
+      for (int k = m; k >= 0; k--) { s_path[k] = j; j = tr.parent[j]; }
+      s_m = m;
+      EpState &s = st[e];
+      int *ot = out_tok + blockIdx.x * (SV_MAX_DEPTH + 1);
+      int *op = out_path + blockIdx.x * (SV_MAX_DEPTH + 1);
+      for (int k = 0; k <= SV_MAX_DEPTH; k++) { ot[k] = -1; op[k] = -1; }
+      for (int k = 1; k <= m; k++) ot[k - 1] = tr.tok[s_path[k]];
+      ot[m] = greedy[base + best];
+      for (int k = 0; k <= m; k++) { op[k] = s_path[k]; s.pending_tok[k] = ot[k]; }
+      out_m[blockIdx.x] = m;
+      s.root = ot[m];
+      s.n_pending = m + 1;
+      // s.P is advanced by the compaction kernel, which still needs the old value
+    }
+  }
+  __syncthreads();
+  const int m = s_m;
+  for (int k = 0; k <= m; k++) {
+    const float *src = feat + (size_t)(base + s_path[k]) * d;
+    float *dst = pend_feat + (size_t)(e * SV_MAX_PENDING + k) * d;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) dst[i] = src[i];
+  }
+}
+
+// In-place KV compaction: accepted row path[j] moves from slot P + path[j] to slot P + j
+// (j = 1..m) in every layer, K and V. path[j] >= j and path is increasing, so copying in
+// ascending j never overwrites a source that is still needed; every 16-byte column chunk is
+// handled by one thread, which keeps that order. grid = (layers * 2, episodes).
+__global__ void __launch_bounds__(256)
+kv_compact_kernel(EpArgs a, const EpState *__restrict__ st,
+                  const int *__restrict__ out_m, const int *__restrict__ out_path,
+                  bf16 *__restrict__ cache, size_t ep_stride, size_t layer_stride, int max_seq, int hd) {
+  const int e = a.eps[blockIdx.y];
+  const int m = out_m[blockIdx.y];
+  const int P = st[e].P;
+  const int *path = out_path + blockIdx.y * (SV_MAX_DEPTH + 1);
+  const int layer = blockIdx.x >> 1, which = blockIdx.x & 1;
+  uint4 *base = reinterpret_cast<uint4 *>(cache + (size_t)e * ep_stride + (size_t)layer * layer_stride +
+                                          (size_t)which * max_seq * hd);
+  const int chunks = hd / 8;
+  for (int j = 1; j <= m; j++) {
+    const int src = P + path[j], dst = P + j;
+    if (src == dst) continue;
+    for (int c = threadIdx.x; c < chunks; c += blockDim.x)
+      base[(size_t)dst * chunks + c] = base[(size_t)src * chunks + c];
+  }
+}
+
+// P <- P + 1 + m after compaction.
+__global__ void advance_state_kernel(EpArgs a, EpState *st, const int *__restrict__ out_m) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < a.n_ep) st[a.eps[i]].P += 1 + out_m[i];
+}
+
+// State after prefill: P = len, Pd = len - 1, root = a_1, one pending pair (f_{P-1}, a_1).
+// a.nrows = prefix lengths, a.aux = last row of each episode.
+__global__ void prefill_commit_kernel(EpArgs a, EpState *st,
+                                      const int *__restrict__ greedy, const float *__restrict__ feat,
+                                      int d, float *__restrict__ pend_feat) {
+  const int e = a.eps[blockIdx.x];
+  if (threadIdx.x == 0) {
+    EpState &s = st[e];
+    s.P = a.nrows[blockIdx.x];
+    s.Pd = a.nrows[blockIdx.x] - 1;
+    s.root = greedy[blockIdx.x];
+    s.n_pending = 1;
+    s.pending_tok[0] = greedy[blockIdx.x];
+  }
+  const float *src = feat + (size_t)a.aux[blockIdx.x] * d;
+  float *dst = pend_feat + (size_t)e * SV_MAX_PENDING * d;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) dst[i] = src[i];
+}
+
+}  // namespace tree
