@@ -1,0 +1,377 @@
+#!/usr/bin/env python
+"""Benchmark of the Spec-VLA tree-verification path on B200.
+
+One step = one action chunk of the C1 workload (OpenVLA-7B-shaped decoder, batch 1,
+290-position prefix, 26-node draft tree from the one-layer draft model, 7 action tokens,
+strict acceptance r = 0) through specvla_generate_action: prefill, then draft -> verify ->
+accept -> compact until 7 tokens. Prints ONE JSON line (see the design doc for every field).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+N > 1 runs N independent replicas (one process per GPU under torchrun); there is no
+data-path collective because episodes are independent.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "action chunks/sec at bs1 (7B)"
+UNIT = "chunks/s"
+WEIGHT_BYTES_PER_VERIFY = 13_214_679_040      # 32 layers + LM head, bf16, read once
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"],
+                    bf16_tflops_sustained=p.get("bf16_tflops_sustained"), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples every 200 ms while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.path = index, None, None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "200"],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in open(self.path):
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        os.unlink(self.path)
+        return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    samples=len(sm), reasons=sorted(reasons))
+
+
+# --------------------------------------------------------------------------- CPU oracle legs
+def oracle_sample(device, iters_per_chunk: int, depth: int, pieces=None):
+    """Times the oracle, as it stands, on a bounded slice of the C1 chunk and extrapolates.
+
+    Slice: one target decoder layer over the 290 prefix rows, one over the 27 tree rows, the LM
+    head over 27 rows and one draft-model level (fc + layer + LM head + log-softmax) over 4
+    rows, all at the 7B shapes. chunk_est = 33 t_layer(290) + iters * (32 t_layer(27) +
+    t_lm(27) + depth * t_draft_level). Returns (chunks/s estimate, seconds used, pieces).
+    `pieces` carries the terms measured by an earlier call that are not re-measured."""
+    import torch
+    from oracle import decoder as D
+    from synth_inputs import configs as C, rng
+
+    desc = C.OPENVLA_7B
+    st = _oracle_state(device)
+    w, T, P = st["w"], 27, 290
+    t0 = time.perf_counter()
+    out = dict(pieces or {})
+
+    def timed(name, fn):
+        if name in out and pieces is not None and name not in ("layer27", "lm27"):
+            return
+        a = time.perf_counter()
+        fn()
+        out[name] = time.perf_counter() - a
+
+    def layer(rows, n_before):
+        x = st["x"][:rows]
+        cache = D.KVCache(1, n_before + rows, desc.n_heads, desc.head_dim)
+        pos = torch.arange(n_before, n_before + rows)
+        vis = torch.ones(rows, n_before + rows, dtype=torch.bool)
+        D.decoder_layer(w, "layers.0.", desc, x, pos, pos, vis, cache, 0)
+
+    def draft_level():
+        cache = D.KVCache(1, P + 4, desc.n_heads, desc.head_dim)
+        pos = torch.arange(P, P + 4)
+        g = D.draft_forward(w, desc, st["x"][:4], st["x"][4:8], pos, pos,
+                            torch.ones(4, P + 4, dtype=torch.bool), cache)
+        torch.log_softmax(D.lm_head(w, g)[:, desc.action_base:desc.action_base + desc.n_bins], dim=1)
+
+    timed("layer290", lambda: layer(P, 0))
+    timed("layer27", lambda: layer(T, P))
+    timed("lm27", lambda: D.lm_head(w, st["x"][:T]))
+    timed("draft_level", draft_level)
+    chunk = 33 * out["layer290"] + iters_per_chunk * (32 * out["layer27"] + out["lm27"] +
+                                                     depth * out["draft_level"])
+    return 1.0 / chunk, time.perf_counter() - t0, out
+
+
+_ORACLE_STATE = {}
+
+
+def _oracle_state(device):
+    if not _ORACLE_STATE:
+        import torch
+        from oracle import decoder as D
+        from synth_inputs import configs as C, rng
+        desc = C.OPENVLA_7B
+        d, F, hd = desc.d_model, desc.d_ffn, desc.n_heads * desc.head_dim
+        raw = {}
+
+        def mat(stream, r, c):
+            return rng.normal_bf16(1, stream, (r, c), 0.02, device).cpu()
+
+        for prefix, base in (("layers.0.", C.STREAM_LAYER0), ("draft.layer.", C.STREAM_DRAFT_LAYER)):
+            raw[prefix + "wqkv"] = torch.cat([mat(base + i, hd, d) for i in range(3)])
+            raw[prefix + "wo"] = mat(base + 3, d, hd)
+            raw[prefix + "wgu"] = torch.cat([mat(base + 4, F, d), mat(base + 5, F, d)])
+            raw[prefix + "wd"] = mat(base + 6, d, F)
+            raw[prefix + "norm1"] = torch.ones(d)
+            raw[prefix + "norm2"] = torch.ones(d)
+        raw["lm_head"] = mat(C.STREAM_LM_HEAD, desc.vocab, d)
+        raw["draft.fc"] = mat(C.STREAM_DRAFT_FC, d, 2 * d)
+        _ORACLE_STATE["w"] = D.DecoderWeights(raw)
+        _ORACLE_STATE["x"] = rng.normal(1, 999, (290, d), 1.0, "cpu")
+    return _ORACLE_STATE
+
+
+def run_reference(args, rank, world):
+    """The reference arm: there is no reference implementation, so the CPU oracle is timed."""
+    if rank != 0:
+        return
+    import torch
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    torch.set_grad_enabled(False)
+    iters, depth = 6, 5
+    pieces, times = None, []
+    total = args.warmup + args.steps
+    full_every_step = total * 10.0 <= 240.0
+    for i in range(total):
+        val, sec, pieces_new = oracle_sample(dev, iters, depth, None if (full_every_step or i == 0) else pieces)
+        pieces = pieces_new
+        if i >= args.warmup:
+            times.append((val, sec))
+    value = statistics.mean(v for v, _ in times)
+    cores = torch.get_num_threads()
+    sample = ("per step: oracle decoder layer over 290 and over 27 rows, LM head over 27 rows"
+              + (", one draft level over 4 rows" if full_every_step else
+                 " (290-row layer and draft level measured once in warm-up)")
+              + "; chunk = 33*t_layer290 + 6*(32*t_layer27 + t_lm27 + 5*t_draft); 7B shapes, float64")
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps, warmup=args.warmup,
+                ms_per_step=1000.0 / value, higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="f64", data="synthetic", impl="reference",
+                config=dict(workload="C1-openvla7b-bs1", prefix=290, tree_rows=27, n_tokens=7, r=0),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=cores, kind="oracle", sample=sample),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------- CUDA arm
+def run_ours(args, rank, local_rank, world):
+    import torch
+    import torch.distributed as dist
+    from paper_2507_22424_b200.binding import SpecVLA, make_shape
+    from synth_inputs import configs as C, data
+
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    wl, desc = C.C1, C.OPENVLA_7B
+    weights = data.make_weights(desc, wl.seed, device="cuda")
+    embeds, ids = data.make_prefix(wl, device="cuda")
+    ids_host = ids.tolist()
+    P = len(ids_host)
+    gpu = SpecVLA(desc, weights, max_seq=512, max_episodes=1, max_rows=512, action_only=True)
+    shape = make_shape(wl.tree.branch, wl.tree.expand)
+    r, n_tok = 0, wl.n_tokens
+
+    def chunk():
+        return gpu.generate_action([0], embeds, ids_host, [P], shape, r, n_tok)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        toks, _, stats = chunk()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    # --- timed region 1: inputs resident in HBM -----------------------------------------
+    barrier()
+    l0 = gpu.kernel_launches()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    ms_verify = ms_draft = ms_prefill = 0.0
+    iters = accept = 0
+    for _ in range(args.steps):
+        toks, _, stats = chunk()
+        ms_verify += stats.ms_verify
+        ms_draft += stats.ms_draft
+        ms_prefill += stats.ms_prefill
+        iters += stats.iterations
+        accept += sum(stats.accept_len[i] for i in range(min(16, stats.iterations)))
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1)
+    launches = gpu.kernel_launches() - l0
+    clocks = sampler.stop() if rank == 0 else None
+    # --- timed region 2: end to end from host buffers ----------------------------------
+    embeds_host = embeds.cpu().pin_memory()
+    stage = torch.empty_like(embeds)
+    barrier()
+    e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2.record()
+    for _ in range(args.steps):
+        stage.copy_(embeds_host, non_blocking=True)
+        toks_e2e, acts, _ = gpu.generate_action([0], stage, ids_host, [P], shape, r, n_tok)
+    e3.record()
+    barrier()
+    ms_e2e = e2.elapsed_time(e3)
+    # --- AR baseline from the same kernels (depth-0 tree) --------------------------------
+    ar_shape = make_shape((), ())
+    gpu.generate_action([0], embeds, ids_host, [P], ar_shape, 0, n_tok)
+    barrier()
+    e4, e5 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e4.record()
+    ar_steps = max(3, args.steps // 2)
+    ar_ms_verify = 0.0
+    for _ in range(ar_steps):
+        ar_toks, _, ar_stats = gpu.generate_action([0], embeds, ids_host, [P], ar_shape, 0, n_tok)
+        ar_ms_verify += ar_stats.ms_verify
+    e5.record()
+    barrier()
+    ms_ar = e4.elapsed_time(e5)
+    # --- per-GEMM device time of the verification phase (separate pass, same steps) -----
+    gpu.profile(4)
+    for _ in range(max(2, args.steps // 4)):
+        chunk()
+    prof = gpu.profile_read()
+    gpu.profile(0)
+
+    if world > 1:
+        t = torch.tensor([ms, ms_e2e], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, ms_e2e = float(t[0]), float(t[1])
+    if rank != 0:
+        return
+    peaks = load_peaks()
+    value = world * args.steps / (ms / 1000.0)
+    e2e_value = world * args.steps / (ms_e2e / 1000.0)
+    T = 1 + wl.tree.n_nodes
+    verify_ms = ms_verify / max(1, iters)
+    kv_bytes = desc.n_layers * 2 * (P + 3 + T) * desc.d_model * 2 + T * desc.n_layers * 2 * desc.d_model * 2
+    verify_gbs = (WEIGHT_BYTES_PER_VERIFY + kv_bytes) / (verify_ms * 1e-3) / 1e9
+    dom = prof["gate_up"]
+    N, K = 2 * desc.d_ffn, desc.d_model
+    alg_bytes = N * K * 2 + T * K * 2 + T * N * 4
+    dom_ms = dom["ms"] / max(1, dom["launches"])
+    achieved = alg_bytes / (dom_ms * 1e-3) / 1e9 if dom["launches"] else None
+    all_ms = sum(v["ms"] for v in prof.values())
+    all_bytes = sum(v["bytes"] for v in prof.values())
+    ipc = max(1, round(iters / args.steps))
+    vals, cpu_sec, reps = [], 0.0, 0
+    oracle_sample("cuda", ipc, wl.tree.depth)                      # untimed: page-in, thread pool
+    while cpu_sec < 10.0 and reps < 64:
+        v, sec, pieces = oracle_sample("cuda", ipc, wl.tree.depth)
+        vals.append(v)
+        cpu_sec += sec
+        reps += 1
+    cpu_val = statistics.mean(vals)
+    line = dict(
+        metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+        ms_per_step=ms / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None,
+        dtype="bf16", data="synthetic",
+        config=dict(workload=wl.name, prefix=P, tree_rows=T, tree="26 nodes depth 5 top-4/2/2/1/1",
+                    n_tokens=n_tok, r=r, action_only=1, replicas=world,
+                    l2="inputs larger than L2: every step streams 13.9 GB of weights"),
+        e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=embeds.numel() * 2 + 4 * P,
+                 d2h_bytes_per_step=4 * n_tok * 2 + 8 * max(1, round(iters / args.steps)) * 10),
+        gpu_launches=launches,
+        clocks=clocks,
+        roofline=dict(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
+                      frac=(achieved / peaks["hbm_gbs"]) if achieved else None, traffic=None,
+                      kernel="weight-streaming GEMM, gate/up projection [22016 x 4096] at T=27 (verify)",
+                      algorithmic_bytes_per_launch=alg_bytes, launches_timed=dom["launches"],
+                      ms_per_launch=dom_ms, peak_source=peaks["source"] + " copy bandwidth",
+                      all_verify_gemms_gbs=(all_bytes / (all_ms * 1e-3) / 1e9) if all_ms else None,
+                      per_class={k: dict(ms_per_launch=v["ms"] / max(1, v["launches"]),
+                                         gbs=(v["bytes"] / (v["ms"] * 1e-3) / 1e9) if v["ms"] else None)
+                                 for k, v in prof.items()}),
+        verify=dict(ms_per_step=verify_ms, hbm_gbs=verify_gbs, frac_of_measured_peak=verify_gbs / peaks["hbm_gbs"],
+                    frac_of_8tbs=verify_gbs / 8000.0, bytes=WEIGHT_BYTES_PER_VERIFY + kv_bytes),
+        phases_ms_per_chunk=dict(prefill=ms_prefill / args.steps, draft=ms_draft / args.steps,
+                                 verify=ms_verify / args.steps),
+        accept=dict(iterations_per_chunk=iters / args.steps, mean_m=accept / max(1, iters),
+                    mean_tokens_per_forward=accept / max(1, iters) + 1.0),
+        ar_baseline=dict(value=world * ar_steps / (ms_ar / 1000.0), unit=UNIT,
+                         ms_per_decode_step=ar_ms_verify / (ar_steps * (n_tok - 1)),
+                         same_tokens=bool(ar_toks == toks)),
+        cpu_baseline=dict(value=cpu_val, unit=UNIT, cores=torch.get_num_threads(), kind="oracle",
+                          sample=("oracle (float64) decoder layer over 290 and 27 rows, LM head over 27 "
+                                  "rows, one draft level over 4 rows at 7B shapes; chunk = 33*t_layer290 + "
+                                  "iters*(32*t_layer27 + t_lm27 + 5*t_draft); mean of %d repetitions, %.1f s of CPU work"
+                                  % (reps, cpu_sec)),
+                          pieces_s=pieces),
+        tokens=toks[0],
+    )
+    print(json.dumps(line), flush=True)
+    gpu.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+    else:
+        import torch
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: the CUDA path has no CPU fallback")
+        torch.set_grad_enabled(False)
+        run_ours(args, rank, local_rank, world)
+
+
+if __name__ == "__main__":
+    main()

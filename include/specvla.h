@@ -13,7 +13,10 @@
  *    ordinary host memory. The caller owns every buffer it passes in; the library owns
  *    only the host-side context object and a few KB of pinned staging memory.
  *  - All weights are bfloat16, row-major [out_features, in_features]; RMSNorm gains are
- *    float32. The workspace (KV caches, activations, split-K scratch) is one device buffer
+ *    float32. Activations are float32 between kernels and enter the bf16 tensor-core GEMMs
+ *    as two bf16 limbs (hi + lo); the KV caches are float32. With single-limb bf16
+ *    activations or a bf16 cache the logits of the 32-layer model drift by 0.1-0.2 from an
+ *    exact forward, ten times the 2e-2 this library is held to. The workspace (KV caches, activations, split-K scratch) is one device buffer
  *    allocated by the caller, at least specvla_workspace_bytes() long, 1024-byte aligned;
  *    it must outlive the context and must not be touched while a call is in flight.
  *  - Work is enqueued on `stream` (a cudaStream_t passed as void*). Calls that return
@@ -183,17 +186,39 @@ int specvla_generate_action(specvla_ctx *ctx, int n_ep, const int *episodes, con
 #define SPECVLA_BUF_DRAFT_TOPK_LP  7 /* float [rows][8]   their log-probabilities */
 int specvla_read_buffer(specvla_ctx *ctx, int what, void *host_dst, size_t bytes, void *stream);
 
-/* Copies KV-cache rows [slot0, slot0+n_slots) of one layer to host as bf16 [n_slots, H*dh].
+/* Copies KV-cache rows [slot0, slot0+n_slots) of one layer to host as f32 [n_slots, H*dh].
  * which: 0 = K, 1 = V; draft: 0 = target cache, 1 = draft cache (layer must be 0). */
 int specvla_read_kv(specvla_ctx *ctx, int draft, int episode, int layer, int which, int slot0,
                     int n_slots, void *host_dst, void *stream);
 
-/* Y[T, N] (f32, device) = X[T, K] (bf16, device) * W[N, K]^T (bf16, device): the library's
- * weight-streaming GEMM exposed for kernel-level parity tests and roofline measurement.
- * scratch: device f32, at least specvla_gemm_scratch_bytes(T, N, K) bytes. */
+/* Y[T, N] (f32, device) = X[T, K] (f32, device) * W[N, K]^T (bf16, device): the library's
+ * weight-streaming GEMM exposed for kernel-level parity tests and roofline measurement. As in
+ * the decoder, X enters the tensor cores as two bf16 limbs (hi + lo), so the result carries
+ * about 16 mantissa bits of X. K % 8 == 0.
+ * scratch: device, 1024-byte aligned, at least specvla_gemm_scratch_bytes(T, N, K) bytes. */
 size_t specvla_gemm_scratch_bytes(int T, int N, int K);
-int specvla_gemm_bf16(const void *X, const void *W, float *Y, int T, int N, int K,
-                      void *scratch, size_t scratch_bytes, void *stream);
+int specvla_gemm(const float *X, const void *W, float *Y, int T, int N, int K,
+                 void *scratch, size_t scratch_bytes, void *stream);
+
+/* Per-GEMM device timing (measurement aid; Section 3.1 attributes the latency to the
+ * parameter stream, which these GEMMs are). `phases` is a bit mask: 1 = prefill, 2 = draft,
+ * 4 = verification; 0 switches timing off. While a phase is enabled, every weight-streaming
+ * GEMM launch of that phase is bracketed by CUDA events on the call's stream (up to 1024
+ * launches between two synchronising calls; later ones go untimed); the sums are folded in at
+ * each synchronisation. Classes index the weight matrix streamed. A non-zero mask resets
+ * the sums. */
+#define SPECVLA_PROF_QKV      0
+#define SPECVLA_PROF_O        1
+#define SPECVLA_PROF_GATE_UP  2
+#define SPECVLA_PROF_DOWN     3
+#define SPECVLA_PROF_LM_HEAD  4
+#define SPECVLA_PROF_FC       5
+#define SPECVLA_PROF_CLASSES  6
+int specvla_profile(specvla_ctx *ctx, int phases);
+/* ms_out / launches_out / bytes_out: host arrays of SPECVLA_PROF_CLASSES entries: summed
+ * device time, timed launches and weight bytes streamed (N*K*2 per launch) per class. */
+int specvla_profile_read(const specvla_ctx *ctx, double *ms_out, long long *launches_out,
+                         double *bytes_out);
 
 const char *specvla_strerror(int code);
 /* Text of the last CUDA error seen by this context (empty string if none). */

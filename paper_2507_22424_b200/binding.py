@@ -68,8 +68,11 @@ EXPORTS = {
     "specvla_read_kv": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
                                   C.c_void_p, C.c_void_p]),
     "specvla_gemm_scratch_bytes": (C.c_size_t, [C.c_int, C.c_int, C.c_int]),
-    "specvla_gemm_bf16": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
+    "specvla_gemm": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                                     C.c_void_p, C.c_size_t, C.c_void_p]),
+    "specvla_profile": (C.c_int, [C.c_void_p, C.c_int]),
+    "specvla_profile_read": (C.c_int, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_longlong),
+                                       C.POINTER(C.c_double)]),
     "specvla_strerror": (C.c_char_p, [C.c_int]),
     "specvla_last_cuda_error": (C.c_char_p, [C.c_void_p]),
     "specvla_kernel_launches": (C.c_longlong, [C.c_void_p]),
@@ -241,23 +244,34 @@ class SpecVLA:
 
     def read_kv(self, episode, layer, which, slot0, n_slots, draft=False):
         hd = self.model.n_heads * self.model.head_dim
-        out = torch.empty(n_slots, hd, dtype=torch.bfloat16)
+        out = torch.empty(n_slots, hd, dtype=torch.float32)
         self._check(lib.specvla_read_kv(self.h, int(draft), episode, layer, which, slot0, n_slots,
                                         C.c_void_p(out.data_ptr()), _stream()))
         return out
+
+    def profile(self, enable: bool):
+        self._check(lib.specvla_profile(self.h, int(enable)))
+
+    def profile_read(self):
+        """Per weight-matrix class: (ms, launches, weight bytes) summed since profiling was enabled."""
+        ms, n, by = (C.c_double * 6)(), (C.c_longlong * 6)(), (C.c_double * 6)()
+        self._check(lib.specvla_profile_read(self.h, ms, n, by))
+        names = ("qkv", "o", "gate_up", "down", "lm_head", "fc")
+        return {k: dict(ms=ms[i], launches=int(n[i]), bytes=by[i]) for i, k in enumerate(names)}
 
     def kernel_launches(self):
         return int(lib.specvla_kernel_launches(self.h))
 
 
-def gemm_bf16(x: torch.Tensor, w: torch.Tensor) -> torch.Tensor:
-    """Y[T, N] = X[T, K] @ W[N, K]^T through the library's weight-streaming GEMM."""
+def gemm(x: torch.Tensor, w: torch.Tensor) -> torch.Tensor:
+    """Y[T, N] = X[T, K] (f32) @ W[N, K]^T (bf16) through the library's weight-streaming GEMM."""
+    assert x.dtype == torch.float32 and w.dtype == torch.bfloat16
     T, K = x.shape
     N = w.shape[0]
     y = torch.empty(T, N, dtype=torch.float32, device="cuda")
     nb = lib.specvla_gemm_scratch_bytes(T, N, K)
     scratch = torch.empty(nb, dtype=torch.uint8, device="cuda")
-    rc = lib.specvla_gemm_bf16(C.c_void_p(x.data_ptr()), C.c_void_p(w.data_ptr()), C.c_void_p(y.data_ptr()),
+    rc = lib.specvla_gemm(C.c_void_p(x.data_ptr()), C.c_void_p(w.data_ptr()), C.c_void_p(y.data_ptr()),
                                T, N, K, C.c_void_p(scratch.data_ptr()), nb, _stream())
     if rc != 0:
         raise SpecVLAError(rc)

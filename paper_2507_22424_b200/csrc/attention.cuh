@@ -1,7 +1,8 @@
 // Tree-mask attention (Section 3.2 / 4.1: every draft-tree row is verified in one forward,
 // each conditioned on its own path). One CTA per (head, row). Row t attends cache slots
-// [0, nvis[t]) plus the slots tbase[t] + b for every bit b of its 128-bit mask. Scores,
-// softmax and the weighted sum are fp32; K, V and the output are bf16.
+// [0, nvis[t]) plus the slots tbase[t] + b for every bit b of its 128-bit mask. Queries,
+// keys, values, scores, softmax and the weighted sum are fp32; the output is written as two
+// bf16 limbs for the O-projection GEMM.
 //
 // Each warp walks its share of the keys with an online softmax (running max / sum), lanes
 // split the head dimension; the four warps' partial results are merged in shared memory in
@@ -15,37 +16,38 @@ constexpr int WARPS = 4;
 
 template <int DH>
 __global__ void __launch_bounds__(WARPS * 32)
-tree_attention_kernel(const bf16 *__restrict__ q, const bf16 *__restrict__ cache, size_t ep_stride,
-                      int max_seq, int H, RowTable rt, float scale, bf16 *__restrict__ out) {
+tree_attention_kernel(const float *__restrict__ q, const float *__restrict__ cache, size_t ep_stride,
+                      int max_seq, int H, RowTable rt, float scale, bf16 *__restrict__ out,
+                      size_t out_plane) {
   constexpr int PER = DH / 32;           // head-dim elements per lane
   const int h = blockIdx.x, t = blockIdx.y;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int hd = H * DH;
-  const bf16 *kbase = cache + (size_t)rt.ep[t] * ep_stride + (size_t)h * DH + lane * PER;
-  const bf16 *vbase = kbase + (size_t)max_seq * hd;
+  const float *kbase = cache + (size_t)rt.ep[t] * ep_stride + (size_t)h * DH + lane * PER;
+  const float *vbase = kbase + (size_t)max_seq * hd;
   const int nvis = rt.nvis[t], tbase = rt.tbase[t];
 
   float qv[PER];
 #pragma unroll
   for (int i = 0; i < PER; i++)
-    qv[i] = __bfloat162float(q[(size_t)t * hd + h * DH + lane * PER + i]) * scale;
+    qv[i] = q[(size_t)t * hd + h * DH + lane * PER + i] * scale;
 
   float m = -INFINITY, l = 0.f, acc[PER];
 #pragma unroll
   for (int i = 0; i < PER; i++) acc[i] = 0.f;
 
   auto visit = [&](int slot) {
-    const bf16 *kp = kbase + (size_t)slot * hd;
-    const bf16 *vp = vbase + (size_t)slot * hd;
+    const float *kp = kbase + (size_t)slot * hd;
+    const float *vp = vbase + (size_t)slot * hd;
     float s = 0.f;
 #pragma unroll
-    for (int i = 0; i < PER; i++) s += qv[i] * __bfloat162float(kp[i]);
+    for (int i = 0; i < PER; i++) s += qv[i] * kp[i];
     s = warp_sum(s);
     const float mn = fmaxf(m, s);
     const float corr = __expf(m - mn), p = __expf(s - mn);
     l = l * corr + p;
 #pragma unroll
-    for (int i = 0; i < PER; i++) acc[i] = acc[i] * corr + p * __bfloat162float(vp[i]);
+    for (int i = 0; i < PER; i++) acc[i] = acc[i] * corr + p * vp[i];
     m = mn;
   };
 
@@ -77,8 +79,13 @@ tree_attention_kernel(const bf16 *__restrict__ q, const bf16 *__restrict__ cache
     }
     const float inv = 1.f / L;
 #pragma unroll
-    for (int i = 0; i < PER; i++)
-      out[(size_t)t * hd + h * DH + lane * PER + i] = __float2bfloat16(o[i] * inv);
+    for (int i = 0; i < PER; i++) {
+      const size_t idx = (size_t)t * hd + h * DH + lane * PER + i;
+      const float v = o[i] * inv;
+      const bf16 hi = __float2bfloat16(v);
+      out[idx] = hi;
+      out[out_plane + idx] = __float2bfloat16(v - __bfloat162float(hi));
+    }
   }
 }
 

@@ -1,13 +1,21 @@
 // Row-wise kernels around the GEMMs: input embedding, split-K reduction fused with
-// RMSNorm / RoPE + KV append / SwiGLU / argmax / log-softmax top-k. All arithmetic is fp32;
-// bf16 appears only where a value becomes a GEMM operand or a cache entry. Split-K partials
-// are summed in ascending split order, so results do not depend on scheduling.
+// RMSNorm / RoPE + KV append / SwiGLU / argmax / log-softmax top-k. All arithmetic is fp32.
+// A value that becomes a GEMM operand is written as two bf16 limbs (hi, lo with hi + lo equal
+// to the fp32 value to 16 mantissa bits), lo limb `plane` elements after the hi limb; queries
+// and cache entries stay fp32. Split-K partials are summed in ascending split order, so
+// results do not depend on scheduling.
 #pragma once
 #include "common.cuh"
 
 namespace epi {
 
 constexpr int THREADS = 256;
+
+__device__ __forceinline__ void store2(bf16 *hi_plane, size_t plane, size_t idx, float v) {
+  const bf16 hi = __float2bfloat16(v);
+  hi_plane[idx] = hi;
+  hi_plane[plane + idx] = __float2bfloat16(v - __bfloat162float(hi));
+}
 
 __device__ __forceinline__ float block_sum(float v, float *red) {
   v = warp_sum(v);
@@ -24,11 +32,11 @@ __device__ __forceinline__ float block_sum(float v, float *red) {
   return red[0];
 }
 
-// x[t] = input row (embeds[src] or E[tok]); xn[t] = bf16(rmsnorm(x[t]) * gain).
+// x[t] = input row (embeds[src] or E[tok]); xn[t] = limbs(rmsnorm(x[t]) * gain).
 __global__ void __launch_bounds__(THREADS)
 embed_norm_kernel(RowTable rt, const bf16 *__restrict__ embeds, const bf16 *__restrict__ E,
                   const float *__restrict__ gain, float eps, int d, float *__restrict__ x,
-                  bf16 *__restrict__ xn) {
+                  bf16 *__restrict__ xn, size_t plane) {
   __shared__ float red[32];
   const int t = blockIdx.x;
   const int tok = rt.tok[t];
@@ -42,16 +50,16 @@ embed_norm_kernel(RowTable rt, const bf16 *__restrict__ embeds, const bf16 *__re
   ss = block_sum(ss, red);
   const float rs = rsqrtf(ss / d + eps);
   for (int i = threadIdx.x; i < d; i += blockDim.x)
-    xn[(size_t)t * d + i] = __float2bfloat16(x[(size_t)t * d + i] * rs * gain[i]);
+    store2(xn, plane, (size_t)t * d + i, x[(size_t)t * d + i] * rs * gain[i]);
 }
 
 // Residual update + next norm:  x[t] (+)= sum_s part[s][t];  then
-//   gain != NULL: xn[t] = bf16(rmsnorm(x[t]) * gain), feat[t] = rmsnorm(x[t]) * gain (if feat)
-//   gain == NULL: xn[t] = bf16(x[t])
+//   gain != NULL: xn[t] = limbs(rmsnorm(x[t]) * gain), feat[t] = rmsnorm(x[t]) * gain (if feat)
+//   gain == NULL: xn[t] = limbs(x[t])
 __global__ void __launch_bounds__(THREADS)
 residual_norm_kernel(const float *__restrict__ part, int splits, int T, int d, int accumulate,
                      const float *__restrict__ gain, float eps, float *__restrict__ x,
-                     bf16 *__restrict__ xn, float *__restrict__ feat) {
+                     bf16 *__restrict__ xn, size_t plane, float *__restrict__ feat) {
   __shared__ float red[32];
   const int t = blockIdx.x;
   float ss = 0.f;
@@ -63,30 +71,30 @@ residual_norm_kernel(const float *__restrict__ part, int splits, int T, int d, i
   }
   if (gain == nullptr) {
     for (int i = threadIdx.x; i < d; i += blockDim.x)
-      xn[(size_t)t * d + i] = __float2bfloat16(x[(size_t)t * d + i]);
+      store2(xn, plane, (size_t)t * d + i, x[(size_t)t * d + i]);
     return;
   }
   ss = block_sum(ss, red);
   const float rs = rsqrtf(ss / d + eps);
   for (int i = threadIdx.x; i < d; i += blockDim.x) {
     float v = x[(size_t)t * d + i] * rs * gain[i];
-    xn[(size_t)t * d + i] = __float2bfloat16(v);
+    store2(xn, plane, (size_t)t * d + i, v);
     if (feat) feat[(size_t)t * d + i] = v;
   }
 }
 
 // q, k, v = sum_s part[s][t][...]; rotate q and k by the row's position (rotate-half pairs
-// (i, i + dh/2), angle from the precomputed table); write q as bf16 and k, v into the row's
-// cache slot. Cache layout per episode: [2 (K, V)][max_seq][H * dh] bf16.
+// (i, i + dh/2), angle from the precomputed table); write q and, into the row's cache slot,
+// k and v, all fp32. Cache layout per episode: [2 (K, V)][max_seq][H * dh] fp32.
 __global__ void __launch_bounds__(THREADS)
 qkv_rope_append_kernel(const float *__restrict__ part, int splits, int T, int H, int dh,
-                       RowTable rt, const float2 *__restrict__ rope_tab, bf16 *__restrict__ q,
-                       bf16 *__restrict__ cache, size_t ep_stride, int max_seq) {
+                       RowTable rt, const float2 *__restrict__ rope_tab, float *__restrict__ q,
+                       float *__restrict__ cache, size_t ep_stride, int max_seq) {
   const int t = blockIdx.x;
   const int hd = H * dh, half = dh >> 1, N = 3 * hd;
   const int pos = rt.pos[t], slot = rt.slot[t];
-  bf16 *kdst = cache + (size_t)rt.ep[t] * ep_stride + (size_t)slot * hd;
-  bf16 *vdst = kdst + (size_t)max_seq * hd;
+  float *kdst = cache + (size_t)rt.ep[t] * ep_stride + (size_t)slot * hd;
+  float *vdst = kdst + (size_t)max_seq * hd;
   for (int i = threadIdx.x; i < H * half; i += blockDim.x) {
     const int h = i / half, j = i - h * half;
     const int c0 = h * dh + j, c1 = c0 + half;
@@ -98,18 +106,19 @@ qkv_rope_append_kernel(const float *__restrict__ part, int splits, int T, int H,
       vlo += p[2 * hd + c0]; vhi += p[2 * hd + c1];
     }
     const float2 cs = rope_tab[(size_t)pos * half + j];
-    q[(size_t)t * hd + c0] = __float2bfloat16(qlo * cs.x - qhi * cs.y);
-    q[(size_t)t * hd + c1] = __float2bfloat16(qhi * cs.x + qlo * cs.y);
-    kdst[c0] = __float2bfloat16(klo * cs.x - khi * cs.y);
-    kdst[c1] = __float2bfloat16(khi * cs.x + klo * cs.y);
-    vdst[c0] = __float2bfloat16(vlo);
-    vdst[c1] = __float2bfloat16(vhi);
+    q[(size_t)t * hd + c0] = qlo * cs.x - qhi * cs.y;
+    q[(size_t)t * hd + c1] = qhi * cs.x + qlo * cs.y;
+    kdst[c0] = klo * cs.x - khi * cs.y;
+    kdst[c1] = khi * cs.x + klo * cs.y;
+    vdst[c0] = vlo;
+    vdst[c1] = vhi;
   }
 }
 
-// hid[t][n] = bf16( silu(g) * u ), g = sum_s part[s][t][n], u = sum_s part[s][t][F + n].
+// hid[t][n] = limbs( silu(g) * u ), g = sum_s part[s][t][n], u = sum_s part[s][t][F + n].
 __global__ void __launch_bounds__(THREADS)
-swiglu_kernel(const float *__restrict__ part, int splits, int T, int F, bf16 *__restrict__ hid) {
+swiglu_kernel(const float *__restrict__ part, int splits, int T, int F, bf16 *__restrict__ hid,
+              size_t plane) {
   const int t = blockIdx.y;
   const int n = blockIdx.x * blockDim.x + threadIdx.x;
   if (n >= F) return;
@@ -119,7 +128,7 @@ swiglu_kernel(const float *__restrict__ part, int splits, int T, int F, bf16 *__
     g += p[n];
     u += p[F + n];
   }
-  hid[(size_t)t * F + n] = __float2bfloat16(g / (1.f + expf(-g)) * u);
+  store2(hid, plane, (size_t)t * F + n, g / (1.f + expf(-g)) * u);
 }
 
 // cos/sin table in double precision: tab[pos][j] = (cos, sin)(pos * theta^(-2j/dh)).
@@ -131,12 +140,21 @@ __global__ void rope_table_kernel(float2 *tab, int max_pos, int half, double the
   tab[i] = make_float2((float)cos(ang), (float)sin(ang));
 }
 
-// dst[i] = bf16 row src_rows[i] of src (row gather, e.g. the last prefix row of each episode).
-__global__ void gather_rows_kernel(const bf16 *__restrict__ src, const int *__restrict__ rows,
-                                   int d, bf16 *__restrict__ dst) {
+// dst[i] = row rows[i] of src, both limbs (e.g. the last prefix row of each episode).
+__global__ void gather_rows_kernel(const bf16 *__restrict__ src, size_t src_plane,
+                                   const int *__restrict__ rows, int d, bf16 *__restrict__ dst,
+                                   size_t dst_plane) {
   const int r = rows[blockIdx.x];
-  for (int i = threadIdx.x; i < d; i += blockDim.x)
+  for (int i = threadIdx.x; i < d; i += blockDim.x) {
     dst[(size_t)blockIdx.x * d + i] = src[(size_t)r * d + i];
+    dst[dst_plane + (size_t)blockIdx.x * d + i] = src[src_plane + (size_t)r * d + i];
+  }
+}
+
+// Two-limb split of an fp32 matrix (stand-alone GEMM entry point).
+__global__ void split_limbs_kernel(const float *__restrict__ x, size_t n, bf16 *__restrict__ out) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) store2(out, n, i, x[i]);
 }
 
 struct Top2 {

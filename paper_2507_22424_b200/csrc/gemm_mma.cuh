@@ -1,9 +1,13 @@
 // Skinny weight-streaming GEMM, warp-level MMA version.
-//   part[z][t][n] = sum over the z-th K range of X[t][k] * W[n][k]      (fp32 accumulate)
-// X [T, K] and W [N, K] are bf16 with K contiguous. The 128 weight rows of a CTA tile sit on
-// the MMA's M axis, the (few) activation rows on its N axis, so one pass over W serves every
-// row of the tree. K ranges (split-K) are summed by the consuming epilogue in fixed order.
-// Requires K % 8 == 0 (16-byte chunks); ragged N, T and K tails are zero-filled.
+//   part[z][t][n] = sum over the z-th K range of (Xhi[t][k] + Xlo[t][k]) * W[n][k]   (fp32 acc)
+// W [N, K] is bf16 with K contiguous. The activations come as TWO bf16 limbs (hi = bf16(x),
+// lo = bf16(x - hi)), each [T, K]: the weight stream is the cost of this kernel, so spending a
+// second MMA per weight tile buys fp32-grade activations for free, which the 32-layer model
+// needs to stay within 2e-2 of a float64 forward (single-limb bf16 activations drift by 0.2).
+// The 128 weight rows of a CTA tile sit on the MMA's M axis, the (few) activation rows on its
+// N axis, so one pass over W serves every row of the tree. K ranges (split-K) are summed by
+// the consuming epilogue in fixed order. Requires K % 8 == 0 (16-byte chunks); ragged N, T
+// and K tails are zero-filled.
 #pragma once
 #include "common.cuh"
 
@@ -39,8 +43,8 @@ __device__ __forceinline__ bf16 *tile_ptr(bf16 *tile, int row, int chunk) {
 
 template <int BT, int WARPS_T>
 __global__ void __launch_bounds__(128 * WARPS_T)
-gemm_kernel(const bf16 *__restrict__ X, const bf16 *__restrict__ W, float *__restrict__ part,
-            int T, int N, int K, int kb_per_split) {
+gemm_kernel(const bf16 *__restrict__ X, size_t x_plane, const bf16 *__restrict__ W,
+            float *__restrict__ part, int T, int N, int K, int kb_per_split) {
   constexpr int NT = 128 * WARPS_T;
   constexpr int WT = BT / WARPS_T;       // activation rows per warp
   constexpr int NTILES = WT / 8;
@@ -57,7 +61,7 @@ gemm_kernel(const bf16 *__restrict__ X, const bf16 *__restrict__ W, float *__res
 
   auto load_stage = [&](int stage, int kb) {
     bf16 *w = sW + stage * BN * BK;
-    bf16 *x = sX + stage * BT * BK;
+    bf16 *x = sX + stage * 2 * BT * BK;
     const int k0 = kb * BK;
     for (int c = tid; c < BN * 8; c += NT) {
       int row = c >> 3, ch = c & 7;
@@ -66,11 +70,11 @@ gemm_kernel(const bf16 *__restrict__ X, const bf16 *__restrict__ W, float *__res
       const bf16 *src = W + (size_t)(ok ? n : 0) * K + (ok ? k : 0);
       cp_async16(tile_ptr(w, row, ch), src, ok ? 16 : 0);
     }
-    for (int c = tid; c < BT * 8; c += NT) {
-      int row = c >> 3, ch = c & 7;
-      int t = t0 + row, k = k0 + ch * 8;
+    for (int c = tid; c < 2 * BT * 8; c += NT) {
+      int row = c >> 3, ch = c & 7;              // rows [0, BT): hi limb, [BT, 2BT): lo limb
+      int limb = row >= BT, t = t0 + row - limb * BT, k = k0 + ch * 8;
       bool ok = (t < T) && (k < K);
-      const bf16 *src = X + (size_t)(ok ? t : 0) * K + (ok ? k : 0);
+      const bf16 *src = X + (size_t)limb * x_plane + (size_t)(ok ? t : 0) * K + (ok ? k : 0);
       cp_async16(tile_ptr(x, row, ch), src, ok ? 16 : 0);
     }
   };
@@ -95,7 +99,7 @@ gemm_kernel(const bf16 *__restrict__ X, const bf16 *__restrict__ W, float *__res
     if (nxt < nk) load_stage(nxt % STAGES, kb0 + nxt);
     cp_async_commit();
     bf16 *w = sW + (it % STAGES) * BN * BK;
-    bf16 *x = sX + (it % STAGES) * BT * BK;
+    bf16 *x = sX + (it % STAGES) * 2 * BT * BK;
 #pragma unroll
     for (int kk = 0; kk < BK / 16; kk++) {
       uint32_t a[2][4];
@@ -105,16 +109,18 @@ gemm_kernel(const bf16 *__restrict__ X, const bf16 *__restrict__ W, float *__res
         ldmatrix_x4(a[mt][0], a[mt][1], a[mt][2], a[mt][3], tile_ptr(w, row, kk * 2 + (lane >> 4)));
       }
 #pragma unroll
-      for (int p = 0; p < NTILES / 2; p++) {
-        uint32_t b0, b1, b2, b3;
-        int row = warp_t * WT + p * 16 + ((lane >> 4) << 3) + (lane & 7);
-        ldmatrix_x4(b0, b1, b2, b3, tile_ptr(x, row, kk * 2 + ((lane >> 3) & 1)));
+      for (int limb = 0; limb < 2; limb++)
 #pragma unroll
-        for (int mt = 0; mt < 2; mt++) {
-          mma_bf16(acc[mt][2 * p], a[mt], b0, b1);
-          mma_bf16(acc[mt][2 * p + 1], a[mt], b2, b3);
+        for (int p = 0; p < NTILES / 2; p++) {
+          uint32_t b0, b1, b2, b3;
+          int row = limb * BT + warp_t * WT + p * 16 + ((lane >> 4) << 3) + (lane & 7);
+          ldmatrix_x4(b0, b1, b2, b3, tile_ptr(x, row, kk * 2 + ((lane >> 3) & 1)));
+#pragma unroll
+          for (int mt = 0; mt < 2; mt++) {
+            mma_bf16(acc[mt][2 * p], a[mt], b0, b1);
+            mma_bf16(acc[mt][2 * p + 1], a[mt], b2, b3);
+          }
         }
-      }
     }
   }
   cp_async_wait<0>();
@@ -134,10 +140,10 @@ gemm_kernel(const bf16 *__restrict__ X, const bf16 *__restrict__ W, float *__res
 }
 
 template <int BT, int WARPS_T>
-inline cudaError_t launch_cfg(const bf16 *X, const bf16 *W, float *part, int T, int N, int K,
-                              int splits, cudaStream_t st) {
+inline cudaError_t launch_cfg(const bf16 *X, size_t x_plane, const bf16 *W, float *part, int T, int N,
+                              int K, int splits, cudaStream_t st) {
   static bool attr_set = false;
-  const int smem = STAGES * (BN + BT) * BK * (int)sizeof(bf16);
+  const int smem = STAGES * (BN + 2 * BT) * BK * (int)sizeof(bf16);
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(gemm_kernel<BT, WARPS_T>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -147,7 +153,7 @@ inline cudaError_t launch_cfg(const bf16 *X, const bf16 *W, float *part, int T, 
   const int nkb = (K + BK - 1) / BK;
   const int kbs = (nkb + splits - 1) / splits;
   dim3 grid((N + BN - 1) / BN, (T + BT - 1) / BT, (nkb + kbs - 1) / kbs);
-  gemm_kernel<BT, WARPS_T><<<grid, 128 * WARPS_T, smem, st>>>(X, W, part, T, N, K, kbs);
+  gemm_kernel<BT, WARPS_T><<<grid, 128 * WARPS_T, smem, st>>>(X, x_plane, W, part, T, N, K, kbs);
   return cudaGetLastError();
 }
 
@@ -164,11 +170,12 @@ inline int plan_splits(int T, int N, int K, int max_splits) {
   return (nkb + kbs - 1) / kbs;
 }
 
-inline cudaError_t launch(const bf16 *X, const bf16 *W, float *part, int T, int N, int K,
+// X: hi limb [T, K]; the lo limb starts x_plane elements after it.
+inline cudaError_t launch(const bf16 *X, size_t x_plane, const bf16 *W, float *part, int T, int N, int K,
                           int splits, cudaStream_t st) {
-  if (T <= 32) return launch_cfg<32, 1>(X, W, part, T, N, K, splits, st);
-  if (T <= 64) return launch_cfg<64, 1>(X, W, part, T, N, K, splits, st);
-  return launch_cfg<128, 2>(X, W, part, T, N, K, splits, st);
+  if (T <= 32) return launch_cfg<32, 1>(X, x_plane, W, part, T, N, K, splits, st);
+  if (T <= 64) return launch_cfg<64, 1>(X, x_plane, W, part, T, N, K, splits, st);
+  return launch_cfg<128, 2>(X, x_plane, W, part, T, N, K, splits, st);
 }
 
 }  // namespace gemm_mma

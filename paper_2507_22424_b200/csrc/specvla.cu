@@ -51,12 +51,14 @@ struct specvla_ctx {
   bool has_draft;
 
   // workspace carve-up (device)
-  bf16 *kv_t, *kv_d;            // target [ep][layer][2][max_seq][hd], draft [ep][2][max_seq][hd]
+  float *kv_t, *kv_d;           // target [ep][layer][2][max_seq][hd], draft [ep][2][max_seq][hd], fp32
   size_t kv_t_ep_stride, kv_t_layer_stride, kv_d_ep_stride;
   float2 *rope_tab;
-  float *x, *feat, *part, *lgs, *pend_feat, *dout, *margin, *top_lp;
+  float *x, *feat, *part, *lgs, *pend_feat, *dout, *margin, *top_lp, *q;
   size_t part_floats;
-  bf16 *xn, *xin, *q, *ao, *hid, *lm_in;
+  // GEMM operands, two bf16 limbs each: hi plane, then the lo plane *_pl elements later
+  bf16 *xn, *xin, *ao, *hid, *lm_in;
+  size_t xn_pl, xin_pl, ao_pl, hid_pl, lm_pl;
   RowTable rt;
   int *feat_src, *dst_row, *lm_rows, *greedy, *top_tok, *out_m, *out_tok, *out_path;
   EpState *st;
@@ -74,6 +76,17 @@ struct specvla_ctx {
   long long launches;
   char cuda_err[256];
   cudaEvent_t ev[4];
+
+  // optional per-GEMM timing (specvla_profile): events around every GEMM launch, summed per
+  // weight-matrix class when the stream is next synchronised
+  int prof_mask;                        // phases timed: 1 prefill, 2 draft, 4 verify
+  int phase;                            // phase of the call in flight
+  std::vector<cudaEvent_t> prof_ev;     // pairs (start, stop)
+  std::vector<int> prof_cls;            // class of each recorded pair
+  int prof_used;
+  double prof_ms[SPECVLA_PROF_CLASSES];
+  long long prof_n[SPECVLA_PROF_CLASSES];
+  double prof_bytes[SPECVLA_PROF_CLASSES];
 };
 
 namespace {
@@ -119,17 +132,22 @@ size_t carve(specvla_ctx *c, char *base) {
   c->kv_t_layer_stride = (size_t)2 * d.max_seq * hd;
   c->kv_t_ep_stride = c->kv_t_layer_stride * d.n_layers;
   c->kv_d_ep_stride = (size_t)2 * d.max_seq * hd;
-  c->kv_t = cv.take<bf16>(E * c->kv_t_ep_stride);
-  c->kv_d = cv.take<bf16>(E * c->kv_d_ep_stride);
+  c->kv_t = cv.take<float>(E * c->kv_t_ep_stride);
+  c->kv_d = cv.take<float>(E * c->kv_d_ep_stride);
   c->rope_tab = cv.take<float2>((size_t)d.max_seq * (d.head_dim / 2));
   c->x = cv.take<float>(R * d.d_model);
   c->feat = cv.take<float>(R * d.d_model);
-  c->xn = cv.take<bf16>(R * d.d_model);
-  c->xin = cv.take<bf16>(R * 2 * d.d_model);
-  c->q = cv.take<bf16>(R * hd);
-  c->ao = cv.take<bf16>(R * hd);
-  c->hid = cv.take<bf16>(R * d.d_ffn);
-  c->lm_in = cv.take<bf16>(lm_rows * d.d_model);
+  c->xn_pl = R * d.d_model;
+  c->xin_pl = R * 2 * d.d_model;
+  c->ao_pl = R * hd;
+  c->hid_pl = R * d.d_ffn;
+  c->lm_pl = lm_rows * d.d_model;
+  c->xn = cv.take<bf16>(2 * c->xn_pl);
+  c->xin = cv.take<bf16>(2 * c->xin_pl);
+  c->q = cv.take<float>(R * hd);
+  c->ao = cv.take<bf16>(2 * c->ao_pl);
+  c->hid = cv.take<bf16>(2 * c->hid_pl);
+  c->lm_in = cv.take<bf16>(2 * c->lm_pl);
   size_t widest = (size_t)3 * hd;
   if ((size_t)2 * d.d_ffn > widest) widest = (size_t)2 * d.d_ffn;
   size_t pf = R * widest;                                  // one split over all rows
@@ -175,29 +193,48 @@ void derive_caps(specvla_ctx *c) {
   c->max_draft_rows = (int)dr;
 }
 
+// Folds the recorded GEMM event pairs into the per-class sums. The stream must be idle.
+void prof_collect(specvla_ctx *ctx) {
+  for (int i = 0; i < ctx->prof_used; i++) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, ctx->prof_ev[2 * i], ctx->prof_ev[2 * i + 1]) == cudaSuccess) {
+      ctx->prof_ms[ctx->prof_cls[i]] += ms;
+      ctx->prof_n[ctx->prof_cls[i]]++;
+    }
+  }
+  ctx->prof_used = 0;
+}
+
 // part <- A[R, K] * W[N, K]^T split over K; returns the number of splits to sum.
-int gemm(specvla_ctx *ctx, const bf16 *A, const bf16 *W, int R, int N, int K, cudaStream_t st,
-         int *splits_out) {
+int gemm(specvla_ctx *ctx, const bf16 *A, size_t a_plane, const bf16 *W, int R, int N, int K,
+         cudaStream_t st, int *splits_out, int cls) {
   int cap = (int)(ctx->part_floats / ((size_t)R * N));
   if (cap < 1) return SPECVLA_ERR_CAPACITY;
   if (cap > MAX_SPLITS) cap = MAX_SPLITS;
   const int splits = gemm_mma::plan_splits(R, N, K, cap);
-  CU(gemm_mma::launch(A, W, ctx->part, R, N, K, splits, st));
+  const bool prof = (ctx->prof_mask & ctx->phase) && 2 * (ctx->prof_used + 1) <= (int)ctx->prof_ev.size();
+  if (prof) CU(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used], st));
+  CU(gemm_mma::launch(A, a_plane, W, ctx->part, R, N, K, splits, st));
+  if (prof) {
+    CU(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used + 1], st));
+    ctx->prof_cls[ctx->prof_used++] = cls;
+    ctx->prof_bytes[cls] += (double)N * K * sizeof(bf16);
+  }
   ctx->launches++;
   *splits_out = splits;
   return SPECVLA_OK;
 }
 
-int attention(specvla_ctx *ctx, int R, const bf16 *cache, size_t ep_stride, cudaStream_t st) {
+int attention(specvla_ctx *ctx, int R, const float *cache, size_t ep_stride, cudaStream_t st) {
   const specvla_model_desc &d = ctx->desc;
   const float scale = 1.f / sqrtf((float)d.head_dim);
   dim3 grid(d.n_heads, R);
   if (d.head_dim == 128)
     attn::tree_attention_kernel<128><<<grid, attn::WARPS * 32, 0, st>>>(
-        ctx->q, cache, ep_stride, d.max_seq, d.n_heads, ctx->rt, scale, ctx->ao);
+        ctx->q, cache, ep_stride, d.max_seq, d.n_heads, ctx->rt, scale, ctx->ao, ctx->ao_pl);
   else
     attn::tree_attention_kernel<64><<<grid, attn::WARPS * 32, 0, st>>>(
-        ctx->q, cache, ep_stride, d.max_seq, d.n_heads, ctx->rt, scale, ctx->ao);
+        ctx->q, cache, ep_stride, d.max_seq, d.n_heads, ctx->rt, scale, ctx->ao, ctx->ao_pl);
   LAUNCHED();
   return SPECVLA_OK;
 }
@@ -205,28 +242,28 @@ int attention(specvla_ctx *ctx, int R, const bf16 *cache, size_t ep_stride, cuda
 // One pre-norm decoder layer over R rows. In: x (residual, fp32) and xn = bf16(norm1(x)).
 // Out: x updated; xn = bf16(rmsnorm(x) * next_gain) (or bf16(x) when next_gain is NULL);
 // feat_out (optional) receives the normalised rows in fp32.
-int run_layer(specvla_ctx *ctx, const LayerW &w, int R, bf16 *cache, size_t ep_stride,
+int run_layer(specvla_ctx *ctx, const LayerW &w, int R, float *cache, size_t ep_stride,
               const float *next_gain, float *feat_out, cudaStream_t st) {
   const specvla_model_desc &d = ctx->desc;
   const int hd = ctx->hd, D = d.d_model, F = d.d_ffn;
   int s;
-  TRY(gemm(ctx, ctx->xn, w.wqkv, R, 3 * hd, D, st, &s));
+  TRY(gemm(ctx, ctx->xn, ctx->xn_pl, w.wqkv, R, 3 * hd, D, st, &s, SPECVLA_PROF_QKV));
   epi::qkv_rope_append_kernel<<<R, epi::THREADS, 0, st>>>(ctx->part, s, R, d.n_heads, d.head_dim, ctx->rt,
                                                           ctx->rope_tab, ctx->q, cache, ep_stride,
                                                           d.max_seq);
   LAUNCHED();
   TRY(attention(ctx, R, cache, ep_stride, st));
-  TRY(gemm(ctx, ctx->ao, w.wo, R, D, hd, st, &s));
+  TRY(gemm(ctx, ctx->ao, ctx->ao_pl, w.wo, R, D, hd, st, &s, SPECVLA_PROF_O));
   epi::residual_norm_kernel<<<R, epi::THREADS, 0, st>>>(ctx->part, s, R, D, 1, w.norm2, d.rms_eps, ctx->x,
-                                                        ctx->xn, nullptr);
+                                                        ctx->xn, ctx->xn_pl, nullptr);
   LAUNCHED();
-  TRY(gemm(ctx, ctx->xn, w.wgu, R, 2 * F, D, st, &s));
+  TRY(gemm(ctx, ctx->xn, ctx->xn_pl, w.wgu, R, 2 * F, D, st, &s, SPECVLA_PROF_GATE_UP));
   epi::swiglu_kernel<<<dim3((F + epi::THREADS - 1) / epi::THREADS, R), epi::THREADS, 0, st>>>(
-      ctx->part, s, R, F, ctx->hid);
+      ctx->part, s, R, F, ctx->hid, ctx->hid_pl);
   LAUNCHED();
-  TRY(gemm(ctx, ctx->hid, w.wd, R, D, F, st, &s));
+  TRY(gemm(ctx, ctx->hid, ctx->hid_pl, w.wd, R, D, F, st, &s, SPECVLA_PROF_DOWN));
   epi::residual_norm_kernel<<<R, epi::THREADS, 0, st>>>(ctx->part, s, R, D, 1, next_gain, d.rms_eps,
-                                                        ctx->x, ctx->xn, feat_out);
+                                                        ctx->x, ctx->xn, ctx->xn_pl, feat_out);
   LAUNCHED();
   return SPECVLA_OK;
 }
@@ -236,7 +273,7 @@ int run_layer(specvla_ctx *ctx, const LayerW &w, int R, bf16 *cache, size_t ep_s
 int target_forward(specvla_ctx *ctx, int R, const bf16 *embeds, cudaStream_t st) {
   const specvla_model_desc &d = ctx->desc;
   epi::embed_norm_kernel<<<R, epi::THREADS, 0, st>>>(ctx->rt, embeds, ctx->embed, ctx->layers[0].norm1,
-                                                     d.rms_eps, d.d_model, ctx->x, ctx->xn);
+                                                     d.rms_eps, d.d_model, ctx->x, ctx->xn, ctx->xn_pl);
   LAUNCHED();
   for (int l = 0; l < d.n_layers; l++) {
     const bool last = (l + 1 == d.n_layers);
@@ -253,17 +290,17 @@ int target_forward(specvla_ctx *ctx, int R, const bf16 *embeds, cudaStream_t st)
 int draft_forward(specvla_ctx *ctx, int R, cudaStream_t st) {
   const specvla_model_desc &d = ctx->desc;
   int s;
-  TRY(gemm(ctx, ctx->xin, ctx->draft_fc, R, d.d_model, 2 * d.d_model, st, &s));
+  TRY(gemm(ctx, ctx->xin, ctx->xin_pl, ctx->draft_fc, R, d.d_model, 2 * d.d_model, st, &s, SPECVLA_PROF_FC));
   epi::residual_norm_kernel<<<R, epi::THREADS, 0, st>>>(ctx->part, s, R, d.d_model, 0, ctx->dlayer.norm1,
-                                                        d.rms_eps, ctx->x, ctx->xn, nullptr);
+                                                        d.rms_eps, ctx->x, ctx->xn, ctx->xn_pl, nullptr);
   LAUNCHED();
   return run_layer(ctx, ctx->dlayer, R, ctx->kv_d, ctx->kv_d_ep_stride, nullptr, nullptr, st);
 }
 
 // LM head over `rows` bf16 rows of A: partial logits land in ctx->part; returns splits.
-int lm_head(specvla_ctx *ctx, const bf16 *A, int rows, cudaStream_t st, int *splits) {
+int lm_head(specvla_ctx *ctx, const bf16 *A, size_t a_plane, int rows, cudaStream_t st, int *splits) {
   if (rows > ctx->max_lm_rows) return SPECVLA_ERR_CAPACITY;
-  return gemm(ctx, A, ctx->lm_head, rows, ctx->desc.vocab, ctx->desc.d_model, st, splits);
+  return gemm(ctx, A, a_plane, ctx->lm_head, rows, ctx->desc.vocab, ctx->desc.d_model, st, splits, SPECVLA_PROF_LM_HEAD);
 }
 
 void argmax_range(const specvla_ctx *ctx, int *lo, int *hi) {
@@ -389,6 +426,10 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
   ctx->pin_trees = reinterpret_cast<DevTree *>(static_cast<char *>(ctx->pinned) + small_b);
   ctx->pin_rows = reinterpret_cast<int *>(static_cast<char *>(ctx->pinned) + small_b + trees_b);
   for (int i = 0; i < 4; i++) cudaEventCreate(&ctx->ev[i]);
+  ctx->prof_mask = 0;
+  ctx->phase = 0;
+  ctx->prof_used = 0;
+  for (int i = 0; i < SPECVLA_PROF_CLASSES; i++) { ctx->prof_ms[i] = 0; ctx->prof_n[i] = 0; ctx->prof_bytes[i] = 0; }
   // device-side initialisation: RoPE table, zeroed state
   const int half = desc->head_dim / 2, n = desc->max_seq * half;
   epi::rope_table_kernel<<<(n + 255) / 256, 256>>>(ctx->rope_tab, desc->max_seq, half, (double)desc->rope_theta);
@@ -407,6 +448,7 @@ int specvla_destroy(specvla_ctx *ctx) {
   if (!ctx) return SPECVLA_ERR_INVALID_ARG;
   cudaDeviceSynchronize();
   for (int i = 0; i < 4; i++) cudaEventDestroy(ctx->ev[i]);
+  for (cudaEvent_t e : ctx->prof_ev) cudaEventDestroy(e);
   cudaFreeHost(ctx->pinned);
   delete ctx;
   return SPECVLA_OK;
@@ -466,17 +508,19 @@ int specvla_prefill(specvla_ctx *ctx, int n_ep, const int *episodes, const void 
   CU(cudaMemsetAsync(ctx->rt.mask, 0, rb * 4, st));
 
   const bf16 *emb = static_cast<const bf16 *>(embeds);
+  ctx->phase = 1;
   TRY(target_forward(ctx, R, emb, st));
 
   // first token: LM head on each episode's last row
   int *h_last = h + 5 * R;
   for (int i = 0; i < n_ep; i++) h_last[i] = ea.aux[i];
   CU(cudaMemcpyAsync(ctx->lm_rows, h_last, n_ep * sizeof(int), cudaMemcpyHostToDevice, st));
-  epi::gather_rows_kernel<<<n_ep, 256, 0, st>>>(ctx->xn, ctx->lm_rows, d.d_model, ctx->lm_in);
+  epi::gather_rows_kernel<<<n_ep, 256, 0, st>>>(ctx->xn, ctx->xn_pl, ctx->lm_rows, d.d_model, ctx->lm_in,
+                                                ctx->lm_pl);
   LAUNCHED();
   int s, lo, hi;
   argmax_range(ctx, &lo, &hi);
-  TRY(lm_head(ctx, ctx->lm_in, n_ep, st, &s));
+  TRY(lm_head(ctx, ctx->lm_in, ctx->lm_pl, n_ep, st, &s));
   epi::argmax_kernel<<<n_ep, epi::THREADS, 0, st>>>(ctx->part, s, n_ep, d.vocab, lo, hi, ctx->greedy,
                                                     ctx->margin, logits_out);
   LAUNCHED();
@@ -504,6 +548,7 @@ int specvla_prefill(specvla_ctx *ctx, int n_ep, const int *episodes, const void 
       // the uploads above are ordered before these on the same stream, but the pinned rows
       // are being rewritten: wait until the first batch has been consumed
       CU(cudaStreamSynchronize(st));
+      prof_collect(ctx);
       CU(cudaMemcpyAsync(ctx->rt.tok, h_tok, db, cudaMemcpyHostToDevice, st));
       CU(cudaMemcpyAsync(ctx->rt.src, h_src, db, cudaMemcpyHostToDevice, st));
       CU(cudaMemcpyAsync(ctx->rt.ep, h_ep, db, cudaMemcpyHostToDevice, st));
@@ -512,7 +557,7 @@ int specvla_prefill(specvla_ctx *ctx, int n_ep, const int *episodes, const void 
       CU(cudaMemcpyAsync(ctx->rt.nvis, h_nvis, db, cudaMemcpyHostToDevice, st));
       CU(cudaMemcpyAsync(ctx->feat_src, h_fs, db, cudaMemcpyHostToDevice, st));
       tree::draft_input_kernel<<<Rd, 256, 0, st>>>(ctx->rt, ctx->feat_src, ctx->feat, emb, ctx->embed,
-                                                   d.d_model, ctx->xin);
+                                                   d.d_model, ctx->xin, ctx->xin_pl);
       LAUNCHED();
       TRY(draft_forward(ctx, Rd, st));
     }
@@ -520,6 +565,7 @@ int specvla_prefill(specvla_ctx *ctx, int n_ep, const int *episodes, const void 
   int *h_g = ctx->pin_small;
   CU(cudaMemcpyAsync(h_g, ctx->greedy, n_ep * sizeof(int), cudaMemcpyDeviceToHost, st));
   CU(cudaStreamSynchronize(st));
+  prof_collect(ctx);
   for (int i = 0; i < n_ep; i++) {
     ctx->hP[episodes[i]] = lens[i];
     ctx->hPending[episodes[i]] = 1;
@@ -553,6 +599,7 @@ int specvla_draft_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const sp
   int lo, hi, s;
   argmax_range(ctx, &lo, &hi);
 
+  ctx->phase = 2;
   // catch-up over the pending rows; the last row of each episode scores the root's children
   tree::build_catchup_rows_kernel<<<(n_ep + 63) / 64, 64, 0, st>>>(ea, ctx->st, ctx->trees, ctx->rt,
                                                                    ctx->feat_src);
@@ -560,7 +607,7 @@ int specvla_draft_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const sp
   tree::catchup_dst_kernel<<<(n_ep + 63) / 64, 64, 0, st>>>(ea, ctx->dst_row, ctx->lm_rows);
   LAUNCHED();
   tree::draft_input_kernel<<<R, 256, 0, st>>>(ctx->rt, ctx->feat_src, ctx->pend_feat, nullptr, ctx->embed,
-                                              d.d_model, ctx->xin);
+                                              d.d_model, ctx->xin, ctx->xin_pl);
   LAUNCHED();
   TRY(draft_forward(ctx, R, st));
   tree::save_draft_out_kernel<<<R, 256, 0, st>>>(ctx->x, ctx->dst_row, d.d_model, ctx->dout);
@@ -574,12 +621,15 @@ int specvla_draft_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const sp
   bool gathered = true;              // round 0 scores the gathered last rows
   for (int l = 0; l < shape->depth; l++) {
     const bf16 *A = ctx->xn;
+    size_t a_plane = ctx->xn_pl;
     if (gathered) {
-      epi::gather_rows_kernel<<<n_ep, 256, 0, st>>>(ctx->xn, ctx->lm_rows, d.d_model, ctx->lm_in);
+      epi::gather_rows_kernel<<<n_ep, 256, 0, st>>>(ctx->xn, ctx->xn_pl, ctx->lm_rows, d.d_model, ctx->lm_in,
+                                                    ctx->lm_pl);
       LAUNCHED();
       A = ctx->lm_in;
+      a_plane = ctx->lm_pl;
     }
-    TRY(lm_head(ctx, A, scored_rows, st, &s));
+    TRY(lm_head(ctx, A, a_plane, scored_rows, st, &s));
     epi::logsoftmax_topk_kernel<<<scored_rows, epi::THREADS, 0, st>>>(
         ctx->part, s, scored_rows, d.vocab, lo, hi, ctx->lgs, ctx->top_tok, ctx->top_lp);
     LAUNCHED();
@@ -597,7 +647,7 @@ int specvla_draft_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const sp
     if (next == 0) break;
     const int Rn = n_ep * next;
     tree::draft_input_kernel<<<Rn, 256, 0, st>>>(ctx->rt, ctx->feat_src, ctx->dout, nullptr, ctx->embed,
-                                                 d.d_model, ctx->xin);
+                                                 d.d_model, ctx->xin, ctx->xin_pl);
     LAUNCHED();
     TRY(draft_forward(ctx, Rn, st));
     tree::save_draft_out_kernel<<<Rn, 256, 0, st>>>(ctx->x, ctx->dst_row, d.d_model, ctx->dout);
@@ -633,12 +683,13 @@ static int verify_device_trees(specvla_ctx *ctx, const EpArgs &ea, int R, int r,
                                cudaStream_t st) {
   const specvla_model_desc &d = ctx->desc;
   const int n_ep = ea.n_ep;
+  ctx->phase = 4;
   tree::build_verify_rows_kernel<<<n_ep, 128, 0, st>>>(ea, ctx->trees, ctx->st, ctx->rt);
   LAUNCHED();
   TRY(target_forward(ctx, R, nullptr, st));
   int s, lo, hi;
   argmax_range(ctx, &lo, &hi);
-  TRY(lm_head(ctx, ctx->xn, R, st, &s));
+  TRY(lm_head(ctx, ctx->xn, ctx->xn_pl, R, st, &s));
   epi::argmax_kernel<<<R, epi::THREADS, 0, st>>>(ctx->part, s, R, d.vocab, lo, hi, ctx->greedy, ctx->margin,
                                                  logits_out);
   LAUNCHED();
@@ -663,6 +714,7 @@ static int finish_verify(specvla_ctx *ctx, const EpArgs &ea, int *accept_len_out
   CU(cudaMemcpyAsync(h, ctx->out_m, n_ep * sizeof(int), cudaMemcpyDeviceToHost, st));
   CU(cudaMemcpyAsync(h + SV_MAX_EP, ctx->out_tok, n_ep * W * sizeof(int), cudaMemcpyDeviceToHost, st));
   CU(cudaStreamSynchronize(st));
+  prof_collect(ctx);
   for (int i = 0; i < n_ep; i++) {
     const int e = ea.eps[i], m = h[i];
     if (m < 0 || m > SV_MAX_DEPTH) return SPECVLA_ERR_BAD_STATE;
@@ -850,11 +902,11 @@ int specvla_read_kv(specvla_ctx *ctx, int draft, int episode, int layer, int whi
       slot0 + n_slots > d.max_seq)
     return SPECVLA_ERR_INVALID_ARG;
   if (draft ? (layer != 0) : (layer < 0 || layer >= d.n_layers)) return SPECVLA_ERR_INVALID_ARG;
-  const bf16 *base = draft ? ctx->kv_d + (size_t)episode * ctx->kv_d_ep_stride
+  const float *base = draft ? ctx->kv_d + (size_t)episode * ctx->kv_d_ep_stride
                            : ctx->kv_t + (size_t)episode * ctx->kv_t_ep_stride + (size_t)layer * ctx->kv_t_layer_stride;
   base += ((size_t)which * d.max_seq + slot0) * ctx->hd;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  CU(cudaMemcpyAsync(host_dst, base, (size_t)n_slots * ctx->hd * sizeof(bf16), cudaMemcpyDeviceToHost, st));
+  CU(cudaMemcpyAsync(host_dst, base, (size_t)n_slots * ctx->hd * sizeof(float), cudaMemcpyDeviceToHost, st));
   CU(cudaStreamSynchronize(st));
   return SPECVLA_OK;
 }
@@ -868,23 +920,55 @@ __global__ void sum_splits_kernel(const float *__restrict__ part, int splits, si
   y[i] = v;
 }
 
+// scratch layout: [two bf16 limbs of X | split-K partials]
+static size_t gemm_limb_bytes(int T, int K) { return ((size_t)2 * T * K * sizeof(bf16) + 1023) / 1024 * 1024; }
+
 size_t specvla_gemm_scratch_bytes(int T, int N, int K) {
   if (T < 1 || N < 1 || K < 8) return 0;
-  return (size_t)gemm_mma::plan_splits(T, N, K, MAX_SPLITS) * T * N * sizeof(float);
+  return gemm_limb_bytes(T, K) + (size_t)gemm_mma::plan_splits(T, N, K, MAX_SPLITS) * T * N * sizeof(float);
 }
 
-int specvla_gemm_bf16(const void *X, const void *W, float *Y, int T, int N, int K, void *scratch,
-                      size_t scratch_bytes, void *stream) {
+int specvla_gemm(const float *X, const void *W, float *Y, int T, int N, int K, void *scratch,
+                 size_t scratch_bytes, void *stream) {
   if (!X || !W || !Y || !scratch || T < 1 || N < 1 || K < 8 || (K % 8)) return SPECVLA_ERR_INVALID_ARG;
   const int splits = gemm_mma::plan_splits(T, N, K, MAX_SPLITS);
-  if (scratch_bytes < (size_t)splits * T * N * sizeof(float)) return SPECVLA_ERR_CAPACITY;
+  if (scratch_bytes < specvla_gemm_scratch_bytes(T, N, K)) return SPECVLA_ERR_CAPACITY;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (gemm_mma::launch(static_cast<const bf16 *>(X), static_cast<const bf16 *>(W), static_cast<float *>(scratch),
-                       T, N, K, splits, st) != cudaSuccess)
+  bf16 *limbs = static_cast<bf16 *>(scratch);
+  float *part = reinterpret_cast<float *>(static_cast<char *>(scratch) + gemm_limb_bytes(T, K));
+  const size_t nx = (size_t)T * K, n = (size_t)T * N;
+  epi::split_limbs_kernel<<<(unsigned)((nx + 255) / 256), 256, 0, st>>>(X, nx, limbs);
+  if (gemm_mma::launch(limbs, nx, static_cast<const bf16 *>(W), part, T, N, K, splits, st) != cudaSuccess)
     return SPECVLA_ERR_CUDA;
-  const size_t n = (size_t)T * N;
-  sum_splits_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(static_cast<const float *>(scratch), splits, n, Y);
+  sum_splits_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(part, splits, n, Y);
   return cudaGetLastError() == cudaSuccess ? SPECVLA_OK : SPECVLA_ERR_CUDA;
+}
+
+int specvla_profile(specvla_ctx *ctx, int enable) {
+  if (!ctx) return SPECVLA_ERR_INVALID_ARG;
+  if (enable && ctx->prof_ev.empty()) {
+    const int pairs = 1024;            // GEMM launches between two synchronisations
+    ctx->prof_ev.resize(2 * pairs);
+    ctx->prof_cls.resize(pairs);
+    for (auto &e : ctx->prof_ev)
+      if (cudaEventCreate(&e) != cudaSuccess) return SPECVLA_ERR_CUDA;
+  }
+  if (enable) {
+    for (int i = 0; i < SPECVLA_PROF_CLASSES; i++) { ctx->prof_ms[i] = 0; ctx->prof_n[i] = 0; ctx->prof_bytes[i] = 0; }
+    ctx->prof_used = 0;
+  }
+  ctx->prof_mask = enable & 7;
+  return SPECVLA_OK;
+}
+
+int specvla_profile_read(const specvla_ctx *ctx, double *ms_out, long long *launches_out, double *bytes_out) {
+  if (!ctx || !ms_out || !launches_out || !bytes_out) return SPECVLA_ERR_INVALID_ARG;
+  for (int i = 0; i < SPECVLA_PROF_CLASSES; i++) {
+    ms_out[i] = ctx->prof_ms[i];
+    launches_out[i] = ctx->prof_n[i];
+    bytes_out[i] = ctx->prof_bytes[i];
+  }
+  return SPECVLA_OK;
 }
 
 const char *specvla_strerror(int code) {

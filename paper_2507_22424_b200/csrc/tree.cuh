@@ -70,18 +70,21 @@ __global__ void build_catchup_rows_kernel(EpArgs a, EpState *st, DevTree *trees,
   tr.sel[0] = 0;
 }
 
-// Draft-model input rows: xin[r] = bf16([feature ; embedding]) with the feature taken from
+// Draft-model input rows: xin[r] = limbs([feature ; embedding]) with the feature taken from
 // row feat_src[r] of `feat` and the embedding from E[tok] (or embeds[src] when tok < 0).
 __global__ void draft_input_kernel(RowTable rt, const int *__restrict__ feat_src,
                                    const float *__restrict__ feat, const bf16 *__restrict__ embeds,
-                                   const bf16 *__restrict__ E, int d, bf16 *__restrict__ xin) {
+                                   const bf16 *__restrict__ E, int d, bf16 *__restrict__ xin, size_t plane) {
   const int r = blockIdx.x;
   const float *f = feat + (size_t)feat_src[r] * d;
   const int tok = rt.tok[r];
   const bf16 *e = tok >= 0 ? E + (size_t)tok * d : embeds + (size_t)rt.src[r] * d;
   for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    xin[(size_t)r * 2 * d + i] = __float2bfloat16(f[i]);
+    const bf16 hi = __float2bfloat16(f[i]);
+    xin[(size_t)r * 2 * d + i] = hi;
+    xin[plane + (size_t)r * 2 * d + i] = __float2bfloat16(f[i] - __bfloat162float(hi));
     xin[(size_t)r * 2 * d + d + i] = e[i];
+    xin[plane + (size_t)r * 2 * d + d + i] = __float2bfloat16(0.f);
   }
 }
 
@@ -259,7 +262,7 @@ accept_select_kernel(EpArgs ea, DevTree *trees, EpState *st, const int *__restri
 __global__ void __launch_bounds__(256)
 kv_compact_kernel(EpArgs a, const EpState *__restrict__ st,
                   const int *__restrict__ out_m, const int *__restrict__ out_path,
-                  bf16 *__restrict__ cache, size_t ep_stride, size_t layer_stride, int max_seq, int hd) {
+                  float *__restrict__ cache, size_t ep_stride, size_t layer_stride, int max_seq, int hd) {
   const int e = a.eps[blockIdx.y];
   const int m = out_m[blockIdx.y];
   const int P = st[e].P;
@@ -267,7 +270,7 @@ kv_compact_kernel(EpArgs a, const EpState *__restrict__ st,
   const int layer = blockIdx.x >> 1, which = blockIdx.x & 1;
   uint4 *base = reinterpret_cast<uint4 *>(cache + (size_t)e * ep_stride + (size_t)layer * layer_stride +
                                           (size_t)which * max_seq * hd);
-  const int chunks = hd / 8;
+  const int chunks = hd / 4;
   for (int j = 1; j <= m; j++) {
     const int src = P + path[j], dst = P + j;
     if (src == dst) continue;

@@ -144,3 +144,28 @@ def plant_children(greedy_bin: int, n_children: int, desc: C.ModelDesc, offsets)
         used.add(b)
         toks.append(desc.action_base + b)
     return toks
+
+
+def plant_tree(shape: C.TreeShape, root_token: int, desc: C.ModelDesc, greedy_fn, seed: int, call: int):
+    """Planted draft tree on the fixed topology of `shape`: the children of every expanded node
+    are the target's greedy action bin after that node plus seeded offsets.
+
+    greedy_fn(tokens, parent, depth) must return the target's greedy token after every row of
+    the partial tree it is given (it is called once per level, root-only tree first).
+    Returns (tokens, parent, depth)."""
+    parent, depth = static_topology(shape)
+    offs = iter(planted_offsets(seed, call, 4096))
+    tokens = [int(root_token)]
+    level_start = 1
+    for l in range(shape.depth):
+        g = greedy_fn(tokens, parent[:len(tokens)], depth[:len(tokens)])
+        n_level = shape.level_sizes[l]
+        parents_in_order = []
+        for i in range(level_start, level_start + n_level):
+            if parent[i] not in parents_in_order:
+                parents_in_order.append(parent[i])
+        for p in parents_in_order:
+            gb = min(max(g[p] - desc.action_base, 0), desc.n_bins - 1)
+            tokens += plant_children(gb, shape.branch[l], desc, offs)
+        level_start += n_level
+    return tokens, parent, depth

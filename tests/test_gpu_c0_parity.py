@@ -27,12 +27,12 @@ def _gpu(c0, wcuda, **kw):
                                    (33, 1000, 1024), (64, 136, 72), (128, 512, 2048), (130, 384, 520),
                                    (290, 768, 512)])
 def test_gemm_matches_float64_matmul(T, N, K):
-    from paper_2507_22424_b200.binding import gemm_bf16
-    x = rng.normal_bf16(11, 1, (T, K), 1.0)
+    from paper_2507_22424_b200.binding import gemm
+    x = rng.normal(11, 1, (T, K), 1.0, dtype=torch.float32)
     w = rng.normal_bf16(11, 2, (N, K), 0.02)
     ref = x.double() @ w.double().T
-    y = gemm_bf16(x.cuda(), w.cuda()).cpu().double()
-    # fp32 accumulation of exact bf16 products; outputs have magnitude ~0.02 * sqrt(K)
+    y = gemm(x.cuda(), w.cuda()).cpu().double()
+    # two-limb activations (2^-18 relative) and fp32 accumulation; outputs ~0.02 * sqrt(K)
     tol = 1e-4 * 0.02 * (K ** 0.5) + 1e-6
     assert (y - ref).abs().max() < tol, float((y - ref).abs().max())
 
@@ -81,7 +81,7 @@ def test_verify_tree_matches_oracle(c0, wcuda, n_rows, seed):
             for which, ref in ((0, ep.cache.k[l]), (1, ep.cache.v[l])):
                 got = gpu.read_kv(0, l, which, 0, ep.P).double()
                 want = ref[:ep.P].reshape(ep.P, -1)
-                assert (got - want).abs().max() < 3e-2
+                assert (got - want).abs().max() < 2e-3
         st = gpu.read_buffer(5, 4, torch.int32).tolist()       # P, Pd, root, n_pending
         assert (st[0], st[2], st[3]) == (ep.P, ep.root, m_ref + 1) and P + 1 + m_ref == ep.P
     print("\n".join(log))
