@@ -353,17 +353,58 @@ def run_ours(args, rank, local_rank, world):
         dist.destroy_process_group()
 
 
+
+# --------------------------------------------------------------------------- kernel micro-run
+def run_micro(spec: str, steps: int, warmup: int):
+    """`--micro gemm:T:N:K[:M]`: the stand-alone weight-streaming GEMM (specvla_gemm) over M
+    distinct weight matrices in turn (default: enough to exceed the 126 MB L2 twice), timed
+    with CUDA events per launch. One JSON line; the target of the ncu captures under profiles/."""
+    import torch
+    from paper_2507_22424_b200 import binding as B
+    from synth_inputs import rng
+    f = spec.split(":")
+    assert f[0] == "gemm" and len(f) in (4, 5), spec
+    T, N, K = int(f[1]), int(f[2]), int(f[3])
+    wbytes = N * K * 2
+    M = int(f[4]) if len(f) == 5 else max(2, -(-2 * 126_000_000 // wbytes) + 1)
+    torch.cuda.set_device(0)
+    ws = [rng.normal_bf16(5, 10 + i, (N, K), 0.02, "cuda") for i in range(M)]
+    x = rng.normal(5, 1, (T, K), 1.0, "cuda", dtype=torch.float32)
+    g = B.GemmRunner(T, N, K)
+    for i in range(warmup):
+        g(x, ws[i % M])
+    torch.cuda.synchronize()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for i, (a, b) in enumerate(ev):
+        a.record()
+        g(x, ws[(warmup + i) % M])
+        b.record()
+    torch.cuda.synchronize()
+    ms = sorted(a.elapsed_time(b) for a, b in ev)
+    med = ms[len(ms) // 2]
+    peaks = load_peaks()
+    alg = wbytes + T * K * 4 + T * N * 4
+    print(json.dumps(dict(micro="gemm", T=T, N=N, K=K, matrices=M, steps=steps, ms_median=med, ms_min=ms[0],
+                          note="whole specvla_gemm call: limb split + GEMM + plane sum",
+                          algorithmic_bytes=alg, gbs_median=alg / med / 1e6, gbs_best=alg / ms[0] / 1e6,
+                          frac_of_peak=alg / med / 1e6 / peaks["hbm_gbs"], peak=peaks["hbm_gbs"],
+                          peak_source=peaks["source"])), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--micro", default=None, help="gemm:T:N:K[:M] - time one kernel alone (see run_micro)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
-    if args.impl == "reference":
+    if args.micro:
+        run_micro(args.micro, args.steps, args.warmup)
+    elif args.impl == "reference":
         run_reference(args, rank, world)
     else:
         import torch

@@ -1,0 +1,451 @@
+// Skinny weight-streaming GEMM on the sm_100a tensor cores (tcgen05 + TMEM, operands by TMA).
+//   part[seg][t][n] = sum over a K range of (Xhi[t][k] + Xlo[t][k]) * W[n][k]     (fp32 acc)
+// for T <= 128 activation rows: the verification forward over one draft tree and every
+// draft-model level. At these sizes the cost is the single pass over W, so the kernel is
+// built around keeping every SM's share of that stream in flight:
+//
+//  * W [N, K] (bf16, K contiguous) is cut into tiles of 256 rows x 64 columns (32 KB, one TMA
+//    box, 128-byte swizzle). The tile sits on the MMA's M axis (two M = 128 halves), the
+//    activation rows on its N axis (TN = T rounded up to 16/32/64/128). Both bf16 limbs of
+//    X are multiplied against the same W tile into the same TMEM accumulator, so fp32-grade
+//    activations cost no extra bytes of the weight stream.
+//  * The tiles x K-blocks form one linear list of units (tile-major, K inner) that is cut
+//    into gridDim.x equal contiguous ranges, one per CTA (one CTA per SM). A CTA therefore
+//    covers the end of one tile, some whole tiles and the start of another; every
+//    (CTA, tile) segment writes its partial sum to plane `seg` = CTA - first CTA of that tile,
+//    and the consuming kernel adds the planes in ascending order (deterministic).
+//  * Warp 0 issues TMA loads into a ring of stages, warp 1 issues the MMAs and releases
+//    stages through tcgen05.commit, warps 2-5 move finished accumulators (double-buffered in
+//    TMEM) to global memory.
+//  * The weight loads of the first ring-full do not depend on the previous kernel, so they
+//    are issued BEFORE griddepcontrol.wait: launched with programmatic stream serialisation
+//    the kernel streams weights while its predecessor drains.
+//
+// Every mbarrier wait is bounded (two seconds of %globaltimer); on expiry the kernel records
+// a code in *err, lets copies in flight land, frees its TMEM and returns.
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace gemm_tc {
+
+constexpr int BM = 256;                   // weight rows per tile (two UMMA halves of 128)
+constexpr int BK = 64;                    // K per stage: 128 bytes = one swizzle row
+constexpr int THREADS = 192;
+constexpr int W_STAGE_BYTES = BM * BK * 2;
+constexpr int SMEM_BUDGET = 227 * 1024;
+constexpr int MAX_T = 128;
+
+// Partition of the unit list; passed by value to the kernels that consume the partials.
+// uniform > 0: every column has exactly `uniform` planes (plain split-K producers).
+struct SegPlan {
+  int uniform;
+  int G;        // CTAs
+  int KB;       // K blocks per tile
+  int U;        // units = tiles * KB
+};
+
+__host__ __device__ inline int owner_of(const SegPlan &p, long long u) {
+  return (int)(((u + 1) * p.G - 1) / p.U);
+}
+// Planes holding partial sums of column n.
+__host__ __device__ inline int nseg_of(const SegPlan &p, int n) {
+  if (p.uniform) return p.uniform;
+  const long long f = (long long)(n / BM) * p.KB;
+  return owner_of(p, f + p.KB - 1) - owner_of(p, f) + 1;
+}
+
+constexpr int tn_of(int T) { return T <= 16 ? 16 : (T <= 32 ? 32 : (T <= 64 ? 64 : 128)); }
+constexpr int stage_bytes(int TN) { return W_STAGE_BYTES + 2 * TN * BK * 2; }
+constexpr int stages_of(int TN) {
+  return (SMEM_BUDGET - 2048) / stage_bytes(TN) > 8 ? 8 : (SMEM_BUDGET - 2048) / stage_bytes(TN);
+}
+constexpr int smem_bytes(int TN) { return stages_of(TN) * stage_bytes(TN) + 1024 + 256; }
+constexpr int tmem_cols(int TN) { return 4 * TN < 32 ? 32 : 4 * TN; }      // 64, 128, 256, 512
+
+inline SegPlan make_plan(int N, int K, int num_sms) {
+  SegPlan p;
+  p.uniform = 0;
+  p.KB = (K + BK - 1) / BK;
+  p.U = ((N + BM - 1) / BM) * p.KB;
+  p.G = p.U < num_sms ? p.U : num_sms;
+  return p;
+}
+// Largest number of planes any tile needs under `p`.
+inline int max_segments(const SegPlan &p) {
+  int m = 1;
+  for (int t = 0; t < p.U / p.KB; t++) {
+    const int s = nseg_of(p, t * BM);
+    if (s > m) m = s;
+  }
+  return m;
+}
+
+// ------------------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
+// Bounded wait: false after WAIT_LIMIT_NS without the phase completing.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 128; i++)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (global_ns() - t0 > WAIT_LIMIT_NS) return false;
+  }
+}
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm, int x, int y, uint32_t bar,
+                                            uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%2, %3}], [%4], %5;"
+      ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar), "l"(pol) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm, int x, int y, int z,
+                                            uint32_t bar, uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%2, %3, %4}], [%5], %6;"
+      ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(bar), "l"(pol) : "memory");
+}
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_alloc(uint32_t smem_dst, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tc_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 x bf16 -> f32, one CTA.
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// The mbarrier receives one arrival when every MMA issued so far by this thread has finished.
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 16 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major tile of 128-byte rows, 128-byte swizzle, 8-row
+// groups 1024 bytes apart; the tile starts on a 1024-byte boundary (plus a K offset of
+// 32 bytes per MMA step inside the swizzled row).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+  return (uint64_t)((addr >> 4) & 0x3FFF) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: f32 accumulator, bf16 x bf16, both K-major, M = 128, N = n.
+constexpr uint32_t instr_desc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+
+#define SV_ERR_WAIT_EMPTY 1
+#define SV_ERR_WAIT_FULL 2
+#define SV_ERR_WAIT_TMEM_EMPTY 3
+#define SV_ERR_WAIT_TMEM_FULL 4
+
+template <int TN>
+__global__ void __launch_bounds__(THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
+               float *__restrict__ part, int T, int N, SegPlan plan, int *__restrict__ err) {
+  constexpr int STAGES = stages_of(TN);
+  constexpr int STAGE = stage_bytes(TN);
+  constexpr uint32_t IDESC = instr_desc(TN);
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bars = base + STAGES * STAGE;
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int b) { return bars + 8u * (2 * STAGES + b); };
+  auto tempty_bar = [&](int b) { return bars + 8u * (2 * STAGES + 2 + b); };
+  const uint32_t tmem_slot = bars + 8u * (2 * STAGES + 4);
+  __shared__ uint32_t s_dummy;    // keeps a static allocation so the dynamic base is stable
+  (void)s_dummy;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long u0 = (long long)blockIdx.x * plan.U / plan.G;
+  const long long u1 = (long long)(blockIdx.x + 1) * plan.U / plan.G;
+  const int n_units = (int)(u1 - u0);
+  const int KB = plan.KB;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; s++) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int b = 0; b < 2; b++) {
+      mbar_init(tfull_bar(b), 1);
+      mbar_init(tempty_bar(b), 4);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    grid_dep_launch();
+  }
+  if (warp == 1) {
+    tc_alloc(tmem_slot, tmem_cols(TN));
+    tc_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  uint32_t tmem_base;
+  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0 && n_units > 0) {
+      const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
+      const int npre = n_units < STAGES ? n_units : STAGES;
+      bool ok = true;
+      for (int it = 0; it < n_units && ok; it++) {
+        const int st = it % STAGES, rnd = it / STAGES;
+        if (rnd > 0 && !mbar_wait(empty_bar(st), (rnd - 1) & 1)) {
+          atomicExch(err, SV_ERR_WAIT_EMPTY);
+          ok = false;
+          break;
+        }
+        const long long u = u0 + it;
+        const int tile = (int)(u / KB), kb = (int)(u % KB);
+        const uint32_t sW = base + st * STAGE;
+        mbar_expect_tx(full_bar(st), STAGE);
+        tma_load_2d(sW, &tmW, kb * BK, tile * BM, full_bar(st), pol_w);
+        if (it >= npre) tma_load_3d(sW + W_STAGE_BYTES, &tmX, kb * BK, 0, 0, full_bar(st), pol_x);
+        if (it == npre - 1) {
+          // the activations are the previous kernel's output: wait for it only now
+          grid_dep_wait();
+          for (int j = 0; j < npre; j++) {
+            const long long uj = u0 + j;
+            tma_load_3d(base + j * STAGE + W_STAGE_BYTES, &tmX, (int)(uj % KB) * BK, 0, 0, full_bar(j), pol_x);
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0 && n_units > 0) {
+      int buf = 0, uses[2] = {0, 0};
+      int prev_tile = -1;
+      for (int it = 0; it < n_units; it++) {
+        const int st = it % STAGES, rnd = it / STAGES;
+        const long long u = u0 + it;
+        const int tile = (int)(u / KB);
+        const bool first = tile != prev_tile;
+        prev_tile = tile;
+        if (first && uses[buf] > 0) {
+          if (!mbar_wait(tempty_bar(buf), (uses[buf] - 1) & 1)) {
+            atomicExch(err, SV_ERR_WAIT_TMEM_EMPTY);
+            break;
+          }
+        }
+        if (!mbar_wait(full_bar(st), rnd & 1)) {
+          atomicExch(err, SV_ERR_WAIT_FULL);
+          break;
+        }
+        tc_fence_after();
+        const uint32_t sW = base + st * STAGE, sX = sW + W_STAGE_BYTES;
+#pragma unroll
+        for (int kk = 0; kk < BK / 16; kk++) {
+#pragma unroll
+          for (int h = 0; h < 2; h++) {
+            const uint64_t adesc = smem_desc(sW + h * (128 * BK * 2) + kk * 32);
+            const uint32_t d = tmem_base + (uint32_t)((buf * 2 + h) * TN);
+#pragma unroll
+            for (int limb = 0; limb < 2; limb++) {
+              const uint64_t bdesc = smem_desc(sX + limb * (TN * BK * 2) + kk * 32);
+              tc_mma(d, adesc, bdesc, IDESC, (first && kk == 0 && limb == 0) ? 0u : 1u);
+            }
+          }
+        }
+        tc_commit(empty_bar(st));
+        const bool last = (it == n_units - 1) || ((int)((u + 1) / KB) != tile);
+        if (last) {
+          tc_commit(tfull_bar(buf));
+          uses[buf]++;
+          buf ^= 1;
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    grid_dep_wait();
+    const int q = warp & 3;                       // TMEM lane quarter this warp may access
+    int buf = 0, uses[2] = {0, 0};
+    int it = 0;
+    while (it < n_units) {
+      const long long u = u0 + it;
+      const int tile = (int)(u / KB), kb0 = (int)(u % KB);
+      int cnt = KB - kb0;
+      if (cnt > n_units - it) cnt = n_units - it;
+      if (!mbar_wait(tfull_bar(buf), uses[buf] & 1)) {
+        if (lane == 0) atomicExch(err, SV_ERR_WAIT_TMEM_FULL);
+        break;
+      }
+      tc_fence_after();
+      const int seg = (int)blockIdx.x - owner_of(plan, (long long)tile * KB);
+      float *out = part + (size_t)seg * T * N;
+#pragma unroll
+      for (int h = 0; h < 2; h++) {
+        const int n = tile * BM + h * 128 + q * 32 + lane;
+#pragma unroll
+        for (int c0 = 0; c0 < TN; c0 += 16) {
+          uint32_t r[16];
+          tc_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)((buf * 2 + h) * TN + c0), r);
+          tc_wait_ld();
+          if (n < N) {
+#pragma unroll
+            for (int j = 0; j < 16; j++)
+              if (c0 + j < T) out[(size_t)(c0 + j) * N + n] = __uint_as_float(r[j]);
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(buf));
+      uses[buf]++;
+      buf ^= 1;
+      it += cnt;
+    }
+  }
+
+  if (*reinterpret_cast<volatile int *>(err) != 0) {
+    // a wait gave up somewhere: give copies in flight time to land before the smem goes away
+    const uint64_t t0 = global_ns();
+    while (global_ns() - t0 < 200000ull) __nanosleep(1000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 1) tc_dealloc(tmem_base, tmem_cols(TN));
+}
+
+// ------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+inline EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// Weight matrix [N, K] bf16, K contiguous: boxes of 256 rows x 64 columns.
+inline bool make_w_map(CUtensorMap *tm, const bf16 *W, int N, int K) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)N};
+  cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+  cuuint32_t box[2] = {BK, BM};
+  cuuint32_t es[2] = {1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<bf16 *>(W), dims, strides, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+// Activation limbs [2][rows][K] bf16 (lo limb `plane` elements after hi): boxes of
+// 2 limbs x TN rows x 64 columns. Rows past `rows` read as zero.
+inline bool make_x_map(CUtensorMap *tm, const bf16 *X, size_t plane, int rows, int K, int TN) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)rows, 2};
+  cuuint64_t strides[2] = {(cuuint64_t)K * 2, (cuuint64_t)plane * 2};
+  cuuint32_t box[3] = {BK, (cuuint32_t)TN, 2};
+  cuuint32_t es[3] = {1, 1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<bf16 *>(X), dims, strides, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int TN>
+inline cudaError_t launch_tn(const CUtensorMap &tmW, const CUtensorMap &tmX, float *part, int T, int N,
+                             const SegPlan &plan, int *err, cudaStream_t st, bool pdl) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<TN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         smem_bytes(TN));
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(plan.G);
+  cfg.blockDim = dim3(THREADS);
+  cfg.dynamicSmemBytes = smem_bytes(TN);
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<TN>, tmW, tmX, part, T, N, plan, err);
+}
+
+// tmX must have been made with TN = tn_of(T).
+inline cudaError_t launch(const CUtensorMap &tmW, const CUtensorMap &tmX, float *part, int T, int N,
+                          const SegPlan &plan, int *err, cudaStream_t st, bool pdl) {
+  switch (tn_of(T)) {
+    case 16: return launch_tn<16>(tmW, tmX, part, T, N, plan, err, st, pdl);
+    case 32: return launch_tn<32>(tmW, tmX, part, T, N, plan, err, st, pdl);
+    case 64: return launch_tn<64>(tmW, tmX, part, T, N, plan, err, st, pdl);
+    default: return launch_tn<128>(tmW, tmX, part, T, N, plan, err, st, pdl);
+  }
+}
+
+}  // namespace gemm_tc
