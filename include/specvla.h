@@ -199,6 +199,10 @@ int specvla_read_kv(specvla_ctx *ctx, int draft, int episode, int layer, int whi
 size_t specvla_gemm_scratch_bytes(int T, int N, int K);
 int specvla_gemm(const float *X, const void *W, float *Y, int T, int N, int K,
                  void *scratch, size_t scratch_bytes, void *stream);
+/* Synchronises `stream` and reports whether the specvla_gemm calls that used `scratch` ran
+ * to completion: SPECVLA_ERR_TIMEOUT if a bounded device-side wait gave up (Y is then
+ * undefined), SPECVLA_ERR_CUDA if the stream is in error, else SPECVLA_OK. */
+int specvla_gemm_status(const void *scratch, void *stream);
 
 /* Per-GEMM device timing (measurement aid; Section 3.1 attributes the latency to the
  * parameter stream, which these GEMMs are). `phases` is a bit mask: 1 = prefill, 2 = draft,

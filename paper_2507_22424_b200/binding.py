@@ -70,6 +70,7 @@ EXPORTS = {
     "specvla_gemm_scratch_bytes": (C.c_size_t, [C.c_int, C.c_int, C.c_int]),
     "specvla_gemm": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                                     C.c_void_p, C.c_size_t, C.c_void_p]),
+    "specvla_gemm_status": (C.c_int, [C.c_void_p, C.c_void_p]),
     "specvla_profile": (C.c_int, [C.c_void_p, C.c_int]),
     "specvla_profile_read": (C.c_int, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_longlong),
                                        C.POINTER(C.c_double)]),
@@ -274,6 +275,8 @@ def gemm(x: torch.Tensor, w: torch.Tensor) -> torch.Tensor:
     sp = (scratch.data_ptr() + 1023) // 1024 * 1024
     rc = lib.specvla_gemm(C.c_void_p(x.data_ptr()), C.c_void_p(w.data_ptr()), C.c_void_p(y.data_ptr()),
                                T, N, K, C.c_void_p(sp), nb, _stream())
+    if rc == 0:
+        rc = lib.specvla_gemm_status(C.c_void_p(sp), _stream())
     if rc != 0:
         raise SpecVLAError(rc)
     return y

@@ -17,6 +17,15 @@ __device__ __forceinline__ void store2(bf16 *hi_plane, size_t plane, size_t idx,
   hi_plane[plane + idx] = __float2bfloat16(v - __bfloat162float(hi));
 }
 
+// Output element (t, n) of a GEMM: its planes added in ascending order.
+__device__ __forceinline__ float col_sum(const float *__restrict__ part, const SegPlan &sp, int T, int N,
+                                         int t, int n) {
+  const int planes = nseg_of(sp, n);
+  float v = 0.f;
+  for (int s = 0; s < planes; s++) v += part[((size_t)s * T + t) * N + n];
+  return v;
+}
+
 __device__ __forceinline__ float block_sum(float v, float *red) {
   v = warp_sum(v);
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -57,7 +66,7 @@ embed_norm_kernel(RowTable rt, const bf16 *__restrict__ embeds, const bf16 *__re
 //   gain != NULL: xn[t] = limbs(rmsnorm(x[t]) * gain), feat[t] = rmsnorm(x[t]) * gain (if feat)
 //   gain == NULL: xn[t] = limbs(x[t])
 __global__ void __launch_bounds__(THREADS)
-residual_norm_kernel(const float *__restrict__ part, int splits, int T, int d, int accumulate,
+residual_norm_kernel(const float *__restrict__ part, SegPlan sp, int T, int d, int accumulate,
                      const float *__restrict__ gain, float eps, float *__restrict__ x,
                      bf16 *__restrict__ xn, size_t plane, float *__restrict__ feat) {
   __shared__ float red[32];
@@ -65,6 +74,7 @@ residual_norm_kernel(const float *__restrict__ part, int splits, int T, int d, i
   float ss = 0.f;
   for (int i = threadIdx.x; i < d; i += blockDim.x) {
     float v = accumulate ? x[(size_t)t * d + i] : 0.f;
+    const int splits = nseg_of(sp, i);
     for (int s = 0; s < splits; s++) v += part[((size_t)s * T + t) * d + i];
     x[(size_t)t * d + i] = v;
     ss += v * v;
@@ -87,7 +97,7 @@ residual_norm_kernel(const float *__restrict__ part, int splits, int T, int d, i
 // (i, i + dh/2), angle from the precomputed table); write q and, into the row's cache slot,
 // k and v, all fp32. Cache layout per episode: [2 (K, V)][max_seq][H * dh] fp32.
 __global__ void __launch_bounds__(THREADS)
-qkv_rope_append_kernel(const float *__restrict__ part, int splits, int T, int H, int dh,
+qkv_rope_append_kernel(const float *__restrict__ part, SegPlan sp, int T, int H, int dh,
                        RowTable rt, const float2 *__restrict__ rope_tab, float *__restrict__ q,
                        float *__restrict__ cache, size_t ep_stride, int max_seq) {
   const int t = blockIdx.x;
@@ -98,13 +108,9 @@ qkv_rope_append_kernel(const float *__restrict__ part, int splits, int T, int H,
   for (int i = threadIdx.x; i < H * half; i += blockDim.x) {
     const int h = i / half, j = i - h * half;
     const int c0 = h * dh + j, c1 = c0 + half;
-    float qlo = 0.f, qhi = 0.f, klo = 0.f, khi = 0.f, vlo = 0.f, vhi = 0.f;
-    for (int s = 0; s < splits; s++) {
-      const float *p = part + ((size_t)s * T + t) * N;
-      qlo += p[c0]; qhi += p[c1];
-      klo += p[hd + c0]; khi += p[hd + c1];
-      vlo += p[2 * hd + c0]; vhi += p[2 * hd + c1];
-    }
+    const float qlo = col_sum(part, sp, T, N, t, c0), qhi = col_sum(part, sp, T, N, t, c1);
+    const float klo = col_sum(part, sp, T, N, t, hd + c0), khi = col_sum(part, sp, T, N, t, hd + c1);
+    const float vlo = col_sum(part, sp, T, N, t, 2 * hd + c0), vhi = col_sum(part, sp, T, N, t, 2 * hd + c1);
     const float2 cs = rope_tab[(size_t)pos * half + j];
     q[(size_t)t * hd + c0] = qlo * cs.x - qhi * cs.y;
     q[(size_t)t * hd + c1] = qhi * cs.x + qlo * cs.y;
@@ -117,17 +123,12 @@ qkv_rope_append_kernel(const float *__restrict__ part, int splits, int T, int H,
 
 // hid[t][n] = limbs( silu(g) * u ), g = sum_s part[s][t][n], u = sum_s part[s][t][F + n].
 __global__ void __launch_bounds__(THREADS)
-swiglu_kernel(const float *__restrict__ part, int splits, int T, int F, bf16 *__restrict__ hid,
+swiglu_kernel(const float *__restrict__ part, SegPlan sp, int T, int F, bf16 *__restrict__ hid,
               size_t plane) {
   const int t = blockIdx.y;
   const int n = blockIdx.x * blockDim.x + threadIdx.x;
   if (n >= F) return;
-  float g = 0.f, u = 0.f;
-  for (int s = 0; s < splits; s++) {
-    const float *p = part + ((size_t)s * T + t) * 2 * F;
-    g += p[n];
-    u += p[F + n];
-  }
+  const float g = col_sum(part, sp, T, 2 * F, t, n), u = col_sum(part, sp, T, 2 * F, t, F + n);
   store2(hid, plane, (size_t)t * F + n, g / (1.f + expf(-g)) * u);
 }
 
@@ -183,14 +184,13 @@ __device__ __forceinline__ void top2_merge(Top2 &a, const Top2 &b) {
 // Greedy token per row: logits = sum_s part[s][t][:]; argmax over [lo, hi) with ties to the
 // lowest id; margin = top-1 minus top-2 over the same range. Optionally dumps the logits.
 __global__ void __launch_bounds__(THREADS)
-argmax_kernel(const float *__restrict__ part, int splits, int T, int V, int lo, int hi,
+argmax_kernel(const float *__restrict__ part, SegPlan sp, int T, int V, int lo, int hi,
               int *__restrict__ greedy, float *__restrict__ margin, float *__restrict__ logits_out) {
   __shared__ Top2 red[THREADS / 32];
   const int t = blockIdx.x;
   Top2 best{-INFINITY, -INFINITY, 0x7fffffff};
   for (int v = threadIdx.x; v < V; v += blockDim.x) {
-    float x = 0.f;
-    for (int s = 0; s < splits; s++) x += part[((size_t)s * T + t) * V + v];
+    const float x = col_sum(part, sp, T, V, t, v);
     if (logits_out) logits_out[(size_t)t * V + v] = x;
     if (v >= lo && v < hi) top2_push(best, x, v);
   }
@@ -214,7 +214,7 @@ argmax_kernel(const float *__restrict__ part, int splits, int T, int V, int lo, 
 // Draft scoring per row: log-softmax of the logits over [lo, hi) and its top-K entries
 // (ties to the lowest id), K = SV_TOPK. Selection by K rounds of block argmax.
 __global__ void __launch_bounds__(THREADS)
-logsoftmax_topk_kernel(const float *__restrict__ part, int splits, int T, int V, int lo, int hi,
+logsoftmax_topk_kernel(const float *__restrict__ part, SegPlan sp, int T, int V, int lo, int hi,
                        float *__restrict__ scratch_logits, int *__restrict__ top_tok,
                        float *__restrict__ top_lp) {
   __shared__ float redf[32];
@@ -225,8 +225,7 @@ logsoftmax_topk_kernel(const float *__restrict__ part, int splits, int T, int V,
   float *lg = scratch_logits + (size_t)t * V;
   float mx = -INFINITY;
   for (int v = lo + threadIdx.x; v < hi; v += blockDim.x) {
-    float x = 0.f;
-    for (int s = 0; s < splits; s++) x += part[((size_t)s * T + t) * V + v];
+    const float x = col_sum(part, sp, T, V, t, v);
     lg[v] = x;
     mx = fmaxf(mx, x);
   }

@@ -30,39 +30,20 @@
 
 namespace gemm_tc {
 
-constexpr int BM = 256;                   // weight rows per tile (two UMMA halves of 128)
+constexpr int BM = SV_TILE_ROWS;          // weight rows per tile (two UMMA halves of 128)
 constexpr int BK = 64;                    // K per stage: 128 bytes = one swizzle row
 constexpr int THREADS = 192;
 constexpr int W_STAGE_BYTES = BM * BK * 2;
 constexpr int SMEM_BUDGET = 227 * 1024;
 constexpr int MAX_T = 128;
 
-// Partition of the unit list; passed by value to the kernels that consume the partials.
-// uniform > 0: every column has exactly `uniform` planes (plain split-K producers).
-struct SegPlan {
-  int uniform;
-  int G;        // CTAs
-  int KB;       // K blocks per tile
-  int U;        // units = tiles * KB
-};
-
-__host__ __device__ inline int owner_of(const SegPlan &p, long long u) {
-  return (int)(((u + 1) * p.G - 1) / p.U);
-}
-// Planes holding partial sums of column n.
-__host__ __device__ inline int nseg_of(const SegPlan &p, int n) {
-  if (p.uniform) return p.uniform;
-  const long long f = (long long)(n / BM) * p.KB;
-  return owner_of(p, f + p.KB - 1) - owner_of(p, f) + 1;
-}
-
-constexpr int tn_of(int T) { return T <= 16 ? 16 : (T <= 32 ? 32 : (T <= 64 ? 64 : 128)); }
-constexpr int stage_bytes(int TN) { return W_STAGE_BYTES + 2 * TN * BK * 2; }
-constexpr int stages_of(int TN) {
+__host__ __device__ constexpr int tn_of(int T) { return T <= 16 ? 16 : (T <= 32 ? 32 : (T <= 64 ? 64 : 128)); }
+__host__ __device__ constexpr int stage_bytes(int TN) { return W_STAGE_BYTES + 2 * TN * BK * 2; }
+__host__ __device__ constexpr int stages_of(int TN) {
   return (SMEM_BUDGET - 2048) / stage_bytes(TN) > 8 ? 8 : (SMEM_BUDGET - 2048) / stage_bytes(TN);
 }
-constexpr int smem_bytes(int TN) { return stages_of(TN) * stage_bytes(TN) + 1024 + 256; }
-constexpr int tmem_cols(int TN) { return 4 * TN < 32 ? 32 : 4 * TN; }      // 64, 128, 256, 512
+__host__ __device__ constexpr int smem_bytes(int TN) { return stages_of(TN) * stage_bytes(TN) + 1024 + 256; }
+__host__ __device__ constexpr int tmem_cols(int TN) { return 4 * TN < 32 ? 32 : 4 * TN; }      // 64, 128, 256, 512
 
 inline SegPlan make_plan(int N, int K, int num_sms) {
   SegPlan p;
@@ -187,7 +168,7 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
   return (uint64_t)((addr >> 4) & 0x3FFF) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
 }
 // Instruction descriptor: f32 accumulator, bf16 x bf16, both K-major, M = 128, N = n.
-constexpr uint32_t instr_desc(int n) {
+__host__ __device__ constexpr uint32_t instr_desc(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
@@ -211,8 +192,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   auto tfull_bar = [&](int b) { return bars + 8u * (2 * STAGES + b); };
   auto tempty_bar = [&](int b) { return bars + 8u * (2 * STAGES + 2 + b); };
   const uint32_t tmem_slot = bars + 8u * (2 * STAGES + 4);
-  __shared__ uint32_t s_dummy;    // keeps a static allocation so the dynamic base is stable
-  (void)s_dummy;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long long u0 = (long long)blockIdx.x * plan.U / plan.G;
@@ -275,7 +254,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0 && n_units > 0) {
-      int buf = 0, uses[2] = {0, 0};
+      int sidx = -1;                 // segment number; accumulator buffer = sidx & 1
       int prev_tile = -1;
       for (int it = 0; it < n_units; it++) {
         const int st = it % STAGES, rnd = it / STAGES;
@@ -283,12 +262,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         const int tile = (int)(u / KB);
         const bool first = tile != prev_tile;
         prev_tile = tile;
-        if (first && uses[buf] > 0) {
-          if (!mbar_wait(tempty_bar(buf), (uses[buf] - 1) & 1)) {
+        if (first) {
+          sidx++;
+          // the buffer's previous accumulator (segment sidx - 2) must have been read out
+          if (sidx >= 2 && !mbar_wait(tempty_bar(sidx & 1), ((sidx >> 1) - 1) & 1)) {
             atomicExch(err, SV_ERR_WAIT_TMEM_EMPTY);
             break;
           }
         }
+        const int buf = sidx & 1;
         if (!mbar_wait(full_bar(st), rnd & 1)) {
           atomicExch(err, SV_ERR_WAIT_FULL);
           break;
@@ -310,25 +292,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         }
         tc_commit(empty_bar(st));
         const bool last = (it == n_units - 1) || ((int)((u + 1) / KB) != tile);
-        if (last) {
-          tc_commit(tfull_bar(buf));
-          uses[buf]++;
-          buf ^= 1;
-        }
+        if (last) tc_commit(tfull_bar(buf));
       }
     }
   } else {
     // ------------------------------------------------------------------ epilogue (warps 2..5)
     grid_dep_wait();
     const int q = warp & 3;                       // TMEM lane quarter this warp may access
-    int buf = 0, uses[2] = {0, 0};
+    int sidx = 0;
     int it = 0;
     while (it < n_units) {
+      const int buf = sidx & 1;
       const long long u = u0 + it;
       const int tile = (int)(u / KB), kb0 = (int)(u % KB);
       int cnt = KB - kb0;
       if (cnt > n_units - it) cnt = n_units - it;
-      if (!mbar_wait(tfull_bar(buf), uses[buf] & 1)) {
+      if (!mbar_wait(tfull_bar(buf), (sidx >> 1) & 1)) {
         if (lane == 0) atomicExch(err, SV_ERR_WAIT_TMEM_FULL);
         break;
       }
@@ -353,8 +332,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(buf));
-      uses[buf]++;
-      buf ^= 1;
+      sidx++;
       it += cnt;
     }
   }

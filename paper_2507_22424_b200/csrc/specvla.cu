@@ -14,14 +14,34 @@
 #include "common.cuh"
 #include "epilogue.cuh"
 #include "gemm_mma.cuh"
+#include "gemm_tc.cuh"
 #include "tree.cuh"
 
 namespace {
 
+// A weight matrix [N, K] and its TMA map (boxes of the tensor-core GEMM).
+struct WMat {
+  const bf16 *p;
+  int N, K;
+  bool has_map;
+  CUtensorMap map;
+};
+// A two-limb activation buffer [2][rows][K] and its TMA maps, one per row-tile size 16/32/64/128.
+struct XBuf {
+  bf16 *p;
+  size_t plane;
+  int rows, K;
+  bool has_map;
+  CUtensorMap map[4];
+};
+inline int tn_index(int TN) { return TN == 16 ? 0 : (TN == 32 ? 1 : (TN == 64 ? 2 : 3)); }
+
 struct LayerW {
-  const bf16 *wqkv, *wo, *wgu, *wd;
+  WMat wqkv, wo, wgu, wd;
   const float *norm1, *norm2;
 };
+
+constexpr int MAX_CTAS = 148;     // grid of the tensor-core GEMM assumed when sizing the workspace
 
 constexpr int MAX_SPLITS = 8;
 constexpr size_t ALIGN = 1024;
@@ -46,9 +66,13 @@ struct specvla_ctx {
   int max_draft_rows;           // rows of one draft-tree level summed over episodes
   std::vector<LayerW> layers;
   LayerW dlayer;
-  const bf16 *embed, *lm_head, *draft_fc;
+  const bf16 *embed;
+  WMat lm_head, draft_fc;
   const float *final_norm;
   bool has_draft;
+  int num_ctas;                 // CTAs of the tensor-core GEMM: min(SM count, MAX_CTAS)
+  bool use_tc;                  // tensor-core (tcgen05) GEMM for calls of <= 128 rows
+  bool use_pdl;                 // programmatic dependent launch between the kernels of a forward
 
   // workspace carve-up (device)
   float *kv_t, *kv_d;           // target [ep][layer][2][max_seq][hd], draft [ep][2][max_seq][hd], fp32
@@ -56,9 +80,9 @@ struct specvla_ctx {
   float2 *rope_tab;
   float *x, *feat, *part, *lgs, *pend_feat, *dout, *margin, *top_lp, *q;
   size_t part_floats;
-  // GEMM operands, two bf16 limbs each: hi plane, then the lo plane *_pl elements later
-  bf16 *xn, *xin, *ao, *hid, *lm_in;
-  size_t xn_pl, xin_pl, ao_pl, hid_pl, lm_pl;
+  // GEMM operands, two bf16 limbs each: hi plane, then the lo plane `plane` elements later
+  XBuf xn, xin, ao, hid, lm_in;
+  int *err;                     // device status word written by bounded waits that gave up
   RowTable rt;
   int *feat_src, *dst_row, *lm_rows, *greedy, *top_tok, *out_m, *out_tok, *out_path;
   EpState *st;
@@ -137,23 +161,36 @@ size_t carve(specvla_ctx *c, char *base) {
   c->rope_tab = cv.take<float2>((size_t)d.max_seq * (d.head_dim / 2));
   c->x = cv.take<float>(R * d.d_model);
   c->feat = cv.take<float>(R * d.d_model);
-  c->xn_pl = R * d.d_model;
-  c->xin_pl = R * 2 * d.d_model;
-  c->ao_pl = R * hd;
-  c->hid_pl = R * d.d_ffn;
-  c->lm_pl = lm_rows * d.d_model;
-  c->xn = cv.take<bf16>(2 * c->xn_pl);
-  c->xin = cv.take<bf16>(2 * c->xin_pl);
+  auto limbs = [&](XBuf &b, size_t rows, size_t K) {
+    b.rows = (int)rows;
+    b.K = (int)K;
+    b.plane = rows * K;
+    b.p = cv.take<bf16>(2 * b.plane);
+  };
+  limbs(c->xn, R, d.d_model);
+  limbs(c->xin, R, 2 * d.d_model);
   c->q = cv.take<float>(R * hd);
-  c->ao = cv.take<bf16>(2 * c->ao_pl);
-  c->hid = cv.take<bf16>(2 * c->hid_pl);
-  c->lm_in = cv.take<bf16>(2 * c->lm_pl);
+  limbs(c->ao, R, hd);
+  limbs(c->hid, R, d.d_ffn);
+  limbs(c->lm_in, lm_rows, d.d_model);
   size_t widest = (size_t)3 * hd;
   if ((size_t)2 * d.d_ffn > widest) widest = (size_t)2 * d.d_ffn;
   size_t pf = R * widest;                                  // one split over all rows
   const size_t small_rows = lm_rows < R ? lm_rows : R;
   if ((size_t)MAX_SPLITS * small_rows * widest > pf) pf = (size_t)MAX_SPLITS * small_rows * widest;
   if (lm_rows * d.vocab > pf) pf = lm_rows * (size_t)d.vocab;
+  // tensor-core path (calls of <= 128 rows): one plane per (CTA, tile) segment
+  auto tc_need = [&](size_t rows, int N, int K) {
+    if (rows > (size_t)gemm_tc::MAX_T) rows = gemm_tc::MAX_T;
+    const size_t need = (size_t)gemm_tc::max_segments(gemm_tc::make_plan(N, K, c->num_ctas)) * rows * N;
+    if (need > pf) pf = need;
+  };
+  tc_need(R, 3 * hd, d.d_model);
+  tc_need(R, d.d_model, hd);
+  tc_need(R, 2 * d.d_ffn, d.d_model);
+  tc_need(R, d.d_model, d.d_ffn);
+  tc_need(R, d.d_model, 2 * d.d_model);
+  tc_need(lm_rows, d.vocab, d.d_model);
   c->part_floats = pf;
   c->part = cv.take<float>(pf);
   c->lgs = cv.take<float>(dr * d.vocab);
@@ -179,6 +216,7 @@ size_t carve(specvla_ctx *c, char *base) {
   c->out_path = cv.take<int>(E * (SV_MAX_DEPTH + 1));
   c->st = cv.take<EpState>(E);
   c->trees = cv.take<DevTree>(E);
+  c->err = cv.take<int>(32);
   return (cv.off + ALIGN - 1) / ALIGN * ALIGN;
 }
 
@@ -205,23 +243,33 @@ void prof_collect(specvla_ctx *ctx) {
   ctx->prof_used = 0;
 }
 
-// part <- A[R, K] * W[N, K]^T split over K; returns the number of splits to sum.
-int gemm(specvla_ctx *ctx, const bf16 *A, size_t a_plane, const bf16 *W, int R, int N, int K,
-         cudaStream_t st, int *splits_out, int cls) {
-  int cap = (int)(ctx->part_floats / ((size_t)R * N));
-  if (cap < 1) return SPECVLA_ERR_CAPACITY;
-  if (cap > MAX_SPLITS) cap = MAX_SPLITS;
-  const int splits = gemm_mma::plan_splits(R, N, K, cap);
+// part <- A[R, K] * W[N, K]^T as planes of partial sums; *plan says how many planes each
+// output column has. Calls of <= 128 rows go to the tensor-core streaming kernel.
+int gemm(specvla_ctx *ctx, const XBuf &A, const WMat &W, int R, cudaStream_t st, SegPlan *plan,
+         int cls) {
+  const int N = W.N, K = W.K;
+  const bool tc = ctx->use_tc && R <= gemm_tc::MAX_T && W.has_map && A.has_map && A.K == K;
   const bool prof = (ctx->prof_mask & ctx->phase) && 2 * (ctx->prof_used + 1) <= (int)ctx->prof_ev.size();
   if (prof) CU(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used], st));
-  CU(gemm_mma::launch(A, a_plane, W, ctx->part, R, N, K, splits, st));
+  if (tc) {
+    *plan = gemm_tc::make_plan(N, K, ctx->num_ctas);
+    if ((size_t)gemm_tc::max_segments(*plan) * R * N > ctx->part_floats) return SPECVLA_ERR_CAPACITY;
+    CU(gemm_tc::launch(W.map, A.map[tn_index(gemm_tc::tn_of(R))], ctx->part, R, N, *plan, ctx->err, st,
+                       ctx->use_pdl));
+  } else {
+    int cap = (int)(ctx->part_floats / ((size_t)R * N));
+    if (cap < 1) return SPECVLA_ERR_CAPACITY;
+    if (cap > MAX_SPLITS) cap = MAX_SPLITS;
+    const int splits = gemm_mma::plan_splits(R, N, K, cap);
+    CU(gemm_mma::launch(A.p, A.plane, W.p, ctx->part, R, N, K, splits, st));
+    *plan = SegPlan{splits, 1, 1, 1};
+  }
   if (prof) {
     CU(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used + 1], st));
     ctx->prof_cls[ctx->prof_used++] = cls;
     ctx->prof_bytes[cls] += (double)N * K * sizeof(bf16);
   }
   ctx->launches++;
-  *splits_out = splits;
   return SPECVLA_OK;
 }
 
@@ -231,10 +279,10 @@ int attention(specvla_ctx *ctx, int R, const float *cache, size_t ep_stride, cud
   dim3 grid(d.n_heads, R);
   if (d.head_dim == 128)
     attn::tree_attention_kernel<128><<<grid, attn::WARPS * 32, 0, st>>>(
-        ctx->q, cache, ep_stride, d.max_seq, d.n_heads, ctx->rt, scale, ctx->ao, ctx->ao_pl);
+        ctx->q, cache, ep_stride, d.max_seq, d.n_heads, ctx->rt, scale, ctx->ao.p, ctx->ao.plane);
   else
     attn::tree_attention_kernel<64><<<grid, attn::WARPS * 32, 0, st>>>(
-        ctx->q, cache, ep_stride, d.max_seq, d.n_heads, ctx->rt, scale, ctx->ao, ctx->ao_pl);
+        ctx->q, cache, ep_stride, d.max_seq, d.n_heads, ctx->rt, scale, ctx->ao.p, ctx->ao.plane);
   LAUNCHED();
   return SPECVLA_OK;
 }
@@ -246,34 +294,34 @@ int run_layer(specvla_ctx *ctx, const LayerW &w, int R, float *cache, size_t ep_
               const float *next_gain, float *feat_out, cudaStream_t st) {
   const specvla_model_desc &d = ctx->desc;
   const int hd = ctx->hd, D = d.d_model, F = d.d_ffn;
-  int s;
-  TRY(gemm(ctx, ctx->xn, ctx->xn_pl, w.wqkv, R, 3 * hd, D, st, &s, SPECVLA_PROF_QKV));
+  SegPlan s;
+  TRY(gemm(ctx, ctx->xn, w.wqkv, R, st, &s, SPECVLA_PROF_QKV));
   epi::qkv_rope_append_kernel<<<R, epi::THREADS, 0, st>>>(ctx->part, s, R, d.n_heads, d.head_dim, ctx->rt,
                                                           ctx->rope_tab, ctx->q, cache, ep_stride,
                                                           d.max_seq);
   LAUNCHED();
   TRY(attention(ctx, R, cache, ep_stride, st));
-  TRY(gemm(ctx, ctx->ao, ctx->ao_pl, w.wo, R, D, hd, st, &s, SPECVLA_PROF_O));
+  TRY(gemm(ctx, ctx->ao, w.wo, R, st, &s, SPECVLA_PROF_O));
   epi::residual_norm_kernel<<<R, epi::THREADS, 0, st>>>(ctx->part, s, R, D, 1, w.norm2, d.rms_eps, ctx->x,
-                                                        ctx->xn, ctx->xn_pl, nullptr);
+                                                        ctx->xn.p, ctx->xn.plane, nullptr);
   LAUNCHED();
-  TRY(gemm(ctx, ctx->xn, ctx->xn_pl, w.wgu, R, 2 * F, D, st, &s, SPECVLA_PROF_GATE_UP));
+  TRY(gemm(ctx, ctx->xn, w.wgu, R, st, &s, SPECVLA_PROF_GATE_UP));
   epi::swiglu_kernel<<<dim3((F + epi::THREADS - 1) / epi::THREADS, R), epi::THREADS, 0, st>>>(
-      ctx->part, s, R, F, ctx->hid, ctx->hid_pl);
+      ctx->part, s, R, F, ctx->hid.p, ctx->hid.plane);
   LAUNCHED();
-  TRY(gemm(ctx, ctx->hid, ctx->hid_pl, w.wd, R, D, F, st, &s, SPECVLA_PROF_DOWN));
+  TRY(gemm(ctx, ctx->hid, w.wd, R, st, &s, SPECVLA_PROF_DOWN));
   epi::residual_norm_kernel<<<R, epi::THREADS, 0, st>>>(ctx->part, s, R, D, 1, next_gain, d.rms_eps,
-                                                        ctx->x, ctx->xn, ctx->xn_pl, feat_out);
+                                                        ctx->x, ctx->xn.p, ctx->xn.plane, feat_out);
   LAUNCHED();
   return SPECVLA_OK;
 }
 
 // Target model over the R rows described by ctx->rt: embedding, all layers, final norm.
-// Leaves features in ctx->feat (fp32) and ctx->xn (bf16).
+// Leaves features in ctx->feat (fp32) and ctx->xn.p (bf16).
 int target_forward(specvla_ctx *ctx, int R, const bf16 *embeds, cudaStream_t st) {
   const specvla_model_desc &d = ctx->desc;
   epi::embed_norm_kernel<<<R, epi::THREADS, 0, st>>>(ctx->rt, embeds, ctx->embed, ctx->layers[0].norm1,
-                                                     d.rms_eps, d.d_model, ctx->x, ctx->xn, ctx->xn_pl);
+                                                     d.rms_eps, d.d_model, ctx->x, ctx->xn.p, ctx->xn.plane);
   LAUNCHED();
   for (int l = 0; l < d.n_layers; l++) {
     const bool last = (l + 1 == d.n_layers);
@@ -285,22 +333,22 @@ int target_forward(specvla_ctx *ctx, int R, const bf16 *embeds, cudaStream_t st)
   return SPECVLA_OK;
 }
 
-// Draft model over R rows: ctx->xin = [feature ; embedding] rows are already built.
-// Leaves the layer outputs in ctx->x (fp32) and ctx->xn (bf16, un-normalised).
+// Draft model over R rows: ctx->xin.p = [feature ; embedding] rows are already built.
+// Leaves the layer outputs in ctx->x (fp32) and ctx->xn.p (bf16, un-normalised).
 int draft_forward(specvla_ctx *ctx, int R, cudaStream_t st) {
   const specvla_model_desc &d = ctx->desc;
-  int s;
-  TRY(gemm(ctx, ctx->xin, ctx->xin_pl, ctx->draft_fc, R, d.d_model, 2 * d.d_model, st, &s, SPECVLA_PROF_FC));
+  SegPlan s;
+  TRY(gemm(ctx, ctx->xin, ctx->draft_fc, R, st, &s, SPECVLA_PROF_FC));
   epi::residual_norm_kernel<<<R, epi::THREADS, 0, st>>>(ctx->part, s, R, d.d_model, 0, ctx->dlayer.norm1,
-                                                        d.rms_eps, ctx->x, ctx->xn, ctx->xn_pl, nullptr);
+                                                        d.rms_eps, ctx->x, ctx->xn.p, ctx->xn.plane, nullptr);
   LAUNCHED();
   return run_layer(ctx, ctx->dlayer, R, ctx->kv_d, ctx->kv_d_ep_stride, nullptr, nullptr, st);
 }
 
-// LM head over `rows` bf16 rows of A: partial logits land in ctx->part; returns splits.
-int lm_head(specvla_ctx *ctx, const bf16 *A, size_t a_plane, int rows, cudaStream_t st, int *splits) {
+// LM head over `rows` two-limb rows of A: partial logits land in ctx->part.
+int lm_head(specvla_ctx *ctx, const XBuf &A, int rows, cudaStream_t st, SegPlan *plan) {
   if (rows > ctx->max_lm_rows) return SPECVLA_ERR_CAPACITY;
-  return gemm(ctx, A, a_plane, ctx->lm_head, rows, ctx->desc.vocab, ctx->desc.d_model, st, splits, SPECVLA_PROF_LM_HEAD);
+  return gemm(ctx, A, ctx->lm_head, rows, st, plan, SPECVLA_PROF_LM_HEAD);
 }
 
 void argmax_range(const specvla_ctx *ctx, int *lo, int *hi) {
@@ -361,6 +409,7 @@ size_t specvla_workspace_bytes(const specvla_model_desc *desc) {
   if (!desc_ok(desc)) return 0;
   specvla_ctx tmp{};
   tmp.desc = *desc;
+  tmp.num_ctas = MAX_CTAS;
   derive_caps(&tmp);
   return carve(&tmp, nullptr);
 }
@@ -384,6 +433,7 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
   specvla_ctx *ctx = new (std::nothrow) specvla_ctx();
   if (!ctx) return SPECVLA_ERR_INVALID_ARG;
   ctx->desc = *desc;
+  ctx->num_ctas = prop.multiProcessorCount < MAX_CTAS ? prop.multiProcessorCount : MAX_CTAS;
   derive_caps(ctx);
   const size_t need = carve(ctx, nullptr);
   if (workspace_bytes < need) {
@@ -391,25 +441,45 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
     return SPECVLA_ERR_CAPACITY;
   }
   carve(ctx, static_cast<char *>(workspace));
+  const int hd = ctx->hd, D = desc->d_model, F = desc->d_ffn;
+  ctx->use_tc = getenv("SPECVLA_NO_TC") == nullptr;
+  ctx->use_pdl = getenv("SPECVLA_NO_PDL") == nullptr;
+  auto wmat = [&](const void *p, int N, int K) {
+    WMat w{};
+    w.p = static_cast<const bf16 *>(p);
+    w.N = N;
+    w.K = K;
+    w.has_map = ctx->use_tc && p && gemm_tc::make_w_map(&w.map, w.p, N, K);
+    return w;
+  };
+  auto xmaps = [&](XBuf &b) {
+    b.has_map = ctx->use_tc;
+    const int tns[4] = {16, 32, 64, 128};
+    for (int i = 0; i < 4 && b.has_map; i++)
+      b.has_map = gemm_tc::make_x_map(&b.map[i], b.p, b.plane, b.rows, b.K, tns[i]);
+  };
+  xmaps(ctx->xn);
+  xmaps(ctx->xin);
+  xmaps(ctx->ao);
+  xmaps(ctx->hid);
+  xmaps(ctx->lm_in);
   ctx->embed = static_cast<const bf16 *>(tw->embed);
-  ctx->lm_head = static_cast<const bf16 *>(tw->lm_head);
+  ctx->lm_head = wmat(tw->lm_head, desc->vocab, D);
   ctx->final_norm = tw->final_norm;
   ctx->layers.resize(desc->n_layers);
   for (int l = 0; l < desc->n_layers; l++) {
-    ctx->layers[l] = LayerW{static_cast<const bf16 *>(tw->wqkv[l]), static_cast<const bf16 *>(tw->wo[l]),
-                            static_cast<const bf16 *>(tw->wgu[l]), static_cast<const bf16 *>(tw->wd[l]),
-                            tw->norm1[l], tw->norm2[l]};
     if (!tw->wqkv[l] || !tw->wo[l] || !tw->wgu[l] || !tw->wd[l] || !tw->norm1[l] || !tw->norm2[l]) {
       delete ctx;
       return SPECVLA_ERR_INVALID_ARG;
     }
+    ctx->layers[l] = LayerW{wmat(tw->wqkv[l], 3 * hd, D), wmat(tw->wo[l], D, hd), wmat(tw->wgu[l], 2 * F, D),
+                            wmat(tw->wd[l], D, F), tw->norm1[l], tw->norm2[l]};
   }
   ctx->has_draft = dw && dw->fc && dw->wqkv && dw->wo && dw->wgu && dw->wd && dw->norm1 && dw->norm2;
   if (ctx->has_draft) {
-    ctx->draft_fc = static_cast<const bf16 *>(dw->fc);
-    ctx->dlayer = LayerW{static_cast<const bf16 *>(dw->wqkv), static_cast<const bf16 *>(dw->wo),
-                         static_cast<const bf16 *>(dw->wgu), static_cast<const bf16 *>(dw->wd),
-                         dw->norm1, dw->norm2};
+    ctx->draft_fc = wmat(dw->fc, D, 2 * D);
+    ctx->dlayer = LayerW{wmat(dw->wqkv, 3 * hd, D), wmat(dw->wo, D, hd), wmat(dw->wgu, 2 * F, D),
+                         wmat(dw->wd, D, F), dw->norm1, dw->norm2};
   }
   ctx->hP.assign(desc->max_episodes, -1);
   ctx->hPending.assign(desc->max_episodes, 0);
@@ -435,6 +505,7 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
   epi::rope_table_kernel<<<(n + 255) / 256, 256>>>(ctx->rope_tab, desc->max_seq, half, (double)desc->rope_theta);
   cudaMemsetAsync(ctx->st, 0, sizeof(EpState) * desc->max_episodes);
   cudaMemsetAsync(ctx->trees, 0, sizeof(DevTree) * desc->max_episodes);
+  cudaMemsetAsync(ctx->err, 0, 32 * sizeof(int));
   if (cudaDeviceSynchronize() != cudaSuccess) {
     cudaFreeHost(ctx->pinned);
     delete ctx;
@@ -515,12 +586,13 @@ int specvla_prefill(specvla_ctx *ctx, int n_ep, const int *episodes, const void 
   int *h_last = h + 5 * R;
   for (int i = 0; i < n_ep; i++) h_last[i] = ea.aux[i];
   CU(cudaMemcpyAsync(ctx->lm_rows, h_last, n_ep * sizeof(int), cudaMemcpyHostToDevice, st));
-  epi::gather_rows_kernel<<<n_ep, 256, 0, st>>>(ctx->xn, ctx->xn_pl, ctx->lm_rows, d.d_model, ctx->lm_in,
-                                                ctx->lm_pl);
+  epi::gather_rows_kernel<<<n_ep, 256, 0, st>>>(ctx->xn.p, ctx->xn.plane, ctx->lm_rows, d.d_model, ctx->lm_in.p,
+                                                ctx->lm_in.plane);
   LAUNCHED();
-  int s, lo, hi;
+  SegPlan s;
+  int lo, hi;
   argmax_range(ctx, &lo, &hi);
-  TRY(lm_head(ctx, ctx->lm_in, ctx->lm_pl, n_ep, st, &s));
+  TRY(lm_head(ctx, ctx->lm_in, n_ep, st, &s));
   epi::argmax_kernel<<<n_ep, epi::THREADS, 0, st>>>(ctx->part, s, n_ep, d.vocab, lo, hi, ctx->greedy,
                                                     ctx->margin, logits_out);
   LAUNCHED();
@@ -557,7 +629,7 @@ int specvla_prefill(specvla_ctx *ctx, int n_ep, const int *episodes, const void 
       CU(cudaMemcpyAsync(ctx->rt.nvis, h_nvis, db, cudaMemcpyHostToDevice, st));
       CU(cudaMemcpyAsync(ctx->feat_src, h_fs, db, cudaMemcpyHostToDevice, st));
       tree::draft_input_kernel<<<Rd, 256, 0, st>>>(ctx->rt, ctx->feat_src, ctx->feat, emb, ctx->embed,
-                                                   d.d_model, ctx->xin, ctx->xin_pl);
+                                                   d.d_model, ctx->xin.p, ctx->xin.plane);
       LAUNCHED();
       TRY(draft_forward(ctx, Rd, st));
     }
@@ -596,7 +668,8 @@ int specvla_draft_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const sp
     R += ctx->hPending[e];
   }
   if (R > d.max_rows || n_ep * 16 > ctx->max_draft_rows) return SPECVLA_ERR_CAPACITY;
-  int lo, hi, s;
+  int lo, hi;
+  SegPlan s;
   argmax_range(ctx, &lo, &hi);
 
   ctx->phase = 2;
@@ -607,7 +680,7 @@ int specvla_draft_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const sp
   tree::catchup_dst_kernel<<<(n_ep + 63) / 64, 64, 0, st>>>(ea, ctx->dst_row, ctx->lm_rows);
   LAUNCHED();
   tree::draft_input_kernel<<<R, 256, 0, st>>>(ctx->rt, ctx->feat_src, ctx->pend_feat, nullptr, ctx->embed,
-                                              d.d_model, ctx->xin, ctx->xin_pl);
+                                              d.d_model, ctx->xin.p, ctx->xin.plane);
   LAUNCHED();
   TRY(draft_forward(ctx, R, st));
   tree::save_draft_out_kernel<<<R, 256, 0, st>>>(ctx->x, ctx->dst_row, d.d_model, ctx->dout);
@@ -620,16 +693,14 @@ int specvla_draft_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const sp
   int scored_rows = n_ep;            // rows scored by the LM head in the current round
   bool gathered = true;              // round 0 scores the gathered last rows
   for (int l = 0; l < shape->depth; l++) {
-    const bf16 *A = ctx->xn;
-    size_t a_plane = ctx->xn_pl;
+    const XBuf *A = &ctx->xn;
     if (gathered) {
-      epi::gather_rows_kernel<<<n_ep, 256, 0, st>>>(ctx->xn, ctx->xn_pl, ctx->lm_rows, d.d_model, ctx->lm_in,
-                                                    ctx->lm_pl);
+      epi::gather_rows_kernel<<<n_ep, 256, 0, st>>>(ctx->xn.p, ctx->xn.plane, ctx->lm_rows, d.d_model, ctx->lm_in.p,
+                                                    ctx->lm_in.plane);
       LAUNCHED();
-      A = ctx->lm_in;
-      a_plane = ctx->lm_pl;
+      A = &ctx->lm_in;
     }
-    TRY(lm_head(ctx, A, a_plane, scored_rows, st, &s));
+    TRY(lm_head(ctx, *A, scored_rows, st, &s));
     epi::logsoftmax_topk_kernel<<<scored_rows, epi::THREADS, 0, st>>>(
         ctx->part, s, scored_rows, d.vocab, lo, hi, ctx->lgs, ctx->top_tok, ctx->top_lp);
     LAUNCHED();
@@ -647,7 +718,7 @@ int specvla_draft_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const sp
     if (next == 0) break;
     const int Rn = n_ep * next;
     tree::draft_input_kernel<<<Rn, 256, 0, st>>>(ctx->rt, ctx->feat_src, ctx->dout, nullptr, ctx->embed,
-                                                 d.d_model, ctx->xin, ctx->xin_pl);
+                                                 d.d_model, ctx->xin.p, ctx->xin.plane);
     LAUNCHED();
     TRY(draft_forward(ctx, Rn, st));
     tree::save_draft_out_kernel<<<Rn, 256, 0, st>>>(ctx->x, ctx->dst_row, d.d_model, ctx->dout);
@@ -687,9 +758,10 @@ static int verify_device_trees(specvla_ctx *ctx, const EpArgs &ea, int R, int r,
   tree::build_verify_rows_kernel<<<n_ep, 128, 0, st>>>(ea, ctx->trees, ctx->st, ctx->rt);
   LAUNCHED();
   TRY(target_forward(ctx, R, nullptr, st));
-  int s, lo, hi;
+  SegPlan s;
+  int lo, hi;
   argmax_range(ctx, &lo, &hi);
-  TRY(lm_head(ctx, ctx->xn, ctx->xn_pl, R, st, &s));
+  TRY(lm_head(ctx, ctx->xn, R, st, &s));
   epi::argmax_kernel<<<R, epi::THREADS, 0, st>>>(ctx->part, s, R, d.vocab, lo, hi, ctx->greedy, ctx->margin,
                                                  logits_out);
   LAUNCHED();
@@ -912,36 +984,83 @@ int specvla_read_kv(specvla_ctx *ctx, int draft, int episode, int layer, int whi
 }
 
 // ------------------------------------------------------------------ stand-alone GEMM
-__global__ void sum_splits_kernel(const float *__restrict__ part, int splits, size_t n, float *__restrict__ y) {
+__global__ void sum_planes_kernel(const float *__restrict__ part, SegPlan sp, int T, int N, float *__restrict__ y) {
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= n) return;
-  float v = 0.f;
-  for (int s = 0; s < splits; s++) v += part[(size_t)s * n + i];
-  y[i] = v;
+  if (i >= (size_t)T * N) return;
+  const int t = (int)(i / N), n = (int)(i - (size_t)t * N);
+  y[i] = epi::col_sum(part, sp, T, N, t, n);
 }
 
-// scratch layout: [two bf16 limbs of X | split-K partials]
+// scratch layout: [status word, 1 KB | two bf16 limbs of X | planes of partial sums]
 static size_t gemm_limb_bytes(int T, int K) { return ((size_t)2 * T * K * sizeof(bf16) + 1023) / 1024 * 1024; }
+static bool gemm_uses_tc(int T) { return T <= gemm_tc::MAX_T && getenv("SPECVLA_NO_TC") == nullptr; }
+static int gemm_ctas() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+      n = sms < MAX_CTAS ? sms : MAX_CTAS;
+    else
+      return MAX_CTAS;
+  }
+  return n;
+}
+static size_t gemm_planes(int T, int N, int K) {
+  if (gemm_uses_tc(T)) return gemm_tc::max_segments(gemm_tc::make_plan(N, K, gemm_ctas()));
+  return gemm_mma::plan_splits(T, N, K, MAX_SPLITS);
+}
 
 size_t specvla_gemm_scratch_bytes(int T, int N, int K) {
   if (T < 1 || N < 1 || K < 8) return 0;
-  return gemm_limb_bytes(T, K) + (size_t)gemm_mma::plan_splits(T, N, K, MAX_SPLITS) * T * N * sizeof(float);
+  return 1024 + gemm_limb_bytes(T, K) + gemm_planes(T, N, K) * T * N * sizeof(float);
 }
 
 int specvla_gemm(const float *X, const void *W, float *Y, int T, int N, int K, void *scratch,
                  size_t scratch_bytes, void *stream) {
   if (!X || !W || !Y || !scratch || T < 1 || N < 1 || K < 8 || (K % 8)) return SPECVLA_ERR_INVALID_ARG;
-  const int splits = gemm_mma::plan_splits(T, N, K, MAX_SPLITS);
+  if ((reinterpret_cast<uintptr_t>(scratch) % 1024) != 0) return SPECVLA_ERR_INVALID_ARG;
   if (scratch_bytes < specvla_gemm_scratch_bytes(T, N, K)) return SPECVLA_ERR_CAPACITY;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  bf16 *limbs = static_cast<bf16 *>(scratch);
-  float *part = reinterpret_cast<float *>(static_cast<char *>(scratch) + gemm_limb_bytes(T, K));
+  int *err = static_cast<int *>(scratch);
+  bf16 *limbs = reinterpret_cast<bf16 *>(static_cast<char *>(scratch) + 1024);
+  float *part = reinterpret_cast<float *>(static_cast<char *>(scratch) + 1024 + gemm_limb_bytes(T, K));
   const size_t nx = (size_t)T * K, n = (size_t)T * N;
+  if (cudaMemsetAsync(err, 0, sizeof(int), st) != cudaSuccess) return SPECVLA_ERR_CUDA;
   epi::split_limbs_kernel<<<(unsigned)((nx + 255) / 256), 256, 0, st>>>(X, nx, limbs);
-  if (gemm_mma::launch(limbs, nx, static_cast<const bf16 *>(W), part, T, N, K, splits, st) != cudaSuccess)
-    return SPECVLA_ERR_CUDA;
-  sum_splits_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(part, splits, n, Y);
+  SegPlan plan;
+  bool done = false;
+  if (gemm_uses_tc(T)) {
+    CUtensorMap mw, mx;
+    if (gemm_tc::make_w_map(&mw, static_cast<const bf16 *>(W), N, K) &&
+        gemm_tc::make_x_map(&mx, limbs, nx, T, K, gemm_tc::tn_of(T))) {
+      plan = gemm_tc::make_plan(N, K, gemm_ctas());
+      if (gemm_tc::launch(mw, mx, part, T, N, plan, err, st, false) != cudaSuccess) return SPECVLA_ERR_CUDA;
+      done = true;
+    }
+  }
+  if (!done) {
+    // scratch was sized for the tensor-core plan; the split-K plan must fit as well
+    int cap = (int)((scratch_bytes - 1024 - gemm_limb_bytes(T, K)) / (n * sizeof(float)));
+    if (cap < 1) return SPECVLA_ERR_CAPACITY;
+    if (cap > MAX_SPLITS) cap = MAX_SPLITS;
+    const int splits = gemm_mma::plan_splits(T, N, K, cap);
+    if (gemm_mma::launch(limbs, nx, static_cast<const bf16 *>(W), part, T, N, K, splits, st) != cudaSuccess)
+      return SPECVLA_ERR_CUDA;
+    plan = SegPlan{splits, 1, 1, 1};
+  }
+  sum_planes_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(part, plan, T, N, Y);
   return cudaGetLastError() == cudaSuccess ? SPECVLA_OK : SPECVLA_ERR_CUDA;
+}
+
+int specvla_gemm_status(const void *scratch, void *stream) {
+  if (!scratch) return SPECVLA_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int word = 0;
+  if (cudaMemcpyAsync(&word, scratch, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess)
+    return SPECVLA_ERR_CUDA;
+  return word == 0 ? SPECVLA_OK : SPECVLA_ERR_TIMEOUT;
 }
 
 int specvla_profile(specvla_ctx *ctx, int enable) {
