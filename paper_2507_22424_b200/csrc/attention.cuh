@@ -1,90 +1,281 @@
 // Tree-mask attention (Section 3.2 / 4.1: every draft-tree row is verified in one forward,
-// each conditioned on its own path). One CTA per (head, row). Row t attends cache slots
-// [0, nvis[t]) plus the slots tbase[t] + b for every bit b of its 128-bit mask. Queries,
-// keys, values, scores, softmax and the weighted sum are fp32; the output is written as two
-// bf16 limbs for the O-projection GEMM.
+// each conditioned on its own path). Row t attends cache slots [0, nvis[t]) plus the slots
+// tbase[t] + b for every bit b of its 128-bit mask. Queries, keys, values, scores, softmax
+// and the weighted sum are fp32; the output is written as two bf16 limbs for the
+// O-projection GEMM.
 //
-// Each warp walks its share of the keys with an online softmax (running max / sum), lanes
-// split the head dimension; the four warps' partial results are merged in shared memory in
-// warp order, so the result is deterministic.
+// One CTA handles one head, a block of up to 32 consecutive rows of ONE episode and one slice
+// of that block's key range (split-KV). Keys and values go through shared memory in tiles of
+// 32 slots, so a K/V row is read from L2/HBM once per row block instead of once per row; the
+// next tile is fetched into registers while the current one is used. For the scores a lane
+// owns a key and a warp four rows; softmax statistics are reduced across the warp (online
+// softmax, running max / sum); for the weighted sum a lane owns head-dim columns. With several
+// key slices each CTA parks (max, sum, unnormalised output) and bumps a counter; the CTA that
+// arrives last merges the slices in ascending order (deterministic, nobody waits).
 #pragma once
 #include "common.cuh"
 
 namespace attn {
 
-constexpr int WARPS = 4;
+constexpr int RB = 32;            // rows per block
+constexpr int KT = 32;            // key slots per tile
+constexpr int THREADS = 256;      // 8 warps x 4 rows
+constexpr int MAX_SPLITS = 8;
+constexpr int MAX_SPLIT_CTAS = 148;   // CTAs of a launch that uses more than one key slice
+
+struct Args {
+  const float *q;          // [rows][H * DH], already rotated
+  const float *cache;      // [episode][2 (K, V)][max_seq][H * DH]
+  size_t ep_stride;
+  int max_seq, H;
+  RowTable rt;
+  float scale;
+  bf16 *out;               // two limbs, [rows][H * DH] each
+  size_t out_plane;
+  int splits;              // key slices per row block
+  float *part;             // [block * H + head][split][RB][DH + 2] parked slices (splits > 1)
+  int *counters;           // [block * H + head], zero between launches
+};
+
+__host__ __device__ inline int blocks_of(const EpArgs &ea) {
+  int n = 0;
+  for (int i = 0; i < ea.n_ep; i++) n += (ea.nrows[i] + RB - 1) / RB;
+  return n;
+}
+template <int DH> constexpr int smem_bytes() {
+  return (RB * DH + 2 * KT * (DH + 4) + RB * (KT + 1)) * (int)sizeof(float);
+}
 
 template <int DH>
-__global__ void __launch_bounds__(WARPS * 32)
-tree_attention_kernel(const float *__restrict__ q, const float *__restrict__ cache, size_t ep_stride,
-                      int max_seq, int H, RowTable rt, float scale, bf16 *__restrict__ out,
-                      size_t out_plane) {
-  constexpr int PER = DH / 32;           // head-dim elements per lane
-  const int h = blockIdx.x, t = blockIdx.y;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int hd = H * DH;
-  const float *kbase = cache + (size_t)rt.ep[t] * ep_stride + (size_t)h * DH + lane * PER;
-  const float *vbase = kbase + (size_t)max_seq * hd;
-  const int nvis = rt.nvis[t], tbase = rt.tbase[t];
+__global__ void __launch_bounds__(THREADS)
+tree_attention_kernel(const EpArgs ea, const Args a) {
+  constexpr int PER = DH / 32;            // head-dim columns per lane in the weighted sum
+  constexpr int C4 = DH / 4;              // float4 per row
+  constexpr int LD = DH + 4;              // padded K/V row (conflict-free float4 reads by key)
+  constexpr int NLD = KT * C4 / THREADS;  // float4 per thread per tile
+  extern __shared__ __align__(16) float smem[];
+  float *sQ = smem;                       // [RB][DH]
+  float *sK = sQ + RB * DH;               // [KT][LD]
+  float *sV = sK + KT * LD;               // [KT][LD]
+  float *sP = sV + KT * LD;               // [RB][KT + 1]
+  __shared__ int s_nvis[RB], s_tbase[RB], s_kmax;
+  __shared__ uint32_t s_mask[RB][4];
+  __shared__ int s_last;
+  pdl_launch();
+  pdl_wait();
 
-  float qv[PER];
-#pragma unroll
-  for (int i = 0; i < PER; i++)
-    qv[i] = q[(size_t)t * hd + h * DH + lane * PER + i] * scale;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int h = blockIdx.y, hd = a.H * DH;
+  int bid = blockIdx.x / a.splits;
+  const int sp = blockIdx.x - bid * a.splits;
+  const int gblock = bid;
+  int ei = 0;
+  for (; ei < ea.n_ep; ei++) {
+    const int nb = (ea.nrows[ei] + RB - 1) / RB;
+    if (bid < nb) break;
+    bid -= nb;
+  }
+  if (ei >= ea.n_ep) return;
+  const int row0 = ea.row0[ei] + bid * RB;
+  const int nrows = min(RB, ea.nrows[ei] - bid * RB);
+  const float *kbase = a.cache + (size_t)ea.eps[ei] * a.ep_stride + (size_t)h * DH;
+  const float *vbase = kbase + (size_t)a.max_seq * hd;
 
-  float m = -INFINITY, l = 0.f, acc[PER];
+  if (tid < RB) {
+    int nv = 0, tb = 0, km = 0;
+    uint32_t m[4] = {0, 0, 0, 0};
+    if (tid < nrows) {
+      nv = a.rt.nvis[row0 + tid];
+      tb = a.rt.tbase[row0 + tid];
+      km = nv;
 #pragma unroll
-  for (int i = 0; i < PER; i++) acc[i] = 0.f;
+      for (int w = 0; w < 4; w++) {
+        m[w] = a.rt.mask[(size_t)(row0 + tid) * 4 + w];
+        if (m[w]) km = max(km, tb + 32 * w + 32 - __clz(m[w]));
+      }
+    }
+    s_nvis[tid] = nv;
+    s_tbase[tid] = tb;
+#pragma unroll
+    for (int w = 0; w < 4; w++) s_mask[tid][w] = m[w];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) km = max(km, __shfl_xor_sync(0xffffffffu, km, o));
+    if (tid == 0) s_kmax = min(km, a.max_seq);
+  }
+  for (int i = tid; i < RB * C4; i += THREADS) {
+    const int r = i / C4, c = i - r * C4;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (r < nrows) {
+      v = *reinterpret_cast<const float4 *>(a.q + (size_t)(row0 + r) * hd + h * DH + c * 4);
+      v.x *= a.scale; v.y *= a.scale; v.z *= a.scale; v.w *= a.scale;
+    }
+    *reinterpret_cast<float4 *>(sQ + r * DH + c * 4) = v;
+  }
+  __syncthreads();
+  const int kmax = s_kmax;
+  const int tiles = (kmax + KT - 1) / KT;
+  const int t0 = sp * tiles / a.splits, t1 = (sp + 1) * tiles / a.splits;
 
-  auto visit = [&](int slot) {
-    const float *kp = kbase + (size_t)slot * hd;
-    const float *vp = vbase + (size_t)slot * hd;
-    float s = 0.f;
+  float m_run[4], l_run[4], acc[4][PER];
 #pragma unroll
-    for (int i = 0; i < PER; i++) s += qv[i] * kp[i];
-    s = warp_sum(s);
-    const float mn = fmaxf(m, s);
-    const float corr = __expf(m - mn), p = __expf(s - mn);
-    l = l * corr + p;
+  for (int rr = 0; rr < 4; rr++) {
+    m_run[rr] = -INFINITY;
+    l_run[rr] = 0.f;
 #pragma unroll
-    for (int i = 0; i < PER; i++) acc[i] = acc[i] * corr + p * vp[i];
-    m = mn;
-  };
-
-  for (int s = warp; s < nvis; s += WARPS) visit(s);
-  // masked tree slots: warp w takes the w-th 32-bit word
-  uint32_t word = rt.mask[t * 4 + warp];
-  while (word) {
-    int b = __ffs(word) - 1;
-    word &= word - 1;
-    visit(tbase + warp * 32 + b);
+    for (int k = 0; k < PER; k++) acc[rr][k] = 0.f;
   }
 
-  __shared__ float sm[WARPS], sl[WARPS], sacc[WARPS][DH];
-  if (lane == 0) { sm[warp] = m; sl[warp] = l; }
+  float4 kreg[NLD], vreg[NLD];
+  auto fetch = [&](int t) {
 #pragma unroll
-  for (int i = 0; i < PER; i++) sacc[warp][lane * PER + i] = acc[i];
+    for (int k = 0; k < NLD; k++) {
+      const int i = tid + k * THREADS;
+      const int slot = t * KT + i / C4, c = i % C4;
+      if (slot < kmax) {
+        kreg[k] = *reinterpret_cast<const float4 *>(kbase + (size_t)slot * hd + c * 4);
+        vreg[k] = *reinterpret_cast<const float4 *>(vbase + (size_t)slot * hd + c * 4);
+      } else {
+        kreg[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        vreg[k] = kreg[k];
+      }
+    }
+  };
+  if (t0 < t1) fetch(t0);
+  for (int t = t0; t < t1; t++) {
+    __syncthreads();                       // the previous tile is no longer being read
+#pragma unroll
+    for (int k = 0; k < NLD; k++) {
+      const int i = tid + k * THREADS;
+      const int j = i / C4, c = i % C4;
+      *reinterpret_cast<float4 *>(sK + j * LD + c * 4) = kreg[k];
+      *reinterpret_cast<float4 *>(sV + j * LD + c * 4) = vreg[k];
+    }
+    __syncthreads();
+    if (t + 1 < t1) fetch(t + 1);          // in flight while this tile is used
+
+    // scores: lane = key, warp = rows 4w .. 4w + 3
+    float s[4] = {0.f, 0.f, 0.f, 0.f};
+    const float *kr = sK + lane * LD;
+#pragma unroll 8
+    for (int c = 0; c < C4; c++) {
+      const float4 kv = *reinterpret_cast<const float4 *>(kr + c * 4);
+#pragma unroll
+      for (int rr = 0; rr < 4; rr++) {
+        const float4 qv = *reinterpret_cast<const float4 *>(sQ + (warp * 4 + rr) * DH + c * 4);
+        s[rr] += qv.x * kv.x + qv.y * kv.y + qv.z * kv.z + qv.w * kv.w;
+      }
+    }
+    const int slot = t * KT + lane;
+    float corr[4];
+#pragma unroll
+    for (int rr = 0; rr < 4; rr++) {
+      const int r = warp * 4 + rr;
+      bool vis = slot < s_nvis[r];
+      const int b = slot - s_tbase[r];
+      if (!vis && b >= 0 && b < 128) vis = (s_mask[r][b >> 5] >> (b & 31)) & 1u;
+      const float sv = vis ? s[rr] : -INFINITY;
+      const float mn = fmaxf(m_run[rr], warp_max(sv));
+      const float p = vis ? __expf(sv - mn) : 0.f;
+      corr[rr] = (mn == -INFINITY) ? 1.f : __expf(m_run[rr] - mn);
+      l_run[rr] = l_run[rr] * corr[rr] + warp_sum(p);
+      m_run[rr] = mn;
+      sP[r * (KT + 1) + lane] = p;
+    }
+    __syncwarp();
+    // weighted sum: lane = head-dim columns PER * lane .., same four rows
+#pragma unroll
+    for (int rr = 0; rr < 4; rr++)
+#pragma unroll
+      for (int k = 0; k < PER; k++) acc[rr][k] *= corr[rr];
+#pragma unroll 4
+    for (int j = 0; j < KT; j++) {
+      float vv[PER];
+      if (PER == 4) {
+        const float4 t4 = *reinterpret_cast<const float4 *>(sV + j * LD + lane * 4);
+        vv[0] = t4.x; vv[1] = t4.y; vv[2 % PER] = t4.z; vv[3 % PER] = t4.w;
+      } else {
+        const float2 t2 = *reinterpret_cast<const float2 *>(sV + j * LD + lane * 2);
+        vv[0] = t2.x; vv[1] = t2.y;
+      }
+#pragma unroll
+      for (int rr = 0; rr < 4; rr++) {
+        const float p = sP[(warp * 4 + rr) * (KT + 1) + j];
+#pragma unroll
+        for (int k = 0; k < PER; k++) acc[rr][k] += p * vv[k];
+      }
+    }
+    __syncwarp();
+  }
+
+  if (a.splits == 1) {
+#pragma unroll
+    for (int rr = 0; rr < 4; rr++) {
+      const int r = warp * 4 + rr;
+      if (r >= nrows) continue;
+      const float inv = 1.f / l_run[rr];
+#pragma unroll
+      for (int k = 0; k < PER; k++) {
+        const size_t idx = (size_t)(row0 + r) * hd + h * DH + lane * PER + k;
+        const float v = acc[rr][k] * inv;
+        const bf16 hi = __float2bfloat16(v);
+        a.out[idx] = hi;
+        a.out[a.out_plane + idx] = __float2bfloat16(v - __bfloat162float(hi));
+      }
+    }
+    return;
+  }
+
+  // several key slices: park this one, the last arrival merges
+  const int unit = gblock * a.H + h;
+  float *mine = a.part + ((size_t)unit * a.splits + sp) * RB * (DH + 2);
+#pragma unroll
+  for (int rr = 0; rr < 4; rr++) {
+    const int r = warp * 4 + rr;
+    float *dst = mine + (size_t)r * (DH + 2);
+#pragma unroll
+    for (int k = 0; k < PER; k++) __stcg(dst + lane * PER + k, acc[rr][k]);
+    if (lane == 0) {
+      __stcg(dst + DH, m_run[rr]);
+      __stcg(dst + DH + 1, l_run[rr]);
+    }
+  }
+  __threadfence();
   __syncthreads();
-  if (warp == 0) {
-    float M = sm[0];
-    for (int w = 1; w < WARPS; w++) M = fmaxf(M, sm[w]);
+  if (tid == 0) {
+    const int old = atomicAdd(a.counters + unit, 1);
+    s_last = (old == a.splits - 1);
+    if (s_last) atomicExch(a.counters + unit, 0);
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  const float *all = a.part + (size_t)unit * a.splits * RB * (DH + 2);
+#pragma unroll
+  for (int rr = 0; rr < 4; rr++) {
+    const int r = warp * 4 + rr;
+    if (r >= nrows) continue;
+    float M = -INFINITY;
+    for (int s2 = 0; s2 < a.splits; s2++)
+      M = fmaxf(M, __ldcg(all + ((size_t)s2 * RB + r) * (DH + 2) + DH));
     float L = 0.f, o[PER];
 #pragma unroll
-    for (int i = 0; i < PER; i++) o[i] = 0.f;
-    for (int w = 0; w < WARPS; w++) {
-      const float c = (sm[w] == -INFINITY) ? 0.f : __expf(sm[w] - M);
-      L += sl[w] * c;
+    for (int k = 0; k < PER; k++) o[k] = 0.f;
+    for (int s2 = 0; s2 < a.splits; s2++) {
+      const float *src = all + ((size_t)s2 * RB + r) * (DH + 2);
+      const float ms = __ldcg(src + DH);
+      const float c = (ms == -INFINITY) ? 0.f : __expf(ms - M);
+      L += __ldcg(src + DH + 1) * c;
 #pragma unroll
-      for (int i = 0; i < PER; i++) o[i] += sacc[w][lane * PER + i] * c;
+      for (int k = 0; k < PER; k++) o[k] += __ldcg(src + lane * PER + k) * c;
     }
     const float inv = 1.f / L;
 #pragma unroll
-    for (int i = 0; i < PER; i++) {
-      const size_t idx = (size_t)t * hd + h * DH + lane * PER + i;
-      const float v = o[i] * inv;
+    for (int k = 0; k < PER; k++) {
+      const size_t idx = (size_t)(row0 + r) * hd + h * DH + lane * PER + k;
+      const float v = o[k] * inv;
       const bf16 hi = __float2bfloat16(v);
-      out[idx] = hi;
-      out[out_plane + idx] = __float2bfloat16(v - __bfloat162float(hi));
+      a.out[idx] = hi;
+      a.out[a.out_plane + idx] = __float2bfloat16(v - __bfloat162float(hi));
     }
   }
 }

@@ -82,6 +82,12 @@ __host__ __device__ inline int nseg_of(const SegPlan &p, int n) {
   return owner_of(p, f + p.KB - 1) - owner_of(p, f) + 1;
 }
 
+// Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may
+// start while its predecessor still runs; nothing the predecessor wrote may be touched before
+// pdl_wait() returns. pdl_launch() lets the kernel after this one start likewise.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

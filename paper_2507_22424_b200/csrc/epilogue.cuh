@@ -1,9 +1,14 @@
-// Row-wise kernels around the GEMMs: input embedding, split-K reduction fused with
-// RMSNorm / RoPE + KV append / SwiGLU / argmax / log-softmax top-k. All arithmetic is fp32.
-// A value that becomes a GEMM operand is written as two bf16 limbs (hi, lo with hi + lo equal
-// to the fp32 value to 16 mantissa bits), lo limb `plane` elements after the hi limb; queries
-// and cache entries stay fp32. Split-K partials are summed in ascending split order, so
-// results do not depend on scheduling.
+// Row-wise kernels around the GEMMs: input embedding, RoPE + KV append, greedy argmax and
+// log-softmax top-k over finished logits, feature materialisation. All arithmetic is fp32.
+//
+// RMSNorm is split around the GEMMs: the producer of a residual row x writes the GEMM operand
+// limbs(x * gain) and per-row partial sums of squares ssq[row][0..nt); the GEMM that consumes
+// the operand multiplies its output rows by rsqrt(sum(ssq) / d + eps). Kernels here follow the
+// same convention. A value that becomes a GEMM operand is written as two bf16 limbs (hi, lo
+// with hi + lo equal to the fp32 value to 16 mantissa bits), lo limb `plane` elements after hi.
+//
+// Every kernel starts with pdl_launch(); pdl_wait(): it may be launched while its predecessor
+// still runs and touches nothing before the predecessor has finished.
 #pragma once
 #include "common.cuh"
 
@@ -15,15 +20,6 @@ __device__ __forceinline__ void store2(bf16 *hi_plane, size_t plane, size_t idx,
   const bf16 hi = __float2bfloat16(v);
   hi_plane[idx] = hi;
   hi_plane[plane + idx] = __float2bfloat16(v - __bfloat162float(hi));
-}
-
-// Output element (t, n) of a GEMM: its planes added in ascending order.
-__device__ __forceinline__ float col_sum(const float *__restrict__ part, const SegPlan &sp, int T, int N,
-                                         int t, int n) {
-  const int planes = nseg_of(sp, n);
-  float v = 0.f;
-  for (int s = 0; s < planes; s++) v += part[((size_t)s * T + t) * N + n];
-  return v;
 }
 
 __device__ __forceinline__ float block_sum(float v, float *red) {
@@ -41,95 +37,63 @@ __device__ __forceinline__ float block_sum(float v, float *red) {
   return red[0];
 }
 
-// x[t] = input row (embeds[src] or E[tok]); xn[t] = limbs(rmsnorm(x[t]) * gain).
+// RMSNorm scale of a row from its partial sums of squares.
+__device__ __forceinline__ float row_scale(const float *__restrict__ ssq, int nt, size_t row, int d, float eps) {
+  float ss = 0.f;
+  for (int j = 0; j < nt; j++) ss += ssq[row * nt + j];
+  return rsqrtf(ss / d + eps);
+}
+
+// x[t] = input row (embeds[src] or E[tok]); xn[t] = limbs(x[t] * gain); ssq[t] = (sum x^2, 0, ...).
 __global__ void __launch_bounds__(THREADS)
-embed_norm_kernel(RowTable rt, const bf16 *__restrict__ embeds, const bf16 *__restrict__ E,
-                  const float *__restrict__ gain, float eps, int d, float *__restrict__ x,
-                  bf16 *__restrict__ xn, size_t plane) {
+embed_kernel(RowTable rt, const bf16 *__restrict__ embeds, const bf16 *__restrict__ E,
+             const float *__restrict__ gain, int d, int nt, float *__restrict__ x,
+             bf16 *__restrict__ xn, size_t plane, float *__restrict__ ssq) {
   __shared__ float red[32];
+  pdl_launch();
+  pdl_wait();
   const int t = blockIdx.x;
   const int tok = rt.tok[t];
   const bf16 *src = tok >= 0 ? E + (size_t)tok * d : embeds + (size_t)rt.src[t] * d;
   float ss = 0.f;
   for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    float v = __bfloat162float(src[i]);
+    const float v = __bfloat162float(src[i]);
     x[(size_t)t * d + i] = v;
+    store2(xn, plane, (size_t)t * d + i, v * gain[i]);
     ss += v * v;
   }
   ss = block_sum(ss, red);
-  const float rs = rsqrtf(ss / d + eps);
-  for (int i = threadIdx.x; i < d; i += blockDim.x)
-    store2(xn, plane, (size_t)t * d + i, x[(size_t)t * d + i] * rs * gain[i]);
+  for (int j = threadIdx.x; j < nt; j += blockDim.x) ssq[(size_t)t * nt + j] = (j == 0) ? ss : 0.f;
 }
 
-// Residual update + next norm:  x[t] (+)= sum_s part[s][t];  then
-//   gain != NULL: xn[t] = limbs(rmsnorm(x[t]) * gain), feat[t] = rmsnorm(x[t]) * gain (if feat)
-//   gain == NULL: xn[t] = limbs(x[t])
+// Rotates q and k of row t by its position (rotate-half pairs (i, i + dh/2), angle from the
+// precomputed table) and writes q and, into the row's cache slot, k and v, all fp32.
+// qkv [T][3 * H * dh] = [q | k | v]. Cache layout per episode: [2 (K, V)][max_seq][H * dh].
+// grid = (T, ceil(H * dh / 2 / THREADS)).
 __global__ void __launch_bounds__(THREADS)
-residual_norm_kernel(const float *__restrict__ part, SegPlan sp, int T, int d, int accumulate,
-                     const float *__restrict__ gain, float eps, float *__restrict__ x,
-                     bf16 *__restrict__ xn, size_t plane, float *__restrict__ feat) {
-  __shared__ float red[32];
+rope_append_kernel(const float *__restrict__ qkv, int H, int dh, RowTable rt,
+                   const float2 *__restrict__ rope_tab, float *__restrict__ q,
+                   float *__restrict__ cache, size_t ep_stride, int max_seq) {
+  pdl_launch();
+  pdl_wait();
   const int t = blockIdx.x;
-  float ss = 0.f;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    float v = accumulate ? x[(size_t)t * d + i] : 0.f;
-    const int splits = nseg_of(sp, i);
-    for (int s = 0; s < splits; s++) v += part[((size_t)s * T + t) * d + i];
-    x[(size_t)t * d + i] = v;
-    ss += v * v;
-  }
-  if (gain == nullptr) {
-    for (int i = threadIdx.x; i < d; i += blockDim.x)
-      store2(xn, plane, (size_t)t * d + i, x[(size_t)t * d + i]);
-    return;
-  }
-  ss = block_sum(ss, red);
-  const float rs = rsqrtf(ss / d + eps);
-  for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    float v = x[(size_t)t * d + i] * rs * gain[i];
-    store2(xn, plane, (size_t)t * d + i, v);
-    if (feat) feat[(size_t)t * d + i] = v;
-  }
-}
-
-// q, k, v = sum_s part[s][t][...]; rotate q and k by the row's position (rotate-half pairs
-// (i, i + dh/2), angle from the precomputed table); write q and, into the row's cache slot,
-// k and v, all fp32. Cache layout per episode: [2 (K, V)][max_seq][H * dh] fp32.
-__global__ void __launch_bounds__(THREADS)
-qkv_rope_append_kernel(const float *__restrict__ part, SegPlan sp, int T, int H, int dh,
-                       RowTable rt, const float2 *__restrict__ rope_tab, float *__restrict__ q,
-                       float *__restrict__ cache, size_t ep_stride, int max_seq) {
-  const int t = blockIdx.x;
-  const int hd = H * dh, half = dh >> 1, N = 3 * hd;
+  const int hd = H * dh, half = dh >> 1;
+  const int i = blockIdx.y * blockDim.x + threadIdx.x;
+  if (i >= H * half) return;
   const int pos = rt.pos[t], slot = rt.slot[t];
   float *kdst = cache + (size_t)rt.ep[t] * ep_stride + (size_t)slot * hd;
   float *vdst = kdst + (size_t)max_seq * hd;
-  for (int i = threadIdx.x; i < H * half; i += blockDim.x) {
-    const int h = i / half, j = i - h * half;
-    const int c0 = h * dh + j, c1 = c0 + half;
-    const float qlo = col_sum(part, sp, T, N, t, c0), qhi = col_sum(part, sp, T, N, t, c1);
-    const float klo = col_sum(part, sp, T, N, t, hd + c0), khi = col_sum(part, sp, T, N, t, hd + c1);
-    const float vlo = col_sum(part, sp, T, N, t, 2 * hd + c0), vhi = col_sum(part, sp, T, N, t, 2 * hd + c1);
-    const float2 cs = rope_tab[(size_t)pos * half + j];
-    q[(size_t)t * hd + c0] = qlo * cs.x - qhi * cs.y;
-    q[(size_t)t * hd + c1] = qhi * cs.x + qlo * cs.y;
-    kdst[c0] = klo * cs.x - khi * cs.y;
-    kdst[c1] = khi * cs.x + klo * cs.y;
-    vdst[c0] = vlo;
-    vdst[c1] = vhi;
-  }
-}
-
-// hid[t][n] = limbs( silu(g) * u ), g = sum_s part[s][t][n], u = sum_s part[s][t][F + n].
-__global__ void __launch_bounds__(THREADS)
-swiglu_kernel(const float *__restrict__ part, SegPlan sp, int T, int F, bf16 *__restrict__ hid,
-              size_t plane) {
-  const int t = blockIdx.y;
-  const int n = blockIdx.x * blockDim.x + threadIdx.x;
-  if (n >= F) return;
-  const float g = col_sum(part, sp, T, 2 * F, t, n), u = col_sum(part, sp, T, 2 * F, t, F + n);
-  store2(hid, plane, (size_t)t * F + n, g / (1.f + expf(-g)) * u);
+  const float *p = qkv + (size_t)t * 3 * hd;
+  const int h = i / half, j = i - h * half;
+  const int c0 = h * dh + j, c1 = c0 + half;
+  const float2 cs = rope_tab[(size_t)pos * half + j];
+  const float qlo = p[c0], qhi = p[c1], klo = p[hd + c0], khi = p[hd + c1];
+  q[(size_t)t * hd + c0] = qlo * cs.x - qhi * cs.y;
+  q[(size_t)t * hd + c1] = qhi * cs.x + qlo * cs.y;
+  kdst[c0] = klo * cs.x - khi * cs.y;
+  kdst[c1] = khi * cs.x + klo * cs.y;
+  vdst[c0] = p[2 * hd + c0];
+  vdst[c1] = p[2 * hd + c1];
 }
 
 // cos/sin table in double precision: tab[pos][j] = (cos, sin)(pos * theta^(-2j/dh)).
@@ -141,15 +105,32 @@ __global__ void rope_table_kernel(float2 *tab, int max_pos, int half, double the
   tab[i] = make_float2((float)cos(ang), (float)sin(ang));
 }
 
-// dst[i] = row rows[i] of src, both limbs (e.g. the last prefix row of each episode).
+// dst[i] = row rows[i] of src, both limbs, and its sums of squares (e.g. the last prefix row
+// of each episode, for the LM head).
 __global__ void gather_rows_kernel(const bf16 *__restrict__ src, size_t src_plane,
+                                   const float *__restrict__ src_ssq, int nt,
                                    const int *__restrict__ rows, int d, bf16 *__restrict__ dst,
-                                   size_t dst_plane) {
+                                   size_t dst_plane, float *__restrict__ dst_ssq) {
+  pdl_launch();
+  pdl_wait();
   const int r = rows[blockIdx.x];
   for (int i = threadIdx.x; i < d; i += blockDim.x) {
     dst[(size_t)blockIdx.x * d + i] = src[(size_t)r * d + i];
     dst[dst_plane + (size_t)blockIdx.x * d + i] = src[src_plane + (size_t)r * d + i];
   }
+  for (int j = threadIdx.x; j < nt; j += blockDim.x)
+    dst_ssq[(size_t)blockIdx.x * nt + j] = src_ssq[(size_t)r * nt + j];
+}
+
+// feat[t] = x[t] * rsqrt(mean(x[t]^2) + eps) * gain: the final-norm output (the "feature").
+__global__ void features_kernel(const float *__restrict__ x, const float *__restrict__ ssq, int nt,
+                                const float *__restrict__ gain, float eps, int d, float *__restrict__ feat) {
+  pdl_launch();
+  pdl_wait();
+  const int t = blockIdx.x;
+  const float rs = row_scale(ssq, nt, t, d, eps);
+  for (int i = threadIdx.x; i < d; i += blockDim.x)
+    feat[(size_t)t * d + i] = x[(size_t)t * d + i] * rs * gain[i];
 }
 
 // Two-limb split of an fp32 matrix (stand-alone GEMM entry point).
@@ -181,19 +162,20 @@ __device__ __forceinline__ void top2_merge(Top2 &a, const Top2 &b) {
   }
 }
 
-// Greedy token per row: logits = sum_s part[s][t][:]; argmax over [lo, hi) with ties to the
-// lowest id; margin = top-1 minus top-2 over the same range. Optionally dumps the logits.
+// Greedy token per row of logits [T][V]: argmax over [lo, hi) with ties to the lowest id;
+// margin = top-1 minus top-2 over the same range. Optionally copies the whole row out.
 __global__ void __launch_bounds__(THREADS)
-argmax_kernel(const float *__restrict__ part, SegPlan sp, int T, int V, int lo, int hi,
-              int *__restrict__ greedy, float *__restrict__ margin, float *__restrict__ logits_out) {
+argmax_kernel(const float *__restrict__ logits, int V, int lo, int hi, int *__restrict__ greedy,
+              float *__restrict__ margin, float *__restrict__ logits_out) {
   __shared__ Top2 red[THREADS / 32];
+  pdl_launch();
+  pdl_wait();
   const int t = blockIdx.x;
+  const float *row = logits + (size_t)t * V;
   Top2 best{-INFINITY, -INFINITY, 0x7fffffff};
-  for (int v = threadIdx.x; v < V; v += blockDim.x) {
-    const float x = col_sum(part, sp, T, V, t, v);
-    if (logits_out) logits_out[(size_t)t * V + v] = x;
-    if (v >= lo && v < hi) top2_push(best, x, v);
-  }
+  if (logits_out)
+    for (int v = threadIdx.x; v < V; v += blockDim.x) logits_out[(size_t)t * V + v] = row[v];
+  for (int v = lo + threadIdx.x; v < hi; v += blockDim.x) top2_push(best, row[v], v);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
     Top2 other;
@@ -211,24 +193,21 @@ argmax_kernel(const float *__restrict__ part, SegPlan sp, int T, int V, int lo, 
   }
 }
 
-// Draft scoring per row: log-softmax of the logits over [lo, hi) and its top-K entries
+// Draft scoring per row of logits [T][V]: log-softmax over [lo, hi) and its top-K entries
 // (ties to the lowest id), K = SV_TOPK. Selection by K rounds of block argmax.
 __global__ void __launch_bounds__(THREADS)
-logsoftmax_topk_kernel(const float *__restrict__ part, SegPlan sp, int T, int V, int lo, int hi,
-                       float *__restrict__ scratch_logits, int *__restrict__ top_tok,
-                       float *__restrict__ top_lp) {
+logsoftmax_topk_kernel(const float *__restrict__ logits, int V, int lo, int hi,
+                       int *__restrict__ top_tok, float *__restrict__ top_lp) {
   __shared__ float redf[32];
   __shared__ float sv[THREADS / 32];
   __shared__ int si[THREADS / 32];
   __shared__ int chosen[SV_TOPK];
+  pdl_launch();
+  pdl_wait();
   const int t = blockIdx.x;
-  float *lg = scratch_logits + (size_t)t * V;
+  const float *lg = logits + (size_t)t * V;
   float mx = -INFINITY;
-  for (int v = lo + threadIdx.x; v < hi; v += blockDim.x) {
-    const float x = col_sum(part, sp, T, V, t, v);
-    lg[v] = x;
-    mx = fmaxf(mx, x);
-  }
+  for (int v = lo + threadIdx.x; v < hi; v += blockDim.x) mx = fmaxf(mx, lg[v]);
   mx = warp_max(mx);
   if ((threadIdx.x & 31) == 0) sv[threadIdx.x >> 5] = mx;
   __syncthreads();

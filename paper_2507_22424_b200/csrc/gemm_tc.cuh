@@ -11,12 +11,16 @@
 //    activations cost no extra bytes of the weight stream.
 //  * The tiles x K-blocks form one linear list of units (tile-major, K inner) that is cut
 //    into gridDim.x equal contiguous ranges, one per CTA (one CTA per SM). A CTA therefore
-//    covers the end of one tile, some whole tiles and the start of another; every
-//    (CTA, tile) segment writes its partial sum to plane `seg` = CTA - first CTA of that tile,
-//    and the consuming kernel adds the planes in ascending order (deterministic).
+//    covers the end of one tile, some whole tiles and the start of another. A tile covered by
+//    one CTA is finished straight from TMEM. Otherwise every (CTA, tile) segment writes its
+//    partial sum to plane `seg` = CTA - first CTA of that tile and bumps the tile's counter;
+//    the CTA that arrives last adds the planes in ascending order (so the result does not
+//    depend on which CTA that is) and finishes the tile. Nobody waits for anybody.
+//  * "Finishing" a tile is the fused epilogue: plain store with the RMSNorm row scale, or
+//    residual add + gain + two-limb split + sum of squares for the next norm, or SwiGLU.
 //  * Warp 0 issues TMA loads into a ring of stages, warp 1 issues the MMAs and releases
-//    stages through tcgen05.commit, warps 2-5 move finished accumulators (double-buffered in
-//    TMEM) to global memory.
+//    stages through tcgen05.commit, warps 2-5 run the epilogue on finished accumulators
+//    (double-buffered in TMEM).
 //  * The weight loads of the first ring-full do not depend on the previous kernel, so they
 //    are issued BEFORE griddepcontrol.wait: launched with programmatic stream serialisation
 //    the kernel streams weights while its predecessor drains.
@@ -34,22 +38,23 @@ constexpr int BM = SV_TILE_ROWS;          // weight rows per tile (two UMMA halv
 constexpr int BK = 64;                    // K per stage: 128 bytes = one swizzle row
 constexpr int THREADS = 192;
 constexpr int W_STAGE_BYTES = BM * BK * 2;
-constexpr int SMEM_BUDGET = 227 * 1024;
+constexpr int RING_BUDGET = 164 * 1024;
 constexpr int MAX_T = 128;
 
 __host__ __device__ constexpr int tn_of(int T) { return T <= 16 ? 16 : (T <= 32 ? 32 : (T <= 64 ? 64 : 128)); }
 __host__ __device__ constexpr int stage_bytes(int TN) { return W_STAGE_BYTES + 2 * TN * BK * 2; }
-__host__ __device__ constexpr int stages_of(int TN) {
-  return (SMEM_BUDGET - 2048) / stage_bytes(TN) > 8 ? 8 : (SMEM_BUDGET - 2048) / stage_bytes(TN);
-}
+// The ring leaves ~60 KB of the SM's shared memory free, so that the small kernels between two
+// GEMMs can be resident next to a GEMM CTA while it prefetches weights.
+__host__ __device__ constexpr int stages_of(int TN) { return RING_BUDGET / stage_bytes(TN); }
 __host__ __device__ constexpr int smem_bytes(int TN) { return stages_of(TN) * stage_bytes(TN) + 1024 + 256; }
 __host__ __device__ constexpr int tmem_cols(int TN) { return 4 * TN < 32 ? 32 : 4 * TN; }      // 64, 128, 256, 512
 
-inline SegPlan make_plan(int N, int K, int num_sms) {
+// tiles: 256-column tiles of the output (for SwiGLU: 128 gate + 128 up columns each).
+inline SegPlan make_plan(int tiles, int K, int num_sms) {
   SegPlan p;
   p.uniform = 0;
   p.KB = (K + BK - 1) / BK;
-  p.U = ((N + BM - 1) / BM) * p.KB;
+  p.U = tiles * p.KB;
   p.G = p.U < num_sms ? p.U : num_sms;
   return p;
 }
@@ -124,8 +129,9 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm,
       "[%0], [%1, {%2, %3, %4}], [%5], %6;"
       ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(bar), "l"(pol) : "memory");
 }
-__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_wait() { pdl_wait(); }
+__device__ __forceinline__ void grid_dep_launch() { pdl_launch(); }
+__device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 __device__ __forceinline__ void tc_alloc(uint32_t smem_dst, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
@@ -177,10 +183,50 @@ __host__ __device__ constexpr uint32_t instr_desc(int n) {
 #define SV_ERR_WAIT_TMEM_EMPTY 3
 #define SV_ERR_WAIT_TMEM_FULL 4
 
+// What the CTA that finishes a tile does with the summed accumulator v[t][n].
+enum EpiMode {
+  EPI_PLAIN = 0,    // out[row0 + t][n] = scale_t * v
+  EPI_RESID = 1,    // x[row0 + t][n] = (accumulate ? x : 0) + v;  xn = limbs(x * gain[n]);  ssq_out
+  EPI_SWIGLU = 2    // hid[row0 + t][n] = limbs(silu(scale_t * gate) * (scale_t * up))
+};
+
+struct EpiArgs {
+  int mode;
+  int row0;              // first row of this launch within the call's row range
+  int T;                 // rows of this launch (<= 128)
+  int N;                 // output columns (EPI_SWIGLU: F, the width of gate and of up)
+  int up_off;            // EPI_SWIGLU: row of W where the up projection starts (F)
+  float *part;           // planes [max segments][T][tiles * 256] for tiles shared by several CTAs
+  int *counters;         // [tiles] arrivals per shared tile; zero between launches
+  // row scale of the RMSNorm in front of this GEMM: rsqrt(sum_j ssq_in[row][j] * inv_k + eps)
+  const float *ssq_in;   // [rows][nt_in] partial sums of squares; NULL: scale 1
+  int nt_in;
+  float inv_k, eps;
+  // EPI_PLAIN
+  float *out;
+  int ldo;
+  // EPI_RESID
+  float *x;              // [rows][N] residual stream
+  int accumulate;
+  const float *gain;     // [N] gain of the NEXT RMSNorm, folded into xn; NULL: ones
+  bf16 *xn;              // two limbs, [rows][N] each
+  size_t xn_plane;
+  float *ssq_out;        // [rows][tiles]: sum over this tile's columns of x^2
+  // EPI_SWIGLU
+  bf16 *hid;             // two limbs, [rows][N] each
+  size_t hid_plane;
+};
+
+__device__ __forceinline__ void store_limbs(bf16 *hi_plane, size_t plane, size_t idx, float v) {
+  const bf16 hi = __float2bfloat16(v);
+  hi_plane[idx] = hi;
+  hi_plane[plane + idx] = __float2bfloat16(v - __bfloat162float(hi));
+}
+
 template <int TN>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
-               float *__restrict__ part, int T, int N, SegPlan plan, int *__restrict__ err) {
+               const EpiArgs ea, const SegPlan plan, int *__restrict__ err) {
   constexpr int STAGES = stages_of(TN);
   constexpr int STAGE = stage_bytes(TN);
   constexpr uint32_t IDESC = instr_desc(TN);
@@ -192,12 +238,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   auto tfull_bar = [&](int b) { return bars + 8u * (2 * STAGES + b); };
   auto tempty_bar = [&](int b) { return bars + 8u * (2 * STAGES + 2 + b); };
   const uint32_t tmem_slot = bars + 8u * (2 * STAGES + 4);
+  __shared__ float s_scale[MAX_T];        // RMSNorm row scales
+  __shared__ float s_red[4][MAX_T];       // per-warp sums of squares
+  __shared__ int s_flag[4];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long long u0 = (long long)blockIdx.x * plan.U / plan.G;
   const long long u1 = (long long)(blockIdx.x + 1) * plan.U / plan.G;
   const int n_units = (int)(u1 - u0);
   const int KB = plan.KB;
+  const int T = ea.T;
+  const bool swiglu = ea.mode == EPI_SWIGLU;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; s++) {
@@ -227,26 +278,29 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     if (lane == 0 && n_units > 0) {
       const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
       const int npre = n_units < STAGES ? n_units : STAGES;
-      bool ok = true;
-      for (int it = 0; it < n_units && ok; it++) {
+      for (int it = 0; it < n_units; it++) {
         const int st = it % STAGES, rnd = it / STAGES;
         if (rnd > 0 && !mbar_wait(empty_bar(st), (rnd - 1) & 1)) {
           atomicExch(err, SV_ERR_WAIT_EMPTY);
-          ok = false;
           break;
         }
         const long long u = u0 + it;
         const int tile = (int)(u / KB), kb = (int)(u % KB);
         const uint32_t sW = base + st * STAGE;
+        // the two 128-row halves of the tile: consecutive rows, or gate rows + up rows
+        const int ya = swiglu ? tile * 128 : tile * BM;
+        const int yb = swiglu ? ea.up_off + tile * 128 : tile * BM + 128;
         mbar_expect_tx(full_bar(st), STAGE);
-        tma_load_2d(sW, &tmW, kb * BK, tile * BM, full_bar(st), pol_w);
-        if (it >= npre) tma_load_3d(sW + W_STAGE_BYTES, &tmX, kb * BK, 0, 0, full_bar(st), pol_x);
+        tma_load_2d(sW, &tmW, kb * BK, ya, full_bar(st), pol_w);
+        tma_load_2d(sW + 128 * BK * 2, &tmW, kb * BK, yb, full_bar(st), pol_w);
+        if (it >= npre) tma_load_3d(sW + W_STAGE_BYTES, &tmX, kb * BK, ea.row0, 0, full_bar(st), pol_x);
         if (it == npre - 1) {
           // the activations are the previous kernel's output: wait for it only now
           grid_dep_wait();
           for (int j = 0; j < npre; j++) {
             const long long uj = u0 + j;
-            tma_load_3d(base + j * STAGE + W_STAGE_BYTES, &tmX, (int)(uj % KB) * BK, 0, 0, full_bar(j), pol_x);
+            tma_load_3d(base + j * STAGE + W_STAGE_BYTES, &tmX, (int)(uj % KB) * BK, ea.row0, 0, full_bar(j),
+                        pol_x);
           }
         }
       }
@@ -299,6 +353,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     // ------------------------------------------------------------------ epilogue (warps 2..5)
     grid_dep_wait();
     const int q = warp & 3;                       // TMEM lane quarter this warp may access
+    const int et = threadIdx.x - 64;              // 0..127 among the epilogue threads
+    const int tiles = plan.U / KB;
+    const int ldp = tiles * BM;                   // row pitch of a plane
+    if (et < T) {
+      float sc = 1.f;
+      if (ea.ssq_in) {
+        float ss = 0.f;
+        for (int j = 0; j < ea.nt_in; j++) ss += ea.ssq_in[(size_t)(ea.row0 + et) * ea.nt_in + j];
+        sc = rsqrtf(ss * ea.inv_k + ea.eps);
+      }
+      s_scale[et] = sc;
+    }
+    epi_barrier();
+
     int sidx = 0;
     int it = 0;
     while (it < n_units) {
@@ -307,31 +375,161 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       const int tile = (int)(u / KB), kb0 = (int)(u % KB);
       int cnt = KB - kb0;
       if (cnt > n_units - it) cnt = n_units - it;
-      if (!mbar_wait(tfull_bar(buf), (sidx >> 1) & 1)) {
-        if (lane == 0) atomicExch(err, SV_ERR_WAIT_TMEM_FULL);
+      // all four warps take the same decision on the wait
+      const bool mine = mbar_wait(tfull_bar(buf), (sidx >> 1) & 1);
+      if (lane == 0) s_flag[q] = mine ? 1 : 0;
+      epi_barrier();
+      const bool ok = s_flag[0] && s_flag[1] && s_flag[2] && s_flag[3];
+      epi_barrier();
+      if (!ok) {
+        if (et == 0) atomicExch(err, SV_ERR_WAIT_TMEM_FULL);
         break;
       }
       tc_fence_after();
+      const int nseg = nseg_of(plan, tile * BM);
       const int seg = (int)blockIdx.x - owner_of(plan, (long long)tile * KB);
-      float *out = part + (size_t)seg * T * N;
-#pragma unroll
-      for (int h = 0; h < 2; h++) {
-        const int n = tile * BM + h * 128 + q * 32 + lane;
-#pragma unroll
+      // column of this thread inside the tile's plane, and in the output, for the two halves
+      const int pc = tile * BM + q * 32 + lane;                       // plane column of half 0 (+128: half 1)
+      const int na = swiglu ? tile * 128 + q * 32 + lane : pc;       // output column, half 0
+      const int nb = swiglu ? na : pc + 128;                          // output column, half 1
+      const uint32_t tadr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 2 * TN);
+
+      bool finish = true;
+      if (nseg > 1) {
+        // park this segment's partial sums, then see who is last
+        float *pl = ea.part + (size_t)seg * T * ldp;
+#pragma unroll 1
         for (int c0 = 0; c0 < TN; c0 += 16) {
-          uint32_t r[16];
-          tc_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)((buf * 2 + h) * TN + c0), r);
+          uint32_t ra[16], rb[16];
+          tc_ld16(tadr + c0, ra);
+          tc_ld16(tadr + TN + c0, rb);
           tc_wait_ld();
-          if (n < N) {
+#pragma unroll
+          for (int j = 0; j < 16; j++)
+            if (c0 + j < T) {
+              __stcg(pl + (size_t)(c0 + j) * ldp + pc, __uint_as_float(ra[j]));
+              __stcg(pl + (size_t)(c0 + j) * ldp + pc + 128, __uint_as_float(rb[j]));
+            }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty_bar(buf));
+        __threadfence();
+        epi_barrier();
+        if (et == 0) {
+          const int old = atomicAdd(ea.counters + tile, 1);
+          const int lastone = (old == nseg - 1);
+          if (lastone) atomicExch(ea.counters + tile, 0);
+          s_flag[0] = lastone;
+        }
+        epi_barrier();
+        finish = s_flag[0] != 0;
+        epi_barrier();
+        if (finish) __threadfence();
+      }
+
+      if (finish) {
+        float sq[8];                 // EPI_RESID: this thread's sums of squares, 8 rows at a time
+#pragma unroll 1
+        for (int c0 = 0; c0 < TN; c0 += 16) {
+          float va[16], vb[16];
+          if (nseg > 1) {
+            // planes in ascending order; the 32 loads of one plane are independent and in flight
+            // together
+#pragma unroll
+            for (int j = 0; j < 16; j++) va[j] = vb[j] = 0.f;
+#pragma unroll 1
+            for (int s = 0; s < nseg; s++) {
+              const float *pl = ea.part + ((size_t)s * T + c0) * ldp + pc;
+              float ta[16], tb[16];
+#pragma unroll
+              for (int j = 0; j < 16; j++) {
+                const bool in = c0 + j < T;
+                ta[j] = in ? __ldcg(pl + (size_t)j * ldp) : 0.f;
+                tb[j] = in ? __ldcg(pl + (size_t)j * ldp + 128) : 0.f;
+              }
+#pragma unroll
+              for (int j = 0; j < 16; j++) {
+                va[j] += ta[j];
+                vb[j] += tb[j];
+              }
+            }
+          } else {
+            uint32_t ra[16], rb[16];
+            tc_ld16(tadr + c0, ra);
+            tc_ld16(tadr + TN + c0, rb);
+            tc_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 16; j++) {
+              va[j] = __uint_as_float(ra[j]);
+              vb[j] = __uint_as_float(rb[j]);
+            }
+          }
+          if (ea.mode == EPI_PLAIN) {
 #pragma unroll
             for (int j = 0; j < 16; j++)
-              if (c0 + j < T) out[(size_t)(c0 + j) * N + n] = __uint_as_float(r[j]);
+              if (c0 + j < T) {
+                const float sc = s_scale[c0 + j];
+                float *o = ea.out + (size_t)(ea.row0 + c0 + j) * ea.ldo;
+                if (na < ea.N) o[na] = sc * va[j];
+                if (nb < ea.N) o[nb] = sc * vb[j];
+              }
+          } else if (ea.mode == EPI_SWIGLU) {
+#pragma unroll
+            for (int j = 0; j < 16; j++)
+              if (c0 + j < T && na < ea.N) {
+                const float sc = s_scale[c0 + j];
+                const float g = sc * va[j], up = sc * vb[j];
+                store_limbs(ea.hid, ea.hid_plane, (size_t)(ea.row0 + c0 + j) * ea.N + na,
+                            g / (1.f + expf(-g)) * up);
+              }
+          } else {
+            const float ga = (ea.gain && na < ea.N) ? ea.gain[na] : 1.f;
+            const float gb = (ea.gain && nb < ea.N) ? ea.gain[nb] : 1.f;
+#pragma unroll
+            for (int half8 = 0; half8 < 2; half8++) {
+#pragma unroll
+              for (int j8 = 0; j8 < 8; j8++) {
+                const int j = half8 * 8 + j8;
+                float s2 = 0.f;
+                if (c0 + j < T) {
+                  const size_t r = (size_t)(ea.row0 + c0 + j) * ea.N;
+                  if (na < ea.N) {
+                    const float xv = (ea.accumulate ? ea.x[r + na] : 0.f) + va[j];
+                    ea.x[r + na] = xv;
+                    store_limbs(ea.xn, ea.xn_plane, r + na, xv * ga);
+                    s2 += xv * xv;
+                  }
+                  if (nb < ea.N) {
+                    const float xv = (ea.accumulate ? ea.x[r + nb] : 0.f) + vb[j];
+                    ea.x[r + nb] = xv;
+                    store_limbs(ea.xn, ea.xn_plane, r + nb, xv * gb);
+                    s2 += xv * xv;
+                  }
+                }
+                sq[j8] = s2;
+              }
+#pragma unroll
+              for (int j8 = 0; j8 < 8; j8++) {
+                const float w = warp_sum(sq[j8]);
+                if (lane == 0) s_red[q][c0 + half8 * 8 + j8] = w;
+              }
+            }
           }
         }
+        if (nseg == 1) {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(tempty_bar(buf));
+        }
+        if (ea.mode == EPI_RESID) {
+          epi_barrier();
+          if (et < T)
+            ea.ssq_out[(size_t)(ea.row0 + et) * tiles + tile] =
+                s_red[0][et] + s_red[1][et] + s_red[2][et] + s_red[3][et];
+          epi_barrier();
+        }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar(buf));
       sidx++;
       it += cnt;
     }
@@ -366,13 +564,13 @@ inline EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// Weight matrix [N, K] bf16, K contiguous: boxes of 256 rows x 64 columns.
+// Weight matrix [N, K] bf16, K contiguous: boxes of 128 rows x 64 columns.
 inline bool make_w_map(CUtensorMap *tm, const bf16 *W, int N, int K) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)N};
   cuuint64_t strides[1] = {(cuuint64_t)K * 2};
-  cuuint32_t box[2] = {BK, BM};
+  cuuint32_t box[2] = {BK, 128};
   cuuint32_t es[2] = {1, 1};
   return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<bf16 *>(W), dims, strides, box, es,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -393,7 +591,7 @@ inline bool make_x_map(CUtensorMap *tm, const bf16 *X, size_t plane, int rows, i
 }
 
 template <int TN>
-inline cudaError_t launch_tn(const CUtensorMap &tmW, const CUtensorMap &tmX, float *part, int T, int N,
+inline cudaError_t launch_tn(const CUtensorMap &tmW, const CUtensorMap &tmX, const EpiArgs &ea,
                              const SegPlan &plan, int *err, cudaStream_t st, bool pdl) {
   static bool attr_set = false;
   if (!attr_set) {
@@ -412,17 +610,17 @@ inline cudaError_t launch_tn(const CUtensorMap &tmW, const CUtensorMap &tmX, flo
   at[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = pdl ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<TN>, tmW, tmX, part, T, N, plan, err);
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<TN>, tmW, tmX, ea, plan, err);
 }
 
-// tmX must have been made with TN = tn_of(T).
-inline cudaError_t launch(const CUtensorMap &tmW, const CUtensorMap &tmX, float *part, int T, int N,
+// One launch over ea.T <= 128 rows; tmX must have been made with TN = tn_of(ea.T).
+inline cudaError_t launch(const CUtensorMap &tmW, const CUtensorMap &tmX, const EpiArgs &ea,
                           const SegPlan &plan, int *err, cudaStream_t st, bool pdl) {
-  switch (tn_of(T)) {
-    case 16: return launch_tn<16>(tmW, tmX, part, T, N, plan, err, st, pdl);
-    case 32: return launch_tn<32>(tmW, tmX, part, T, N, plan, err, st, pdl);
-    case 64: return launch_tn<64>(tmW, tmX, part, T, N, plan, err, st, pdl);
-    default: return launch_tn<128>(tmW, tmX, part, T, N, plan, err, st, pdl);
+  switch (tn_of(ea.T)) {
+    case 16: return launch_tn<16>(tmW, tmX, ea, plan, err, st, pdl);
+    case 32: return launch_tn<32>(tmW, tmX, ea, plan, err, st, pdl);
+    case 64: return launch_tn<64>(tmW, tmX, ea, plan, err, st, pdl);
+    default: return launch_tn<128>(tmW, tmX, ea, plan, err, st, pdl);
   }
 }
 

@@ -13,7 +13,6 @@
 #include "attention.cuh"
 #include "common.cuh"
 #include "epilogue.cuh"
-#include "gemm_mma.cuh"
 #include "gemm_tc.cuh"
 #include "tree.cuh"
 
@@ -43,7 +42,6 @@ struct LayerW {
 
 constexpr int MAX_CTAS = 148;     // grid of the tensor-core GEMM assumed when sizing the workspace
 
-constexpr int MAX_SPLITS = 8;
 constexpr size_t ALIGN = 1024;
 
 struct Carver {
@@ -70,16 +68,22 @@ struct specvla_ctx {
   WMat lm_head, draft_fc;
   const float *final_norm;
   bool has_draft;
-  int num_ctas;                 // CTAs of the tensor-core GEMM: min(SM count, MAX_CTAS)
-  bool use_tc;                  // tensor-core (tcgen05) GEMM for calls of <= 128 rows
+  int num_ctas;                 // CTAs of the GEMM: min(SM count, MAX_CTAS)
+  int nt;                       // 256-column tiles of a d_model-wide row (sums-of-squares slots)
   bool use_pdl;                 // programmatic dependent launch between the kernels of a forward
 
   // workspace carve-up (device)
   float *kv_t, *kv_d;           // target [ep][layer][2][max_seq][hd], draft [ep][2][max_seq][hd], fp32
   size_t kv_t_ep_stride, kv_t_layer_stride, kv_d_ep_stride;
   float2 *rope_tab;
-  float *x, *feat, *part, *lgs, *pend_feat, *dout, *margin, *top_lp, *q;
+  float *x, *feat, *part, *lgs, *pend_feat, *dout, *margin, *top_lp, *q, *qkv;
+  float *ssq, *lm_ssq;          // per-row partial sums of squares of x / of the gathered LM-head rows
+  int *counters;                // per-tile arrival counters of the GEMM (zero between launches)
+  float *att_part;              // parked key slices of the attention kernel
+  int *att_counters;            // its arrival counters (zero between launches)
   size_t part_floats;
+  int lgs_rows;                 // rows of the logits buffer
+  int n_counters;
   // GEMM operands, two bf16 limbs each: hi plane, then the lo plane `plane` elements later
   XBuf xn, xin, ao, hid, lm_in;
   int *err;                     // device status word written by bounded waits that gave up
@@ -97,6 +101,7 @@ struct specvla_ctx {
   std::vector<int> hP, hPending;  // host mirror of P and n_pending; -1 = not prefilled
   std::vector<int> hTreeRows;     // rows of the device-resident tree left by the last draft call
   int last_rows;                // rows of the last target forward
+  bool feat_valid;              // ctx->feat holds the features of those rows
   long long launches;
   char cuda_err[256];
   cudaEvent_t ev[4];
@@ -123,11 +128,6 @@ namespace {
                __FILE__, __LINE__);                                                     \
       return SPECVLA_ERR_CUDA;                                                          \
     }                                                                                   \
-  } while (0)
-#define LAUNCHED()            \
-  do {                        \
-    ctx->launches++;          \
-    CU(cudaGetLastError());   \
   } while (0)
 #define TRY(expr)             \
   do {                        \
@@ -173,27 +173,34 @@ size_t carve(specvla_ctx *c, char *base) {
   limbs(c->ao, R, hd);
   limbs(c->hid, R, d.d_ffn);
   limbs(c->lm_in, lm_rows, d.d_model);
-  size_t widest = (size_t)3 * hd;
-  if ((size_t)2 * d.d_ffn > widest) widest = (size_t)2 * d.d_ffn;
-  size_t pf = R * widest;                                  // one split over all rows
-  const size_t small_rows = lm_rows < R ? lm_rows : R;
-  if ((size_t)MAX_SPLITS * small_rows * widest > pf) pf = (size_t)MAX_SPLITS * small_rows * widest;
-  if (lm_rows * d.vocab > pf) pf = lm_rows * (size_t)d.vocab;
-  // tensor-core path (calls of <= 128 rows): one plane per (CTA, tile) segment
-  auto tc_need = [&](size_t rows, int N, int K) {
-    if (rows > (size_t)gemm_tc::MAX_T) rows = gemm_tc::MAX_T;
-    const size_t need = (size_t)gemm_tc::max_segments(gemm_tc::make_plan(N, K, c->num_ctas)) * rows * N;
-    if (need > pf) pf = need;
+  c->qkv = cv.take<float>(R * 3 * hd);
+  c->nt = (d.d_model + SV_TILE_ROWS - 1) / SV_TILE_ROWS;
+  c->ssq = cv.take<float>(R * c->nt);
+  c->lm_ssq = cv.take<float>(lm_rows * c->nt);
+  // planes of partial sums for tiles shared by several CTAs: one launch covers <= 128 rows
+  size_t pf = 0;
+  int max_tiles = 1;
+  auto need = [&](int tiles, int K) {
+    const size_t n = (size_t)gemm_tc::max_segments(gemm_tc::make_plan(tiles, K, c->num_ctas)) *
+                     gemm_tc::MAX_T * tiles * SV_TILE_ROWS;
+    if (n > pf) pf = n;
+    if (tiles > max_tiles) max_tiles = tiles;
   };
-  tc_need(R, 3 * hd, d.d_model);
-  tc_need(R, d.d_model, hd);
-  tc_need(R, 2 * d.d_ffn, d.d_model);
-  tc_need(R, d.d_model, d.d_ffn);
-  tc_need(R, d.d_model, 2 * d.d_model);
-  tc_need(lm_rows, d.vocab, d.d_model);
+  auto tiles256 = [](int N) { return (N + SV_TILE_ROWS - 1) / SV_TILE_ROWS; };
+  need(tiles256(3 * hd), d.d_model);
+  need(tiles256(d.d_model), hd);
+  need((d.d_ffn + 127) / 128, d.d_model);
+  need(tiles256(d.d_model), d.d_ffn);
+  need(tiles256(d.d_model), 2 * d.d_model);
+  need(tiles256(d.vocab), d.d_model);
   c->part_floats = pf;
   c->part = cv.take<float>(pf);
-  c->lgs = cv.take<float>(dr * d.vocab);
+  c->att_part = cv.take<float>((size_t)attn::MAX_SPLIT_CTAS * attn::RB * (d.head_dim + 2));
+  c->att_counters = cv.take<int>(attn::MAX_SPLIT_CTAS);
+  c->n_counters = max_tiles;
+  c->counters = cv.take<int>(max_tiles);
+  c->lgs_rows = (int)(lm_rows > dr ? lm_rows : dr);
+  c->lgs = cv.take<float>((size_t)c->lgs_rows * d.vocab);
   c->pend_feat = cv.take<float>(E * SV_MAX_PENDING * d.d_model);
   c->dout = cv.take<float>(E * SV_MAX_TREE * d.d_model);
   c->margin = cv.take<float>(R);
@@ -243,112 +250,173 @@ void prof_collect(specvla_ctx *ctx) {
   ctx->prof_used = 0;
 }
 
-// part <- A[R, K] * W[N, K]^T as planes of partial sums; *plan says how many planes each
-// output column has. Calls of <= 128 rows go to the tensor-core streaming kernel.
-int gemm(specvla_ctx *ctx, const XBuf &A, const WMat &W, int R, cudaStream_t st, SegPlan *plan,
-         int cls) {
-  const int N = W.N, K = W.K;
-  const bool tc = ctx->use_tc && R <= gemm_tc::MAX_T && W.has_map && A.has_map && A.K == K;
+cudaLaunchConfig_t launch_cfg(dim3 grid, dim3 block, cudaStream_t st, cudaLaunchAttribute *attr, bool pdl) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.stream = st;
+  attr->id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr->val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cfg;
+}
+// Launch of a row-wise / tree kernel on the call's stream, allowed to overlap its predecessor.
+#define LAUNCH(kernel, grid, block, ...)                                                       \
+  do {                                                                                         \
+    cudaLaunchAttribute _at;                                                                   \
+    cudaLaunchConfig_t _cfg = launch_cfg(grid, block, st, &_at, ctx->use_pdl);                 \
+    CU(cudaLaunchKernelEx(&_cfg, kernel, __VA_ARGS__));                                        \
+    ctx->launches++;                                                                           \
+  } while (0)
+
+// One GEMM over R rows of A against W with the fused epilogue described by `ea` (mode and
+// outputs; row range, planes and counters are filled in here). Rows go in launches of 128.
+int gemm(specvla_ctx *ctx, const XBuf &A, const WMat &W, int R, gemm_tc::EpiArgs ea, cudaStream_t st, int cls) {
+  if (!W.has_map || !A.has_map || A.K != W.K) return SPECVLA_ERR_BAD_STATE;
+  const bool swiglu = ea.mode == gemm_tc::EPI_SWIGLU;
+  const int tiles = swiglu ? (ea.N + 127) / 128 : (W.N + SV_TILE_ROWS - 1) / SV_TILE_ROWS;
+  const SegPlan plan = gemm_tc::make_plan(tiles, W.K, ctx->num_ctas);
+  if ((size_t)gemm_tc::max_segments(plan) * gemm_tc::MAX_T * tiles * SV_TILE_ROWS > ctx->part_floats)
+    return SPECVLA_ERR_CAPACITY;
+  ea.part = ctx->part;
+  ea.counters = ctx->counters;
+  ea.inv_k = 1.f / (float)W.K;
+  ea.eps = ctx->desc.rms_eps;
   const bool prof = (ctx->prof_mask & ctx->phase) && 2 * (ctx->prof_used + 1) <= (int)ctx->prof_ev.size();
   if (prof) CU(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used], st));
-  if (tc) {
-    *plan = gemm_tc::make_plan(N, K, ctx->num_ctas);
-    if ((size_t)gemm_tc::max_segments(*plan) * R * N > ctx->part_floats) return SPECVLA_ERR_CAPACITY;
-    CU(gemm_tc::launch(W.map, A.map[tn_index(gemm_tc::tn_of(R))], ctx->part, R, N, *plan, ctx->err, st,
-                       ctx->use_pdl));
-  } else {
-    int cap = (int)(ctx->part_floats / ((size_t)R * N));
-    if (cap < 1) return SPECVLA_ERR_CAPACITY;
-    if (cap > MAX_SPLITS) cap = MAX_SPLITS;
-    const int splits = gemm_mma::plan_splits(R, N, K, cap);
-    CU(gemm_mma::launch(A.p, A.plane, W.p, ctx->part, R, N, K, splits, st));
-    *plan = SegPlan{splits, 1, 1, 1};
+  for (int r0 = 0; r0 < R; r0 += gemm_tc::MAX_T) {
+    ea.row0 = r0;
+    ea.T = R - r0 < gemm_tc::MAX_T ? R - r0 : gemm_tc::MAX_T;
+    CU(gemm_tc::launch(W.map, A.map[tn_index(gemm_tc::tn_of(ea.T))], ea, plan, ctx->err, st, ctx->use_pdl));
+    ctx->launches++;
   }
   if (prof) {
     CU(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used + 1], st));
     ctx->prof_cls[ctx->prof_used++] = cls;
-    ctx->prof_bytes[cls] += (double)N * K * sizeof(bf16);
+    ctx->prof_bytes[cls] += (double)W.N * W.K * sizeof(bf16) * ((R + gemm_tc::MAX_T - 1) / gemm_tc::MAX_T);
+  }
+  return SPECVLA_OK;
+}
+
+gemm_tc::EpiArgs epi_plain(float *out, int ldo, int N, const float *ssq_in, int nt_in) {
+  gemm_tc::EpiArgs e = {};
+  e.mode = gemm_tc::EPI_PLAIN;
+  e.N = N;
+  e.out = out;
+  e.ldo = ldo;
+  e.ssq_in = ssq_in;
+  e.nt_in = nt_in;
+  return e;
+}
+// x (+)= result; xn = limbs(x * gain) (gain may be NULL); ssq = per-tile sums of squares of x.
+gemm_tc::EpiArgs epi_resid(specvla_ctx *ctx, int accumulate, const float *gain) {
+  gemm_tc::EpiArgs e = {};
+  e.mode = gemm_tc::EPI_RESID;
+  e.N = ctx->desc.d_model;
+  e.x = ctx->x;
+  e.accumulate = accumulate;
+  e.gain = gain;
+  e.xn = ctx->xn.p;
+  e.xn_plane = ctx->xn.plane;
+  e.ssq_out = ctx->ssq;
+  return e;
+}
+
+// Tree-mask attention over the rows of `rows` (contiguous per episode) against `cache`.
+int attention(specvla_ctx *ctx, const EpArgs &rows, const float *cache, size_t ep_stride, cudaStream_t st) {
+  const specvla_model_desc &d = ctx->desc;
+  attn::Args a = {};
+  a.q = ctx->q;
+  a.cache = cache;
+  a.ep_stride = ep_stride;
+  a.max_seq = d.max_seq;
+  a.H = d.n_heads;
+  a.rt = ctx->rt;
+  a.scale = 1.f / sqrtf((float)d.head_dim);
+  a.out = ctx->ao.p;
+  a.out_plane = ctx->ao.plane;
+  a.part = ctx->att_part;
+  a.counters = ctx->att_counters;
+  const int blocks = attn::blocks_of(rows);
+  if (blocks < 1) return SPECVLA_OK;
+  // few row blocks: slice the key range so that the launch still covers the SMs
+  const int ctas = blocks * d.n_heads;
+  a.splits = 1;
+  if (ctas < 96) {
+    a.splits = attn::MAX_SPLIT_CTAS / ctas;
+    if (a.splits > attn::MAX_SPLITS) a.splits = attn::MAX_SPLITS;
+    if (a.splits < 1) a.splits = 1;
+  }
+  const dim3 grid(blocks * a.splits, d.n_heads);
+  cudaLaunchAttribute at;
+  cudaLaunchConfig_t cfg = launch_cfg(grid, dim3(attn::THREADS), st, &at, ctx->use_pdl);
+  if (d.head_dim == 128) {
+    cfg.dynamicSmemBytes = attn::smem_bytes<128>();
+    CU(cudaLaunchKernelEx(&cfg, attn::tree_attention_kernel<128>, rows, a));
+  } else {
+    cfg.dynamicSmemBytes = attn::smem_bytes<64>();
+    CU(cudaLaunchKernelEx(&cfg, attn::tree_attention_kernel<64>, rows, a));
   }
   ctx->launches++;
   return SPECVLA_OK;
 }
 
-int attention(specvla_ctx *ctx, int R, const float *cache, size_t ep_stride, cudaStream_t st) {
+// One pre-norm decoder layer over R rows. In: x (residual, fp32), xn = limbs(x * norm1 gain) and
+// ssq = sums of squares of x. Out: x updated; xn = limbs(x * next_gain) (limbs(x) when next_gain
+// is NULL) and ssq for the norm that follows.
+int run_layer(specvla_ctx *ctx, const LayerW &w, int R, const EpArgs &rows, float *cache, size_t ep_stride,
+              const float *next_gain, cudaStream_t st) {
   const specvla_model_desc &d = ctx->desc;
-  const float scale = 1.f / sqrtf((float)d.head_dim);
-  dim3 grid(d.n_heads, R);
-  if (d.head_dim == 128)
-    attn::tree_attention_kernel<128><<<grid, attn::WARPS * 32, 0, st>>>(
-        ctx->q, cache, ep_stride, d.max_seq, d.n_heads, ctx->rt, scale, ctx->ao.p, ctx->ao.plane);
-  else
-    attn::tree_attention_kernel<64><<<grid, attn::WARPS * 32, 0, st>>>(
-        ctx->q, cache, ep_stride, d.max_seq, d.n_heads, ctx->rt, scale, ctx->ao.p, ctx->ao.plane);
-  LAUNCHED();
+  const int hd = ctx->hd, F = d.d_ffn;
+  TRY(gemm(ctx, ctx->xn, w.wqkv, R, epi_plain(ctx->qkv, 3 * hd, 3 * hd, ctx->ssq, ctx->nt), st, SPECVLA_PROF_QKV));
+  LAUNCH(epi::rope_append_kernel, dim3(R, (d.n_heads * d.head_dim / 2 + epi::THREADS - 1) / epi::THREADS),
+         dim3(epi::THREADS), (const float *)ctx->qkv, d.n_heads, d.head_dim, ctx->rt,
+         (const float2 *)ctx->rope_tab, ctx->q, cache, ep_stride, d.max_seq);
+  TRY(attention(ctx, rows, cache, ep_stride, st));
+  TRY(gemm(ctx, ctx->ao, w.wo, R, epi_resid(ctx, 1, w.norm2), st, SPECVLA_PROF_O));
+  gemm_tc::EpiArgs sw = {};
+  sw.mode = gemm_tc::EPI_SWIGLU;
+  sw.N = F;
+  sw.up_off = F;
+  sw.ssq_in = ctx->ssq;
+  sw.nt_in = ctx->nt;
+  sw.hid = ctx->hid.p;
+  sw.hid_plane = ctx->hid.plane;
+  TRY(gemm(ctx, ctx->xn, w.wgu, R, sw, st, SPECVLA_PROF_GATE_UP));
+  TRY(gemm(ctx, ctx->hid, w.wd, R, epi_resid(ctx, 1, next_gain), st, SPECVLA_PROF_DOWN));
   return SPECVLA_OK;
 }
 
-// One pre-norm decoder layer over R rows. In: x (residual, fp32) and xn = bf16(norm1(x)).
-// Out: x updated; xn = bf16(rmsnorm(x) * next_gain) (or bf16(x) when next_gain is NULL);
-// feat_out (optional) receives the normalised rows in fp32.
-int run_layer(specvla_ctx *ctx, const LayerW &w, int R, float *cache, size_t ep_stride,
-              const float *next_gain, float *feat_out, cudaStream_t st) {
+// Target model over the R rows described by ctx->rt: embedding, all layers. Leaves the residual
+// in ctx->x, limbs(x * final-norm gain) in ctx->xn and the sums of squares in ctx->ssq: the
+// final RMSNorm itself is applied by whoever consumes them (LM head epilogue, feature readers).
+int target_forward(specvla_ctx *ctx, int R, const EpArgs &rows, const bf16 *embeds, cudaStream_t st) {
   const specvla_model_desc &d = ctx->desc;
-  const int hd = ctx->hd, D = d.d_model, F = d.d_ffn;
-  SegPlan s;
-  TRY(gemm(ctx, ctx->xn, w.wqkv, R, st, &s, SPECVLA_PROF_QKV));
-  epi::qkv_rope_append_kernel<<<R, epi::THREADS, 0, st>>>(ctx->part, s, R, d.n_heads, d.head_dim, ctx->rt,
-                                                          ctx->rope_tab, ctx->q, cache, ep_stride,
-                                                          d.max_seq);
-  LAUNCHED();
-  TRY(attention(ctx, R, cache, ep_stride, st));
-  TRY(gemm(ctx, ctx->ao, w.wo, R, st, &s, SPECVLA_PROF_O));
-  epi::residual_norm_kernel<<<R, epi::THREADS, 0, st>>>(ctx->part, s, R, D, 1, w.norm2, d.rms_eps, ctx->x,
-                                                        ctx->xn.p, ctx->xn.plane, nullptr);
-  LAUNCHED();
-  TRY(gemm(ctx, ctx->xn, w.wgu, R, st, &s, SPECVLA_PROF_GATE_UP));
-  epi::swiglu_kernel<<<dim3((F + epi::THREADS - 1) / epi::THREADS, R), epi::THREADS, 0, st>>>(
-      ctx->part, s, R, F, ctx->hid.p, ctx->hid.plane);
-  LAUNCHED();
-  TRY(gemm(ctx, ctx->hid, w.wd, R, st, &s, SPECVLA_PROF_DOWN));
-  epi::residual_norm_kernel<<<R, epi::THREADS, 0, st>>>(ctx->part, s, R, D, 1, next_gain, d.rms_eps,
-                                                        ctx->x, ctx->xn.p, ctx->xn.plane, feat_out);
-  LAUNCHED();
-  return SPECVLA_OK;
-}
-
-// Target model over the R rows described by ctx->rt: embedding, all layers, final norm.
-// Leaves features in ctx->feat (fp32) and ctx->xn.p (bf16).
-int target_forward(specvla_ctx *ctx, int R, const bf16 *embeds, cudaStream_t st) {
-  const specvla_model_desc &d = ctx->desc;
-  epi::embed_norm_kernel<<<R, epi::THREADS, 0, st>>>(ctx->rt, embeds, ctx->embed, ctx->layers[0].norm1,
-                                                     d.rms_eps, d.d_model, ctx->x, ctx->xn.p, ctx->xn.plane);
-  LAUNCHED();
+  LAUNCH(epi::embed_kernel, dim3(R), dim3(epi::THREADS), ctx->rt, embeds, ctx->embed, ctx->layers[0].norm1,
+         d.d_model, ctx->nt, ctx->x, ctx->xn.p, ctx->xn.plane, ctx->ssq);
   for (int l = 0; l < d.n_layers; l++) {
     const bool last = (l + 1 == d.n_layers);
-    TRY(run_layer(ctx, ctx->layers[l], R, ctx->kv_t + (size_t)l * ctx->kv_t_layer_stride,
-                  ctx->kv_t_ep_stride, last ? ctx->final_norm : ctx->layers[l + 1].norm1,
-                  last ? ctx->feat : nullptr, st));
+    TRY(run_layer(ctx, ctx->layers[l], R, rows, ctx->kv_t + (size_t)l * ctx->kv_t_layer_stride,
+                  ctx->kv_t_ep_stride, last ? ctx->final_norm : ctx->layers[l + 1].norm1, st));
   }
   ctx->last_rows = R;
   return SPECVLA_OK;
 }
 
-// Draft model over R rows: ctx->xin.p = [feature ; embedding] rows are already built.
-// Leaves the layer outputs in ctx->x (fp32) and ctx->xn.p (bf16, un-normalised).
-int draft_forward(specvla_ctx *ctx, int R, cudaStream_t st) {
-  const specvla_model_desc &d = ctx->desc;
-  SegPlan s;
-  TRY(gemm(ctx, ctx->xin, ctx->draft_fc, R, st, &s, SPECVLA_PROF_FC));
-  epi::residual_norm_kernel<<<R, epi::THREADS, 0, st>>>(ctx->part, s, R, d.d_model, 0, ctx->dlayer.norm1,
-                                                        d.rms_eps, ctx->x, ctx->xn.p, ctx->xn.plane, nullptr);
-  LAUNCHED();
-  return run_layer(ctx, ctx->dlayer, R, ctx->kv_d, ctx->kv_d_ep_stride, nullptr, nullptr, st);
+// Draft model over R rows: ctx->xin = [feature ; embedding] rows are already built.
+// Leaves the layer outputs in ctx->x (fp32) and ctx->xn (limbs, un-normalised).
+int draft_forward(specvla_ctx *ctx, int R, const EpArgs &rows, cudaStream_t st) {
+  TRY(gemm(ctx, ctx->xin, ctx->draft_fc, R, epi_resid(ctx, 0, ctx->dlayer.norm1), st, SPECVLA_PROF_FC));
+  return run_layer(ctx, ctx->dlayer, R, rows, ctx->kv_d, ctx->kv_d_ep_stride, nullptr, st);
 }
 
-// LM head over `rows` two-limb rows of A: partial logits land in ctx->part.
-int lm_head(specvla_ctx *ctx, const XBuf &A, int rows, cudaStream_t st, SegPlan *plan) {
-  if (rows > ctx->max_lm_rows) return SPECVLA_ERR_CAPACITY;
-  return gemm(ctx, A, ctx->lm_head, rows, st, plan, SPECVLA_PROF_LM_HEAD);
+// LM head over `rows` two-limb rows of A into ctx->lgs [rows][vocab]. ssq != NULL: the rows
+// are limbs(x * final gain) and get their RMSNorm scale here.
+int lm_head(specvla_ctx *ctx, const XBuf &A, const float *ssq, int rows, cudaStream_t st) {
+  if (rows > ctx->max_lm_rows || rows > ctx->lgs_rows) return SPECVLA_ERR_CAPACITY;
+  return gemm(ctx, A, ctx->lm_head, rows, epi_plain(ctx->lgs, ctx->desc.vocab, ctx->desc.vocab, ssq, ctx->nt),
+              st, SPECVLA_PROF_LM_HEAD);
 }
 
 void argmax_range(const specvla_ctx *ctx, int *lo, int *hi) {
@@ -442,18 +510,17 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
   }
   carve(ctx, static_cast<char *>(workspace));
   const int hd = ctx->hd, D = desc->d_model, F = desc->d_ffn;
-  ctx->use_tc = getenv("SPECVLA_NO_TC") == nullptr;
   ctx->use_pdl = getenv("SPECVLA_NO_PDL") == nullptr;
   auto wmat = [&](const void *p, int N, int K) {
     WMat w{};
     w.p = static_cast<const bf16 *>(p);
     w.N = N;
     w.K = K;
-    w.has_map = ctx->use_tc && p && gemm_tc::make_w_map(&w.map, w.p, N, K);
+    w.has_map = p && gemm_tc::make_w_map(&w.map, w.p, N, K);
     return w;
   };
   auto xmaps = [&](XBuf &b) {
-    b.has_map = ctx->use_tc;
+    b.has_map = true;
     const int tns[4] = {16, 32, 64, 128};
     for (int i = 0; i < 4 && b.has_map; i++)
       b.has_map = gemm_tc::make_x_map(&b.map[i], b.p, b.plane, b.rows, b.K, tns[i]);
@@ -506,6 +573,12 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
   cudaMemsetAsync(ctx->st, 0, sizeof(EpState) * desc->max_episodes);
   cudaMemsetAsync(ctx->trees, 0, sizeof(DevTree) * desc->max_episodes);
   cudaMemsetAsync(ctx->err, 0, 32 * sizeof(int));
+  cudaMemsetAsync(ctx->counters, 0, ctx->n_counters * sizeof(int));
+  cudaMemsetAsync(ctx->att_counters, 0, attn::MAX_SPLIT_CTAS * sizeof(int));
+  cudaFuncSetAttribute(attn::tree_attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                       attn::smem_bytes<128>());
+  cudaFuncSetAttribute(attn::tree_attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                       attn::smem_bytes<64>());
   if (cudaDeviceSynchronize() != cudaSuccess) {
     cudaFreeHost(ctx->pinned);
     delete ctx;
@@ -580,31 +653,36 @@ int specvla_prefill(specvla_ctx *ctx, int n_ep, const int *episodes, const void 
 
   const bf16 *emb = static_cast<const bf16 *>(embeds);
   ctx->phase = 1;
-  TRY(target_forward(ctx, R, emb, st));
+  TRY(target_forward(ctx, R, ea, emb, st));
 
   // first token: LM head on each episode's last row
   int *h_last = h + 5 * R;
   for (int i = 0; i < n_ep; i++) h_last[i] = ea.aux[i];
   CU(cudaMemcpyAsync(ctx->lm_rows, h_last, n_ep * sizeof(int), cudaMemcpyHostToDevice, st));
-  epi::gather_rows_kernel<<<n_ep, 256, 0, st>>>(ctx->xn.p, ctx->xn.plane, ctx->lm_rows, d.d_model, ctx->lm_in.p,
-                                                ctx->lm_in.plane);
-  LAUNCHED();
-  SegPlan s;
+  LAUNCH(epi::gather_rows_kernel, dim3(n_ep), dim3(256), (const bf16 *)ctx->xn.p, ctx->xn.plane,
+         (const float *)ctx->ssq, ctx->nt, (const int *)ctx->lm_rows, d.d_model, ctx->lm_in.p, ctx->lm_in.plane,
+         ctx->lm_ssq);
   int lo, hi;
   argmax_range(ctx, &lo, &hi);
-  TRY(lm_head(ctx, ctx->lm_in, n_ep, st, &s));
-  epi::argmax_kernel<<<n_ep, epi::THREADS, 0, st>>>(ctx->part, s, n_ep, d.vocab, lo, hi, ctx->greedy,
-                                                    ctx->margin, logits_out);
-  LAUNCHED();
-  tree::prefill_commit_kernel<<<n_ep, 256, 0, st>>>(ea, ctx->st, ctx->greedy, ctx->feat, d.d_model,
-                                                    ctx->pend_feat);
-  LAUNCHED();
+  TRY(lm_head(ctx, ctx->lm_in, ctx->lm_ssq, n_ep, st));
+  LAUNCH(epi::argmax_kernel, dim3(n_ep), dim3(epi::THREADS), (const float *)ctx->lgs, d.vocab, lo, hi, ctx->greedy,
+         ctx->margin, logits_out);
+  LAUNCH(tree::prefill_commit_kernel, dim3(n_ep), dim3(256), ea, ctx->st, (const int *)ctx->greedy,
+         (const float *)ctx->x, (const float *)ctx->ssq, ctx->nt, ctx->final_norm, d.rms_eps, d.d_model,
+         ctx->pend_feat);
+  // the features of every prefix row, kept for inspection (the draft pass below reuses x)
+  LAUNCH(epi::features_kernel, dim3(R), dim3(256), (const float *)ctx->x, (const float *)ctx->ssq, ctx->nt,
+         ctx->final_norm, d.rms_eps, d.d_model, ctx->feat);
+  ctx->feat_valid = true;
 
   // draft model over the shifted pairs (feature_i, input_{i+1}), i = 0 .. len-2
   if (ctx->has_draft) {
     int Rd = 0;
     int *h_fs = h + 5 * R + n_ep;          // feature source rows
-    for (int i = 0; i < n_ep; i++)
+    EpArgs ed = ea;
+    for (int i = 0; i < n_ep; i++) {
+      ed.row0[i] = Rd;
+      ed.nrows[i] = lens[i] - 1;
       for (int j = 0; j + 1 < lens[i]; j++) {
         const int r = Rd++;
         const int tr = ea.row0[i] + j;     // target row of f_j; the embedding comes from row tr+1
@@ -615,6 +693,7 @@ int specvla_prefill(specvla_ctx *ctx, int n_ep, const int *episodes, const void 
         h_nvis[r] = j + 1;
         h_fs[r] = tr;
       }
+    }
     if (Rd > 0) {
       const size_t db = (size_t)Rd * sizeof(int);
       // the uploads above are ordered before these on the same stream, but the pinned rows
@@ -628,16 +707,18 @@ int specvla_prefill(specvla_ctx *ctx, int n_ep, const int *episodes, const void 
       CU(cudaMemcpyAsync(ctx->rt.slot, h_pos, db, cudaMemcpyHostToDevice, st));
       CU(cudaMemcpyAsync(ctx->rt.nvis, h_nvis, db, cudaMemcpyHostToDevice, st));
       CU(cudaMemcpyAsync(ctx->feat_src, h_fs, db, cudaMemcpyHostToDevice, st));
-      tree::draft_input_kernel<<<Rd, 256, 0, st>>>(ctx->rt, ctx->feat_src, ctx->feat, emb, ctx->embed,
-                                                   d.d_model, ctx->xin.p, ctx->xin.plane);
-      LAUNCHED();
-      TRY(draft_forward(ctx, Rd, st));
+      LAUNCH(tree::draft_input_kernel, dim3(Rd), dim3(256), ctx->rt, (const int *)ctx->feat_src,
+             (const float *)ctx->feat, (const float *)nullptr, 0, (const float *)nullptr, 0.f, emb, ctx->embed,
+             d.d_model, ctx->xin.p, ctx->xin.plane);
+      TRY(draft_forward(ctx, Rd, ed, st));
     }
   }
   int *h_g = ctx->pin_small;
   CU(cudaMemcpyAsync(h_g, ctx->greedy, n_ep * sizeof(int), cudaMemcpyDeviceToHost, st));
+  CU(cudaMemcpyAsync(h_g + 4000, ctx->err, sizeof(int), cudaMemcpyDeviceToHost, st));
   CU(cudaStreamSynchronize(st));
   prof_collect(ctx);
+  if (h_g[4000] != 0) return SPECVLA_ERR_TIMEOUT;
   for (int i = 0; i < n_ep; i++) {
     ctx->hP[episodes[i]] = lens[i];
     ctx->hPending[episodes[i]] = 1;
@@ -669,22 +750,22 @@ int specvla_draft_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const sp
   }
   if (R > d.max_rows || n_ep * 16 > ctx->max_draft_rows) return SPECVLA_ERR_CAPACITY;
   int lo, hi;
-  SegPlan s;
   argmax_range(ctx, &lo, &hi);
 
   ctx->phase = 2;
   // catch-up over the pending rows; the last row of each episode scores the root's children
-  tree::build_catchup_rows_kernel<<<(n_ep + 63) / 64, 64, 0, st>>>(ea, ctx->st, ctx->trees, ctx->rt,
-                                                                   ctx->feat_src);
-  LAUNCHED();
-  tree::catchup_dst_kernel<<<(n_ep + 63) / 64, 64, 0, st>>>(ea, ctx->dst_row, ctx->lm_rows);
-  LAUNCHED();
-  tree::draft_input_kernel<<<R, 256, 0, st>>>(ctx->rt, ctx->feat_src, ctx->pend_feat, nullptr, ctx->embed,
-                                              d.d_model, ctx->xin.p, ctx->xin.plane);
-  LAUNCHED();
-  TRY(draft_forward(ctx, R, st));
-  tree::save_draft_out_kernel<<<R, 256, 0, st>>>(ctx->x, ctx->dst_row, d.d_model, ctx->dout);
-  LAUNCHED();
+  const bf16 *no_embeds = nullptr;
+  const float *no_f = nullptr;
+  LAUNCH(tree::build_catchup_rows_kernel, dim3((n_ep + 63) / 64), dim3(64), ea, ctx->st, ctx->trees, ctx->rt,
+         ctx->feat_src);
+  LAUNCH(tree::catchup_dst_kernel, dim3((n_ep + 63) / 64), dim3(64), ea, ctx->dst_row, ctx->lm_rows);
+  LAUNCH(tree::draft_input_kernel, dim3(R), dim3(256), ctx->rt, (const int *)ctx->feat_src,
+         (const float *)ctx->pend_feat, no_f, 0, no_f, 0.f, no_embeds, ctx->embed, d.d_model, ctx->xin.p,
+         ctx->xin.plane);
+  TRY(draft_forward(ctx, R, ea, st));
+  LAUNCH(tree::save_draft_out_kernel, dim3(R), dim3(256), (const float *)ctx->x, (const int *)ctx->dst_row,
+         d.d_model, ctx->dout);
+  ctx->feat_valid = false;
   for (int i = 0; i < n_ep; i++) {
     ctx->hPending[episodes[i]] = 0;
     ctx->hTreeRows[episodes[i]] = 1 + n_nodes;
@@ -695,15 +776,15 @@ int specvla_draft_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const sp
   for (int l = 0; l < shape->depth; l++) {
     const XBuf *A = &ctx->xn;
     if (gathered) {
-      epi::gather_rows_kernel<<<n_ep, 256, 0, st>>>(ctx->xn.p, ctx->xn.plane, ctx->lm_rows, d.d_model, ctx->lm_in.p,
-                                                    ctx->lm_in.plane);
-      LAUNCHED();
+      LAUNCH(epi::gather_rows_kernel, dim3(n_ep), dim3(256), (const bf16 *)ctx->xn.p, ctx->xn.plane,
+             (const float *)ctx->ssq, ctx->nt, (const int *)ctx->lm_rows, d.d_model, ctx->lm_in.p,
+             ctx->lm_in.plane, ctx->lm_ssq);
       A = &ctx->lm_in;
     }
-    TRY(lm_head(ctx, *A, scored_rows, st, &s));
-    epi::logsoftmax_topk_kernel<<<scored_rows, epi::THREADS, 0, st>>>(
-        ctx->part, s, scored_rows, d.vocab, lo, hi, ctx->lgs, ctx->top_tok, ctx->top_lp);
-    LAUNCHED();
+    // the draft layer's output feeds the shared LM head as it is: no norm, no row scale
+    TRY(lm_head(ctx, *A, nullptr, scored_rows, st));
+    LAUNCH(epi::logsoftmax_topk_kernel, dim3(scored_rows), dim3(epi::THREADS), (const float *)ctx->lgs, d.vocab,
+           lo, hi, ctx->top_tok, ctx->top_lp);
     const int cur = (l == 0) ? 1 : shape->expand[l];            // parents scored per episode
     const int next = (l + 1 < shape->depth) ? shape->expand[l + 1] : 0;
     EpArgs la = ea;
@@ -711,18 +792,22 @@ int specvla_draft_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const sp
       la.row0[i] = i * cur;
       la.aux[i] = i * next;
     }
-    tree::expand_level_kernel<<<(n_ep + 63) / 64, 64, 0, st>>>(la, l, shape->branch[l], next, ctx->top_tok,
-                                                               ctx->top_lp, ctx->trees, ctx->st, ctx->rt,
-                                                               ctx->feat_src, ctx->dst_row);
-    LAUNCHED();
+    LAUNCH(tree::expand_level_kernel, dim3((n_ep + 63) / 64), dim3(64), la, l, shape->branch[l], next,
+           (const int *)ctx->top_tok, (const float *)ctx->top_lp, ctx->trees, (const EpState *)ctx->st, ctx->rt,
+           ctx->feat_src, ctx->dst_row);
     if (next == 0) break;
     const int Rn = n_ep * next;
-    tree::draft_input_kernel<<<Rn, 256, 0, st>>>(ctx->rt, ctx->feat_src, ctx->dout, nullptr, ctx->embed,
-                                                 d.d_model, ctx->xin.p, ctx->xin.plane);
-    LAUNCHED();
-    TRY(draft_forward(ctx, Rn, st));
-    tree::save_draft_out_kernel<<<Rn, 256, 0, st>>>(ctx->x, ctx->dst_row, d.d_model, ctx->dout);
-    LAUNCHED();
+    LAUNCH(tree::draft_input_kernel, dim3(Rn), dim3(256), ctx->rt, (const int *)ctx->feat_src,
+           (const float *)ctx->dout, no_f, 0, no_f, 0.f, no_embeds, ctx->embed, d.d_model, ctx->xin.p,
+           ctx->xin.plane);
+    EpArgs ln = ea;
+    for (int i = 0; i < n_ep; i++) {
+      ln.row0[i] = i * next;
+      ln.nrows[i] = next;
+    }
+    TRY(draft_forward(ctx, Rn, ln, st));
+    LAUNCH(tree::save_draft_out_kernel, dim3(Rn), dim3(256), (const float *)ctx->x, (const int *)ctx->dst_row,
+           d.d_model, ctx->dout);
     scored_rows = Rn;
     gathered = false;
   }
@@ -755,26 +840,21 @@ static int verify_device_trees(specvla_ctx *ctx, const EpArgs &ea, int R, int r,
   const specvla_model_desc &d = ctx->desc;
   const int n_ep = ea.n_ep;
   ctx->phase = 4;
-  tree::build_verify_rows_kernel<<<n_ep, 128, 0, st>>>(ea, ctx->trees, ctx->st, ctx->rt);
-  LAUNCHED();
-  TRY(target_forward(ctx, R, nullptr, st));
-  SegPlan s;
+  LAUNCH(tree::build_verify_rows_kernel, dim3(n_ep), dim3(128), ea, ctx->trees, (const EpState *)ctx->st, ctx->rt);
+  TRY(target_forward(ctx, R, ea, nullptr, st));
+  ctx->feat_valid = false;
   int lo, hi;
   argmax_range(ctx, &lo, &hi);
-  TRY(lm_head(ctx, ctx->xn, R, st, &s));
-  epi::argmax_kernel<<<R, epi::THREADS, 0, st>>>(ctx->part, s, R, d.vocab, lo, hi, ctx->greedy, ctx->margin,
-                                                 logits_out);
-  LAUNCHED();
-  tree::accept_select_kernel<<<n_ep, 128, 0, st>>>(ea, ctx->trees, ctx->st, ctx->greedy, r, d.action_base,
-                                                   d.n_bins, ctx->feat, d.d_model, ctx->pend_feat,
-                                                   ctx->out_m, ctx->out_tok, ctx->out_path);
-  LAUNCHED();
-  tree::kv_compact_kernel<<<dim3(d.n_layers * 2, n_ep), 256, 0, st>>>(
-      ea, ctx->st, ctx->out_m, ctx->out_path, ctx->kv_t, ctx->kv_t_ep_stride, ctx->kv_t_layer_stride,
-      d.max_seq, ctx->hd);
-  LAUNCHED();
-  tree::advance_state_kernel<<<(n_ep + 63) / 64, 64, 0, st>>>(ea, ctx->st, ctx->out_m);
-  LAUNCHED();
+  TRY(lm_head(ctx, ctx->xn, ctx->ssq, R, st));
+  LAUNCH(epi::argmax_kernel, dim3(R), dim3(epi::THREADS), (const float *)ctx->lgs, d.vocab, lo, hi, ctx->greedy,
+         ctx->margin, logits_out);
+  LAUNCH(tree::accept_select_kernel, dim3(n_ep), dim3(128), ea, ctx->trees, ctx->st, (const int *)ctx->greedy, r,
+         d.action_base, d.n_bins, (const float *)ctx->x, (const float *)ctx->ssq, ctx->nt, ctx->final_norm,
+         d.rms_eps, d.d_model, ctx->pend_feat, ctx->out_m, ctx->out_tok, ctx->out_path);
+  LAUNCH(tree::kv_compact_kernel, dim3(d.n_layers * 2, n_ep), dim3(256), ea, (const EpState *)ctx->st,
+         (const int *)ctx->out_m, (const int *)ctx->out_path, ctx->kv_t, ctx->kv_t_ep_stride,
+         ctx->kv_t_layer_stride, d.max_seq, ctx->hd);
+  LAUNCH(tree::advance_state_kernel, dim3((n_ep + 63) / 64), dim3(64), ea, ctx->st, (const int *)ctx->out_m);
   return SPECVLA_OK;
 }
 
@@ -785,8 +865,10 @@ static int finish_verify(specvla_ctx *ctx, const EpArgs &ea, int *accept_len_out
   int *h = ctx->pin_small;
   CU(cudaMemcpyAsync(h, ctx->out_m, n_ep * sizeof(int), cudaMemcpyDeviceToHost, st));
   CU(cudaMemcpyAsync(h + SV_MAX_EP, ctx->out_tok, n_ep * W * sizeof(int), cudaMemcpyDeviceToHost, st));
+  CU(cudaMemcpyAsync(h + 4000, ctx->err, sizeof(int), cudaMemcpyDeviceToHost, st));
   CU(cudaStreamSynchronize(st));
   prof_collect(ctx);
+  if (h[4000] != 0) return SPECVLA_ERR_TIMEOUT;
   for (int i = 0; i < n_ep; i++) {
     const int e = ea.eps[i], m = h[i];
     if (m < 0 || m > SV_MAX_DEPTH) return SPECVLA_ERR_BAD_STATE;
@@ -945,7 +1027,19 @@ int specvla_read_buffer(specvla_ctx *ctx, int what, void *host_dst, size_t bytes
   switch (what) {
     case SPECVLA_BUF_GREEDY: src = ctx->greedy; avail = (size_t)d.max_rows * sizeof(int); break;
     case SPECVLA_BUF_MARGIN: src = ctx->margin; avail = (size_t)d.max_rows * sizeof(float); break;
-    case SPECVLA_BUF_FEATURES: src = ctx->feat; avail = (size_t)d.max_rows * d.d_model * sizeof(float); break;
+    case SPECVLA_BUF_FEATURES: {
+      // after a verification the features exist only as residual + sums of squares
+      if (!ctx->feat_valid) {
+        if (ctx->last_rows < 1) return SPECVLA_ERR_BAD_STATE;
+        cudaStream_t st = static_cast<cudaStream_t>(stream);
+        LAUNCH(epi::features_kernel, dim3(ctx->last_rows), dim3(256), (const float *)ctx->x,
+               (const float *)ctx->ssq, ctx->nt, ctx->final_norm, d.rms_eps, d.d_model, ctx->feat);
+        ctx->feat_valid = true;
+      }
+      src = ctx->feat;
+      avail = (size_t)d.max_rows * d.d_model * sizeof(float);
+      break;
+    }
     case SPECVLA_BUF_PATH: src = ctx->out_path; avail = (size_t)d.max_episodes * (SV_MAX_DEPTH + 1) * sizeof(int); break;
     case SPECVLA_BUF_DRAFT_TOPK_TOK: src = ctx->top_tok; avail = (size_t)ctx->max_draft_rows * SV_TOPK * sizeof(int); break;
     case SPECVLA_BUF_DRAFT_TOPK_LP: src = ctx->top_lp; avail = (size_t)ctx->max_draft_rows * SV_TOPK * sizeof(float); break;
@@ -984,16 +1078,9 @@ int specvla_read_kv(specvla_ctx *ctx, int draft, int episode, int layer, int whi
 }
 
 // ------------------------------------------------------------------ stand-alone GEMM
-__global__ void sum_planes_kernel(const float *__restrict__ part, SegPlan sp, int T, int N, float *__restrict__ y) {
-  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= (size_t)T * N) return;
-  const int t = (int)(i / N), n = (int)(i - (size_t)t * N);
-  y[i] = epi::col_sum(part, sp, T, N, t, n);
-}
-
-// scratch layout: [status word, 1 KB | two bf16 limbs of X | planes of partial sums]
+// scratch layout: [status word, 1 KB | tile counters, 4 KB | two bf16 limbs of X | planes]
+static const size_t GEMM_HDR = 1024 + 4096;
 static size_t gemm_limb_bytes(int T, int K) { return ((size_t)2 * T * K * sizeof(bf16) + 1023) / 1024 * 1024; }
-static bool gemm_uses_tc(int T) { return T <= gemm_tc::MAX_T && getenv("SPECVLA_NO_TC") == nullptr; }
 static int gemm_ctas() {
   static int n = 0;
   if (!n) {
@@ -1006,50 +1093,51 @@ static int gemm_ctas() {
   }
   return n;
 }
-static size_t gemm_planes(int T, int N, int K) {
-  if (gemm_uses_tc(T)) return gemm_tc::max_segments(gemm_tc::make_plan(N, K, gemm_ctas()));
-  return gemm_mma::plan_splits(T, N, K, MAX_SPLITS);
+static size_t gemm_plane_floats(int T, int N, int K) {
+  const int tiles = (N + SV_TILE_ROWS - 1) / SV_TILE_ROWS;
+  const int rows = T < gemm_tc::MAX_T ? T : gemm_tc::MAX_T;
+  return (size_t)gemm_tc::max_segments(gemm_tc::make_plan(tiles, K, gemm_ctas())) * rows * tiles * SV_TILE_ROWS;
 }
 
 size_t specvla_gemm_scratch_bytes(int T, int N, int K) {
-  if (T < 1 || N < 1 || K < 8) return 0;
-  return 1024 + gemm_limb_bytes(T, K) + gemm_planes(T, N, K) * T * N * sizeof(float);
+  if (T < 1 || N < 1 || K < 8 || N > 1024 * SV_TILE_ROWS) return 0;
+  return GEMM_HDR + gemm_limb_bytes(T, K) + gemm_plane_floats(T, N, K) * sizeof(float);
 }
 
 int specvla_gemm(const float *X, const void *W, float *Y, int T, int N, int K, void *scratch,
                  size_t scratch_bytes, void *stream) {
-  if (!X || !W || !Y || !scratch || T < 1 || N < 1 || K < 8 || (K % 8)) return SPECVLA_ERR_INVALID_ARG;
+  if (!X || !W || !Y || !scratch || T < 1 || N < 1 || K < 8 || (K % 8) || N > 1024 * SV_TILE_ROWS)
+    return SPECVLA_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(scratch) % 1024) != 0) return SPECVLA_ERR_INVALID_ARG;
   if (scratch_bytes < specvla_gemm_scratch_bytes(T, N, K)) return SPECVLA_ERR_CAPACITY;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  int *err = static_cast<int *>(scratch);
-  bf16 *limbs = reinterpret_cast<bf16 *>(static_cast<char *>(scratch) + 1024);
-  float *part = reinterpret_cast<float *>(static_cast<char *>(scratch) + 1024 + gemm_limb_bytes(T, K));
-  const size_t nx = (size_t)T * K, n = (size_t)T * N;
-  if (cudaMemsetAsync(err, 0, sizeof(int), st) != cudaSuccess) return SPECVLA_ERR_CUDA;
+  char *base = static_cast<char *>(scratch);
+  int *err = reinterpret_cast<int *>(base);
+  bf16 *limbs = reinterpret_cast<bf16 *>(base + GEMM_HDR);
+  const size_t nx = (size_t)T * K;
+  // status word and tile counters start at zero
+  if (cudaMemsetAsync(base, 0, GEMM_HDR, st) != cudaSuccess) return SPECVLA_ERR_CUDA;
   epi::split_limbs_kernel<<<(unsigned)((nx + 255) / 256), 256, 0, st>>>(X, nx, limbs);
-  SegPlan plan;
-  bool done = false;
-  if (gemm_uses_tc(T)) {
-    CUtensorMap mw, mx;
-    if (gemm_tc::make_w_map(&mw, static_cast<const bf16 *>(W), N, K) &&
-        gemm_tc::make_x_map(&mx, limbs, nx, T, K, gemm_tc::tn_of(T))) {
-      plan = gemm_tc::make_plan(N, K, gemm_ctas());
-      if (gemm_tc::launch(mw, mx, part, T, N, plan, err, st, false) != cudaSuccess) return SPECVLA_ERR_CUDA;
-      done = true;
-    }
-  }
-  if (!done) {
-    // scratch was sized for the tensor-core plan; the split-K plan must fit as well
-    int cap = (int)((scratch_bytes - 1024 - gemm_limb_bytes(T, K)) / (n * sizeof(float)));
-    if (cap < 1) return SPECVLA_ERR_CAPACITY;
-    if (cap > MAX_SPLITS) cap = MAX_SPLITS;
-    const int splits = gemm_mma::plan_splits(T, N, K, cap);
-    if (gemm_mma::launch(limbs, nx, static_cast<const bf16 *>(W), part, T, N, K, splits, st) != cudaSuccess)
+  CUtensorMap mw, mx[4];
+  if (!gemm_tc::make_w_map(&mw, static_cast<const bf16 *>(W), N, K)) return SPECVLA_ERR_CUDA;
+  const int tns[4] = {16, 32, 64, 128};
+  for (int i = 0; i < 4; i++)
+    if (!gemm_tc::make_x_map(&mx[i], limbs, nx, T, K, tns[i])) return SPECVLA_ERR_CUDA;
+  const int tiles = (N + SV_TILE_ROWS - 1) / SV_TILE_ROWS;
+  const SegPlan plan = gemm_tc::make_plan(tiles, K, gemm_ctas());
+  gemm_tc::EpiArgs ea = {};
+  ea.mode = gemm_tc::EPI_PLAIN;
+  ea.N = N;
+  ea.out = Y;
+  ea.ldo = N;
+  ea.part = reinterpret_cast<float *>(base + GEMM_HDR + gemm_limb_bytes(T, K));
+  ea.counters = reinterpret_cast<int *>(base + 1024);
+  for (int r0 = 0; r0 < T; r0 += gemm_tc::MAX_T) {
+    ea.row0 = r0;
+    ea.T = T - r0 < gemm_tc::MAX_T ? T - r0 : gemm_tc::MAX_T;
+    if (gemm_tc::launch(mw, mx[tn_index(gemm_tc::tn_of(ea.T))], ea, plan, err, st, false) != cudaSuccess)
       return SPECVLA_ERR_CUDA;
-    plan = SegPlan{splits, 1, 1, 1};
   }
-  sum_planes_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(part, plan, T, N, Y);
   return cudaGetLastError() == cudaSuccess ? SPECVLA_OK : SPECVLA_ERR_CUDA;
 }
 

@@ -12,6 +12,8 @@ namespace tree {
 // caller-supplied trees need only tok / parent / depth. One CTA per episode.
 __global__ void build_verify_rows_kernel(EpArgs a, DevTree *trees, const EpState *__restrict__ st,
                                          RowTable rt) {
+  pdl_launch();
+  pdl_wait();
   const int e = a.eps[blockIdx.x];
   DevTree &tr = trees[e];
   const int P = st[e].P;
@@ -38,6 +40,8 @@ __global__ void build_verify_rows_kernel(EpArgs a, DevTree *trees, const EpState
 // root is the episode's last emitted token. One thread per episode.
 __global__ void build_catchup_rows_kernel(EpArgs a, EpState *st, DevTree *trees, RowTable rt,
                                           int *__restrict__ feat_src) {
+  pdl_launch();
+  pdl_wait();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= a.n_ep) return;
   const int e = a.eps[i];
@@ -70,19 +74,34 @@ __global__ void build_catchup_rows_kernel(EpArgs a, EpState *st, DevTree *trees,
   tr.sel[0] = 0;
 }
 
+// RMSNorm scale of a residual row from its partial sums of squares ssq[row][0..nt).
+__device__ __forceinline__ float norm_scale(const float *__restrict__ ssq, int nt, size_t row, int d, float eps) {
+  float ss = 0.f;
+  for (int j = 0; j < nt; j++) ss += ssq[row * nt + j];
+  return rsqrtf(ss / d + eps);
+}
+
 // Draft-model input rows: xin[r] = limbs([feature ; embedding]) with the feature taken from
 // row feat_src[r] of `feat` and the embedding from E[tok] (or embeds[src] when tok < 0).
+// With ssq != NULL, `feat` holds residual rows and the feature is their RMSNorm
+// (x * rsqrt(mean x^2 + eps) * gain), computed here.
 __global__ void draft_input_kernel(RowTable rt, const int *__restrict__ feat_src,
-                                   const float *__restrict__ feat, const bf16 *__restrict__ embeds,
+                                   const float *__restrict__ feat, const float *__restrict__ ssq, int nt,
+                                   const float *__restrict__ gain, float eps,
+                                   const bf16 *__restrict__ embeds,
                                    const bf16 *__restrict__ E, int d, bf16 *__restrict__ xin, size_t plane) {
+  pdl_launch();
+  pdl_wait();
   const int r = blockIdx.x;
   const float *f = feat + (size_t)feat_src[r] * d;
+  const float rs = ssq ? norm_scale(ssq, nt, (size_t)feat_src[r], d, eps) : 1.f;
   const int tok = rt.tok[r];
   const bf16 *e = tok >= 0 ? E + (size_t)tok * d : embeds + (size_t)rt.src[r] * d;
   for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    const bf16 hi = __float2bfloat16(f[i]);
+    const float fv = ssq ? f[i] * rs * gain[i] : f[i];
+    const bf16 hi = __float2bfloat16(fv);
     xin[(size_t)r * 2 * d + i] = hi;
-    xin[plane + (size_t)r * 2 * d + i] = __float2bfloat16(f[i] - __bfloat162float(hi));
+    xin[plane + (size_t)r * 2 * d + i] = __float2bfloat16(fv - __bfloat162float(hi));
     xin[(size_t)r * 2 * d + d + i] = e[i];
     xin[plane + (size_t)r * 2 * d + d + i] = __float2bfloat16(0.f);
   }
@@ -92,6 +111,8 @@ __global__ void draft_input_kernel(RowTable rt, const int *__restrict__ feat_src
 // call only each episode's last row is kept, as draft row 0.
 __global__ void save_draft_out_kernel(const float *__restrict__ x, const int *__restrict__ dst_row,
                                       int d, float *__restrict__ dout) {
+  pdl_launch();
+  pdl_wait();
   const int r = blockIdx.x;
   const int dst = dst_row[r];
   if (dst < 0) return;
@@ -100,6 +121,8 @@ __global__ void save_draft_out_kernel(const float *__restrict__ x, const int *__
 
 // dst_row for the catch-up call: last pending row of episode i -> dout row e * SV_MAX_TREE.
 __global__ void catchup_dst_kernel(EpArgs a, int *__restrict__ dst_row, int *__restrict__ lm_rows) {
+  pdl_launch();
+  pdl_wait();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= a.n_ep) return;
   for (int j = 0; j < a.nrows[i]; j++) dst_row[a.row0[i] + j] = -1;
@@ -119,6 +142,8 @@ __global__ void expand_level_kernel(EpArgs a, int level, int branch, int expand_
                                     const int *__restrict__ top_tok, const float *__restrict__ top_lp,
                                     DevTree *trees, const EpState *__restrict__ st, RowTable rt,
                                     int *__restrict__ feat_src, int *__restrict__ dst_row) {
+  pdl_launch();
+  pdl_wait();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= a.n_ep) return;
   const int e = a.eps[i];
@@ -184,8 +209,11 @@ __global__ void expand_level_kernel(EpArgs a, int level, int branch, int expand_
 // commits the state for the next iteration and gathers the features on the path.
 __global__ void __launch_bounds__(128)
 accept_select_kernel(EpArgs ea, DevTree *trees, EpState *st, const int *__restrict__ greedy, int r, int a0, int nb,
-                     const float *__restrict__ feat, int d, float *__restrict__ pend_feat,
+                     const float *__restrict__ x, const float *__restrict__ ssq, int nt,
+                     const float *__restrict__ gain, float eps, int d, float *__restrict__ pend_feat,
                      int *__restrict__ out_m, int *__restrict__ out_tok, int *__restrict__ out_path) {
+  pdl_launch();
+  pdl_wait();
   __shared__ int s_path[SV_MAX_DEPTH + 1], s_m;
   const int e = ea.eps[blockIdx.x];
   const int base = ea.row0[blockIdx.x];
@@ -248,10 +276,13 @@ accept_select_kernel(EpArgs ea, DevTree *trees, EpState *st, const int *__restri
   }
   __syncthreads();
   const int m = s_m;
+  // features (final-norm outputs) of the rows on the path, for the draft model's next call
   for (int k = 0; k <= m; k++) {
-    const float *src = feat + (size_t)(base + s_path[k]) * d;
+    const size_t row = (size_t)(base + s_path[k]);
+    const float *src = x + row * d;
+    const float rs = norm_scale(ssq, nt, row, d, eps);
     float *dst = pend_feat + (size_t)(e * SV_MAX_PENDING + k) * d;
-    for (int i = threadIdx.x; i < d; i += blockDim.x) dst[i] = src[i];
+    for (int i = threadIdx.x; i < d; i += blockDim.x) dst[i] = src[i] * rs * gain[i];
   }
 }
 
@@ -263,6 +294,8 @@ __global__ void __launch_bounds__(256)
 kv_compact_kernel(EpArgs a, const EpState *__restrict__ st,
                   const int *__restrict__ out_m, const int *__restrict__ out_path,
                   float *__restrict__ cache, size_t ep_stride, size_t layer_stride, int max_seq, int hd) {
+  pdl_launch();
+  pdl_wait();
   const int e = a.eps[blockIdx.y];
   const int m = out_m[blockIdx.y];
   const int P = st[e].P;
@@ -281,6 +314,8 @@ kv_compact_kernel(EpArgs a, const EpState *__restrict__ st,
 
 // P <- P + 1 + m after compaction.
 __global__ void advance_state_kernel(EpArgs a, EpState *st, const int *__restrict__ out_m) {
+  pdl_launch();
+  pdl_wait();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < a.n_ep) st[a.eps[i]].P += 1 + out_m[i];
 }
@@ -288,8 +323,12 @@ __global__ void advance_state_kernel(EpArgs a, EpState *st, const int *__restric
 // State after prefill: P = len, Pd = len - 1, root = a_1, one pending pair (f_{P-1}, a_1).
 // a.nrows = prefix lengths, a.aux = last row of each episode.
 __global__ void prefill_commit_kernel(EpArgs a, EpState *st,
-                                      const int *__restrict__ greedy, const float *__restrict__ feat,
+                                      const int *__restrict__ greedy, const float *__restrict__ x,
+                                      const float *__restrict__ ssq, int nt,
+                                      const float *__restrict__ gain, float eps,
                                       int d, float *__restrict__ pend_feat) {
+  pdl_launch();
+  pdl_wait();
   const int e = a.eps[blockIdx.x];
   if (threadIdx.x == 0) {
     EpState &s = st[e];
@@ -299,9 +338,11 @@ __global__ void prefill_commit_kernel(EpArgs a, EpState *st,
     s.n_pending = 1;
     s.pending_tok[0] = greedy[blockIdx.x];
   }
-  const float *src = feat + (size_t)a.aux[blockIdx.x] * d;
+  const size_t row = (size_t)a.aux[blockIdx.x];
+  const float *src = x + row * d;
+  const float rs = norm_scale(ssq, nt, row, d, eps);
   float *dst = pend_feat + (size_t)e * SV_MAX_PENDING * d;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) dst[i] = src[i];
+  for (int i = threadIdx.x; i < d; i += blockDim.x) dst[i] = src[i] * rs * gain[i];
 }
 
 }  // namespace tree
