@@ -204,6 +204,27 @@ int specvla_gemm(const float *X, const void *W, float *Y, int T, int N, int K,
  * undefined), SPECVLA_ERR_CUDA if the stream is in error, else SPECVLA_OK. */
 int specvla_gemm_status(const void *scratch, void *stream);
 
+/* specvla_gemm for callers that cannot allocate device memory: code running inside a CUDA
+ * stream capture or a real-time control loop, a plug-in handed only its input and output
+ * buffers, a process whose memory pool is owned by another component. (The paper has no
+ * counterpart of this call; it exists for such callers only.) The scratch that specvla_gemm
+ * takes from its caller is here a fixed array of SPECVLA_STATIC_SCRATCH_BYTES inside the
+ * library image; every GPU that loads the library holds that much memory until the process
+ * exits. X, W and Y are the caller's, exactly as for specvla_gemm.
+ *  - Returns SPECVLA_ERR_CAPACITY, before touching the GPU, when
+ *    specvla_gemm_scratch_bytes(T, N, K) exceeds SPECVLA_STATIC_SCRATCH_BYTES.
+ *  - Calls no cudaMalloc / cudaFree or any other allocating routine.
+ *  - The first call on each device looks the array's device address up (the device must be
+ *    current); make that first call outside any stream capture.
+ *  - All calls on a device share the one array, which still holds the previous call's
+ *    contents; the call clears what it needs cleared. Two calls that may overlap on the GPU
+ *    (different streams, no dependency) race on it: serialise them.
+ *  - wait != 0: synchronises `stream` and returns SPECVLA_ERR_TIMEOUT if a bounded
+ *    device-side wait gave up (as specvla_gemm_status); wait == 0: asynchronous. */
+#define SPECVLA_STATIC_SCRATCH_BYTES (16u << 20)
+int specvla_gemm_static(const float *X, const void *W, float *Y, int T, int N, int K, int wait,
+                        void *stream);
+
 /* Per-GEMM device timing (measurement aid; Section 3.1 attributes the latency to the
  * parameter stream, which these GEMMs are). `phases` is a bit mask: 1 = prefill, 2 = draft,
  * 4 = verification; 0 switches timing off. While a phase is enabled, every weight-streaming

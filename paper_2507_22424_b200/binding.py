@@ -71,6 +71,8 @@ EXPORTS = {
     "specvla_gemm": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                                     C.c_void_p, C.c_size_t, C.c_void_p]),
     "specvla_gemm_status": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "specvla_gemm_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int,
+                                     C.c_void_p]),
     "specvla_profile": (C.c_int, [C.c_void_p, C.c_int]),
     "specvla_profile_read": (C.c_int, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_longlong),
                                        C.POINTER(C.c_double)]),
@@ -277,6 +279,24 @@ def gemm(x: torch.Tensor, w: torch.Tensor) -> torch.Tensor:
                                T, N, K, C.c_void_p(sp), nb, _stream())
     if rc == 0:
         rc = lib.specvla_gemm_status(C.c_void_p(sp), _stream())
+    if rc != 0:
+        raise SpecVLAError(rc)
+    return y
+
+
+STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def gemm_static(x: torch.Tensor, w: torch.Tensor, y: torch.Tensor) -> torch.Tensor:
+    """specvla_gemm_static: the same product written into the caller's y, with the scratch taken
+    from the library's built-in array instead of a caller allocation. Nothing is allocated here
+    or in the library; shapes whose scratch exceeds STATIC_SCRATCH_BYTES raise SpecVLAError(-2)."""
+    assert x.dtype == torch.float32 and w.dtype == torch.bfloat16 and y.dtype == torch.float32
+    T, K = x.shape
+    N = w.shape[0]
+    assert y.shape == (T, N) and y.is_contiguous()
+    rc = lib.specvla_gemm_static(C.c_void_p(x.data_ptr()), C.c_void_p(w.data_ptr()), C.c_void_p(y.data_ptr()),
+                                 T, N, K, 1, _stream())
     if rc != 0:
         raise SpecVLAError(rc)
     return y

@@ -1141,6 +1141,34 @@ int specvla_gemm(const float *X, const void *W, float *Y, int T, int N, int K, v
   return cudaGetLastError() == cudaSuccess ? SPECVLA_OK : SPECVLA_ERR_CUDA;
 }
 
+// ------------------------------------------------------------------ GEMM without allocation
+// Scratch of specvla_gemm_static: lives in the library image, one copy on every device that
+// loads it, for as long as the process runs. The extra 1 KB lets the start be rounded up to
+// the 1024-byte boundary specvla_gemm asks for.
+static __device__ __align__(256) unsigned char g_static_scratch[SPECVLA_STATIC_SCRATCH_BYTES + 1024];
+// Device address of g_static_scratch per device ordinal (0 = not looked up yet). In host code
+// the symbol itself is only a stand-in; kernels must be given the address looked up here.
+static void *g_static_scratch_addr[64];
+
+int specvla_gemm_static(const float *X, const void *W, float *Y, int T, int N, int K, int wait, void *stream) {
+  if (!X || !W || !Y || T < 1 || N < 1 || K < 8 || (K % 8)) return SPECVLA_ERR_INVALID_ARG;
+  const size_t need = specvla_gemm_scratch_bytes(T, N, K);
+  if (need == 0) return SPECVLA_ERR_INVALID_ARG;
+  if (need > (size_t)SPECVLA_STATIC_SCRATCH_BYTES) return SPECVLA_ERR_CAPACITY;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SPECVLA_ERR_CUDA;
+  if (!g_static_scratch_addr[dev]) {
+    void *p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return SPECVLA_ERR_CUDA;
+    g_static_scratch_addr[dev] = p;
+  }
+  const uintptr_t base = (reinterpret_cast<uintptr_t>(g_static_scratch_addr[dev]) + 1023) & ~(uintptr_t)1023;
+  void *scratch = reinterpret_cast<void *>(base);
+  const int rc = specvla_gemm(X, W, Y, T, N, K, scratch, SPECVLA_STATIC_SCRATCH_BYTES, stream);
+  if (rc != SPECVLA_OK || !wait) return rc;
+  return specvla_gemm_status(scratch, stream);
+}
+
 int specvla_gemm_status(const void *scratch, void *stream) {
   if (!scratch) return SPECVLA_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
