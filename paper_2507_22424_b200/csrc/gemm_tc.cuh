@@ -129,6 +129,13 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm,
       "[%0], [%1, {%2, %3, %4}], [%5], %6;"
       ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(bar), "l"(pol) : "memory");
 }
+// Linear bulk copy global -> shared (both 16-byte aligned, size a multiple of 16).
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar,
+                                          uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+      ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(pol) : "memory");
+}
 __device__ __forceinline__ void grid_dep_wait() { pdl_wait(); }
 __device__ __forceinline__ void grid_dep_launch() { pdl_launch(); }
 __device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
@@ -196,6 +203,8 @@ struct EpiArgs {
   int T;                 // rows of this launch (<= 128)
   int N;                 // output columns (EPI_SWIGLU: F, the width of gate and of up)
   int up_off;            // EPI_SWIGLU: row of W where the up projection starts (F)
+  const bf16 *wpacked;   // weights repacked by pack_weights_kernel (one contiguous 32 KB block per
+                         // (tile, K block), in unit order); NULL: strided boxes through the W map
   float *part;           // planes [max segments][T][tiles * 256] for tiles shared by several CTAs
   int *counters;         // [tiles] arrivals per shared tile; zero between launches
   // row scale of the RMSNorm in front of this GEMM: rsqrt(sum_j ssq_in[row][j] * inv_k + eps)
@@ -291,8 +300,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         const int ya = swiglu ? tile * 128 : tile * BM;
         const int yb = swiglu ? ea.up_off + tile * 128 : tile * BM + 128;
         mbar_expect_tx(full_bar(st), STAGE);
-        tma_load_2d(sW, &tmW, kb * BK, ya, full_bar(st), pol_w);
-        tma_load_2d(sW + 128 * BK * 2, &tmW, kb * BK, yb, full_bar(st), pol_w);
+        if (ea.wpacked) {
+          bulk_load(sW, ea.wpacked + (size_t)u * (BM * BK), W_STAGE_BYTES, full_bar(st), pol_w);
+        } else {
+          tma_load_2d(sW, &tmW, kb * BK, ya, full_bar(st), pol_w);
+          tma_load_2d(sW + 128 * BK * 2, &tmW, kb * BK, yb, full_bar(st), pol_w);
+        }
         if (it >= npre) tma_load_3d(sW + W_STAGE_BYTES, &tmX, kb * BK, ea.row0, 0, full_bar(st), pol_x);
         if (it == npre - 1) {
           // the activations are the previous kernel's output: wait for it only now
@@ -434,24 +447,38 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         for (int c0 = 0; c0 < TN; c0 += 16) {
           float va[16], vb[16];
           if (nseg > 1) {
-            // planes in ascending order; the 32 loads of one plane are independent and in flight
-            // together
+            // planes are added in ascending order; two planes (64 independent loads per thread)
+            // are in flight per round
 #pragma unroll
             for (int j = 0; j < 16; j++) va[j] = vb[j] = 0.f;
+            const float *pl = ea.part + (size_t)c0 * ldp + pc;
+            const size_t pstride = (size_t)T * ldp;
+            int sgn = 0;
 #pragma unroll 1
-            for (int s = 0; s < nseg; s++) {
-              const float *pl = ea.part + ((size_t)s * T + c0) * ldp + pc;
-              float ta[16], tb[16];
+            for (; sgn + 1 < nseg; sgn += 2) {
+              float ta[16], tb[16], ua[16], ub[16];
 #pragma unroll
               for (int j = 0; j < 16; j++) {
                 const bool in = c0 + j < T;
-                ta[j] = in ? __ldcg(pl + (size_t)j * ldp) : 0.f;
-                tb[j] = in ? __ldcg(pl + (size_t)j * ldp + 128) : 0.f;
+                const float *p0 = pl + (size_t)sgn * pstride + (size_t)j * ldp;
+                ta[j] = in ? __ldcg(p0) : 0.f;
+                tb[j] = in ? __ldcg(p0 + 128) : 0.f;
+                ua[j] = in ? __ldcg(p0 + pstride) : 0.f;
+                ub[j] = in ? __ldcg(p0 + pstride + 128) : 0.f;
               }
 #pragma unroll
               for (int j = 0; j < 16; j++) {
-                va[j] += ta[j];
-                vb[j] += tb[j];
+                va[j] = (va[j] + ta[j]) + ua[j];
+                vb[j] = (vb[j] + tb[j]) + ub[j];
+              }
+            }
+            if (sgn < nseg) {
+#pragma unroll
+              for (int j = 0; j < 16; j++) {
+                const bool in = c0 + j < T;
+                const float *p0 = pl + (size_t)sgn * pstride + (size_t)j * ldp;
+                va[j] += in ? __ldcg(p0) : 0.f;
+                vb[j] += in ? __ldcg(p0 + 128) : 0.f;
               }
             }
           } else {
@@ -486,6 +513,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           } else {
             const float ga = (ea.gain && na < ea.N) ? ea.gain[na] : 1.f;
             const float gb = (ea.gain && nb < ea.N) ? ea.gain[nb] : 1.f;
+            // all residual loads of the 16 rows first: they are independent of the stores below
+            float xa[16], xb[16];
+#pragma unroll
+            for (int j = 0; j < 16; j++) {
+              const bool in = ea.accumulate && c0 + j < T;
+              const size_t r = (size_t)(ea.row0 + c0 + j) * ea.N;
+              xa[j] = (in && na < ea.N) ? __ldcg(ea.x + r + na) : 0.f;
+              xb[j] = (in && nb < ea.N) ? __ldcg(ea.x + r + nb) : 0.f;
+            }
 #pragma unroll
             for (int half8 = 0; half8 < 2; half8++) {
 #pragma unroll
@@ -495,13 +531,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
                 if (c0 + j < T) {
                   const size_t r = (size_t)(ea.row0 + c0 + j) * ea.N;
                   if (na < ea.N) {
-                    const float xv = (ea.accumulate ? ea.x[r + na] : 0.f) + va[j];
+                    const float xv = xa[j] + va[j];
                     ea.x[r + na] = xv;
                     store_limbs(ea.xn, ea.xn_plane, r + na, xv * ga);
                     s2 += xv * xv;
                   }
                   if (nb < ea.N) {
-                    const float xv = (ea.accumulate ? ea.x[r + nb] : 0.f) + vb[j];
+                    const float xv = xb[j] + vb[j];
                     ea.x[r + nb] = xv;
                     store_limbs(ea.xn, ea.xn_plane, r + nb, xv * gb);
                     s2 += xv * xv;
@@ -545,6 +581,38 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   tc_fence_after();
   if (warp == 1) tc_dealloc(tmem_base, tmem_cols(TN));
 }
+
+// Repacks W [N, K] (row-major) into the order the kernel streams it: one contiguous 32 KB block
+// per unit (tile, K block), tile-major, each block being the shared-memory image of a stage
+// (256 rows of 64 bf16, the eight 16-byte chunks of a row XOR-swizzled by row & 7, exactly what
+// a 128-byte-swizzle TMA box would have written). A CTA's share of the stream is then one
+// contiguous range of HBM instead of 128-byte pieces one row pitch apart. Rows / columns past
+// the matrix are zero. swiglu: tile j = gate rows j*128.. then up rows F + j*128.. (N = 2F).
+__global__ void pack_weights_kernel(const bf16 *__restrict__ W, int N, int K, int tiles, int KB, int swiglu,
+                                    int F, bf16 *__restrict__ out) {
+  const size_t total = (size_t)tiles * KB * BM * 8;
+  for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+       idx += (size_t)gridDim.x * blockDim.x) {
+    const int c = (int)(idx & 7), r = (int)((idx >> 3) & (BM - 1));
+    const size_t unit = idx >> 11;
+    const int kb = (int)(unit % KB), tile = (int)(unit / KB);
+    int n;
+    bool ok;
+    if (swiglu) {
+      n = (r < 128) ? tile * 128 + r : F + tile * 128 + (r - 128);
+      ok = tile * 128 + (r & 127) < F;
+    } else {
+      n = tile * BM + r;
+      ok = n < N;
+    }
+    const int k = kb * BK + c * 8;
+    ok = ok && k < K;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (ok) v = *reinterpret_cast<const uint4 *>(W + (size_t)n * K + k);
+    *reinterpret_cast<uint4 *>(out + unit * (BM * BK) + (size_t)r * BK + ((c ^ (r & 7)) << 3)) = v;
+  }
+}
+inline size_t packed_elems(int tiles, int K) { return (size_t)tiles * ((K + BK - 1) / BK) * BM * BK; }
 
 // ------------------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,

@@ -24,6 +24,7 @@ struct WMat {
   int N, K;
   bool has_map;
   CUtensorMap map;
+  const bf16 *packed;     // the library's repacked copy (gemm_tc::pack_weights_kernel), in the workspace
 };
 // A two-limb activation buffer [2][rows][K] and its TMA maps, one per row-tile size 16/32/64/128.
 struct XBuf {
@@ -79,6 +80,8 @@ struct specvla_ctx {
   float *x, *feat, *part, *lgs, *pend_feat, *dout, *margin, *top_lp, *q, *qkv;
   float *ssq, *lm_ssq;          // per-row partial sums of squares of x / of the gathered LM-head rows
   int *counters;                // per-tile arrival counters of the GEMM (zero between launches)
+  bf16 *packed;                 // repacked weight matrices, one after the other
+  size_t packed_elems;
   float *att_part;              // parked key slices of the attention kernel
   int *att_counters;            // its arrival counters (zero between launches)
   size_t part_floats;
@@ -195,6 +198,16 @@ size_t carve(specvla_ctx *c, char *base) {
   need(tiles256(d.vocab), d.d_model);
   c->part_floats = pf;
   c->part = cv.take<float>(pf);
+  {
+    // repacked weights: every target layer, the LM head, the draft fc and the draft layer
+    const size_t layer = gemm_tc::packed_elems(tiles256(3 * hd), d.d_model) +
+                         gemm_tc::packed_elems(tiles256(d.d_model), hd) +
+                         gemm_tc::packed_elems((d.d_ffn + 127) / 128, d.d_model) +
+                         gemm_tc::packed_elems(tiles256(d.d_model), d.d_ffn);
+    c->packed_elems = layer * ((size_t)d.n_layers + 1) + gemm_tc::packed_elems(tiles256(d.vocab), d.d_model) +
+                      gemm_tc::packed_elems(tiles256(d.d_model), 2 * d.d_model);
+    c->packed = cv.take<bf16>(c->packed_elems);
+  }
   c->att_part = cv.take<float>((size_t)attn::MAX_SPLIT_CTAS * attn::RB * (d.head_dim + 2));
   c->att_counters = cv.take<int>(attn::MAX_SPLIT_CTAS);
   c->n_counters = max_tiles;
@@ -281,6 +294,7 @@ int gemm(specvla_ctx *ctx, const XBuf &A, const WMat &W, int R, gemm_tc::EpiArgs
     return SPECVLA_ERR_CAPACITY;
   ea.part = ctx->part;
   ea.counters = ctx->counters;
+  ea.wpacked = W.packed;
   ea.inv_k = 1.f / (float)W.K;
   ea.eps = ctx->desc.rms_eps;
   const bool prof = (ctx->prof_mask & ctx->phase) && 2 * (ctx->prof_used + 1) <= (int)ctx->prof_ev.size();
@@ -511,12 +525,30 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
   carve(ctx, static_cast<char *>(workspace));
   const int hd = ctx->hd, D = desc->d_model, F = desc->d_ffn;
   ctx->use_pdl = getenv("SPECVLA_NO_PDL") == nullptr;
-  auto wmat = [&](const void *p, int N, int K) {
+  size_t packed_used = 0;
+  bool pack_ok = true;
+  // swiglu: the matrix is [gate; up] stacked ([2F, K]) and is packed as tiles of 128 + 128 rows
+  auto wmat = [&](const void *p, int N, int K, bool swiglu = false) {
     WMat w{};
     w.p = static_cast<const bf16 *>(p);
     w.N = N;
     w.K = K;
     w.has_map = p && gemm_tc::make_w_map(&w.map, w.p, N, K);
+    w.packed = nullptr;
+    if (p) {
+      const int F = N / 2;
+      const int tiles = swiglu ? (F + 127) / 128 : (N + SV_TILE_ROWS - 1) / SV_TILE_ROWS;
+      const size_t elems = gemm_tc::packed_elems(tiles, K);
+      if (packed_used + elems > ctx->packed_elems) {
+        pack_ok = false;
+        return w;
+      }
+      bf16 *dst = ctx->packed + packed_used;
+      packed_used += elems;
+      gemm_tc::pack_weights_kernel<<<148 * 8, 256>>>(w.p, N, K, tiles, (K + gemm_tc::BK - 1) / gemm_tc::BK,
+                                                     swiglu ? 1 : 0, F, dst);
+      w.packed = dst;
+    }
     return w;
   };
   auto xmaps = [&](XBuf &b) {
@@ -539,13 +571,13 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
       delete ctx;
       return SPECVLA_ERR_INVALID_ARG;
     }
-    ctx->layers[l] = LayerW{wmat(tw->wqkv[l], 3 * hd, D), wmat(tw->wo[l], D, hd), wmat(tw->wgu[l], 2 * F, D),
+    ctx->layers[l] = LayerW{wmat(tw->wqkv[l], 3 * hd, D), wmat(tw->wo[l], D, hd), wmat(tw->wgu[l], 2 * F, D, true),
                             wmat(tw->wd[l], D, F), tw->norm1[l], tw->norm2[l]};
   }
   ctx->has_draft = dw && dw->fc && dw->wqkv && dw->wo && dw->wgu && dw->wd && dw->norm1 && dw->norm2;
   if (ctx->has_draft) {
     ctx->draft_fc = wmat(dw->fc, D, 2 * D);
-    ctx->dlayer = LayerW{wmat(dw->wqkv, 3 * hd, D), wmat(dw->wo, D, hd), wmat(dw->wgu, 2 * F, D),
+    ctx->dlayer = LayerW{wmat(dw->wqkv, 3 * hd, D), wmat(dw->wo, D, hd), wmat(dw->wgu, 2 * F, D, true),
                          wmat(dw->wd, D, F), dw->norm1, dw->norm2};
   }
   ctx->hP.assign(desc->max_episodes, -1);
@@ -579,10 +611,10 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
                        attn::smem_bytes<128>());
   cudaFuncSetAttribute(attn::tree_attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                        attn::smem_bytes<64>());
-  if (cudaDeviceSynchronize() != cudaSuccess) {
+  if (cudaDeviceSynchronize() != cudaSuccess || !pack_ok) {
     cudaFreeHost(ctx->pinned);
     delete ctx;
-    return SPECVLA_ERR_CUDA;
+    return pack_ok ? SPECVLA_ERR_CUDA : SPECVLA_ERR_CAPACITY;
   }
   *out = ctx;
   return SPECVLA_OK;
