@@ -88,6 +88,30 @@ __host__ __device__ inline int nseg_of(const SegPlan &p, int n) {
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// Four consecutive elements at a time (every row length here is a multiple of 8 elements and
+// every buffer starts on a 1024-byte boundary, so these accesses are aligned).
+__device__ __forceinline__ float4 load_bf16x4(const bf16 *p) {
+  const uint2 raw = *reinterpret_cast<const uint2 *>(p);
+  const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162 *>(&raw.x);
+  const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162 *>(&raw.y);
+  const float2 fa = __bfloat1622float2(a), fb = __bfloat1622float2(b);
+  return make_float4(fa.x, fa.y, fb.x, fb.y);
+}
+__device__ __forceinline__ void store_bf16x4(bf16 *p, float4 v) {
+  __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+  uint2 raw;
+  raw.x = *reinterpret_cast<uint32_t *>(&a);
+  raw.y = *reinterpret_cast<uint32_t *>(&b);
+  *reinterpret_cast<uint2 *>(p) = raw;
+}
+// Two-limb split of four values: hi = bf16(v), lo = bf16(v - hi), lo plane `plane` elements on.
+__device__ __forceinline__ void store_limbs4(bf16 *hi_plane, size_t plane, size_t idx, float4 v) {
+  const float4 h = make_float4(__bfloat162float(__float2bfloat16(v.x)), __bfloat162float(__float2bfloat16(v.y)),
+                               __bfloat162float(__float2bfloat16(v.z)), __bfloat162float(__float2bfloat16(v.w)));
+  store_bf16x4(hi_plane + idx, h);
+  store_bf16x4(hi_plane + plane + idx, make_float4(v.x - h.x, v.y - h.y, v.z - h.z, v.w - h.w));
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

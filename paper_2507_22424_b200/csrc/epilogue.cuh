@@ -56,11 +56,13 @@ embed_kernel(RowTable rt, const bf16 *__restrict__ embeds, const bf16 *__restric
   const int tok = rt.tok[t];
   const bf16 *src = tok >= 0 ? E + (size_t)tok * d : embeds + (size_t)rt.src[t] * d;
   float ss = 0.f;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    const float v = __bfloat162float(src[i]);
-    x[(size_t)t * d + i] = v;
-    store2(xn, plane, (size_t)t * d + i, v * gain[i]);
-    ss += v * v;
+#pragma unroll 2
+  for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
+    const float4 v = load_bf16x4(src + i);
+    const float4 g = *reinterpret_cast<const float4 *>(gain + i);
+    *reinterpret_cast<float4 *>(x + (size_t)t * d + i) = v;
+    store_limbs4(xn, plane, (size_t)t * d + i, make_float4(v.x * g.x, v.y * g.y, v.z * g.z, v.w * g.w));
+    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
   }
   ss = block_sum(ss, red);
   for (int j = threadIdx.x; j < nt; j += blockDim.x) ssq[(size_t)t * nt + j] = (j == 0) ? ss : 0.f;
@@ -114,9 +116,12 @@ __global__ void gather_rows_kernel(const bf16 *__restrict__ src, size_t src_plan
   pdl_launch();
   pdl_wait();
   const int r = rows[blockIdx.x];
-  for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    dst[(size_t)blockIdx.x * d + i] = src[(size_t)r * d + i];
-    dst[dst_plane + (size_t)blockIdx.x * d + i] = src[src_plane + (size_t)r * d + i];
+#pragma unroll 2
+  for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
+    *reinterpret_cast<uint2 *>(dst + (size_t)blockIdx.x * d + i) =
+        *reinterpret_cast<const uint2 *>(src + (size_t)r * d + i);
+    *reinterpret_cast<uint2 *>(dst + dst_plane + (size_t)blockIdx.x * d + i) =
+        *reinterpret_cast<const uint2 *>(src + src_plane + (size_t)r * d + i);
   }
   for (int j = threadIdx.x; j < nt; j += blockDim.x)
     dst_ssq[(size_t)blockIdx.x * nt + j] = src_ssq[(size_t)r * nt + j];
@@ -129,8 +134,13 @@ __global__ void features_kernel(const float *__restrict__ x, const float *__rest
   pdl_wait();
   const int t = blockIdx.x;
   const float rs = row_scale(ssq, nt, t, d, eps);
-  for (int i = threadIdx.x; i < d; i += blockDim.x)
-    feat[(size_t)t * d + i] = x[(size_t)t * d + i] * rs * gain[i];
+#pragma unroll 2
+  for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
+    const float4 v = *reinterpret_cast<const float4 *>(x + (size_t)t * d + i);
+    const float4 g = *reinterpret_cast<const float4 *>(gain + i);
+    *reinterpret_cast<float4 *>(feat + (size_t)t * d + i) =
+        make_float4(v.x * rs * g.x, v.y * rs * g.y, v.z * rs * g.z, v.w * rs * g.w);
+  }
 }
 
 // Two-limb split of an fp32 matrix (stand-alone GEMM entry point).

@@ -19,7 +19,7 @@
 //  * "Finishing" a tile is the fused epilogue: plain store with the RMSNorm row scale, or
 //    residual add + gain + two-limb split + sum of squares for the next norm, or SwiGLU.
 //  * Warp 0 issues TMA loads into a ring of stages, warp 1 issues the MMAs and releases
-//    stages through tcgen05.commit, warps 2-5 run the epilogue on finished accumulators
+//    stages through tcgen05.commit, warps 2-9 run the epilogue on finished accumulators
 //    (double-buffered in TMEM).
 //  * The weight loads of the first ring-full do not depend on the previous kernel, so they
 //    are issued BEFORE griddepcontrol.wait: launched with programmatic stream serialisation
@@ -36,7 +36,7 @@ namespace gemm_tc {
 
 constexpr int BM = SV_TILE_ROWS;          // weight rows per tile (two UMMA halves of 128)
 constexpr int BK = 64;                    // K per stage: 128 bytes = one swizzle row
-constexpr int THREADS = 192;
+constexpr int THREADS = 320;               // warp 0 TMA, warp 1 MMA, warps 2-9 epilogue
 constexpr int W_STAGE_BYTES = BM * BK * 2;
 constexpr int RING_BUDGET = 164 * 1024;
 constexpr int MAX_T = 128;
@@ -47,7 +47,12 @@ __host__ __device__ constexpr int stage_bytes(int TN) { return W_STAGE_BYTES + 2
 // GEMMs can be resident next to a GEMM CTA while it prefetches weights.
 __host__ __device__ constexpr int stages_of(int TN) { return RING_BUDGET / stage_bytes(TN); }
 __host__ __device__ constexpr int smem_bytes(int TN) { return stages_of(TN) * stage_bytes(TN) + 1024 + 256; }
-__host__ __device__ constexpr int tmem_cols(int TN) { return 4 * TN < 32 ? 32 : 4 * TN; }      // 64, 128, 256, 512
+// Up to 64 rows both limbs of X form ONE MMA operand (N = 2 TN: hi rows, then lo rows) and the
+// two column groups are added in the epilogue; at 128 rows the limbs are two MMAs into the
+// same TN columns. Either way an accumulator is acc_width(TN) TMEM columns wide.
+__host__ __device__ constexpr bool merged_limbs(int TN) { return TN <= 64; }
+__host__ __device__ constexpr int acc_width(int TN) { return merged_limbs(TN) ? 2 * TN : TN; }
+__host__ __device__ constexpr int tmem_cols(int TN) { return 4 * acc_width(TN); }      // 128, 256, 512, 512
 
 // tiles: 256-column tiles of the output (for SwiGLU: 128 gate + 128 up columns each).
 inline SegPlan make_plan(int tiles, int K, int num_sms) {
@@ -138,7 +143,10 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_
 }
 __device__ __forceinline__ void grid_dep_wait() { pdl_wait(); }
 __device__ __forceinline__ void grid_dep_launch() { pdl_launch(); }
-__device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *tm) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(tm) : "memory");
+}
 
 __device__ __forceinline__ void tc_alloc(uint32_t smem_dst, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
@@ -238,7 +246,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
                const EpiArgs ea, const SegPlan plan, int *__restrict__ err) {
   constexpr int STAGES = stages_of(TN);
   constexpr int STAGE = stage_bytes(TN);
-  constexpr uint32_t IDESC = instr_desc(TN);
+  constexpr bool MERGE = merged_limbs(TN);
+  constexpr int AW = acc_width(TN);
+  constexpr uint32_t IDESC = instr_desc(AW);
   extern __shared__ unsigned char smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t bars = base + STAGES * STAGE;
@@ -249,7 +259,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   const uint32_t tmem_slot = bars + 8u * (2 * STAGES + 4);
   __shared__ float s_scale[MAX_T];        // RMSNorm row scales
   __shared__ float s_red[4][MAX_T];       // per-warp sums of squares
-  __shared__ int s_flag[4];
+  __shared__ int s_flag[8];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const long long u0 = (long long)blockIdx.x * plan.U / plan.G;
@@ -259,18 +269,42 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   const int T = ea.T;
   const bool swiglu = ea.mode == EPI_SWIGLU;
 
+  const int npre = n_units < STAGES ? n_units : STAGES;
+  uint64_t pol_w = 0;
+  auto load_w = [&](int it) {
+    const int st = it % STAGES;
+    const long long u = u0 + it;
+    const int tile = (int)(u / KB), kb = (int)(u % KB);
+    const uint32_t sW = base + st * STAGE;
+    mbar_expect_tx(full_bar(st), STAGE);
+    if (ea.wpacked) {
+      bulk_load(sW, ea.wpacked + (size_t)u * (BM * BK), W_STAGE_BYTES, full_bar(st), pol_w);
+    } else {
+      // the two 128-row halves of the tile: consecutive rows, or gate rows + up rows
+      const int ya = swiglu ? tile * 128 : tile * BM;
+      const int yb = swiglu ? ea.up_off + tile * 128 : tile * BM + 128;
+      tma_load_2d(sW, &tmW, kb * BK, ya, full_bar(st), pol_w);
+      tma_load_2d(sW + 128 * BK * 2, &tmW, kb * BK, yb, full_bar(st), pol_w);
+    }
+  };
   if (threadIdx.x == 0) {
+    prefetch_tensormap(&tmX);
+    if (!ea.wpacked) prefetch_tensormap(&tmW);
     for (int s = 0; s < STAGES; s++) {
       mbar_init(full_bar(s), 1);
       mbar_init(empty_bar(s), 1);
     }
     for (int b = 0; b < 2; b++) {
       mbar_init(tfull_bar(b), 1);
-      mbar_init(tempty_bar(b), 4);
+      mbar_init(tempty_bar(b), 8);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     grid_dep_launch();
+    // the first ring-full of weights needs nothing from the previous kernel nor from the rest
+    // of this CTA's set-up: get it moving at once
+    pol_w = policy_evict_first();
+    for (int it = 0; it < npre; it++) load_w(it);
   }
   if (warp == 1) {
     tc_alloc(tmem_slot, tmem_cols(TN));
@@ -285,37 +319,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0 && n_units > 0) {
-      const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
-      const int npre = n_units < STAGES ? n_units : STAGES;
-      for (int it = 0; it < n_units; it++) {
+      const uint64_t pol_x = policy_evict_last();
+      // the activations are the previous kernel's output: wait for it only now
+      grid_dep_wait();
+      for (int j = 0; j < npre; j++)
+        tma_load_3d(base + j * STAGE + W_STAGE_BYTES, &tmX, (int)((u0 + j) % KB) * BK, ea.row0, 0, full_bar(j),
+                    pol_x);
+      for (int it = npre; it < n_units; it++) {
         const int st = it % STAGES, rnd = it / STAGES;
-        if (rnd > 0 && !mbar_wait(empty_bar(st), (rnd - 1) & 1)) {
+        if (!mbar_wait(empty_bar(st), (rnd - 1) & 1)) {
           atomicExch(err, SV_ERR_WAIT_EMPTY);
           break;
         }
-        const long long u = u0 + it;
-        const int tile = (int)(u / KB), kb = (int)(u % KB);
-        const uint32_t sW = base + st * STAGE;
-        // the two 128-row halves of the tile: consecutive rows, or gate rows + up rows
-        const int ya = swiglu ? tile * 128 : tile * BM;
-        const int yb = swiglu ? ea.up_off + tile * 128 : tile * BM + 128;
-        mbar_expect_tx(full_bar(st), STAGE);
-        if (ea.wpacked) {
-          bulk_load(sW, ea.wpacked + (size_t)u * (BM * BK), W_STAGE_BYTES, full_bar(st), pol_w);
-        } else {
-          tma_load_2d(sW, &tmW, kb * BK, ya, full_bar(st), pol_w);
-          tma_load_2d(sW + 128 * BK * 2, &tmW, kb * BK, yb, full_bar(st), pol_w);
-        }
-        if (it >= npre) tma_load_3d(sW + W_STAGE_BYTES, &tmX, kb * BK, ea.row0, 0, full_bar(st), pol_x);
-        if (it == npre - 1) {
-          // the activations are the previous kernel's output: wait for it only now
-          grid_dep_wait();
-          for (int j = 0; j < npre; j++) {
-            const long long uj = u0 + j;
-            tma_load_3d(base + j * STAGE + W_STAGE_BYTES, &tmX, (int)(uj % KB) * BK, ea.row0, 0, full_bar(j),
-                        pol_x);
-          }
-        }
+        load_w(it);
+        tma_load_3d(base + st * STAGE + W_STAGE_BYTES, &tmX, (int)((u0 + it) % KB) * BK, ea.row0, 0,
+                    full_bar(st), pol_x);
       }
     }
   } else if (warp == 1) {
@@ -349,11 +367,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 #pragma unroll
           for (int h = 0; h < 2; h++) {
             const uint64_t adesc = smem_desc(sW + h * (128 * BK * 2) + kk * 32);
-            const uint32_t d = tmem_base + (uint32_t)((buf * 2 + h) * TN);
+            const uint32_t d = tmem_base + (uint32_t)((buf * 2 + h) * AW);
+            if (MERGE) {
+              tc_mma(d, adesc, smem_desc(sX + kk * 32), IDESC, (first && kk == 0) ? 0u : 1u);
+            } else {
 #pragma unroll
-            for (int limb = 0; limb < 2; limb++) {
-              const uint64_t bdesc = smem_desc(sX + limb * (TN * BK * 2) + kk * 32);
-              tc_mma(d, adesc, bdesc, IDESC, (first && kk == 0 && limb == 0) ? 0u : 1u);
+              for (int limb = 0; limb < 2; limb++) {
+                const uint64_t bdesc = smem_desc(sX + limb * (TN * BK * 2) + kk * 32);
+                tc_mma(d, adesc, bdesc, IDESC, (first && kk == 0 && limb == 0) ? 0u : 1u);
+              }
             }
           }
         }
@@ -363,10 +385,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    // ------------------------------------------------------------------ epilogue (warps 2..9)
+    // Two warps per TMEM lane quarter; they take alternate 16-row chunks of the accumulator.
     grid_dep_wait();
     const int q = warp & 3;                       // TMEM lane quarter this warp may access
-    const int et = threadIdx.x - 64;              // 0..127 among the epilogue threads
+    const int wp = (warp - 2) >> 2;               // which of the quarter's two warps
+    const int et = threadIdx.x - 64;              // 0..255 among the epilogue threads
+    // accumulator chunk: 16 rows (TMEM columns c0..c0+15 of half hf) of this thread's column
+    auto load_acc = [&](uint32_t tadr, int hf, int c0, float (&v)[16]) {
+      uint32_t r0[16];
+      tc_ld16(tadr + hf * AW + c0, r0);
+      if (MERGE) {
+        uint32_t r1[16];
+        tc_ld16(tadr + hf * AW + TN + c0, r1);
+        tc_wait_ld();
+#pragma unroll
+        for (int j = 0; j < 16; j++) v[j] = __uint_as_float(r0[j]) + __uint_as_float(r1[j]);
+      } else {
+        tc_wait_ld();
+#pragma unroll
+        for (int j = 0; j < 16; j++) v[j] = __uint_as_float(r0[j]);
+      }
+    };
     const int tiles = plan.U / KB;
     const int ldp = tiles * BM;                   // row pitch of a plane
     if (et < T) {
@@ -388,11 +428,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       const int tile = (int)(u / KB), kb0 = (int)(u % KB);
       int cnt = KB - kb0;
       if (cnt > n_units - it) cnt = n_units - it;
-      // all four warps take the same decision on the wait
+      // all eight warps take the same decision on the wait
       const bool mine = mbar_wait(tfull_bar(buf), (sidx >> 1) & 1);
-      if (lane == 0) s_flag[q] = mine ? 1 : 0;
+      if (lane == 0) s_flag[warp - 2] = mine ? 1 : 0;
       epi_barrier();
-      const bool ok = s_flag[0] && s_flag[1] && s_flag[2] && s_flag[3];
+      const bool ok = s_flag[0] && s_flag[1] && s_flag[2] && s_flag[3] && s_flag[4] && s_flag[5] && s_flag[6] &&
+                      s_flag[7];
       epi_barrier();
       if (!ok) {
         if (et == 0) atomicExch(err, SV_ERR_WAIT_TMEM_FULL);
@@ -405,23 +446,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       const int pc = tile * BM + q * 32 + lane;                       // plane column of half 0 (+128: half 1)
       const int na = swiglu ? tile * 128 + q * 32 + lane : pc;       // output column, half 0
       const int nb = swiglu ? na : pc + 128;                          // output column, half 1
-      const uint32_t tadr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 2 * TN);
+      const uint32_t tadr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 2 * AW);
 
       bool finish = true;
       if (nseg > 1) {
         // park this segment's partial sums, then see who is last
         float *pl = ea.part + (size_t)seg * T * ldp;
 #pragma unroll 1
-        for (int c0 = 0; c0 < TN; c0 += 16) {
-          uint32_t ra[16], rb[16];
-          tc_ld16(tadr + c0, ra);
-          tc_ld16(tadr + TN + c0, rb);
-          tc_wait_ld();
+        for (int c0 = 16 * wp; c0 < TN; c0 += 32) {
+          float ra[16], rb[16];
+          load_acc(tadr, 0, c0, ra);
+          load_acc(tadr, 1, c0, rb);
 #pragma unroll
           for (int j = 0; j < 16; j++)
             if (c0 + j < T) {
-              __stcg(pl + (size_t)(c0 + j) * ldp + pc, __uint_as_float(ra[j]));
-              __stcg(pl + (size_t)(c0 + j) * ldp + pc + 128, __uint_as_float(rb[j]));
+              __stcg(pl + (size_t)(c0 + j) * ldp + pc, ra[j]);
+              __stcg(pl + (size_t)(c0 + j) * ldp + pc + 128, rb[j]);
             }
         }
         tc_fence_before();
@@ -444,7 +484,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       if (finish) {
         float sq[8];                 // EPI_RESID: this thread's sums of squares, 8 rows at a time
 #pragma unroll 1
-        for (int c0 = 0; c0 < TN; c0 += 16) {
+        for (int c0 = 16 * wp; c0 < TN; c0 += 32) {
           float va[16], vb[16];
           if (nseg > 1) {
             // planes are added in ascending order; two planes (64 independent loads per thread)
@@ -482,15 +522,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
               }
             }
           } else {
-            uint32_t ra[16], rb[16];
-            tc_ld16(tadr + c0, ra);
-            tc_ld16(tadr + TN + c0, rb);
-            tc_wait_ld();
-#pragma unroll
-            for (int j = 0; j < 16; j++) {
-              va[j] = __uint_as_float(ra[j]);
-              vb[j] = __uint_as_float(rb[j]);
-            }
+            load_acc(tadr, 0, c0, va);
+            load_acc(tadr, 1, c0, vb);
           }
           if (ea.mode == EPI_PLAIN) {
 #pragma unroll

@@ -97,13 +97,16 @@ __global__ void draft_input_kernel(RowTable rt, const int *__restrict__ feat_src
   const float rs = ssq ? norm_scale(ssq, nt, (size_t)feat_src[r], d, eps) : 1.f;
   const int tok = rt.tok[r];
   const bf16 *e = tok >= 0 ? E + (size_t)tok * d : embeds + (size_t)rt.src[r] * d;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    const float fv = ssq ? f[i] * rs * gain[i] : f[i];
-    const bf16 hi = __float2bfloat16(fv);
-    xin[(size_t)r * 2 * d + i] = hi;
-    xin[plane + (size_t)r * 2 * d + i] = __float2bfloat16(fv - __bfloat162float(hi));
-    xin[(size_t)r * 2 * d + d + i] = e[i];
-    xin[plane + (size_t)r * 2 * d + d + i] = __float2bfloat16(0.f);
+#pragma unroll 2
+  for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
+    float4 fv = *reinterpret_cast<const float4 *>(f + i);
+    if (ssq) {
+      const float4 g = *reinterpret_cast<const float4 *>(gain + i);
+      fv = make_float4(fv.x * rs * g.x, fv.y * rs * g.y, fv.z * rs * g.z, fv.w * rs * g.w);
+    }
+    store_limbs4(xin, plane, (size_t)r * 2 * d + i, fv);
+    *reinterpret_cast<uint2 *>(xin + (size_t)r * 2 * d + d + i) = *reinterpret_cast<const uint2 *>(e + i);
+    *reinterpret_cast<uint2 *>(xin + plane + (size_t)r * 2 * d + d + i) = make_uint2(0u, 0u);
   }
 }
 
@@ -116,7 +119,9 @@ __global__ void save_draft_out_kernel(const float *__restrict__ x, const int *__
   const int r = blockIdx.x;
   const int dst = dst_row[r];
   if (dst < 0) return;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) dout[(size_t)dst * d + i] = x[(size_t)r * d + i];
+#pragma unroll 2
+  for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4)
+    *reinterpret_cast<float4 *>(dout + (size_t)dst * d + i) = *reinterpret_cast<const float4 *>(x + (size_t)r * d + i);
 }
 
 // dst_row for the catch-up call: last pending row of episode i -> dout row e * SV_MAX_TREE.
@@ -282,7 +287,11 @@ accept_select_kernel(EpArgs ea, DevTree *trees, EpState *st, const int *__restri
     const float *src = x + row * d;
     const float rs = norm_scale(ssq, nt, row, d, eps);
     float *dst = pend_feat + (size_t)(e * SV_MAX_PENDING + k) * d;
-    for (int i = threadIdx.x; i < d; i += blockDim.x) dst[i] = src[i] * rs * gain[i];
+    for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
+      const float4 v = *reinterpret_cast<const float4 *>(src + i);
+      const float4 g = *reinterpret_cast<const float4 *>(gain + i);
+      *reinterpret_cast<float4 *>(dst + i) = make_float4(v.x * rs * g.x, v.y * rs * g.y, v.z * rs * g.z, v.w * rs * g.w);
+    }
   }
 }
 
@@ -342,7 +351,11 @@ __global__ void prefill_commit_kernel(EpArgs a, EpState *st,
   const float *src = x + row * d;
   const float rs = norm_scale(ssq, nt, row, d, eps);
   float *dst = pend_feat + (size_t)e * SV_MAX_PENDING * d;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) dst[i] = src[i] * rs * gain[i];
+  for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
+    const float4 v = *reinterpret_cast<const float4 *>(src + i);
+    const float4 g = *reinterpret_cast<const float4 *>(gain + i);
+    *reinterpret_cast<float4 *>(dst + i) = make_float4(v.x * rs * g.x, v.y * rs * g.y, v.z * rs * g.z, v.w * rs * g.w);
+  }
 }
 
 }  // namespace tree
