@@ -195,8 +195,9 @@ int specvla_read_kv(specvla_ctx *ctx, int draft, int episode, int layer, int whi
 /* Y[T, N] (f32, device) = X[T, K] (f32, device) * W[N, K]^T (bf16, device): the library's
  * weight-streaming GEMM exposed for kernel-level parity tests and roofline measurement. As in
  * the decoder, X enters the tensor cores as two bf16 limbs (hi + lo), so the result carries
- * about 16 mantissa bits of X. K % 8 == 0.
- * scratch: device, 1024-byte aligned, at least specvla_gemm_scratch_bytes(T, N, K) bytes. */
+ * about 16 mantissa bits of X. K % 8 == 0, N % 4 == 0.
+ * scratch: device, 1024-byte aligned, at least specvla_gemm_scratch_bytes(T, N, K) bytes (a
+ * status word and the two bf16 limbs of X). */
 size_t specvla_gemm_scratch_bytes(int T, int N, int K);
 int specvla_gemm(const float *X, const void *W, float *Y, int T, int N, int K,
                  void *scratch, size_t scratch_bytes, void *stream);

@@ -59,28 +59,7 @@ struct DevTree {
   uint32_t dmask[SV_MAX_TREE][4]; // ancestors-and-self over draft rows (draft mask), by draft row
 };
 
-// How a GEMM's partial sums are spread over planes part[plane][row][column].
-// uniform > 0: every column has exactly `uniform` planes (plain split-K).
-// uniform == 0: stream-K. The matrix is cut into tiles of SV_TILE_ROWS output columns x KB
-// blocks of K; the U = tiles * KB units, tile-major, are dealt to G CTAs in equal contiguous
-// ranges, and CTA c writes its share of tile t to plane c - (first CTA touching t).
-#define SV_TILE_ROWS 256
-struct SegPlan {
-  int uniform;
-  int G;        // CTAs
-  int KB;       // K blocks per tile
-  int U;        // units = tiles * KB
-};
-// CTA whose range [c * U / G, (c + 1) * U / G) contains unit u.
-__host__ __device__ inline int owner_of(const SegPlan &p, long long u) {
-  return (int)(((u + 1) * p.G - 1) / p.U);
-}
-// Planes holding partial sums of output column n.
-__host__ __device__ inline int nseg_of(const SegPlan &p, int n) {
-  if (p.uniform) return p.uniform;
-  const long long f = (long long)(n / SV_TILE_ROWS) * p.KB;
-  return owner_of(p, f + p.KB - 1) - owner_of(p, f) + 1;
-}
+#define SV_TILE_ROWS 256         // output columns per GEMM tile
 
 // Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may
 // start while its predecessor still runs; nothing the predecessor wrote may be touched before

@@ -203,10 +203,11 @@ argmax_kernel(const float *__restrict__ logits, int V, int lo, int hi, int *__re
   }
 }
 
-// Draft scoring per row of logits [T][V]: log-softmax over [lo, hi) and its top-K entries
-// (ties to the lowest id), K = SV_TOPK. Selection by K rounds of block argmax.
+// Draft scoring per row of logits [T][V]: log-softmax over columns [lo, hi) and its top-K
+// entries (ties to the lowest id), K = SV_TOPK. Column c stands for token tok_offset + c (the
+// logits may cover only a slice of the vocabulary). Selection by K rounds of block argmax.
 __global__ void __launch_bounds__(THREADS)
-logsoftmax_topk_kernel(const float *__restrict__ logits, int V, int lo, int hi,
+logsoftmax_topk_kernel(const float *__restrict__ logits, int V, int lo, int hi, int tok_offset,
                        int *__restrict__ top_tok, float *__restrict__ top_lp) {
   __shared__ float redf[32];
   __shared__ float sv[THREADS / 32];
@@ -249,7 +250,7 @@ logsoftmax_topk_kernel(const float *__restrict__ logits, int V, int lo, int hi,
       for (int w = 1; w < THREADS / 32; w++)
         if (sv[w] > bv || (sv[w] == bv && si[w] < bi)) { bv = sv[w]; bi = si[w]; }
       chosen[k] = bi;
-      top_tok[t * SV_TOPK + k] = bi;
+      top_tok[t * SV_TOPK + k] = bi + tok_offset;
       top_lp[t * SV_TOPK + k] = bv - lse;
     }
     __syncthreads();

@@ -1,0 +1,409 @@
+// Weight-streaming GEMM, one 256-column output tile per CTA or per small cluster of CTAs.
+//
+// A B200 SM can pull well over 100 GB/s through TMA, so ~64 streaming CTAs already saturate
+// HBM: there is no need to spread a matrix over all 148 SMs. Every GEMM of the decoder is
+// therefore cut into whole tiles first (LM head: 126 tiles = 126 CTAs, gate/up: 86, each
+// finishing its tile straight from TMEM with the fused epilogue), and only matrices with few
+// tiles are split along K as well: the S (<= 4) CTAs that share a tile form one thread-block
+// cluster, CTA r streams K blocks [r KB / S, (r + 1) KB / S) through the TMA ring / tcgen05
+// pipeline, drops its fp32 partial tile into its own shared memory, and after one cluster
+// barrier every CTA finishes the rows t = r, r + S, ... of the tile, reading the S partials
+// over DSMEM in rank order (deterministic). Nothing is parked in global memory, the epilogue
+// work is spread over all CTAs, and a second cluster barrier keeps every CTA's shared memory
+// alive until its peers have read it.
+//
+// Pipeline inside a CTA (as in gemm_tc.cuh, whose helpers are used): thread 0 issues the
+// weight ring before the rest of the set-up and before griddepcontrol.wait, warp 0 keeps it
+// full, warp 1 issues the MMAs (both limbs of X as one operand up to 64 rows), warps 2-9 run
+// the epilogue: row scale of the preceding RMSNorm, or residual add + gain + two-limb split +
+// sums of squares for the next norm, or SwiGLU.
+//
+// Waits on mbarriers are bounded as in gemm_tc; the cluster barriers are hardware barriers
+// between co-scheduled CTAs and every path through the kernel reaches both of them.
+#pragma once
+#include <cooperative_groups.h>
+
+#include "gemm_tc.cuh"
+
+namespace gemm_ck {
+
+using namespace gemm_tc;
+
+constexpr int MAX_S = 8;                   // largest cluster = K slices per tile (portable limit)
+
+__device__ __forceinline__ uint32_t cluster_size() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__host__ __device__ constexpr int ck_tmem_cols(int TN) { return 2 * acc_width(TN) < 32 ? 32 : 2 * acc_width(TN); }
+
+// EpiArgs as in gemm_tc (EPI_PLAIN or EPI_RESID; part / counters unused). KB = K blocks per tile.
+template <int TN>
+__global__ void __launch_bounds__(THREADS, 1)
+gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
+               const EpiArgs ea, const int KB, int *__restrict__ err) {
+  constexpr int STAGES = stages_of(TN);
+  constexpr int STAGE = stage_bytes(TN);
+  constexpr bool MERGE = merged_limbs(TN);
+  constexpr int AW = acc_width(TN);
+  constexpr uint32_t IDESC = instr_desc(AW);
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bars = base + STAGES * STAGE;
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
+  const uint32_t tfull_bar = bars + 8u * (2 * STAGES);
+  const uint32_t tmem_slot = bars + 8u * (2 * STAGES + 1);
+  __shared__ float s_scale[MAX_T];
+  __shared__ float s_red[8][MAX_T];
+  __shared__ int s_flag[8];
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int S = (int)cluster_size();
+  const int rank = (int)cluster_rank();
+  const bool swiglu = ea.mode == EPI_SWIGLU;
+  const int tile = blockIdx.x / S;
+  const int kb0 = rank * KB / S, kb1 = (rank + 1) * KB / S;
+  const int n_units = kb1 - kb0;
+  const long long u0 = (long long)tile * KB + kb0;
+  const int T = ea.T;
+  const int tiles = gridDim.x / S;
+
+  const int npre = n_units < STAGES ? n_units : STAGES;
+  uint64_t pol_w = 0;
+  auto load_w = [&](int it) {
+    const int st = it % STAGES;
+    const uint32_t sW = base + st * STAGE;
+    mbar_expect_tx(full_bar(st), STAGE);
+    if (ea.wpacked) {
+      bulk_load(sW, ea.wpacked + (size_t)(u0 + it) * (BM * BK), W_STAGE_BYTES, full_bar(st), pol_w);
+    } else {
+      // the two 128-row halves of the tile: consecutive rows, or gate rows + up rows
+      const int ya = swiglu ? tile * 128 : tile * BM;
+      const int yb = swiglu ? ea.up_off + tile * 128 : tile * BM + 128;
+      tma_load_2d(sW, &tmW, (kb0 + it) * BK, ya, full_bar(st), pol_w);
+      tma_load_2d(sW + 128 * BK * 2, &tmW, (kb0 + it) * BK, yb, full_bar(st), pol_w);
+    }
+  };
+  if (threadIdx.x == 0) {
+    prefetch_tensormap(&tmX);
+    if (!ea.wpacked) prefetch_tensormap(&tmW);
+    for (int s = 0; s < STAGES; s++) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    mbar_init(tfull_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    grid_dep_launch();
+    pol_w = policy_evict_first();
+    for (int it = 0; it < npre; it++) load_w(it);
+  }
+  if (warp == 1) {
+    tc_alloc(tmem_slot, ck_tmem_cols(TN));
+    tc_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  uint32_t tmem_base;
+  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0 && n_units > 0) {
+      const uint64_t pol_x = policy_evict_last();
+      grid_dep_wait();
+      for (int j = 0; j < npre; j++)
+        tma_load_3d(base + j * STAGE + W_STAGE_BYTES, &tmX, (kb0 + j) * BK, ea.row0, 0, full_bar(j), pol_x);
+      for (int it = npre; it < n_units; it++) {
+        const int st = it % STAGES, rnd = it / STAGES;
+        if (!mbar_wait(empty_bar(st), (rnd - 1) & 1)) {
+          atomicExch(err, SV_ERR_WAIT_EMPTY);
+          break;
+        }
+        load_w(it);
+        tma_load_3d(base + st * STAGE + W_STAGE_BYTES, &tmX, (kb0 + it) * BK, ea.row0, 0, full_bar(st), pol_x);
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0 && n_units > 0) {
+      for (int it = 0; it < n_units; it++) {
+        const int st = it % STAGES, rnd = it / STAGES;
+        if (!mbar_wait(full_bar(st), rnd & 1)) {
+          atomicExch(err, SV_ERR_WAIT_FULL);
+          break;
+        }
+        tc_fence_after();
+        const uint32_t sW = base + st * STAGE, sX = sW + W_STAGE_BYTES;
+#pragma unroll
+        for (int kk = 0; kk < BK / 16; kk++) {
+#pragma unroll
+          for (int h = 0; h < 2; h++) {
+            const uint64_t adesc = smem_desc(sW + h * (128 * BK * 2) + kk * 32);
+            const uint32_t d = tmem_base + (uint32_t)(h * AW);
+            if (MERGE) {
+              tc_mma(d, adesc, smem_desc(sX + kk * 32), IDESC, (it == 0 && kk == 0) ? 0u : 1u);
+            } else {
+#pragma unroll
+              for (int limb = 0; limb < 2; limb++) {
+                const uint64_t bdesc = smem_desc(sX + limb * (TN * BK * 2) + kk * 32);
+                tc_mma(d, adesc, bdesc, IDESC, (it == 0 && kk == 0 && limb == 0) ? 0u : 1u);
+              }
+            }
+          }
+        }
+        tc_commit(empty_bar(st));
+        if (it == n_units - 1) tc_commit(tfull_bar);
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------------ epilogue, part 1:
+    // accumulator -> this CTA's partial tile P[t][256] in shared memory (the ring is idle by then)
+    grid_dep_wait();
+    const int q = warp & 3, wp = (warp - 2) >> 2;
+    const int et = threadIdx.x - 64;
+    if (et < T) {
+      float sc = 1.f;
+      if (ea.ssq_in) {
+        float ss = 0.f;
+        for (int j = 0; j < ea.nt_in; j++) ss += ea.ssq_in[(size_t)(ea.row0 + et) * ea.nt_in + j];
+        sc = rsqrtf(ss * ea.inv_k + ea.eps);
+      }
+      s_scale[et] = sc;
+    }
+    bool have = n_units > 0;
+    if (have) {
+      const bool mine = mbar_wait(tfull_bar, 0);
+      if (lane == 0) s_flag[warp - 2] = mine ? 1 : 0;
+      epi_barrier();
+      have = s_flag[0] && s_flag[1] && s_flag[2] && s_flag[3] && s_flag[4] && s_flag[5] && s_flag[6] && s_flag[7];
+      if (!have && et == 0) atomicExch(err, SV_ERR_WAIT_TMEM_FULL);
+      tc_fence_after();
+    }
+    const uint32_t tadr = tmem_base + ((uint32_t)(q * 32) << 16);
+    const int col = q * 32 + lane;                       // column within a 128-column half
+#pragma unroll 1
+    for (int c0 = 16 * wp; c0 < TN; c0 += 32) {
+#pragma unroll 1
+      for (int hf = 0; hf < 2; hf++) {
+        float v[16];
+        if (have) {
+          uint32_t r0[16];
+          tc_ld16(tadr + hf * AW + c0, r0);
+          if (MERGE) {
+            uint32_t r1[16];
+            tc_ld16(tadr + hf * AW + TN + c0, r1);
+            tc_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 16; j++) v[j] = __uint_as_float(r0[j]) + __uint_as_float(r1[j]);
+          } else {
+            tc_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 16; j++) v[j] = __uint_as_float(r0[j]);
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; j++) v[j] = 0.f;
+        }
+#pragma unroll
+        for (int j = 0; j < 16; j++)
+          if (c0 + j < T) {
+            const uint32_t a = base + (uint32_t)(((c0 + j) * BM + hf * 128 + col) * 4);
+            asm volatile("st.shared.f32 [%0], %1;" ::"r"(a), "f"(v[j]) : "memory");
+          }
+      }
+    }
+    tc_fence_before();
+  }
+
+  // every CTA's partial tile is in place
+  if (S > 1) cluster_sync_all(); else __syncthreads();
+
+  if (warp >= 2) {
+    // ------------------------------------------------------------------ epilogue, part 2:
+    // rows rank, rank + S, ... of the tile. A thread owns four consecutive columns (64 column
+    // groups) and every fourth of those rows; the S partials are added in rank order. The
+    // code is kept small on purpose: it runs once per CTA, straight from a cold instruction
+    // cache.
+    const int et = threadIdx.x - 64;
+    const int rg = et >> 6, cg = et & 63;                // row group 0..3, column group 0..63
+    const int c4 = swiglu ? (cg & 31) * 4 : cg * 4;      // first of the four columns within the tile
+    const int n = swiglu ? tile * 128 + c4 : tile * BM + c4;
+    const bool col_ok = n < ea.N && !(swiglu && cg >= 32);   // N % 4 == 0: all four or none
+    const float *P_own = reinterpret_cast<const float *>(smem_raw + (base - smem_u32(smem_raw)));
+    const float *P_of[MAX_S];
+    {
+      cooperative_groups::cluster_group cluster = cooperative_groups::this_cluster();
+#pragma unroll
+      for (int sl = 0; sl < MAX_S; sl++)
+        P_of[sl] = S == 1 ? P_own
+                          : cluster.map_shared_rank(const_cast<float *>(P_own), (unsigned)(sl < S ? sl : S - 1));
+    }
+    float4 gain = make_float4(1.f, 1.f, 1.f, 1.f);
+    if (ea.mode == EPI_RESID && ea.gain && col_ok) gain = *reinterpret_cast<const float4 *>(ea.gain + n);
+    auto partial_sum = [&](int off) {
+      float4 acc = *reinterpret_cast<const float4 *>(P_of[0] + off);
+      if (S > 1) {
+        float4 p[MAX_S];
+#pragma unroll
+        for (int sl = 1; sl < MAX_S; sl++) p[sl] = *reinterpret_cast<const float4 *>(P_of[sl] + off);
+#pragma unroll
+        for (int sl = 1; sl < MAX_S; sl++)
+          if (sl < S) {
+            acc.x += p[sl].x;
+            acc.y += p[sl].y;
+            acc.z += p[sl].z;
+            acc.w += p[sl].w;
+          }
+      }
+      return acc;
+    };
+#pragma unroll 2
+    for (int t = rank + rg * S; t < T; t += 4 * S) {
+      const size_t row = (size_t)(ea.row0 + t);
+      const float sc = s_scale[t];
+      float4 v = partial_sum(t * BM + c4);
+      if (ea.mode == EPI_PLAIN) {
+        if (col_ok)
+          *reinterpret_cast<float4 *>(ea.out + row * ea.ldo + n) = make_float4(sc * v.x, sc * v.y, sc * v.z, sc * v.w);
+      } else if (swiglu) {
+        const float4 u = partial_sum(t * BM + 128 + c4);
+        if (col_ok) {
+          const float gx = sc * v.x, gy = sc * v.y, gz = sc * v.z, gw = sc * v.w;
+          store_limbs4(ea.hid, ea.hid_plane, row * ea.N + n,
+                       make_float4(gx / (1.f + expf(-gx)) * (sc * u.x), gy / (1.f + expf(-gy)) * (sc * u.y),
+                                   gz / (1.f + expf(-gz)) * (sc * u.z), gw / (1.f + expf(-gw)) * (sc * u.w)));
+        }
+      } else {
+        float s2 = 0.f;
+        if (col_ok) {
+          float *xp = ea.x + row * ea.N + n;
+          if (ea.accumulate) {
+            const float4 xo = *reinterpret_cast<const float4 *>(xp);
+            v.x += xo.x;
+            v.y += xo.y;
+            v.z += xo.z;
+            v.w += xo.w;
+          }
+          *reinterpret_cast<float4 *>(xp) = v;
+          store_limbs4(ea.xn, ea.xn_plane, row * ea.N + n,
+                       make_float4(v.x * gain.x, v.y * gain.y, v.z * gain.z, v.w * gain.w));
+          s2 = (v.x * v.x + v.y * v.y) + (v.z * v.z + v.w * v.w);
+        }
+        s2 = warp_sum(s2);
+        if (lane == 0) s_red[warp - 2][t] = s2;
+      }
+    }
+    if (ea.mode == EPI_RESID) {
+      epi_barrier();
+      // thread i finishes this CTA's i-th row, which row group i % 4 (two warps) handled
+      const int t = rank + et * S;
+      if (t < T) {
+        const int w0 = 2 * (et & 3);
+        ea.ssq_out[(size_t)(ea.row0 + t) * tiles + tile] = s_red[w0][t] + s_red[w0 + 1][t];
+      }
+    }
+  }
+
+  // nobody leaves while a peer may still be reading its shared memory
+  if (S > 1) cluster_sync_all();
+
+  if (*reinterpret_cast<volatile int *>(err) != 0) {
+    const uint64_t t0 = global_ns();
+    while (global_ns() - t0 < 200000ull) __nanosleep(1000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 1) tc_dealloc(tmem_base, ck_tmem_cols(TN));
+}
+
+template <int TN>
+inline cudaError_t launch_tn(const CUtensorMap &tmW, const CUtensorMap &tmX, const EpiArgs &ea, int tiles, int KB,
+                             int S, int *err, cudaStream_t st, bool pdl) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_ck_kernel<TN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         smem_bytes(TN));
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(tiles * S);
+  cfg.blockDim = dim3(THREADS);
+  cfg.dynamicSmemBytes = smem_bytes(TN);
+  cfg.stream = st;
+  cudaLaunchAttribute at[2];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = S;
+  at[0].val.clusterDim.y = 1;
+  at[0].val.clusterDim.z = 1;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = pdl ? 2 : 1;
+  return cudaLaunchKernelEx(&cfg, gemm_ck_kernel<TN>, tmW, tmX, ea, KB, err);
+}
+
+// How many clusters of each size 1..MAX_S can be resident at once (index = size; 0 = unknown).
+struct ClusterFit {
+  int max_active[MAX_S + 1];
+};
+// Asks the occupancy calculator about the TN = 32 instantiation (all instantiations use about
+// the same shared memory and one CTA per SM).
+inline ClusterFit query_cluster_fit() {
+  ClusterFit f = {};
+  cudaFuncSetAttribute(gemm_ck_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(32));
+  for (int S = 1; S <= MAX_S; S++) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(S * 64);
+    cfg.blockDim = dim3(THREADS);
+    cfg.dynamicSmemBytes = smem_bytes(32);
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = S;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_ck_kernel<32>, &cfg) == cudaSuccess) f.max_active[S] = n;
+  }
+  cudaGetLastError();
+  return f;
+}
+// K slices per tile: the largest cluster size whose `tiles` clusters are all resident at once
+// (a second wave would double the time), each slice keeping at least four K blocks.
+inline int slices_for(int tiles, int KB, const ClusterFit &fit) {
+  int best = 1;
+  for (int S = 2; S <= MAX_S; S++)
+    if (fit.max_active[S] >= tiles && KB / S >= 4) best = S;
+  return best;
+}
+
+// One launch over ea.T <= 128 rows; tmX must have been made with TN = tn_of(ea.T).
+inline cudaError_t launch(const CUtensorMap &tmW, const CUtensorMap &tmX, const EpiArgs &ea, int tiles, int KB,
+                          int S, int *err, cudaStream_t st, bool pdl) {
+  switch (tn_of(ea.T)) {
+    case 16: return launch_tn<16>(tmW, tmX, ea, tiles, KB, S, err, st, pdl);
+    case 32: return launch_tn<32>(tmW, tmX, ea, tiles, KB, S, err, st, pdl);
+    case 64: return launch_tn<64>(tmW, tmX, ea, tiles, KB, S, err, st, pdl);
+    default: return launch_tn<128>(tmW, tmX, ea, tiles, KB, S, err, st, pdl);
+  }
+}
+
+}  // namespace gemm_ck

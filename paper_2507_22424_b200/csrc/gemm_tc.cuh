@@ -1,29 +1,23 @@
-// Skinny weight-streaming GEMM on the sm_100a tensor cores (tcgen05 + TMEM, operands by TMA).
-//   part[seg][t][n] = sum over a K range of (Xhi[t][k] + Xlo[t][k]) * W[n][k]     (fp32 acc)
-// for T <= 128 activation rows: the verification forward over one draft tree and every
-// draft-model level. At these sizes the cost is the single pass over W, so the kernel is
-// built around keeping every SM's share of that stream in flight:
+// Building blocks of the weight-streaming GEMM on the sm_100a tensor cores (tcgen05 + TMEM,
+// operands by TMA); the kernel itself is in gemm_ck.cuh.
+//   Y[t][n] = sum_k (Xhi[t][k] + Xlo[t][k]) * W[n][k]        (fp32 accumulate)
+// for T <= 128 activation rows per launch: the verification forward over one draft tree, every
+// draft-model level, and the prefill in launches of 128 rows. At these sizes the cost is the
+// single pass over W, so everything is built around streaming W:
 //
-//  * W [N, K] (bf16, K contiguous) is cut into tiles of 256 rows x 64 columns (32 KB, one TMA
-//    box, 128-byte swizzle). The tile sits on the MMA's M axis (two M = 128 halves), the
-//    activation rows on its N axis (TN = T rounded up to 16/32/64/128). Both bf16 limbs of
-//    X are multiplied against the same W tile into the same TMEM accumulator, so fp32-grade
-//    activations cost no extra bytes of the weight stream.
-//  * The tiles x K-blocks form one linear list of units (tile-major, K inner) that is cut
-//    into gridDim.x equal contiguous ranges, one per CTA (one CTA per SM). A CTA therefore
-//    covers the end of one tile, some whole tiles and the start of another. A tile covered by
-//    one CTA is finished straight from TMEM. Otherwise every (CTA, tile) segment writes its
-//    partial sum to plane `seg` = CTA - first CTA of that tile and bumps the tile's counter;
-//    the CTA that arrives last adds the planes in ascending order (so the result does not
-//    depend on which CTA that is) and finishes the tile. Nobody waits for anybody.
-//  * "Finishing" a tile is the fused epilogue: plain store with the RMSNorm row scale, or
-//    residual add + gain + two-limb split + sum of squares for the next norm, or SwiGLU.
-//  * Warp 0 issues TMA loads into a ring of stages, warp 1 issues the MMAs and releases
-//    stages through tcgen05.commit, warps 2-9 run the epilogue on finished accumulators
-//    (double-buffered in TMEM).
-//  * The weight loads of the first ring-full do not depend on the previous kernel, so they
-//    are issued BEFORE griddepcontrol.wait: launched with programmatic stream serialisation
-//    the kernel streams weights while its predecessor drains.
+//  * W [N, K] (bf16, K contiguous) is cut into tiles of 256 rows x 64 columns (32 KB, 128-byte
+//    swizzle). A tile sits on the MMA's M axis (two M = 128 halves), the activation rows on its
+//    N axis (TN = T rounded up to 16/32/64/128). Both bf16 limbs of X are multiplied against
+//    the same W tile (as one operand of 2 TN rows up to TN = 64), so fp32-grade activations
+//    cost no extra bytes of the weight stream.
+//  * The library keeps its own repacked copy of every weight matrix (pack_weights_kernel):
+//    one contiguous 32 KB block per (tile, K block) in streaming order, already swizzled, so
+//    a CTA's share of the stream is one contiguous range of HBM fetched by plain bulk copies.
+//  * The epilogue is fused (EpiArgs): plain store with the RMSNorm row scale, or residual add
+//    + gain + two-limb split + sums of squares for the next norm, or SwiGLU.
+//  * The first ring-full of weight loads does not depend on the previous kernel, so it is
+//    issued BEFORE griddepcontrol.wait: launched with programmatic stream serialisation a GEMM
+//    streams weights while its predecessor drains.
 //
 // Every mbarrier wait is bounded (two seconds of %globaltimer); on expiry the kernel records
 // a code in *err, lets copies in flight land, frees its TMEM and returns.
@@ -53,25 +47,6 @@ __host__ __device__ constexpr int smem_bytes(int TN) { return stages_of(TN) * st
 __host__ __device__ constexpr bool merged_limbs(int TN) { return TN <= 64; }
 __host__ __device__ constexpr int acc_width(int TN) { return merged_limbs(TN) ? 2 * TN : TN; }
 __host__ __device__ constexpr int tmem_cols(int TN) { return 4 * acc_width(TN); }      // 128, 256, 512, 512
-
-// tiles: 256-column tiles of the output (for SwiGLU: 128 gate + 128 up columns each).
-inline SegPlan make_plan(int tiles, int K, int num_sms) {
-  SegPlan p;
-  p.uniform = 0;
-  p.KB = (K + BK - 1) / BK;
-  p.U = tiles * p.KB;
-  p.G = p.U < num_sms ? p.U : num_sms;
-  return p;
-}
-// Largest number of planes any tile needs under `p`.
-inline int max_segments(const SegPlan &p) {
-  int m = 1;
-  for (int t = 0; t < p.U / p.KB; t++) {
-    const int s = nseg_of(p, t * BM);
-    if (s > m) m = s;
-  }
-  return m;
-}
 
 // ------------------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -143,6 +118,7 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_
 }
 __device__ __forceinline__ void grid_dep_wait() { pdl_wait(); }
 __device__ __forceinline__ void grid_dep_launch() { pdl_launch(); }
+// barrier among the 256 epilogue threads (warps 2-9)
 __device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *tm) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(tm) : "memory");
@@ -213,8 +189,6 @@ struct EpiArgs {
   int up_off;            // EPI_SWIGLU: row of W where the up projection starts (F)
   const bf16 *wpacked;   // weights repacked by pack_weights_kernel (one contiguous 32 KB block per
                          // (tile, K block), in unit order); NULL: strided boxes through the W map
-  float *part;           // planes [max segments][T][tiles * 256] for tiles shared by several CTAs
-  int *counters;         // [tiles] arrivals per shared tile; zero between launches
   // row scale of the RMSNorm in front of this GEMM: rsqrt(sum_j ssq_in[row][j] * inv_k + eps)
   const float *ssq_in;   // [rows][nt_in] partial sums of squares; NULL: scale 1
   int nt_in;
@@ -238,381 +212,6 @@ __device__ __forceinline__ void store_limbs(bf16 *hi_plane, size_t plane, size_t
   const bf16 hi = __float2bfloat16(v);
   hi_plane[idx] = hi;
   hi_plane[plane + idx] = __float2bfloat16(v - __bfloat162float(hi));
-}
-
-template <int TN>
-__global__ void __launch_bounds__(THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
-               const EpiArgs ea, const SegPlan plan, int *__restrict__ err) {
-  constexpr int STAGES = stages_of(TN);
-  constexpr int STAGE = stage_bytes(TN);
-  constexpr bool MERGE = merged_limbs(TN);
-  constexpr int AW = acc_width(TN);
-  constexpr uint32_t IDESC = instr_desc(AW);
-  extern __shared__ unsigned char smem_raw[];
-  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t bars = base + STAGES * STAGE;
-  auto full_bar = [&](int s) { return bars + 8u * s; };
-  auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
-  auto tfull_bar = [&](int b) { return bars + 8u * (2 * STAGES + b); };
-  auto tempty_bar = [&](int b) { return bars + 8u * (2 * STAGES + 2 + b); };
-  const uint32_t tmem_slot = bars + 8u * (2 * STAGES + 4);
-  __shared__ float s_scale[MAX_T];        // RMSNorm row scales
-  __shared__ float s_red[4][MAX_T];       // per-warp sums of squares
-  __shared__ int s_flag[8];
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const long long u0 = (long long)blockIdx.x * plan.U / plan.G;
-  const long long u1 = (long long)(blockIdx.x + 1) * plan.U / plan.G;
-  const int n_units = (int)(u1 - u0);
-  const int KB = plan.KB;
-  const int T = ea.T;
-  const bool swiglu = ea.mode == EPI_SWIGLU;
-
-  const int npre = n_units < STAGES ? n_units : STAGES;
-  uint64_t pol_w = 0;
-  auto load_w = [&](int it) {
-    const int st = it % STAGES;
-    const long long u = u0 + it;
-    const int tile = (int)(u / KB), kb = (int)(u % KB);
-    const uint32_t sW = base + st * STAGE;
-    mbar_expect_tx(full_bar(st), STAGE);
-    if (ea.wpacked) {
-      bulk_load(sW, ea.wpacked + (size_t)u * (BM * BK), W_STAGE_BYTES, full_bar(st), pol_w);
-    } else {
-      // the two 128-row halves of the tile: consecutive rows, or gate rows + up rows
-      const int ya = swiglu ? tile * 128 : tile * BM;
-      const int yb = swiglu ? ea.up_off + tile * 128 : tile * BM + 128;
-      tma_load_2d(sW, &tmW, kb * BK, ya, full_bar(st), pol_w);
-      tma_load_2d(sW + 128 * BK * 2, &tmW, kb * BK, yb, full_bar(st), pol_w);
-    }
-  };
-  if (threadIdx.x == 0) {
-    prefetch_tensormap(&tmX);
-    if (!ea.wpacked) prefetch_tensormap(&tmW);
-    for (int s = 0; s < STAGES; s++) {
-      mbar_init(full_bar(s), 1);
-      mbar_init(empty_bar(s), 1);
-    }
-    for (int b = 0; b < 2; b++) {
-      mbar_init(tfull_bar(b), 1);
-      mbar_init(tempty_bar(b), 8);
-    }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    grid_dep_launch();
-    // the first ring-full of weights needs nothing from the previous kernel nor from the rest
-    // of this CTA's set-up: get it moving at once
-    pol_w = policy_evict_first();
-    for (int it = 0; it < npre; it++) load_w(it);
-  }
-  if (warp == 1) {
-    tc_alloc(tmem_slot, tmem_cols(TN));
-    tc_relinquish();
-  }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  uint32_t tmem_base;
-  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
-
-  if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
-    if (lane == 0 && n_units > 0) {
-      const uint64_t pol_x = policy_evict_last();
-      // the activations are the previous kernel's output: wait for it only now
-      grid_dep_wait();
-      for (int j = 0; j < npre; j++)
-        tma_load_3d(base + j * STAGE + W_STAGE_BYTES, &tmX, (int)((u0 + j) % KB) * BK, ea.row0, 0, full_bar(j),
-                    pol_x);
-      for (int it = npre; it < n_units; it++) {
-        const int st = it % STAGES, rnd = it / STAGES;
-        if (!mbar_wait(empty_bar(st), (rnd - 1) & 1)) {
-          atomicExch(err, SV_ERR_WAIT_EMPTY);
-          break;
-        }
-        load_w(it);
-        tma_load_3d(base + st * STAGE + W_STAGE_BYTES, &tmX, (int)((u0 + it) % KB) * BK, ea.row0, 0,
-                    full_bar(st), pol_x);
-      }
-    }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0 && n_units > 0) {
-      int sidx = -1;                 // segment number; accumulator buffer = sidx & 1
-      int prev_tile = -1;
-      for (int it = 0; it < n_units; it++) {
-        const int st = it % STAGES, rnd = it / STAGES;
-        const long long u = u0 + it;
-        const int tile = (int)(u / KB);
-        const bool first = tile != prev_tile;
-        prev_tile = tile;
-        if (first) {
-          sidx++;
-          // the buffer's previous accumulator (segment sidx - 2) must have been read out
-          if (sidx >= 2 && !mbar_wait(tempty_bar(sidx & 1), ((sidx >> 1) - 1) & 1)) {
-            atomicExch(err, SV_ERR_WAIT_TMEM_EMPTY);
-            break;
-          }
-        }
-        const int buf = sidx & 1;
-        if (!mbar_wait(full_bar(st), rnd & 1)) {
-          atomicExch(err, SV_ERR_WAIT_FULL);
-          break;
-        }
-        tc_fence_after();
-        const uint32_t sW = base + st * STAGE, sX = sW + W_STAGE_BYTES;
-#pragma unroll
-        for (int kk = 0; kk < BK / 16; kk++) {
-#pragma unroll
-          for (int h = 0; h < 2; h++) {
-            const uint64_t adesc = smem_desc(sW + h * (128 * BK * 2) + kk * 32);
-            const uint32_t d = tmem_base + (uint32_t)((buf * 2 + h) * AW);
-            if (MERGE) {
-              tc_mma(d, adesc, smem_desc(sX + kk * 32), IDESC, (first && kk == 0) ? 0u : 1u);
-            } else {
-#pragma unroll
-              for (int limb = 0; limb < 2; limb++) {
-                const uint64_t bdesc = smem_desc(sX + limb * (TN * BK * 2) + kk * 32);
-                tc_mma(d, adesc, bdesc, IDESC, (first && kk == 0 && limb == 0) ? 0u : 1u);
-              }
-            }
-          }
-        }
-        tc_commit(empty_bar(st));
-        const bool last = (it == n_units - 1) || ((int)((u + 1) / KB) != tile);
-        if (last) tc_commit(tfull_bar(buf));
-      }
-    }
-  } else {
-    // ------------------------------------------------------------------ epilogue (warps 2..9)
-    // Two warps per TMEM lane quarter; they take alternate 16-row chunks of the accumulator.
-    grid_dep_wait();
-    const int q = warp & 3;                       // TMEM lane quarter this warp may access
-    const int wp = (warp - 2) >> 2;               // which of the quarter's two warps
-    const int et = threadIdx.x - 64;              // 0..255 among the epilogue threads
-    // accumulator chunk: 16 rows (TMEM columns c0..c0+15 of half hf) of this thread's column
-    auto load_acc = [&](uint32_t tadr, int hf, int c0, float (&v)[16]) {
-      uint32_t r0[16];
-      tc_ld16(tadr + hf * AW + c0, r0);
-      if (MERGE) {
-        uint32_t r1[16];
-        tc_ld16(tadr + hf * AW + TN + c0, r1);
-        tc_wait_ld();
-#pragma unroll
-        for (int j = 0; j < 16; j++) v[j] = __uint_as_float(r0[j]) + __uint_as_float(r1[j]);
-      } else {
-        tc_wait_ld();
-#pragma unroll
-        for (int j = 0; j < 16; j++) v[j] = __uint_as_float(r0[j]);
-      }
-    };
-    const int tiles = plan.U / KB;
-    const int ldp = tiles * BM;                   // row pitch of a plane
-    if (et < T) {
-      float sc = 1.f;
-      if (ea.ssq_in) {
-        float ss = 0.f;
-        for (int j = 0; j < ea.nt_in; j++) ss += ea.ssq_in[(size_t)(ea.row0 + et) * ea.nt_in + j];
-        sc = rsqrtf(ss * ea.inv_k + ea.eps);
-      }
-      s_scale[et] = sc;
-    }
-    epi_barrier();
-
-    int sidx = 0;
-    int it = 0;
-    while (it < n_units) {
-      const int buf = sidx & 1;
-      const long long u = u0 + it;
-      const int tile = (int)(u / KB), kb0 = (int)(u % KB);
-      int cnt = KB - kb0;
-      if (cnt > n_units - it) cnt = n_units - it;
-      // all eight warps take the same decision on the wait
-      const bool mine = mbar_wait(tfull_bar(buf), (sidx >> 1) & 1);
-      if (lane == 0) s_flag[warp - 2] = mine ? 1 : 0;
-      epi_barrier();
-      const bool ok = s_flag[0] && s_flag[1] && s_flag[2] && s_flag[3] && s_flag[4] && s_flag[5] && s_flag[6] &&
-                      s_flag[7];
-      epi_barrier();
-      if (!ok) {
-        if (et == 0) atomicExch(err, SV_ERR_WAIT_TMEM_FULL);
-        break;
-      }
-      tc_fence_after();
-      const int nseg = nseg_of(plan, tile * BM);
-      const int seg = (int)blockIdx.x - owner_of(plan, (long long)tile * KB);
-      // column of this thread inside the tile's plane, and in the output, for the two halves
-      const int pc = tile * BM + q * 32 + lane;                       // plane column of half 0 (+128: half 1)
-      const int na = swiglu ? tile * 128 + q * 32 + lane : pc;       // output column, half 0
-      const int nb = swiglu ? na : pc + 128;                          // output column, half 1
-      const uint32_t tadr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 2 * AW);
-
-      bool finish = true;
-      if (nseg > 1) {
-        // park this segment's partial sums, then see who is last
-        float *pl = ea.part + (size_t)seg * T * ldp;
-#pragma unroll 1
-        for (int c0 = 16 * wp; c0 < TN; c0 += 32) {
-          float ra[16], rb[16];
-          load_acc(tadr, 0, c0, ra);
-          load_acc(tadr, 1, c0, rb);
-#pragma unroll
-          for (int j = 0; j < 16; j++)
-            if (c0 + j < T) {
-              __stcg(pl + (size_t)(c0 + j) * ldp + pc, ra[j]);
-              __stcg(pl + (size_t)(c0 + j) * ldp + pc + 128, rb[j]);
-            }
-        }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(tempty_bar(buf));
-        __threadfence();
-        epi_barrier();
-        if (et == 0) {
-          const int old = atomicAdd(ea.counters + tile, 1);
-          const int lastone = (old == nseg - 1);
-          if (lastone) atomicExch(ea.counters + tile, 0);
-          s_flag[0] = lastone;
-        }
-        epi_barrier();
-        finish = s_flag[0] != 0;
-        epi_barrier();
-        if (finish) __threadfence();
-      }
-
-      if (finish) {
-        float sq[8];                 // EPI_RESID: this thread's sums of squares, 8 rows at a time
-#pragma unroll 1
-        for (int c0 = 16 * wp; c0 < TN; c0 += 32) {
-          float va[16], vb[16];
-          if (nseg > 1) {
-            // planes are added in ascending order; two planes (64 independent loads per thread)
-            // are in flight per round
-#pragma unroll
-            for (int j = 0; j < 16; j++) va[j] = vb[j] = 0.f;
-            const float *pl = ea.part + (size_t)c0 * ldp + pc;
-            const size_t pstride = (size_t)T * ldp;
-            int sgn = 0;
-#pragma unroll 1
-            for (; sgn + 1 < nseg; sgn += 2) {
-              float ta[16], tb[16], ua[16], ub[16];
-#pragma unroll
-              for (int j = 0; j < 16; j++) {
-                const bool in = c0 + j < T;
-                const float *p0 = pl + (size_t)sgn * pstride + (size_t)j * ldp;
-                ta[j] = in ? __ldcg(p0) : 0.f;
-                tb[j] = in ? __ldcg(p0 + 128) : 0.f;
-                ua[j] = in ? __ldcg(p0 + pstride) : 0.f;
-                ub[j] = in ? __ldcg(p0 + pstride + 128) : 0.f;
-              }
-#pragma unroll
-              for (int j = 0; j < 16; j++) {
-                va[j] = (va[j] + ta[j]) + ua[j];
-                vb[j] = (vb[j] + tb[j]) + ub[j];
-              }
-            }
-            if (sgn < nseg) {
-#pragma unroll
-              for (int j = 0; j < 16; j++) {
-                const bool in = c0 + j < T;
-                const float *p0 = pl + (size_t)sgn * pstride + (size_t)j * ldp;
-                va[j] += in ? __ldcg(p0) : 0.f;
-                vb[j] += in ? __ldcg(p0 + 128) : 0.f;
-              }
-            }
-          } else {
-            load_acc(tadr, 0, c0, va);
-            load_acc(tadr, 1, c0, vb);
-          }
-          if (ea.mode == EPI_PLAIN) {
-#pragma unroll
-            for (int j = 0; j < 16; j++)
-              if (c0 + j < T) {
-                const float sc = s_scale[c0 + j];
-                float *o = ea.out + (size_t)(ea.row0 + c0 + j) * ea.ldo;
-                if (na < ea.N) o[na] = sc * va[j];
-                if (nb < ea.N) o[nb] = sc * vb[j];
-              }
-          } else if (ea.mode == EPI_SWIGLU) {
-#pragma unroll
-            for (int j = 0; j < 16; j++)
-              if (c0 + j < T && na < ea.N) {
-                const float sc = s_scale[c0 + j];
-                const float g = sc * va[j], up = sc * vb[j];
-                store_limbs(ea.hid, ea.hid_plane, (size_t)(ea.row0 + c0 + j) * ea.N + na,
-                            g / (1.f + expf(-g)) * up);
-              }
-          } else {
-            const float ga = (ea.gain && na < ea.N) ? ea.gain[na] : 1.f;
-            const float gb = (ea.gain && nb < ea.N) ? ea.gain[nb] : 1.f;
-            // all residual loads of the 16 rows first: they are independent of the stores below
-            float xa[16], xb[16];
-#pragma unroll
-            for (int j = 0; j < 16; j++) {
-              const bool in = ea.accumulate && c0 + j < T;
-              const size_t r = (size_t)(ea.row0 + c0 + j) * ea.N;
-              xa[j] = (in && na < ea.N) ? __ldcg(ea.x + r + na) : 0.f;
-              xb[j] = (in && nb < ea.N) ? __ldcg(ea.x + r + nb) : 0.f;
-            }
-#pragma unroll
-            for (int half8 = 0; half8 < 2; half8++) {
-#pragma unroll
-              for (int j8 = 0; j8 < 8; j8++) {
-                const int j = half8 * 8 + j8;
-                float s2 = 0.f;
-                if (c0 + j < T) {
-                  const size_t r = (size_t)(ea.row0 + c0 + j) * ea.N;
-                  if (na < ea.N) {
-                    const float xv = xa[j] + va[j];
-                    ea.x[r + na] = xv;
-                    store_limbs(ea.xn, ea.xn_plane, r + na, xv * ga);
-                    s2 += xv * xv;
-                  }
-                  if (nb < ea.N) {
-                    const float xv = xb[j] + vb[j];
-                    ea.x[r + nb] = xv;
-                    store_limbs(ea.xn, ea.xn_plane, r + nb, xv * gb);
-                    s2 += xv * xv;
-                  }
-                }
-                sq[j8] = s2;
-              }
-#pragma unroll
-              for (int j8 = 0; j8 < 8; j8++) {
-                const float w = warp_sum(sq[j8]);
-                if (lane == 0) s_red[q][c0 + half8 * 8 + j8] = w;
-              }
-            }
-          }
-        }
-        if (nseg == 1) {
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(tempty_bar(buf));
-        }
-        if (ea.mode == EPI_RESID) {
-          epi_barrier();
-          if (et < T)
-            ea.ssq_out[(size_t)(ea.row0 + et) * tiles + tile] =
-                s_red[0][et] + s_red[1][et] + s_red[2][et] + s_red[3][et];
-          epi_barrier();
-        }
-      }
-      sidx++;
-      it += cnt;
-    }
-  }
-
-  if (*reinterpret_cast<volatile int *>(err) != 0) {
-    // a wait gave up somewhere: give copies in flight time to land before the smem goes away
-    const uint64_t t0 = global_ns();
-    while (global_ns() - t0 < 200000ull) __nanosleep(1000);
-  }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  if (warp == 1) tc_dealloc(tmem_base, tmem_cols(TN));
 }
 
 // Repacks W [N, K] (row-major) into the order the kernel streams it: one contiguous 32 KB block
@@ -689,40 +288,6 @@ inline bool make_x_map(CUtensorMap *tm, const bf16 *X, size_t plane, int rows, i
   return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<bf16 *>(X), dims, strides, box, es,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-template <int TN>
-inline cudaError_t launch_tn(const CUtensorMap &tmW, const CUtensorMap &tmX, const EpiArgs &ea,
-                             const SegPlan &plan, int *err, cudaStream_t st, bool pdl) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<TN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         smem_bytes(TN));
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(plan.G);
-  cfg.blockDim = dim3(THREADS);
-  cfg.dynamicSmemBytes = smem_bytes(TN);
-  cfg.stream = st;
-  cudaLaunchAttribute at[1];
-  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  at[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = at;
-  cfg.numAttrs = pdl ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<TN>, tmW, tmX, ea, plan, err);
-}
-
-// One launch over ea.T <= 128 rows; tmX must have been made with TN = tn_of(ea.T).
-inline cudaError_t launch(const CUtensorMap &tmW, const CUtensorMap &tmX, const EpiArgs &ea,
-                          const SegPlan &plan, int *err, cudaStream_t st, bool pdl) {
-  switch (tn_of(ea.T)) {
-    case 16: return launch_tn<16>(tmW, tmX, ea, plan, err, st, pdl);
-    case 32: return launch_tn<32>(tmW, tmX, ea, plan, err, st, pdl);
-    case 64: return launch_tn<64>(tmW, tmX, ea, plan, err, st, pdl);
-    default: return launch_tn<128>(tmW, tmX, ea, plan, err, st, pdl);
-  }
 }
 
 }  // namespace gemm_tc

@@ -13,6 +13,7 @@
 #include "attention.cuh"
 #include "common.cuh"
 #include "epilogue.cuh"
+#include "gemm_ck.cuh"
 #include "gemm_tc.cuh"
 #include "tree.cuh"
 
@@ -41,7 +42,6 @@ struct LayerW {
   const float *norm1, *norm2;
 };
 
-constexpr int MAX_CTAS = 148;     // grid of the tensor-core GEMM assumed when sizing the workspace
 
 constexpr size_t ALIGN = 1024;
 
@@ -67,26 +67,25 @@ struct specvla_ctx {
   LayerW dlayer;
   const bf16 *embed;
   WMat lm_head, draft_fc;
+  WMat lm_head_act;             // rows [action_base, action_base + n_bins) of the LM head (draft scoring)
   const float *final_norm;
   bool has_draft;
-  int num_ctas;                 // CTAs of the GEMM: min(SM count, MAX_CTAS)
   int nt;                       // 256-column tiles of a d_model-wide row (sums-of-squares slots)
   bool use_pdl;                 // programmatic dependent launch between the kernels of a forward
+  gemm_ck::ClusterFit fit;      // clusters of each size that can be resident at once
 
   // workspace carve-up (device)
   float *kv_t, *kv_d;           // target [ep][layer][2][max_seq][hd], draft [ep][2][max_seq][hd], fp32
   size_t kv_t_ep_stride, kv_t_layer_stride, kv_d_ep_stride;
   float2 *rope_tab;
-  float *x, *feat, *part, *lgs, *pend_feat, *dout, *margin, *top_lp, *q, *qkv;
+  float *x, *feat, *lgs, *pend_feat, *dout, *margin, *top_lp, *q, *qkv;
   float *ssq, *lm_ssq;          // per-row partial sums of squares of x / of the gathered LM-head rows
-  int *counters;                // per-tile arrival counters of the GEMM (zero between launches)
   bf16 *packed;                 // repacked weight matrices, one after the other
   size_t packed_elems;
   float *att_part;              // parked key slices of the attention kernel
   int *att_counters;            // its arrival counters (zero between launches)
-  size_t part_floats;
   int lgs_rows;                 // rows of the logits buffer
-  int n_counters;
+
   // GEMM operands, two bf16 limbs each: hi plane, then the lo plane `plane` elements later
   XBuf xn, xin, ao, hid, lm_in;
   int *err;                     // device status word written by bounded waits that gave up
@@ -142,7 +141,7 @@ bool desc_ok(const specvla_model_desc *d) {
   if (!d) return false;
   if (d->n_layers < 1 || d->d_model < 64 || d->n_heads < 1 || d->d_ffn < 8 || d->vocab < 16) return false;
   if (d->head_dim != 64 && d->head_dim != 128) return false;
-  if (d->d_model % 8 || d->d_ffn % 8 || (d->n_heads * d->head_dim) % 8) return false;
+  if (d->d_model % 8 || d->d_ffn % 8 || (d->n_heads * d->head_dim) % 8 || d->vocab % 4 || d->n_bins % 4) return false;
   if (d->n_bins < 1 || d->action_base < 0 || d->action_base + d->n_bins > d->vocab) return false;
   if (d->max_seq < 2 || d->max_episodes < 1 || d->max_episodes > SV_MAX_EP || d->max_rows < 1) return false;
   if (!(d->rms_eps > 0.f) || !(d->rope_theta > 1.f)) return false;
@@ -180,38 +179,21 @@ size_t carve(specvla_ctx *c, char *base) {
   c->nt = (d.d_model + SV_TILE_ROWS - 1) / SV_TILE_ROWS;
   c->ssq = cv.take<float>(R * c->nt);
   c->lm_ssq = cv.take<float>(lm_rows * c->nt);
-  // planes of partial sums for tiles shared by several CTAs: one launch covers <= 128 rows
-  size_t pf = 0;
-  int max_tiles = 1;
-  auto need = [&](int tiles, int K) {
-    const size_t n = (size_t)gemm_tc::max_segments(gemm_tc::make_plan(tiles, K, c->num_ctas)) *
-                     gemm_tc::MAX_T * tiles * SV_TILE_ROWS;
-    if (n > pf) pf = n;
-    if (tiles > max_tiles) max_tiles = tiles;
-  };
   auto tiles256 = [](int N) { return (N + SV_TILE_ROWS - 1) / SV_TILE_ROWS; };
-  need(tiles256(3 * hd), d.d_model);
-  need(tiles256(d.d_model), hd);
-  need((d.d_ffn + 127) / 128, d.d_model);
-  need(tiles256(d.d_model), d.d_ffn);
-  need(tiles256(d.d_model), 2 * d.d_model);
-  need(tiles256(d.vocab), d.d_model);
-  c->part_floats = pf;
-  c->part = cv.take<float>(pf);
   {
-    // repacked weights: every target layer, the LM head, the draft fc and the draft layer
+    // repacked weights: every target layer, the LM head and its action rows, the draft fc and
+    // the draft layer
     const size_t layer = gemm_tc::packed_elems(tiles256(3 * hd), d.d_model) +
                          gemm_tc::packed_elems(tiles256(d.d_model), hd) +
                          gemm_tc::packed_elems((d.d_ffn + 127) / 128, d.d_model) +
                          gemm_tc::packed_elems(tiles256(d.d_model), d.d_ffn);
     c->packed_elems = layer * ((size_t)d.n_layers + 1) + gemm_tc::packed_elems(tiles256(d.vocab), d.d_model) +
+                      gemm_tc::packed_elems(tiles256(d.n_bins), d.d_model) +
                       gemm_tc::packed_elems(tiles256(d.d_model), 2 * d.d_model);
     c->packed = cv.take<bf16>(c->packed_elems);
   }
   c->att_part = cv.take<float>((size_t)attn::MAX_SPLIT_CTAS * attn::RB * (d.head_dim + 2));
   c->att_counters = cv.take<int>(attn::MAX_SPLIT_CTAS);
-  c->n_counters = max_tiles;
-  c->counters = cv.take<int>(max_tiles);
   c->lgs_rows = (int)(lm_rows > dr ? lm_rows : dr);
   c->lgs = cv.take<float>((size_t)c->lgs_rows * d.vocab);
   c->pend_feat = cv.take<float>(E * SV_MAX_PENDING * d.d_model);
@@ -284,25 +266,23 @@ cudaLaunchConfig_t launch_cfg(dim3 grid, dim3 block, cudaStream_t st, cudaLaunch
   } while (0)
 
 // One GEMM over R rows of A against W with the fused epilogue described by `ea` (mode and
-// outputs; row range, planes and counters are filled in here). Rows go in launches of 128.
+// outputs; the row range is filled in here). Rows go in launches of 128.
 int gemm(specvla_ctx *ctx, const XBuf &A, const WMat &W, int R, gemm_tc::EpiArgs ea, cudaStream_t st, int cls) {
   if (!W.has_map || !A.has_map || A.K != W.K) return SPECVLA_ERR_BAD_STATE;
   const bool swiglu = ea.mode == gemm_tc::EPI_SWIGLU;
   const int tiles = swiglu ? (ea.N + 127) / 128 : (W.N + SV_TILE_ROWS - 1) / SV_TILE_ROWS;
-  const SegPlan plan = gemm_tc::make_plan(tiles, W.K, ctx->num_ctas);
-  if ((size_t)gemm_tc::max_segments(plan) * gemm_tc::MAX_T * tiles * SV_TILE_ROWS > ctx->part_floats)
-    return SPECVLA_ERR_CAPACITY;
-  ea.part = ctx->part;
-  ea.counters = ctx->counters;
+  const int KB = (W.K + gemm_tc::BK - 1) / gemm_tc::BK;
   ea.wpacked = W.packed;
   ea.inv_k = 1.f / (float)W.K;
   ea.eps = ctx->desc.rms_eps;
   const bool prof = (ctx->prof_mask & ctx->phase) && 2 * (ctx->prof_used + 1) <= (int)ctx->prof_ev.size();
   if (prof) CU(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used], st));
+  const int S = gemm_ck::slices_for(tiles, KB, ctx->fit);
   for (int r0 = 0; r0 < R; r0 += gemm_tc::MAX_T) {
     ea.row0 = r0;
     ea.T = R - r0 < gemm_tc::MAX_T ? R - r0 : gemm_tc::MAX_T;
-    CU(gemm_tc::launch(W.map, A.map[tn_index(gemm_tc::tn_of(ea.T))], ea, plan, ctx->err, st, ctx->use_pdl));
+    CU(gemm_ck::launch(W.map, A.map[tn_index(gemm_tc::tn_of(ea.T))], ea, tiles, KB, S, ctx->err, st,
+                       ctx->use_pdl));
     ctx->launches++;
   }
   if (prof) {
@@ -491,7 +471,6 @@ size_t specvla_workspace_bytes(const specvla_model_desc *desc) {
   if (!desc_ok(desc)) return 0;
   specvla_ctx tmp{};
   tmp.desc = *desc;
-  tmp.num_ctas = MAX_CTAS;
   derive_caps(&tmp);
   return carve(&tmp, nullptr);
 }
@@ -515,7 +494,6 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
   specvla_ctx *ctx = new (std::nothrow) specvla_ctx();
   if (!ctx) return SPECVLA_ERR_INVALID_ARG;
   ctx->desc = *desc;
-  ctx->num_ctas = prop.multiProcessorCount < MAX_CTAS ? prop.multiProcessorCount : MAX_CTAS;
   derive_caps(ctx);
   const size_t need = carve(ctx, nullptr);
   if (workspace_bytes < need) {
@@ -525,6 +503,12 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
   carve(ctx, static_cast<char *>(workspace));
   const int hd = ctx->hd, D = desc->d_model, F = desc->d_ffn;
   ctx->use_pdl = getenv("SPECVLA_NO_PDL") == nullptr;
+  ctx->fit = gemm_ck::query_cluster_fit();
+  if (getenv("SPECVLA_DEBUG")) {
+    fprintf(stderr, "specvla: resident clusters by size:");
+    for (int i = 1; i <= gemm_ck::MAX_S; i++) fprintf(stderr, " %d:%d", i, ctx->fit.max_active[i]);
+    fprintf(stderr, "\n");
+  }
   size_t packed_used = 0;
   bool pack_ok = true;
   // swiglu: the matrix is [gate; up] stacked ([2F, K]) and is packed as tiles of 128 + 128 rows
@@ -576,6 +560,8 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
   }
   ctx->has_draft = dw && dw->fc && dw->wqkv && dw->wo && dw->wgu && dw->wd && dw->norm1 && dw->norm2;
   if (ctx->has_draft) {
+    // the draft only ranks action tokens when action_only is set: those rows of the LM head suffice
+    ctx->lm_head_act = wmat(static_cast<const bf16 *>(tw->lm_head) + (size_t)desc->action_base * D, desc->n_bins, D);
     ctx->draft_fc = wmat(dw->fc, D, 2 * D);
     ctx->dlayer = LayerW{wmat(dw->wqkv, 3 * hd, D), wmat(dw->wo, D, hd), wmat(dw->wgu, 2 * F, D, true),
                          wmat(dw->wd, D, F), dw->norm1, dw->norm2};
@@ -605,7 +591,6 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
   cudaMemsetAsync(ctx->st, 0, sizeof(EpState) * desc->max_episodes);
   cudaMemsetAsync(ctx->trees, 0, sizeof(DevTree) * desc->max_episodes);
   cudaMemsetAsync(ctx->err, 0, 32 * sizeof(int));
-  cudaMemsetAsync(ctx->counters, 0, ctx->n_counters * sizeof(int));
   cudaMemsetAsync(ctx->att_counters, 0, attn::MAX_SPLIT_CTAS * sizeof(int));
   cudaFuncSetAttribute(attn::tree_attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                        attn::smem_bytes<128>());
@@ -814,9 +799,18 @@ int specvla_draft_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const sp
       A = &ctx->lm_in;
     }
     // the draft layer's output feeds the shared LM head as it is: no norm, no row scale
-    TRY(lm_head(ctx, *A, nullptr, scored_rows, st));
-    LAUNCH(epi::logsoftmax_topk_kernel, dim3(scored_rows), dim3(epi::THREADS), (const float *)ctx->lgs, d.vocab,
-           lo, hi, ctx->top_tok, ctx->top_lp);
+    if (d.action_only) {
+      // log-softmax and top-k range over the action ids only, so only their logits are computed
+      if (scored_rows > ctx->lgs_rows) return SPECVLA_ERR_CAPACITY;
+      TRY(gemm(ctx, *A, ctx->lm_head_act, scored_rows, epi_plain(ctx->lgs, d.n_bins, d.n_bins, nullptr, ctx->nt), st,
+               SPECVLA_PROF_LM_HEAD));
+      LAUNCH(epi::logsoftmax_topk_kernel, dim3(scored_rows), dim3(epi::THREADS), (const float *)ctx->lgs, d.n_bins,
+             0, d.n_bins, d.action_base, ctx->top_tok, ctx->top_lp);
+    } else {
+      TRY(lm_head(ctx, *A, nullptr, scored_rows, st));
+      LAUNCH(epi::logsoftmax_topk_kernel, dim3(scored_rows), dim3(epi::THREADS), (const float *)ctx->lgs, d.vocab,
+             lo, hi, 0, ctx->top_tok, ctx->top_lp);
+    }
     const int cur = (l == 0) ? 1 : shape->expand[l];            // parents scored per episode
     const int next = (l + 1 < shape->depth) ? shape->expand[l + 1] : 0;
     EpArgs la = ea;
@@ -1110,36 +1104,17 @@ int specvla_read_kv(specvla_ctx *ctx, int draft, int episode, int layer, int whi
 }
 
 // ------------------------------------------------------------------ stand-alone GEMM
-// scratch layout: [status word, 1 KB | tile counters, 4 KB | two bf16 limbs of X | planes]
-static const size_t GEMM_HDR = 1024 + 4096;
+// scratch layout: [status word, 1 KB | two bf16 limbs of X]
+static const size_t GEMM_HDR = 1024;
 static size_t gemm_limb_bytes(int T, int K) { return ((size_t)2 * T * K * sizeof(bf16) + 1023) / 1024 * 1024; }
-static int gemm_ctas() {
-  static int n = 0;
-  if (!n) {
-    int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess &&
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
-      n = sms < MAX_CTAS ? sms : MAX_CTAS;
-    else
-      return MAX_CTAS;
-  }
-  return n;
-}
-static size_t gemm_plane_floats(int T, int N, int K) {
-  const int tiles = (N + SV_TILE_ROWS - 1) / SV_TILE_ROWS;
-  const int rows = T < gemm_tc::MAX_T ? T : gemm_tc::MAX_T;
-  return (size_t)gemm_tc::max_segments(gemm_tc::make_plan(tiles, K, gemm_ctas())) * rows * tiles * SV_TILE_ROWS;
-}
-
 size_t specvla_gemm_scratch_bytes(int T, int N, int K) {
-  if (T < 1 || N < 1 || K < 8 || N > 1024 * SV_TILE_ROWS) return 0;
-  return GEMM_HDR + gemm_limb_bytes(T, K) + gemm_plane_floats(T, N, K) * sizeof(float);
+  if (T < 1 || N < 4 || (N % 4) || K < 8) return 0;
+  return GEMM_HDR + gemm_limb_bytes(T, K);
 }
 
 int specvla_gemm(const float *X, const void *W, float *Y, int T, int N, int K, void *scratch,
                  size_t scratch_bytes, void *stream) {
-  if (!X || !W || !Y || !scratch || T < 1 || N < 1 || K < 8 || (K % 8) || N > 1024 * SV_TILE_ROWS)
-    return SPECVLA_ERR_INVALID_ARG;
+  if (!X || !W || !Y || !scratch || T < 1 || N < 4 || (N % 4) || K < 8 || (K % 8)) return SPECVLA_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(scratch) % 1024) != 0) return SPECVLA_ERR_INVALID_ARG;
   if (scratch_bytes < specvla_gemm_scratch_bytes(T, N, K)) return SPECVLA_ERR_CAPACITY;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -1147,7 +1122,7 @@ int specvla_gemm(const float *X, const void *W, float *Y, int T, int N, int K, v
   int *err = reinterpret_cast<int *>(base);
   bf16 *limbs = reinterpret_cast<bf16 *>(base + GEMM_HDR);
   const size_t nx = (size_t)T * K;
-  // status word and tile counters start at zero
+  // the status word starts at zero
   if (cudaMemsetAsync(base, 0, GEMM_HDR, st) != cudaSuccess) return SPECVLA_ERR_CUDA;
   epi::split_limbs_kernel<<<(unsigned)((nx + 255) / 256), 256, 0, st>>>(X, nx, limbs);
   CUtensorMap mw, mx[4];
@@ -1156,18 +1131,19 @@ int specvla_gemm(const float *X, const void *W, float *Y, int T, int N, int K, v
   for (int i = 0; i < 4; i++)
     if (!gemm_tc::make_x_map(&mx[i], limbs, nx, T, K, tns[i])) return SPECVLA_ERR_CUDA;
   const int tiles = (N + SV_TILE_ROWS - 1) / SV_TILE_ROWS;
-  const SegPlan plan = gemm_tc::make_plan(tiles, K, gemm_ctas());
+  const int KB = (K + gemm_tc::BK - 1) / gemm_tc::BK;
   gemm_tc::EpiArgs ea = {};
   ea.mode = gemm_tc::EPI_PLAIN;
   ea.N = N;
   ea.out = Y;
   ea.ldo = N;
-  ea.part = reinterpret_cast<float *>(base + GEMM_HDR + gemm_limb_bytes(T, K));
-  ea.counters = reinterpret_cast<int *>(base + 1024);
+  static const gemm_ck::ClusterFit fit = gemm_ck::query_cluster_fit();
+  const int S = gemm_ck::slices_for(tiles, KB, fit);
   for (int r0 = 0; r0 < T; r0 += gemm_tc::MAX_T) {
     ea.row0 = r0;
     ea.T = T - r0 < gemm_tc::MAX_T ? T - r0 : gemm_tc::MAX_T;
-    if (gemm_tc::launch(mw, mx[tn_index(gemm_tc::tn_of(ea.T))], ea, plan, err, st, false) != cudaSuccess)
+    if (gemm_ck::launch(mw, mx[tn_index(gemm_tc::tn_of(ea.T))], ea, tiles, KB, S, err, st, false) !=
+        cudaSuccess)
       return SPECVLA_ERR_CUDA;
   }
   return cudaGetLastError() == cudaSuccess ? SPECVLA_OK : SPECVLA_ERR_CUDA;
@@ -1183,7 +1159,7 @@ static __device__ __align__(256) unsigned char g_static_scratch[SPECVLA_STATIC_S
 static void *g_static_scratch_addr[64];
 
 int specvla_gemm_static(const float *X, const void *W, float *Y, int T, int N, int K, int wait, void *stream) {
-  if (!X || !W || !Y || T < 1 || N < 1 || K < 8 || (K % 8)) return SPECVLA_ERR_INVALID_ARG;
+  if (!X || !W || !Y || T < 1 || N < 4 || (N % 4) || K < 8 || (K % 8)) return SPECVLA_ERR_INVALID_ARG;
   const size_t need = specvla_gemm_scratch_bytes(T, N, K);
   if (need == 0) return SPECVLA_ERR_INVALID_ARG;
   if (need > (size_t)SPECVLA_STATIC_SCRATCH_BYTES) return SPECVLA_ERR_CAPACITY;

@@ -36,7 +36,7 @@ def test_static_scratch_gemm_matches_allocating_gemm_twice():
 
 def test_static_scratch_gemm_rejects_oversize():
     from paper_2507_22424_b200 import binding as B
-    T, N, K = 128, 32064, 4096
+    T, N, K = 1024, 256, 8192          # the two limbs of X alone need 32 MiB
     assert B.lib.specvla_gemm_scratch_bytes(T, N, K) > B.STATIC_SCRATCH_BYTES
     x = torch.zeros(T, K, dtype=torch.float32, device="cuda")
     w = torch.zeros(N, K, dtype=torch.bfloat16, device="cuda")
