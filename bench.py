@@ -363,6 +363,8 @@ def run_micro(spec: str, steps: int, warmup: int):
     from paper_2507_22424_b200 import binding as B
     from synth_inputs import rng
     f = spec.split(":")
+    if f[0] == "verify":
+        return run_micro_verify(int(f[1]), int(f[2]) if len(f) > 2 else 27, steps, warmup)
     assert f[0] == "gemm" and len(f) in (4, 5), spec
     T, N, K = int(f[1]), int(f[2]), int(f[3])
     wbytes = N * K * 2
@@ -391,13 +393,56 @@ def run_micro(spec: str, steps: int, warmup: int):
                           peak_source=peaks["source"])), flush=True)
 
 
+def run_micro_verify(n_layers: int, rows: int, steps: int, warmup: int):
+    """`--micro verify:L[:T]`: verification steps of a 7B-SHAPED decoder cut down to L layers (a few
+    GB on the device instead of 28), random T-row trees, strict acceptance. The small case of the
+    real kernels (repacked weights, fused epilogues, PDL) for ncu --set full captures; also prints
+    the per-GEMM device times of the verification phase."""
+    import dataclasses
+    import torch
+    from paper_2507_22424_b200.binding import SpecVLA
+    from synth_inputs import configs as C, data
+    torch.cuda.set_device(0)
+    desc = dataclasses.replace(C.OPENVLA_7B, n_layers=n_layers)
+    wl = dataclasses.replace(C.C1, model=desc)
+    weights = data.make_weights(desc, wl.seed, device="cuda", with_draft=False)
+    embeds, ids = data.make_prefix(wl, device="cuda")
+    ids_host, P = ids.tolist(), len(ids)
+    gpu = SpecVLA(desc, weights, max_seq=1024, max_episodes=1, max_rows=512, action_only=True)
+    first = gpu.prefill([0], embeds, ids_host, [P])
+    trees = []
+    for i in range(warmup + steps):
+        tok, par, dep = data.random_tree(rows, desc, seed=2, max_depth=8, stream_offset=10 * i)
+        trees.append(dict(tokens=[-1] + tok[1:], parent=par, depth=dep))
+    for i in range(warmup):
+        gpu.verify_tree([0], [trees[i]], 0)
+    gpu.profile(4)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for i in range(steps):
+        gpu.verify_tree([0], [trees[warmup + i]], 0)
+    b.record()
+    torch.cuda.synchronize()
+    prof = gpu.profile_read()
+    ms = a.elapsed_time(b) / steps
+    wbytes = n_layers * 404_750_336 + 262_668_288
+    print(json.dumps(dict(micro="verify", layers=n_layers, rows=rows, steps=steps, ms_per_step=ms,
+                          weight_bytes=wbytes, gbs=wbytes / ms / 1e6,
+                          note="ms_per_step includes the per-GEMM timing events and the host read-back",
+                          per_class={k: dict(us_per_launch=1e3 * v["ms"] / max(1, v["launches"]),
+                                             gbs=(v["bytes"] / (v["ms"] * 1e-3) / 1e9) if v["ms"] else None)
+                                     for k, v in prof.items()})), flush=True)
+    gpu.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--micro", default=None, help="gemm:T:N:K[:M] - time one kernel alone (see run_micro)")
+    ap.add_argument("--micro", default=None, help="gemm:T:N:K[:M] or verify:L[:T] - small cases for kernel timing / ncu (see run_micro)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

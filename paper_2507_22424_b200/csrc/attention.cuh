@@ -9,16 +9,15 @@
 // 32 slots, so a K/V row is read from L2/HBM once per row block instead of once per row; the
 // next tile is fetched into registers while the current one is used.
 //
-// Both products run on the tensor cores as warp-level m16n8k8 TF32 MMAs with fp32-grade
-// operands: every operand value x is split into hi = tf32(x) and lo = tf32(x - hi) and each
-// product is the sum of lo*hi, hi*lo and hi*hi (21 mantissa bits per operand, fp32
-// accumulation). For the scores the eight warps tile the 32 rows x 32 keys of a tile as
-// 2 x 4 fragments of 16 x 8; the softmax statistics of a row (online softmax: running max and
-// sum) are combined across the four warps that hold its keys through shared memory. For the
-// weighted sum each warp owns 16 rows x (head_dim / 4) columns of the output, kept in
-// registers across tiles. With several key slices each CTA parks (max, sum, unnormalised
-// output) and bumps a counter; the CTA that arrives last merges the slices in ascending
-// order (deterministic, nobody waits).
+// All arithmetic is fp32 FMA, organised so that shared-memory traffic does not limit it:
+// a warp owns four rows. For the scores a lane owns four keys of the tile (k, k + 8, k + 16,
+// k + 24) and a quarter of the head dimension, with that quarter of its four query rows kept
+// in registers for the whole kernel, so that a step costs four conflict-free K loads per 64
+// FMAs; the quarters are added with two warp shuffles. The softmax statistics of a row
+// (online softmax: running max and sum) live entirely inside its warp. For the weighted sum
+// a lane owns head-dim columns and reads P four keys at a time. With several key slices each
+// CTA parks (max, sum, unnormalised output) and bumps a counter; the CTA that arrives last
+// merges the slices in ascending order (deterministic, nobody waits).
 #pragma once
 #include "common.cuh"
 
@@ -49,57 +48,35 @@ __host__ __device__ inline int blocks_of(const EpArgs &ea) {
   for (int i = 0; i < ea.n_ep; i++) n += (ea.nrows[i] + RB - 1) / RB;
   return n;
 }
-// Row pitches (floats) chosen so that the MMA fragment loads hit 32 distinct banks.
+// K and V tiles (rows padded by 4 floats: conflict-free float4 reads by key) and P.
 template <int DH> constexpr int smem_bytes() {
-  return (RB * (DH + 4) + KT * (DH + 4) + KT * (DH + 8) + RB * (KT + 4) + 8 * RB) * (int)sizeof(float);
-}
-
-__device__ __forceinline__ void tf32_split(float x, uint32_t &hi, uint32_t &lo) {
-  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(hi) : "f"(x));
-  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(lo) : "f"(x - __uint_as_float(hi)));
-}
-// c += a (16 x 8, row-major) * b (8 x 8, column-major), TF32 operands, fp32 accumulate.
-__device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
-}
-// c += a * b with both operands carried as (hi, lo) pairs: small terms first.
-__device__ __forceinline__ void mma_3x(float (&c)[4], const uint32_t (&ah)[4], const uint32_t (&al)[4],
-                                       const uint32_t (&bh)[2], const uint32_t (&bl)[2]) {
-  mma_tf32(c, al, bh);
-  mma_tf32(c, ah, bl);
-  mma_tf32(c, ah, bh);
+  return (2 * KT * (DH + 4) + RB * (KT + 4)) * (int)sizeof(float);
 }
 
 template <int DH>
-__global__ void __launch_bounds__(THREADS)
+__global__ void __launch_bounds__(THREADS, 1)
 tree_attention_kernel(const EpArgs ea, const Args a) {
-  constexpr int PER = DH / 32;            // head-dim columns per lane in the slice merge
+  constexpr int PER = DH / 32;            // head-dim columns per lane in the weighted sum
   constexpr int C4 = DH / 4;              // float4 per row
-  constexpr int LQ = DH + 4;              // pitch of sQ and sK rows
-  constexpr int LV = DH + 8;              // pitch of sV rows
+  constexpr int LK = DH + 4;              // pitch of sK and sV rows
   constexpr int LP = KT + 4;              // pitch of sP rows
   constexpr int NLD = KT * C4 / THREADS;  // float4 per thread per tile
-  constexpr int NTW = DH / 32;            // 8-column output fragments per warp
+  constexpr int DPG = DH / 4;             // head-dim elements per lane group in the scores
+  constexpr int NS = DPG / 4;             // float4 steps over them
   extern __shared__ __align__(16) float smem[];
-  float *sQ = smem;                       // [RB][LQ]
-  float *sK = sQ + RB * LQ;               // [KT][LQ]
-  float *sV = sK + KT * LQ;               // [KT][LV]
-  float *sP = sV + KT * LV;               // [RB][LP]
-  float *s_pm = sP + RB * LP;             // [4][RB] per-warp-column partial row maxima
-  float *s_ps = s_pm + 4 * RB;            // [4][RB] ... and partial row sums
+  float *sK = smem;                       // [KT][LK]
+  float *sV = sK + KT * LK;               // [KT][LK]
+  float *sP = sV + KT * LK;               // [RB][LP]
   __shared__ int s_nvis[RB], s_tbase[RB], s_kmax;
   __shared__ uint32_t s_mask[RB][4];
   __shared__ int s_last;
-  pdl_launch();
+  // This kernel needs the whole register file of its SM (the query rows live in registers):
+  // the GEMM that follows is let in only once the tile loop is over (pdl_launch below), not
+  // at the start, or its waiting CTAs would take the registers and push this grid into waves.
   pdl_wait();
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int g = lane >> 2, tg = lane & 3;          // MMA fragment coordinates
-  const int mt = warp & 1, nt = warp >> 1;         // 16-row block / 8-key block (or column group)
-  const int r0 = 16 * mt + g, r1 = r0 + 8;         // the two rows this thread holds values of
+  const int gk = lane >> 3, tc = lane & 7;         // quarter of the head dimension / key column
   const int h = blockIdx.y, hd = a.H * DH;
   int bid = blockIdx.x / a.splits;
   const int sp = blockIdx.x - bid * a.splits;
@@ -110,7 +87,10 @@ tree_attention_kernel(const EpArgs ea, const Args a) {
     if (bid < nb) break;
     bid -= nb;
   }
-  if (ei >= ea.n_ep) return;
+  if (ei >= ea.n_ep) {
+    pdl_launch();
+    return;
+  }
   const int row0 = ea.row0[ei] + bid * RB;
   const int nrows = min(RB, ea.nrows[ei] - bid * RB);
   const float *kbase = a.cache + (size_t)ea.eps[ei] * a.ep_stride + (size_t)h * DH;
@@ -137,33 +117,34 @@ tree_attention_kernel(const EpArgs ea, const Args a) {
     for (int o = 16; o > 0; o >>= 1) km = max(km, __shfl_xor_sync(0xffffffffu, km, o));
     if (tid == 0) s_kmax = min(km, a.max_seq);
   }
-  for (int i = tid; i < RB * C4; i += THREADS) {
-    const int r = i / C4, c = i - r * C4;
-    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (r < nrows) {
-      v = *reinterpret_cast<const float4 *>(a.q + (size_t)(row0 + r) * hd + h * DH + c * 4);
-      v.x *= a.scale; v.y *= a.scale; v.z *= a.scale; v.w *= a.scale;
+  // this lane's quarter of its warp's four query rows, scaled, for the whole kernel
+  float4 qreg[4][NS];
+#pragma unroll
+  for (int i = 0; i < 4; i++) {
+    const int r = warp * 4 + i;
+#pragma unroll
+    for (int s4 = 0; s4 < NS; s4++) {
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (r < nrows) {
+        v = *reinterpret_cast<const float4 *>(a.q + (size_t)(row0 + r) * hd + h * DH + DPG * gk + 4 * s4);
+        v.x *= a.scale; v.y *= a.scale; v.z *= a.scale; v.w *= a.scale;
+      }
+      qreg[i][s4] = v;
     }
-    *reinterpret_cast<float4 *>(sQ + r * LQ + c * 4) = v;
   }
   __syncthreads();
   const int kmax = s_kmax;
   const int tiles = (kmax + KT - 1) / KT;
   const int t0 = sp * tiles / a.splits, t1 = (sp + 1) * tiles / a.splits;
 
-  // running softmax statistics of rows r0, r1 (identical in every thread that holds the row)
-  float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
-  float o[NTW][4];                          // output fragments: rows r0 / r1, columns 32 nt + 8 j + 2 tg (+1)
+  float m_run[4], l_run[4], acc[4][PER];
 #pragma unroll
-  for (int j = 0; j < NTW; j++)
+  for (int rr = 0; rr < 4; rr++) {
+    m_run[rr] = -INFINITY;
+    l_run[rr] = 0.f;
 #pragma unroll
-    for (int k = 0; k < 4; k++) o[j][k] = 0.f;
-  auto visible = [&](int r, int slot) {
-    bool vis = slot < s_nvis[r];
-    const int b = slot - s_tbase[r];
-    if (!vis && b >= 0 && b < 128) vis = (s_mask[r][b >> 5] >> (b & 31)) & 1u;
-    return vis;
-  };
+    for (int k = 0; k < PER; k++) acc[rr][k] = 0.f;
+  }
 
   float4 kreg[NLD], vreg[NLD];
   auto fetch = [&](int t) {
@@ -187,118 +168,120 @@ tree_attention_kernel(const EpArgs ea, const Args a) {
     for (int k = 0; k < NLD; k++) {
       const int i = tid + k * THREADS;
       const int j = i / C4, c = i % C4;
-      *reinterpret_cast<float4 *>(sK + j * LQ + c * 4) = kreg[k];
-      *reinterpret_cast<float4 *>(sV + j * LV + c * 4) = vreg[k];
+      *reinterpret_cast<float4 *>(sK + j * LK + c * 4) = kreg[k];
+      *reinterpret_cast<float4 *>(sV + j * LK + c * 4) = vreg[k];
     }
     __syncthreads();
     if (t + 1 < t1) fetch(t + 1);          // in flight while this tile is used
 
-    // ---- scores of rows 16 mt .. +15 against keys 8 nt .. +7 of the tile
-    float sc[4] = {0.f, 0.f, 0.f, 0.f};
+    // ---- scores: rows 4 warp + i against keys tc + 8 j, this lane's quarter of the head dim
+    float sc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; i++)
+#pragma unroll
+      for (int j = 0; j < 4; j++) sc[i][j] = 0.f;
     {
-      const float *qa = sQ + r0 * LQ + tg, *qb = sQ + r1 * LQ + tg;
-      const float *kp = sK + (8 * nt + g) * LQ + tg;
-#pragma unroll 4
-      for (int k0 = 0; k0 < DH; k0 += 8) {
-        uint32_t ah[4], al[4], bh[2], bl[2];
-        tf32_split(qa[k0], ah[0], al[0]);
-        tf32_split(qb[k0], ah[1], al[1]);
-        tf32_split(qa[k0 + 4], ah[2], al[2]);
-        tf32_split(qb[k0 + 4], ah[3], al[3]);
-        tf32_split(kp[k0], bh[0], bl[0]);
-        tf32_split(kp[k0 + 4], bh[1], bl[1]);
-        mma_3x(sc, ah, al, bh, bl);
+      const float *kp = sK + tc * LK + DPG * gk;
+#pragma unroll
+      for (int s4 = 0; s4 < NS; s4++) {
+        float4 kf[4];
+#pragma unroll
+        for (int j = 0; j < 4; j++) kf[j] = *reinterpret_cast<const float4 *>(kp + 8 * j * LK + 4 * s4);
+#pragma unroll
+        for (int i = 0; i < 4; i++)
+#pragma unroll
+          for (int j = 0; j < 4; j++)
+            sc[i][j] += (qreg[i][s4].x * kf[j].x + qreg[i][s4].y * kf[j].y) +
+                        (qreg[i][s4].z * kf[j].z + qreg[i][s4].w * kf[j].w);
       }
     }
-    // sc[0], sc[1]: row r0, keys 8 nt + 2 tg (+1); sc[2], sc[3]: row r1, same keys
-    const int slot = t * KT + 8 * nt + 2 * tg;
-    const bool v00 = visible(r0, slot), v01 = visible(r0, slot + 1);
-    const bool v10 = visible(r1, slot), v11 = visible(r1, slot + 1);
-    float pm0 = fmaxf(v00 ? sc[0] : -INFINITY, v01 ? sc[1] : -INFINITY);
-    float pm1 = fmaxf(v10 ? sc[2] : -INFINITY, v11 ? sc[3] : -INFINITY);
-    pm0 = fmaxf(pm0, __shfl_xor_sync(0xffffffffu, pm0, 1));
-    pm0 = fmaxf(pm0, __shfl_xor_sync(0xffffffffu, pm0, 2));
-    pm1 = fmaxf(pm1, __shfl_xor_sync(0xffffffffu, pm1, 1));
-    pm1 = fmaxf(pm1, __shfl_xor_sync(0xffffffffu, pm1, 2));
-    if (tg == 0) {
-      s_pm[nt * RB + r0] = pm0;
-      s_pm[nt * RB + r1] = pm1;
-    }
-    __syncthreads();
-    float corr[2];
-    {
-      const float tm0 = fmaxf(fmaxf(s_pm[r0], s_pm[RB + r0]), fmaxf(s_pm[2 * RB + r0], s_pm[3 * RB + r0]));
-      const float tm1 = fmaxf(fmaxf(s_pm[r1], s_pm[RB + r1]), fmaxf(s_pm[2 * RB + r1], s_pm[3 * RB + r1]));
-      const float mn0 = fmaxf(m_run[0], tm0), mn1 = fmaxf(m_run[1], tm1);
-      corr[0] = (mn0 == -INFINITY) ? 1.f : __expf(m_run[0] - mn0);
-      corr[1] = (mn1 == -INFINITY) ? 1.f : __expf(m_run[1] - mn1);
-      m_run[0] = mn0;
-      m_run[1] = mn1;
-      const float p00 = v00 ? __expf(sc[0] - mn0) : 0.f, p01 = v01 ? __expf(sc[1] - mn0) : 0.f;
-      const float p10 = v10 ? __expf(sc[2] - mn1) : 0.f, p11 = v11 ? __expf(sc[3] - mn1) : 0.f;
-      *reinterpret_cast<float2 *>(sP + r0 * LP + 8 * nt + 2 * tg) = make_float2(p00, p01);
-      *reinterpret_cast<float2 *>(sP + r1 * LP + 8 * nt + 2 * tg) = make_float2(p10, p11);
-      float ps0 = p00 + p01, ps1 = p10 + p11;
-      ps0 += __shfl_xor_sync(0xffffffffu, ps0, 1);
-      ps0 += __shfl_xor_sync(0xffffffffu, ps0, 2);
-      ps1 += __shfl_xor_sync(0xffffffffu, ps1, 1);
-      ps1 += __shfl_xor_sync(0xffffffffu, ps1, 2);
-      if (tg == 0) {
-        s_ps[nt * RB + r0] = ps0;
-        s_ps[nt * RB + r1] = ps1;
+    // add the four quarters: afterwards all four lane groups hold the full scores
+#pragma unroll
+    for (int i = 0; i < 4; i++)
+#pragma unroll
+      for (int j = 0; j < 4; j++) {
+        sc[i][j] += __shfl_xor_sync(0xffffffffu, sc[i][j], 8);
+        sc[i][j] += __shfl_xor_sync(0xffffffffu, sc[i][j], 16);
       }
+    float corr[4];
+#pragma unroll
+    for (int i = 0; i < 4; i++) {
+      const int r = warp * 4 + i;
+      bool vis[4];
+      float mx = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < 4; j++) {
+        const int slot = t * KT + tc + 8 * j;
+        vis[j] = slot < s_nvis[r];
+        const int b = slot - s_tbase[r];
+        if (!vis[j] && b >= 0 && b < 128) vis[j] = (s_mask[r][b >> 5] >> (b & 31)) & 1u;
+        if (vis[j]) mx = fmaxf(mx, sc[i][j]);
+      }
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+      const float mn = fmaxf(m_run[i], mx);
+      corr[i] = (mn == -INFINITY) ? 1.f : __expf(m_run[i] - mn);
+      m_run[i] = mn;
+      float ps = 0.f;
+#pragma unroll
+      for (int j = 0; j < 4; j++) {
+        const float p = vis[j] ? __expf(sc[i][j] - mn) : 0.f;
+        ps += p;
+        if (gk == 0) sP[r * LP + tc + 8 * j] = p;
+      }
+      ps += __shfl_xor_sync(0xffffffffu, ps, 1);
+      ps += __shfl_xor_sync(0xffffffffu, ps, 2);
+      ps += __shfl_xor_sync(0xffffffffu, ps, 4);
+      l_run[i] = l_run[i] * corr[i] + ps;
     }
-    __syncthreads();
-    l_run[0] = l_run[0] * corr[0] + ((s_ps[r0] + s_ps[RB + r0]) + (s_ps[2 * RB + r0] + s_ps[3 * RB + r0]));
-    l_run[1] = l_run[1] * corr[1] + ((s_ps[r1] + s_ps[RB + r1]) + (s_ps[2 * RB + r1] + s_ps[3 * RB + r1]));
-
-    // ---- weighted sum: rows 16 mt .. +15, output columns (DH / 4) nt .. of the head
+    __syncwarp();
+    // ---- weighted sum: lane = head-dim columns PER * lane .., same four rows, four keys a step
 #pragma unroll
-    for (int j = 0; j < NTW; j++) {
-      o[j][0] *= corr[0];
-      o[j][1] *= corr[0];
-      o[j][2] *= corr[1];
-      o[j][3] *= corr[1];
-    }
-    {
-      const float *pa = sP + r0 * LP + tg, *pb = sP + r1 * LP + tg;
+    for (int rr = 0; rr < 4; rr++)
 #pragma unroll
-      for (int k0 = 0; k0 < KT; k0 += 8) {
-        uint32_t ah[4], al[4];
-        tf32_split(pa[k0], ah[0], al[0]);
-        tf32_split(pb[k0], ah[1], al[1]);
-        tf32_split(pa[k0 + 4], ah[2], al[2]);
-        tf32_split(pb[k0 + 4], ah[3], al[3]);
-        const float *vp = sV + (k0 + tg) * LV + NTW * 8 * nt + g;
+      for (int k = 0; k < PER; k++) acc[rr][k] *= corr[rr];
+#pragma unroll 2
+    for (int j4 = 0; j4 < KT; j4 += 4) {
+      float4 pf[4];
 #pragma unroll
-        for (int j = 0; j < NTW; j++) {
-          uint32_t bh[2], bl[2];
-          tf32_split(vp[8 * j], bh[0], bl[0]);
-          tf32_split(vp[4 * LV + 8 * j], bh[1], bl[1]);
-          mma_3x(o[j], ah, al, bh, bl);
+      for (int rr = 0; rr < 4; rr++) pf[rr] = *reinterpret_cast<const float4 *>(sP + (warp * 4 + rr) * LP + j4);
+#pragma unroll
+      for (int jj = 0; jj < 4; jj++) {
+        float vv[PER];
+        if (PER == 4) {
+          const float4 t4 = *reinterpret_cast<const float4 *>(sV + (j4 + jj) * LK + lane * 4);
+          vv[0] = t4.x; vv[1] = t4.y; vv[2 % PER] = t4.z; vv[3 % PER] = t4.w;
+        } else {
+          const float2 t2 = *reinterpret_cast<const float2 *>(sV + (j4 + jj) * LK + lane * 2);
+          vv[0] = t2.x; vv[1] = t2.y;
+        }
+#pragma unroll
+        for (int rr = 0; rr < 4; rr++) {
+          const float p = jj == 0 ? pf[rr].x : (jj == 1 ? pf[rr].y : (jj == 2 ? pf[rr].z : pf[rr].w));
+#pragma unroll
+          for (int k = 0; k < PER; k++) acc[rr][k] += p * vv[k];
         }
       }
     }
+    __syncwarp();
   }
 
-  // o[j][0..1]: row r0, columns cbase + 8 j + 2 tg (+1); o[j][2..3]: row r1
-  const int cbase = NTW * 8 * nt + 2 * tg;
+  pdl_launch();
   if (a.splits == 1) {
 #pragma unroll
-    for (int hh = 0; hh < 2; hh++) {
-      const int r = hh ? r1 : r0;
+    for (int rr = 0; rr < 4; rr++) {
+      const int r = warp * 4 + rr;
       if (r >= nrows) continue;
-      const float inv = 1.f / l_run[hh];
+      const float inv = 1.f / l_run[rr];
 #pragma unroll
-      for (int j = 0; j < NTW; j++)
-#pragma unroll
-        for (int e = 0; e < 2; e++) {
-          const size_t idx = (size_t)(row0 + r) * hd + h * DH + cbase + 8 * j + e;
-          const float v = o[j][2 * hh + e] * inv;
-          const bf16 hi = __float2bfloat16(v);
-          a.out[idx] = hi;
-          a.out[a.out_plane + idx] = __float2bfloat16(v - __bfloat162float(hi));
-        }
+      for (int k = 0; k < PER; k++) {
+        const size_t idx = (size_t)(row0 + r) * hd + h * DH + lane * PER + k;
+        const float v = acc[rr][k] * inv;
+        const bf16 hi = __float2bfloat16(v);
+        a.out[idx] = hi;
+        a.out[a.out_plane + idx] = __float2bfloat16(v - __bfloat162float(hi));
+      }
     }
     return;
   }
@@ -307,17 +290,14 @@ tree_attention_kernel(const EpArgs ea, const Args a) {
   const int unit = gblock * a.H + h;
   float *mine = a.part + ((size_t)unit * a.splits + sp) * RB * (DH + 2);
 #pragma unroll
-  for (int hh = 0; hh < 2; hh++) {
-    const int r = hh ? r1 : r0;
+  for (int rr = 0; rr < 4; rr++) {
+    const int r = warp * 4 + rr;
     float *dst = mine + (size_t)r * (DH + 2);
 #pragma unroll
-    for (int j = 0; j < NTW; j++) {
-      __stcg(dst + cbase + 8 * j, o[j][2 * hh]);
-      __stcg(dst + cbase + 8 * j + 1, o[j][2 * hh + 1]);
-    }
-    if (nt == 0 && tg == 0) {
-      __stcg(dst + DH, m_run[hh]);
-      __stcg(dst + DH + 1, l_run[hh]);
+    for (int k = 0; k < PER; k++) __stcg(dst + lane * PER + k, acc[rr][k]);
+    if (lane == 0) {
+      __stcg(dst + DH, m_run[rr]);
+      __stcg(dst + DH + 1, l_run[rr]);
     }
   }
   __threadfence();

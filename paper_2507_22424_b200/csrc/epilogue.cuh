@@ -1,4 +1,4 @@
-// Row-wise kernels around the GEMMs: input embedding, RoPE + KV append, greedy argmax and
+// Row-wise kernels around the GEMMs: input embedding, the RoPE table, greedy argmax and
 // log-softmax top-k over finished logits, feature materialisation. All arithmetic is fp32.
 //
 // RMSNorm is split around the GEMMs: the producer of a residual row x writes the GEMM operand
@@ -66,36 +66,6 @@ embed_kernel(RowTable rt, const bf16 *__restrict__ embeds, const bf16 *__restric
   }
   ss = block_sum(ss, red);
   for (int j = threadIdx.x; j < nt; j += blockDim.x) ssq[(size_t)t * nt + j] = (j == 0) ? ss : 0.f;
-}
-
-// Rotates q and k of row t by its position (rotate-half pairs (i, i + dh/2), angle from the
-// precomputed table) and writes q and, into the row's cache slot, k and v, all fp32.
-// qkv [T][3 * H * dh] = [q | k | v]. Cache layout per episode: [2 (K, V)][max_seq][H * dh].
-// grid = (T, ceil(H * dh / 2 / THREADS)).
-__global__ void __launch_bounds__(THREADS)
-rope_append_kernel(const float *__restrict__ qkv, int H, int dh, RowTable rt,
-                   const float2 *__restrict__ rope_tab, float *__restrict__ q,
-                   float *__restrict__ cache, size_t ep_stride, int max_seq) {
-  pdl_launch();
-  pdl_wait();
-  const int t = blockIdx.x;
-  const int hd = H * dh, half = dh >> 1;
-  const int i = blockIdx.y * blockDim.x + threadIdx.x;
-  if (i >= H * half) return;
-  const int pos = rt.pos[t], slot = rt.slot[t];
-  float *kdst = cache + (size_t)rt.ep[t] * ep_stride + (size_t)slot * hd;
-  float *vdst = kdst + (size_t)max_seq * hd;
-  const float *p = qkv + (size_t)t * 3 * hd;
-  const int h = i / half, j = i - h * half;
-  const int c0 = h * dh + j, c1 = c0 + half;
-  const float2 cs = rope_tab[(size_t)pos * half + j];
-  const float qlo = p[c0], qhi = p[c1], klo = p[hd + c0], khi = p[hd + c1];
-  q[(size_t)t * hd + c0] = qlo * cs.x - qhi * cs.y;
-  q[(size_t)t * hd + c1] = qhi * cs.x + qlo * cs.y;
-  kdst[c0] = klo * cs.x - khi * cs.y;
-  kdst[c1] = khi * cs.x + klo * cs.y;
-  vdst[c0] = p[2 * hd + c0];
-  vdst[c1] = p[2 * hd + c1];
 }
 
 // cos/sin table in double precision: tab[pos][j] = (cos, sin)(pos * theta^(-2j/dh)).

@@ -232,74 +232,122 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 
   // every CTA's partial tile is in place
   if (S > 1) cluster_sync_all(); else __syncthreads();
+  if (warp == 0 && lane == 0 && ea.pf_w) {
+    // head of the next GEMM's weight stream into L2, one request per range (its CTA c reads
+    // units [tile KB + r KB / S, tile KB + (r + 1) KB / S) with tile = c / S, r = c % S).
+    // Issued here, off the critical path of the epilogue warps.
+    const int nct = ea.pf_tiles * ea.pf_S;
+    for (int c = blockIdx.x; c < nct; c += gridDim.x) {
+      const int ptile = c / ea.pf_S, r = c - ptile * ea.pf_S;
+      const int pk0 = r * ea.pf_KB / ea.pf_S;
+      int n = (r + 1) * ea.pf_KB / ea.pf_S - pk0;
+      if (n > ea.pf_units) n = ea.pf_units;
+      if (n > 0) prefetch_l2(ea.pf_w + ((size_t)ptile * ea.pf_KB + pk0) * (BM * BK), (uint32_t)n * W_STAGE_BYTES);
+    }
+  }
 
   if (warp >= 2) {
     // ------------------------------------------------------------------ epilogue, part 2:
-    // rows rank, rank + S, ... of the tile. A thread owns four consecutive columns (64 column
-    // groups) and every fourth of those rows; the S partials are added in rank order. The
-    // code is kept small on purpose: it runs once per CTA, straight from a cold instruction
-    // cache.
+    // rows rank, rank + S, ... of the tile. A thread owns four consecutive columns and every
+    // RG-th of those rows (64 column groups x 4 row groups; SwiGLU, whose 128 outputs come
+    // from column pairs, 32 x 8); the S partials are added in rank order. Everything this code
+    // needs from global memory (residual, positions, RoPE factors) is requested BEFORE the
+    // partial tiles are read, so that the latencies overlap instead of adding up.
     const int et = threadIdx.x - 64;
-    const int rg = et >> 6, cg = et & 63;                // row group 0..3, column group 0..63
-    const int c4 = swiglu ? (cg & 31) * 4 : cg * 4;      // first of the four columns within the tile
+    const int RG = swiglu ? 8 : 4;
+    const int rg = swiglu ? et >> 5 : et >> 6;
+    const int c4 = swiglu ? (et & 31) * 4 : (et & 63) * 4;    // first of the four columns within the tile
     const int n = swiglu ? tile * 128 + c4 : tile * BM + c4;
-    const bool col_ok = n < ea.N && !(swiglu && cg >= 32);   // N % 4 == 0: all four or none
+    const bool col_ok = n < ea.N;                             // N % 4 == 0: all four or none
     const float *P_own = reinterpret_cast<const float *>(smem_raw + (base - smem_u32(smem_raw)));
     const float *P_of[MAX_S];
     {
       cooperative_groups::cluster_group cluster = cooperative_groups::this_cluster();
 #pragma unroll
       for (int sl = 0; sl < MAX_S; sl++)
-        P_of[sl] = S == 1 ? P_own
-                          : cluster.map_shared_rank(const_cast<float *>(P_own), (unsigned)(sl < S ? sl : S - 1));
+        P_of[sl] = (S == 1 || sl >= S) ? P_own : cluster.map_shared_rank(const_cast<float *>(P_own), (unsigned)sl);
     }
     float4 gain = make_float4(1.f, 1.f, 1.f, 1.f);
     if (ea.mode == EPI_RESID && ea.gain && col_ok) gain = *reinterpret_cast<const float4 *>(ea.gain + n);
+    // QKV: which of q / k / v and which half of a head the four columns lie in
+    const int which = ea.mode == EPI_QKV ? n / ea.hd : 2;
+    const int cq = ea.mode == EPI_QKV ? n - which * ea.hd : 0;
+    const int half = ea.dh >> 1, jq = ea.mode == EPI_QKV ? cq % ea.dh : 0;
+    const bool lo = jq < half, rot = ea.mode == EPI_QKV && which < 2;
     auto partial_sum = [&](int off) {
-      float4 acc = *reinterpret_cast<const float4 *>(P_of[0] + off);
-      if (S > 1) {
-        float4 p[MAX_S];
+      float4 p[MAX_S];
 #pragma unroll
-        for (int sl = 1; sl < MAX_S; sl++) p[sl] = *reinterpret_cast<const float4 *>(P_of[sl] + off);
+      for (int sl = 0; sl < MAX_S; sl++)
+        if (sl < S) p[sl] = *reinterpret_cast<const float4 *>(P_of[sl] + off);
+      float4 acc = p[0];
 #pragma unroll
-        for (int sl = 1; sl < MAX_S; sl++)
-          if (sl < S) {
-            acc.x += p[sl].x;
-            acc.y += p[sl].y;
-            acc.z += p[sl].z;
-            acc.w += p[sl].w;
-          }
-      }
+      for (int sl = 1; sl < MAX_S; sl++)
+        if (sl < S) {
+          acc.x += p[sl].x;
+          acc.y += p[sl].y;
+          acc.z += p[sl].z;
+          acc.w += p[sl].w;
+        }
       return acc;
     };
-#pragma unroll 2
-    for (int t = rank + rg * S; t < T; t += 4 * S) {
+    for (int t = rank + rg * S; t < T; t += RG * S) {
       const size_t row = (size_t)(ea.row0 + t);
       const float sc = s_scale[t];
+      // global operands first
+      float4 xo = make_float4(0.f, 0.f, 0.f, 0.f), cs01 = xo, cs23 = xo;
+      int slot = 0, ep = 0;
+      if (ea.mode == EPI_RESID && ea.accumulate && col_ok)
+        xo = *reinterpret_cast<const float4 *>(ea.x + row * ea.N + n);
+      if (ea.mode == EPI_QKV) {
+        if (rot) {
+          const float2 *cs = ea.rope_tab + (size_t)ea.rt.pos[row] * half + (lo ? jq : jq - half);
+          cs01 = *reinterpret_cast<const float4 *>(cs);
+          cs23 = *reinterpret_cast<const float4 *>(cs + 2);
+        }
+        if (which > 0) {
+          slot = ea.rt.slot[row];
+          ep = ea.rt.ep[row];
+        }
+      }
       float4 v = partial_sum(t * BM + c4);
       if (ea.mode == EPI_PLAIN) {
         if (col_ok)
           *reinterpret_cast<float4 *>(ea.out + row * ea.ldo + n) = make_float4(sc * v.x, sc * v.y, sc * v.z, sc * v.w);
+      } else if (ea.mode == EPI_QKV) {
+        // the partner columns of the rotation (dh / 2 away) are in the same tile
+        float4 o = make_float4(sc * v.x, sc * v.y, sc * v.z, sc * v.w);
+        if (rot) {
+          const float4 w = partial_sum(t * BM + c4 + (lo ? half : -half));
+          const float sg = lo ? -sc : sc;
+          o.x = o.x * cs01.x + sg * w.x * cs01.y;
+          o.y = o.y * cs01.z + sg * w.y * cs01.w;
+          o.z = o.z * cs23.x + sg * w.z * cs23.y;
+          o.w = o.w * cs23.z + sg * w.w * cs23.w;
+        }
+        if (col_ok) {
+          float *dst = which == 0 ? ea.q + row * ea.hd + cq
+                                  : ea.cache + (size_t)ep * ea.ep_stride +
+                                        ((size_t)(which - 1) * ea.max_seq + slot) * ea.hd + cq;
+          *reinterpret_cast<float4 *>(dst) = o;
+        }
       } else if (swiglu) {
         const float4 u = partial_sum(t * BM + 128 + c4);
         if (col_ok) {
           const float gx = sc * v.x, gy = sc * v.y, gz = sc * v.z, gw = sc * v.w;
           store_limbs4(ea.hid, ea.hid_plane, row * ea.N + n,
-                       make_float4(gx / (1.f + expf(-gx)) * (sc * u.x), gy / (1.f + expf(-gy)) * (sc * u.y),
-                                   gz / (1.f + expf(-gz)) * (sc * u.z), gw / (1.f + expf(-gw)) * (sc * u.w)));
+                       make_float4(__fdividef(gx, 1.f + __expf(-gx)) * (sc * u.x),
+                                   __fdividef(gy, 1.f + __expf(-gy)) * (sc * u.y),
+                                   __fdividef(gz, 1.f + __expf(-gz)) * (sc * u.z),
+                                   __fdividef(gw, 1.f + __expf(-gw)) * (sc * u.w)));
         }
       } else {
         float s2 = 0.f;
         if (col_ok) {
-          float *xp = ea.x + row * ea.N + n;
-          if (ea.accumulate) {
-            const float4 xo = *reinterpret_cast<const float4 *>(xp);
-            v.x += xo.x;
-            v.y += xo.y;
-            v.z += xo.z;
-            v.w += xo.w;
-          }
-          *reinterpret_cast<float4 *>(xp) = v;
+          v.x += xo.x;
+          v.y += xo.y;
+          v.z += xo.z;
+          v.w += xo.w;
+          *reinterpret_cast<float4 *>(ea.x + row * ea.N + n) = v;
           store_limbs4(ea.xn, ea.xn_plane, row * ea.N + n,
                        make_float4(v.x * gain.x, v.y * gain.y, v.z * gain.z, v.w * gain.w));
           s2 = (v.x * v.x + v.y * v.y) + (v.z * v.z + v.w * v.w);

@@ -116,6 +116,9 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_
       "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
       ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(pol) : "memory");
 }
+__device__ __forceinline__ void prefetch_l2(const void *src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ void grid_dep_wait() { pdl_wait(); }
 __device__ __forceinline__ void grid_dep_launch() { pdl_launch(); }
 // barrier among the 256 epilogue threads (warps 2-9)
@@ -178,7 +181,9 @@ __host__ __device__ constexpr uint32_t instr_desc(int n) {
 enum EpiMode {
   EPI_PLAIN = 0,    // out[row0 + t][n] = scale_t * v
   EPI_RESID = 1,    // x[row0 + t][n] = (accumulate ? x : 0) + v;  xn = limbs(x * gain[n]);  ssq_out
-  EPI_SWIGLU = 2    // hid[row0 + t][n] = limbs(silu(scale_t * gate) * (scale_t * up))
+  EPI_SWIGLU = 2,   // hid[row0 + t][n] = limbs(silu(scale_t * gate) * (scale_t * up))
+  EPI_QKV = 3       // scale_t * v is [q | k | v]: rotate q and k by the row's position (rotate-half
+                    // pairs (i, i + dh/2)), write q and, into the row's cache slot, k and v
 };
 
 struct EpiArgs {
@@ -189,6 +194,11 @@ struct EpiArgs {
   int up_off;            // EPI_SWIGLU: row of W where the up projection starts (F)
   const bf16 *wpacked;   // weights repacked by pack_weights_kernel (one contiguous 32 KB block per
                          // (tile, K block), in unit order); NULL: strided boxes through the W map
+  // L2 prefetch for the GEMM that follows: once its own loads are issued, every CTA asks for
+  // the first pf_units 32 KB blocks of some of the next GEMM's per-CTA ranges, so that HBM keeps
+  // working through this kernel's epilogue, the kernel boundary and the next kernel's start.
+  const bf16 *pf_w;      // packed weights of the next GEMM; NULL: no prefetch
+  int pf_tiles, pf_KB, pf_S, pf_units;
   // row scale of the RMSNorm in front of this GEMM: rsqrt(sum_j ssq_in[row][j] * inv_k + eps)
   const float *ssq_in;   // [rows][nt_in] partial sums of squares; NULL: scale 1
   int nt_in;
@@ -206,6 +216,13 @@ struct EpiArgs {
   // EPI_SWIGLU
   bf16 *hid;             // two limbs, [rows][N] each
   size_t hid_plane;
+  // EPI_QKV (N = 3 * H * dh)
+  RowTable rt;           // per-row position, cache slot and episode
+  const float2 *rope_tab;  // [position][dh / 2] (cos, sin)
+  float *q;              // [rows][H * dh]
+  float *cache;          // [episode][2 (K, V)][max_seq][H * dh]
+  size_t ep_stride;
+  int max_seq, hd, dh;
 };
 
 __device__ __forceinline__ void store_limbs(bf16 *hi_plane, size_t plane, size_t idx, float v) {

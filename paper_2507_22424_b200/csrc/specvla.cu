@@ -44,6 +44,7 @@ struct LayerW {
 
 
 constexpr size_t ALIGN = 1024;
+constexpr size_t L2_PREFETCH_BYTES = 48u << 20;   // of the next GEMM's weights, out of 126 MB of L2
 
 struct Carver {
   char *base;
@@ -73,12 +74,13 @@ struct specvla_ctx {
   int nt;                       // 256-column tiles of a d_model-wide row (sums-of-squares slots)
   bool use_pdl;                 // programmatic dependent launch between the kernels of a forward
   gemm_ck::ClusterFit fit;      // clusters of each size that can be resident at once
+  bool use_l2_prefetch;         // GEMMs prefetch the head of the next GEMM's weights into L2
 
   // workspace carve-up (device)
   float *kv_t, *kv_d;           // target [ep][layer][2][max_seq][hd], draft [ep][2][max_seq][hd], fp32
   size_t kv_t_ep_stride, kv_t_layer_stride, kv_d_ep_stride;
   float2 *rope_tab;
-  float *x, *feat, *lgs, *pend_feat, *dout, *margin, *top_lp, *q, *qkv;
+  float *x, *feat, *lgs, *pend_feat, *dout, *margin, *top_lp, *q;
   float *ssq, *lm_ssq;          // per-row partial sums of squares of x / of the gathered LM-head rows
   bf16 *packed;                 // repacked weight matrices, one after the other
   size_t packed_elems;
@@ -175,7 +177,6 @@ size_t carve(specvla_ctx *c, char *base) {
   limbs(c->ao, R, hd);
   limbs(c->hid, R, d.d_ffn);
   limbs(c->lm_in, lm_rows, d.d_model);
-  c->qkv = cv.take<float>(R * 3 * hd);
   c->nt = (d.d_model + SV_TILE_ROWS - 1) / SV_TILE_ROWS;
   c->ssq = cv.take<float>(R * c->nt);
   c->lm_ssq = cv.take<float>(lm_rows * c->nt);
@@ -267,7 +268,9 @@ cudaLaunchConfig_t launch_cfg(dim3 grid, dim3 block, cudaStream_t st, cudaLaunch
 
 // One GEMM over R rows of A against W with the fused epilogue described by `ea` (mode and
 // outputs; the row range is filled in here). Rows go in launches of 128.
-int gemm(specvla_ctx *ctx, const XBuf &A, const WMat &W, int R, gemm_tc::EpiArgs ea, cudaStream_t st, int cls) {
+// next: the matrix of the GEMM that will follow (its head is prefetched into L2), or NULL.
+int gemm(specvla_ctx *ctx, const XBuf &A, const WMat &W, int R, gemm_tc::EpiArgs ea, cudaStream_t st, int cls,
+         const WMat *next = nullptr, bool next_swiglu = false) {
   if (!W.has_map || !A.has_map || A.K != W.K) return SPECVLA_ERR_BAD_STATE;
   const bool swiglu = ea.mode == gemm_tc::EPI_SWIGLU;
   const int tiles = swiglu ? (ea.N + 127) / 128 : (W.N + SV_TILE_ROWS - 1) / SV_TILE_ROWS;
@@ -281,6 +284,16 @@ int gemm(specvla_ctx *ctx, const XBuf &A, const WMat &W, int R, gemm_tc::EpiArgs
   for (int r0 = 0; r0 < R; r0 += gemm_tc::MAX_T) {
     ea.row0 = r0;
     ea.T = R - r0 < gemm_tc::MAX_T ? R - r0 : gemm_tc::MAX_T;
+    ea.pf_w = nullptr;
+    if (next && next->packed && ctx->use_l2_prefetch && r0 + gemm_tc::MAX_T >= R) {
+      // last launch over W: start pulling the next matrix (up to L2_PREFETCH_BYTES of it)
+      ea.pf_tiles = next_swiglu ? (next->N / 2 + 127) / 128 : (next->N + SV_TILE_ROWS - 1) / SV_TILE_ROWS;
+      ea.pf_KB = (next->K + gemm_tc::BK - 1) / gemm_tc::BK;
+      ea.pf_S = gemm_ck::slices_for(ea.pf_tiles, ea.pf_KB, ctx->fit);
+      const size_t per_cta = L2_PREFETCH_BYTES / ((size_t)ea.pf_tiles * ea.pf_S) / gemm_tc::W_STAGE_BYTES;
+      ea.pf_units = per_cta < 1 ? 1 : (int)per_cta;
+      ea.pf_w = next->packed;
+    }
     CU(gemm_ck::launch(W.map, A.map[tn_index(gemm_tc::tn_of(ea.T))], ea, tiles, KB, S, ctx->err, st,
                        ctx->use_pdl));
     ctx->launches++;
@@ -359,16 +372,28 @@ int attention(specvla_ctx *ctx, const EpArgs &rows, const float *cache, size_t e
 // One pre-norm decoder layer over R rows. In: x (residual, fp32), xn = limbs(x * norm1 gain) and
 // ssq = sums of squares of x. Out: x updated; xn = limbs(x * next_gain) (limbs(x) when next_gain
 // is NULL) and ssq for the norm that follows.
+// after: the matrix of the GEMM that follows this layer (next layer's QKV, the LM head), or NULL.
 int run_layer(specvla_ctx *ctx, const LayerW &w, int R, const EpArgs &rows, float *cache, size_t ep_stride,
-              const float *next_gain, cudaStream_t st) {
+              const float *next_gain, const WMat *after, cudaStream_t st) {
   const specvla_model_desc &d = ctx->desc;
   const int hd = ctx->hd, F = d.d_ffn;
-  TRY(gemm(ctx, ctx->xn, w.wqkv, R, epi_plain(ctx->qkv, 3 * hd, 3 * hd, ctx->ssq, ctx->nt), st, SPECVLA_PROF_QKV));
-  LAUNCH(epi::rope_append_kernel, dim3(R, (d.n_heads * d.head_dim / 2 + epi::THREADS - 1) / epi::THREADS),
-         dim3(epi::THREADS), (const float *)ctx->qkv, d.n_heads, d.head_dim, ctx->rt,
-         (const float2 *)ctx->rope_tab, ctx->q, cache, ep_stride, d.max_seq);
+  // QKV projection; its epilogue applies the norm's row scale and RoPE and appends K, V to the cache
+  gemm_tc::EpiArgs qk = {};
+  qk.mode = gemm_tc::EPI_QKV;
+  qk.N = 3 * hd;
+  qk.ssq_in = ctx->ssq;
+  qk.nt_in = ctx->nt;
+  qk.rt = ctx->rt;
+  qk.rope_tab = ctx->rope_tab;
+  qk.q = ctx->q;
+  qk.cache = cache;
+  qk.ep_stride = ep_stride;
+  qk.max_seq = d.max_seq;
+  qk.hd = hd;
+  qk.dh = d.head_dim;
+  TRY(gemm(ctx, ctx->xn, w.wqkv, R, qk, st, SPECVLA_PROF_QKV, &w.wo));
   TRY(attention(ctx, rows, cache, ep_stride, st));
-  TRY(gemm(ctx, ctx->ao, w.wo, R, epi_resid(ctx, 1, w.norm2), st, SPECVLA_PROF_O));
+  TRY(gemm(ctx, ctx->ao, w.wo, R, epi_resid(ctx, 1, w.norm2), st, SPECVLA_PROF_O, &w.wgu, true));
   gemm_tc::EpiArgs sw = {};
   sw.mode = gemm_tc::EPI_SWIGLU;
   sw.N = F;
@@ -377,8 +402,8 @@ int run_layer(specvla_ctx *ctx, const LayerW &w, int R, const EpArgs &rows, floa
   sw.nt_in = ctx->nt;
   sw.hid = ctx->hid.p;
   sw.hid_plane = ctx->hid.plane;
-  TRY(gemm(ctx, ctx->xn, w.wgu, R, sw, st, SPECVLA_PROF_GATE_UP));
-  TRY(gemm(ctx, ctx->hid, w.wd, R, epi_resid(ctx, 1, next_gain), st, SPECVLA_PROF_DOWN));
+  TRY(gemm(ctx, ctx->xn, w.wgu, R, sw, st, SPECVLA_PROF_GATE_UP, &w.wd));
+  TRY(gemm(ctx, ctx->hid, w.wd, R, epi_resid(ctx, 1, next_gain), st, SPECVLA_PROF_DOWN, after));
   return SPECVLA_OK;
 }
 
@@ -392,7 +417,8 @@ int target_forward(specvla_ctx *ctx, int R, const EpArgs &rows, const bf16 *embe
   for (int l = 0; l < d.n_layers; l++) {
     const bool last = (l + 1 == d.n_layers);
     TRY(run_layer(ctx, ctx->layers[l], R, rows, ctx->kv_t + (size_t)l * ctx->kv_t_layer_stride,
-                  ctx->kv_t_ep_stride, last ? ctx->final_norm : ctx->layers[l + 1].norm1, st));
+                  ctx->kv_t_ep_stride, last ? ctx->final_norm : ctx->layers[l + 1].norm1,
+                  last ? &ctx->lm_head : &ctx->layers[l + 1].wqkv, st));
   }
   ctx->last_rows = R;
   return SPECVLA_OK;
@@ -401,8 +427,10 @@ int target_forward(specvla_ctx *ctx, int R, const EpArgs &rows, const bf16 *embe
 // Draft model over R rows: ctx->xin = [feature ; embedding] rows are already built.
 // Leaves the layer outputs in ctx->x (fp32) and ctx->xn (limbs, un-normalised).
 int draft_forward(specvla_ctx *ctx, int R, const EpArgs &rows, cudaStream_t st) {
-  TRY(gemm(ctx, ctx->xin, ctx->draft_fc, R, epi_resid(ctx, 0, ctx->dlayer.norm1), st, SPECVLA_PROF_FC));
-  return run_layer(ctx, ctx->dlayer, R, rows, ctx->kv_d, ctx->kv_d_ep_stride, nullptr, st);
+  TRY(gemm(ctx, ctx->xin, ctx->draft_fc, R, epi_resid(ctx, 0, ctx->dlayer.norm1), st, SPECVLA_PROF_FC,
+           &ctx->dlayer.wqkv));
+  return run_layer(ctx, ctx->dlayer, R, rows, ctx->kv_d, ctx->kv_d_ep_stride, nullptr,
+                   ctx->desc.action_only ? &ctx->lm_head_act : &ctx->lm_head, st);
 }
 
 // LM head over `rows` two-limb rows of A into ctx->lgs [rows][vocab]. ssq != NULL: the rows
@@ -503,6 +531,7 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
   carve(ctx, static_cast<char *>(workspace));
   const int hd = ctx->hd, D = desc->d_model, F = desc->d_ffn;
   ctx->use_pdl = getenv("SPECVLA_NO_PDL") == nullptr;
+  ctx->use_l2_prefetch = getenv("SPECVLA_NO_L2_PREFETCH") == nullptr;
   ctx->fit = gemm_ck::query_cluster_fit();
   if (getenv("SPECVLA_DEBUG")) {
     fprintf(stderr, "specvla: resident clusters by size:");
