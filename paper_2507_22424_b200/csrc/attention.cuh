@@ -311,24 +311,35 @@ tree_attention_kernel(const EpArgs ea, const Args a) {
   if (!s_last) return;
   __threadfence();
   const float *all = a.part + (size_t)unit * a.splits * RB * (DH + 2);
+  // every load of a row's slices is issued before any is used: one latency, not one per slice
 #pragma unroll
   for (int rr = 0; rr < 4; rr++) {
     const int r = warp * 4 + rr;
     if (r >= nrows) continue;
+    float ms[MAX_SPLITS], ls[MAX_SPLITS], os[MAX_SPLITS][PER];
+#pragma unroll
+    for (int s2 = 0; s2 < MAX_SPLITS; s2++) {
+      const float *src = all + ((size_t)(s2 < a.splits ? s2 : 0) * RB + r) * (DH + 2);
+      ms[s2] = __ldcg(src + DH);
+      ls[s2] = __ldcg(src + DH + 1);
+#pragma unroll
+      for (int k = 0; k < PER; k++) os[s2][k] = __ldcg(src + lane * PER + k);
+    }
     float M = -INFINITY;
-    for (int s2 = 0; s2 < a.splits; s2++)
-      M = fmaxf(M, __ldcg(all + ((size_t)s2 * RB + r) * (DH + 2) + DH));
+#pragma unroll
+    for (int s2 = 0; s2 < MAX_SPLITS; s2++)
+      if (s2 < a.splits) M = fmaxf(M, ms[s2]);
     float L = 0.f, o[PER];
 #pragma unroll
     for (int k = 0; k < PER; k++) o[k] = 0.f;
-    for (int s2 = 0; s2 < a.splits; s2++) {
-      const float *src = all + ((size_t)s2 * RB + r) * (DH + 2);
-      const float ms = __ldcg(src + DH);
-      const float c = (ms == -INFINITY) ? 0.f : __expf(ms - M);
-      L += __ldcg(src + DH + 1) * c;
 #pragma unroll
-      for (int k = 0; k < PER; k++) o[k] += __ldcg(src + lane * PER + k) * c;
-    }
+    for (int s2 = 0; s2 < MAX_SPLITS; s2++)
+      if (s2 < a.splits) {
+        const float c = (ms[s2] == -INFINITY) ? 0.f : __expf(ms[s2] - M);
+        L += ls[s2] * c;
+#pragma unroll
+        for (int k = 0; k < PER; k++) o[k] += os[s2][k] * c;
+      }
     const float inv = 1.f / L;
 #pragma unroll
     for (int k = 0; k < PER; k++) {
