@@ -51,12 +51,11 @@ __host__ __device__ constexpr int ck_tmem_cols(int TN) { return 2 * acc_width(TN
 template <int TN>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
-               const EpiArgs ea, const int KB, int *__restrict__ err) {
+               const __grid_constant__ CUtensorMap tmXtail, const EpiArgs ea, const int KB,
+               int *__restrict__ err) {
   constexpr int STAGES = stages_of(TN);
   constexpr int STAGE = stage_bytes(TN);
-  constexpr bool MERGE = merged_limbs(TN);
   constexpr int AW = acc_width(TN);
-  constexpr uint32_t IDESC = instr_desc(AW);
   extern __shared__ unsigned char smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t bars = base + STAGES * STAGE;
@@ -65,6 +64,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   const uint32_t tfull_bar = bars + 8u * (2 * STAGES);
   const uint32_t tmem_slot = bars + 8u * (2 * STAGES + 1);
   __shared__ float s_scale[MAX_T];
+  __shared__ int s_pos[MAX_T], s_slot[MAX_T], s_ep[MAX_T];
   __shared__ float s_red[8][MAX_T];
   __shared__ int s_flag[8];
 
@@ -76,15 +76,23 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   const int kb0 = rank * KB / S, kb1 = (rank + 1) * KB / S;
   const int n_units = kb1 - kb0;
   const long long u0 = (long long)tile * KB + kb0;
-  const int T = ea.T;
   const int tiles = gridDim.x / S;
+  // rows of this CTA: the blockIdx.y-th 128-row chunk. The last chunk of a multi-chunk launch may
+  // be narrower than TN: it has a tensor map with its own box and MMAs of its own width.
+  const int row0 = ea.row0 + (int)blockIdx.y * MAX_T;
+  const int T = ea.T - (int)blockIdx.y * MAX_T < MAX_T ? ea.T - (int)blockIdx.y * MAX_T : MAX_T;
+  const bool tail = TN == MAX_T && blockIdx.y == gridDim.y - 1;
+  const int tn = tail ? ea.tn_tail : TN;
+  const CUtensorMap *xmap = tail ? &tmXtail : &tmX;
+  const uint32_t stage_tx = (uint32_t)(W_STAGE_BYTES + 2 * tn * BK * 2);
+  const uint32_t idesc = instr_desc(2 * tn);
 
   const int npre = n_units < STAGES ? n_units : STAGES;
   uint64_t pol_w = 0;
   auto load_w = [&](int it) {
     const int st = it % STAGES;
     const uint32_t sW = base + st * STAGE;
-    mbar_expect_tx(full_bar(st), STAGE);
+    mbar_expect_tx(full_bar(st), stage_tx);
     if (ea.wpacked) {
       bulk_load(sW, ea.wpacked + (size_t)(u0 + it) * (BM * BK), W_STAGE_BYTES, full_bar(st), pol_w);
     } else {
@@ -96,7 +104,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     }
   };
   if (threadIdx.x == 0) {
-    prefetch_tensormap(&tmX);
+    prefetch_tensormap(xmap);
     if (!ea.wpacked) prefetch_tensormap(&tmW);
     for (int s = 0; s < STAGES; s++) {
       mbar_init(full_bar(s), 1);
@@ -125,7 +133,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       const uint64_t pol_x = policy_evict_last();
       grid_dep_wait();
       for (int j = 0; j < npre; j++)
-        tma_load_3d(base + j * STAGE + W_STAGE_BYTES, &tmX, (kb0 + j) * BK, ea.row0, 0, full_bar(j), pol_x);
+        tma_load_3d(base + j * STAGE + W_STAGE_BYTES, xmap, (kb0 + j) * BK, row0, 0, full_bar(j), pol_x);
       for (int it = npre; it < n_units; it++) {
         const int st = it % STAGES, rnd = it / STAGES;
         if (!mbar_wait(empty_bar(st), (rnd - 1) & 1)) {
@@ -133,7 +141,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           break;
         }
         load_w(it);
-        tma_load_3d(base + st * STAGE + W_STAGE_BYTES, &tmX, (kb0 + it) * BK, ea.row0, 0, full_bar(st), pol_x);
+        tma_load_3d(base + st * STAGE + W_STAGE_BYTES, xmap, (kb0 + it) * BK, row0, 0, full_bar(st), pol_x);
       }
     }
     __syncwarp();
@@ -154,15 +162,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           for (int h = 0; h < 2; h++) {
             const uint64_t adesc = smem_desc(sW + h * (128 * BK * 2) + kk * 32);
             const uint32_t d = tmem_base + (uint32_t)(h * AW);
-            if (MERGE) {
-              tc_mma(d, adesc, smem_desc(sX + kk * 32), IDESC, (it == 0 && kk == 0) ? 0u : 1u);
-            } else {
-#pragma unroll
-              for (int limb = 0; limb < 2; limb++) {
-                const uint64_t bdesc = smem_desc(sX + limb * (TN * BK * 2) + kk * 32);
-                tc_mma(d, adesc, bdesc, IDESC, (it == 0 && kk == 0 && limb == 0) ? 0u : 1u);
-              }
-            }
+            tc_mma(d, adesc, smem_desc(sX + kk * 32), idesc, (it == 0 && kk == 0) ? 0u : 1u);
           }
         }
         tc_commit(empty_bar(st));
@@ -180,10 +180,15 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       float sc = 1.f;
       if (ea.ssq_in) {
         float ss = 0.f;
-        for (int j = 0; j < ea.nt_in; j++) ss += ea.ssq_in[(size_t)(ea.row0 + et) * ea.nt_in + j];
+        for (int j = 0; j < ea.nt_in; j++) ss += ea.ssq_in[(size_t)(row0 + et) * ea.nt_in + j];
         sc = rsqrtf(ss * ea.inv_k + ea.eps);
       }
       s_scale[et] = sc;
+      if (ea.mode == EPI_QKV) {
+        s_pos[et] = ea.rt.pos[row0 + et];
+        s_slot[et] = ea.rt.slot[row0 + et];
+        s_ep[et] = ea.rt.ep[row0 + et];
+      }
     }
     bool have = n_units > 0;
     if (have) {
@@ -197,24 +202,17 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     const uint32_t tadr = tmem_base + ((uint32_t)(q * 32) << 16);
     const int col = q * 32 + lane;                       // column within a 128-column half
 #pragma unroll 1
-    for (int c0 = 16 * wp; c0 < TN; c0 += 32) {
+    for (int c0 = 16 * wp; c0 < tn; c0 += 32) {
 #pragma unroll 1
       for (int hf = 0; hf < 2; hf++) {
         float v[16];
         if (have) {
-          uint32_t r0[16];
+          uint32_t r0[16], r1[16];
           tc_ld16(tadr + hf * AW + c0, r0);
-          if (MERGE) {
-            uint32_t r1[16];
-            tc_ld16(tadr + hf * AW + TN + c0, r1);
-            tc_wait_ld();
+          tc_ld16(tadr + hf * AW + tn + c0, r1);
+          tc_wait_ld();
 #pragma unroll
-            for (int j = 0; j < 16; j++) v[j] = __uint_as_float(r0[j]) + __uint_as_float(r1[j]);
-          } else {
-            tc_wait_ld();
-#pragma unroll
-            for (int j = 0; j < 16; j++) v[j] = __uint_as_float(r0[j]);
-          }
+          for (int j = 0; j < 16; j++) v[j] = __uint_as_float(r0[j]) + __uint_as_float(r1[j]);
         } else {
 #pragma unroll
           for (int j = 0; j < 16; j++) v[j] = 0.f;
@@ -237,7 +235,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     // units [tile KB + r KB / S, tile KB + (r + 1) KB / S) with tile = c / S, r = c % S).
     // Issued here, off the critical path of the epilogue warps.
     const int nct = ea.pf_tiles * ea.pf_S;
-    for (int c = blockIdx.x; c < nct; c += gridDim.x) {
+    for (int c = blockIdx.y * gridDim.x + blockIdx.x; c < nct; c += gridDim.x * gridDim.y) {
       const int ptile = c / ea.pf_S, r = c - ptile * ea.pf_S;
       const int pk0 = r * ea.pf_KB / ea.pf_S;
       int n = (r + 1) * ea.pf_KB / ea.pf_S - pk0;
@@ -260,13 +258,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     const int n = swiglu ? tile * 128 + c4 : tile * BM + c4;
     const bool col_ok = n < ea.N;                             // N % 4 == 0: all four or none
     const float *P_own = reinterpret_cast<const float *>(smem_raw + (base - smem_u32(smem_raw)));
-    const float *P_of[MAX_S];
-    {
-      cooperative_groups::cluster_group cluster = cooperative_groups::this_cluster();
-#pragma unroll
-      for (int sl = 0; sl < MAX_S; sl++)
-        P_of[sl] = (S == 1 || sl >= S) ? P_own : cluster.map_shared_rank(const_cast<float *>(P_own), (unsigned)sl);
-    }
+    cooperative_groups::cluster_group cluster = cooperative_groups::this_cluster();
     float4 gain = make_float4(1.f, 1.f, 1.f, 1.f);
     if (ea.mode == EPI_RESID && ea.gain && col_ok) gain = *reinterpret_cast<const float4 *>(ea.gain + n);
     // QKV: which of q / k / v and which half of a head the four columns lie in
@@ -278,7 +270,12 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       float4 p[MAX_S];
 #pragma unroll
       for (int sl = 0; sl < MAX_S; sl++)
-        if (sl < S) p[sl] = *reinterpret_cast<const float4 *>(P_of[sl] + off);
+        if (sl < S) {
+          // rank sl's copy of the same shared-memory address (mapped on the spot: an array of
+          // eight mapped pointers would cost sixteen registers)
+          const float *P = S == 1 ? P_own : cluster.map_shared_rank(const_cast<float *>(P_own), (unsigned)sl);
+          p[sl] = *reinterpret_cast<const float4 *>(P + off);
+        }
       float4 acc = p[0];
 #pragma unroll
       for (int sl = 1; sl < MAX_S; sl++)
@@ -291,24 +288,18 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       return acc;
     };
     for (int t = rank + rg * S; t < T; t += RG * S) {
-      const size_t row = (size_t)(ea.row0 + t);
+      const size_t row = (size_t)(row0 + t);
       const float sc = s_scale[t];
       // global operands first
       float4 xo = make_float4(0.f, 0.f, 0.f, 0.f), cs01 = xo, cs23 = xo;
-      int slot = 0, ep = 0;
       if (ea.mode == EPI_RESID && ea.accumulate && col_ok)
         xo = *reinterpret_cast<const float4 *>(ea.x + row * ea.N + n);
-      if (ea.mode == EPI_QKV) {
-        if (rot) {
-          const float2 *cs = ea.rope_tab + (size_t)ea.rt.pos[row] * half + (lo ? jq : jq - half);
-          cs01 = *reinterpret_cast<const float4 *>(cs);
-          cs23 = *reinterpret_cast<const float4 *>(cs + 2);
-        }
-        if (which > 0) {
-          slot = ea.rt.slot[row];
-          ep = ea.rt.ep[row];
-        }
+      if (rot) {
+        const float2 *cs = ea.rope_tab + (size_t)s_pos[t] * half + (lo ? jq : jq - half);
+        cs01 = *reinterpret_cast<const float4 *>(cs);
+        cs23 = *reinterpret_cast<const float4 *>(cs + 2);
       }
+      const int slot = ea.mode == EPI_QKV ? s_slot[t] : 0, ep = ea.mode == EPI_QKV ? s_ep[t] : 0;
       float4 v = partial_sum(t * BM + c4);
       if (ea.mode == EPI_PLAIN) {
         if (col_ok)
@@ -362,7 +353,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       const int t = rank + et * S;
       if (t < T) {
         const int w0 = 2 * (et & 3);
-        ea.ssq_out[(size_t)(ea.row0 + t) * tiles + tile] = s_red[w0][t] + s_red[w0 + 1][t];
+        ea.ssq_out[(size_t)(row0 + t) * tiles + tile] = s_red[w0][t] + s_red[w0 + 1][t];
       }
     }
   }
@@ -381,8 +372,8 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 }
 
 template <int TN>
-inline cudaError_t launch_tn(const CUtensorMap &tmW, const CUtensorMap &tmX, const EpiArgs &ea, int tiles, int KB,
-                             int S, int *err, cudaStream_t st, bool pdl) {
+inline cudaError_t launch_tn(const CUtensorMap &tmW, const CUtensorMap &tmX, const CUtensorMap &tmXtail,
+                             const EpiArgs &ea, int tiles, int KB, int S, int *err, cudaStream_t st, bool pdl) {
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(gemm_ck_kernel<TN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -391,7 +382,7 @@ inline cudaError_t launch_tn(const CUtensorMap &tmW, const CUtensorMap &tmX, con
     attr_set = true;
   }
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(tiles * S);
+  cfg.gridDim = dim3(tiles * S, (ea.T + MAX_T - 1) / MAX_T);
   cfg.blockDim = dim3(THREADS);
   cfg.dynamicSmemBytes = smem_bytes(TN);
   cfg.stream = st;
@@ -404,15 +395,15 @@ inline cudaError_t launch_tn(const CUtensorMap &tmW, const CUtensorMap &tmX, con
   at[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = pdl ? 2 : 1;
-  return cudaLaunchKernelEx(&cfg, gemm_ck_kernel<TN>, tmW, tmX, ea, KB, err);
+  return cudaLaunchKernelEx(&cfg, gemm_ck_kernel<TN>, tmW, tmX, tmXtail, ea, KB, err);
 }
 
 // How many clusters of each size 1..MAX_S can be resident at once (index = size; 0 = unknown).
 struct ClusterFit {
   int max_active[MAX_S + 1];
 };
-// Asks the occupancy calculator about the TN = 32 instantiation (all instantiations use about
-// the same shared memory and one CTA per SM).
+// Asks the occupancy calculator about the TN = 32 instantiation (every instantiation uses most
+// of an SM's shared memory: one CTA per SM).
 inline ClusterFit query_cluster_fit() {
   ClusterFit f = {};
   cudaFuncSetAttribute(gemm_ck_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(32));
@@ -434,23 +425,43 @@ inline ClusterFit query_cluster_fit() {
   cudaGetLastError();
   return f;
 }
-// K slices per tile: the largest cluster size whose `tiles` clusters are all resident at once
-// (a second wave would double the time), each slice keeping at least four K blocks.
-inline int slices_for(int tiles, int KB, const ClusterFit &fit) {
+// K slices per tile for `units` (tile, row chunk) pairs of KB blocks each; every slice keeps at
+// least four K blocks. When the units fit on the GPU at once: the largest cluster size whose
+// `units` clusters are all resident together (a second wave would double the time). Otherwise
+// (more units than SMs: prefill) clusters run in waves and a CTA's time is a fixed part (start,
+// reduction, epilogue: about what 16 K blocks take) plus its K blocks, so the cost of a choice
+// is waves x (16 + blocks per slice), ties to the smaller cluster.
+inline int slices_for(int units, int KB, const ClusterFit &fit) {
+  const int fit1 = fit.max_active[1] > 0 ? fit.max_active[1] : 148;
   int best = 1;
-  for (int S = 2; S <= MAX_S; S++)
-    if (fit.max_active[S] >= tiles && KB / S >= 4) best = S;
+  if (units <= fit1) {
+    for (int S = 2; S <= MAX_S; S++)
+      if (fit.max_active[S] >= units && KB / S >= 4) best = S;
+    return best;
+  }
+  long best_cost = -1;
+  for (int S = 1; S <= MAX_S; S++) {
+    const int fits = S == 1 ? fit1 : fit.max_active[S];
+    if (fits <= 0 || (S > 1 && KB / S < 4)) continue;
+    const long cost = (long)((units + fits - 1) / fits) * (16 + (KB + S - 1) / S);
+    if (best_cost < 0 || cost < best_cost) {
+      best_cost = cost;
+      best = S;
+    }
+  }
   return best;
 }
 
-// One launch over ea.T <= 128 rows; tmX must have been made with TN = tn_of(ea.T).
-inline cudaError_t launch(const CUtensorMap &tmW, const CUtensorMap &tmX, const EpiArgs &ea, int tiles, int KB,
-                          int S, int *err, cudaStream_t st, bool pdl) {
+// One launch over ea.T rows in chunks of 128 (grid y). tmX: the X map with box rows
+// tn_of(min(ea.T, 128)); tmXtail: the map for the last chunk when ea.T > 128 (box rows
+// ea.tn_tail), else unused.
+inline cudaError_t launch(const CUtensorMap &tmW, const CUtensorMap &tmX, const CUtensorMap &tmXtail,
+                          const EpiArgs &ea, int tiles, int KB, int S, int *err, cudaStream_t st, bool pdl) {
   switch (tn_of(ea.T)) {
-    case 16: return launch_tn<16>(tmW, tmX, ea, tiles, KB, S, err, st, pdl);
-    case 32: return launch_tn<32>(tmW, tmX, ea, tiles, KB, S, err, st, pdl);
-    case 64: return launch_tn<64>(tmW, tmX, ea, tiles, KB, S, err, st, pdl);
-    default: return launch_tn<128>(tmW, tmX, ea, tiles, KB, S, err, st, pdl);
+    case 16: return launch_tn<16>(tmW, tmX, tmX, ea, tiles, KB, S, err, st, pdl);
+    case 32: return launch_tn<32>(tmW, tmX, tmX, ea, tiles, KB, S, err, st, pdl);
+    case 64: return launch_tn<64>(tmW, tmX, tmX, ea, tiles, KB, S, err, st, pdl);
+    default: return launch_tn<128>(tmW, tmX, tmXtail, ea, tiles, KB, S, err, st, pdl);
   }
 }
 

@@ -37,16 +37,16 @@ constexpr int MAX_T = 128;
 
 __host__ __device__ constexpr int tn_of(int T) { return T <= 16 ? 16 : (T <= 32 ? 32 : (T <= 64 ? 64 : 128)); }
 __host__ __device__ constexpr int stage_bytes(int TN) { return W_STAGE_BYTES + 2 * TN * BK * 2; }
-// The ring leaves ~60 KB of the SM's shared memory free, so that the small kernels between two
-// GEMMs can be resident next to a GEMM CTA while it prefetches weights.
-__host__ __device__ constexpr int stages_of(int TN) { return RING_BUDGET / stage_bytes(TN); }
+// Up to 64 rows the ring leaves ~60 KB of the SM's shared memory free, so that the small kernels
+// between two GEMMs can be resident next to a GEMM CTA while it prefetches weights. At 128 rows
+// (prefill) a stage is 64 KB and two of them cannot cover the load latency: the ring takes a
+// third and most of the SM's shared memory.
+__host__ __device__ constexpr int stages_of(int TN) { return TN > 64 ? 3 : RING_BUDGET / stage_bytes(TN); }
 __host__ __device__ constexpr int smem_bytes(int TN) { return stages_of(TN) * stage_bytes(TN) + 1024 + 256; }
-// Up to 64 rows both limbs of X form ONE MMA operand (N = 2 TN: hi rows, then lo rows) and the
-// two column groups are added in the epilogue; at 128 rows the limbs are two MMAs into the
-// same TN columns. Either way an accumulator is acc_width(TN) TMEM columns wide.
-__host__ __device__ constexpr bool merged_limbs(int TN) { return TN <= 64; }
-__host__ __device__ constexpr int acc_width(int TN) { return merged_limbs(TN) ? 2 * TN : TN; }
-__host__ __device__ constexpr int tmem_cols(int TN) { return 4 * acc_width(TN); }      // 128, 256, 512, 512
+// Both limbs of X form ONE MMA operand (N = 2 TN: hi rows, then lo rows; 256 at most, the
+// largest N of an M = 128 MMA), which reads the weight operand from shared memory once for
+// both; the two column groups of the accumulator are added in the epilogue.
+__host__ __device__ constexpr int acc_width(int TN) { return 2 * TN; }
 
 // ------------------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -189,7 +189,8 @@ enum EpiMode {
 struct EpiArgs {
   int mode;
   int row0;              // first row of this launch within the call's row range
-  int T;                 // rows of this launch (<= 128)
+  int T;                 // rows of this launch; CTAs with blockIdx.y = c take rows [128 c, 128 c + 128)
+  int tn_tail;           // tn_of(rows of the last 128-row chunk): its X box and MMA width
   int N;                 // output columns (EPI_SWIGLU: F, the width of gate and of up)
   int up_off;            // EPI_SWIGLU: row of W where the up projection starts (F)
   const bf16 *wpacked;   // weights repacked by pack_weights_kernel (one contiguous 32 KB block per

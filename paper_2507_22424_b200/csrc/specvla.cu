@@ -267,7 +267,7 @@ cudaLaunchConfig_t launch_cfg(dim3 grid, dim3 block, cudaStream_t st, cudaLaunch
   } while (0)
 
 // One GEMM over R rows of A against W with the fused epilogue described by `ea` (mode and
-// outputs; the row range is filled in here). Rows go in launches of 128.
+// outputs; the row range is filled in here): one launch, 128 rows per CTA.
 // next: the matrix of the GEMM that will follow (its head is prefetched into L2), or NULL.
 int gemm(specvla_ctx *ctx, const XBuf &A, const WMat &W, int R, gemm_tc::EpiArgs ea, cudaStream_t st, int cls,
          const WMat *next = nullptr, bool next_swiglu = false) {
@@ -280,28 +280,28 @@ int gemm(specvla_ctx *ctx, const XBuf &A, const WMat &W, int R, gemm_tc::EpiArgs
   ea.eps = ctx->desc.rms_eps;
   const bool prof = (ctx->prof_mask & ctx->phase) && 2 * (ctx->prof_used + 1) <= (int)ctx->prof_ev.size();
   if (prof) CU(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used], st));
-  const int S = gemm_ck::slices_for(tiles, KB, ctx->fit);
-  for (int r0 = 0; r0 < R; r0 += gemm_tc::MAX_T) {
-    ea.row0 = r0;
-    ea.T = R - r0 < gemm_tc::MAX_T ? R - r0 : gemm_tc::MAX_T;
-    ea.pf_w = nullptr;
-    if (next && next->packed && ctx->use_l2_prefetch && r0 + gemm_tc::MAX_T >= R) {
-      // last launch over W: start pulling the next matrix (up to L2_PREFETCH_BYTES of it)
-      ea.pf_tiles = next_swiglu ? (next->N / 2 + 127) / 128 : (next->N + SV_TILE_ROWS - 1) / SV_TILE_ROWS;
-      ea.pf_KB = (next->K + gemm_tc::BK - 1) / gemm_tc::BK;
-      ea.pf_S = gemm_ck::slices_for(ea.pf_tiles, ea.pf_KB, ctx->fit);
-      const size_t per_cta = L2_PREFETCH_BYTES / ((size_t)ea.pf_tiles * ea.pf_S) / gemm_tc::W_STAGE_BYTES;
-      ea.pf_units = per_cta < 1 ? 1 : (int)per_cta;
-      ea.pf_w = next->packed;
-    }
-    CU(gemm_ck::launch(W.map, A.map[tn_index(gemm_tc::tn_of(ea.T))], ea, tiles, KB, S, ctx->err, st,
-                       ctx->use_pdl));
-    ctx->launches++;
+  const int chunks = (R + gemm_tc::MAX_T - 1) / gemm_tc::MAX_T;
+  const int S = gemm_ck::slices_for(tiles * chunks, KB, ctx->fit);
+  ea.row0 = 0;
+  ea.T = R;
+  ea.tn_tail = gemm_tc::tn_of(R - (chunks - 1) * gemm_tc::MAX_T);
+  ea.pf_w = nullptr;
+  if (next && next->packed && ctx->use_l2_prefetch) {
+    // start pulling the next matrix (up to L2_PREFETCH_BYTES of it)
+    ea.pf_tiles = next_swiglu ? (next->N / 2 + 127) / 128 : (next->N + SV_TILE_ROWS - 1) / SV_TILE_ROWS;
+    ea.pf_KB = (next->K + gemm_tc::BK - 1) / gemm_tc::BK;
+    ea.pf_S = gemm_ck::slices_for(ea.pf_tiles * chunks, ea.pf_KB, ctx->fit);
+    const size_t per_cta = L2_PREFETCH_BYTES / ((size_t)ea.pf_tiles * ea.pf_S) / gemm_tc::W_STAGE_BYTES;
+    ea.pf_units = per_cta < 1 ? 1 : (int)per_cta;
+    ea.pf_w = next->packed;
   }
+  CU(gemm_ck::launch(W.map, A.map[tn_index(gemm_tc::tn_of(R))], A.map[tn_index(ea.tn_tail)], ea, tiles, KB, S,
+                     ctx->err, st, ctx->use_pdl));
+  ctx->launches++;
   if (prof) {
     CU(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used + 1], st));
     ctx->prof_cls[ctx->prof_used++] = cls;
-    ctx->prof_bytes[cls] += (double)W.N * W.K * sizeof(bf16) * ((R + gemm_tc::MAX_T - 1) / gemm_tc::MAX_T);
+    ctx->prof_bytes[cls] += (double)W.N * W.K * sizeof(bf16);
   }
   return SPECVLA_OK;
 }
@@ -1167,14 +1167,14 @@ int specvla_gemm(const float *X, const void *W, float *Y, int T, int N, int K, v
   ea.out = Y;
   ea.ldo = N;
   static const gemm_ck::ClusterFit fit = gemm_ck::query_cluster_fit();
-  const int S = gemm_ck::slices_for(tiles, KB, fit);
-  for (int r0 = 0; r0 < T; r0 += gemm_tc::MAX_T) {
-    ea.row0 = r0;
-    ea.T = T - r0 < gemm_tc::MAX_T ? T - r0 : gemm_tc::MAX_T;
-    if (gemm_ck::launch(mw, mx[tn_index(gemm_tc::tn_of(ea.T))], ea, tiles, KB, S, err, st, false) !=
-        cudaSuccess)
-      return SPECVLA_ERR_CUDA;
-  }
+  const int chunks = (T + gemm_tc::MAX_T - 1) / gemm_tc::MAX_T;
+  const int S = gemm_ck::slices_for(tiles * chunks, KB, fit);
+  ea.row0 = 0;
+  ea.T = T;
+  ea.tn_tail = gemm_tc::tn_of(T - (chunks - 1) * gemm_tc::MAX_T);
+  if (gemm_ck::launch(mw, mx[tn_index(gemm_tc::tn_of(T))], mx[tn_index(ea.tn_tail)], ea, tiles, KB, S, err, st,
+                      false) != cudaSuccess)
+    return SPECVLA_ERR_CUDA;
   return cudaGetLastError() == cudaSuccess ? SPECVLA_OK : SPECVLA_ERR_CUDA;
 }
 
