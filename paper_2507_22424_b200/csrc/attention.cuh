@@ -1,7 +1,7 @@
 // Tree-mask attention (Section 3.2 / 4.1: every draft-tree row is verified in one forward,
 // each conditioned on its own path). Row t attends cache slots [0, nvis[t]) plus the slots
-// tbase[t] + b for every bit b of its 128-bit mask. Queries, keys, values, scores, softmax
-// and the weighted sum are fp32; the output is written as two bf16 limbs for the
+// tbase[t] + b for every bit b of its 128-bit mask. Queries, keys and values are fp32 in
+// memory; softmax and accumulation are fp32; the output is written as two bf16 limbs for the
 // O-projection GEMM.
 //
 // One CTA handles one head, a block of up to 32 consecutive rows of ONE episode and one slice
@@ -9,15 +9,15 @@
 // 32 slots, so a K/V row is read from L2/HBM once per row block instead of once per row; the
 // next tile is fetched into registers while the current one is used.
 //
-// All arithmetic is fp32 FMA, organised so that shared-memory traffic does not limit it:
-// a warp owns four rows. For the scores a lane owns four keys of the tile (k, k + 8, k + 16,
-// k + 24) and a quarter of the head dimension, with that quarter of its four query rows kept
-// in registers for the whole kernel, so that a step costs four conflict-free K loads per 64
-// FMAs; the quarters are added with two warp shuffles. The softmax statistics of a row
-// (online softmax: running max and sum) live entirely inside its warp. For the weighted sum
-// a lane owns head-dim columns and reads P four keys at a time. With several key slices each
-// CTA parks (max, sum, unnormalised output) and bumps a counter; the CTA that arrives last
-// merges the slices in ascending order (deterministic, nobody waits).
+// The two contractions run on the tensor cores with fp32-grade operands: every operand (q
+// scaled, k, v, the softmax weights p) is split into two bf16 limbs (hi = bf16(x), lo =
+// bf16(x - hi): 16 mantissa bits) when it is written to shared memory, and a product is three
+// m16n8k16 MMAs (hi hi + hi lo + lo hi) accumulated in fp32. A tile goes through three phases
+// separated by CTA barriers: scores (warp = 16 rows x 8 keys, q fragments kept in registers
+// for the whole kernel), online softmax (warp = 4 rows, lane = key; running max and sum live
+// in that warp's registers), weighted sum (warp = 16 rows x a quarter of the head dimension).
+// With several key slices each CTA parks (max, sum, unnormalised output) and bumps a counter;
+// the CTA that arrives last merges the slices in ascending order (deterministic, nobody waits).
 #pragma once
 #include "common.cuh"
 
@@ -48,35 +48,68 @@ __host__ __device__ inline int blocks_of(const EpArgs &ea) {
   for (int i = 0; i < ea.n_ep; i++) n += (ea.nrows[i] + RB - 1) / RB;
   return n;
 }
-// K and V tiles (rows padded by 4 floats: conflict-free float4 reads by key) and P.
+// Shared memory: bf16 limb planes of Q [RB], K [KT], V [KT] (row pitch DH + 8: rows 16-byte
+// aligned and ldmatrix conflict-free), of P [RB][KT + 8], and the fp32 scores [RB][KT + 4].
 template <int DH> constexpr int smem_bytes() {
-  return (2 * KT * (DH + 4) + RB * (KT + 4)) * (int)sizeof(float);
+  return (2 * (RB + 2 * KT) * (DH + 8) + 2 * RB * (KT + 8)) * (int)sizeof(bf16) + RB * (KT + 4) * (int)sizeof(float);
+}
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+// c += a (16 x 16, row) * b (16 x 8, col), bf16 operands, fp32 accumulator
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// four floats -> four hi limbs and four lo limbs, 8 bytes each
+__device__ __forceinline__ void split4(const float4 v, uint2 &hi, uint2 &lo) {
+  const __nv_bfloat162 h01 = __floats2bfloat162_rn(v.x, v.y), h23 = __floats2bfloat162_rn(v.z, v.w);
+  const float2 f01 = __bfloat1622float2(h01), f23 = __bfloat1622float2(h23);
+  const __nv_bfloat162 l01 = __floats2bfloat162_rn(v.x - f01.x, v.y - f01.y);
+  const __nv_bfloat162 l23 = __floats2bfloat162_rn(v.z - f23.x, v.w - f23.y);
+  hi = make_uint2(*reinterpret_cast<const uint32_t *>(&h01), *reinterpret_cast<const uint32_t *>(&h23));
+  lo = make_uint2(*reinterpret_cast<const uint32_t *>(&l01), *reinterpret_cast<const uint32_t *>(&l23));
 }
 
 template <int DH>
 __global__ void __launch_bounds__(THREADS, 1)
 tree_attention_kernel(const EpArgs ea, const Args a) {
-  constexpr int PER = DH / 32;            // head-dim columns per lane in the weighted sum
+  constexpr int PER = DH / 32;            // head-dim columns per lane in the slice merge
   constexpr int C4 = DH / 4;              // float4 per row
-  constexpr int LK = DH + 4;              // pitch of sK and sV rows
-  constexpr int LP = KT + 4;              // pitch of sP rows
+  constexpr int LD = DH + 8;              // pitch (bf16) of the Q, K, V limb planes
+  constexpr int LP = KT + 8;              // pitch (bf16) of the P limb planes
+  constexpr int LS = KT + 4;              // pitch (float) of the scores
   constexpr int NLD = KT * C4 / THREADS;  // float4 per thread per tile
-  constexpr int DPG = DH / 4;             // head-dim elements per lane group in the scores
-  constexpr int NS = DPG / 4;             // float4 steps over them
-  extern __shared__ __align__(16) float smem[];
-  float *sK = smem;                       // [KT][LK]
-  float *sV = sK + KT * LK;               // [KT][LK]
-  float *sP = sV + KT * LK;               // [RB][LP]
+  constexpr int KS = DH / 16;             // k steps of the score MMAs
+  constexpr int NB = DH / 32;             // 8-column blocks of a warp's quarter of the head dim
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  bf16 *sQh = reinterpret_cast<bf16 *>(smem_raw);   // [RB][LD]
+  bf16 *sQl = sQh + RB * LD;
+  bf16 *sKh = sQl + RB * LD;                        // [KT][LD]
+  bf16 *sKl = sKh + KT * LD;
+  bf16 *sVh = sKl + KT * LD;
+  bf16 *sVl = sVh + KT * LD;
+  bf16 *sPh = sVl + KT * LD;                        // [RB][LP]
+  bf16 *sPl = sPh + RB * LP;
+  float *sS = reinterpret_cast<float *>(sPl + RB * LP);   // [RB][LS]
   __shared__ int s_nvis[RB], s_tbase[RB], s_kmax;
   __shared__ uint32_t s_mask[RB][4];
+  __shared__ float s_corr[RB], s_m[RB], s_l[RB];
   __shared__ int s_last;
-  // This kernel needs the whole register file of its SM (the query rows live in registers):
-  // the GEMM that follows is let in only once the tile loop is over (pdl_launch below), not
-  // at the start, or its waiting CTAs would take the registers and push this grid into waves.
+  // The GEMM that follows is let in only once the tile loop is over (pdl_launch below): its
+  // waiting CTAs would otherwise take registers and shared memory and push this grid into waves.
   pdl_wait();
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int gk = lane >> 3, tc = lane & 7;         // quarter of the head dimension / key column
+  const int mb = warp & 1, wq = warp >> 1;         // 16-row block; key octet (scores) / head-dim quarter (sum)
   const int h = blockIdx.y, hd = a.H * DH;
   int bid = blockIdx.x / a.splits;
   const int sp = blockIdx.x - bid * a.splits;
@@ -117,34 +150,47 @@ tree_attention_kernel(const EpArgs ea, const Args a) {
     for (int o = 16; o > 0; o >>= 1) km = max(km, __shfl_xor_sync(0xffffffffu, km, o));
     if (tid == 0) s_kmax = min(km, a.max_seq);
   }
-  // this lane's quarter of its warp's four query rows, scaled, for the whole kernel
-  float4 qreg[4][NS];
+  // the block's query rows, scaled, as limbs (rows past nrows are zero)
 #pragma unroll
-  for (int i = 0; i < 4; i++) {
-    const int r = warp * 4 + i;
-#pragma unroll
-    for (int s4 = 0; s4 < NS; s4++) {
-      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (r < nrows) {
-        v = *reinterpret_cast<const float4 *>(a.q + (size_t)(row0 + r) * hd + h * DH + DPG * gk + 4 * s4);
-        v.x *= a.scale; v.y *= a.scale; v.z *= a.scale; v.w *= a.scale;
-      }
-      qreg[i][s4] = v;
+  for (int k = 0; k < RB * C4 / THREADS; k++) {
+    const int i = tid + k * THREADS;
+    const int r = i / C4, c = i % C4;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (r < nrows) {
+      v = *reinterpret_cast<const float4 *>(a.q + (size_t)(row0 + r) * hd + h * DH + c * 4);
+      v.x *= a.scale; v.y *= a.scale; v.z *= a.scale; v.w *= a.scale;
     }
+    uint2 hi, lo;
+    split4(v, hi, lo);
+    *reinterpret_cast<uint2 *>(sQh + r * LD + c * 4) = hi;
+    *reinterpret_cast<uint2 *>(sQl + r * LD + c * 4) = lo;
   }
   __syncthreads();
   const int kmax = s_kmax;
   const int tiles = (kmax + KT - 1) / KT;
   const int t0 = sp * tiles / a.splits, t1 = (sp + 1) * tiles / a.splits;
 
-  float m_run[4], l_run[4], acc[4][PER];
+  // A fragments of this warp's 16 query rows, both limbs, for the whole kernel
+  uint32_t qh[KS][4], ql[KS][4];
+  {
+    const int r = 16 * mb + (lane & 15), c = (lane >> 4) * 8;
 #pragma unroll
-  for (int rr = 0; rr < 4; rr++) {
-    m_run[rr] = -INFINITY;
-    l_run[rr] = 0.f;
-#pragma unroll
-    for (int k = 0; k < PER; k++) acc[rr][k] = 0.f;
+    for (int ks = 0; ks < KS; ks++) {
+      ldsm_x4(smem_addr(sQh + r * LD + 16 * ks + c), qh[ks]);
+      ldsm_x4(smem_addr(sQl + r * LD + 16 * ks + c), ql[ks]);
+    }
   }
+  float m_run[4], l_run[4];               // softmax statistics of rows 4 warp + i
+#pragma unroll
+  for (int i = 0; i < 4; i++) {
+    m_run[i] = -INFINITY;
+    l_run[i] = 0.f;
+  }
+  float acc[NB][4];                       // rows 16 mb + lane / 4 (+ 8), columns (DH / 4) wq + 8 nb + 2 (lane % 4) (+ 1)
+#pragma unroll
+  for (int nb = 0; nb < NB; nb++)
+#pragma unroll
+    for (int k = 0; k < 4; k++) acc[nb][k] = 0.f;
 
   float4 kreg[NLD], vreg[NLD];
   auto fetch = [&](int t) {
@@ -168,119 +214,122 @@ tree_attention_kernel(const EpArgs ea, const Args a) {
     for (int k = 0; k < NLD; k++) {
       const int i = tid + k * THREADS;
       const int j = i / C4, c = i % C4;
-      *reinterpret_cast<float4 *>(sK + j * LK + c * 4) = kreg[k];
-      *reinterpret_cast<float4 *>(sV + j * LK + c * 4) = vreg[k];
+      uint2 hi, lo;
+      split4(kreg[k], hi, lo);
+      *reinterpret_cast<uint2 *>(sKh + j * LD + c * 4) = hi;
+      *reinterpret_cast<uint2 *>(sKl + j * LD + c * 4) = lo;
+      split4(vreg[k], hi, lo);
+      *reinterpret_cast<uint2 *>(sVh + j * LD + c * 4) = hi;
+      *reinterpret_cast<uint2 *>(sVl + j * LD + c * 4) = lo;
     }
     __syncthreads();
     if (t + 1 < t1) fetch(t + 1);          // in flight while this tile is used
 
-    // ---- scores: rows 4 warp + i against keys tc + 8 j, this lane's quarter of the head dim
-    float sc[4][4];
-#pragma unroll
-    for (int i = 0; i < 4; i++)
-#pragma unroll
-      for (int j = 0; j < 4; j++) sc[i][j] = 0.f;
+    // ---- scores of rows 16 mb .. + 16 against keys 8 wq .. + 8
     {
-      const float *kp = sK + tc * LK + DPG * gk;
+      float sc[4] = {0.f, 0.f, 0.f, 0.f};
+      // B fragments two k steps at a time: lanes 0-7 / 8-15 address the keys' columns
+      // 32 kp, 32 kp + 8 (first step), lanes 16-23 / 24-31 the columns 32 kp + 16, + 24 (second)
+      const int key = 8 * wq + (lane & 7), c = (lane >> 3) * 8;
 #pragma unroll
-      for (int s4 = 0; s4 < NS; s4++) {
-        float4 kf[4];
-#pragma unroll
-        for (int j = 0; j < 4; j++) kf[j] = *reinterpret_cast<const float4 *>(kp + 8 * j * LK + 4 * s4);
-#pragma unroll
-        for (int i = 0; i < 4; i++)
-#pragma unroll
-          for (int j = 0; j < 4; j++)
-            sc[i][j] += (qreg[i][s4].x * kf[j].x + qreg[i][s4].y * kf[j].y) +
-                        (qreg[i][s4].z * kf[j].z + qreg[i][s4].w * kf[j].w);
+      for (int kp = 0; kp < KS / 2; kp++) {
+        uint32_t bh[4], bl[4];
+        ldsm_x4(smem_addr(sKh + key * LD + 32 * kp + c), bh);
+        ldsm_x4(smem_addr(sKl + key * LD + 32 * kp + c), bl);
+        mma_bf16(sc, qh[2 * kp], bh[0], bh[1]);
+        mma_bf16(sc, qh[2 * kp], bl[0], bl[1]);
+        mma_bf16(sc, ql[2 * kp], bh[0], bh[1]);
+        mma_bf16(sc, qh[2 * kp + 1], bh[2], bh[3]);
+        mma_bf16(sc, qh[2 * kp + 1], bl[2], bl[3]);
+        mma_bf16(sc, ql[2 * kp + 1], bh[2], bh[3]);
       }
+      float *dst = sS + (16 * mb + (lane >> 2)) * LS + 8 * wq + 2 * (lane & 3);
+      *reinterpret_cast<float2 *>(dst) = make_float2(sc[0], sc[1]);
+      *reinterpret_cast<float2 *>(dst + 8 * LS) = make_float2(sc[2], sc[3]);
     }
-    // add the four quarters: afterwards all four lane groups hold the full scores
-#pragma unroll
-    for (int i = 0; i < 4; i++)
-#pragma unroll
-      for (int j = 0; j < 4; j++) {
-        sc[i][j] += __shfl_xor_sync(0xffffffffu, sc[i][j], 8);
-        sc[i][j] += __shfl_xor_sync(0xffffffffu, sc[i][j], 16);
-      }
-    float corr[4];
+    __syncthreads();
+    // ---- online softmax of rows 4 warp + i, lane = key of the tile
 #pragma unroll
     for (int i = 0; i < 4; i++) {
       const int r = warp * 4 + i;
-      bool vis[4];
-      float mx = -INFINITY;
-#pragma unroll
-      for (int j = 0; j < 4; j++) {
-        const int slot = t * KT + tc + 8 * j;
-        vis[j] = slot < s_nvis[r];
-        const int b = slot - s_tbase[r];
-        if (!vis[j] && b >= 0 && b < 128) vis[j] = (s_mask[r][b >> 5] >> (b & 31)) & 1u;
-        if (vis[j]) mx = fmaxf(mx, sc[i][j]);
-      }
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+      const int slot = t * KT + lane;
+      bool vis = slot < s_nvis[r];
+      const int b = slot - s_tbase[r];
+      if (!vis && b >= 0 && b < 128) vis = (s_mask[r][b >> 5] >> (b & 31)) & 1u;
+      const float s = sS[r * LS + lane];
+      const float mx = warp_max(vis ? s : -INFINITY);
       const float mn = fmaxf(m_run[i], mx);
-      corr[i] = (mn == -INFINITY) ? 1.f : __expf(m_run[i] - mn);
+      const float corr = (mn == -INFINITY) ? 1.f : __expf(m_run[i] - mn);
       m_run[i] = mn;
-      float ps = 0.f;
-#pragma unroll
-      for (int j = 0; j < 4; j++) {
-        const float p = vis[j] ? __expf(sc[i][j] - mn) : 0.f;
-        ps += p;
-        if (gk == 0) sP[r * LP + tc + 8 * j] = p;
-      }
-      ps += __shfl_xor_sync(0xffffffffu, ps, 1);
-      ps += __shfl_xor_sync(0xffffffffu, ps, 2);
-      ps += __shfl_xor_sync(0xffffffffu, ps, 4);
-      l_run[i] = l_run[i] * corr[i] + ps;
+      const float p = vis ? __expf(s - mn) : 0.f;
+      l_run[i] = l_run[i] * corr + warp_sum(p);
+      const bf16 ph = __float2bfloat16(p);
+      sPh[r * LP + lane] = ph;
+      sPl[r * LP + lane] = __float2bfloat16(p - __bfloat162float(ph));
+      if (lane == 0) s_corr[r] = corr;
     }
-    __syncwarp();
-    // ---- weighted sum: lane = head-dim columns PER * lane .., same four rows, four keys a step
+    __syncthreads();
+    // ---- weighted sum: rows 16 mb .. + 16, head-dim columns (DH / 4) wq .. + DH / 4
+    {
+      const float c0 = s_corr[16 * mb + (lane >> 2)], c1 = s_corr[16 * mb + (lane >> 2) + 8];
 #pragma unroll
-    for (int rr = 0; rr < 4; rr++)
+      for (int nb = 0; nb < NB; nb++) {
+        acc[nb][0] *= c0;
+        acc[nb][1] *= c0;
+        acc[nb][2] *= c1;
+        acc[nb][3] *= c1;
+      }
+      const int pr = 16 * mb + (lane & 15), pc = (lane >> 4) * 8;
+      // V fragments (transposed loads): lanes 0-7 / 8-15 address keys 16 ks .. + 8 / + 8 .. + 16
+      // at one 8-column block, lanes 16-31 the same keys at the next block
+      const int vk = (lane & 7) + ((lane >> 3) & 1) * 8, vc = (DH / 4) * wq + (lane >> 4) * 8;
 #pragma unroll
-      for (int k = 0; k < PER; k++) acc[rr][k] *= corr[rr];
-#pragma unroll 2
-    for (int j4 = 0; j4 < KT; j4 += 4) {
-      float4 pf[4];
+      for (int ks = 0; ks < KT / 16; ks++) {
+        uint32_t ph[4], pl[4];
+        ldsm_x4(smem_addr(sPh + pr * LP + 16 * ks + pc), ph);
+        ldsm_x4(smem_addr(sPl + pr * LP + 16 * ks + pc), pl);
 #pragma unroll
-      for (int rr = 0; rr < 4; rr++) pf[rr] = *reinterpret_cast<const float4 *>(sP + (warp * 4 + rr) * LP + j4);
-#pragma unroll
-      for (int jj = 0; jj < 4; jj++) {
-        float vv[PER];
-        if (PER == 4) {
-          const float4 t4 = *reinterpret_cast<const float4 *>(sV + (j4 + jj) * LK + lane * 4);
-          vv[0] = t4.x; vv[1] = t4.y; vv[2 % PER] = t4.z; vv[3 % PER] = t4.w;
-        } else {
-          const float2 t2 = *reinterpret_cast<const float2 *>(sV + (j4 + jj) * LK + lane * 2);
-          vv[0] = t2.x; vv[1] = t2.y;
-        }
-#pragma unroll
-        for (int rr = 0; rr < 4; rr++) {
-          const float p = jj == 0 ? pf[rr].x : (jj == 1 ? pf[rr].y : (jj == 2 ? pf[rr].z : pf[rr].w));
-#pragma unroll
-          for (int k = 0; k < PER; k++) acc[rr][k] += p * vv[k];
+        for (int np = 0; np < NB / 2; np++) {
+          uint32_t vh[4], vl[4];
+          ldsm_x4_trans(smem_addr(sVh + (16 * ks + vk) * LD + vc + 16 * np), vh);
+          ldsm_x4_trans(smem_addr(sVl + (16 * ks + vk) * LD + vc + 16 * np), vl);
+          mma_bf16(acc[2 * np], ph, vh[0], vh[1]);
+          mma_bf16(acc[2 * np], ph, vl[0], vl[1]);
+          mma_bf16(acc[2 * np], pl, vh[0], vh[1]);
+          mma_bf16(acc[2 * np + 1], ph, vh[2], vh[3]);
+          mma_bf16(acc[2 * np + 1], ph, vl[2], vl[3]);
+          mma_bf16(acc[2 * np + 1], pl, vh[2], vh[3]);
         }
       }
     }
-    __syncwarp();
   }
 
   pdl_launch();
+  if (lane == 0) {
+#pragma unroll
+    for (int i = 0; i < 4; i++) {
+      s_m[warp * 4 + i] = m_run[i];
+      s_l[warp * 4 + i] = l_run[i];
+    }
+  }
+  __syncthreads();
+  const int ra = 16 * mb + (lane >> 2), rb = ra + 8;        // this thread's two rows
+  const int cbase = (DH / 4) * wq + 2 * (lane & 3);          // + 8 nb: its column pairs
   if (a.splits == 1) {
+    const float ia = 1.f / s_l[ra], ib = 1.f / s_l[rb];
 #pragma unroll
-    for (int rr = 0; rr < 4; rr++) {
-      const int r = warp * 4 + rr;
-      if (r >= nrows) continue;
-      const float inv = 1.f / l_run[rr];
+    for (int nb = 0; nb < NB; nb++) {
 #pragma unroll
-      for (int k = 0; k < PER; k++) {
-        const size_t idx = (size_t)(row0 + r) * hd + h * DH + lane * PER + k;
-        const float v = acc[rr][k] * inv;
-        const bf16 hi = __float2bfloat16(v);
-        a.out[idx] = hi;
-        a.out[a.out_plane + idx] = __float2bfloat16(v - __bfloat162float(hi));
+      for (int half = 0; half < 2; half++) {
+        const int r = half ? rb : ra;
+        if (r >= nrows) continue;
+        const float inv = half ? ib : ia;
+        const float v0 = acc[nb][2 * half] * inv, v1 = acc[nb][2 * half + 1] * inv;
+        const size_t idx = (size_t)(row0 + r) * hd + h * DH + cbase + 8 * nb;
+        const __nv_bfloat162 hi = __floats2bfloat162_rn(v0, v1);
+        const float2 hf = __bfloat1622float2(hi);
+        *reinterpret_cast<__nv_bfloat162 *>(a.out + idx) = hi;
+        *reinterpret_cast<__nv_bfloat162 *>(a.out + a.out_plane + idx) = __floats2bfloat162_rn(v0 - hf.x, v1 - hf.y);
       }
     }
     return;
@@ -290,15 +339,13 @@ tree_attention_kernel(const EpArgs ea, const Args a) {
   const int unit = gblock * a.H + h;
   float *mine = a.part + ((size_t)unit * a.splits + sp) * RB * (DH + 2);
 #pragma unroll
-  for (int rr = 0; rr < 4; rr++) {
-    const int r = warp * 4 + rr;
-    float *dst = mine + (size_t)r * (DH + 2);
-#pragma unroll
-    for (int k = 0; k < PER; k++) __stcg(dst + lane * PER + k, acc[rr][k]);
-    if (lane == 0) {
-      __stcg(dst + DH, m_run[rr]);
-      __stcg(dst + DH + 1, l_run[rr]);
-    }
+  for (int nb = 0; nb < NB; nb++) {
+    __stcg(reinterpret_cast<float2 *>(mine + (size_t)ra * (DH + 2) + cbase + 8 * nb), make_float2(acc[nb][0], acc[nb][1]));
+    __stcg(reinterpret_cast<float2 *>(mine + (size_t)rb * (DH + 2) + cbase + 8 * nb), make_float2(acc[nb][2], acc[nb][3]));
+  }
+  if (tid < RB) {
+    __stcg(mine + (size_t)tid * (DH + 2) + DH, s_m[tid]);
+    __stcg(mine + (size_t)tid * (DH + 2) + DH + 1, s_l[tid]);
   }
   __threadfence();
   __syncthreads();
