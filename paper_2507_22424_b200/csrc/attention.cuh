@@ -129,6 +129,15 @@ tree_attention_kernel(const EpArgs ea, const Args a) {
   const float *kbase = a.cache + (size_t)ea.eps[ei] * a.ep_stride + (size_t)h * DH;
   const float *vbase = kbase + (size_t)a.max_seq * hd;
 
+  // the block's query rows (rows past nrows are zero): requested first, used after the metadata
+  float4 qv[RB * C4 / THREADS];
+#pragma unroll
+  for (int k = 0; k < RB * C4 / THREADS; k++) {
+    const int i = tid + k * THREADS;
+    const int r = i / C4, c = i % C4;
+    qv[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (r < nrows) qv[k] = *reinterpret_cast<const float4 *>(a.q + (size_t)(row0 + r) * hd + h * DH + c * 4);
+  }
   if (tid < RB) {
     int nv = 0, tb = 0, km = 0;
     uint32_t m[4] = {0, 0, 0, 0};
@@ -150,47 +159,10 @@ tree_attention_kernel(const EpArgs ea, const Args a) {
     for (int o = 16; o > 0; o >>= 1) km = max(km, __shfl_xor_sync(0xffffffffu, km, o));
     if (tid == 0) s_kmax = min(km, a.max_seq);
   }
-  // the block's query rows, scaled, as limbs (rows past nrows are zero)
-#pragma unroll
-  for (int k = 0; k < RB * C4 / THREADS; k++) {
-    const int i = tid + k * THREADS;
-    const int r = i / C4, c = i % C4;
-    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (r < nrows) {
-      v = *reinterpret_cast<const float4 *>(a.q + (size_t)(row0 + r) * hd + h * DH + c * 4);
-      v.x *= a.scale; v.y *= a.scale; v.z *= a.scale; v.w *= a.scale;
-    }
-    uint2 hi, lo;
-    split4(v, hi, lo);
-    *reinterpret_cast<uint2 *>(sQh + r * LD + c * 4) = hi;
-    *reinterpret_cast<uint2 *>(sQl + r * LD + c * 4) = lo;
-  }
   __syncthreads();
   const int kmax = s_kmax;
   const int tiles = (kmax + KT - 1) / KT;
   const int t0 = sp * tiles / a.splits, t1 = (sp + 1) * tiles / a.splits;
-
-  // A fragments of this warp's 16 query rows, both limbs, for the whole kernel
-  uint32_t qh[KS][4], ql[KS][4];
-  {
-    const int r = 16 * mb + (lane & 15), c = (lane >> 4) * 8;
-#pragma unroll
-    for (int ks = 0; ks < KS; ks++) {
-      ldsm_x4(smem_addr(sQh + r * LD + 16 * ks + c), qh[ks]);
-      ldsm_x4(smem_addr(sQl + r * LD + 16 * ks + c), ql[ks]);
-    }
-  }
-  float m_run[4], l_run[4];               // softmax statistics of rows 4 warp + i
-#pragma unroll
-  for (int i = 0; i < 4; i++) {
-    m_run[i] = -INFINITY;
-    l_run[i] = 0.f;
-  }
-  float acc[NB][4];                       // rows 16 mb + lane / 4 (+ 8), columns (DH / 4) wq + 8 nb + 2 (lane % 4) (+ 1)
-#pragma unroll
-  for (int nb = 0; nb < NB; nb++)
-#pragma unroll
-    for (int k = 0; k < 4; k++) acc[nb][k] = 0.f;
 
   float4 kreg[NLD], vreg[NLD];
   auto fetch = [&](int t) {
@@ -207,7 +179,39 @@ tree_attention_kernel(const EpArgs ea, const Args a) {
       }
     }
   };
-  if (t0 < t1) fetch(t0);
+  if (t0 < t1) fetch(t0);                  // in flight while the queries are split
+
+  // the query rows, scaled, as limbs
+#pragma unroll
+  for (int k = 0; k < RB * C4 / THREADS; k++) {
+    const int i = tid + k * THREADS;
+    const int r = i / C4, c = i % C4;
+    float4 v = qv[k];
+    v.x *= a.scale; v.y *= a.scale; v.z *= a.scale; v.w *= a.scale;
+    uint2 hi, lo;
+    split4(v, hi, lo);
+    *reinterpret_cast<uint2 *>(sQh + r * LD + c * 4) = hi;
+    *reinterpret_cast<uint2 *>(sQl + r * LD + c * 4) = lo;
+  }
+  __syncthreads();
+
+  // A fragments of this warp's 16 query rows, both limbs, for the whole kernel
+  uint32_t qh[KS][4], ql[KS][4];
+  {
+    const int r = 16 * mb + (lane & 15), c = (lane >> 4) * 8;
+#pragma unroll
+    for (int ks = 0; ks < KS; ks++) {
+      ldsm_x4(smem_addr(sQh + r * LD + 16 * ks + c), qh[ks]);
+      ldsm_x4(smem_addr(sQl + r * LD + 16 * ks + c), ql[ks]);
+    }
+  }
+  float m_run = -INFINITY, l_run = 0.f;   // softmax statistics of row 4 warp + lane / 8
+  float acc[NB][4];                       // rows 16 mb + lane / 4 (+ 8), columns (DH / 4) wq + 8 nb + 2 (lane % 4) (+ 1)
+#pragma unroll
+  for (int nb = 0; nb < NB; nb++)
+#pragma unroll
+    for (int k = 0; k < 4; k++) acc[nb][k] = 0.f;
+
   for (int t = t0; t < t1; t++) {
     __syncthreads();                       // the previous tile is no longer being read
 #pragma unroll
@@ -227,7 +231,8 @@ tree_attention_kernel(const EpArgs ea, const Args a) {
 
     // ---- scores of rows 16 mb .. + 16 against keys 8 wq .. + 8
     {
-      float sc[4] = {0.f, 0.f, 0.f, 0.f};
+      // three chains (hi hi, hi lo, lo hi) instead of one of 3 DH / 16 dependent MMAs
+      float sc[4] = {0.f, 0.f, 0.f, 0.f}, sc1[4] = {0.f, 0.f, 0.f, 0.f}, sc2[4] = {0.f, 0.f, 0.f, 0.f};
       // B fragments two k steps at a time: lanes 0-7 / 8-15 address the keys' columns
       // 32 kp, 32 kp + 8 (first step), lanes 16-23 / 24-31 the columns 32 kp + 16, + 24 (second)
       const int key = 8 * wq + (lane & 7), c = (lane >> 3) * 8;
@@ -237,36 +242,56 @@ tree_attention_kernel(const EpArgs ea, const Args a) {
         ldsm_x4(smem_addr(sKh + key * LD + 32 * kp + c), bh);
         ldsm_x4(smem_addr(sKl + key * LD + 32 * kp + c), bl);
         mma_bf16(sc, qh[2 * kp], bh[0], bh[1]);
-        mma_bf16(sc, qh[2 * kp], bl[0], bl[1]);
-        mma_bf16(sc, ql[2 * kp], bh[0], bh[1]);
+        mma_bf16(sc1, qh[2 * kp], bl[0], bl[1]);
+        mma_bf16(sc2, ql[2 * kp], bh[0], bh[1]);
         mma_bf16(sc, qh[2 * kp + 1], bh[2], bh[3]);
-        mma_bf16(sc, qh[2 * kp + 1], bl[2], bl[3]);
-        mma_bf16(sc, ql[2 * kp + 1], bh[2], bh[3]);
+        mma_bf16(sc1, qh[2 * kp + 1], bl[2], bl[3]);
+        mma_bf16(sc2, ql[2 * kp + 1], bh[2], bh[3]);
       }
+#pragma unroll
+      for (int k = 0; k < 4; k++) sc[k] += sc1[k] + sc2[k];
       float *dst = sS + (16 * mb + (lane >> 2)) * LS + 8 * wq + 2 * (lane & 3);
       *reinterpret_cast<float2 *>(dst) = make_float2(sc[0], sc[1]);
       *reinterpret_cast<float2 *>(dst + 8 * LS) = make_float2(sc[2], sc[3]);
     }
     __syncthreads();
-    // ---- online softmax of rows 4 warp + i, lane = key of the tile
+    // ---- online softmax: eight lanes per row (row 4 warp + lane / 8), a lane has the keys
+    // lane % 8 + 8 j of the tile
+    {
+      const int r = warp * 4 + (lane >> 3), tc = lane & 7;
+      const int nv = s_nvis[r], tb = s_tbase[r];
+      float sv[4];
+      bool vis[4];
+      float mx = -INFINITY;
 #pragma unroll
-    for (int i = 0; i < 4; i++) {
-      const int r = warp * 4 + i;
-      const int slot = t * KT + lane;
-      bool vis = slot < s_nvis[r];
-      const int b = slot - s_tbase[r];
-      if (!vis && b >= 0 && b < 128) vis = (s_mask[r][b >> 5] >> (b & 31)) & 1u;
-      const float s = sS[r * LS + lane];
-      const float mx = warp_max(vis ? s : -INFINITY);
-      const float mn = fmaxf(m_run[i], mx);
-      const float corr = (mn == -INFINITY) ? 1.f : __expf(m_run[i] - mn);
-      m_run[i] = mn;
-      const float p = vis ? __expf(s - mn) : 0.f;
-      l_run[i] = l_run[i] * corr + warp_sum(p);
-      const bf16 ph = __float2bfloat16(p);
-      sPh[r * LP + lane] = ph;
-      sPl[r * LP + lane] = __float2bfloat16(p - __bfloat162float(ph));
-      if (lane == 0) s_corr[r] = corr;
+      for (int j = 0; j < 4; j++) {
+        const int slot = t * KT + tc + 8 * j;
+        vis[j] = slot < nv;
+        const int b = slot - tb;
+        if (!vis[j] && b >= 0 && b < 128) vis[j] = (s_mask[r][b >> 5] >> (b & 31)) & 1u;
+        sv[j] = sS[r * LS + tc + 8 * j];
+        if (vis[j]) mx = fmaxf(mx, sv[j]);
+      }
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+      const float mn = fmaxf(m_run, mx);
+      const float corr = (mn == -INFINITY) ? 1.f : __expf(m_run - mn);
+      m_run = mn;
+      float ps = 0.f;
+#pragma unroll
+      for (int j = 0; j < 4; j++) {
+        const float p = vis[j] ? __expf(sv[j] - mn) : 0.f;
+        ps += p;
+        const bf16 ph = __float2bfloat16(p);
+        sPh[r * LP + tc + 8 * j] = ph;
+        sPl[r * LP + tc + 8 * j] = __float2bfloat16(p - __bfloat162float(ph));
+      }
+      ps += __shfl_xor_sync(0xffffffffu, ps, 1);
+      ps += __shfl_xor_sync(0xffffffffu, ps, 2);
+      ps += __shfl_xor_sync(0xffffffffu, ps, 4);
+      l_run = l_run * corr + ps;
+      if (tc == 0) s_corr[r] = corr;
     }
     __syncthreads();
     // ---- weighted sum: rows 16 mb .. + 16, head-dim columns (DH / 4) wq .. + DH / 4
@@ -305,12 +330,9 @@ tree_attention_kernel(const EpArgs ea, const Args a) {
   }
 
   pdl_launch();
-  if (lane == 0) {
-#pragma unroll
-    for (int i = 0; i < 4; i++) {
-      s_m[warp * 4 + i] = m_run[i];
-      s_l[warp * 4 + i] = l_run[i];
-    }
+  if ((lane & 7) == 0) {
+    s_m[warp * 4 + (lane >> 3)] = m_run;
+    s_l[warp * 4 + (lane >> 3)] = l_run;
   }
   __syncthreads();
   const int ra = 16 * mb + (lane >> 2), rb = ra + 8;        // this thread's two rows
