@@ -16,9 +16,12 @@
 // separated by CTA barriers: scores (warp = 16 rows x 8 keys, q fragments kept in registers
 // for the whole kernel), online softmax (warp = 4 rows, lane = key; running max and sum live
 // in that warp's registers), weighted sum (warp = 16 rows x a quarter of the head dimension).
-// With several key slices each CTA parks (max, sum, unnormalised output) and bumps a counter;
-// the CTA that arrives last merges the slices in ascending order (deterministic, nobody waits).
+// With several key slices the CTAs of a row block form a thread-block cluster: each leaves
+// (max, sum, unnormalised output) in its own shared memory, and after one cluster barrier
+// every CTA merges a share of the rows, reading the slices over distributed shared memory in
+// ascending order (deterministic; nothing goes through global memory).
 #pragma once
+#include <cooperative_groups.h>
 #include "common.cuh"
 
 namespace attn {
@@ -26,7 +29,7 @@ namespace attn {
 constexpr int RB = 32;            // rows per block
 constexpr int KT = 32;            // key slots per tile
 constexpr int THREADS = 256;      // 8 warps x 4 rows
-constexpr int MAX_SPLITS = 8;
+constexpr int MAX_SPLITS = 8;         // key slices per row block = cluster size (8: the portable limit)
 constexpr int MAX_SPLIT_CTAS = 148;   // CTAs of a launch that uses more than one key slice
 
 struct Args {
@@ -38,9 +41,7 @@ struct Args {
   float scale;
   bf16 *out;               // two limbs, [rows][H * DH] each
   size_t out_plane;
-  int splits;              // key slices per row block
-  float *part;             // [block * H + head][split][RB][DH + 2] parked slices (splits > 1)
-  int *counters;           // [block * H + head], zero between launches
+  int splits;              // key slices per row block; the launch's cluster is (splits, 1, 1)
 };
 
 __host__ __device__ inline int blocks_of(const EpArgs &ea) {
@@ -103,7 +104,6 @@ tree_attention_kernel(const EpArgs ea, const Args a) {
   __shared__ int s_nvis[RB], s_tbase[RB], s_kmax;
   __shared__ uint32_t s_mask[RB][4];
   __shared__ float s_corr[RB], s_m[RB], s_l[RB];
-  __shared__ int s_last;
   // The GEMM that follows is let in only once the tile loop is over (pdl_launch below): its
   // waiting CTAs would otherwise take registers and shared memory and push this grid into waves.
   pdl_wait();
@@ -113,7 +113,6 @@ tree_attention_kernel(const EpArgs ea, const Args a) {
   const int h = blockIdx.y, hd = a.H * DH;
   int bid = blockIdx.x / a.splits;
   const int sp = blockIdx.x - bid * a.splits;
-  const int gblock = bid;
   int ei = 0;
   for (; ei < ea.n_ep; ei++) {
     const int nb = (ea.nrows[ei] + RB - 1) / RB;
@@ -357,42 +356,39 @@ tree_attention_kernel(const EpArgs ea, const Args a) {
     return;
   }
 
-  // several key slices: park this one, the last arrival merges
-  const int unit = gblock * a.H + h;
-  float *mine = a.part + ((size_t)unit * a.splits + sp) * RB * (DH + 2);
+  // several key slices: leave this one in shared memory (over the query planes, which were
+  // only needed for the fragments), then merge rows sp, sp + splits, ... from all slices
+  constexpr int LO = DH + 4;
+  float *sO = reinterpret_cast<float *>(smem_raw);          // [RB][LO]: output, then max and sum
 #pragma unroll
   for (int nb = 0; nb < NB; nb++) {
-    __stcg(reinterpret_cast<float2 *>(mine + (size_t)ra * (DH + 2) + cbase + 8 * nb), make_float2(acc[nb][0], acc[nb][1]));
-    __stcg(reinterpret_cast<float2 *>(mine + (size_t)rb * (DH + 2) + cbase + 8 * nb), make_float2(acc[nb][2], acc[nb][3]));
+    *reinterpret_cast<float2 *>(sO + ra * LO + cbase + 8 * nb) = make_float2(acc[nb][0], acc[nb][1]);
+    *reinterpret_cast<float2 *>(sO + rb * LO + cbase + 8 * nb) = make_float2(acc[nb][2], acc[nb][3]);
   }
   if (tid < RB) {
-    __stcg(mine + (size_t)tid * (DH + 2) + DH, s_m[tid]);
-    __stcg(mine + (size_t)tid * (DH + 2) + DH + 1, s_l[tid]);
+    sO[tid * LO + DH] = s_m[tid];
+    sO[tid * LO + DH + 1] = s_l[tid];
   }
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    const int old = atomicAdd(a.counters + unit, 1);
-    s_last = (old == a.splits - 1);
-    if (s_last) atomicExch(a.counters + unit, 0);
-  }
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
-  const float *all = a.part + (size_t)unit * a.splits * RB * (DH + 2);
-  // every load of a row's slices is issued before any is used: one latency, not one per slice
-#pragma unroll
-  for (int rr = 0; rr < 4; rr++) {
-    const int r = warp * 4 + rr;
-    if (r >= nrows) continue;
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+  cooperative_groups::cluster_group cluster = cooperative_groups::this_cluster();
+  for (int r = sp + a.splits * warp; r < nrows; r += a.splits * (THREADS / 32)) {
+    // every load of the row's slices is issued before any is used: one latency, not one per slice
     float ms[MAX_SPLITS], ls[MAX_SPLITS], os[MAX_SPLITS][PER];
 #pragma unroll
     for (int s2 = 0; s2 < MAX_SPLITS; s2++) {
-      const float *src = all + ((size_t)(s2 < a.splits ? s2 : 0) * RB + r) * (DH + 2);
-      ms[s2] = __ldcg(src + DH);
-      ls[s2] = __ldcg(src + DH + 1);
-#pragma unroll
-      for (int k = 0; k < PER; k++) os[s2][k] = __ldcg(src + lane * PER + k);
+      if (s2 < a.splits) {
+        const float *src = cluster.map_shared_rank(sO, (unsigned)s2) + r * LO;
+        ms[s2] = src[DH];
+        ls[s2] = src[DH + 1];
+        if (PER == 4) {
+          const float4 t4 = *reinterpret_cast<const float4 *>(src + lane * 4);
+          os[s2][0] = t4.x; os[s2][1] = t4.y; os[s2][2 % PER] = t4.z; os[s2][3 % PER] = t4.w;
+        } else {
+          const float2 t2 = *reinterpret_cast<const float2 *>(src + lane * 2);
+          os[s2][0] = t2.x; os[s2][1] = t2.y;
+        }
+      }
     }
     float M = -INFINITY;
 #pragma unroll
@@ -419,6 +415,9 @@ tree_attention_kernel(const EpArgs ea, const Args a) {
       a.out[a.out_plane + idx] = __float2bfloat16(v - __bfloat162float(hi));
     }
   }
+  // nobody leaves while a peer may still be reading its shared memory
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
 }  // namespace attn

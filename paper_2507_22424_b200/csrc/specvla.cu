@@ -84,8 +84,6 @@ struct specvla_ctx {
   float *ssq, *lm_ssq;          // per-row partial sums of squares of x / of the gathered LM-head rows
   bf16 *packed;                 // repacked weight matrices, one after the other
   size_t packed_elems;
-  float *att_part;              // parked key slices of the attention kernel
-  int *att_counters;            // its arrival counters (zero between launches)
   int lgs_rows;                 // rows of the logits buffer
 
   // GEMM operands, two bf16 limbs each: hi plane, then the lo plane `plane` elements later
@@ -193,8 +191,6 @@ size_t carve(specvla_ctx *c, char *base) {
                       gemm_tc::packed_elems(tiles256(d.d_model), 2 * d.d_model);
     c->packed = cv.take<bf16>(c->packed_elems);
   }
-  c->att_part = cv.take<float>((size_t)attn::MAX_SPLIT_CTAS * attn::RB * (d.head_dim + 2));
-  c->att_counters = cv.take<int>(attn::MAX_SPLIT_CTAS);
   c->lgs_rows = (int)(lm_rows > dr ? lm_rows : dr);
   c->lgs = cv.take<float>((size_t)c->lgs_rows * d.vocab);
   c->pend_feat = cv.take<float>(E * SV_MAX_PENDING * d.d_model);
@@ -343,8 +339,6 @@ int attention(specvla_ctx *ctx, const EpArgs &rows, const float *cache, size_t e
   a.scale = 1.f / sqrtf((float)d.head_dim);
   a.out = ctx->ao.p;
   a.out_plane = ctx->ao.plane;
-  a.part = ctx->att_part;
-  a.counters = ctx->att_counters;
   const int blocks = attn::blocks_of(rows);
   if (blocks < 1) return SPECVLA_OK;
   // few row blocks: slice the key range so that the launch still covers the SMs
@@ -355,9 +349,15 @@ int attention(specvla_ctx *ctx, const EpArgs &rows, const float *cache, size_t e
     if (a.splits > attn::MAX_SPLITS) a.splits = attn::MAX_SPLITS;
     if (a.splits < 1) a.splits = 1;
   }
+  // the key slices of a row block are one cluster (they merge through distributed shared memory)
   const dim3 grid(blocks * a.splits, d.n_heads);
-  cudaLaunchAttribute at;
-  cudaLaunchConfig_t cfg = launch_cfg(grid, dim3(attn::THREADS), st, &at, ctx->use_pdl);
+  cudaLaunchAttribute at[2];
+  cudaLaunchConfig_t cfg = launch_cfg(grid, dim3(attn::THREADS), st, &at[0], ctx->use_pdl);
+  at[cfg.numAttrs].id = cudaLaunchAttributeClusterDimension;
+  at[cfg.numAttrs].val.clusterDim.x = a.splits;
+  at[cfg.numAttrs].val.clusterDim.y = 1;
+  at[cfg.numAttrs].val.clusterDim.z = 1;
+  cfg.numAttrs++;
   if (d.head_dim == 128) {
     cfg.dynamicSmemBytes = attn::smem_bytes<128>();
     CU(cudaLaunchKernelEx(&cfg, attn::tree_attention_kernel<128>, rows, a));
@@ -620,7 +620,6 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
   cudaMemsetAsync(ctx->st, 0, sizeof(EpState) * desc->max_episodes);
   cudaMemsetAsync(ctx->trees, 0, sizeof(DevTree) * desc->max_episodes);
   cudaMemsetAsync(ctx->err, 0, 32 * sizeof(int));
-  cudaMemsetAsync(ctx->att_counters, 0, attn::MAX_SPLIT_CTAS * sizeof(int));
   cudaFuncSetAttribute(attn::tree_attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                        attn::smem_bytes<128>());
   cudaFuncSetAttribute(attn::tree_attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
