@@ -31,6 +31,11 @@ UNIT = "chunks/s"
 WEIGHT_BYTES_PER_VERIFY = 13_214_679_040      # 32 layers + LM head, bf16, read once
 
 
+# DRAM traffic of one gate/up launch at T = 27 from the ncu capture under profiles/ (bytes); to be
+# re-taken (or set to None) whenever gemm_ck.cuh changes.
+GATE_UP_DRAM_BYTES = 203_312_640 + 3_463_424
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -322,7 +327,10 @@ def run_ours(args, rank, local_rank, world):
         gpu_launches=launches,
         clocks=clocks,
         roofline=dict(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
-                      frac=(achieved / peaks["hbm_gbs"]) if achieved else None, traffic=None,
+                      frac=(achieved / peaks["hbm_gbs"]) if achieved else None, traffic=GATE_UP_DRAM_BYTES,
+                      traffic_source="ncu dram__bytes_read.sum + dram__bytes_write.sum of this launch "
+                                     "(profiles/gemm_ck_verify_T27_ncu_full.md); the ~20 MB above the weights "
+                                     "are the L2 prefetch of the next GEMM's weights",
                       kernel="weight-streaming GEMM, gate/up projection [22016 x 4096] at T=27 (verify)",
                       algorithmic_bytes_per_launch=alg_bytes, launches_timed=dom["launches"],
                       ms_per_launch=dom_ms, peak_source=peaks["source"] + " copy bandwidth",

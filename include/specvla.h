@@ -16,7 +16,7 @@
  *    float32. Activations are float32 between kernels and enter the bf16 tensor-core GEMMs
  *    as two bf16 limbs (hi + lo); the KV caches are float32. With single-limb bf16
  *    activations or a bf16 cache the logits of the 32-layer model drift by 0.1-0.2 from an
- *    exact forward, ten times the 2e-2 this library is held to. The workspace (KV caches, activations, partial-sum planes and the library's
+ *    exact forward, ten times the 2e-2 this library is held to. The workspace (KV caches, activations and the library's
  *    repacked copy of every weight matrix, about the size of the weights themselves) is one
  *    device buffer allocated by the caller, at least specvla_workspace_bytes() long, 1024-byte aligned;
  *    it must outlive the context and must not be touched while a call is in flight.
