@@ -202,6 +202,24 @@ def run_reference(args, rank, world):
     print(json.dumps(line), flush=True)
 
 
+# --------------------------------------------------------------------------- replicas
+def max_over_ranks(values, device, world):
+    """Each value's maximum over the ranks of the job: N GPUs run N independent replicas, and a
+    timed region lasts as long as its slowest replica. No other data crosses ranks."""
+    if world == 1:
+        return [float(v) for v in values]
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(v) for v in values], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def replica_throughput(world, steps, ms):
+    """Whole-job chunks/s: every rank finished `steps` chunks within `ms` (the slowest rank's time)."""
+    return world * steps / (ms / 1000.0)
+
+
 # --------------------------------------------------------------------------- CUDA arm
 def run_ours(args, rank, local_rank, world):
     import torch
@@ -286,15 +304,14 @@ def run_ours(args, rank, local_rank, world):
     prof = gpu.profile_read()
     gpu.profile(0)
 
-    if world > 1:
-        t = torch.tensor([ms, ms_e2e], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, ms_e2e = float(t[0]), float(t[1])
+    ms, ms_e2e = max_over_ranks([ms, ms_e2e], "cuda", world)
     if rank != 0:
+        gpu.close()
+        dist.destroy_process_group()
         return
     peaks = load_peaks()
-    value = world * args.steps / (ms / 1000.0)
-    e2e_value = world * args.steps / (ms_e2e / 1000.0)
+    value = replica_throughput(world, args.steps, ms)
+    e2e_value = replica_throughput(world, args.steps, ms_e2e)
     T = 1 + wl.tree.n_nodes
     verify_ms = ms_verify / max(1, iters)
     kv_bytes = desc.n_layers * 2 * (P + 3 + T) * desc.d_model * 2 + T * desc.n_layers * 2 * desc.d_model * 2
