@@ -297,6 +297,17 @@ def run_ours(args, rank, local_rank, world):
     e5.record()
     barrier()
     ms_ar = e4.elapsed_time(e5)
+    # --- depth pruning: an iteration drafts no deeper than the tokens still missing ------------
+    pr_shape = make_shape(wl.tree.branch, wl.tree.expand, prune=True)
+    gpu.generate_action([0], embeds, ids_host, [P], pr_shape, r, n_tok)
+    barrier()
+    e6, e7 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e6.record()
+    for _ in range(ar_steps):
+        pr_toks, _, pr_stats = gpu.generate_action([0], embeds, ids_host, [P], pr_shape, r, n_tok)
+    e7.record()
+    barrier()
+    ms_pr = e6.elapsed_time(e7)
     # --- per-GEMM device time of the verification phase (separate pass, same steps) -----
     gpu.profile(4)
     for _ in range(max(2, args.steps // 4)):
@@ -364,6 +375,9 @@ def run_ours(args, rank, local_rank, world):
         ar_baseline=dict(value=world * ar_steps / (ms_ar / 1000.0), unit=UNIT,
                          ms_per_decode_step=ar_ms_verify / (ar_steps * (n_tok - 1)),
                          same_tokens=bool(ar_toks == toks)),
+        depth_pruned=dict(value=world * ar_steps / (ms_pr / 1000.0), unit=UNIT, same_tokens=bool(pr_toks == toks),
+                          note="same call with tree_shape.prune = 1 (not Algorithm 1 as printed: iterations "
+                               "draft min(depth, missing tokens - 1) levels); `value` above is unpruned"),
         cpu_baseline=dict(value=cpu_val, unit=UNIT, cores=torch.get_num_threads(), kind="oracle",
                           sample=("oracle (float64) decoder layer over 290 and 27 rows, LM head over 27 "
                                   "rows, one draft level over 4 rows at 7B shapes; chunk = 33*t_layer290 + "
@@ -390,6 +404,8 @@ def run_micro(spec: str, steps: int, warmup: int):
     f = spec.split(":")
     if f[0] == "verify":
         return run_micro_verify(int(f[1]), int(f[2]) if len(f) > 2 else 27, steps, warmup)
+    if f[0] == "batch":
+        return run_micro_batch(int(f[1]) if len(f) > 1 else 16, steps, warmup)
     assert f[0] == "gemm" and len(f) in (4, 5), spec
     T, N, K = int(f[1]), int(f[2]), int(f[3])
     wbytes = N * K * 2
@@ -461,13 +477,63 @@ def run_micro_verify(n_layers: int, rows: int, steps: int, warmup: int):
     gpu.close()
 
 
+def run_micro_batch(n_ep: int, steps: int, warmup: int):
+    """`--micro batch[:E]`: the batched workload (C4: E ragged episodes of 276-316 prefix rows, 27-row
+    random trees, r = 4) on the full 7B-shaped target: prefill of all episodes in one call and
+    verification of all trees in one call, both tensor-bound; times and algorithmic TFLOP/s
+    (2 x 6.607e9 flop per row; the two-limb arithmetic does twice that)."""
+    import torch
+    from paper_2507_22424_b200.binding import SpecVLA
+    from synth_inputs import configs as C, data
+    torch.cuda.set_device(0)
+    desc = C.OPENVLA_7B
+    weights = data.make_weights(desc, C.C4.seed, device="cuda", with_draft=False)
+    pre = [data.make_prefix(C.C4, episode=e, device="cuda", prefix_seed=C.C4.extra["prefix_seed"])
+           for e in range(n_ep)]
+    lens = [len(i) for _, i in pre]
+    emb = torch.cat([e for e, _ in pre])
+    ids = torch.cat([i for _, i in pre]).tolist()
+    eps = list(range(n_ep))
+    gpu = SpecVLA(desc, weights, max_seq=512, max_episodes=n_ep, max_rows=n_ep * 320, action_only=True)
+    ms_p, ms_v = [], []
+    for i in range(warmup + steps):
+        a, b, c = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        a.record()
+        first = gpu.prefill(eps, emb, ids, lens)
+        b.record()
+        trees = []
+        for e in eps:
+            tok, par, dep = data.random_tree(27, desc, seed=50 + e, max_depth=5, root_token=first[e])
+            trees.append(dict(tokens=tok, parent=par, depth=dep))
+        torch.cuda.synchronize()
+        b2 = torch.cuda.Event(enable_timing=True)
+        b2.record()
+        gpu.verify_tree(eps, trees, C.C4.extra["r"])
+        c.record()
+        torch.cuda.synchronize()
+        if i >= warmup:
+            ms_p.append(a.elapsed_time(b))
+            ms_v.append(b2.elapsed_time(c))
+    mp, mv = statistics.median(ms_p), statistics.median(ms_v)
+    rows_p, rows_v = sum(lens), 27 * n_ep
+    peaks = load_peaks()
+    print(json.dumps(dict(micro="batch", episodes=n_ep, prefix_rows=rows_p, tree_rows=rows_v, steps=steps,
+                          prefill_ms=mp, verify_ms=mv,
+                          prefill_tflops=2 * 6.607e9 * rows_p / mp / 1e9,
+                          verify_tflops=2 * 6.607e9 * rows_v / mv / 1e9,
+                          bf16_peak_tflops=peaks.get("bf16_tflops"), peak_source=peaks["source"],
+                          note="algorithmic flops (one bf16 pass); the kernels run two limbs, i.e. twice these")),
+          flush=True)
+    gpu.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--micro", default=None, help="gemm:T:N:K[:M] or verify:L[:T] - small cases for kernel timing / ncu (see run_micro)")
+    ap.add_argument("--micro", default=None, help="gemm:T:N:K[:M], verify:L[:T] or batch[:E] - small cases for kernel timing / ncu (see run_micro)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

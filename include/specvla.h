@@ -93,6 +93,12 @@ typedef struct {
   int depth;
   int branch[SPECVLA_MAX_DEPTH];
   int expand[SPECVLA_MAX_DEPTH];
+  int prune;   /* read by specvla_generate_action only. 0: every iteration drafts `depth` levels and
+                * the chunk is clipped at the end (Algorithm 1 as printed). 1: an iteration whose
+                * episodes still miss at most k tokens drafts min(depth, k - 1) levels (the
+                * verification adds one token itself, deeper nodes could only be clipped), and
+                * none at all when k = 1. Same tokens at r = 0; at r > 0 the accepted path may be
+                * another equally valid one. */
 } specvla_tree_shape;
 
 /* One draft tree in HOST memory. Row 0 is the root (the last emitted token, not yet in the

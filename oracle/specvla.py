@@ -269,15 +269,29 @@ class SpecVLAOracle:
 
     # ------------------------------------------------------------------ Algorithm 1, outer loop
     def generate_action(self, embeds, token_ids, shape, r: int, n_tokens: int = 7,
-                        tree_fn=None):
+                        tree_fn=None, prune: bool = False):
         """Prefill, then draft -> verify -> accept until n_tokens are emitted; clip.
         tree_fn(ep, iteration) may supply the tree instead of the draft model (planted or
-        random drafts). Returns (tokens [n_tokens], accept lengths per iteration)."""
+        random drafts). Returns (tokens [n_tokens], accept lengths per iteration).
+
+        prune (not in Algorithm 1, which drafts to a fixed depth and clips the chunk at the end):
+        an iteration that still misses k tokens drafts only k - 1 levels deep, since the
+        verification adds one token of its own and everything beyond is clipped; with k = 1 it
+        drafts nothing and verifies the root alone."""
         ep = self.prefill(embeds, token_ids)
         accept_lens = []
         it = 0
         while len(ep.emitted) < n_tokens:
-            tree = tree_fn(ep, it) if tree_fn is not None else self.draft_tree(ep, shape)
+            if tree_fn is not None:
+                tree = tree_fn(ep, it)
+            elif prune:
+                k = min(shape.depth, n_tokens - len(ep.emitted) - 1)
+                if k == 0:
+                    tree = Tree([ep.root], [-1], [0], [0.0])
+                else:
+                    tree = self.draft_tree(ep, type(shape)(tuple(shape.branch[:k]), tuple(shape.expand[:k])))
+            else:
+                tree = self.draft_tree(ep, shape)
             m, _ = self.verify_tree(ep, tree, r)
             accept_lens.append(m)
             it += 1

@@ -35,7 +35,8 @@ class DraftWeights(C.Structure):
 
 
 class TreeShape(C.Structure):
-    _fields_ = [("depth", C.c_int), ("branch", C.c_int * MAX_DEPTH), ("expand", C.c_int * MAX_DEPTH)]
+    _fields_ = [("depth", C.c_int), ("branch", C.c_int * MAX_DEPTH), ("expand", C.c_int * MAX_DEPTH),
+                ("prune", C.c_int)]
 
 
 class Tree(C.Structure):
@@ -110,9 +111,10 @@ def _stream():
     return C.c_void_p(torch.cuda.current_stream().cuda_stream)
 
 
-def make_shape(branch, expand) -> TreeShape:
+def make_shape(branch, expand, prune: bool = False) -> TreeShape:
     s = TreeShape()
     s.depth = len(branch)
+    s.prune = 1 if prune else 0
     for i, (b, e) in enumerate(zip(branch, expand)):
         s.branch[i], s.expand[i] = int(b), int(e)
     return s

@@ -65,6 +65,10 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   const uint32_t tmem_slot = bars + 8u * (2 * STAGES + 1);
   __shared__ float s_scale[MAX_T];
   __shared__ int s_pos[MAX_T], s_slot[MAX_T], s_ep[MAX_T];
+  // RoPE factors of the CTA's rows (EPI_QKV, up to 32 rows of up to 64 pairs): fetched while the
+  // MMAs run, so that the finishing loop does not wait for them row after row
+  constexpr int ROPE_ROWS = TN <= 32 ? 32 : 1, ROPE_HALF = TN <= 32 ? 64 : 1;
+  __shared__ __align__(16) float2 s_rope[ROPE_ROWS * ROPE_HALF];
   __shared__ float s_red[8][MAX_T];
   __shared__ int s_flag[8];
 
@@ -127,6 +131,10 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   uint32_t tmem_base;
   asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
 
+  // finishing-loop operands that the epilogue warps fetch while the MMAs run (part 1)
+  const bool rope_staged = ea.mode == EPI_QKV && T <= ROPE_ROWS && (ea.dh >> 1) <= ROPE_HALF;
+  float4 xpre0 = make_float4(0.f, 0.f, 0.f, 0.f), xpre1 = xpre0;
+
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0 && n_units > 0) {
@@ -188,6 +196,23 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         s_pos[et] = ea.rt.pos[row0 + et];
         s_slot[et] = ea.rt.slot[row0 + et];
         s_ep[et] = ea.rt.ep[row0 + et];
+      }
+    }
+    // operands of the finishing loop that do not depend on this GEMM, requested now
+    const bool p2_swiglu = ea.mode == EPI_SWIGLU;
+    const int p2_rg = p2_swiglu ? et >> 5 : et >> 6, p2_RG = p2_swiglu ? 8 : 4;
+    const int p2_n = p2_swiglu ? tile * 128 + (et & 31) * 4 : tile * BM + (et & 63) * 4;
+    const int p2_t0 = rank + p2_rg * S, p2_t1 = p2_t0 + p2_RG * S;
+    if (ea.mode == EPI_RESID && ea.accumulate && p2_n < ea.N) {
+      if (p2_t0 < T) xpre0 = *reinterpret_cast<const float4 *>(ea.x + (size_t)(row0 + p2_t0) * ea.N + p2_n);
+      if (p2_t1 < T) xpre1 = *reinterpret_cast<const float4 *>(ea.x + (size_t)(row0 + p2_t1) * ea.N + p2_n);
+    }
+    if (rope_staged) {
+      epi_barrier();                                       // s_pos is in place
+      const int half = ea.dh >> 1;
+      for (int i = et; i < T * half; i += 256) {
+        const int t = i / half, j = i - t * half;
+        s_rope[t * ROPE_HALF + j] = ea.rope_tab[(size_t)s_pos[t] * half + j];
       }
     }
     bool have = n_units > 0;
@@ -287,15 +312,18 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         }
       return acc;
     };
-    for (int t = rank + rg * S; t < T; t += RG * S) {
+    int iter = 0;
+    for (int t = rank + rg * S; t < T; t += RG * S, iter++) {
       const size_t row = (size_t)(row0 + t);
       const float sc = s_scale[t];
-      // global operands first
-      float4 xo = make_float4(0.f, 0.f, 0.f, 0.f), cs01 = xo, cs23 = xo;
-      if (ea.mode == EPI_RESID && ea.accumulate && col_ok)
+      // global operands first (the first two rows' residuals and, up to 32 rows, the RoPE
+      // factors were fetched in part 1)
+      float4 xo = iter == 0 ? xpre0 : xpre1, cs01 = make_float4(0.f, 0.f, 0.f, 0.f), cs23 = cs01;
+      if (ea.mode == EPI_RESID && ea.accumulate && col_ok && iter >= 2)
         xo = *reinterpret_cast<const float4 *>(ea.x + row * ea.N + n);
       if (rot) {
-        const float2 *cs = ea.rope_tab + (size_t)s_pos[t] * half + (lo ? jq : jq - half);
+        const float2 *cs = rope_staged ? s_rope + t * ROPE_HALF + (lo ? jq : jq - half)
+                                       : ea.rope_tab + (size_t)s_pos[t] * half + (lo ? jq : jq - half);
         cs01 = *reinterpret_cast<const float4 *>(cs);
         cs23 = *reinterpret_cast<const float4 *>(cs + 2);
       }

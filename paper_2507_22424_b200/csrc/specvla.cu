@@ -1019,8 +1019,16 @@ int specvla_generate_action(specvla_ctx *ctx, int n_ep, const int *episodes, con
     ea.n_ep = n_ep;
     int R = 0;
     CU(cudaEventRecord(ctx->ev[0], st));
-    if (shape->depth > 0) {
-      TRY(specvla_draft_tree(ctx, n_ep, episodes, shape, nullptr, stream));
+    // levels to draft: all of them, or (prune) no more than the tokens still missing minus the
+    // one the verification adds itself
+    specvla_tree_shape now = *shape;
+    if (shape->prune) {
+      int missing = 0;
+      for (int i = 0; i < n_ep; i++) missing = std::max(missing, n_tokens - count[i]);
+      now.depth = std::min(shape->depth, missing - 1);
+    }
+    if (now.depth > 0) {
+      TRY(specvla_draft_tree(ctx, n_ep, episodes, &now, nullptr, stream));
     } else {
       // no drafting: a one-row tree (the root) per episode = one autoregressive step
       DevTree *h = ctx->pin_trees;

@@ -92,6 +92,9 @@ def test_c1_generate_action_strict_equals_greedy(env):
     ar, _, _ = gpu.generate_action([0], env["emb"], env["ids"].tolist(), [len(env["ids"])],
                                    make_shape((), ()), 0, 7)
     assert toks == ar
+    pruned, _, st3 = gpu.generate_action([0], env["emb"], env["ids"].tolist(), [len(env["ids"])],
+                                         make_shape(C.TREE_26.branch, C.TREE_26.expand, prune=True), 0, 7)
+    assert pruned == toks and st3.ms_draft < stats.ms_draft
     for i in range(7):
         if mg[i] <= G.MARGIN:
             print(f"position {i}: margin {mg[i]:.4f}; comparison stops here")

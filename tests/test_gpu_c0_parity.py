@@ -181,6 +181,10 @@ def test_generate_action_strict_equals_greedy_decoding(c0, wcuda):
                                      make_shape((), ()), 0, 7)
     assert st2.iterations == 6
     assert toks[0] == ar[0]          # lossless inside the CUDA path itself, whatever the margins
+    # depth pruning (an iteration drafts no deeper than the tokens still missing): same chunk
+    pr, _, st3 = gpu.generate_action([0], c0["embeds"].cuda(), c0["ids"].tolist(), [64],
+                                     make_shape(shape.branch, shape.expand, prune=True), 0, 7)
+    assert pr[0] == toks[0] and st3.iterations >= stats.iterations
     for i in range(7):
         if mg[i] <= G.MARGIN:
             print(f"position {i}: margin {mg[i]:.4f}, comparison stops")

@@ -150,6 +150,27 @@ def test_strict_acceptance_is_lossless_with_draft_model(c0, ar_tokens):
     assert len(lens) >= 1 and all(0 <= m <= 3 for m in lens)
 
 
+def test_depth_pruning_is_lossless_and_never_drafts_past_the_chunk(c0, ar_tokens, monkeypatch):
+    """prune: an iteration drafts at most (missing tokens - 1) levels, nothing when one token is
+    missing, and at r = 0 the chunk is still the greedy one."""
+    orc = c0["make"]()
+    depths, missing = [], []
+    real = orc.draft_tree
+
+    def spy(ep, shape, want_debug=False):
+        depths.append(shape.depth)
+        missing.append(7 - len(ep.emitted))
+        return real(ep, shape, want_debug)
+
+    monkeypatch.setattr(orc, "draft_tree", spy)
+    toks, lens = orc.generate_action(c0["embeds"], c0["ids"], c0["wl"].tree, r=0, prune=True)
+    assert toks == ar_tokens
+    assert depths and all(d == min(c0["wl"].tree.depth, k - 1) and d >= 1 for d, k in zip(depths, missing))
+    assert all(m <= d for m, d in zip(lens, depths + [0]))
+    # the last iteration of a chunk that ends one token short verifies the root alone
+    assert sum(m + 1 for m in lens) + 1 >= 7 and len(lens) >= len(depths)
+
+
 @pytest.mark.parametrize("action_only", [True, False])
 def test_strict_acceptance_is_lossless_with_arbitrary_trees(c0, action_only):
     orc = c0["make"](action_only=action_only)
