@@ -26,7 +26,7 @@ Only tests, the smoke check and the benchmark's CPU-baseline leg may import this
 """
 from __future__ import annotations
 
-from dataclasses import dataclass, field
+from dataclasses import dataclass, field, replace
 
 import torch
 
@@ -73,6 +73,24 @@ def accept_and_select(tokens, parent, depth, g, r, action_base, n_bins):
 
 
 # ----------------------------------------------------------------------------- state
+def rerank_and_keep(tree, keep: int):
+    """Dynamic draft tree (Section 4.1: the Eagle-2 strategy; Section 5.1: at most 50 nodes):
+    after the last level every drafted node is ranked by its cumulative log-probability (ties to
+    the lower node index) and only the `keep` best are verified. A node never outranks its
+    parent (log-probabilities are <= 0 and a parent has the lower index), so the kept set is
+    closed under ancestors; kept nodes keep their relative (creation) order."""
+    n = len(tree.tokens)
+    if n - 1 <= keep:
+        return tree
+    best = sorted(range(1, n), key=lambda i: (-tree.score[i], i))[:keep]
+    kept = [0] + sorted(best)
+    new_index = {old: new for new, old in enumerate(kept)}
+    return Tree([tree.tokens[i] for i in kept],
+                [-1 if tree.parent[i] < 0 else new_index[tree.parent[i]] for i in kept],
+                [tree.depth[i] for i in kept],
+                [tree.score[i] for i in kept])
+
+
 @dataclass
 class Episode:
     """Decoding state of one episode."""
@@ -226,6 +244,8 @@ class SpecVLAOracle:
                     score.append(score[n] + float(lp_all[v]))
             level = nxt
         tree = Tree(tokens, parent, depth, score)
+        if getattr(shape, "keep", 0) > 0:
+            tree = rerank_and_keep(tree, shape.keep)
         if want_debug:
             return tree, debug
         return tree
@@ -289,7 +309,8 @@ class SpecVLAOracle:
                 if k == 0:
                     tree = Tree([ep.root], [-1], [0], [0.0])
                 else:
-                    tree = self.draft_tree(ep, type(shape)(tuple(shape.branch[:k]), tuple(shape.expand[:k])))
+                    tree = self.draft_tree(ep, replace(shape, branch=tuple(shape.branch[:k]),
+                                                       expand=tuple(shape.expand[:k])))
             else:
                 tree = self.draft_tree(ep, shape)
             m, _ = self.verify_tree(ep, tree, r)

@@ -35,6 +35,7 @@ class TreeShape:
     """
     branch: tuple
     expand: tuple
+    keep: int = 0             # > 0: after the last level only the `keep` best nodes are verified
 
     @property
     def depth(self):

@@ -150,6 +150,73 @@ def test_strict_acceptance_is_lossless_with_draft_model(c0, ar_tokens):
     assert len(lens) >= 1 and all(0 <= m <= 3 for m in lens)
 
 
+def _random_scored_tree(seed, n, max_depth=5):
+    import random
+    rnd = random.Random(seed)
+    parent, depth, score = [-1], [0], [0.0]
+    for i in range(1, n):
+        p = rnd.choice([j for j in range(i) if depth[j] < max_depth])
+        parent.append(p)
+        depth.append(depth[p] + 1)
+        # cumulative log-probability: the parent's plus something <= 0 (sometimes exactly 0: a tie)
+        score.append(score[p] - (0.0 if rnd.random() < 0.1 else rnd.expovariate(1.0)))
+    return parent, depth, score
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_rerank_keeps_the_best_nodes_and_their_ancestors(seed):
+    """Dynamic tree (Section 4.1 / 5.1): the kept nodes are the `keep` best by cumulative
+    log-probability, the set is closed under ancestors, order and structure are preserved."""
+    from oracle.specvla import Tree, rerank_and_keep
+    n = 6 + 5 * seed
+    parent, depth, score = _random_scored_tree(seed, n)
+    tokens = [1000 + i for i in range(n)]                  # the token identifies the old node
+    for keep in (1, 3, n // 2, n - 2, n - 1, n + 5):
+        t = rerank_and_keep(Tree(tokens, parent, depth, score), keep)
+        kept = [tok - 1000 for tok in t.tokens]
+        assert kept[0] == 0 and kept == sorted(kept) and len(kept) == 1 + min(keep, n - 1)
+        dropped = [i for i in range(1, n) if i not in kept]
+        if dropped:
+            assert min(score[i] for i in kept[1:]) >= max(score[i] for i in dropped)
+            # among equal scores the lower index wins
+            edge = min(score[i] for i in kept[1:])
+            assert all(i > max(k for k in kept if score[k] == edge) for i in dropped if score[i] == edge)
+        for new, old in enumerate(kept):
+            if old:
+                assert parent[old] in kept and t.parent[new] == kept.index(parent[old]) < new
+            assert t.depth[new] == depth[old] and t.score[new] == score[old]
+
+
+def test_dynamic_tree_of_the_draft_model_is_lossless_and_consistent(c0, ar_tokens):
+    """Top-4 expansion to depth 3, best 10 nodes kept: a valid tree whose scores are sums of the
+    draft model's log-probabilities along each path, and r = 0 still gives the greedy chunk."""
+    from synth_inputs.configs import TreeShape
+    shape = TreeShape((4, 4, 4), (1, 4, 4), keep=10)
+    full = TreeShape((4, 4, 4), (1, 4, 4))
+    orc = c0["make"]()
+    ep = orc.prefill(c0["embeds"], c0["ids"])
+    import copy
+    t_full = orc.draft_tree(copy.deepcopy(ep), full)
+    t = orc.draft_tree(ep, shape)
+    assert len(t_full.tokens) == 1 + 4 + 16 + 16 and len(t.tokens) == 11
+    for i in range(1, 11):
+        assert 0 <= t.parent[i] < i and t.depth[i] == t.depth[t.parent[i]] + 1
+        assert t.score[i] <= t.score[t.parent[i]]
+    # every kept node is a node of the full tree with the same path of tokens
+    def path(tr, i):
+        out = []
+        while i > 0:
+            out.append(tr.tokens[i])
+            i = tr.parent[i]
+        return tuple(reversed(out))
+    full_paths = {path(t_full, i): t_full.score[i] for i in range(1, len(t_full.tokens))}
+    for i in range(1, 11):
+        assert abs(full_paths[path(t, i)] - t.score[i]) < 1e-12
+    assert sorted(full_paths.values(), reverse=True)[9] == min(t.score[1:])
+    toks, lens = c0["make"]().generate_action(c0["embeds"], c0["ids"], shape, r=0)
+    assert toks == ar_tokens
+
+
 def test_depth_pruning_is_lossless_and_never_drafts_past_the_chunk(c0, ar_tokens, monkeypatch):
     """prune: an iteration drafts at most (missing tokens - 1) levels, nothing when one token is
     missing, and at r = 0 the chunk is still the greedy one."""
