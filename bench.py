@@ -308,6 +308,17 @@ def run_ours(args, rank, local_rank, world):
     e7.record()
     barrier()
     ms_pr = e6.elapsed_time(e7)
+    # --- the paper's dynamic tree: top-8, depth 5, best 50 of the 264 drafted nodes verified ----
+    dy_shape = make_shape((8,) * 5, (1, 8, 8, 8, 8), keep=50)
+    gpu.generate_action([0], embeds, ids_host, [P], dy_shape, r, n_tok)
+    barrier()
+    e8, e9 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e8.record()
+    for _ in range(ar_steps):
+        dy_toks, _, dy_stats = gpu.generate_action([0], embeds, ids_host, [P], dy_shape, r, n_tok)
+    e9.record()
+    barrier()
+    ms_dy = e8.elapsed_time(e9)
     # --- per-GEMM device time of the verification phase (separate pass, same steps) -----
     gpu.profile(4)
     for _ in range(max(2, args.steps // 4)):
@@ -378,6 +389,8 @@ def run_ours(args, rank, local_rank, world):
         depth_pruned=dict(value=world * ar_steps / (ms_pr / 1000.0), unit=UNIT, same_tokens=bool(pr_toks == toks),
                           note="same call with tree_shape.prune = 1 (not Algorithm 1 as printed: iterations "
                                "draft min(depth, missing tokens - 1) levels); `value` above is unpruned"),
+        dynamic_tree=dict(value=world * ar_steps / (ms_dy / 1000.0), unit=UNIT, same_tokens=bool(dy_toks == toks),
+                          note="top-8, depth 5, best 50 of 264 drafted nodes verified (51 rows per step)"),
         cpu_baseline=dict(value=cpu_val, unit=UNIT, cores=torch.get_num_threads(), kind="oracle",
                           sample=("oracle (float64) decoder layer over 290 and 27 rows, LM head over 27 "
                                   "rows, one draft level over 4 rows at 7B shapes; chunk = 33*t_layer290 + "

@@ -87,7 +87,7 @@ typedef struct {
 } specvla_draft_weights;
 
 /* Static-size draft tree (Section 4.1, Eagle-2 style): level l (0-based) expands the
- * expand[l] best nodes of level l-1 (expand[0] must be 1: the root) into branch[l] children
+ * expand[l] best nodes of level l-1 (expand[0] must be 1: the root) into branch[l] <= 8 children
  * each. depth = 0 means no drafting: every iteration is one plain autoregressive step. */
 typedef struct {
   int depth;
@@ -99,6 +99,11 @@ typedef struct {
                 * verification adds one token itself, deeper nodes could only be clipped), and
                 * none at all when k = 1. Same tokens at r = 0; at r > 0 the accepted path may be
                 * another equally valid one. */
+  int keep;    /* 0: every drafted node is verified (at most 16 nodes per level, 127 in all).
+                * N > 0: dynamic tree (Section 4.1: the Eagle-2 strategy; Section 5.1: 50 nodes,
+                * top-8): levels may hold up to 64 nodes (16 of them expanded), 319 in all; after the
+                * last level the nodes are ranked by cumulative log-probability (ties to the lower
+                * node index) and only the N best (N <= 127) are kept and verified. */
 } specvla_tree_shape;
 
 /* One draft tree in HOST memory. Row 0 is the root (the last emitted token, not yet in the

@@ -36,7 +36,7 @@ class DraftWeights(C.Structure):
 
 class TreeShape(C.Structure):
     _fields_ = [("depth", C.c_int), ("branch", C.c_int * MAX_DEPTH), ("expand", C.c_int * MAX_DEPTH),
-                ("prune", C.c_int)]
+                ("prune", C.c_int), ("keep", C.c_int)]
 
 
 class Tree(C.Structure):
@@ -111,10 +111,11 @@ def _stream():
     return C.c_void_p(torch.cuda.current_stream().cuda_stream)
 
 
-def make_shape(branch, expand, prune: bool = False) -> TreeShape:
+def make_shape(branch, expand, prune: bool = False, keep: int = 0) -> TreeShape:
     s = TreeShape()
     s.depth = len(branch)
     s.prune = 1 if prune else 0
+    s.keep = int(keep)
     for i, (b, e) in enumerate(zip(branch, expand)):
         s.branch[i], s.expand[i] = int(b), int(e)
     return s

@@ -7,7 +7,8 @@
 
 typedef __nv_bfloat16 bf16;
 
-#define SV_MAX_TREE 128          // rows of one tree, root included
+#define SV_MAX_TREE 128          // rows of one tree as it is verified, root included
+#define SV_MAX_CAND 320          // nodes a dynamic tree may draft before re-ranking, root included
 #define SV_MAX_DEPTH 8
 #define SV_MAX_BRANCH 8
 #define SV_MAX_PENDING (SV_MAX_DEPTH + 1)
@@ -52,10 +53,9 @@ struct DevTree {
   int level_begin, level_end;     // nodes of the level built last
   int sel_count;                  // nodes selected for expansion at the next level
   int sel[16];                    // ... in rank order
-  int tok[SV_MAX_TREE], parent[SV_MAX_TREE], depth[SV_MAX_TREE];
-  float score[SV_MAX_TREE];
-  int drow[SV_MAX_TREE];          // draft row that scored the node's children (-1: none)
-  uint32_t vmask[SV_MAX_TREE][4]; // ancestors-and-self over tree rows (verification mask)
+  int tok[SV_MAX_CAND], parent[SV_MAX_CAND], depth[SV_MAX_CAND];
+  float score[SV_MAX_CAND];
+  int drow[SV_MAX_CAND];          // draft row that scored the node's children (-1: none)
   uint32_t dmask[SV_MAX_TREE][4]; // ancestors-and-self over draft rows (draft mask), by draft row
 };
 

@@ -474,19 +474,23 @@ int validate_tree(const specvla_tree &t) {
   return SPECVLA_OK;
 }
 
-int validate_shape(const specvla_tree_shape *s, int *n_nodes) {
-  if (!s || s->depth < 0 || s->depth > SV_MAX_DEPTH) return SPECVLA_ERR_INVALID_ARG;
+// n_nodes: nodes drafted; n_rows_out (may be NULL): rows verified (root + nodes kept).
+int validate_shape(const specvla_tree_shape *s, int *n_nodes, int *n_rows_out = nullptr) {
+  if (!s || s->depth < 0 || s->depth > SV_MAX_DEPTH || s->keep < 0) return SPECVLA_ERR_INVALID_ARG;
+  const int level_max = s->keep > 0 ? 64 : 16;            // nodes of one level
   int prev = 1, total = 0;
   for (int l = 0; l < s->depth; l++) {
     if (s->branch[l] < 1 || s->branch[l] > SV_MAX_BRANCH) return SPECVLA_ERR_INVALID_ARG;
     if (s->expand[l] < 1 || s->expand[l] > 16 || s->expand[l] > prev) return SPECVLA_ERR_INVALID_ARG;
     if (l == 0 && s->expand[0] != 1) return SPECVLA_ERR_INVALID_ARG;
     prev = s->branch[l] * s->expand[l];
-    if (prev > 16) return SPECVLA_ERR_INVALID_ARG;   // one level: at most 16 nodes
+    if (prev > level_max) return SPECVLA_ERR_INVALID_ARG;
     total += prev;
   }
-  if (1 + total > SV_MAX_TREE) return SPECVLA_ERR_INVALID_ARG;
+  const int kept = (s->keep > 0 && s->keep < total) ? s->keep : total;
+  if (1 + total > SV_MAX_CAND || 1 + kept > SV_MAX_TREE) return SPECVLA_ERR_INVALID_ARG;
   *n_nodes = total;
+  if (n_rows_out) *n_rows_out = 1 + kept;
   return SPECVLA_OK;
 }
 
@@ -777,8 +781,9 @@ int specvla_draft_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const sp
                        specvla_tree *trees_out, void *stream) {
   TRY(check_episodes(ctx, n_ep, episodes));
   if (!ctx->has_draft) return SPECVLA_ERR_BAD_STATE;
-  int n_nodes = 0;
-  TRY(validate_shape(shape, &n_nodes));
+  int n_nodes = 0, n_tree_rows = 0, n_draft_rows = 0;
+  TRY(validate_shape(shape, &n_nodes, &n_tree_rows));
+  for (int l = 1; l < shape->depth; l++) n_draft_rows += shape->expand[l];
   const specvla_model_desc &d = ctx->desc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   EpArgs ea{};
@@ -787,7 +792,8 @@ int specvla_draft_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const sp
   for (int i = 0; i < n_ep; i++) {
     const int e = episodes[i];
     if (ctx->hP[e] < 0 || ctx->hPending[e] < 1) return SPECVLA_ERR_BAD_STATE;
-    if (ctx->hP[e] + 1 + n_nodes > d.max_seq) return SPECVLA_ERR_CAPACITY;
+    // target cache: the rows verified; draft cache: one row per node expanded below the root
+    if (ctx->hP[e] + n_tree_rows > d.max_seq || ctx->hP[e] + n_draft_rows > d.max_seq) return SPECVLA_ERR_CAPACITY;
     ea.eps[i] = e;
     ea.row0[i] = R;
     ea.nrows[i] = ctx->hPending[e];
@@ -813,7 +819,7 @@ int specvla_draft_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const sp
   ctx->feat_valid = false;
   for (int i = 0; i < n_ep; i++) {
     ctx->hPending[episodes[i]] = 0;
-    ctx->hTreeRows[episodes[i]] = 1 + n_nodes;
+    ctx->hTreeRows[episodes[i]] = n_tree_rows;
   }
 
   int scored_rows = n_ep;            // rows scored by the LM head in the current round
@@ -865,6 +871,9 @@ int specvla_draft_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const sp
     scored_rows = Rn;
     gathered = false;
   }
+
+  if (n_tree_rows < 1 + n_nodes)
+    LAUNCH(tree::rerank_keep_kernel, dim3(n_ep), dim3(SV_MAX_CAND), ea, ctx->trees, n_tree_rows - 1);
 
   if (trees_out) {
     DevTree *h = ctx->pin_trees;

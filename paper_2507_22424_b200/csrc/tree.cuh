@@ -8,8 +8,8 @@ namespace tree {
 
 // ---------------------------------------------------------------------------------------
 // Verification rows of each episode's tree: row i sits at position P + depth[i], slot P + i,
-// sees the P committed slots, its ancestors and itself. Also (re)computes vmask so that
-// caller-supplied trees need only tok / parent / depth. One CTA per episode.
+// sees the P committed slots, its ancestors and itself (the mask is computed here from the
+// parents, so trees need only tok / parent / depth). One CTA per episode.
 __global__ void build_verify_rows_kernel(EpArgs a, DevTree *trees, const EpState *__restrict__ st,
                                          RowTable rt) {
   pdl_launch();
@@ -29,7 +29,7 @@ __global__ void build_verify_rows_kernel(EpArgs a, DevTree *trees, const EpState
     rt.nvis[r] = P;
     rt.tbase[r] = P;
 #pragma unroll
-    for (int w = 0; w < 4; w++) { rt.mask[r * 4 + w] = m[w]; tr.vmask[i][w] = m[w]; }
+    for (int w = 0; w < 4; w++) rt.mask[r * 4 + w] = m[w];
   }
   if (threadIdx.x == 0 && tr.tok[0] < 0) tr.tok[0] = st[e].root;
 }
@@ -67,7 +67,7 @@ __global__ void build_catchup_rows_kernel(EpArgs a, EpState *st, DevTree *trees,
   tr.depth[0] = 0;
   tr.score[0] = 0.f;
   tr.drow[0] = 0;
-  for (int w = 0; w < 4; w++) { tr.vmask[0][w] = (w == 0); tr.dmask[0][w] = 0; }
+  for (int w = 0; w < 4; w++) tr.dmask[0][w] = 0;
   tr.level_begin = 0;
   tr.level_end = 1;
   tr.sel_count = 1;
@@ -141,7 +141,7 @@ __global__ void catchup_dst_kernel(EpArgs a, int *__restrict__ dst_row, int *__r
 // (score = parent score + log-prob). Then the `expand_next` best new nodes (by score, ties
 // to the lower node index) are selected, in rank order, and their draft rows are laid out
 // for the next level: input feature = output of the row that scored them, token = their own.
-// One thread per episode (at most 128 nodes, 16 per level).
+// One thread per episode (at most 64 nodes per level, 16 of them expanded).
 // a.row0 = first scored row of each episode, a.aux = first row of its next level.
 __global__ void expand_level_kernel(EpArgs a, int level, int branch, int expand_next,
                                     const int *__restrict__ top_tok, const float *__restrict__ top_lp,
@@ -164,22 +164,20 @@ __global__ void expand_level_kernel(EpArgs a, int level, int branch, int expand_
       tr.depth[n] = level + 1;
       tr.score[n] = tr.score[p] + top_lp[srow * SV_TOPK + b];
       tr.drow[n] = -1;
-      for (int w = 0; w < 4; w++) tr.vmask[n][w] = tr.vmask[p][w];
-      tr.vmask[n][n >> 5] |= 1u << (n & 31);
     }
   }
   tr.level_begin = begin;
   tr.level_end = tr.n_rows;
-  // selection of the next level's parents: repeated arg-best (<= 16 x 16 comparisons)
+  // selection of the next level's parents: repeated arg-best (<= 16 x 64 comparisons)
   int cnt = 0;
-  uint32_t used = 0;
+  unsigned long long used = 0;
   for (; cnt < expand_next && cnt < tr.level_end - begin; cnt++) {
     int best = -1;
     for (int n = begin; n < tr.level_end; n++) {
-      if (used & (1u << (n - begin))) continue;
+      if (used & (1ull << (n - begin))) continue;
       if (best < 0 || tr.score[n] > tr.score[best]) best = n;
     }
-    used |= 1u << (best - begin);
+    used |= 1ull << (best - begin);
     tr.sel[cnt] = best;
   }
   tr.sel_count = cnt;
@@ -203,6 +201,52 @@ __global__ void expand_level_kernel(EpArgs a, int level, int branch, int expand_
     feat_src[r] = e * SV_MAX_TREE + pdr;   // row of dout
     dst_row[r] = e * SV_MAX_TREE + dr;
   }
+}
+
+// ---------------------------------------------------------------------------------------
+// Dynamic draft tree (Section 4.1: the Eagle-2 strategy; Section 5.1: at most 50 nodes): once
+// the last level is drafted, every node is ranked by its cumulative log-probability (ties to
+// the lower node index) and only the `keep` best stay, in their creation order. A node never
+// outranks its parent (log-probabilities are <= 0 and the parent has the lower index), so the
+// set is closed under ancestors. One CTA per episode; ranks by counting (n <= 320).
+__global__ void __launch_bounds__(SV_MAX_CAND)
+rerank_keep_kernel(EpArgs a, DevTree *trees, int keep) {
+  __shared__ float s_score[SV_MAX_CAND];
+  __shared__ int s_tok[SV_MAX_CAND], s_parent[SV_MAX_CAND], s_depth[SV_MAX_CAND], s_new[SV_MAX_CAND];
+  pdl_launch();
+  pdl_wait();
+  DevTree &tr = trees[a.eps[blockIdx.x]];
+  const int n = tr.n_rows, i = threadIdx.x;
+  if (n - 1 <= keep) return;
+  if (i < n) {
+    s_score[i] = tr.score[i];
+    s_tok[i] = tr.tok[i];
+    s_parent[i] = tr.parent[i];
+    s_depth[i] = tr.depth[i];
+  }
+  __syncthreads();
+  bool kept = false;
+  if (i < n) {
+    int rank = 0;
+    for (int j = 1; j < n; j++) rank += (s_score[j] > s_score[i]) || (s_score[j] == s_score[i] && j < i);
+    kept = (i == 0) || rank < keep;
+  }
+  // new index = kept nodes before this one (block-wide exclusive count through ballots)
+  __shared__ int s_warp[SV_MAX_CAND / 32];
+  const unsigned b = __ballot_sync(0xffffffffu, kept);
+  if ((i & 31) == 0) s_warp[i >> 5] = __popc(b);
+  __syncthreads();
+  int before = __popc(b & ((1u << (i & 31)) - 1u));
+  for (int w = 0; w < (i >> 5); w++) before += s_warp[w];
+  s_new[i] = kept ? before : -1;
+  __syncthreads();
+  if (kept) {
+    tr.tok[before] = s_tok[i];
+    tr.parent[before] = i == 0 ? -1 : s_new[s_parent[i]];
+    tr.depth[before] = s_depth[i];
+    tr.score[before] = s_score[i];
+  }
+  if (i == 0) tr.n_rows = 1 + keep;
 }
 
 // ---------------------------------------------------------------------------------------

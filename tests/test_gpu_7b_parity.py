@@ -95,6 +95,10 @@ def test_c1_generate_action_strict_equals_greedy(env):
     pruned, _, st3 = gpu.generate_action([0], env["emb"], env["ids"].tolist(), [len(env["ids"])],
                                          make_shape(C.TREE_26.branch, C.TREE_26.expand, prune=True), 0, 7)
     assert pruned == toks and st3.ms_draft < stats.ms_draft
+    # the paper's own tree (Section 5.1 / Table 4): top-8, depth 5, the best 50 of 264 drafted nodes
+    dyn, _, st4 = gpu.generate_action([0], env["emb"], env["ids"].tolist(), [len(env["ids"])],
+                                      make_shape((8,) * 5, (1, 8, 8, 8, 8), keep=50), 0, 7)
+    assert dyn == toks
     for i in range(7):
         if mg[i] <= G.MARGIN:
             print(f"position {i}: margin {mg[i]:.4f}; comparison stops here")

@@ -135,6 +135,57 @@ def test_draft_tree_matches_oracle(c0, wcuda):
     gpu.close()
 
 
+@pytest.mark.parametrize("branch,expand,keep", [((4, 4, 4), (1, 4, 4), 10), ((8, 8, 8), (1, 8, 8), 50),
+                                                ((8, 8), (1, 8), 100)])
+def test_dynamic_draft_tree_matches_oracle(c0, wcuda, branch, expand, keep):
+    """Dynamic tree: wide levels (up to 64 nodes), the best `keep` nodes by cumulative
+    log-probability stay. Structure always valid; tokens, parents and scores equal the oracle's
+    unless two candidates' scores are closer than the comparison margin."""
+    from paper_2507_22424_b200.binding import make_shape
+    from synth_inputs.configs import TreeShape
+    import copy
+    shape = TreeShape(branch, expand, keep=keep)
+    orc = c0["make"]()
+    ep = orc.prefill(c0["embeds"], c0["ids"])
+    full = orc.draft_tree(copy.deepcopy(ep), TreeShape(branch, expand))
+    ref = orc.draft_tree(ep, shape)
+    gpu = _gpu(c0, wcuda)
+    gpu.prefill([0], c0["embeds"].cuda(), c0["ids"].tolist(), [64])
+    got = gpu.draft_tree([0], make_shape(branch, expand, keep=keep))[0]
+    n = 1 + min(keep, shape.n_nodes)
+    assert len(got["tokens"]) == n == len(ref.tokens)
+    assert got["parent"][0] == -1 and got["tokens"][0] == ep.root
+    for i in range(1, n):
+        assert 0 <= got["parent"][i] < i and got["depth"][i] == got["depth"][got["parent"][i]] + 1
+        assert got["score"][i] <= got["score"][got["parent"][i]] + 1e-6
+    if got["tokens"] == ref.tokens and got["parent"] == ref.parent:
+        assert max(abs(a - b) for a, b in zip(got["score"], ref.score)) < 5e-2
+    else:
+        ranked = sorted(full.score[1:], reverse=True)
+        gap = min(a - b for a, b in zip(ranked, ranked[1:]))
+        assert gap < G.MARGIN, (got["tokens"], ref.tokens)
+        print("dynamic tree differs where two candidates are", gap, "apart")
+    # the tree is verified as it stands (device-resident), strict acceptance
+    m_ref, emitted_ref, dbg = orc.verify_tree(ep, ref, 0, want_debug=True)
+    if got["tokens"] == ref.tokens and got["parent"] == ref.parent:
+        m, emitted = gpu.verify_tree([0], [dict(tokens=got["tokens"], parent=got["parent"], depth=got["depth"])], 0)
+        g_gpu = gpu.read_buffer(1, n, torch.int32).tolist()
+        if g_gpu == dbg["g"]:
+            assert (m[0], emitted[0]) == (m_ref, emitted_ref)
+    gpu.close()
+
+
+def test_generate_action_with_dynamic_tree_is_lossless(c0, wcuda):
+    from paper_2507_22424_b200.binding import make_shape
+    gpu = _gpu(c0, wcuda)
+    args = ([0], c0["embeds"].cuda(), c0["ids"].tolist(), [64])
+    ar, _, _ = gpu.generate_action(*args, make_shape((), ()), 0, 7)
+    dyn, _, st = gpu.generate_action(*args, make_shape((8, 8, 8), (1, 8, 8), keep=50), 0, 7)
+    both, _, _ = gpu.generate_action(*args, make_shape((8, 8, 8), (1, 8, 8), keep=50, prune=True), 0, 7)
+    assert dyn[0] == ar[0] and both[0] == ar[0] and st.iterations <= 6
+    gpu.close()
+
+
 @pytest.mark.parametrize("r", [0, 4])
 @pytest.mark.parametrize("action_only", [True, False])
 def test_generate_action_lockstep_with_oracle(c0, wcuda, r, action_only):
