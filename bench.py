@@ -4,7 +4,7 @@
 One step = one action chunk of the C1 workload (OpenVLA-7B-shaped decoder, batch 1,
 290-position prefix, 26-node draft tree from the one-layer draft model, 7 action tokens,
 strict acceptance r = 0) through specvla_generate_action: prefill, then draft -> verify ->
-accept -> compact until 7 tokens. Prints ONE JSON line (see the design doc for every field).
+accept -> compact until 7 tokens. Prints ONE JSON line.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
