@@ -476,7 +476,8 @@ int validate_tree(const specvla_tree &t) {
 
 // n_nodes: nodes drafted; n_rows_out (may be NULL): rows verified (root + nodes kept).
 int validate_shape(const specvla_tree_shape *s, int *n_nodes, int *n_rows_out = nullptr) {
-  if (!s || s->depth < 0 || s->depth > SV_MAX_DEPTH || s->keep < 0) return SPECVLA_ERR_INVALID_ARG;
+  if (!s || s->depth < 0 || s->depth > SV_MAX_DEPTH || s->keep < 0 || s->keep > SV_MAX_TREE - 1)
+    return SPECVLA_ERR_INVALID_ARG;
   const int level_max = s->keep > 0 ? 64 : 16;            // nodes of one level
   int prev = 1, total = 0;
   for (int l = 0; l < s->depth; l++) {

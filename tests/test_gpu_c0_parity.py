@@ -299,5 +299,15 @@ def test_bad_arguments_are_rejected_before_any_launch(c0, wcuda):
     assert e.value.code == -2
     with pytest.raises(SpecVLAError):
         gpu.verify_tree([3], [bad[0]], 0)
+    # tree shapes: a level wider than 16 nodes needs the dynamic tree (keep > 0); at most 127 kept
+    # nodes and 319 drafted ones; level 0 expands the root alone; capacity of the caches
+    from paper_2507_22424_b200.binding import make_shape
+    for sh, code in [(make_shape((8, 8), (1, 8)), -1), (make_shape((8, 8), (1, 8), keep=128), -1),
+                     (make_shape((8,) * 7, (1,) + (8,) * 6, keep=50), -1), (make_shape((4, 4), (2, 4)), -1),
+                     (make_shape((4, 4), (1, 5)), -1), (make_shape((9,), (1,)), -1),
+                     (make_shape((8, 8), (1, 8), keep=40), -2)]:          # 64 + 41 rows > max_seq
+        with pytest.raises(SpecVLAError) as e:
+            gpu.draft_tree([0], sh, want_trees=False)
+        assert e.value.code == code, (e.value.code, code)
     assert gpu.kernel_launches() == n0
     gpu.close()
