@@ -25,7 +25,7 @@ def _gpu(c0, wcuda, **kw):
 
 @pytest.mark.parametrize("T,N,K", [(1, 256, 256), (15, 1376, 256), (15, 256, 688), (27, 4096, 4096),
                                    (33, 1000, 1024), (64, 136, 72), (128, 512, 2048), (130, 384, 520),
-                                   (290, 768, 512)])
+                                   (290, 768, 512), (27, 8448, 1024), (9, 16384, 768)])
 def test_gemm_matches_float64_matmul(T, N, K):
     from paper_2507_22424_b200.binding import gemm
     x = rng.normal(11, 1, (T, K), 1.0, dtype=torch.float32)
