@@ -48,7 +48,7 @@ __device__ __forceinline__ void cluster_sync_all() {
 __host__ __device__ constexpr int ck_tmem_cols(int TN) { return 2 * acc_width(TN) < 32 ? 32 : 2 * acc_width(TN); }
 
 // EpiArgs as in gemm_tc (EPI_PLAIN or EPI_RESID; part / counters unused). KB = K blocks per tile.
-template <int TN>
+template <int TN, int MODE>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                const __grid_constant__ CUtensorMap tmXtail, const EpiArgs ea, const int KB,
@@ -67,7 +67,8 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   __shared__ int s_pos[MAX_T], s_slot[MAX_T], s_ep[MAX_T];
   // RoPE factors of the CTA's rows (EPI_QKV, up to 32 rows of up to 64 pairs): fetched while the
   // MMAs run, so that the finishing loop does not wait for them row after row
-  constexpr int ROPE_ROWS = TN <= 32 ? 32 : 1, ROPE_HALF = TN <= 32 ? 64 : 1;
+  constexpr bool ROPE_SMEM = TN <= 32 && MODE == EPI_QKV;
+  constexpr int ROPE_ROWS = ROPE_SMEM ? 32 : 1, ROPE_HALF = ROPE_SMEM ? 64 : 1;
   __shared__ __align__(16) float2 s_rope[ROPE_ROWS * ROPE_HALF];
   __shared__ float s_red[8][MAX_T];
   __shared__ int s_flag[8];
@@ -75,7 +76,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int S = (int)cluster_size();
   const int rank = (int)cluster_rank();
-  const bool swiglu = ea.mode == EPI_SWIGLU;
+  constexpr bool swiglu = MODE == EPI_SWIGLU;
   const int tile = blockIdx.x / S;
   const int kb0 = rank * KB / S, kb1 = (rank + 1) * KB / S;
   const int n_units = kb1 - kb0;
@@ -132,7 +133,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   asm volatile("ld.shared.b32 %0, [%1];" : "=r"(tmem_base) : "r"(tmem_slot));
 
   // finishing-loop operands that the epilogue warps fetch while the MMAs run (part 1)
-  const bool rope_staged = ea.mode == EPI_QKV && T <= ROPE_ROWS && (ea.dh >> 1) <= ROPE_HALF;
+  const bool rope_staged = MODE == EPI_QKV && T <= ROPE_ROWS && (ea.dh >> 1) <= ROPE_HALF;
   float4 xpre0 = make_float4(0.f, 0.f, 0.f, 0.f), xpre1 = xpre0;
 
   if (warp == 0) {
@@ -192,18 +193,18 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         sc = rsqrtf(ss * ea.inv_k + ea.eps);
       }
       s_scale[et] = sc;
-      if (ea.mode == EPI_QKV) {
+      if (MODE == EPI_QKV) {
         s_pos[et] = ea.rt.pos[row0 + et];
         s_slot[et] = ea.rt.slot[row0 + et];
         s_ep[et] = ea.rt.ep[row0 + et];
       }
     }
     // operands of the finishing loop that do not depend on this GEMM, requested now
-    const bool p2_swiglu = ea.mode == EPI_SWIGLU;
+    constexpr bool p2_swiglu = MODE == EPI_SWIGLU;
     const int p2_rg = p2_swiglu ? et >> 5 : et >> 6, p2_RG = p2_swiglu ? 8 : 4;
     const int p2_n = p2_swiglu ? tile * 128 + (et & 31) * 4 : tile * BM + (et & 63) * 4;
     const int p2_t0 = rank + p2_rg * S, p2_t1 = p2_t0 + p2_RG * S;
-    if (ea.mode == EPI_RESID && ea.accumulate && p2_n < ea.N) {
+    if (MODE == EPI_RESID && ea.accumulate && p2_n < ea.N) {
       if (p2_t0 < T) xpre0 = *reinterpret_cast<const float4 *>(ea.x + (size_t)(row0 + p2_t0) * ea.N + p2_n);
       if (p2_t1 < T) xpre1 = *reinterpret_cast<const float4 *>(ea.x + (size_t)(row0 + p2_t1) * ea.N + p2_n);
     }
@@ -285,12 +286,12 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     const float *P_own = reinterpret_cast<const float *>(smem_raw + (base - smem_u32(smem_raw)));
     cooperative_groups::cluster_group cluster = cooperative_groups::this_cluster();
     float4 gain = make_float4(1.f, 1.f, 1.f, 1.f);
-    if (ea.mode == EPI_RESID && ea.gain && col_ok) gain = *reinterpret_cast<const float4 *>(ea.gain + n);
+    if (MODE == EPI_RESID && ea.gain && col_ok) gain = *reinterpret_cast<const float4 *>(ea.gain + n);
     // QKV: which of q / k / v and which half of a head the four columns lie in
-    const int which = ea.mode == EPI_QKV ? n / ea.hd : 2;
-    const int cq = ea.mode == EPI_QKV ? n - which * ea.hd : 0;
-    const int half = ea.dh >> 1, jq = ea.mode == EPI_QKV ? cq % ea.dh : 0;
-    const bool lo = jq < half, rot = ea.mode == EPI_QKV && which < 2;
+    const int which = MODE == EPI_QKV ? n / ea.hd : 2;
+    const int cq = MODE == EPI_QKV ? n - which * ea.hd : 0;
+    const int half = ea.dh >> 1, jq = MODE == EPI_QKV ? cq % ea.dh : 0;
+    const bool lo = jq < half, rot = MODE == EPI_QKV && which < 2;
     auto partial_sum = [&](int off) {
       float4 p[MAX_S];
 #pragma unroll
@@ -319,7 +320,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       // global operands first (the first two rows' residuals and, up to 32 rows, the RoPE
       // factors were fetched in part 1)
       float4 xo = iter == 0 ? xpre0 : xpre1, cs01 = make_float4(0.f, 0.f, 0.f, 0.f), cs23 = cs01;
-      if (ea.mode == EPI_RESID && ea.accumulate && col_ok && iter >= 2)
+      if (MODE == EPI_RESID && ea.accumulate && col_ok && iter >= 2)
         xo = *reinterpret_cast<const float4 *>(ea.x + row * ea.N + n);
       if (rot) {
         const float2 *cs = rope_staged ? s_rope + t * ROPE_HALF + (lo ? jq : jq - half)
@@ -327,12 +328,12 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         cs01 = *reinterpret_cast<const float4 *>(cs);
         cs23 = *reinterpret_cast<const float4 *>(cs + 2);
       }
-      const int slot = ea.mode == EPI_QKV ? s_slot[t] : 0, ep = ea.mode == EPI_QKV ? s_ep[t] : 0;
+      const int slot = MODE == EPI_QKV ? s_slot[t] : 0, ep = MODE == EPI_QKV ? s_ep[t] : 0;
       float4 v = partial_sum(t * BM + c4);
-      if (ea.mode == EPI_PLAIN) {
+      if (MODE == EPI_PLAIN) {
         if (col_ok)
           *reinterpret_cast<float4 *>(ea.out + row * ea.ldo + n) = make_float4(sc * v.x, sc * v.y, sc * v.z, sc * v.w);
-      } else if (ea.mode == EPI_QKV) {
+      } else if (MODE == EPI_QKV) {
         // the partner columns of the rotation (dh / 2 away) are in the same tile
         float4 o = make_float4(sc * v.x, sc * v.y, sc * v.z, sc * v.w);
         if (rot) {
@@ -375,7 +376,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         if (lane == 0) s_red[warp - 2][t] = s2;
       }
     }
-    if (ea.mode == EPI_RESID) {
+    if (MODE == EPI_RESID) {
       epi_barrier();
       // thread i finishes this CTA's i-th row, which row group i % 4 (two warps) handled
       const int t = rank + et * S;
@@ -399,12 +400,12 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   if (warp == 1) tc_dealloc(tmem_base, ck_tmem_cols(TN));
 }
 
-template <int TN>
-inline cudaError_t launch_tn(const CUtensorMap &tmW, const CUtensorMap &tmX, const CUtensorMap &tmXtail,
+template <int TN, int MODE>
+inline cudaError_t launch_tm(const CUtensorMap &tmW, const CUtensorMap &tmX, const CUtensorMap &tmXtail,
                              const EpiArgs &ea, int tiles, int KB, int S, int *err, cudaStream_t st, bool pdl) {
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_ck_kernel<TN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(gemm_ck_kernel<TN, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          smem_bytes(TN));
     if (e != cudaSuccess) return e;
     attr_set = true;
@@ -423,7 +424,20 @@ inline cudaError_t launch_tn(const CUtensorMap &tmW, const CUtensorMap &tmX, con
   at[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = pdl ? 2 : 1;
-  return cudaLaunchKernelEx(&cfg, gemm_ck_kernel<TN>, tmW, tmX, tmXtail, ea, KB, err);
+  return cudaLaunchKernelEx(&cfg, gemm_ck_kernel<TN, MODE>, tmW, tmX, tmXtail, ea, KB, err);
+}
+
+// The epilogue mode is a template parameter: each instantiation carries only its own finishing
+// code (the epilogue runs once per CTA from a cold instruction cache, so its size matters).
+template <int TN>
+inline cudaError_t launch_tn(const CUtensorMap &tmW, const CUtensorMap &tmX, const CUtensorMap &tmXtail,
+                             const EpiArgs &ea, int tiles, int KB, int S, int *err, cudaStream_t st, bool pdl) {
+  switch (ea.mode) {
+    case EPI_PLAIN: return launch_tm<TN, EPI_PLAIN>(tmW, tmX, tmXtail, ea, tiles, KB, S, err, st, pdl);
+    case EPI_RESID: return launch_tm<TN, EPI_RESID>(tmW, tmX, tmXtail, ea, tiles, KB, S, err, st, pdl);
+    case EPI_SWIGLU: return launch_tm<TN, EPI_SWIGLU>(tmW, tmX, tmXtail, ea, tiles, KB, S, err, st, pdl);
+    default: return launch_tm<TN, EPI_QKV>(tmW, tmX, tmXtail, ea, tiles, KB, S, err, st, pdl);
+  }
 }
 
 // How many clusters of each size 1..MAX_S can be resident at once (index = size; 0 = unknown).
@@ -434,7 +448,7 @@ struct ClusterFit {
 // of an SM's shared memory: one CTA per SM).
 inline ClusterFit query_cluster_fit() {
   ClusterFit f = {};
-  cudaFuncSetAttribute(gemm_ck_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(32));
+  cudaFuncSetAttribute(gemm_ck_kernel<32, EPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(32));
   for (int S = 1; S <= MAX_S; S++) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(S * 64);
@@ -448,7 +462,7 @@ inline ClusterFit query_cluster_fit() {
     cfg.attrs = at;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, gemm_ck_kernel<32>, &cfg) == cudaSuccess) f.max_active[S] = n;
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_ck_kernel<32, EPI_RESID>, &cfg) == cudaSuccess) f.max_active[S] = n;
   }
   cudaGetLastError();
   return f;
