@@ -376,19 +376,22 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         if (lane == 0) s_red[warp - 2][t] = s2;
       }
     }
-    if (MODE == EPI_RESID) {
-      epi_barrier();
-      // thread i finishes this CTA's i-th row, which row group i % 4 (two warps) handled
-      const int t = rank + et * S;
-      if (t < T) {
-        const int w0 = 2 * (et & 3);
-        ea.ssq_out[(size_t)(row0 + t) * tiles + tile] = s_red[w0][t] + s_red[w0 + 1][t];
-      }
+  }
+  // This CTA has read all it needs from its peers: say so now, and wait for the peers' word only
+  // before leaving (nobody leaves while a peer may still be reading its shared memory), so that
+  // the barrier's latency passes behind the rest of the epilogue.
+  if (S > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  if (warp >= 2 && MODE == EPI_RESID) {
+    const int et = threadIdx.x - 64;
+    epi_barrier();
+    // thread i finishes this CTA's i-th row, which row group i % 4 (two warps) handled
+    const int t = rank + et * S;
+    if (t < T) {
+      const int w0 = 2 * (et & 3);
+      ea.ssq_out[(size_t)(row0 + t) * tiles + tile] = s_red[w0][t] + s_red[w0 + 1][t];
     }
   }
-
-  // nobody leaves while a peer may still be reading its shared memory
-  if (S > 1) cluster_sync_all();
+  if (S > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 
   if (*reinterpret_cast<volatile int *>(err) != 0) {
     const uint64_t t0 = global_ns();
