@@ -175,6 +175,32 @@ def test_dynamic_draft_tree_matches_oracle(c0, wcuda, branch, expand, keep):
     gpu.close()
 
 
+def test_dynamic_tree_two_ragged_episodes_in_one_call(c0, wcuda):
+    """Two episodes of different prefix lengths drafted, re-ranked and verified together equal
+    the same episodes run alone."""
+    from paper_2507_22424_b200.binding import make_shape
+    desc = c0["desc"]
+    emb2 = rng.normal_bf16(5, 1, (40, desc.d_model), 1.0)
+    ids2 = torch.full((40,), -1, dtype=torch.int32)
+    ids2[30:] = rng.integers(5, 2, 10, 0, desc.action_base).to(torch.int32)
+    shape = make_shape((8, 8, 8), (1, 8, 8), keep=30)
+    gpu = _gpu(c0, wcuda)
+    alone = []
+    for emb, ids, n in ((c0["embeds"], c0["ids"], 64), (emb2, ids2, 40)):
+        gpu.prefill([0], emb.cuda(), ids.tolist(), [n])
+        tree = gpu.draft_tree([0], shape)[0]
+        alone.append((tree, gpu.verify_tree([0], None, 4)))
+    emb = torch.cat([c0["embeds"], emb2]).cuda()
+    gpu.prefill([1, 0], emb, c0["ids"].tolist() + ids2.tolist(), [64, 40])
+    trees = gpu.draft_tree([1, 0], shape)
+    m, emitted = gpu.verify_tree([1, 0], None, 4)
+    for k in range(2):
+        assert len(trees[k]["tokens"]) == 31
+        assert trees[k]["tokens"] == alone[k][0]["tokens"] and trees[k]["parent"] == alone[k][0]["parent"]
+        assert (m[k], emitted[k]) == (alone[k][1][0][0], alone[k][1][1][0])
+    gpu.close()
+
+
 def test_generate_action_with_dynamic_tree_is_lossless(c0, wcuda):
     from paper_2507_22424_b200.binding import make_shape
     gpu = _gpu(c0, wcuda)
