@@ -18,7 +18,8 @@ for). No blocking, fusion or reordering: one matmul per projection, one softmax 
 
 Only tests, the smoke check and the benchmark's CPU-baseline leg may import this package.
 Pins (tests/test_oracle_*.py): logits against the HuggingFace Llama implementation under a
-causal mask and under a tree mask; tree rows against sequential decoding of each path.
+causal mask and under a tree mask; tree rows against sequential decoding of each path;
+draft_forward against a one-layer library Llama fed the fc output, read before any final norm.
 """
 from __future__ import annotations
 

@@ -18,9 +18,11 @@ pseudo-code prints. Readings taken where the paper is silent or inconsistent:
 Pins (tests/test_oracle_*.py): r = 0 reproduces greedy autoregressive decoding (SD is
 lossless); r >= 255 accepts every action-token draft; path selection equals brute force
 over all root-to-leaf paths; a one-node tree is one autoregressive step; the cache after
-compaction equals a fresh prefill of prefix + emitted tokens. The draft model's numerics
-have no independent pin beyond the shared decoder layer: "parity unpinned" for Eq. 2's
-fc + shared-head composition.
+compaction equals a fresh prefill of prefix + emitted tokens. The draft model: every tree
+row equals sequential causal draft decoding of its own path (masks, slots, positions of the
+draft levels), and draft_forward equals a one-layer library Llama fed the fc output (Eq. 2's
+composition and the [feature ; embedding] order). Parity unpinned: only the paper's acceptance
+statistics, which need its data and trained weights.
 
 Only tests, the smoke check and the benchmark's CPU-baseline leg may import this package.
 """
@@ -155,9 +157,19 @@ class SpecVLAOracle:
         return vis
 
     # ------------------------------------------------------------------ Section 4.1, prefill
-    def prefill(self, embeds, token_ids, want_logits: bool = False):
+    def _follow(self, logits_row, own: int, other, margin: float) -> int:
+        """Re-synchronisation used by parity tests: where the top-2 margin of this row is at most
+        `margin`, the two best tokens are equally valid at the compared precision, and decoding
+        continues with the token `other` that the implementation under test chose, so that the
+        rest of the chunk stays comparable. Everywhere else the oracle's own token stands."""
+        if other is None or D.top2_margin(logits_row, self.desc, self.action_only) > margin:
+            return own
+        return int(other)
+
+    def prefill(self, embeds, token_ids, want_logits: bool = False, follow=None):
         """Target forward over the P prefix rows (causal); first token a_1 = greedy token of
-        the last row; draft forward over the P-1 shifted pairs (feature_i, input_{i+1})."""
+        the last row; draft forward over the P-1 shifted pairs (feature_i, input_{i+1}).
+        follow = (token, margin): see _follow."""
         ep = self._new_episode()
         x = D.embed_rows(self.w, embeds, token_ids)
         P = x.shape[0]
@@ -165,6 +177,8 @@ class SpecVLAOracle:
         feats = D.target_forward(self.w, self.desc, x, pos, pos, self._causal(0, P), ep.cache)
         logits_last = D.lm_head(self.w, feats[P - 1:P])[0]
         a1 = self._greedy(logits_last)
+        if follow is not None:
+            a1 = self._follow(logits_last, a1, follow[0], follow[1])
         if P > 1:
             dpos = torch.arange(P - 1)
             D.draft_forward(self.w, self.desc, feats[:P - 1], x[1:], dpos, dpos,
@@ -235,7 +249,7 @@ class SpecVLAOracle:
                     base = 0
                 order = sorted(range(lp_all.numel()), key=lambda v: (-float(lp_all[v]), v))
                 if want_debug:
-                    debug.append((n, lp_all.clone(), base))
+                    debug.append((n, lp_all.clone(), base, produced_by[n]))
                 for v in order[:shape.branch[l]]:
                     nxt.append(len(tokens))
                     tokens.append(base + v)
@@ -263,12 +277,15 @@ class SpecVLAOracle:
                                  self._tree_visible(P, tree.parent), ep.cache)
         return D.lm_head(self.w, feats), feats
 
-    def verify_tree(self, ep: Episode, tree: Tree, r: int, want_debug: bool = False):
+    def verify_tree(self, ep: Episode, tree: Tree, r: int, want_debug: bool = False, follow=None):
         """Verify, accept (Eq. 4), select the longest accepted path, compact the cache and set
-        up the next iteration. Returns (m, emitted tokens [m + 1])."""
+        up the next iteration. Returns (m, emitted tokens [m + 1]).
+        follow = (tokens per row, margin): see _follow."""
         desc = self.desc
         logits, feats = self.verify_forward(ep, tree)
-        g = [self._greedy(logits[i]) for i in range(len(tree.tokens))]
+        g_own = [self._greedy(logits[i]) for i in range(len(tree.tokens))]
+        g = g_own if follow is None else [self._follow(logits[i], g_own[i], follow[0][i], follow[1])
+                                          for i in range(len(tree.tokens))]
         m, path, emitted = accept_and_select(tree.tokens, tree.parent, tree.depth, g, r,
                                              desc.action_base, desc.n_bins)
         # compaction: accepted rows move next to the root (ascending j: a destination slot
@@ -284,7 +301,7 @@ class SpecVLAOracle:
         ep.pending_feat = [feats[j] for j in path]
         ep.pending_tok = list(emitted)
         if want_debug:
-            return m, emitted, dict(logits=logits, feats=feats, g=g, path=path)
+            return m, emitted, dict(logits=logits, feats=feats, g=g, g_own=g_own, path=path)
         return m, emitted
 
     # ------------------------------------------------------------------ Algorithm 1, outer loop
@@ -319,8 +336,10 @@ class SpecVLAOracle:
         return ep.emitted[:n_tokens], accept_lens
 
     # ------------------------------------------------------------------ Eq. 1
-    def ar_generate(self, embeds, token_ids, n_tokens: int = 7, want_margins: bool = False):
-        """Plain greedy autoregressive decoding with the verification model alone."""
+    def ar_generate(self, embeds, token_ids, n_tokens: int = 7, want_margins: bool = False, follow=None):
+        """Plain greedy autoregressive decoding with the verification model alone.
+        follow = (tokens, margin): see _follow; with it the returned list holds the oracle's own
+        greedy token at every position, each conditioned on the tokens actually continued with."""
         d = self.desc
         cache = D.KVCache(d.n_layers, self.max_seq, d.n_heads, d.head_dim, self.dtype)
         x = D.embed_rows(self.w, embeds, token_ids)
@@ -332,7 +351,9 @@ class SpecVLAOracle:
         margins = [D.top2_margin(logits, d, self.action_only)]
         while len(toks) < n_tokens:
             p = torch.tensor([P])
-            feats = D.target_forward(self.w, d, self._embed([toks[-1]]), p, p,
+            last = toks[-1] if follow is None else self._follow(logits, toks[-1], follow[0][len(toks) - 1],
+                                                                follow[1])
+            feats = D.target_forward(self.w, d, self._embed([last]), p, p,
                                      self._causal(P, 1), cache)
             logits = D.lm_head(self.w, feats)[0]
             toks.append(self._greedy(logits))

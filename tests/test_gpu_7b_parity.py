@@ -29,64 +29,78 @@ def env():
     gpu.close()
 
 
-def _prefill_both(env, emb, ids, episode=0):
-    ep, ref_logits, _ = env["orc"].prefill(emb.cpu(), ids.cpu(), want_logits=True)
-    first, logits = env["gpu"].prefill([episode], emb, ids.tolist(), [len(ids)], want_logits=True)
-    return ep, ref_logits, first[0], logits[0]
+KV_LAYERS = (0, 13, 31)      # layers whose committed cache is read back and compared
 
 
-def _check_verify(env, ep, tree, r, episode=0, log=None, dbg_ref=None):
-    """Verifies `tree` on both sides; returns True when the states stay comparable."""
-    log = [] if log is None else log
-    if dbg_ref is None:
-        m_ref, emitted_ref, dbg = env["orc"].verify_tree(ep, tree, r, want_debug=True)
-    else:
-        m_ref, emitted_ref, dbg = dbg_ref
+def _check_state_and_cache(gpu, tally, cache, P_before, m_ref, path, root, episode):
+    """State of `episode` after a commit and its cache slots [0, P + 1 + m): prefix rows as they
+    were, then the rows of `path` (oracle cache still holds the tree rows at slots P + row)."""
+    st = gpu.read_buffer(5, 4 * (episode + 1), torch.int32).tolist()[4 * episode:4 * episode + 4]
+    assert (st[0], st[2], st[3]) == (P_before + 1 + m_ref, root, m_ref + 1), st
+    src = list(range(P_before)) + [P_before + j for j in path]
+    worst = 0.0
+    for l in KV_LAYERS:
+        for which, refc in ((0, cache.k[l]), (1, cache.v[l])):
+            got = gpu.read_kv(episode, l, which, 0, len(src)).double()
+            want = refc[src].reshape(len(src), -1)
+            worst = max(worst, float((got - want).abs().max()))
+    assert worst < G.KV_TOL, worst
+    tally.caches += 1
+
+
+def _verify_against_logits(env, tree, r, logits, cache, P, tally, where, episode=0, index=0, n_ep=1,
+                           call=None):
+    """Verification of `tree` on the GPU against oracle logits of (a superset of) its rows computed
+    beforehand: logits, greedy tokens, then acceptance, path and tokens through the oracle's
+    accept_and_select on the greedy vector with the GPU's token at logged low-margin rows."""
+    gpu = env["gpu"]
     n = len(tree.tokens)
-    m, emitted, logits = env["gpu"].verify_tree([episode], [G.tree_dict(tree)], r, want_logits=True)
-    err = float((logits.cpu().double() - dbg["logits"][:n]).abs().max())
+    if call is None:
+        m, emitted, glog = gpu.verify_tree([episode], [G.tree_dict(tree)], r, want_logits=True)
+        g_gpu = gpu.read_buffer(1, n, torch.int32).tolist()
+    else:
+        m, emitted, glog, g_gpu = call
+    err = float((glog.cpu().double() - logits[:n]).abs().max())
+    tally.max_logit_err = max(tally.max_logit_err, err)
     assert err < G.LOGIT_TOL, err
-    g_gpu = env["gpu"].read_buffer(1, n, torch.int32).tolist()
-    G.compare_tokens(g_gpu, dbg["g"][:n], G.margins(dbg["logits"][:n], DESC, True).tolist(), log, "g")
-    if g_gpu != dbg["g"][:n]:
-        return False, err
-    assert (m[0], emitted[0]) == (m_ref, emitted_ref)
-    return True, err
+    mg = G.margins(logits[:n], DESC, True).tolist()
+    g_own = [env["orc"]._greedy(logits[i]) for i in range(n)]
+    G.compare_tokens(g_gpu, g_own, mg, tally, where)
+    g = [g_gpu[i] if mg[i] <= G.MARGIN else g_own[i] for i in range(n)]
+    m_ref, path, emitted_ref = accept_and_select(tree.tokens, tree.parent, tree.depth, g, r,
+                                                 DESC.action_base, DESC.n_bins)
+    assert (m[index], emitted[index]) == (m_ref, emitted_ref), (m[index], emitted[index], m_ref, emitted_ref)
+    got_path = gpu.read_buffer(4, 9 * n_ep, torch.int32).tolist()[9 * index:9 * index + m_ref + 1]
+    assert got_path == path
+    tally.accepts += 1
+    tally.iterations += 1
+    _check_state_and_cache(gpu, tally, cache, P, m_ref, path, emitted_ref[-1], episode)
+    return m_ref, err
 
 
 def test_c1_prefill_draft_verify_lockstep(env):
+    """C1 iteration by iteration until the chunk is complete: draft tree against the oracle's, then
+    the oracle's tree verified on both sides with everything compared (all 32 layers of the cache)."""
     orc, gpu = env["orc"], env["gpu"]
-    ep, ref_logits, first, logits = _prefill_both(env, env["emb"], env["ids"])
-    err = float((logits.cpu().double() - ref_logits).abs().max())
-    print("C1 prefill logits max-abs err", err)
-    assert err < G.LOGIT_TOL
-    from oracle import decoder as D
-    log = []
-    G.compare_tokens([first], [ep.root], [D.top2_margin(ref_logits, DESC, True)], log, "a1")
-    if first != ep.root:
-        pytest.skip("first token at a low margin")
-    for it in range(6):
+    tally = G.Tally()
+    ep, _, _ = G.prefill_both(orc, gpu, env["emb"], env["ids"], 0, tally, DESC)
+    print("C1 prefill logits max-abs err", tally.max_logit_err)
+    same = []
+    while len(ep.emitted) < 7:
         ref_tree, dbg = orc.draft_tree(ep, C.TREE_26, want_debug=True)
         got = gpu.draft_tree([0], env["shape"])[0]
-        assert len(got["tokens"]) == 27 and got["tokens"][0] == ep.root
-        if got["tokens"] == ref_tree.tokens:
-            assert got["parent"] == ref_tree.parent and got["depth"] == ref_tree.depth
-            assert max(abs(a - b) for a, b in zip(got["score"], ref_tree.score)) < 5e-2
-        else:
-            gap = min(float(torch.sort(lp, descending=True).values[:5].diff().abs().min()) for _, lp, _ in dbg)
-            log.append(f"it{it}: draft tree differs; smallest ranking gap {gap:.4f}")
-            assert gap < G.MARGIN
-        ok, err = _check_verify(env, ep, ref_tree, 0, log=log)
-        print(f"it{it}: verify logits err {err:.4f}")
-        if not ok or len(ep.emitted) >= 7:
-            break
-    print("\n".join(log))
+        same.append(G.compare_draft_trees(got, ref_tree, dbg, C.TREE_26, tally))
+        G.verify_both(orc, gpu, ep, ref_tree, 0, tally, DESC, where=f"it{tally.iterations}.g")
+    tally.report("C1 lockstep")
+    print("identical leading draft-tree nodes per iteration:", same)
+    assert tally.iterations >= 3 and tally.accepts == tally.caches == tally.iterations
+    assert tally.rows_exact >= 2 * tally.rows_low            # sigma_logit = 1.3: most rows are decided
+    assert max(same) == 27                                    # some iteration's tree is identical throughout
 
 
 def test_c1_generate_action_strict_equals_greedy(env):
     orc, gpu = env["orc"], env["gpu"]
     from paper_2507_22424_b200.binding import make_shape
-    ref, mg = orc.ar_generate(env["emb"].cpu(), env["ids"].cpu(), 7, want_margins=True)
     toks, acts, stats = gpu.generate_action([0], env["emb"], env["ids"].tolist(), [len(env["ids"])],
                                             env["shape"], 0, 7)
     ar, _, _ = gpu.generate_action([0], env["emb"], env["ids"].tolist(), [len(env["ids"])],
@@ -99,37 +113,36 @@ def test_c1_generate_action_strict_equals_greedy(env):
     dyn, _, st4 = gpu.generate_action([0], env["emb"], env["ids"].tolist(), [len(env["ids"])],
                                       make_shape((8,) * 5, (1, 8, 8, 8, 8), keep=50), 0, 7)
     assert dyn == toks
-    for i in range(7):
-        if mg[i] <= G.MARGIN:
-            print(f"position {i}: margin {mg[i]:.4f}; comparison stops here")
-            break
-        assert toks[0][i] == ref[i]
+    ref, mg = orc.ar_generate(env["emb"].cpu(), env["ids"].cpu(), 7, want_margins=True,
+                              follow=(toks[0], G.MARGIN))
+    tally = G.Tally()
+    G.compare_tokens(toks[0], ref, mg, tally, "chunk")
+    tally.report("C1 generate r=0")
+    assert tally.rows_exact + tally.rows_low == 7 and tally.rows_exact >= 4
     print("chunk", toks[0], "oracle", ref, "margins", [round(x, 3) for x in mg])
 
 
 def test_c3_verify_sweep_tree_sizes(env):
     """Rows {1, 8, 26, 27, 60, 128}: every size is a prefix of the same 128-row random tree, and a
     row's logits depend only on its ancestors, so one oracle pass over 128 rows gives the
-    expected logits of all of them."""
+    expected logits and cache rows of all of them."""
     orc, gpu = env["orc"], env["gpu"]
     emb, ids = data.make_prefix(C.C3, device="cuda")
     assert 290 <= len(ids) <= 297
-    ep = orc.prefill(emb.cpu(), ids.cpu())
+    tally = G.Tally()
+    ep, _, _ = G.prefill_both(orc, gpu, emb, ids, 0, tally, DESC)
+    P = ep.P
     tok, par, dep = data.random_tree(128, DESC, seed=C.C3.extra["tree_seed"], max_depth=8, root_token=ep.root)
     logits, _ = orc.verify_forward(ep, Tree(tok, par, dep, [0.0] * 128))
-    g = [orc._greedy(logits[i]) for i in range(128)]
     r = 16
     for n in C.C3.extra["rows"] + (27,):
         first = gpu.prefill([0], emb, ids.tolist(), [len(ids)])
-        if first[0] != ep.root:
-            pytest.skip("first token at a low margin")
+        assert first[0] == ep.root                       # same call as above: deterministic
         sub = Tree(tok[:n], par[:n], dep[:n], [0.0] * n)
-        m_ref, path, emitted_ref = accept_and_select(sub.tokens, sub.parent, sub.depth, g[:n], r,
-                                                     DESC.action_base, DESC.n_bins)
-        log = []
-        ok, err = _check_verify(env, None, sub, r, log=log,
-                                dbg_ref=(m_ref, emitted_ref, dict(logits=logits, g=g)))
-        print(f"T={n}: logits err {err:.4f}, m={m_ref}, comparable={ok}; " + "; ".join(log))
+        m_ref, err = _verify_against_logits(env, sub, r, logits, ep.cache, P, tally, f"g(T={n})")
+        print(f"T={n}: logits err {err:.4f}, m={m_ref}")
+    tally.report("C3 sweep")
+    assert tally.accepts == tally.caches == 6 and tally.rows_exact >= 150
 
 
 def _oracle_planted(orc, ep, seed, call):
@@ -143,40 +156,38 @@ def _oracle_planted(orc, ep, seed, call):
 def test_c2_planted_drafts_threshold_sweep(env):
     """Three oracle-planted trees of the first iteration, each verified at every threshold."""
     orc, gpu = env["orc"], env["gpu"]
-    ep = orc.prefill(env["emb"].cpu(), env["ids"].cpu())
+    tally = G.Tally()
+    ep, _, _ = G.prefill_both(orc, gpu, env["emb"], env["ids"], 0, tally, DESC)
+    P = ep.P
     for call in (0, 1, 2):
         tree = _oracle_planted(orc, ep, C.C2.seed, call)
         logits, _ = orc.verify_forward(ep, tree)
-        g = [orc._greedy(logits[i]) for i in range(27)]
         ms = []
         for r in C.C2.extra["r"]:
             first = gpu.prefill([0], env["emb"], env["ids"].tolist(), [len(env["ids"])])
-            if first[0] != ep.root:
-                pytest.skip("first token at a low margin")
-            m_ref, path, emitted_ref = accept_and_select(tree.tokens, tree.parent, tree.depth, g, r,
-                                                         DESC.action_base, DESC.n_bins)
-            ok, err = _check_verify(env, None, tree, r, dbg_ref=(m_ref, emitted_ref, dict(logits=logits, g=g)))
-            ms.append((r, m_ref, ok))
-        print(f"C2 planted tree {call}, (r, accepted length, comparable):", ms)
-        assert [m for _, m, _ in ms] == sorted(m for _, m, _ in ms)  # accepted length grows with r
+            assert first[0] == ep.root
+            m_ref, err = _verify_against_logits(env, tree, r, logits, ep.cache, P, tally, f"tree{call}.r{r}.g")
+            ms.append((r, m_ref))
+        print(f"C2 planted tree {call}, (r, accepted length):", ms)
+        assert [m for _, m in ms] == sorted(m for _, m in ms)  # accepted length grows with r
+    tally.report("C2 threshold sweep")
+    assert tally.accepts == tally.caches == 18
 
 
 def test_c2_planted_chunk_lockstep_r4(env):
     """A whole chunk with oracle-planted trees at r = 4, iteration by iteration."""
     orc, gpu = env["orc"], env["gpu"]
-    ep, _, first, _ = _prefill_both(env, env["emb"], env["ids"])
-    if first != ep.root:
-        pytest.skip("first token at a low margin")
-    log, lens = [], []
-    for it in range(6):
-        tree = _oracle_planted(orc, ep, C.C2.seed, 10 + it)
+    tally = G.Tally()
+    ep, _, _ = G.prefill_both(orc, gpu, env["emb"], env["ids"], 0, tally, DESC)
+    lens = []
+    while len(ep.emitted) < 7:
+        tree = _oracle_planted(orc, ep, C.C2.seed, 10 + tally.iterations)
         gpu.draft_tree([0], env["shape"], want_trees=False)       # keeps the draft state in step
-        n_before = len(ep.emitted)
-        ok, err = _check_verify(env, ep, tree, 4, log=log)
-        lens.append(len(ep.emitted) - n_before - 1)
-        if not ok or len(ep.emitted) >= 7:
-            break
-    print("accepted lengths", lens, "emitted", ep.emitted[:7], "\n".join(log))
+        ref = G.verify_both(orc, gpu, ep, tree, 4, tally, DESC, where=f"it{tally.iterations}.g")
+        lens.append(ref[0])
+    tally.report("C2 chunk r=4")
+    print("accepted lengths", lens, "emitted", ep.emitted[:7])
+    assert tally.accepts == tally.caches == tally.iterations == len(lens) and sum(lens) >= 1
 
 
 def test_c4_sixteen_ragged_episodes(env):
@@ -191,33 +202,35 @@ def test_c4_sixteen_ragged_episodes(env):
     emb = torch.cat([e for e, _ in pre])
     ids = torch.cat([i for _, i in pre]).tolist()
     first, logits = gpu.prefill(list(range(n_ep)), emb, ids, lens, want_logits=True)
+    tally = G.Tally()
     trees, refs = [], {}
+    from oracle import decoder as D
     for e in range(n_ep):
         if e in (0, 15):
-            ep, ref_logits, _ = orc.prefill(pre[e][0].cpu(), pre[e][1].cpu(), want_logits=True)
+            ep, ref_logits, _ = orc.prefill(pre[e][0].cpu(), pre[e][1].cpu(), want_logits=True,
+                                            follow=(first[e], G.MARGIN))
             assert float((logits[e].cpu().double() - ref_logits).abs().max()) < G.LOGIT_TOL
+            G.compare_tokens([first[e]], [D.greedy_token(ref_logits, DESC, True)],
+                             [D.top2_margin(ref_logits, DESC, True)], tally, f"ep{e}.a1")
             t = _oracle_planted(orc, ep, C.C4.extra["prefix_seed"], 100 + e)
-            refs[e] = (ep, t, orc.verify_tree(ep, t, r, want_debug=True))
+            refs[e] = (ep, t, orc.verify_forward(ep, t)[0])
             trees.append(G.tree_dict(t))
         else:
             tok, par, dep = data.random_tree(27, DESC, seed=50 + e, max_depth=5, root_token=first[e])
             trees.append(dict(tokens=tok, parent=par, depth=dep))
-    if any(first[e] != refs[e][0].emitted[0] for e in refs):
-        pytest.skip("first token at a low margin")
     m, emitted, vlogits = gpu.verify_tree(list(range(n_ep)), trees, r, want_logits=True)
     g_all = gpu.read_buffer(1, 27 * n_ep, torch.int32).tolist()
-    for e, (ep, t, (m_ref, emitted_ref, dbg)) in refs.items():
+    for e, (ep, t, ref_logits) in refs.items():
         rows = slice(27 * e, 27 * e + 27)
-        err = float((vlogits[rows].cpu().double() - dbg["logits"]).abs().max())
-        assert err < G.LOGIT_TOL, err
-        log = []
-        G.compare_tokens(g_all[rows], dbg["g"], G.margins(dbg["logits"], DESC, True).tolist(), log, f"ep{e}.g")
-        if g_all[rows] == dbg["g"]:
-            assert (m[e], emitted[e]) == (m_ref, emitted_ref)
-        print(f"episode {e}: P={lens[e]}, logits err {err:.4f}, m={m_ref}; " + "; ".join(log))
+        m_ref, err = _verify_against_logits(env, t, r, ref_logits, ep.cache, lens[e], tally, f"ep{e}.g",
+                                            episode=e, index=e, n_ep=n_ep,
+                                            call=(m, emitted, vlogits[rows], g_all[rows]))
+        print(f"episode {e}: P={lens[e]}, logits err {err:.4f}, m={m_ref}")
     st = gpu.read_buffer(5, 4 * n_ep, torch.int32).reshape(n_ep, 4).tolist()
     for e in range(n_ep):
         assert st[e][0] == lens[e] + 1 + m[e] and st[e][3] == m[e] + 1
+    tally.report("C4 batch")
+    assert tally.accepts == tally.caches == 2
 
 
 @pytest.mark.parametrize("T,N,K", [(27, 22016, 4096), (27, 4096, 11008), (128, 12288, 4096),

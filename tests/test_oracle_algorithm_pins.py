@@ -344,6 +344,93 @@ def test_draft_state_after_commit_equals_fresh_prefill(c0):
     assert max(abs(a - b) for a, b in zip(ref.score, nxt.score)) < 1e-9
 
 
+@pytest.mark.parametrize("shape", [C.TREE_C0, C.TreeShape((3, 2, 2, 1), (1, 2, 3, 2)),
+                                   C.TreeShape((4, 4, 4), (1, 3, 4), keep=0)])
+def test_draft_tree_rows_equal_sequential_draft_decoding(c0, shape):
+    """Eq. 2 on a tree is Eq. 2 on each path: the predicted feature of every expanded node (the
+    draft output that scores its children) equals the last row of one ordinary causal draft
+    forward over the prefix pairs (f_i, e_{i+1}), the pair (f_{P-1}, e(a_1)) and the node's own
+    path of (predicted feature of the parent, embedding of the node's token) pairs at positions
+    0, 1, 2, ... - which fixes the draft-level masks, cache slots and positions."""
+    desc = c0["desc"]
+    orc = c0["make"]()
+    ep, _, feats = orc.prefill(c0["embeds"], c0["ids"], want_logits=True)
+    x0 = D.embed_rows(orc.w, c0["embeds"], c0["ids"])
+    P = x0.shape[0]
+    tree, dbg = orc.draft_tree(ep, shape, want_debug=True)
+    out_of = {node: out for node, _, _, out in dbg}
+    assert len(out_of) == 1 + sum(shape.expand[1:]) and max(tree.depth[n] for n in out_of) == shape.depth - 1
+    for node, out in out_of.items():
+        path = []
+        j = node
+        while j != -1:
+            path.append(j)
+            j = tree.parent[j]
+        path.reverse()                                          # root .. node
+        feat_in = [feats[i] for i in range(P)] + [out_of[tree.parent[j]] for j in path[1:]]
+        emb_in = [x0[i] for i in range(1, P)] + [orc._embed([tree.tokens[j]])[0] for j in path]
+        n = len(feat_in)
+        assert n == len(emb_in) == P + len(path) - 1
+        cache = D.KVCache(1, n, desc.n_heads, desc.head_dim)
+        seq = D.draft_forward(orc.w, desc, torch.stack(feat_in), torch.stack(emb_in), torch.arange(n),
+                              torch.arange(n), orc._causal(0, n), cache)
+        assert (seq[-1] - out).abs().max() < 1e-10, (node, float((seq[-1] - out).abs().max()))
+
+
+def test_draft_forward_matches_one_layer_hf_llama(c0):
+    """Eq. 2 / Eq. 5 composition: fc over [feature ; embedding] followed by one decoder layer, the
+    layer's output taken BEFORE any final norm. Library pin: a one-layer HuggingFace Llama fed
+    inputs_embeds = feature @ Wfc[:, :d]^T + embedding @ Wfc[:, d:]^T, output read by a forward
+    hook on its decoder layer."""
+    from transformers import LlamaConfig, LlamaForCausalLM
+    desc, w = c0["desc"], c0["weights"]
+    d, hd, F = desc.d_model, desc.n_heads * desc.head_dim, desc.d_ffn
+    cfg = LlamaConfig(vocab_size=desc.vocab, hidden_size=d, intermediate_size=F, num_hidden_layers=1,
+                      num_attention_heads=desc.n_heads, num_key_value_heads=desc.n_heads,
+                      head_dim=desc.head_dim, rms_norm_eps=desc.rms_eps, rope_theta=desc.rope_theta,
+                      max_position_embeddings=1024, attention_bias=False, mlp_bias=False,
+                      tie_word_embeddings=False)
+    cfg._attn_implementation = "eager"
+    m = LlamaForCausalLM(cfg).double().eval()
+    q = "draft.layer."
+    sd = {"model.layers.0.self_attn.q_proj.weight": w[q + "wqkv"][:hd],
+          "model.layers.0.self_attn.k_proj.weight": w[q + "wqkv"][hd:2 * hd],
+          "model.layers.0.self_attn.v_proj.weight": w[q + "wqkv"][2 * hd:],
+          "model.layers.0.self_attn.o_proj.weight": w[q + "wo"],
+          "model.layers.0.mlp.gate_proj.weight": w[q + "wgu"][:F],
+          "model.layers.0.mlp.up_proj.weight": w[q + "wgu"][F:],
+          "model.layers.0.mlp.down_proj.weight": w[q + "wd"],
+          "model.layers.0.input_layernorm.weight": w[q + "norm1"],
+          "model.layers.0.post_attention_layernorm.weight": w[q + "norm2"]}
+    m.load_state_dict({k: v.double() for k, v in sd.items()}, strict=False)
+    grabbed = []
+    m.model.layers[0].register_forward_hook(
+        lambda mod, args, out: grabbed.append(out[0] if isinstance(out, tuple) else out))
+    orc = c0["make"]()
+    n = 23
+    g = torch.Generator().manual_seed(3)
+    feat = torch.randn(n, d, generator=g, dtype=torch.float64)
+    emb = torch.randn(n, d, generator=g, dtype=torch.float64)
+    # a tree-ish mask and per-row positions, as the draft levels use them
+    vis = orc._causal(0, n).clone()
+    vis[15:, 10:15] = False
+    pos = torch.cat([torch.arange(15), torch.tensor([15, 15, 16, 16, 16, 17, 17, 18])])
+    cache = D.KVCache(1, n, desc.n_heads, desc.head_dim)
+    mine = D.draft_forward(orc.w, desc, feat, emb, pos, torch.arange(n), vis, cache)
+    Wfc = w["draft.fc"].double()
+    z = feat @ Wfc[:, :d].T + emb @ Wfc[:, d:].T
+    mask = torch.zeros(n, n, dtype=torch.float64)
+    mask[~vis] = torch.finfo(torch.float64).min
+    with torch.no_grad():
+        m(inputs_embeds=z[None], attention_mask=mask[None, None], position_ids=pos[None])
+    ref = grabbed[0].reshape(n, d)
+    assert torch.allclose(mine, ref, atol=5e-6, rtol=0), float((mine - ref).abs().max())
+    # [feature ; embedding] order: swapping the halves must be visible
+    swapped = D.draft_forward(orc.w, desc, emb, feat, pos, torch.arange(n), vis,
+                              D.KVCache(1, n, desc.n_heads, desc.head_dim))
+    assert (swapped - ref).abs().max() > 1e-2
+
+
 def test_draft_tree_invariants(c0):
     shape = c0["wl"].tree
     for action_only in (True, False):
@@ -360,7 +447,7 @@ def test_draft_tree_invariants(c0):
             assert tree.score[i] <= tree.score[p] + 1e-12          # log-probs are <= 0
             if action_only:
                 assert A0 <= tree.tokens[i] < A0 + NB
-        for node, lp, base in dbg:
+        for node, lp, base, _ in dbg:
             kids = [i for i in range(n) if tree.parent[i] == node]
             assert abs(float(torch.exp(lp).sum()) - 1.0) < 1e-9
             top = torch.topk(lp, len(kids))
