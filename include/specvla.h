@@ -134,6 +134,23 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *target
                    specvla_ctx **out);
 int specvla_destroy(specvla_ctx *ctx);
 
+/* Execution options of a context (all default to the fastest setting; they exist for A/B
+ * measurements and tests, and change no result beyond rounding order):
+ *   SPECVLA_OPT_PERSISTENT_FORWARD  1: forwards of one episode and at most 32 rows (the batch-1
+ *       verification step of Algorithm 1, an autoregressive step) run as ONE cooperative kernel
+ *       whose weight stream continues across all GEMMs of all layers; 0: one launch per GEMM.
+ *   SPECVLA_OPT_DEPENDENT_LAUNCH    1: kernels of the per-GEMM path are launched with programmatic
+ *       stream serialisation (a GEMM streams weights while its predecessor drains).
+ *   SPECVLA_OPT_L2_PREFETCH         1: a GEMM of the per-GEMM path prefetches the head of the next
+ *       matrix into L2.
+ *   SPECVLA_OPT_WAIT_LIMIT_NS       limit of every device-side wait of the persistent kernel in
+ *       nanoseconds (default 2e9); a wait that runs out makes the call return SPECVLA_ERR_TIMEOUT. */
+#define SPECVLA_OPT_PERSISTENT_FORWARD 1
+#define SPECVLA_OPT_DEPENDENT_LAUNCH   2
+#define SPECVLA_OPT_L2_PREFETCH        3
+#define SPECVLA_OPT_WAIT_LIMIT_NS      4
+int specvla_set_option(specvla_ctx *ctx, int option, long long value);
+
 /* Forgets an episode's state (its caches are simply overwritten by the next prefill). */
 int specvla_reset(specvla_ctx *ctx, int episode);
 

@@ -15,6 +15,7 @@ from .build import LIB_PATH
 MAX_DEPTH = 8
 MAX_TREE_ROWS = 128
 
+OPT_PERSISTENT_FORWARD, OPT_DEPENDENT_LAUNCH, OPT_L2_PREFETCH, OPT_WAIT_LIMIT_NS = 1, 2, 3, 4
 BUF_GREEDY, BUF_MARGIN, BUF_FEATURES, BUF_PATH, BUF_STATE, BUF_TOPK_TOK, BUF_TOPK_LP = 1, 2, 3, 4, 5, 6, 7
 
 
@@ -55,6 +56,7 @@ EXPORTS = {
                                  C.c_void_p, C.c_size_t, C.POINTER(C.c_void_p)]),
     "specvla_destroy": (C.c_int, [C.c_void_p]),
     "specvla_reset": (C.c_int, [C.c_void_p, C.c_int]),
+    "specvla_set_option": (C.c_int, [C.c_void_p, C.c_int, C.c_longlong]),
     "specvla_prefill": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_int), C.c_void_p, C.POINTER(C.c_int),
                                   C.POINTER(C.c_int), C.POINTER(C.c_int), C.c_void_p, C.c_void_p]),
     "specvla_draft_tree": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_int), C.POINTER(TreeShape),
@@ -167,6 +169,9 @@ class SpecVLA:
             self.close()
         except Exception:
             pass
+
+    def set_option(self, option: int, value: int):
+        self._check(lib.specvla_set_option(self.h, int(option), int(value)))
 
     def _check(self, rc):
         if rc != 0:

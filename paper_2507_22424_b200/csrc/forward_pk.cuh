@@ -74,7 +74,8 @@ struct Op {
   const float *gain;           // EPI_RESID: gain of the next RMSNorm folded into the operand written
   float *cache;                // EPI_QKV / attention: this layer's cache, [episode][2][max_seq][hd]
   size_t ep_stride;
-  float *out;                  // EPI_PLAIN: [rows][ldo] logits (may be NULL)
+  float *out;                  // EPI_PLAIN: [rows][ldo] logits (may be NULL); POST_ARGMAX phases write
+                               // to Params::logits_out instead
   int ldo, lo, hi;             // EPI_PLAIN: argmax / top-k range over output columns
   int post;                    // PostKind after an EPI_PLAIN phase
   int tok_offset;              // POST_TOPK: token id of output column 0
@@ -100,6 +101,7 @@ struct Params {
   int splits;
   const float2 *rope_tab;
   float4 *cand;                // [32][2 * tiles]: (top-1 value, top-1 id, top-2 value, -) per 128 columns
+  float *logits_out;           // [rows][ldo] of the POST_ARGMAX phase, or NULL
   int *greedy;                 // POST_ARGMAX
   float *margin;
   int *top_tok;                // POST_TOPK: [rows][SV_TOPK]
@@ -176,10 +178,13 @@ struct Cta {
 // ------------------------------------------------------------------------- grid barrier
 // All 256 epilogue threads of every CTA call this the same number of times. `epoch` counts calls.
 __device__ __forceinline__ bool grid_barrier(const Params &p, int G, unsigned &epoch, int et, volatile int *s_ok) {
+  // what this thread wrote is about to be read by other CTAs, partly through bulk copies (async proxy)
+  asm volatile("fence.proxy.async.global;" ::: "memory");
   __threadfence();
   epi_sync();
   if (et == 0) {
     epoch++;
+    __threadfence();
     atomicAdd(p.bar, 1u);
     const unsigned target = epoch * (unsigned)G;
     bool ok = true;
@@ -193,6 +198,7 @@ __device__ __forceinline__ bool grid_barrier(const Params &p, int G, unsigned &e
         }
       }
     }
+    __threadfence();
     if (!ok) atomicCAS(p.err, 0, SV_ERR_WAIT_GRID);
     *s_ok = ok ? 1 : 0;
   }
@@ -234,7 +240,7 @@ __device__ void attention_unit(const Params &p, const Op &op, unsigned char *sme
     const int i = tid + k * EPI_THREADS;
     const int r = i / C4, c = i % C4;
     qv[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (r < nrows) qv[k] = *reinterpret_cast<const float4 *>(p.q + (size_t)r * hd + h * DH + c * 4);
+    if (r < nrows) qv[k] = __ldcg(reinterpret_cast<const float4 *>(p.q + (size_t)r * hd + h * DH + c * 4));
   }
   epi_sync();                               // the previous unit's shared state is no longer read
   if (tid < RB) {
@@ -270,8 +276,8 @@ __device__ void attention_unit(const Params &p, const Op &op, unsigned char *sme
       const int i = tid + k * EPI_THREADS;
       const int slot = t * KT + i / C4, c = i % C4;
       if (slot < kmax) {
-        kreg[k] = *reinterpret_cast<const float4 *>(kbase + (size_t)slot * hd + c * 4);
-        vreg[k] = *reinterpret_cast<const float4 *>(vbase + (size_t)slot * hd + c * 4);
+        kreg[k] = __ldcg(reinterpret_cast<const float4 *>(kbase + (size_t)slot * hd + c * 4));
+        vreg[k] = __ldcg(reinterpret_cast<const float4 *>(vbase + (size_t)slot * hd + c * 4));
       } else {
         kreg[k] = make_float4(0.f, 0.f, 0.f, 0.f);
         vreg[k] = kreg[k];
@@ -433,10 +439,10 @@ __device__ void attention_unit(const Params &p, const Op &op, unsigned char *sme
   }
 }
 
-template <int DH> constexpr int attn_smem_bytes() {
+template <int DH> __host__ __device__ constexpr int attn_smem_bytes() {
   return (2 * (32 + 2 * 32) * (DH + 8) + 2 * 32 * (32 + 8)) * (int)sizeof(bf16) + 32 * (32 + 4) * (int)sizeof(float);
 }
-template <int DH> constexpr int smem_bytes() { return STAGES * STAGE_BYTES + attn_smem_bytes<DH>() + 1024 + 128; }
+template <int DH> __host__ __device__ constexpr int smem_bytes() { return STAGES * STAGE_BYTES + attn_smem_bytes<DH>() + 1024 + 128; }
 
 // ------------------------------------------------------------------------- the kernel
 template <int DH>
@@ -452,8 +458,7 @@ __global__ void __launch_bounds__(THREADS, 1) forward_pk_kernel(const __grid_con
   auto tempty_bar = [&](int b) { return bars + 8u * (2 * STAGES + 2 + b); };
   const uint32_t xready_bar = bars + 8u * (2 * STAGES + 4);
   const uint32_t tmem_slot = bars + 8u * (2 * STAGES + 5);
-  __shared__ int s_ok;
-  __shared__ float s_scale[TN];
+  __shared__ int s_ok, s_gok;              // results of bounded waits, shared by the epilogue threads
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int c = blockIdx.x, G = gridDim.x;
@@ -541,6 +546,7 @@ __global__ void __launch_bounds__(THREADS, 1) forward_pk_kernel(const __grid_con
           break;
         }
         g++;
+        asm volatile("fence.proxy.async.global;" ::: "memory");
         const int U = o.tiles * o.KB;
         const int ub = ubegin(U, c, G), ue = ubegin(U, c + 1, G);
         for (int u = ub; u < ue; u++, it++) {
@@ -632,13 +638,13 @@ __global__ void __launch_bounds__(THREADS, 1) forward_pk_kernel(const __grid_con
           const float ss = warp_sum(v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w);
           if (lane == 0) p.ssq[t * p.nt + ch] = ss;
         }
-        if (!grid_barrier(p, G, epoch, et, &s_ok)) break;
+        if (!grid_barrier(p, G, epoch, et, &s_gok)) break;
         continue;
       }
       if (o.kind == OP_ATTN) {
         const int units = p.H * p.splits;
         for (int un = c; un < units; un += G) attention_unit<DH>(p, o, attn_smem, et, un / p.splits, un % p.splits);
-        if (!grid_barrier(p, G, epoch, et, &s_ok)) break;
+        if (!grid_barrier(p, G, epoch, et, &s_gok)) break;
         // merge of the key slices: one warp per (row, head); the O projection's operand
         constexpr int LO = DH + 4, PER = DH / 32;
         for (int item = gw; item < T * p.H; item += GW) {
@@ -648,13 +654,13 @@ __global__ void __launch_bounds__(THREADS, 1) forward_pk_kernel(const __grid_con
           for (int s2 = 0; s2 < MAX_SPLITS; s2++)
             if (s2 < p.splits) {
               const float *src = p.apart + ((size_t)(h * p.splits + s2) * 32 + t) * LO;
-              ms[s2] = src[DH];
-              ls[s2] = src[DH + 1];
+              ms[s2] = __ldcg(src + DH);
+              ls[s2] = __ldcg(src + DH + 1);
               if (PER == 4) {
-                const float4 t4 = *reinterpret_cast<const float4 *>(src + lane * 4);
+                const float4 t4 = __ldcg(reinterpret_cast<const float4 *>(src + lane * 4));
                 os[s2][0] = t4.x; os[s2][1] = t4.y; os[s2][2 % PER] = t4.z; os[s2][3 % PER] = t4.w;
               } else {
-                const float2 t2 = *reinterpret_cast<const float2 *>(src + lane * 2);
+                const float2 t2 = __ldcg(reinterpret_cast<const float2 *>(src + lane * 2));
                 os[s2][0] = t2.x; os[s2][1] = t2.y;
               }
             }
@@ -686,7 +692,7 @@ __global__ void __launch_bounds__(THREADS, 1) forward_pk_kernel(const __grid_con
                 __floats2bfloat162_rn(ov[0] * inv - hf.x, ov[1] * inv - hf.y);
           }
         }
-        if (!grid_barrier(p, G, epoch, et, &s_ok)) break;
+        if (!grid_barrier(p, G, epoch, et, &s_gok)) break;
         continue;
       }
       // -------------------------------------------------------------- GEMM phase
@@ -732,7 +738,7 @@ __global__ void __launch_bounds__(THREADS, 1) forward_pk_kernel(const __grid_con
         }
         if (!alive) break;
       }
-      if (!grid_barrier(p, G, epoch, et, &s_ok)) break;
+      if (!grid_barrier(p, G, epoch, et, &s_gok)) break;
       // part 2: sum the partial tiles of every output tile in CTA order and finish
       const bool swiglu = o.mode == EPI_SWIGLU;
       const int halves = swiglu ? 1 : 2;
@@ -746,18 +752,20 @@ __global__ void __launch_bounds__(THREADS, 1) forward_pk_kernel(const __grid_con
         float sc = 1.f;
         if (o.use_scale) {
           float ss = 0.f;
-          for (int i = lane; i < p.nt; i += 32) ss += p.ssq[t * p.nt + i];
+          for (int i = lane; i < p.nt; i += 32) ss += __ldcg(p.ssq + t * p.nt + i);
           ss = warp_sum(ss);
           sc = rsqrtf(ss / (float)p.d + p.eps);
         }
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f), v2 = v;
         for (int cc = cf; cc <= cl; cc++) {
-          const int seg = j - ubegin(U, cc, G) / o.KB;
+          const int cb = ubegin(U, cc, G);
+          if (cb == ubegin(U, cc + 1, G)) continue;                    // a CTA without units
+          const int seg = j - cb / o.KB;
           const float *src = p.part + (((size_t)cc * p.max_seg + seg) * TN + t) * BM + col;
-          const float4 a = *reinterpret_cast<const float4 *>(src);
+          const float4 a = __ldcg(reinterpret_cast<const float4 *>(src));
           v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w;
           if (swiglu) {
-            const float4 b = *reinterpret_cast<const float4 *>(src + 128);
+            const float4 b = __ldcg(reinterpret_cast<const float4 *>(src + 128));
             v2.x += b.x; v2.y += b.y; v2.z += b.z; v2.w += b.w;
           }
         }
@@ -803,7 +811,7 @@ __global__ void __launch_bounds__(THREADS, 1) forward_pk_kernel(const __grid_con
           if (n < o.N) {
             float *xp = p.x + (size_t)t * o.N + n;
             if (o.accumulate) {
-              const float4 xo = *reinterpret_cast<const float4 *>(xp);
+              const float4 xo = __ldcg(reinterpret_cast<const float4 *>(xp));
               v.x += xo.x; v.y += xo.y; v.z += xo.z; v.w += xo.w;
             }
             *reinterpret_cast<float4 *>(xp) = v;
@@ -818,7 +826,8 @@ __global__ void __launch_bounds__(THREADS, 1) forward_pk_kernel(const __grid_con
           // EPI_PLAIN: logits of 128 columns; their top-2 over [lo, hi) for the argmax / top-k
           const int n = j * BM + col;
           const float4 ov = make_float4(sc * v.x, sc * v.y, sc * v.z, sc * v.w);
-          if (o.out && n < o.N) *reinterpret_cast<float4 *>(o.out + (size_t)t * o.ldo + n) = ov;
+          float *outp = o.post == POST_ARGMAX ? p.logits_out : o.out;
+          if (outp && n < o.N) *reinterpret_cast<float4 *>(outp + (size_t)t * o.ldo + n) = ov;
           if (o.post == POST_ARGMAX) {
             epi::Top2 b{-INFINITY, -INFINITY, 0x7fffffff};
             const float vv[4] = {ov.x, ov.y, ov.z, ov.w};
@@ -830,13 +839,13 @@ __global__ void __launch_bounds__(THREADS, 1) forward_pk_kernel(const __grid_con
           }
         }
       }
-      if (!grid_barrier(p, G, epoch, et, &s_ok)) break;
+      if (!grid_barrier(p, G, epoch, et, &s_gok)) break;
       if (o.post == POST_ARGMAX) {
         // one warp per row merges the per-128-column candidates (ties to the lowest id)
         for (int t = gw; t < T; t += GW) {
           epi::Top2 b{-INFINITY, -INFINITY, 0x7fffffff};
           for (int i = lane; i < 2 * o.tiles; i += 32) {
-            const float4 cd = p.cand[(size_t)t * (2 * o.tiles) + i];
+            const float4 cd = __ldcg(p.cand + (size_t)t * (2 * o.tiles) + i);
             epi::Top2 other{cd.x, cd.z, __float_as_int(cd.y)};
             epi::top2_merge(b, other);
           }
@@ -852,10 +861,10 @@ __global__ void __launch_bounds__(THREADS, 1) forward_pk_kernel(const __grid_con
         for (int t = gw; t < T; t += GW) {
           const float *lg = o.out + (size_t)t * o.ldo;
           float mx = -INFINITY;
-          for (int v = o.lo + lane; v < o.hi; v += 32) mx = fmaxf(mx, lg[v]);
+          for (int v = o.lo + lane; v < o.hi; v += 32) mx = fmaxf(mx, __ldcg(lg + v));
           mx = warp_max(mx);
           float se = 0.f;
-          for (int v = o.lo + lane; v < o.hi; v += 32) se += expf(lg[v] - mx);
+          for (int v = o.lo + lane; v < o.hi; v += 32) se += expf(__ldcg(lg + v) - mx);
           se = warp_sum(se);
           const float lse = mx + logf(se);
           int chosen[SV_TOPK];
@@ -865,7 +874,7 @@ __global__ void __launch_bounds__(THREADS, 1) forward_pk_kernel(const __grid_con
             for (int v = o.lo + lane; v < o.hi; v += 32) {
               bool taken = false;
               for (int jj = 0; jj < k; jj++) taken |= (chosen[jj] == v);
-              const float xv = lg[v];
+              const float xv = __ldcg(lg + v);
               if (!taken && (xv > bv || (xv == bv && v < bi))) { bv = xv; bi = v; }
             }
 #pragma unroll

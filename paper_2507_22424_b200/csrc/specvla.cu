@@ -7,12 +7,14 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <algorithm>
 #include <new>
 #include <vector>
 
 #include "attention.cuh"
 #include "common.cuh"
 #include "epilogue.cuh"
+#include "forward_pk.cuh"
 #include "gemm_ck.cuh"
 #include "gemm_tc.cuh"
 #include "tree.cuh"
@@ -94,6 +96,21 @@ struct specvla_ctx {
   EpState *st;
   DevTree *trees;
 
+  // persistent forward kernel (forward_pk.cuh): calls of one episode and at most 32 rows
+  bool pk_ok;                   // shapes allow it and all CTAs of its grid are resident together
+  bool use_pk;
+  int pk_G;                     // its grid: one CTA per SM
+  int pk_max_seg, pk_splits, pk_nt;
+  pk::Op *pk_ops_t;             // phase list of the target forward (device)
+  int pk_n_ops_t;
+  float *pk_part, *pk_apart, *pk_ssq;
+  float4 *pk_cand;
+  bf16 *pk_xn, *pk_ao, *pk_hid;
+  unsigned *pk_bar;
+  unsigned long long wait_ns;   // limit of every device-side wait
+  const float *last_ssq;        // sums of squares (and their slots per row) left by the last target forward
+  int last_nt;
+
   // host side
   void *pinned;                 // pinned staging: [small results | tree staging | row tables]
   size_t pinned_bytes;
@@ -146,6 +163,43 @@ bool desc_ok(const specvla_model_desc *d) {
   if (d->max_seq < 2 || d->max_episodes < 1 || d->max_episodes > SV_MAX_EP || d->max_rows < 1) return false;
   if (!(d->rms_eps > 0.f) || !(d->rope_theta > 1.f)) return false;
   return true;
+}
+
+// The persistent forward kernel needs rows of 128-column groups (sums of squares, RoPE partner
+// lanes) and one of its two head sizes.
+bool pk_shapes_ok(const specvla_model_desc &d) {
+  const int hd = d.n_heads * d.head_dim;
+  return d.d_model % 128 == 0 && hd % 128 == 0 && d.d_model / 128 <= 64 * 32 && d.n_heads <= 148;
+}
+int sm_count() {
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1)
+    n = 148;
+  return n;
+}
+int pk_splits_for(const specvla_model_desc &d, int G) {
+  int s = G / d.n_heads;
+  return s < 1 ? 1 : (s > pk::MAX_SPLITS ? pk::MAX_SPLITS : s);
+}
+// Most output tiles any CTA's unit range touches in one GEMM phase of this model.
+int pk_max_segments(const specvla_model_desc &d, int G) {
+  const int hd = d.n_heads * d.head_dim;
+  auto kb = [](int K) { return (K + gemm_tc::BK - 1) / gemm_tc::BK; };
+  auto t256 = [](int N) { return (N + SV_TILE_ROWS - 1) / SV_TILE_ROWS; };
+  const int shapes[7][2] = {{t256(3 * hd), kb(d.d_model)}, {t256(d.d_model), kb(hd)},
+                            {(d.d_ffn + 127) / 128, kb(d.d_model)}, {t256(d.d_model), kb(d.d_ffn)},
+                            {t256(d.vocab), kb(d.d_model)}, {t256(d.n_bins), kb(d.d_model)},
+                            {t256(d.d_model), kb(2 * d.d_model)}};
+  int worst = 1;
+  for (auto &sh : shapes) {
+    const long long U = (long long)sh[0] * sh[1];
+    for (int c = 0; c < G; c++) {
+      const long long b = U * c / G, e = U * (c + 1) / G;
+      if (e > b) worst = std::max(worst, (int)((e - 1) / sh[1] - b / sh[1] + 1));
+    }
+  }
+  return worst;
 }
 
 // Lays the workspace out; with base == NULL only measures it.
@@ -216,12 +270,30 @@ size_t carve(specvla_ctx *c, char *base) {
   c->st = cv.take<EpState>(E);
   c->trees = cv.take<DevTree>(E);
   c->err = cv.take<int>(32);
+  // persistent forward kernel: packed operands, partial tiles, attention slices, candidates
+  if (pk_shapes_ok(d)) {
+    const size_t G = c->pk_G;
+    auto kblocks = [](int K) { return (size_t)((K + gemm_tc::BK - 1) / gemm_tc::BK); };
+    c->pk_nt = d.d_model / 128;
+    c->pk_splits = pk_splits_for(d, (int)G);
+    c->pk_max_seg = pk_max_segments(d, (int)G);
+    c->pk_xn = cv.take<bf16>(kblocks(d.d_model) * pk::X_BLOCK_ELEMS);
+    c->pk_ao = cv.take<bf16>(kblocks(hd) * pk::X_BLOCK_ELEMS);
+    c->pk_hid = cv.take<bf16>(kblocks(d.d_ffn) * pk::X_BLOCK_ELEMS);
+    c->pk_part = cv.take<float>(G * c->pk_max_seg * pk::PART_ELEMS);
+    c->pk_apart = cv.take<float>((size_t)d.n_heads * c->pk_splits * 32 * (d.head_dim + 4));
+    c->pk_ssq = cv.take<float>((size_t)32 * c->pk_nt);
+    c->pk_cand = cv.take<float4>((size_t)32 * 2 * tiles256(d.vocab));
+    c->pk_ops_t = cv.take<pk::Op>((size_t)5 * d.n_layers + 2);
+    c->pk_bar = cv.take<unsigned>(32);
+  }
   return (cv.off + ALIGN - 1) / ALIGN * ALIGN;
 }
 
 void derive_caps(specvla_ctx *c) {
   const specvla_model_desc &d = c->desc;
   c->hd = d.n_heads * d.head_dim;
+  c->pk_G = sm_count();
   size_t lm = (size_t)d.max_episodes * SV_MAX_TREE;
   if (lm > (size_t)d.max_rows) lm = d.max_rows;
   c->max_lm_rows = (int)lm;
@@ -421,6 +493,8 @@ int target_forward(specvla_ctx *ctx, int R, const EpArgs &rows, const bf16 *embe
                   last ? &ctx->lm_head : &ctx->layers[l + 1].wqkv, st));
   }
   ctx->last_rows = R;
+  ctx->last_ssq = ctx->ssq;
+  ctx->last_nt = ctx->nt;
   return SPECVLA_OK;
 }
 
@@ -449,6 +523,154 @@ void argmax_range(const specvla_ctx *ctx, int *lo, int *hi) {
     *lo = 0;
     *hi = ctx->desc.vocab;
   }
+}
+
+// Phase list of the target forward for the persistent kernel: embedding, the layers, the LM head
+// with the greedy argmax. Built on the host, kept in the workspace.
+void pk_build_target_ops(specvla_ctx *ctx) {
+  const specvla_model_desc &d = ctx->desc;
+  const int hd = ctx->hd, F = d.d_ffn;
+  auto kb = [](int K) { return (K + gemm_tc::BK - 1) / gemm_tc::BK; };
+  auto t256 = [](int N) { return (N + SV_TILE_ROWS - 1) / SV_TILE_ROWS; };
+  std::vector<pk::Op> ops;
+  auto gemm_op = [&](int mode, const WMat &w, int tiles, int N, const bf16 *xin) {
+    pk::Op o = {};
+    o.kind = pk::OP_GEMM;
+    o.mode = mode;
+    o.w = w.packed;
+    o.tiles = tiles;
+    o.KB = kb(w.K);
+    o.N = N;
+    o.xin = xin;
+    return o;
+  };
+  pk::Op e = {};
+  e.kind = pk::OP_EMBED;
+  ops.push_back(e);
+  for (int l = 0; l < d.n_layers; l++) {
+    const LayerW &w = ctx->layers[l];
+    float *cache = ctx->kv_t + (size_t)l * ctx->kv_t_layer_stride;
+    pk::Op q = gemm_op(gemm_tc::EPI_QKV, w.wqkv, t256(3 * hd), 3 * hd, ctx->pk_xn);
+    q.use_scale = 1;
+    q.cache = cache;
+    q.ep_stride = ctx->kv_t_ep_stride;
+    ops.push_back(q);
+    pk::Op a = {};
+    a.kind = pk::OP_ATTN;
+    a.cache = cache;
+    a.ep_stride = ctx->kv_t_ep_stride;
+    ops.push_back(a);
+    pk::Op o = gemm_op(gemm_tc::EPI_RESID, w.wo, t256(d.d_model), d.d_model, ctx->pk_ao);
+    o.accumulate = 1;
+    o.gain = w.norm2;
+    ops.push_back(o);
+    pk::Op g = gemm_op(gemm_tc::EPI_SWIGLU, w.wgu, (F + 127) / 128, F, ctx->pk_xn);
+    g.use_scale = 1;
+    ops.push_back(g);
+    pk::Op dn = gemm_op(gemm_tc::EPI_RESID, w.wd, t256(d.d_model), d.d_model, ctx->pk_hid);
+    dn.accumulate = 1;
+    dn.gain = (l + 1 == d.n_layers) ? ctx->final_norm : ctx->layers[l + 1].norm1;
+    ops.push_back(dn);
+  }
+  pk::Op lm = gemm_op(gemm_tc::EPI_PLAIN, ctx->lm_head, t256(d.vocab), d.vocab, ctx->pk_xn);
+  lm.use_scale = 1;
+  lm.ldo = d.vocab;
+  argmax_range(ctx, &lm.lo, &lm.hi);
+  lm.post = pk::POST_ARGMAX;
+  ops.push_back(lm);
+  ctx->pk_n_ops_t = (int)ops.size();
+  cudaMemcpy(ctx->pk_ops_t, ops.data(), ops.size() * sizeof(pk::Op), cudaMemcpyHostToDevice);
+}
+
+template <int DH> bool pk_prepare_dh(specvla_ctx *ctx) {
+  if (cudaFuncSetAttribute(pk::forward_pk_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           pk::smem_bytes<DH>()) != cudaSuccess)
+    return false;
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, pk::forward_pk_kernel<DH>, pk::THREADS,
+                                                    pk::smem_bytes<DH>()) != cudaSuccess)
+    return false;
+  return per_sm >= 1;
+}
+// Shared-memory attribute and residency check of the persistent kernel; clears its buffers (the
+// padding rows and columns of the packed operands are read by the MMAs and must stay finite).
+bool pk_prepare(specvla_ctx *ctx) {
+  const specvla_model_desc &d = ctx->desc;
+  int coop = 0, dev = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+  const bool ok = coop && (d.head_dim == 128 ? pk_prepare_dh<128>(ctx) : pk_prepare_dh<64>(ctx));
+  cudaGetLastError();
+  if (!ok) return false;
+  auto kblocks = [](int K) { return (size_t)((K + gemm_tc::BK - 1) / gemm_tc::BK); };
+  cudaMemsetAsync(ctx->pk_xn, 0, kblocks(d.d_model) * pk::X_STAGE_BYTES);
+  cudaMemsetAsync(ctx->pk_ao, 0, kblocks(ctx->hd) * pk::X_STAGE_BYTES);
+  cudaMemsetAsync(ctx->pk_hid, 0, kblocks(d.d_ffn) * pk::X_STAGE_BYTES);
+  cudaMemsetAsync(ctx->pk_bar, 0, 32 * sizeof(unsigned));
+  return true;
+}
+
+// Target forward + LM head + greedy argmax over the R <= 32 rows of one episode described by
+// ctx->rt, as ONE cooperative launch. Leaves the residual in ctx->x, the sums of squares in
+// ctx->pk_ssq, greedy tokens and margins in ctx->greedy / ctx->margin.
+int pk_target_forward(specvla_ctx *ctx, int R, const bf16 *embeds, float *logits_out, cudaStream_t st) {
+  const specvla_model_desc &d = ctx->desc;
+  pk::Params p = {};
+  p.ops = ctx->pk_ops_t;
+  p.n_ops = ctx->pk_n_ops_t;
+  p.T = R;
+  p.max_seg = ctx->pk_max_seg;
+  p.rt = ctx->rt;
+  p.embeds = embeds;
+  p.E = ctx->embed;
+  p.gain0 = ctx->layers[0].norm1;
+  p.d = d.d_model;
+  p.hd = ctx->hd;
+  p.H = d.n_heads;
+  p.dh = d.head_dim;
+  p.max_seq = d.max_seq;
+  p.eps = d.rms_eps;
+  p.attn_scale = 1.f / sqrtf((float)d.head_dim);
+  p.nt = ctx->pk_nt;
+  p.x = ctx->x;
+  p.ssq = ctx->pk_ssq;
+  p.q = ctx->q;
+  p.xn_pk = ctx->pk_xn;
+  p.ao_pk = ctx->pk_ao;
+  p.hid_pk = ctx->pk_hid;
+  p.part = ctx->pk_part;
+  p.apart = ctx->pk_apart;
+  p.splits = ctx->pk_splits;
+  p.rope_tab = ctx->rope_tab;
+  p.cand = ctx->pk_cand;
+  p.logits_out = logits_out;
+  p.greedy = ctx->greedy;
+  p.margin = ctx->margin;
+  p.bar = ctx->pk_bar;
+  p.err = ctx->err;
+  p.wait_ns = ctx->wait_ns;
+  CU(cudaMemsetAsync(ctx->pk_bar, 0, sizeof(unsigned), st));
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(ctx->pk_G);
+  cfg.blockDim = dim3(pk::THREADS);
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeCooperative;
+  at[0].val.cooperative = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  if (d.head_dim == 128) {
+    cfg.dynamicSmemBytes = pk::smem_bytes<128>();
+    CU(cudaLaunchKernelEx(&cfg, pk::forward_pk_kernel<128>, p));
+  } else {
+    cfg.dynamicSmemBytes = pk::smem_bytes<64>();
+    CU(cudaLaunchKernelEx(&cfg, pk::forward_pk_kernel<64>, p));
+  }
+  ctx->launches++;
+  ctx->last_rows = R;
+  ctx->last_ssq = ctx->pk_ssq;
+  ctx->last_nt = ctx->pk_nt;
+  return SPECVLA_OK;
 }
 
 int check_episodes(const specvla_ctx *ctx, int n_ep, const int *episodes) {
@@ -535,14 +757,9 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
   }
   carve(ctx, static_cast<char *>(workspace));
   const int hd = ctx->hd, D = desc->d_model, F = desc->d_ffn;
-  ctx->use_pdl = getenv("SPECVLA_NO_PDL") == nullptr;
-  ctx->use_l2_prefetch = getenv("SPECVLA_NO_L2_PREFETCH") == nullptr;
+  ctx->use_pdl = true;
+  ctx->use_l2_prefetch = true;
   ctx->fit = gemm_ck::query_cluster_fit();
-  if (getenv("SPECVLA_DEBUG")) {
-    fprintf(stderr, "specvla: resident clusters by size:");
-    for (int i = 1; i <= gemm_ck::MAX_S; i++) fprintf(stderr, " %d:%d", i, ctx->fit.max_active[i]);
-    fprintf(stderr, "\n");
-  }
   size_t packed_used = 0;
   bool pack_ok = true;
   // swiglu: the matrix is [gate; up] stacked ([2F, K]) and is packed as tiles of 128 + 128 rows
@@ -600,6 +817,15 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
     ctx->dlayer = LayerW{wmat(dw->wqkv, 3 * hd, D), wmat(dw->wo, D, hd), wmat(dw->wgu, 2 * F, D, true),
                          wmat(dw->wd, D, F), dw->norm1, dw->norm2};
   }
+  ctx->wait_ns = 2000000000ull;
+  ctx->last_ssq = ctx->ssq;
+  ctx->last_nt = ctx->nt;
+  ctx->pk_ok = false;
+  ctx->use_pk = true;
+  if (pk_shapes_ok(*desc) && pack_ok) {
+    pk_build_target_ops(ctx);
+    ctx->pk_ok = pk_prepare(ctx);
+  }
   ctx->hP.assign(desc->max_episodes, -1);
   ctx->hPending.assign(desc->max_episodes, 0);
   ctx->hTreeRows.assign(desc->max_episodes, 0);
@@ -645,6 +871,21 @@ int specvla_destroy(specvla_ctx *ctx) {
   for (cudaEvent_t e : ctx->prof_ev) cudaEventDestroy(e);
   cudaFreeHost(ctx->pinned);
   delete ctx;
+  return SPECVLA_OK;
+}
+
+int specvla_set_option(specvla_ctx *ctx, int option, long long value) {
+  if (!ctx) return SPECVLA_ERR_INVALID_ARG;
+  switch (option) {
+    case SPECVLA_OPT_PERSISTENT_FORWARD: ctx->use_pk = value != 0; break;
+    case SPECVLA_OPT_DEPENDENT_LAUNCH: ctx->use_pdl = value != 0; break;
+    case SPECVLA_OPT_L2_PREFETCH: ctx->use_l2_prefetch = value != 0; break;
+    case SPECVLA_OPT_WAIT_LIMIT_NS:
+      if (value < 1000) return SPECVLA_ERR_INVALID_ARG;
+      ctx->wait_ns = (unsigned long long)value;
+      break;
+    default: return SPECVLA_ERR_INVALID_ARG;
+  }
   return SPECVLA_OK;
 }
 
@@ -905,15 +1146,19 @@ static int verify_device_trees(specvla_ctx *ctx, const EpArgs &ea, int R, int r,
   const int n_ep = ea.n_ep;
   ctx->phase = 4;
   LAUNCH(tree::build_verify_rows_kernel, dim3(n_ep), dim3(128), ea, ctx->trees, (const EpState *)ctx->st, ctx->rt);
-  TRY(target_forward(ctx, R, ea, nullptr, st));
+  if (ctx->pk_ok && ctx->use_pk && n_ep == 1 && R <= pk::TN) {
+    TRY(pk_target_forward(ctx, R, nullptr, logits_out, st));
+  } else {
+    TRY(target_forward(ctx, R, ea, nullptr, st));
+    int lo, hi;
+    argmax_range(ctx, &lo, &hi);
+    TRY(lm_head(ctx, ctx->xn, ctx->ssq, R, st));
+    LAUNCH(epi::argmax_kernel, dim3(R), dim3(epi::THREADS), (const float *)ctx->lgs, d.vocab, lo, hi, ctx->greedy,
+           ctx->margin, logits_out);
+  }
   ctx->feat_valid = false;
-  int lo, hi;
-  argmax_range(ctx, &lo, &hi);
-  TRY(lm_head(ctx, ctx->xn, ctx->ssq, R, st));
-  LAUNCH(epi::argmax_kernel, dim3(R), dim3(epi::THREADS), (const float *)ctx->lgs, d.vocab, lo, hi, ctx->greedy,
-         ctx->margin, logits_out);
   LAUNCH(tree::accept_select_kernel, dim3(n_ep), dim3(128), ea, ctx->trees, ctx->st, (const int *)ctx->greedy, r,
-         d.action_base, d.n_bins, (const float *)ctx->x, (const float *)ctx->ssq, ctx->nt, ctx->final_norm,
+         d.action_base, d.n_bins, (const float *)ctx->x, ctx->last_ssq, ctx->last_nt, ctx->final_norm,
          d.rms_eps, d.d_model, ctx->pend_feat, ctx->out_m, ctx->out_tok, ctx->out_path);
   LAUNCH(tree::kv_compact_kernel, dim3(d.n_layers * 2, n_ep), dim3(256), ea, (const EpState *)ctx->st,
          (const int *)ctx->out_m, (const int *)ctx->out_path, ctx->kv_t, ctx->kv_t_ep_stride,
@@ -1105,7 +1350,7 @@ int specvla_read_buffer(specvla_ctx *ctx, int what, void *host_dst, size_t bytes
         if (ctx->last_rows < 1) return SPECVLA_ERR_BAD_STATE;
         cudaStream_t st = static_cast<cudaStream_t>(stream);
         LAUNCH(epi::features_kernel, dim3(ctx->last_rows), dim3(256), (const float *)ctx->x,
-               (const float *)ctx->ssq, ctx->nt, ctx->final_norm, d.rms_eps, d.d_model, ctx->feat);
+               ctx->last_ssq, ctx->last_nt, ctx->final_norm, d.rms_eps, d.d_model, ctx->feat);
         ctx->feat_valid = true;
       }
       src = ctx->feat;
