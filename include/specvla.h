@@ -134,11 +134,13 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *target
                    specvla_ctx **out);
 int specvla_destroy(specvla_ctx *ctx);
 
-/* Execution options of a context (all default to the fastest setting; they exist for A/B
- * measurements and tests, and change no result beyond rounding order):
+/* Execution options of a context (each defaults to the setting measured fastest on B200; they
+ * exist for A/B measurements and tests, and change no result beyond rounding order):
  *   SPECVLA_OPT_PERSISTENT_FORWARD  1: forwards of one episode and at most 32 rows (the batch-1
  *       verification step of Algorithm 1, an autoregressive step) run as ONE cooperative kernel
- *       whose weight stream continues across all GEMMs of all layers; 0: one launch per GEMM.
+ *       whose weight stream continues across all GEMMs of all layers; 0 (default): one launch per
+ *       GEMM. The persistent kernel needs two grid-wide barriers per GEMM at about 2 us each and
+ *       measures 25 % slower than the per-GEMM path on the 7B-shaped model.
  *   SPECVLA_OPT_DEPENDENT_LAUNCH    1: kernels of the per-GEMM path are launched with programmatic
  *       stream serialisation (a GEMM streams weights while its predecessor drains).
  *   SPECVLA_OPT_L2_PREFETCH         1: a GEMM of the per-GEMM path prefetches the head of the next

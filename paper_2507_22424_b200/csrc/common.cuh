@@ -56,6 +56,7 @@ struct DevTree {
   int tok[SV_MAX_CAND], parent[SV_MAX_CAND], depth[SV_MAX_CAND];
   float score[SV_MAX_CAND];
   int drow[SV_MAX_CAND];          // draft row that scored the node's children (-1: none)
+  int xrow[SV_MAX_CAND];          // row of the draft forward that ran the node (its output feeds its children)
   uint32_t dmask[SV_MAX_TREE][4]; // ancestors-and-self over draft rows (draft mask), by draft row
 };
 
@@ -101,3 +102,40 @@ __device__ __forceinline__ float warp_max(float v) {
   for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
   return v;
 }
+
+// Running (top-1 value, its index, top-2 value) of a set of values; ties go to the lowest index.
+namespace sv {
+struct Top2 {
+  float v1, v2;
+  int i1;
+};
+__device__ __forceinline__ void top2_push(Top2 &a, float v, int i) {
+  if (v > a.v1 || (v == a.v1 && i < a.i1)) {
+    a.v2 = a.v1;
+    a.v1 = v;
+    a.i1 = i;
+  } else if (v > a.v2) {
+    a.v2 = v;
+  }
+}
+__device__ __forceinline__ void top2_merge(Top2 &a, const Top2 &b) {
+  if (b.v1 > a.v1 || (b.v1 == a.v1 && b.i1 < a.i1)) {
+    a.v2 = fmaxf(a.v1, b.v2);
+    a.v1 = b.v1;
+    a.i1 = b.i1;
+  } else {
+    a.v2 = fmaxf(a.v2, b.v1);
+  }
+}
+
+__device__ __forceinline__ void top2_warp(Top2 &b) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    Top2 other;
+    other.v1 = __shfl_xor_sync(0xffffffffu, b.v1, o);
+    other.v2 = __shfl_xor_sync(0xffffffffu, b.v2, o);
+    other.i1 = __shfl_xor_sync(0xffffffffu, b.i1, o);
+    top2_merge(b, other);
+  }
+}
+}  // namespace sv

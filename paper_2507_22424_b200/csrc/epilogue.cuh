@@ -119,28 +119,10 @@ __global__ void split_limbs_kernel(const float *__restrict__ x, size_t n, bf16 *
   if (i < n) store2(out, n, i, x[i]);
 }
 
-struct Top2 {
-  float v1, v2;
-  int i1;
-};
-__device__ __forceinline__ void top2_push(Top2 &a, float v, int i) {
-  if (v > a.v1 || (v == a.v1 && i < a.i1)) {
-    a.v2 = a.v1;
-    a.v1 = v;
-    a.i1 = i;
-  } else if (v > a.v2) {
-    a.v2 = v;
-  }
-}
-__device__ __forceinline__ void top2_merge(Top2 &a, const Top2 &b) {
-  if (b.v1 > a.v1 || (b.v1 == a.v1 && b.i1 < a.i1)) {
-    a.v2 = fmaxf(a.v1, b.v2);
-    a.v1 = b.v1;
-    a.i1 = b.i1;
-  } else {
-    a.v2 = fmaxf(a.v2, b.v1);
-  }
-}
+using sv::Top2;
+using sv::top2_push;
+using sv::top2_merge;
+using sv::top2_warp;
 
 // Greedy token per row of logits [T][V]: argmax over [lo, hi) with ties to the lowest id;
 // margin = top-1 minus top-2 over the same range. Optionally copies the whole row out.
@@ -168,6 +150,29 @@ argmax_kernel(const float *__restrict__ logits, int V, int lo, int hi, int *__re
   __syncthreads();
   if (threadIdx.x == 0) {
     for (int w = 1; w < THREADS / 32; w++) top2_merge(best, red[w]);
+    greedy[t] = best.i1;
+    margin[t] = best.v1 - best.v2;
+  }
+}
+
+// Greedy token per row from the candidates a GEMM epilogue left: cand[row][0..nc) holds the top-2
+// of each 128-column group of the row's logits (value, column as int bits, second value). One
+// warp per row; ties go to the lowest id; margin = top-1 minus top-2.
+__global__ void __launch_bounds__(128)
+argmax_merge_kernel(const float4 *__restrict__ cand, int nc, int rows, int *__restrict__ greedy,
+                    float *__restrict__ margin) {
+  pdl_launch();
+  pdl_wait();
+  const int t = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (t >= rows) return;
+  Top2 best{-INFINITY, -INFINITY, 0x7fffffff};
+  for (int i = lane; i < nc; i += 32) {
+    const float4 c = cand[(size_t)t * nc + i];
+    const Top2 other{c.x, c.z, __float_as_int(c.y)};
+    top2_merge(best, other);
+  }
+  top2_warp(best);
+  if (lane == 0) {
     greedy[t] = best.i1;
     margin[t] = best.v1 - best.v2;
   }

@@ -14,9 +14,8 @@
 //    the matrix shape.
 //  * A producer thread issues those bulk copies into a four-stage shared-memory ring, matrix
 //    after matrix, with no dependency on the computation: it runs ahead of the MMAs as far as the
-//    ring allows, and asks for the units further ahead to be brought into L2
-//    (cp.async.bulk.prefetch.L2), so HBM keeps working while the tensor cores wait for the
-//    activations of the next matrix.
+//    ring allows, so the first stages of the next matrix are already on the SM when its
+//    activations become available.
 //  * The activation operand (both bf16 limbs of up to 32 rows) is kept in global memory in the
 //    same K-block-major, pre-swizzled form (8 KB per K block), written by the epilogue of the
 //    phase that produces it and fetched per stage by a second loader thread once that phase is
@@ -54,7 +53,6 @@ constexpr int ACC_COLS = 2 * TN;                    // accumulator columns of on
 constexpr int TMEM_COLS = 4 * ACC_COLS;             // two buffers x two halves
 constexpr int PART_ELEMS = TN * BM;                 // fp32 elements of one partial tile
 constexpr int MAX_SPLITS = 8;
-constexpr int PF_DISTANCE = 12;                     // units the L2 prefetch runs ahead of the ring
 
 #define SV_ERR_WAIT_GRID 5
 #define SV_ERR_WAIT_XREADY 6
@@ -112,10 +110,11 @@ struct Params {
 };
 
 // ------------------------------------------------------------------------- small helpers
-__device__ __forceinline__ int ubegin(int U, int c, int G) { return (int)((long long)U * c / G); }
+// First unit of CTA c when U units are dealt out to G CTAs (U * G < 2^31, checked by the host).
+__device__ __forceinline__ int ubegin(int U, int c, int G) { return (int)((unsigned)U * (unsigned)c / (unsigned)G); }
 // the CTA whose range holds unit u
 __device__ __forceinline__ int uowner(int U, int u, int G) {
-  int c = (int)(((long long)u * G) / U);
+  int c = (int)(((unsigned)u * (unsigned)G) / (unsigned)U);
   while (c + 1 < G && ubegin(U, c + 1, G) <= u) c++;
   while (c > 0 && ubegin(U, c, G) > u) c--;
   return c;
@@ -157,16 +156,7 @@ __device__ __forceinline__ void store_limbs4_pk(bf16 *buf, int t, int k, float4 
   store_bf16x4(buf + o + TN * BK, make_float4(v.x - h.x, v.y - h.y, v.z - h.z, v.w - h.w));
 }
 
-__device__ __forceinline__ void top2_warp(epi::Top2 &b) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    epi::Top2 other;
-    other.v1 = __shfl_xor_sync(0xffffffffu, b.v1, o);
-    other.v2 = __shfl_xor_sync(0xffffffffu, b.v2, o);
-    other.i1 = __shfl_xor_sync(0xffffffffu, b.i1, o);
-    epi::top2_merge(b, other);
-  }
-}
+using sv::top2_warp;
 
 // Shared state of one CTA.
 struct Cta {
@@ -178,14 +168,15 @@ struct Cta {
 // ------------------------------------------------------------------------- grid barrier
 // All 256 epilogue threads of every CTA call this the same number of times. `epoch` counts calls.
 __device__ __forceinline__ bool grid_barrier(const Params &p, int G, unsigned &epoch, int et, volatile int *s_ok) {
-  // what this thread wrote is about to be read by other CTAs, partly through bulk copies (async proxy)
+  // what this thread wrote is about to be read by other CTAs, partly through bulk copies (async
+  // proxy). The CTA barrier orders every thread's writes before the elected thread's fence, which
+  // is cumulative; its counterpart after the wait covers the reads of all threads.
   asm volatile("fence.proxy.async.global;" ::: "memory");
-  __threadfence();
   epi_sync();
   if (et == 0) {
     epoch++;
     __threadfence();
-    atomicAdd(p.bar, 1u);
+    asm volatile("red.relaxed.gpu.global.add.u32 [%0], 1;" ::"l"(p.bar) : "memory");
     const unsigned target = epoch * (unsigned)G;
     bool ok = true;
     if (ld_acquire(p.bar) < target) {
@@ -439,6 +430,181 @@ __device__ void attention_unit(const Params &p, const Op &op, unsigned char *sme
   }
 }
 
+// ------------------------------------------------------------------------- finishing a GEMM phase
+constexpr int MAX_G = 192;                          // CTAs the unit tables are sized for
+constexpr int MAX_TILES = 512;                      // output tiles of one matrix
+
+struct RowInfo {
+  const float *scale;          // RMSNorm scale per row (shared memory)
+  const int *pos, *slot, *ep;  // RoPE position, cache slot, episode per row (shared memory)
+  const int *begin;            // first unit of every CTA in this phase, [G + 1] (shared memory)
+  const unsigned short *cf, *cl;   // first and last CTA that hold units of each output tile (shared memory)
+};
+
+// What remains of a GEMM phase once every CTA's partial tiles are in global scratch: work items of
+// one row x 128 output columns (SwiGLU: 128 gate + 128 up columns) are dealt out to the epilogue
+// warps of the whole grid; a warp sums the item's partial tiles in CTA order (deterministic) and
+// applies the phase's epilogue. IB items are handled together, the first NB partial tiles of each
+// loaded in one round before anything is used (loads from L2 take a microsecond: a warp that
+// waited for each in turn would need several). A tile shared by more CTAs takes further rounds.
+template <int MODE, int IB, int NB>
+__device__ __forceinline__ void finish_phase(const Params &p, const Op &o, const RowInfo &ri, int T, int G,
+                                             int gw, int GW, int lane) {
+  constexpr bool SW = MODE == EPI_SWIGLU;
+  constexpr int halves = SW ? 1 : 2;
+  const int n_items = o.tiles * T * halves;
+  const int colbase = lane * 4;
+  for (int base = gw; base < n_items; base += GW * IB) {
+    int jj[IB], tt[IB], hh[IB], cfs[IB], cls[IB];
+    float4 a[IB][NB], b[IB][SW ? NB : 1];
+    // operands that do not depend on the partial tiles: residual and gain (EPI_RESID), RoPE factors
+    // (EPI_QKV), requested in the same round
+    float4 ex0[IB], ex1[IB];
+    // round 1 of every item
+#pragma unroll
+    for (int k = 0; k < IB; k++) {
+      const int item = base + k * GW;
+      jj[k] = -1;
+      if (item < n_items) {
+        const int j = item / (T * halves);
+        const int rem = item - j * (T * halves);
+        jj[k] = j;
+        tt[k] = rem / halves;
+        hh[k] = rem - tt[k] * halves;
+        cfs[k] = ri.cf[j];
+        cls[k] = ri.cl[j];
+        const int n = j * BM + hh[k] * 128 + colbase;
+        ex0[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        ex1[k] = make_float4(1.f, 1.f, 1.f, 1.f);
+        if (MODE == EPI_RESID && n < o.N) {
+          if (o.accumulate) ex0[k] = __ldcg(reinterpret_cast<const float4 *>(p.x + (size_t)tt[k] * o.N + n));
+          if (o.gain) ex1[k] = *reinterpret_cast<const float4 *>(o.gain + n);
+        }
+        if (MODE == EPI_QKV) {
+          const int which = n / p.hd, jq = (n - which * p.hd) & (p.dh - 1), half = p.dh >> 1;
+          if (which < 2) {
+            const float2 *cs = p.rope_tab + (size_t)ri.pos[tt[k]] * half + (jq < half ? jq : jq - half);
+            ex0[k] = *reinterpret_cast<const float4 *>(cs);
+            ex1[k] = *reinterpret_cast<const float4 *>(cs + 2);
+          }
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < NB; i++) {
+        a[k][i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (SW) b[k][i] = a[k][i];
+        if (jj[k] >= 0 && cfs[k] + i <= cls[k]) {
+          const int cc = cfs[k] + i;
+          const int cb = ri.begin[cc];
+          if (cb != ri.begin[cc + 1]) {                                 // a CTA without units adds nothing
+            // only the first CTA of a tile can have begun in an earlier tile
+            const int seg = i == 0 ? jj[k] - cb / o.KB : 0;
+            const float *src = p.part + (((size_t)cc * p.max_seg + seg) * TN + tt[k]) * BM + hh[k] * 128 + colbase;
+            a[k][i] = __ldcg(reinterpret_cast<const float4 *>(src));
+            if (SW) b[k][i] = __ldcg(reinterpret_cast<const float4 *>(src + 128));
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < IB; k++) {
+      if (jj[k] < 0) continue;
+      const int j = jj[k], t = tt[k], hf = hh[k];
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f), v2 = v;
+#pragma unroll
+      for (int i = 0; i < NB; i++) {
+        v.x += a[k][i].x; v.y += a[k][i].y; v.z += a[k][i].z; v.w += a[k][i].w;
+        if (SW) { v2.x += b[k][i].x; v2.y += b[k][i].y; v2.z += b[k][i].z; v2.w += b[k][i].w; }
+      }
+      // further rounds (tiles shared by more than NB CTAs)
+      for (int c0 = cfs[k] + NB; c0 <= cls[k]; c0 += NB) {
+        float4 e[NB], f[SW ? NB : 1];
+#pragma unroll
+        for (int i = 0; i < NB; i++) {
+          e[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (SW) f[i] = e[i];
+          const int cc = c0 + i;
+          if (cc <= cls[k] && ri.begin[cc] != ri.begin[cc + 1]) {
+            const float *src = p.part + (((size_t)cc * p.max_seg) * TN + t) * BM + hf * 128 + colbase;
+            e[i] = __ldcg(reinterpret_cast<const float4 *>(src));
+            if (SW) f[i] = __ldcg(reinterpret_cast<const float4 *>(src + 128));
+          }
+        }
+#pragma unroll
+        for (int i = 0; i < NB; i++) {
+          v.x += e[i].x; v.y += e[i].y; v.z += e[i].z; v.w += e[i].w;
+          if (SW) { v2.x += f[i].x; v2.y += f[i].y; v2.z += f[i].z; v2.w += f[i].w; }
+        }
+      }
+      const float sc = o.use_scale ? ri.scale[t] : 1.f;
+      const int col = hf * 128 + colbase;                  // first of this lane's four columns within the tile
+      if (MODE == EPI_QKV) {
+        const int n = j * BM + col;
+        const int which = n / p.hd, cq = n - which * p.hd;
+        const int half = p.dh >> 1, jq = cq & (p.dh - 1);
+        const bool lo = jq < half;
+        float4 ov = make_float4(sc * v.x, sc * v.y, sc * v.z, sc * v.w);
+        // the rotation partner (dh / 2 columns away) sits dh / 8 lanes away in the same warp
+        const int dl = p.dh >> 3;
+        const float wx = __shfl_xor_sync(0xffffffffu, ov.x, dl), wy = __shfl_xor_sync(0xffffffffu, ov.y, dl);
+        const float wz = __shfl_xor_sync(0xffffffffu, ov.z, dl), ww = __shfl_xor_sync(0xffffffffu, ov.w, dl);
+        if (which < 2) {
+          const float4 cs01 = ex0[k], cs23 = ex1[k];
+          const float sg = lo ? -1.f : 1.f;
+          ov.x = ov.x * cs01.x + sg * wx * cs01.y;
+          ov.y = ov.y * cs01.z + sg * wy * cs01.w;
+          ov.z = ov.z * cs23.x + sg * wz * cs23.y;
+          ov.w = ov.w * cs23.z + sg * ww * cs23.w;
+        }
+        if (n < o.N) {
+          float *dst = which == 0 ? p.q + (size_t)t * p.hd + cq
+                                  : o.cache + (size_t)ri.ep[t] * o.ep_stride +
+                                        ((size_t)(which - 1) * p.max_seq + ri.slot[t]) * p.hd + cq;
+          *reinterpret_cast<float4 *>(dst) = ov;
+        }
+      } else if (SW) {
+        const int n = j * 128 + col;
+        if (n < o.N) {
+          const float gx = sc * v.x, gy = sc * v.y, gz = sc * v.z, gw2 = sc * v.w;
+          store_limbs4_pk(p.hid_pk, t, n,
+                          make_float4(__fdividef(gx, 1.f + __expf(-gx)) * (sc * v2.x),
+                                      __fdividef(gy, 1.f + __expf(-gy)) * (sc * v2.y),
+                                      __fdividef(gz, 1.f + __expf(-gz)) * (sc * v2.z),
+                                      __fdividef(gw2, 1.f + __expf(-gw2)) * (sc * v2.w)));
+        }
+      } else if (MODE == EPI_RESID) {
+        const int n = j * BM + col;
+        float s2 = 0.f;
+        if (n < o.N) {
+          float *xp = p.x + (size_t)t * o.N + n;
+          const float4 xo = ex0[k], g = ex1[k];
+          v.x += xo.x; v.y += xo.y; v.z += xo.z; v.w += xo.w;
+          *reinterpret_cast<float4 *>(xp) = v;
+          store_limbs4_pk(p.xn_pk, t, n, make_float4(v.x * g.x, v.y * g.y, v.z * g.z, v.w * g.w));
+          s2 = (v.x * v.x + v.y * v.y) + (v.z * v.z + v.w * v.w);
+        }
+        s2 = warp_sum(s2);
+        if (lane == 0 && j * 2 + hf < p.nt) p.ssq[t * p.nt + j * 2 + hf] = s2;
+      } else {
+        // EPI_PLAIN: logits of 128 columns; their top-2 over [lo, hi) for the argmax
+        const int n = j * BM + col;
+        const float4 ov = make_float4(sc * v.x, sc * v.y, sc * v.z, sc * v.w);
+        float *outp = o.post == POST_ARGMAX ? p.logits_out : o.out;
+        if (outp && n < o.N) *reinterpret_cast<float4 *>(outp + (size_t)t * o.ldo + n) = ov;
+        if (o.post == POST_ARGMAX) {
+          epi::Top2 bb{-INFINITY, -INFINITY, 0x7fffffff};
+          const float vv[4] = {ov.x, ov.y, ov.z, ov.w};
+#pragma unroll
+          for (int e2 = 0; e2 < 4; e2++)
+            if (n + e2 >= o.lo && n + e2 < o.hi) epi::top2_push(bb, vv[e2], n + e2);
+          top2_warp(bb);
+          if (lane == 0) p.cand[(size_t)t * (2 * o.tiles) + j * 2 + hf] = make_float4(bb.v1, __int_as_float(bb.i1), bb.v2, 0.f);
+        }
+      }
+    }
+  }
+}
+
 template <int DH> __host__ __device__ constexpr int attn_smem_bytes() {
   return (2 * (32 + 2 * 32) * (DH + 8) + 2 * 32 * (32 + 8)) * (int)sizeof(bf16) + 32 * (32 + 4) * (int)sizeof(float);
 }
@@ -459,6 +625,10 @@ __global__ void __launch_bounds__(THREADS, 1) forward_pk_kernel(const __grid_con
   const uint32_t xready_bar = bars + 8u * (2 * STAGES + 4);
   const uint32_t tmem_slot = bars + 8u * (2 * STAGES + 5);
   __shared__ int s_ok, s_gok;              // results of bounded waits, shared by the epilogue threads
+  __shared__ int s_begin[MAX_G + 1];       // first unit of every CTA in the GEMM phase being run
+  __shared__ unsigned short s_cf[MAX_TILES], s_cl[MAX_TILES];   // CTAs that share each of its output tiles
+  __shared__ float s_scale[TN];            // RMSNorm scale of each row for the phase being finished
+  __shared__ int s_pos[TN], s_slot[TN], s_ep[TN];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int c = blockIdx.x, G = gridDim.x;
@@ -491,23 +661,6 @@ __global__ void __launch_bounds__(THREADS, 1) forward_pk_kernel(const __grid_con
     // ---------------------------------------------------------------- weight producer
     if (lane == 0) {
       const uint64_t pol_w = policy_evict_first();
-      // prefetch cursor: PF_DISTANCE units ahead of the load cursor in this CTA's unit sequence
-      int pop = 0, pu = 0, pe = 0;
-      const bf16 *pw = nullptr;
-      auto pf_step = [&]() {
-        while (pu >= pe) {
-          if (pop >= p.n_ops) return;
-          const Op &o = p.ops[pop++];
-          if (o.kind != OP_GEMM) continue;
-          const int U = o.tiles * o.KB;
-          pu = ubegin(U, c, G);
-          pe = ubegin(U, c + 1, G);
-          pw = o.w;
-        }
-        prefetch_l2(pw + (size_t)pu * (BM * BK), W_STAGE_BYTES);
-        pu++;
-      };
-      for (int i = 0; i < PF_DISTANCE; i++) pf_step();
       uint32_t it = 0;
       bool ok = true;
       for (int oi = 0; oi < p.n_ops && ok; oi++) {
@@ -526,7 +679,6 @@ __global__ void __launch_bounds__(THREADS, 1) forward_pk_kernel(const __grid_con
           }
           mbar_expect_tx(full_bar(st), W_STAGE_BYTES);
           bulk_load(ring + st * STAGE_BYTES, w + (size_t)u * (BM * BK), W_STAGE_BYTES, full_bar(st), pol_w);
-          pf_step();
         }
       }
     }
@@ -622,8 +774,15 @@ __global__ void __launch_bounds__(THREADS, 1) forward_pk_kernel(const __grid_con
     unsigned epoch = 0;
     uint32_t segc = 0;
     bool alive = true;
+    if (et < TN) {
+      const bool in = et < T;
+      s_pos[et] = in ? p.rt.pos[et] : 0;
+      s_slot[et] = in ? p.rt.slot[et] : 0;
+      s_ep[et] = in ? p.rt.ep[et] : 0;
+    }
+    epi_sync();
     for (int oi = 0; oi < p.n_ops && alive; oi++) {
-      const Op &o = p.ops[oi];
+      const Op o = p.ops[oi];                        // a private copy: the fields are used after fences
       if (o.kind == OP_EMBED) {
         // x = input rows; xn = limbs(x * gain0) packed; ssq per 128 columns
         for (int item = gw; item < T * p.nt; item += GW) {
@@ -697,6 +856,23 @@ __global__ void __launch_bounds__(THREADS, 1) forward_pk_kernel(const __grid_con
       }
       // -------------------------------------------------------------- GEMM phase
       if (et == 0) mbar_arrive(xready_bar);          // everything before this phase is complete
+      // unit tables of this phase (the finishing code would otherwise divide its time away)
+      const int U0 = o.tiles * o.KB;
+      for (int i = et; i <= G; i += EPI_THREADS) s_begin[i] = ubegin(U0, i, G);
+      for (int j = et; j < o.tiles; j += EPI_THREADS) {
+        s_cf[j] = (unsigned short)uowner(U0, j * o.KB, G);
+        s_cl[j] = (unsigned short)uowner(U0, (j + 1) * o.KB - 1, G);
+      }
+      if (o.use_scale) {
+        // RMSNorm scales of the rows (their sums of squares are complete), once per CTA, while the
+        // MMAs run; read after the grid barrier below
+        for (int t = ew; t < T; t += 8) {
+          float ss = 0.f;
+          for (int i = lane; i < p.nt; i += 32) ss += __ldcg(p.ssq + t * p.nt + i);
+          ss = warp_sum(ss);
+          if (lane == 0) s_scale[t] = rsqrtf(ss / (float)p.d + p.eps);
+        }
+      }
       const int U = o.tiles * o.KB;
       const int ub = ubegin(U, c, G), ue = ubegin(U, c + 1, G);
       // part 1: each finished accumulator -> fp32 partial tile [t][256] in global scratch
@@ -740,104 +916,12 @@ __global__ void __launch_bounds__(THREADS, 1) forward_pk_kernel(const __grid_con
       }
       if (!grid_barrier(p, G, epoch, et, &s_gok)) break;
       // part 2: sum the partial tiles of every output tile in CTA order and finish
-      const bool swiglu = o.mode == EPI_SWIGLU;
-      const int halves = swiglu ? 1 : 2;
-      const int n_items = o.tiles * T * halves;
-      for (int item = gw; item < n_items; item += GW) {
-        const int j = item / (T * halves);
-        const int rem = item - j * (T * halves);
-        const int t = rem / halves, hf = rem - t * halves;
-        const int cf = uowner(U, j * o.KB, G), cl = uowner(U, (j + 1) * o.KB - 1, G);
-        const int col = swiglu ? lane * 4 : hf * 128 + lane * 4;       // first column within the tile
-        float sc = 1.f;
-        if (o.use_scale) {
-          float ss = 0.f;
-          for (int i = lane; i < p.nt; i += 32) ss += __ldcg(p.ssq + t * p.nt + i);
-          ss = warp_sum(ss);
-          sc = rsqrtf(ss / (float)p.d + p.eps);
-        }
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f), v2 = v;
-        for (int cc = cf; cc <= cl; cc++) {
-          const int cb = ubegin(U, cc, G);
-          if (cb == ubegin(U, cc + 1, G)) continue;                    // a CTA without units
-          const int seg = j - cb / o.KB;
-          const float *src = p.part + (((size_t)cc * p.max_seg + seg) * TN + t) * BM + col;
-          const float4 a = __ldcg(reinterpret_cast<const float4 *>(src));
-          v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w;
-          if (swiglu) {
-            const float4 b = __ldcg(reinterpret_cast<const float4 *>(src + 128));
-            v2.x += b.x; v2.y += b.y; v2.z += b.z; v2.w += b.w;
-          }
-        }
-        if (o.mode == EPI_QKV) {
-          const int n = j * BM + col;
-          const int which = n / p.hd, cq = n - which * p.hd;
-          const int half = p.dh >> 1, jq = cq % p.dh;
-          const bool lo = jq < half;
-          float4 ov = make_float4(sc * v.x, sc * v.y, sc * v.z, sc * v.w);
-          // the rotation partner (dh / 2 columns away) sits dh / 8 lanes away in the same warp
-          const int dl = p.dh >> 3;
-          const float wx = __shfl_xor_sync(0xffffffffu, ov.x, dl), wy = __shfl_xor_sync(0xffffffffu, ov.y, dl);
-          const float wz = __shfl_xor_sync(0xffffffffu, ov.z, dl), ww = __shfl_xor_sync(0xffffffffu, ov.w, dl);
-          if (which < 2) {
-            const float2 *cs = p.rope_tab + (size_t)p.rt.pos[t] * half + (lo ? jq : jq - half);
-            const float4 cs01 = *reinterpret_cast<const float4 *>(cs);
-            const float4 cs23 = *reinterpret_cast<const float4 *>(cs + 2);
-            const float sg = lo ? -1.f : 1.f;
-            ov.x = ov.x * cs01.x + sg * wx * cs01.y;
-            ov.y = ov.y * cs01.z + sg * wy * cs01.w;
-            ov.z = ov.z * cs23.x + sg * wz * cs23.y;
-            ov.w = ov.w * cs23.z + sg * ww * cs23.w;
-          }
-          if (n < o.N) {
-            float *dst = which == 0 ? p.q + (size_t)t * p.hd + cq
-                                    : o.cache + (size_t)p.rt.ep[t] * o.ep_stride +
-                                          ((size_t)(which - 1) * p.max_seq + p.rt.slot[t]) * p.hd + cq;
-            *reinterpret_cast<float4 *>(dst) = ov;
-          }
-        } else if (swiglu) {
-          const int n = j * 128 + col;
-          if (n < o.N) {
-            const float gx = sc * v.x, gy = sc * v.y, gz = sc * v.z, gw2 = sc * v.w;
-            store_limbs4_pk(p.hid_pk, t, n,
-                            make_float4(__fdividef(gx, 1.f + __expf(-gx)) * (sc * v2.x),
-                                        __fdividef(gy, 1.f + __expf(-gy)) * (sc * v2.y),
-                                        __fdividef(gz, 1.f + __expf(-gz)) * (sc * v2.z),
-                                        __fdividef(gw2, 1.f + __expf(-gw2)) * (sc * v2.w)));
-          }
-        } else if (o.mode == EPI_RESID) {
-          const int n = j * BM + col;
-          float s2 = 0.f;
-          if (n < o.N) {
-            float *xp = p.x + (size_t)t * o.N + n;
-            if (o.accumulate) {
-              const float4 xo = __ldcg(reinterpret_cast<const float4 *>(xp));
-              v.x += xo.x; v.y += xo.y; v.z += xo.z; v.w += xo.w;
-            }
-            *reinterpret_cast<float4 *>(xp) = v;
-            float4 g = make_float4(1.f, 1.f, 1.f, 1.f);
-            if (o.gain) g = *reinterpret_cast<const float4 *>(o.gain + n);
-            store_limbs4_pk(p.xn_pk, t, n, make_float4(v.x * g.x, v.y * g.y, v.z * g.z, v.w * g.w));
-            s2 = (v.x * v.x + v.y * v.y) + (v.z * v.z + v.w * v.w);
-          }
-          s2 = warp_sum(s2);
-          if (lane == 0 && j * 2 + hf < p.nt) p.ssq[t * p.nt + j * 2 + hf] = s2;
-        } else {
-          // EPI_PLAIN: logits of 128 columns; their top-2 over [lo, hi) for the argmax / top-k
-          const int n = j * BM + col;
-          const float4 ov = make_float4(sc * v.x, sc * v.y, sc * v.z, sc * v.w);
-          float *outp = o.post == POST_ARGMAX ? p.logits_out : o.out;
-          if (outp && n < o.N) *reinterpret_cast<float4 *>(outp + (size_t)t * o.ldo + n) = ov;
-          if (o.post == POST_ARGMAX) {
-            epi::Top2 b{-INFINITY, -INFINITY, 0x7fffffff};
-            const float vv[4] = {ov.x, ov.y, ov.z, ov.w};
-#pragma unroll
-            for (int e = 0; e < 4; e++)
-              if (n + e >= o.lo && n + e < o.hi) epi::top2_push(b, vv[e], n + e);
-            top2_warp(b);
-            if (lane == 0) p.cand[(size_t)t * (2 * o.tiles) + j * 2 + hf] = make_float4(b.v1, __int_as_float(b.i1), b.v2, 0.f);
-          }
-        }
+      const RowInfo ri{s_scale, s_pos, s_slot, s_ep, s_begin, s_cf, s_cl};
+      switch (o.mode) {
+        case EPI_QKV: finish_phase<EPI_QKV, 2, 6>(p, o, ri, T, G, gw, GW, lane); break;
+        case EPI_SWIGLU: finish_phase<EPI_SWIGLU, 2, 3>(p, o, ri, T, G, gw, GW, lane); break;
+        case EPI_RESID: finish_phase<EPI_RESID, 1, 12>(p, o, ri, T, G, gw, GW, lane); break;
+        default: finish_phase<EPI_PLAIN, 3, 3>(p, o, ri, T, G, gw, GW, lane); break;
       }
       if (!grid_barrier(p, G, epoch, et, &s_gok)) break;
       if (o.post == POST_ARGMAX) {

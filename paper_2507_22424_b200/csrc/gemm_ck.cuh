@@ -4,7 +4,7 @@
 // HBM: there is no need to spread a matrix over all 148 SMs. Every GEMM of the decoder is
 // therefore cut into whole tiles first (LM head: 126 tiles = 126 CTAs, gate/up: 86, each
 // finishing its tile straight from TMEM with the fused epilogue), and only matrices with few
-// tiles are split along K as well: the S (<= 4) CTAs that share a tile form one thread-block
+// tiles are split along K as well: the S (<= 8) CTAs that share a tile form one thread-block
 // cluster, CTA r streams K blocks [r KB / S, (r + 1) KB / S) through the TMA ring / tcgen05
 // pipeline, drops its fp32 partial tile into its own shared memory, and after one cluster
 // barrier every CTA finishes the rows t = r, r + S, ... of the tile, reading the S partials
@@ -47,7 +47,7 @@ __device__ __forceinline__ void cluster_sync_all() {
 }
 __host__ __device__ constexpr int ck_tmem_cols(int TN) { return 2 * acc_width(TN) < 32 ? 32 : 2 * acc_width(TN); }
 
-// EpiArgs as in gemm_tc (EPI_PLAIN or EPI_RESID; part / counters unused). KB = K blocks per tile.
+// EpiArgs as in gemm_tc: the mode is a template parameter. KB = K blocks per tile.
 template <int TN, int MODE>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
@@ -72,6 +72,8 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   __shared__ __align__(16) float2 s_rope[ROPE_ROWS * ROPE_HALF];
   __shared__ float s_red[8][MAX_T];
   __shared__ int s_flag[8];
+  __shared__ float s_xv[4][2];             // EPI_TOPK: exchange between the two warps of a row group
+  __shared__ int s_xi[4][2];
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int S = (int)cluster_size();
@@ -331,8 +333,82 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       const int slot = MODE == EPI_QKV ? s_slot[t] : 0, ep = MODE == EPI_QKV ? s_ep[t] : 0;
       float4 v = partial_sum(t * BM + c4);
       if (MODE == EPI_PLAIN) {
-        if (col_ok)
-          *reinterpret_cast<float4 *>(ea.out + row * ea.ldo + n) = make_float4(sc * v.x, sc * v.y, sc * v.z, sc * v.w);
+        const float4 ov = make_float4(sc * v.x, sc * v.y, sc * v.z, sc * v.w);
+        if (ea.out && col_ok) *reinterpret_cast<float4 *>(ea.out + row * ea.ldo + n) = ov;
+        if (ea.cand) {
+          // greedy argmax, first step: the top-2 of this warp's 128 columns over [lo, hi)
+          sv::Top2 b{-INFINITY, -INFINITY, 0x7fffffff};
+          const float vv[4] = {ov.x, ov.y, ov.z, ov.w};
+#pragma unroll
+          for (int e = 0; e < 4; e++)
+            if (n + e >= ea.lo && n + e < ea.hi && n + e < ea.N) sv::top2_push(b, vv[e], n + e);
+          sv::top2_warp(b);
+          if (lane == 0)
+            ea.cand[row * (size_t)(2 * tiles) + tile * 2 + ((et >> 5) & 1)] = make_float4(b.v1, __int_as_float(b.i1), b.v2, 0.f);
+        }
+      } else if (MODE == EPI_TOPK) {
+        // the row's 256 scores sit in the two warps of this row group, four per thread
+        const int wg = (et >> 5) & 1;
+        const float xv[4] = {sc * v.x, sc * v.y, sc * v.z, sc * v.w};
+        bool in[4];
+#pragma unroll
+        for (int e = 0; e < 4; e++) in[e] = n + e >= ea.lo && n + e < ea.hi && n + e < ea.N;
+        if (ea.out && col_ok) *reinterpret_cast<float4 *>(ea.out + row * ea.ldo + n) = make_float4(xv[0], xv[1], xv[2], xv[3]);
+        auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(2 + rg) : "memory"); };
+        float mx = -INFINITY;
+#pragma unroll
+        for (int e = 0; e < 4; e++)
+          if (in[e]) mx = fmaxf(mx, xv[e]);
+        mx = warp_max(mx);
+        if (lane == 0) s_xv[rg][wg] = mx;
+        pair_sync();
+        mx = fmaxf(s_xv[rg][0], s_xv[rg][1]);
+        pair_sync();
+        float se = 0.f;
+#pragma unroll
+        for (int e = 0; e < 4; e++)
+          if (in[e]) se += expf(xv[e] - mx);
+        se = warp_sum(se);
+        if (lane == 0) s_xv[rg][wg] = se;
+        pair_sync();
+        const float lse = mx + logf(s_xv[rg][0] + s_xv[rg][1]);
+        pair_sync();
+        unsigned taken = 0;
+        for (int k = 0; k < SV_TOPK; k++) {
+          float bv = -INFINITY;
+          int bi = 0x7fffffff;
+#pragma unroll
+          for (int e = 0; e < 4; e++)
+            if (in[e] && !((taken >> e) & 1u) && (xv[e] > bv || (xv[e] == bv && n + e < bi))) {
+              bv = xv[e];
+              bi = n + e;
+            }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (ov > bv || (ov == bv && oi < bi)) {
+              bv = ov;
+              bi = oi;
+            }
+          }
+          if (lane == 0) {
+            s_xv[rg][wg] = bv;
+            s_xi[rg][wg] = bi;
+          }
+          pair_sync();
+          const float v0 = s_xv[rg][0], v1 = s_xv[rg][1];
+          const int i0 = s_xi[rg][0], i1 = s_xi[rg][1];
+          const bool first = v0 > v1 || (v0 == v1 && i0 < i1);
+          bv = first ? v0 : v1;
+          bi = first ? i0 : i1;
+          pair_sync();
+          if (bi >= n && bi < n + 4) taken |= 1u << (bi - n);
+          if ((et & 63) == 0) {
+            ea.top_tok[row * SV_TOPK + k] = bi + ea.tok_offset;
+            ea.top_lp[row * SV_TOPK + k] = bv - lse;
+          }
+        }
       } else if (MODE == EPI_QKV) {
         // the partner columns of the rotation (dh / 2 away) are in the same tile
         float4 o = make_float4(sc * v.x, sc * v.y, sc * v.z, sc * v.w);
@@ -406,13 +482,10 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 template <int TN, int MODE>
 inline cudaError_t launch_tm(const CUtensorMap &tmW, const CUtensorMap &tmX, const CUtensorMap &tmXtail,
                              const EpiArgs &ea, int tiles, int KB, int S, int *err, cudaStream_t st, bool pdl) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_ck_kernel<TN, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         smem_bytes(TN));
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  // per device and cheap: set on every launch, so that every device of the process has it
+  cudaError_t e = cudaFuncSetAttribute(gemm_ck_kernel<TN, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       smem_bytes(TN));
+  if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(tiles * S, (ea.T + MAX_T - 1) / MAX_T);
   cfg.blockDim = dim3(THREADS);
@@ -439,6 +512,7 @@ inline cudaError_t launch_tn(const CUtensorMap &tmW, const CUtensorMap &tmX, con
     case EPI_PLAIN: return launch_tm<TN, EPI_PLAIN>(tmW, tmX, tmXtail, ea, tiles, KB, S, err, st, pdl);
     case EPI_RESID: return launch_tm<TN, EPI_RESID>(tmW, tmX, tmXtail, ea, tiles, KB, S, err, st, pdl);
     case EPI_SWIGLU: return launch_tm<TN, EPI_SWIGLU>(tmW, tmX, tmXtail, ea, tiles, KB, S, err, st, pdl);
+    case EPI_TOPK: return launch_tm<TN, EPI_TOPK>(tmW, tmX, tmXtail, ea, tiles, KB, S, err, st, pdl);
     default: return launch_tm<TN, EPI_QKV>(tmW, tmX, tmXtail, ea, tiles, KB, S, err, st, pdl);
   }
 }

@@ -8,7 +8,7 @@
 //  * W [N, K] (bf16, K contiguous) is cut into tiles of 256 rows x 64 columns (32 KB, 128-byte
 //    swizzle). A tile sits on the MMA's M axis (two M = 128 halves), the activation rows on its
 //    N axis (TN = T rounded up to 16/32/64/128). Both bf16 limbs of X are multiplied against
-//    the same W tile (as one operand of 2 TN rows up to TN = 64), so fp32-grade activations
+//    the same W tile (as one operand of 2 TN rows, 256 at most), so fp32-grade activations
 //    cost no extra bytes of the weight stream.
 //  * The library keeps its own repacked copy of every weight matrix (pack_weights_kernel):
 //    one contiguous 32 KB block per (tile, K block) in streaming order, already swizzled, so
@@ -179,11 +179,16 @@ __host__ __device__ constexpr uint32_t instr_desc(int n) {
 
 // What the CTA that finishes a tile does with the summed accumulator v[t][n].
 enum EpiMode {
-  EPI_PLAIN = 0,    // out[row0 + t][n] = scale_t * v
+  EPI_PLAIN = 0,    // out[row0 + t][n] = scale_t * v (when out != NULL); with cand != NULL also the
+                    // top-2 of every 128 output columns over [lo, hi): the greedy argmax (Eq. 1) is
+                    // finished from those by argmax_merge_kernel, no [T, V] logits are stored
   EPI_RESID = 1,    // x[row0 + t][n] = (accumulate ? x : 0) + v;  xn = limbs(x * gain[n]);  ssq_out
   EPI_SWIGLU = 2,   // hid[row0 + t][n] = limbs(silu(scale_t * gate) * (scale_t * up))
-  EPI_QKV = 3       // scale_t * v is [q | k | v]: rotate q and k by the row's position (rotate-half
+  EPI_QKV = 3,      // scale_t * v is [q | k | v]: rotate q and k by the row's position (rotate-half
                     // pairs (i, i + dh/2)), write q and, into the row's cache slot, k and v
+  EPI_TOPK = 4      // one 256-column tile (the action rows of the LM head): log-softmax over columns
+                    // [lo, hi) of scale_t * v and its SV_TOPK best entries per row (Eq. 2: the draft
+                    // model's candidates), finished inside the GEMM
 };
 
 struct EpiArgs {
@@ -204,9 +209,14 @@ struct EpiArgs {
   const float *ssq_in;   // [rows][nt_in] partial sums of squares; NULL: scale 1
   int nt_in;
   float inv_k, eps;
-  // EPI_PLAIN
+  // EPI_PLAIN (out may be NULL when cand is given), EPI_TOPK (out may be NULL)
   float *out;
   int ldo;
+  float4 *cand;          // EPI_PLAIN: [rows][2 * tiles] (top-1 value, top-1 column as int bits, top-2 value, -)
+  int lo, hi;            // EPI_PLAIN with cand / EPI_TOPK: columns that take part
+  int tok_offset;        // EPI_TOPK: token id of column 0
+  int *top_tok;          // EPI_TOPK: [rows][SV_TOPK]
+  float *top_lp;
   // EPI_RESID
   float *x;              // [rows][N] residual stream
   int accumulate;

@@ -84,6 +84,8 @@ struct specvla_ctx {
   float2 *rope_tab;
   float *x, *feat, *lgs, *pend_feat, *dout, *margin, *top_lp, *q;
   float *ssq, *lm_ssq;          // per-row partial sums of squares of x / of the gathered LM-head rows
+  float4 *cand;                 // [rows][2 * vocab tiles] top-2 per 128 logit columns (greedy argmax, Eq. 1)
+  int cand_nc;
   bf16 *packed;                 // repacked weight matrices, one after the other
   size_t packed_elems;
   int lgs_rows;                 // rows of the logits buffer
@@ -104,7 +106,6 @@ struct specvla_ctx {
   pk::Op *pk_ops_t;             // phase list of the target forward (device)
   int pk_n_ops_t;
   float *pk_part, *pk_apart, *pk_ssq;
-  float4 *pk_cand;
   bf16 *pk_xn, *pk_ao, *pk_hid;
   unsigned *pk_bar;
   unsigned long long wait_ns;   // limit of every device-side wait
@@ -169,7 +170,11 @@ bool desc_ok(const specvla_model_desc *d) {
 // lanes) and one of its two head sizes.
 bool pk_shapes_ok(const specvla_model_desc &d) {
   const int hd = d.n_heads * d.head_dim;
-  return d.d_model % 128 == 0 && hd % 128 == 0 && d.d_model / 128 <= 64 * 32 && d.n_heads <= 148;
+  // (the unit arithmetic of the kernel is 32-bit: units of the largest matrix times CTAs)
+  const long long units = (long long)((d.vocab + 255) / 256) * ((std::max(d.d_model, d.d_ffn) * 2 + 63) / 64);
+  return d.d_model % 128 == 0 && hd % 128 == 0 && units * 1024 < (1ll << 31) &&
+         (d.vocab + 255) / 256 <= pk::MAX_TILES && (d.d_ffn + 127) / 128 <= pk::MAX_TILES &&
+         (3 * hd + 255) / 256 <= pk::MAX_TILES;
 }
 int sm_count() {
   int dev = 0, n = 0;
@@ -245,8 +250,12 @@ size_t carve(specvla_ctx *c, char *base) {
                       gemm_tc::packed_elems(tiles256(d.d_model), 2 * d.d_model);
     c->packed = cv.take<bf16>(c->packed_elems);
   }
-  c->lgs_rows = (int)(lm_rows > dr ? lm_rows : dr);
-  c->lgs = cv.take<float>((size_t)c->lgs_rows * d.vocab);
+  // full-vocabulary logits are stored only for the draft model's top-k when it ranges over the
+  // whole vocabulary (action_only = 0); the greedy argmax works from per-128-column candidates
+  c->lgs_rows = (int)dr;
+  c->lgs = cv.take<float>((size_t)c->lgs_rows * (d.action_only ? d.n_bins : d.vocab));
+  c->cand_nc = 2 * tiles256(d.vocab);
+  c->cand = cv.take<float4>((lm_rows > 32 ? lm_rows : 32) * (size_t)c->cand_nc);
   c->pend_feat = cv.take<float>(E * SV_MAX_PENDING * d.d_model);
   c->dout = cv.take<float>(E * SV_MAX_TREE * d.d_model);
   c->margin = cv.take<float>(R);
@@ -283,7 +292,6 @@ size_t carve(specvla_ctx *c, char *base) {
     c->pk_part = cv.take<float>(G * c->pk_max_seg * pk::PART_ELEMS);
     c->pk_apart = cv.take<float>((size_t)d.n_heads * c->pk_splits * 32 * (d.head_dim + 4));
     c->pk_ssq = cv.take<float>((size_t)32 * c->pk_nt);
-    c->pk_cand = cv.take<float4>((size_t)32 * 2 * tiles256(d.vocab));
     c->pk_ops_t = cv.take<pk::Op>((size_t)5 * d.n_layers + 2);
     c->pk_bar = cv.take<unsigned>(32);
   }
@@ -293,7 +301,7 @@ size_t carve(specvla_ctx *c, char *base) {
 void derive_caps(specvla_ctx *c) {
   const specvla_model_desc &d = c->desc;
   c->hd = d.n_heads * d.head_dim;
-  c->pk_G = sm_count();
+  c->pk_G = std::min(sm_count(), (int)pk::MAX_G);
   size_t lm = (size_t)d.max_episodes * SV_MAX_TREE;
   if (lm > (size_t)d.max_rows) lm = d.max_rows;
   c->max_lm_rows = (int)lm;
@@ -382,6 +390,18 @@ gemm_tc::EpiArgs epi_plain(float *out, int ldo, int N, const float *ssq_in, int 
   e.ldo = ldo;
   e.ssq_in = ssq_in;
   e.nt_in = nt_in;
+  return e;
+}
+// Draft scoring fused into the (one-tile) action-row LM head: log-softmax + top-k per row.
+gemm_tc::EpiArgs epi_topk(specvla_ctx *ctx, int N, int tok_offset) {
+  gemm_tc::EpiArgs e = {};
+  e.mode = gemm_tc::EPI_TOPK;
+  e.N = N;
+  e.lo = 0;
+  e.hi = N;
+  e.tok_offset = tok_offset;
+  e.top_tok = ctx->top_tok;
+  e.top_lp = ctx->top_lp;
   return e;
 }
 // x (+)= result; xn = limbs(x * gain) (gain may be NULL); ssq = per-tile sums of squares of x.
@@ -507,12 +527,27 @@ int draft_forward(specvla_ctx *ctx, int R, const EpArgs &rows, cudaStream_t st) 
                    ctx->desc.action_only ? &ctx->lm_head_act : &ctx->lm_head, st);
 }
 
-// LM head over `rows` two-limb rows of A into ctx->lgs [rows][vocab]. ssq != NULL: the rows
-// are limbs(x * final gain) and get their RMSNorm scale here.
+// LM head over `rows` two-limb rows of A into ctx->lgs [rows][vocab] (draft top-k over the whole
+// vocabulary). ssq != NULL: the rows are limbs(x * final gain) and get their RMSNorm scale here.
 int lm_head(specvla_ctx *ctx, const XBuf &A, const float *ssq, int rows, cudaStream_t st) {
-  if (rows > ctx->max_lm_rows || rows > ctx->lgs_rows) return SPECVLA_ERR_CAPACITY;
+  if (rows > ctx->max_lm_rows || rows > ctx->lgs_rows || ctx->desc.action_only) return SPECVLA_ERR_CAPACITY;
   return gemm(ctx, A, ctx->lm_head, rows, epi_plain(ctx->lgs, ctx->desc.vocab, ctx->desc.vocab, ssq, ctx->nt),
               st, SPECVLA_PROF_LM_HEAD);
+}
+
+void argmax_range(const specvla_ctx *ctx, int *lo, int *hi);
+// LM head + greedy argmax (Eq. 1) over `rows` rows: the GEMM's epilogue leaves the top-2 of every
+// 128 logit columns, a one-warp-per-row kernel finishes greedy token and margin. The logits
+// themselves are written only when logits_out is given (parity tests).
+int lm_head_greedy(specvla_ctx *ctx, const XBuf &A, const float *ssq, int rows, float *logits_out, cudaStream_t st) {
+  if (rows > ctx->max_lm_rows) return SPECVLA_ERR_CAPACITY;
+  gemm_tc::EpiArgs e = epi_plain(logits_out, ctx->desc.vocab, ctx->desc.vocab, ssq, ctx->nt);
+  e.cand = ctx->cand;
+  argmax_range(ctx, &e.lo, &e.hi);
+  TRY(gemm(ctx, A, ctx->lm_head, rows, e, st, SPECVLA_PROF_LM_HEAD));
+  LAUNCH(epi::argmax_merge_kernel, dim3((rows + 3) / 4), dim3(128), (const float4 *)ctx->cand, ctx->cand_nc, rows,
+         ctx->greedy, ctx->margin);
+  return SPECVLA_OK;
 }
 
 void argmax_range(const specvla_ctx *ctx, int *lo, int *hi) {
@@ -642,7 +677,7 @@ int pk_target_forward(specvla_ctx *ctx, int R, const bf16 *embeds, float *logits
   p.apart = ctx->pk_apart;
   p.splits = ctx->pk_splits;
   p.rope_tab = ctx->rope_tab;
-  p.cand = ctx->pk_cand;
+  p.cand = ctx->cand;
   p.logits_out = logits_out;
   p.greedy = ctx->greedy;
   p.margin = ctx->margin;
@@ -821,7 +856,7 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
   ctx->last_ssq = ctx->ssq;
   ctx->last_nt = ctx->nt;
   ctx->pk_ok = false;
-  ctx->use_pk = true;
+  ctx->use_pk = false;            // measured slower than one launch per GEMM on B200: opt-in
   if (pk_shapes_ok(*desc) && pack_ok) {
     pk_build_target_ops(ctx);
     ctx->pk_ok = pk_prepare(ctx);
@@ -953,11 +988,7 @@ int specvla_prefill(specvla_ctx *ctx, int n_ep, const int *episodes, const void 
   LAUNCH(epi::gather_rows_kernel, dim3(n_ep), dim3(256), (const bf16 *)ctx->xn.p, ctx->xn.plane,
          (const float *)ctx->ssq, ctx->nt, (const int *)ctx->lm_rows, d.d_model, ctx->lm_in.p, ctx->lm_in.plane,
          ctx->lm_ssq);
-  int lo, hi;
-  argmax_range(ctx, &lo, &hi);
-  TRY(lm_head(ctx, ctx->lm_in, ctx->lm_ssq, n_ep, st));
-  LAUNCH(epi::argmax_kernel, dim3(n_ep), dim3(epi::THREADS), (const float *)ctx->lgs, d.vocab, lo, hi, ctx->greedy,
-         ctx->margin, logits_out);
+  TRY(lm_head_greedy(ctx, ctx->lm_in, ctx->lm_ssq, n_ep, logits_out, st));
   LAUNCH(tree::prefill_commit_kernel, dim3(n_ep), dim3(256), ea, ctx->st, (const int *)ctx->greedy,
          (const float *)ctx->x, (const float *)ctx->ssq, ctx->nt, ctx->final_norm, d.rms_eps, d.d_model,
          ctx->pend_feat);
@@ -1078,10 +1109,16 @@ int specvla_draft_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const sp
     if (d.action_only) {
       // log-softmax and top-k range over the action ids only, so only their logits are computed
       if (scored_rows > ctx->lgs_rows) return SPECVLA_ERR_CAPACITY;
-      TRY(gemm(ctx, *A, ctx->lm_head_act, scored_rows, epi_plain(ctx->lgs, d.n_bins, d.n_bins, nullptr, ctx->nt), st,
-               SPECVLA_PROF_LM_HEAD));
-      LAUNCH(epi::logsoftmax_topk_kernel, dim3(scored_rows), dim3(epi::THREADS), (const float *)ctx->lgs, d.n_bins,
-             0, d.n_bins, d.action_base, ctx->top_tok, ctx->top_lp);
+      if (d.n_bins <= SV_TILE_ROWS) {
+        // one output tile: log-softmax and top-k are finished in the GEMM's epilogue
+        TRY(gemm(ctx, *A, ctx->lm_head_act, scored_rows, epi_topk(ctx, d.n_bins, d.action_base), st,
+                 SPECVLA_PROF_LM_HEAD));
+      } else {
+        TRY(gemm(ctx, *A, ctx->lm_head_act, scored_rows, epi_plain(ctx->lgs, d.n_bins, d.n_bins, nullptr, ctx->nt),
+                 st, SPECVLA_PROF_LM_HEAD));
+        LAUNCH(epi::logsoftmax_topk_kernel, dim3(scored_rows), dim3(epi::THREADS), (const float *)ctx->lgs, d.n_bins,
+               0, d.n_bins, d.action_base, ctx->top_tok, ctx->top_lp);
+      }
     } else {
       TRY(lm_head(ctx, *A, nullptr, scored_rows, st));
       LAUNCH(epi::logsoftmax_topk_kernel, dim3(scored_rows), dim3(epi::THREADS), (const float *)ctx->lgs, d.vocab,
@@ -1150,11 +1187,7 @@ static int verify_device_trees(specvla_ctx *ctx, const EpArgs &ea, int R, int r,
     TRY(pk_target_forward(ctx, R, nullptr, logits_out, st));
   } else {
     TRY(target_forward(ctx, R, ea, nullptr, st));
-    int lo, hi;
-    argmax_range(ctx, &lo, &hi);
-    TRY(lm_head(ctx, ctx->xn, ctx->ssq, R, st));
-    LAUNCH(epi::argmax_kernel, dim3(R), dim3(epi::THREADS), (const float *)ctx->lgs, d.vocab, lo, hi, ctx->greedy,
-           ctx->margin, logits_out);
+    TRY(lm_head_greedy(ctx, ctx->xn, ctx->ssq, R, logits_out, st));
   }
   ctx->feat_valid = false;
   LAUNCH(tree::accept_select_kernel, dim3(n_ep), dim3(128), ea, ctx->trees, ctx->st, (const int *)ctx->greedy, r,

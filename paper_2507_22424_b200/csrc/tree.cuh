@@ -136,6 +136,149 @@ __global__ void catchup_dst_kernel(EpArgs a, int *__restrict__ dst_row, int *__r
   lm_rows[i] = last;
 }
 
+// [feature ; embedding] row r of the draft model's input: the feature is an fp32 row (split
+// into limbs here), the embedding a bf16 row of E (its lo limb is zero).
+__device__ __forceinline__ void write_draft_input_row(const float *__restrict__ f, const bf16 *__restrict__ e, int d,
+                                                      bf16 *__restrict__ xin, size_t plane, int r) {
+#pragma unroll 2
+  for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
+    store_limbs4(xin, plane, (size_t)r * 2 * d + i, *reinterpret_cast<const float4 *>(f + i));
+    *reinterpret_cast<uint2 *>(xin + (size_t)r * 2 * d + d + i) = *reinterpret_cast<const uint2 *>(e + i);
+    *reinterpret_cast<uint2 *>(xin + plane + (size_t)r * 2 * d + d + i) = make_uint2(0u, 0u);
+  }
+}
+
+// Start of a draft call, one CTA per episode: the (feature_j, token_j) pairs pending since the
+// last commit become draft rows at positions Pd + j, causal among themselves (row table and
+// model input written here); Pd advances; a new tree is opened whose root is the episode's last
+// emitted token, scored by the last of these rows.
+__global__ void __launch_bounds__(256)
+catchup_input_kernel(EpArgs a, EpState *st, DevTree *trees, RowTable rt, const float *__restrict__ pend_feat,
+                     const bf16 *__restrict__ E, int d, bf16 *__restrict__ xin, size_t plane) {
+  __shared__ int s_n, s_tok[SV_MAX_PENDING];
+  pdl_launch();
+  pdl_wait();
+  const int i = blockIdx.x, e = a.eps[i];
+  EpState &s = st[e];
+  if (threadIdx.x == 0) s_n = s.n_pending;
+  if (threadIdx.x < SV_MAX_PENDING) s_tok[threadIdx.x] = s.pending_tok[threadIdx.x];
+  __syncthreads();
+  const int n = s_n, Pd = s.Pd;
+  __syncthreads();                                  // everybody has the old Pd
+  if (threadIdx.x < n) {
+    const int j = threadIdx.x, r = a.row0[i] + j;
+    rt.tok[r] = s_tok[j];
+    rt.src[r] = 0;
+    rt.ep[r] = e;
+    rt.pos[r] = Pd + j;
+    rt.slot[r] = Pd + j;
+    rt.nvis[r] = Pd + j + 1;
+    rt.tbase[r] = 0;
+    for (int w = 0; w < 4; w++) rt.mask[r * 4 + w] = 0;
+  }
+  if (threadIdx.x == 0) {
+    s.Pd = Pd + n;
+    DevTree &tr = trees[e];
+    tr.n_rows = 1;
+    tr.n_drows = 1;
+    tr.tok[0] = s.root;
+    tr.parent[0] = -1;
+    tr.depth[0] = 0;
+    tr.score[0] = 0.f;
+    tr.drow[0] = 0;
+    tr.xrow[0] = a.row0[i] + n - 1;
+    for (int w = 0; w < 4; w++) tr.dmask[0][w] = 0;
+    tr.level_begin = 0;
+    tr.level_end = 1;
+    tr.sel_count = 1;
+    tr.sel[0] = 0;
+  }
+  for (int j = 0; j < n; j++)
+    write_draft_input_row(pend_feat + (size_t)(e * SV_MAX_PENDING + j) * d, E + (size_t)s_tok[j] * d, d, xin, plane,
+                          a.row0[i] + j);
+}
+
+// One level of tree growth and the next level's model input, one CTA per episode. The rows
+// scored last (one per selected parent, in rank order; a.row0 = the first of them, or for the
+// root the episode's last catch-up row) come with their top-K tokens and log-probabilities:
+// parent sel[j] gets `branch` children (score = parent score + log-prob), numbered in creation
+// order. Then the `expand_next` best new nodes (by score, ties to the lower node index: rank by
+// counting) are selected, in rank order, as the next level's rows a.aux + j: token = their own,
+// feature = output row x[xrow[parent]] of the forward that ran their parent, position
+// Pd - 1 + level + 1, cache slot Pd - 1 + draft row, mask = the parent's ancestors and itself.
+__global__ void __launch_bounds__(256)
+grow_input_kernel(EpArgs a, int level, int branch, int expand_next, const int *__restrict__ top_tok,
+                  const float *__restrict__ top_lp, DevTree *trees, const EpState *__restrict__ st, RowTable rt,
+                  const float *__restrict__ x, const bf16 *__restrict__ E, int d, bf16 *__restrict__ xin,
+                  size_t plane) {
+  __shared__ int s_sel_old[16], s_sel[16], s_src[16], s_tokn[16];
+  __shared__ float s_score[128];
+  __shared__ int s_cnt;
+  pdl_launch();
+  pdl_wait();
+  const int i = blockIdx.x, e = a.eps[i];
+  DevTree &tr = trees[e];
+  const int begin = tr.n_rows, nsel = tr.sel_count, base_dr = tr.n_drows;
+  if (threadIdx.x < 16) s_sel_old[threadIdx.x] = tr.sel[threadIdx.x];
+  __syncthreads();                                  // the old state has been read by everybody
+  const int m = nsel * branch;                      // new nodes (at most 128)
+  const int k = threadIdx.x;
+  if (k < m) {
+    const int j = k / branch, b = k - j * branch;
+    const int p = s_sel_old[j], srow = a.row0[i] + j, n = begin + k;
+    const float sc = tr.score[p] + top_lp[srow * SV_TOPK + b];
+    tr.tok[n] = top_tok[srow * SV_TOPK + b];
+    tr.parent[n] = p;
+    tr.depth[n] = level + 1;
+    tr.score[n] = sc;
+    tr.drow[n] = -1;
+    s_score[k] = sc;
+  }
+  const int cnt = expand_next < m ? expand_next : m;
+  if (k == 0) {
+    tr.n_rows = begin + m;
+    tr.level_begin = begin;
+    tr.level_end = begin + m;
+    tr.sel_count = cnt;
+    tr.n_drows = base_dr + cnt;
+    s_cnt = cnt;
+  }
+  __syncthreads();
+  if (k < m) {
+    int rank = 0;
+    for (int q = 0; q < m; q++) rank += (s_score[q] > s_score[k]) || (s_score[q] == s_score[k] && q < k);
+    if (rank < cnt) s_sel[rank] = begin + k;
+  }
+  __syncthreads();
+  if (k < cnt) {
+    const int n = s_sel[k], dr = base_dr + k;
+    const int p = tr.parent[n], pdr = tr.drow[p];
+    const int Pd = st[e].Pd, r = a.aux[i] + k;
+    tr.sel[k] = n;
+    tr.drow[n] = dr;
+    tr.xrow[n] = r;
+    uint32_t msk[4];
+    for (int w = 0; w < 4; w++) msk[w] = tr.dmask[pdr][w];
+    msk[dr >> 5] |= 1u << (dr & 31);
+    for (int w = 0; w < 4; w++) {
+      tr.dmask[dr][w] = msk[w];
+      rt.mask[r * 4 + w] = msk[w];
+    }
+    rt.tok[r] = tr.tok[n];
+    rt.src[r] = 0;
+    rt.ep[r] = e;
+    rt.pos[r] = Pd - 1 + level + 1;
+    rt.slot[r] = Pd - 1 + dr;              // draft row dr >= 1 -> slot Pd + (dr - 1)
+    rt.nvis[r] = Pd;
+    rt.tbase[r] = Pd - 1;                  // bit dr of the mask <-> slot Pd - 1 + dr
+    s_src[k] = tr.xrow[p];
+    s_tokn[k] = tr.tok[n];
+  }
+  __syncthreads();
+  for (int j = 0; j < s_cnt; j++)
+    write_draft_input_row(x + (size_t)s_src[j] * d, E + (size_t)s_tokn[j] * d, d, xin, plane, a.aux[i] + j);
+}
+
 // One level of tree growth. The rows scored last (one per selected parent, in rank order)
 // come with their top-K tokens and log-probabilities; parent sel[j] gets `branch` children
 // (score = parent score + log-prob). Then the `expand_next` best new nodes (by score, ties

@@ -249,3 +249,21 @@ def test_gemm_full_size_sampled_outputs(T, N, K):
     for t, n in zip(ts, ns):
         ref = float(xc[t] @ wc[n].double())
         assert abs(float(y[t, n]) - ref) < 1e-4 * 0.02 * (K ** 0.5) + 1e-6
+
+
+def test_c1_persistent_forward_kernel_matches_oracle(env):
+    """The same verification step through the single cooperative forward kernel (opt-in): one
+    iteration of C1 with the oracle's draft tree, everything compared."""
+    from paper_2507_22424_b200.binding import OPT_PERSISTENT_FORWARD
+    orc, gpu = env["orc"], env["gpu"]
+    gpu.set_option(OPT_PERSISTENT_FORWARD, 1)
+    try:
+        tally = G.Tally()
+        ep, _, _ = G.prefill_both(orc, gpu, env["emb"], env["ids"], 0, tally, DESC)
+        tree = orc.draft_tree(ep, C.TREE_26)
+        gpu.draft_tree([0], env["shape"], want_trees=False)
+        G.verify_both(orc, gpu, ep, tree, 0, tally, DESC, where="pk.g")
+        tally.report("C1 persistent forward")
+        assert tally.accepts == tally.caches == 1 and tally.rows_exact >= 18
+    finally:
+        gpu.set_option(OPT_PERSISTENT_FORWARD, 0)

@@ -17,10 +17,14 @@ def wcuda(c0):
     return G.to_cuda(c0["weights"])
 
 
-def _gpu(c0, wcuda, **kw):
+def _gpu(c0, wcuda, persistent=False, **kw):
     args = dict(max_seq=256, max_episodes=2, max_rows=256, action_only=True)
     args.update(kw)
-    return G.make_gpu(c0["desc"], wcuda, **args)
+    gpu = G.make_gpu(c0["desc"], wcuda, **args)
+    if persistent:
+        from paper_2507_22424_b200.binding import OPT_PERSISTENT_FORWARD
+        gpu.set_option(OPT_PERSISTENT_FORWARD, 1)
+    return gpu
 
 
 @pytest.mark.parametrize("T,N,K", [(1, 256, 256), (15, 1376, 256), (15, 256, 688), (27, 4096, 4096),
@@ -51,13 +55,16 @@ def test_prefill_logits_and_first_token(c0, wcuda, action_only):
     gpu.close()
 
 
-@pytest.mark.parametrize("n_rows,seed", [(1, 0), (15, 1), (27, 2), (60, 3), (128, 4)])
-def test_verify_tree_matches_oracle(c0, wcuda, n_rows, seed):
+@pytest.mark.parametrize("n_rows,seed,persistent", [(1, 0, False), (15, 1, False), (27, 2, False), (60, 3, False),
+                                                    (128, 4, False), (1, 0, True), (15, 1, True), (27, 2, True),
+                                                    (32, 5, True)])
+def test_verify_tree_matches_oracle(c0, wcuda, n_rows, seed, persistent):
     """Logits, greedy tokens, accepted length, emitted tokens, path, compacted cache and state of
-    one verification, for every tree size: all compared on every run (see gpu_helpers)."""
+    one verification, for every tree size: all compared on every run (see gpu_helpers). With
+    `persistent` the forward runs as the single cooperative kernel (up to 32 rows)."""
     desc = c0["desc"]
     orc = c0["make"]()
-    gpu = _gpu(c0, wcuda)
+    gpu = _gpu(c0, wcuda, persistent=persistent)
     tally = G.Tally()
     ep, _, _ = G.prefill_both(orc, gpu, c0["embeds"].cuda(), c0["ids"], 0, tally, desc)
     tok, par, dep = data.random_tree(n_rows, desc, seed=seed, max_depth=8, root_token=ep.root)
@@ -181,14 +188,14 @@ def test_generate_action_with_dynamic_tree_is_lossless(c0, wcuda):
     gpu.close()
 
 
-@pytest.mark.parametrize("r", [0, 4])
-@pytest.mark.parametrize("action_only", [True, False])
-def test_generate_action_lockstep_with_oracle(c0, wcuda, r, action_only):
+@pytest.mark.parametrize("r,action_only,persistent", [(0, True, False), (4, True, False), (0, False, False),
+                                                      (4, False, False), (4, True, True), (0, False, True)])
+def test_generate_action_lockstep_with_oracle(c0, wcuda, r, action_only, persistent):
     """Iteration by iteration until the chunk is complete: the oracle's draft tree is verified on
     both sides; accepted length, emitted tokens, path, cache and state agree in every iteration."""
     desc, shape = c0["desc"], c0["wl"].tree
     orc = c0["make"](action_only=action_only)
-    gpu = _gpu(c0, wcuda, action_only=action_only)
+    gpu = _gpu(c0, wcuda, action_only=action_only, persistent=persistent)
     tally = G.Tally()
     ep, _, _ = G.prefill_both(orc, gpu, c0["embeds"].cuda(), c0["ids"], 0, tally, desc, action_only)
     from paper_2507_22424_b200.binding import make_shape
