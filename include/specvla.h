@@ -122,6 +122,12 @@ typedef struct {
   int tokens_emitted;             /* before clipping, first episode */
   int accept_len[16];             /* accepted draft tokens m of the first 16 iterations, first episode */
   float ms_prefill, ms_draft, ms_verify;   /* device time, CUDA events */
+  /* Accepted draft tokens by the position at which an iteration starts (Table 3): an iteration
+   * that begins when k + 1 tokens of the chunk exist starts at position k (0 .. n_tokens - 2).
+   * Iterations counted and accepted lengths m summed per position, first episode; positions past
+   * 15 go uncounted. mean = pos_accept_sum[k] / pos_iterations[k]. */
+  int pos_iterations[16];
+  int pos_accept_sum[16];
 } specvla_stats;
 
 /* Bytes of device workspace a context of this description needs. 0 on invalid description. */
@@ -194,6 +200,15 @@ int specvla_verify_tree(specvla_ctx *ctx, int n_ep, const int *episodes,
                         const specvla_tree *trees, int r, int *accept_len_out, int *tokens_out,
                         float *logits_out, void *stream);
 
+/* The verification forward alone (Eq. 1 over every tree row): greedy token of M_V after each row
+ * of caller-supplied trees, WITHOUT acceptance, compaction or any change of the episodes' state
+ * (the tree rows' K/V land in cache slots beyond the committed ones and are overwritten by the next
+ * forward). For harnesses that need the target's opinion on partial trees, e.g. to plant drafts
+ * around its greedy bins. The uploaded trees replace the device-resident ones.
+ *   greedy_out  host [total rows], rows in call order */
+int specvla_score_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const specvla_tree *trees,
+                       int *greedy_out, void *stream);
+
 /* Whole chunk (Algorithm 1): prefill, then draft -> verify -> accept until every episode has
  * n_tokens tokens; the result is clipped to n_tokens. One stream synchronisation per
  * iteration (the accepted length decides termination).
@@ -231,6 +246,26 @@ int specvla_read_kv(specvla_ctx *ctx, int draft, int episode, int layer, int whi
 size_t specvla_gemm_scratch_bytes(int T, int N, int K);
 int specvla_gemm(const float *X, const void *W, float *Y, int T, int N, int K,
                  void *scratch, size_t scratch_bytes, void *stream);
+/* The same product with W given in the library's streaming order (Section 3.1: the cost of
+ * decoding is the parameter stream; the decoder keeps every matrix in this form): one contiguous,
+ * pre-swizzled 32 KB block per (256-row tile, 64-column K block), read by plain bulk copies.
+ * specvla_pack_weights writes that form of W [N, K] into `packed` (device, 1024-byte aligned, at
+ * least specvla_packed_weight_bytes(N, K) bytes; 0 is returned for an invalid shape); pack once,
+ * multiply many times. Scratch and status as for specvla_gemm. */
+size_t specvla_packed_weight_bytes(int N, int K);
+int specvla_pack_weights(const void *W, int N, int K, void *packed, size_t packed_bytes, void *stream);
+int specvla_gemm_prepacked(const float *X, const void *Wpacked, float *Y, int T, int N, int K,
+                           void *scratch, size_t scratch_bytes, void *stream);
+
+/* Failure-handling test hook (no counterpart in the paper). Every device-side wait of the GEMM
+ * is bounded; this call makes the NEXT specvla_gemm / specvla_gemm_prepacked call of the process
+ * run with the given wait limit (nanoseconds, >= 1000) and has the producer of every CTA withhold
+ * the K block of that index within its K range (-1: none), so that the waits for it run out: the
+ * kernel records the failure in the scratch's status word, lets its copies land, frees its
+ * tensor memory and returns, and specvla_gemm_status reports SPECVLA_ERR_TIMEOUT. Nothing faults
+ * or hangs; the context stays usable. Both settings are cleared by that one call. */
+int specvla_gemm_fault_test(long long wait_limit_ns, int withhold_k_block);
+
 /* Synchronises `stream` and reports whether the specvla_gemm calls that used `scratch` ran
  * to completion: SPECVLA_ERR_TIMEOUT if a bounded device-side wait gave up (Y is then
  * undefined), SPECVLA_ERR_CUDA if the stream is in error, else SPECVLA_OK. */
@@ -252,10 +287,13 @@ int specvla_gemm_status(const void *scratch, void *stream);
  *    contents; the call clears what it needs cleared. Two calls that may overlap on the GPU
  *    (different streams, no dependency) race on it: serialise them.
  *  - wait != 0: synchronises `stream` and returns SPECVLA_ERR_TIMEOUT if a bounded
- *    device-side wait gave up (as specvla_gemm_status); wait == 0: asynchronous. */
+ *    device-side wait gave up (as specvla_gemm_status); wait == 0: asynchronous (ask
+ *    specvla_gemm_static_status afterwards). Inside a stream capture wait must be 0. */
 #define SPECVLA_STATIC_SCRATCH_BYTES (16u << 20)
 int specvla_gemm_static(const float *X, const void *W, float *Y, int T, int N, int K, int wait,
                         void *stream);
+/* specvla_gemm_status for the built-in scratch of the current device: synchronises `stream`. */
+int specvla_gemm_static_status(void *stream);
 
 /* Per-GEMM device timing (measurement aid; Section 3.1 attributes the latency to the
  * parameter stream, which these GEMMs are). `phases` is a bit mask: 1 = prefill, 2 = draft,

@@ -47,7 +47,8 @@ class Tree(C.Structure):
 
 class Stats(C.Structure):
     _fields_ = [("iterations", C.c_int), ("tokens_emitted", C.c_int), ("accept_len", C.c_int * 16),
-                ("ms_prefill", C.c_float), ("ms_draft", C.c_float), ("ms_verify", C.c_float)]
+                ("ms_prefill", C.c_float), ("ms_draft", C.c_float), ("ms_verify", C.c_float),
+                ("pos_iterations", C.c_int * 16), ("pos_accept_sum", C.c_int * 16)]
 
 
 EXPORTS = {
@@ -63,6 +64,8 @@ EXPORTS = {
                                      C.POINTER(Tree), C.c_void_p]),
     "specvla_verify_tree": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_int), C.POINTER(Tree), C.c_int,
                                       C.POINTER(C.c_int), C.POINTER(C.c_int), C.c_void_p, C.c_void_p]),
+    "specvla_score_tree": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_int), C.POINTER(Tree), C.POINTER(C.c_int),
+                                     C.c_void_p]),
     "specvla_generate_action": (C.c_int, [C.c_void_p, C.c_int, C.POINTER(C.c_int), C.c_void_p,
                                           C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(TreeShape),
                                           C.c_int, C.c_int, C.POINTER(C.c_int), C.POINTER(C.c_float),
@@ -74,6 +77,12 @@ EXPORTS = {
     "specvla_gemm": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                                     C.c_void_p, C.c_size_t, C.c_void_p]),
     "specvla_gemm_status": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "specvla_packed_weight_bytes": (C.c_size_t, [C.c_int, C.c_int]),
+    "specvla_pack_weights": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "specvla_gemm_prepacked": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
+                                         C.c_void_p, C.c_size_t, C.c_void_p]),
+    "specvla_gemm_fault_test": (C.c_int, [C.c_longlong, C.c_int]),
+    "specvla_gemm_static_status": (C.c_int, [C.c_void_p]),
     "specvla_gemm_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int,
                                      C.c_void_p]),
     "specvla_profile": (C.c_int, [C.c_void_p, C.c_int]),
@@ -234,6 +243,21 @@ class SpecVLA:
         emitted = [list(toks[i * (MAX_DEPTH + 1): i * (MAX_DEPTH + 1) + m[i] + 1]) for i in range(n)]
         return (list(m), emitted, logits) if want_logits else (list(m), emitted)
 
+    def score_tree(self, episodes, trees):
+        """Greedy token of the target after every row of the given trees; episode state untouched."""
+        n = len(episodes)
+        ctrees, keep, rows = (Tree * n)(), [], 0
+        for i, t in enumerate(trees):
+            a, b, c = _ints(t["tokens"]), _ints(t["parent"]), _ints(t["depth"])
+            keep += [a, b, c]
+            ctrees[i].n_rows = len(t["tokens"])
+            ctrees[i].tokens, ctrees[i].parent, ctrees[i].depth = a, b, c
+            ctrees[i].score = None
+            rows += len(t["tokens"])
+        g = (C.c_int * rows)()
+        self._check(lib.specvla_score_tree(self.h, n, _ints(episodes), ctrees, g, _stream()))
+        return list(g)
+
     def generate_action(self, episodes, embeds, token_ids, lens, shape: TreeShape, r, n_tokens=7):
         n = len(episodes)
         toks = (C.c_int * (n * n_tokens))()
@@ -285,6 +309,38 @@ def gemm(x: torch.Tensor, w: torch.Tensor) -> torch.Tensor:
     sp = (scratch.data_ptr() + 1023) // 1024 * 1024
     rc = lib.specvla_gemm(C.c_void_p(x.data_ptr()), C.c_void_p(w.data_ptr()), C.c_void_p(y.data_ptr()),
                                T, N, K, C.c_void_p(sp), nb, _stream())
+    if rc == 0:
+        rc = lib.specvla_gemm_status(C.c_void_p(sp), _stream())
+    if rc != 0:
+        raise SpecVLAError(rc)
+    return y
+
+
+def pack_weights(w: torch.Tensor) -> torch.Tensor:
+    """The library's streaming form of W [N, K] (bf16): specvla_pack_weights into a new buffer."""
+    assert w.dtype == torch.bfloat16 and w.is_contiguous()
+    N, K = w.shape
+    nb = lib.specvla_packed_weight_bytes(N, K)
+    if nb == 0:
+        raise SpecVLAError(-1, "(shape rejected)")
+    buf = torch.empty(nb + 1024, dtype=torch.uint8, device="cuda")
+    off = (-buf.data_ptr()) % 1024
+    packed = buf[off:off + nb]
+    rc = lib.specvla_pack_weights(C.c_void_p(w.data_ptr()), N, K, C.c_void_p(packed.data_ptr()), nb, _stream())
+    if rc != 0:
+        raise SpecVLAError(rc)
+    return packed
+
+
+def gemm_prepacked(x: torch.Tensor, packed: torch.Tensor, N: int) -> torch.Tensor:
+    """Y[T, N] = X[T, K] (f32) @ W^T with W given in packed form (pack_weights)."""
+    T, K = x.shape
+    y = torch.empty(T, N, dtype=torch.float32, device="cuda")
+    nb = lib.specvla_gemm_scratch_bytes(T, N, K)
+    scratch = torch.empty(nb + 1024, dtype=torch.uint8, device="cuda")
+    sp = (scratch.data_ptr() + 1023) // 1024 * 1024
+    rc = lib.specvla_gemm_prepacked(C.c_void_p(x.data_ptr()), C.c_void_p(packed.data_ptr()), C.c_void_p(y.data_ptr()),
+                                    T, N, K, C.c_void_p(sp), nb, _stream())
     if rc == 0:
         rc = lib.specvla_gemm_status(C.c_void_p(sp), _stream())
     if rc != 0:

@@ -124,37 +124,6 @@ using sv::top2_push;
 using sv::top2_merge;
 using sv::top2_warp;
 
-// Greedy token per row of logits [T][V]: argmax over [lo, hi) with ties to the lowest id;
-// margin = top-1 minus top-2 over the same range. Optionally copies the whole row out.
-__global__ void __launch_bounds__(THREADS)
-argmax_kernel(const float *__restrict__ logits, int V, int lo, int hi, int *__restrict__ greedy,
-              float *__restrict__ margin, float *__restrict__ logits_out) {
-  __shared__ Top2 red[THREADS / 32];
-  pdl_launch();
-  pdl_wait();
-  const int t = blockIdx.x;
-  const float *row = logits + (size_t)t * V;
-  Top2 best{-INFINITY, -INFINITY, 0x7fffffff};
-  if (logits_out)
-    for (int v = threadIdx.x; v < V; v += blockDim.x) logits_out[(size_t)t * V + v] = row[v];
-  for (int v = lo + threadIdx.x; v < hi; v += blockDim.x) top2_push(best, row[v], v);
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    Top2 other;
-    other.v1 = __shfl_xor_sync(0xffffffffu, best.v1, o);
-    other.v2 = __shfl_xor_sync(0xffffffffu, best.v2, o);
-    other.i1 = __shfl_xor_sync(0xffffffffu, best.i1, o);
-    top2_merge(best, other);
-  }
-  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = best;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    for (int w = 1; w < THREADS / 32; w++) top2_merge(best, red[w]);
-    greedy[t] = best.i1;
-    margin[t] = best.v1 - best.v2;
-  }
-}
-
 // Greedy token per row from the candidates a GEMM epilogue left: cand[row][0..nc) holds the top-2
 // of each 128-column group of the row's logits (value, column as int bits, second value). One
 // warp per row; ties go to the lowest id; margin = top-1 minus top-2.

@@ -96,7 +96,10 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 
   const int npre = n_units < STAGES ? n_units : STAGES;
   uint64_t pol_w = 0;
+  // test hook: the K block that is never loaded (-1: none)
+  const int withheld = ea.withhold_unit - 1;
   auto load_w = [&](int it) {
+    if (it == withheld) return;
     const int st = it % STAGES;
     const uint32_t sW = base + st * STAGE;
     mbar_expect_tx(full_bar(st), stage_tx);
@@ -144,15 +147,17 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       const uint64_t pol_x = policy_evict_last();
       grid_dep_wait();
       for (int j = 0; j < npre; j++)
-        tma_load_3d(base + j * STAGE + W_STAGE_BYTES, xmap, (kb0 + j) * BK, row0, 0, full_bar(j), pol_x);
+        if (j != withheld)
+          tma_load_3d(base + j * STAGE + W_STAGE_BYTES, xmap, (kb0 + j) * BK, row0, 0, full_bar(j), pol_x);
       for (int it = npre; it < n_units; it++) {
         const int st = it % STAGES, rnd = it / STAGES;
-        if (!mbar_wait(empty_bar(st), (rnd - 1) & 1)) {
+        if (!mbar_wait(empty_bar(st), (rnd - 1) & 1, ea.wait_ns)) {
           atomicExch(err, SV_ERR_WAIT_EMPTY);
           break;
         }
         load_w(it);
-        tma_load_3d(base + st * STAGE + W_STAGE_BYTES, xmap, (kb0 + it) * BK, row0, 0, full_bar(st), pol_x);
+        if (it != withheld)
+          tma_load_3d(base + st * STAGE + W_STAGE_BYTES, xmap, (kb0 + it) * BK, row0, 0, full_bar(st), pol_x);
       }
     }
     __syncwarp();
@@ -161,7 +166,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     if (lane == 0 && n_units > 0) {
       for (int it = 0; it < n_units; it++) {
         const int st = it % STAGES, rnd = it / STAGES;
-        if (!mbar_wait(full_bar(st), rnd & 1)) {
+        if (!mbar_wait(full_bar(st), rnd & 1, ea.wait_ns)) {
           atomicExch(err, SV_ERR_WAIT_FULL);
           break;
         }
@@ -220,7 +225,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     }
     bool have = n_units > 0;
     if (have) {
-      const bool mine = mbar_wait(tfull_bar, 0);
+      const bool mine = mbar_wait(tfull_bar, 0, ea.wait_ns);
       if (lane == 0) s_flag[warp - 2] = mine ? 1 : 0;
       epi_barrier();
       have = s_flag[0] && s_flag[1] && s_flag[2] && s_flag[3] && s_flag[4] && s_flag[5] && s_flag[6] && s_flag[7];

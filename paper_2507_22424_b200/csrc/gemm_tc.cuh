@@ -19,8 +19,8 @@
 //    issued BEFORE griddepcontrol.wait: launched with programmatic stream serialisation a GEMM
 //    streams weights while its predecessor drains.
 //
-// Every mbarrier wait is bounded (two seconds of %globaltimer); on expiry the kernel records
-// a code in *err, lets copies in flight land, frees its TMEM and returns.
+// Every mbarrier wait is bounded (EpiArgs::wait_ns of %globaltimer, two seconds by default); on
+// expiry the kernel records a code in *err, lets copies in flight land, frees its TMEM and returns.
 #pragma once
 #include <cuda.h>
 
@@ -73,16 +73,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
-// Bounded wait: false after WAIT_LIMIT_NS without the phase completing.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;     // default limit of a device-side wait
+// Bounded wait: false after limit_ns without the phase completing.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint64_t limit_ns) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_ns();
   for (;;) {
 #pragma unroll 1
     for (int i = 0; i < 128; i++)
       if (mbar_try_wait(bar, parity)) return true;
-    if (global_ns() - t0 > WAIT_LIMIT_NS) return false;
+    if (global_ns() - t0 > limit_ns) return false;
   }
 }
 __device__ __forceinline__ uint64_t policy_evict_first() {
@@ -198,6 +198,9 @@ struct EpiArgs {
   int tn_tail;           // tn_of(rows of the last 128-row chunk): its X box and MMA width
   int N;                 // output columns (EPI_SWIGLU: F, the width of gate and of up)
   int up_off;            // EPI_SWIGLU: row of W where the up projection starts (F)
+  unsigned long long wait_ns;   // limit of every mbarrier wait
+  int withhold_unit;     // test hook (specvla_gemm_fault_test): > 0: the producer of every CTA skips its
+                         // (withhold_unit - 1)-th K block, so the waits for it run out; 0: off
   const bf16 *wpacked;   // weights repacked by pack_weights_kernel (one contiguous 32 KB block per
                          // (tile, K block), in unit order); NULL: strided boxes through the W map
   // L2 prefetch for the GEMM that follows: once its own loads are issued, every CTA asks for

@@ -8,6 +8,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -82,7 +83,7 @@ struct specvla_ctx {
   float *kv_t, *kv_d;           // target [ep][layer][2][max_seq][hd], draft [ep][2][max_seq][hd], fp32
   size_t kv_t_ep_stride, kv_t_layer_stride, kv_d_ep_stride;
   float2 *rope_tab;
-  float *x, *feat, *lgs, *pend_feat, *dout, *margin, *top_lp, *q;
+  float *x, *feat, *lgs, *pend_feat, *margin, *top_lp, *q;
   float *ssq, *lm_ssq;          // per-row partial sums of squares of x / of the gathered LM-head rows
   float4 *cand;                 // [rows][2 * vocab tiles] top-2 per 128 logit columns (greedy argmax, Eq. 1)
   int cand_nc;
@@ -94,7 +95,7 @@ struct specvla_ctx {
   XBuf xn, xin, ao, hid, lm_in;
   int *err;                     // device status word written by bounded waits that gave up
   RowTable rt;
-  int *feat_src, *dst_row, *lm_rows, *greedy, *top_tok, *out_m, *out_tok, *out_path;
+  int *feat_src, *lm_rows, *greedy, *top_tok, *out_m, *out_tok, *out_path;
   EpState *st;
   DevTree *trees;
 
@@ -117,7 +118,7 @@ struct specvla_ctx {
   size_t pinned_bytes;
   int *pin_small;               // 4096 ints of results read back
   DevTree *pin_trees;           // max_episodes trees
-  int *pin_rows;                // 8 * max_rows ints
+  int *pin_rows;                // 11 * max_rows + SV_MAX_EP ints: row tables of the target and of the draft model
   std::vector<int> hP, hPending;  // host mirror of P and n_pending; -1 = not prefilled
   std::vector<int> hTreeRows;     // rows of the device-resident tree left by the last draft call
   int last_rows;                // rows of the last target forward
@@ -233,10 +234,10 @@ size_t carve(specvla_ctx *c, char *base) {
   c->q = cv.take<float>(R * hd);
   limbs(c->ao, R, hd);
   limbs(c->hid, R, d.d_ffn);
-  limbs(c->lm_in, lm_rows, d.d_model);
+  limbs(c->lm_in, E, d.d_model);                 // last prefix row of each episode (first token)
   c->nt = (d.d_model + SV_TILE_ROWS - 1) / SV_TILE_ROWS;
   c->ssq = cv.take<float>(R * c->nt);
-  c->lm_ssq = cv.take<float>(lm_rows * c->nt);
+  c->lm_ssq = cv.take<float>(E * c->nt);
   auto tiles256 = [](int N) { return (N + SV_TILE_ROWS - 1) / SV_TILE_ROWS; };
   {
     // repacked weights: every target layer, the LM head and its action rows, the draft fc and
@@ -257,7 +258,6 @@ size_t carve(specvla_ctx *c, char *base) {
   c->cand_nc = 2 * tiles256(d.vocab);
   c->cand = cv.take<float4>((lm_rows > 32 ? lm_rows : 32) * (size_t)c->cand_nc);
   c->pend_feat = cv.take<float>(E * SV_MAX_PENDING * d.d_model);
-  c->dout = cv.take<float>(E * SV_MAX_TREE * d.d_model);
   c->margin = cv.take<float>(R);
   c->top_lp = cv.take<float>(dr * SV_TOPK);
   c->rt.tok = cv.take<int>(R);
@@ -269,7 +269,6 @@ size_t carve(specvla_ctx *c, char *base) {
   c->rt.tbase = cv.take<int>(R);
   c->rt.mask = cv.take<uint32_t>(R * 4);
   c->feat_src = cv.take<int>(R);
-  c->dst_row = cv.take<int>(R);
   c->lm_rows = cv.take<int>(R);
   c->greedy = cv.take<int>(R);
   c->top_tok = cv.take<int>(dr * SV_TOPK);
@@ -352,6 +351,7 @@ int gemm(specvla_ctx *ctx, const XBuf &A, const WMat &W, int R, gemm_tc::EpiArgs
   const int tiles = swiglu ? (ea.N + 127) / 128 : (W.N + SV_TILE_ROWS - 1) / SV_TILE_ROWS;
   const int KB = (W.K + gemm_tc::BK - 1) / gemm_tc::BK;
   ea.wpacked = W.packed;
+  ea.wait_ns = ctx->wait_ns;
   ea.inv_k = 1.f / (float)W.K;
   ea.eps = ctx->desc.rms_eps;
   const bool prof = (ctx->prof_mask & ctx->phase) && 2 * (ctx->prof_used + 1) <= (int)ctx->prof_ev.size();
@@ -866,7 +866,7 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
   ctx->hTreeRows.assign(desc->max_episodes, 0);
   const size_t small_b = 4096 * sizeof(int);
   const size_t trees_b = (sizeof(DevTree) * desc->max_episodes + 255) / 256 * 256;
-  ctx->pinned_bytes = small_b + trees_b + ((size_t)desc->max_rows * 8 + 256) * sizeof(int);
+  ctx->pinned_bytes = small_b + trees_b + ((size_t)desc->max_rows * 11 + SV_MAX_EP + 256) * sizeof(int);
   ctx->cuda_err[0] = 0;
   if (cudaHostAlloc(&ctx->pinned, ctx->pinned_bytes, cudaHostAllocDefault) != cudaSuccess) {
     delete ctx;
@@ -1000,7 +1000,11 @@ int specvla_prefill(specvla_ctx *ctx, int n_ep, const int *episodes, const void 
   // draft model over the shifted pairs (feature_i, input_{i+1}), i = 0 .. len-2
   if (ctx->has_draft) {
     int Rd = 0;
-    int *h_fs = h + 5 * R + n_ep;          // feature source rows
+    // The draft model's row tables live in their own part of the pinned staging area: the copies
+    // of the target's tables above may still be pending on the stream.
+    int *hd = h + 5 * R + SV_MAX_EP;
+    int *h_tok = hd, *h_src = hd + R, *h_ep = hd + 2 * R, *h_pos = hd + 3 * R, *h_nvis = hd + 4 * R;
+    int *h_fs = hd + 5 * R;                // feature source rows
     EpArgs ed = ea;
     for (int i = 0; i < n_ep; i++) {
       ed.row0[i] = Rd;
@@ -1018,10 +1022,6 @@ int specvla_prefill(specvla_ctx *ctx, int n_ep, const int *episodes, const void 
     }
     if (Rd > 0) {
       const size_t db = (size_t)Rd * sizeof(int);
-      // the uploads above are ordered before these on the same stream, but the pinned rows
-      // are being rewritten: wait until the first batch has been consumed
-      CU(cudaStreamSynchronize(st));
-      prof_collect(ctx);
       CU(cudaMemcpyAsync(ctx->rt.tok, h_tok, db, cudaMemcpyHostToDevice, st));
       CU(cudaMemcpyAsync(ctx->rt.src, h_src, db, cudaMemcpyHostToDevice, st));
       CU(cudaMemcpyAsync(ctx->rt.ep, h_ep, db, cudaMemcpyHostToDevice, st));
@@ -1078,77 +1078,54 @@ int specvla_draft_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const sp
 
   ctx->phase = 2;
   // catch-up over the pending rows; the last row of each episode scores the root's children
-  const bf16 *no_embeds = nullptr;
-  const float *no_f = nullptr;
-  LAUNCH(tree::build_catchup_rows_kernel, dim3((n_ep + 63) / 64), dim3(64), ea, ctx->st, ctx->trees, ctx->rt,
-         ctx->feat_src);
-  LAUNCH(tree::catchup_dst_kernel, dim3((n_ep + 63) / 64), dim3(64), ea, ctx->dst_row, ctx->lm_rows);
-  LAUNCH(tree::draft_input_kernel, dim3(R), dim3(256), ctx->rt, (const int *)ctx->feat_src,
-         (const float *)ctx->pend_feat, no_f, 0, no_f, 0.f, no_embeds, ctx->embed, d.d_model, ctx->xin.p,
-         ctx->xin.plane);
+  LAUNCH(tree::catchup_input_kernel, dim3(n_ep), dim3(256), ea, ctx->st, ctx->trees, ctx->rt,
+         (const float *)ctx->pend_feat, ctx->embed, d.d_model, ctx->xin.p, ctx->xin.plane);
   TRY(draft_forward(ctx, R, ea, st));
-  LAUNCH(tree::save_draft_out_kernel, dim3(R), dim3(256), (const float *)ctx->x, (const int *)ctx->dst_row,
-         d.d_model, ctx->dout);
   ctx->feat_valid = false;
   for (int i = 0; i < n_ep; i++) {
     ctx->hPending[episodes[i]] = 0;
     ctx->hTreeRows[episodes[i]] = n_tree_rows;
   }
 
-  int scored_rows = n_ep;            // rows scored by the LM head in the current round
-  bool gathered = true;              // round 0 scores the gathered last rows
+  // Per level: the shared LM head over the rows just run (draft layer outputs as they are: no
+  // norm, no row scale) with log-softmax + top-k, then one kernel that grows the tree and writes
+  // the next level's input rows, then the draft model over those.
+  int scored_rows = R;               // round 0 scores every catch-up row; only each episode's last one is used
   for (int l = 0; l < shape->depth; l++) {
-    const XBuf *A = &ctx->xn;
-    if (gathered) {
-      LAUNCH(epi::gather_rows_kernel, dim3(n_ep), dim3(256), (const bf16 *)ctx->xn.p, ctx->xn.plane,
-             (const float *)ctx->ssq, ctx->nt, (const int *)ctx->lm_rows, d.d_model, ctx->lm_in.p,
-             ctx->lm_in.plane, ctx->lm_ssq);
-      A = &ctx->lm_in;
-    }
-    // the draft layer's output feeds the shared LM head as it is: no norm, no row scale
-    if (d.action_only) {
-      // log-softmax and top-k range over the action ids only, so only their logits are computed
-      if (scored_rows > ctx->lgs_rows) return SPECVLA_ERR_CAPACITY;
-      if (d.n_bins <= SV_TILE_ROWS) {
-        // one output tile: log-softmax and top-k are finished in the GEMM's epilogue
-        TRY(gemm(ctx, *A, ctx->lm_head_act, scored_rows, epi_topk(ctx, d.n_bins, d.action_base), st,
-                 SPECVLA_PROF_LM_HEAD));
-      } else {
-        TRY(gemm(ctx, *A, ctx->lm_head_act, scored_rows, epi_plain(ctx->lgs, d.n_bins, d.n_bins, nullptr, ctx->nt),
-                 st, SPECVLA_PROF_LM_HEAD));
-        LAUNCH(epi::logsoftmax_topk_kernel, dim3(scored_rows), dim3(epi::THREADS), (const float *)ctx->lgs, d.n_bins,
-               0, d.n_bins, d.action_base, ctx->top_tok, ctx->top_lp);
-      }
+    if (scored_rows > ctx->lgs_rows) return SPECVLA_ERR_CAPACITY;
+    if (d.action_only && d.n_bins <= SV_TILE_ROWS) {
+      // the action ids are one output tile: log-softmax and top-k are finished in the GEMM's epilogue
+      TRY(gemm(ctx, ctx->xn, ctx->lm_head_act, scored_rows, epi_topk(ctx, d.n_bins, d.action_base), st,
+               SPECVLA_PROF_LM_HEAD));
+    } else if (d.action_only) {
+      TRY(gemm(ctx, ctx->xn, ctx->lm_head_act, scored_rows,
+               epi_plain(ctx->lgs, d.n_bins, d.n_bins, nullptr, ctx->nt), st, SPECVLA_PROF_LM_HEAD));
+      LAUNCH(epi::logsoftmax_topk_kernel, dim3(scored_rows), dim3(epi::THREADS), (const float *)ctx->lgs, d.n_bins,
+             0, d.n_bins, d.action_base, ctx->top_tok, ctx->top_lp);
     } else {
-      TRY(lm_head(ctx, *A, nullptr, scored_rows, st));
+      TRY(lm_head(ctx, ctx->xn, nullptr, scored_rows, st));
       LAUNCH(epi::logsoftmax_topk_kernel, dim3(scored_rows), dim3(epi::THREADS), (const float *)ctx->lgs, d.vocab,
              lo, hi, 0, ctx->top_tok, ctx->top_lp);
     }
-    const int cur = (l == 0) ? 1 : shape->expand[l];            // parents scored per episode
+    const int cur = shape->expand[l];                            // parents scored per episode (level 0: the root)
     const int next = (l + 1 < shape->depth) ? shape->expand[l + 1] : 0;
     EpArgs la = ea;
     for (int i = 0; i < n_ep; i++) {
-      la.row0[i] = i * cur;
+      la.row0[i] = (l == 0) ? ea.row0[i] + ea.nrows[i] - 1 : i * cur;
       la.aux[i] = i * next;
     }
-    LAUNCH(tree::expand_level_kernel, dim3((n_ep + 63) / 64), dim3(64), la, l, shape->branch[l], next,
-           (const int *)ctx->top_tok, (const float *)ctx->top_lp, ctx->trees, (const EpState *)ctx->st, ctx->rt,
-           ctx->feat_src, ctx->dst_row);
+    LAUNCH(tree::grow_input_kernel, dim3(n_ep), dim3(256), la, l, shape->branch[l], next, (const int *)ctx->top_tok,
+           (const float *)ctx->top_lp, ctx->trees, (const EpState *)ctx->st, ctx->rt, (const float *)ctx->x,
+           ctx->embed, d.d_model, ctx->xin.p, ctx->xin.plane);
     if (next == 0) break;
     const int Rn = n_ep * next;
-    LAUNCH(tree::draft_input_kernel, dim3(Rn), dim3(256), ctx->rt, (const int *)ctx->feat_src,
-           (const float *)ctx->dout, no_f, 0, no_f, 0.f, no_embeds, ctx->embed, d.d_model, ctx->xin.p,
-           ctx->xin.plane);
     EpArgs ln = ea;
     for (int i = 0; i < n_ep; i++) {
       ln.row0[i] = i * next;
       ln.nrows[i] = next;
     }
     TRY(draft_forward(ctx, Rn, ln, st));
-    LAUNCH(tree::save_draft_out_kernel, dim3(Rn), dim3(256), (const float *)ctx->x, (const int *)ctx->dst_row,
-           d.d_model, ctx->dout);
     scored_rows = Rn;
-    gathered = false;
   }
 
   if (n_tree_rows < 1 + n_nodes)
@@ -1224,12 +1201,11 @@ static int finish_verify(specvla_ctx *ctx, const EpArgs &ea, int *accept_len_out
   return SPECVLA_OK;
 }
 
-int specvla_verify_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const specvla_tree *trees, int r,
-                        int *accept_len_out, int *tokens_out, float *logits_out, void *stream) {
-  TRY(check_episodes(ctx, n_ep, episodes));
-  if (r < 0 || !accept_len_out || !tokens_out) return SPECVLA_ERR_INVALID_ARG;
+// Validates the call's trees (caller-supplied, or the device-resident ones when trees == NULL),
+// lays the episodes' rows out and uploads caller-supplied trees.
+static int prepare_trees(specvla_ctx *ctx, int n_ep, const int *episodes, const specvla_tree *trees, EpArgs *ea_out,
+                         int *rows_out, cudaStream_t st) {
   const specvla_model_desc &d = ctx->desc;
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
   EpArgs ea{};
   ea.n_ep = n_ep;
   int R = 0;
@@ -1268,8 +1244,50 @@ int specvla_verify_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const s
       CU(cudaMemcpyAsync(&ctx->trees[episodes[i]], &h[i], sizeof(DevTree), cudaMemcpyHostToDevice, st));
     }
   }
+  *ea_out = ea;
+  *rows_out = R;
+  return SPECVLA_OK;
+}
+
+int specvla_verify_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const specvla_tree *trees, int r,
+                        int *accept_len_out, int *tokens_out, float *logits_out, void *stream) {
+  TRY(check_episodes(ctx, n_ep, episodes));
+  if (r < 0 || !accept_len_out || !tokens_out) return SPECVLA_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  EpArgs ea{};
+  int R = 0;
+  TRY(prepare_trees(ctx, n_ep, episodes, trees, &ea, &R, st));
   TRY(verify_device_trees(ctx, ea, R, r, logits_out, st));
   return finish_verify(ctx, ea, accept_len_out, tokens_out, st);
+}
+
+int specvla_score_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const specvla_tree *trees,
+                       int *greedy_out, void *stream) {
+  TRY(check_episodes(ctx, n_ep, episodes));
+  if (!trees || !greedy_out) return SPECVLA_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  EpArgs ea{};
+  int R = 0;
+  TRY(prepare_trees(ctx, n_ep, episodes, trees, &ea, &R, st));
+  if (R > 4096 - 64) return SPECVLA_ERR_CAPACITY;                   // results come back through the small staging area
+  ctx->phase = 4;
+  LAUNCH(tree::build_verify_rows_kernel, dim3(n_ep), dim3(128), ea, ctx->trees, (const EpState *)ctx->st, ctx->rt);
+  if (ctx->pk_ok && ctx->use_pk && n_ep == 1 && R <= pk::TN) {
+    TRY(pk_target_forward(ctx, R, nullptr, nullptr, st));
+  } else {
+    TRY(target_forward(ctx, R, ea, nullptr, st));
+    TRY(lm_head_greedy(ctx, ctx->xn, ctx->ssq, R, nullptr, st));
+  }
+  ctx->feat_valid = false;
+  for (int i = 0; i < n_ep; i++) ctx->hTreeRows[episodes[i]] = ea.nrows[i];
+  int *h = ctx->pin_small;
+  CU(cudaMemcpyAsync(h, ctx->greedy, R * sizeof(int), cudaMemcpyDeviceToHost, st));
+  CU(cudaMemcpyAsync(h + 4000, ctx->err, sizeof(int), cudaMemcpyDeviceToHost, st));
+  CU(cudaStreamSynchronize(st));
+  prof_collect(ctx);
+  if (h[4000] != 0) return SPECVLA_ERR_TIMEOUT;
+  for (int k = 0; k < R; k++) greedy_out[k] = h[k];
+  return SPECVLA_OK;
 }
 
 int specvla_generate_action(specvla_ctx *ctx, int n_ep, const int *episodes, const void *embeds,
@@ -1348,6 +1366,11 @@ int specvla_generate_action(specvla_ctx *ctx, int n_ep, const int *episodes, con
       CU(cudaEventElapsedTime(&ms, ctx->ev[1], ctx->ev[2]));
       stats->ms_verify += ms;
       if (iterations < 16) stats->accept_len[iterations] = m_out[0];
+      const int pos = count[0] - 1;
+      if (pos >= 0 && pos < 16) {
+        stats->pos_iterations[pos]++;
+        stats->pos_accept_sum[pos] += m_out[0];
+      }
     }
     for (int i = 0; i < n_ep; i++)
       for (int k = 0; k <= m_out[i]; k++) {
@@ -1428,6 +1451,21 @@ int specvla_read_kv(specvla_ctx *ctx, int draft, int episode, int layer, int whi
 }
 
 // ------------------------------------------------------------------ stand-alone GEMM
+// Resident-cluster counts per device ordinal, looked up once per device under a lock.
+static std::mutex g_dev_mutex;
+static gemm_ck::ClusterFit g_fit[64];
+static bool g_fit_known[64];
+static gemm_ck::ClusterFit cluster_fit_of_current_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return gemm_ck::query_cluster_fit();
+  std::lock_guard<std::mutex> lock(g_dev_mutex);
+  if (!g_fit_known[dev]) {
+    g_fit[dev] = gemm_ck::query_cluster_fit();
+    g_fit_known[dev] = true;
+  }
+  return g_fit[dev];
+}
+
 // scratch layout: [status word, 1 KB | two bf16 limbs of X]
 static const size_t GEMM_HDR = 1024;
 static size_t gemm_limb_bytes(int T, int K) { return ((size_t)2 * T * K * sizeof(bf16) + 1023) / 1024 * 1024; }
@@ -1436,9 +1474,38 @@ size_t specvla_gemm_scratch_bytes(int T, int N, int K) {
   return GEMM_HDR + gemm_limb_bytes(T, K);
 }
 
-int specvla_gemm(const float *X, const void *W, float *Y, int T, int N, int K, void *scratch,
-                 size_t scratch_bytes, void *stream) {
-  if (!X || !W || !Y || !scratch || T < 1 || N < 4 || (N % 4) || K < 8 || (K % 8)) return SPECVLA_ERR_INVALID_ARG;
+// Test hook of the next stand-alone GEMM call (specvla_gemm_fault_test): wait limit and the K
+// block its producers withhold. Process-wide, consumed by one call.
+static unsigned long long g_gemm_wait_ns = gemm_tc::WAIT_LIMIT_NS;
+static int g_gemm_withhold = 0;
+
+int specvla_gemm_fault_test(long long wait_limit_ns, int withhold_k_block) {
+  if (wait_limit_ns < 1000 || withhold_k_block < -1) return SPECVLA_ERR_INVALID_ARG;
+  g_gemm_wait_ns = (unsigned long long)wait_limit_ns;
+  g_gemm_withhold = withhold_k_block + 1;
+  return SPECVLA_OK;
+}
+
+size_t specvla_packed_weight_bytes(int N, int K) {
+  if (N < 4 || (N % 4) || K < 8 || (K % 8)) return 0;
+  return gemm_tc::packed_elems((N + SV_TILE_ROWS - 1) / SV_TILE_ROWS, K) * sizeof(bf16);
+}
+
+int specvla_pack_weights(const void *W, int N, int K, void *packed, size_t packed_bytes, void *stream) {
+  if (!W || !packed || (reinterpret_cast<uintptr_t>(packed) % 1024) != 0) return SPECVLA_ERR_INVALID_ARG;
+  const size_t need = specvla_packed_weight_bytes(N, K);
+  if (need == 0) return SPECVLA_ERR_INVALID_ARG;
+  if (packed_bytes < need) return SPECVLA_ERR_CAPACITY;
+  const int tiles = (N + SV_TILE_ROWS - 1) / SV_TILE_ROWS, KB = (K + gemm_tc::BK - 1) / gemm_tc::BK;
+  gemm_tc::pack_weights_kernel<<<148 * 8, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const bf16 *>(W), N, K, tiles, KB, 0, N / 2, static_cast<bf16 *>(packed));
+  return cudaGetLastError() == cudaSuccess ? SPECVLA_OK : SPECVLA_ERR_CUDA;
+}
+
+// W (row-major) or Wp (repacked) is given, never both.
+static int gemm_entry(const float *X, const void *W, const void *Wp, float *Y, int T, int N, int K, void *scratch,
+                      size_t scratch_bytes, void *stream) {
+  if (!X || (!W && !Wp) || !Y || !scratch || T < 1 || N < 4 || (N % 4) || K < 8 || (K % 8)) return SPECVLA_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(scratch) % 1024) != 0) return SPECVLA_ERR_INVALID_ARG;
   if (scratch_bytes < specvla_gemm_scratch_bytes(T, N, K)) return SPECVLA_ERR_CAPACITY;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -1449,8 +1516,8 @@ int specvla_gemm(const float *X, const void *W, float *Y, int T, int N, int K, v
   // the status word starts at zero
   if (cudaMemsetAsync(base, 0, GEMM_HDR, st) != cudaSuccess) return SPECVLA_ERR_CUDA;
   epi::split_limbs_kernel<<<(unsigned)((nx + 255) / 256), 256, 0, st>>>(X, nx, limbs);
-  CUtensorMap mw, mx[4];
-  if (!gemm_tc::make_w_map(&mw, static_cast<const bf16 *>(W), N, K)) return SPECVLA_ERR_CUDA;
+  CUtensorMap mw = {}, mx[4];
+  if (W && !gemm_tc::make_w_map(&mw, static_cast<const bf16 *>(W), N, K)) return SPECVLA_ERR_CUDA;
   const int tns[4] = {16, 32, 64, 128};
   for (int i = 0; i < 4; i++)
     if (!gemm_tc::make_x_map(&mx[i], limbs, nx, T, K, tns[i])) return SPECVLA_ERR_CUDA;
@@ -1461,7 +1528,12 @@ int specvla_gemm(const float *X, const void *W, float *Y, int T, int N, int K, v
   ea.N = N;
   ea.out = Y;
   ea.ldo = N;
-  static const gemm_ck::ClusterFit fit = gemm_ck::query_cluster_fit();
+  ea.wpacked = static_cast<const bf16 *>(Wp);
+  ea.wait_ns = g_gemm_wait_ns;
+  ea.withhold_unit = g_gemm_withhold;
+  g_gemm_wait_ns = gemm_tc::WAIT_LIMIT_NS;           // the test hook holds for one call
+  g_gemm_withhold = 0;
+  const gemm_ck::ClusterFit fit = cluster_fit_of_current_device();
   const int chunks = (T + gemm_tc::MAX_T - 1) / gemm_tc::MAX_T;
   const int S = gemm_ck::slices_for(tiles * chunks, KB, fit);
   ea.row0 = 0;
@@ -1471,6 +1543,18 @@ int specvla_gemm(const float *X, const void *W, float *Y, int T, int N, int K, v
                       false) != cudaSuccess)
     return SPECVLA_ERR_CUDA;
   return cudaGetLastError() == cudaSuccess ? SPECVLA_OK : SPECVLA_ERR_CUDA;
+}
+
+int specvla_gemm(const float *X, const void *W, float *Y, int T, int N, int K, void *scratch,
+                 size_t scratch_bytes, void *stream) {
+  if (!W) return SPECVLA_ERR_INVALID_ARG;
+  return gemm_entry(X, W, nullptr, Y, T, N, K, scratch, scratch_bytes, stream);
+}
+
+int specvla_gemm_prepacked(const float *X, const void *Wpacked, float *Y, int T, int N, int K, void *scratch,
+                           size_t scratch_bytes, void *stream) {
+  if (!Wpacked) return SPECVLA_ERR_INVALID_ARG;
+  return gemm_entry(X, nullptr, Wpacked, Y, T, N, K, scratch, scratch_bytes, stream);
 }
 
 // ------------------------------------------------------------------ GEMM without allocation
@@ -1489,16 +1573,34 @@ int specvla_gemm_static(const float *X, const void *W, float *Y, int T, int N, i
   if (need > (size_t)SPECVLA_STATIC_SCRATCH_BYTES) return SPECVLA_ERR_CAPACITY;
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SPECVLA_ERR_CUDA;
-  if (!g_static_scratch_addr[dev]) {
-    void *p = nullptr;
-    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return SPECVLA_ERR_CUDA;
-    g_static_scratch_addr[dev] = p;
+  void *addr = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
+    if (!g_static_scratch_addr[dev]) {
+      void *p = nullptr;
+      if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return SPECVLA_ERR_CUDA;
+      g_static_scratch_addr[dev] = p;
+    }
+    addr = g_static_scratch_addr[dev];
   }
-  const uintptr_t base = (reinterpret_cast<uintptr_t>(g_static_scratch_addr[dev]) + 1023) & ~(uintptr_t)1023;
+  const uintptr_t base = (reinterpret_cast<uintptr_t>(addr) + 1023) & ~(uintptr_t)1023;
   void *scratch = reinterpret_cast<void *>(base);
   const int rc = specvla_gemm(X, W, Y, T, N, K, scratch, SPECVLA_STATIC_SCRATCH_BYTES, stream);
   if (rc != SPECVLA_OK || !wait) return rc;
   return specvla_gemm_status(scratch, stream);
+}
+
+int specvla_gemm_static_status(void *stream) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SPECVLA_ERR_CUDA;
+  void *addr = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
+    addr = g_static_scratch_addr[dev];
+  }
+  if (!addr) return SPECVLA_ERR_BAD_STATE;            // specvla_gemm_static has not run on this device
+  const uintptr_t base = (reinterpret_cast<uintptr_t>(addr) + 1023) & ~(uintptr_t)1023;
+  return specvla_gemm_status(reinterpret_cast<const void *>(base), stream);
 }
 
 int specvla_gemm_status(const void *scratch, void *stream) {

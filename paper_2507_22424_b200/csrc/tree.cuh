@@ -34,46 +34,6 @@ __global__ void build_verify_rows_kernel(EpArgs a, DevTree *trees, const EpState
   if (threadIdx.x == 0 && tr.tok[0] < 0) tr.tok[0] = st[e].root;
 }
 
-// ---------------------------------------------------------------------------------------
-// Draft catch-up rows: the (feature_j, token_j) pairs pending since the last commit run at
-// draft positions Pd + j, causal among themselves. Advances Pd and opens a new tree whose
-// root is the episode's last emitted token. One thread per episode.
-__global__ void build_catchup_rows_kernel(EpArgs a, EpState *st, DevTree *trees, RowTable rt,
-                                          int *__restrict__ feat_src) {
-  pdl_launch();
-  pdl_wait();
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= a.n_ep) return;
-  const int e = a.eps[i];
-  EpState &s = st[e];
-  for (int j = 0; j < s.n_pending; j++) {
-    const int r = a.row0[i] + j;
-    rt.tok[r] = s.pending_tok[j];
-    rt.src[r] = 0;
-    rt.ep[r] = e;
-    rt.pos[r] = s.Pd + j;
-    rt.slot[r] = s.Pd + j;
-    rt.nvis[r] = s.Pd + j + 1;
-    rt.tbase[r] = 0;
-    for (int w = 0; w < 4; w++) rt.mask[r * 4 + w] = 0;
-    feat_src[r] = e * SV_MAX_PENDING + j;          // row of the pending-feature buffer
-  }
-  s.Pd += s.n_pending;
-  DevTree &tr = trees[e];
-  tr.n_rows = 1;
-  tr.n_drows = 1;
-  tr.tok[0] = s.root;
-  tr.parent[0] = -1;
-  tr.depth[0] = 0;
-  tr.score[0] = 0.f;
-  tr.drow[0] = 0;
-  for (int w = 0; w < 4; w++) tr.dmask[0][w] = 0;
-  tr.level_begin = 0;
-  tr.level_end = 1;
-  tr.sel_count = 1;
-  tr.sel[0] = 0;
-}
-
 // RMSNorm scale of a residual row from its partial sums of squares ssq[row][0..nt).
 __device__ __forceinline__ float norm_scale(const float *__restrict__ ssq, int nt, size_t row, int d, float eps) {
   float ss = 0.f;
@@ -108,32 +68,6 @@ __global__ void draft_input_kernel(RowTable rt, const int *__restrict__ feat_src
     *reinterpret_cast<uint2 *>(xin + (size_t)r * 2 * d + d + i) = *reinterpret_cast<const uint2 *>(e + i);
     *reinterpret_cast<uint2 *>(xin + plane + (size_t)r * 2 * d + d + i) = make_uint2(0u, 0u);
   }
-}
-
-// Saves the draft outputs of the rows just run: dout[e][drow] = x[row]. For the catch-up
-// call only each episode's last row is kept, as draft row 0.
-__global__ void save_draft_out_kernel(const float *__restrict__ x, const int *__restrict__ dst_row,
-                                      int d, float *__restrict__ dout) {
-  pdl_launch();
-  pdl_wait();
-  const int r = blockIdx.x;
-  const int dst = dst_row[r];
-  if (dst < 0) return;
-#pragma unroll 2
-  for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4)
-    *reinterpret_cast<float4 *>(dout + (size_t)dst * d + i) = *reinterpret_cast<const float4 *>(x + (size_t)r * d + i);
-}
-
-// dst_row for the catch-up call: last pending row of episode i -> dout row e * SV_MAX_TREE.
-__global__ void catchup_dst_kernel(EpArgs a, int *__restrict__ dst_row, int *__restrict__ lm_rows) {
-  pdl_launch();
-  pdl_wait();
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= a.n_ep) return;
-  for (int j = 0; j < a.nrows[i]; j++) dst_row[a.row0[i] + j] = -1;
-  const int last = a.row0[i] + a.nrows[i] - 1;
-  dst_row[last] = a.eps[i] * SV_MAX_TREE;
-  lm_rows[i] = last;
 }
 
 // [feature ; embedding] row r of the draft model's input: the feature is an fp32 row (split
@@ -277,73 +211,6 @@ grow_input_kernel(EpArgs a, int level, int branch, int expand_next, const int *_
   __syncthreads();
   for (int j = 0; j < s_cnt; j++)
     write_draft_input_row(x + (size_t)s_src[j] * d, E + (size_t)s_tokn[j] * d, d, xin, plane, a.aux[i] + j);
-}
-
-// One level of tree growth. The rows scored last (one per selected parent, in rank order)
-// come with their top-K tokens and log-probabilities; parent sel[j] gets `branch` children
-// (score = parent score + log-prob). Then the `expand_next` best new nodes (by score, ties
-// to the lower node index) are selected, in rank order, and their draft rows are laid out
-// for the next level: input feature = output of the row that scored them, token = their own.
-// One thread per episode (at most 64 nodes per level, 16 of them expanded).
-// a.row0 = first scored row of each episode, a.aux = first row of its next level.
-__global__ void expand_level_kernel(EpArgs a, int level, int branch, int expand_next,
-                                    const int *__restrict__ top_tok, const float *__restrict__ top_lp,
-                                    DevTree *trees, const EpState *__restrict__ st, RowTable rt,
-                                    int *__restrict__ feat_src, int *__restrict__ dst_row) {
-  pdl_launch();
-  pdl_wait();
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= a.n_ep) return;
-  const int e = a.eps[i];
-  DevTree &tr = trees[e];
-  const int begin = tr.n_rows;
-  for (int j = 0; j < tr.sel_count; j++) {
-    const int p = tr.sel[j];
-    const int srow = a.row0[i] + j;
-    for (int b = 0; b < branch; b++) {
-      const int n = tr.n_rows++;
-      tr.tok[n] = top_tok[srow * SV_TOPK + b];
-      tr.parent[n] = p;
-      tr.depth[n] = level + 1;
-      tr.score[n] = tr.score[p] + top_lp[srow * SV_TOPK + b];
-      tr.drow[n] = -1;
-    }
-  }
-  tr.level_begin = begin;
-  tr.level_end = tr.n_rows;
-  // selection of the next level's parents: repeated arg-best (<= 16 x 64 comparisons)
-  int cnt = 0;
-  unsigned long long used = 0;
-  for (; cnt < expand_next && cnt < tr.level_end - begin; cnt++) {
-    int best = -1;
-    for (int n = begin; n < tr.level_end; n++) {
-      if (used & (1ull << (n - begin))) continue;
-      if (best < 0 || tr.score[n] > tr.score[best]) best = n;
-    }
-    used |= 1ull << (best - begin);
-    tr.sel[cnt] = best;
-  }
-  tr.sel_count = cnt;
-  const int Pd = st[e].Pd;
-  for (int j = 0; j < cnt; j++) {
-    const int n = tr.sel[j];
-    const int dr = tr.n_drows++;
-    const int pdr = tr.drow[tr.parent[n]];
-    tr.drow[n] = dr;
-    for (int w = 0; w < 4; w++) tr.dmask[dr][w] = tr.dmask[pdr][w];
-    tr.dmask[dr][dr >> 5] |= 1u << (dr & 31);
-    const int r = a.aux[i] + j;
-    rt.tok[r] = tr.tok[n];
-    rt.src[r] = 0;
-    rt.ep[r] = e;
-    rt.pos[r] = Pd - 1 + level + 1;
-    rt.slot[r] = Pd - 1 + dr;              // draft row dr >= 1 -> slot Pd + (dr - 1)
-    rt.nvis[r] = Pd;
-    rt.tbase[r] = Pd - 1;                  // bit dr of dmask <-> slot Pd - 1 + dr
-    for (int w = 0; w < 4; w++) rt.mask[r * 4 + w] = tr.dmask[dr][w];
-    feat_src[r] = e * SV_MAX_TREE + pdr;   // row of dout
-    dst_row[r] = e * SV_MAX_TREE + dr;
-  }
 }
 
 // ---------------------------------------------------------------------------------------

@@ -233,15 +233,20 @@ def test_c4_sixteen_ragged_episodes(env):
     assert tally.accepts == tally.caches == 2
 
 
-@pytest.mark.parametrize("T,N,K", [(27, 22016, 4096), (27, 4096, 11008), (128, 12288, 4096),
-                                   (27, 32064, 4096), (290, 4096, 4096)])
-def test_gemm_full_size_sampled_outputs(T, N, K):
-    """7B-shaped GEMMs: 256 sampled outputs recomputed one by one in float64."""
-    from paper_2507_22424_b200.binding import gemm
+@pytest.mark.parametrize("T,N,K,packed", [(27, 22016, 4096, False), (27, 4096, 11008, False),
+                                          (128, 12288, 4096, False), (27, 32064, 4096, False),
+                                          (290, 4096, 4096, False), (27, 22016, 4096, True),
+                                          (27, 4096, 11008, True), (27, 32064, 4096, True),
+                                          (290, 12288, 4096, True)])
+def test_gemm_full_size_sampled_outputs(T, N, K, packed):
+    """7B-shaped GEMMs: 256 sampled outputs recomputed one by one in float64. `packed`: through
+    the repacked weights and plain bulk copies, the path the decoder itself uses; else through the
+    strided tensor-map boxes over the caller's row-major matrix."""
+    from paper_2507_22424_b200.binding import gemm, gemm_prepacked, pack_weights
     from synth_inputs import rng
     x = rng.normal(21, 1, (T, K), 1.0, "cuda", dtype=torch.float32)
     w = rng.normal_bf16(21, 2, (N, K), 0.02, "cuda")
-    y = gemm(x, w).cpu()
+    y = (gemm_prepacked(x, pack_weights(w), N) if packed else gemm(x, w)).cpu()
     ts = rng.integers(21, 3, 256, 0, T).tolist()
     ns = rng.integers(21, 4, 256, 0, N).tolist()
     ns[:4] = [0, N - 1, N - 64, 127]

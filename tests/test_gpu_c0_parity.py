@@ -41,6 +41,51 @@ def test_gemm_matches_float64_matmul(T, N, K):
     assert (y - ref).abs().max() < tol, float((y - ref).abs().max())
 
 
+@pytest.mark.parametrize("T,N,K", [(1, 256, 256), (15, 1376, 256), (33, 1000, 1024), (130, 384, 520), (9, 16384, 768)])
+def test_prepacked_gemm_matches_float64_matmul(T, N, K):
+    """The same product through the library's repacked weights (the decoder's own path)."""
+    from paper_2507_22424_b200.binding import gemm_prepacked, pack_weights
+    x = rng.normal(12, 1, (T, K), 1.0, dtype=torch.float32)
+    w = rng.normal_bf16(12, 2, (N, K), 0.02)
+    ref = x.double() @ w.double().T
+    y = gemm_prepacked(x.cuda(), pack_weights(w.cuda()), N).cpu().double()
+    tol = 1e-4 * 0.02 * (K ** 0.5) + 1e-6
+    assert (y - ref).abs().max() < tol, float((y - ref).abs().max())
+
+
+def test_device_side_wait_runs_out_and_the_context_survives():
+    """Failure detection without a fault: the producer of the next GEMM withholds one K block and
+    the wait limit is 2 ms; the kernel must record the failure and RETURN (status word ->
+    SPECVLA_ERR_TIMEOUT), and the very next ordinary call on the same context must be correct."""
+    import ctypes as C
+    from paper_2507_22424_b200 import binding as B
+    T, N, K = 16, 256, 512
+    x = rng.normal(13, 1, (T, K), 1.0, dtype=torch.float32).cuda()
+    w = rng.normal_bf16(13, 2, (N, K), 0.02).cuda()
+    ref = x.cpu().double() @ w.cpu().double().T
+    y = torch.zeros(T, N, dtype=torch.float32, device="cuda")
+    nb = B.lib.specvla_gemm_scratch_bytes(T, N, K)
+    scratch = torch.empty(nb + 1024, dtype=torch.uint8, device="cuda")
+    sp = (scratch.data_ptr() + 1023) // 1024 * 1024
+    assert B.lib.specvla_gemm_fault_test(2_000_000, 1) == 0          # 2 ms, K block 1 of every CTA's range
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    rc = B.lib.specvla_gemm(C.c_void_p(x.data_ptr()), C.c_void_p(w.data_ptr()), C.c_void_p(y.data_ptr()), T, N, K,
+                            C.c_void_p(sp), nb, B._stream())
+    t1.record()
+    assert rc == 0
+    assert B.lib.specvla_gemm_status(C.c_void_p(sp), B._stream()) == -6   # SPECVLA_ERR_TIMEOUT
+    assert 2.0 <= t0.elapsed_time(t1) < 200.0                          # it waited the limit out, and returned
+    # the hook held for that one call: the next call on the same scratch is an ordinary, correct GEMM
+    got = B.gemm(x, w).cpu().double()
+    assert (got - ref).abs().max() < 1e-4 * 0.02 * (K ** 0.5) + 1e-6
+    rc = B.lib.specvla_gemm(C.c_void_p(x.data_ptr()), C.c_void_p(w.data_ptr()), C.c_void_p(y.data_ptr()), T, N, K,
+                            C.c_void_p(sp), nb, B._stream())
+    assert rc == 0 and B.lib.specvla_gemm_status(C.c_void_p(sp), B._stream()) == 0
+    assert (y.cpu().double() - ref).abs().max() < 1e-4 * 0.02 * (K ** 0.5) + 1e-6
+
+
 @pytest.mark.parametrize("action_only", [True, False])
 def test_prefill_logits_and_first_token(c0, wcuda, action_only):
     orc = c0["make"](action_only=action_only)

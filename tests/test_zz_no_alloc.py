@@ -44,3 +44,19 @@ def test_static_scratch_gemm_rejects_oversize():
     with pytest.raises(B.SpecVLAError) as e:
         B.gemm_static(x, w, y)
     assert e.value.code == -2
+
+
+def test_static_scratch_gemm_asynchronous_then_status():
+    """wait = 0 (the form a stream capture needs): the call returns at once; the status of the
+    built-in scratch is asked for afterwards."""
+    import ctypes as C
+    from paper_2507_22424_b200 import binding as B
+    T, N, K = 27, 1024, 1024
+    x, w = _case(41, T, N, K)
+    y = torch.full((T, N), float("nan"), dtype=torch.float32, device="cuda")
+    rc = B.lib.specvla_gemm_static(C.c_void_p(x.data_ptr()), C.c_void_p(w.data_ptr()), C.c_void_p(y.data_ptr()),
+                                   T, N, K, 0, B._stream())
+    assert rc == 0
+    assert B.lib.specvla_gemm_static_status(B._stream()) == 0
+    want = B.gemm(x, w).cpu().double()
+    assert (y.cpu().double() - want).abs().max() < 1e-4 * 0.02 * (K ** 0.5) + 1e-6
