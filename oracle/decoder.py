@@ -36,7 +36,12 @@ class DecoderWeights:
         self.dtype = dtype
 
     def __call__(self, name: str) -> torch.Tensor:
-        return self.raw[name].to(device="cpu", dtype=self.dtype)
+        raw = self.raw[name]
+        if isinstance(raw, tuple):
+            # a quantised matrix (oracle/quant.py): int8 codes and one float32 scale per output row
+            q, scale = raw
+            return q.to(device="cpu", dtype=self.dtype) * scale.to(device="cpu", dtype=self.dtype)[:, None]
+        return raw.to(device="cpu", dtype=self.dtype)
 
 
 def rmsnorm(x: torch.Tensor, gain: torch.Tensor, eps: float) -> torch.Tensor:
@@ -114,8 +119,8 @@ def target_forward(w: DecoderWeights, desc, x, pos, slots, visible, cache: KVCac
     return rmsnorm(x, w("final_norm"), desc.rms_eps)
 
 
-def lm_head(w: DecoderWeights, features: torch.Tensor) -> torch.Tensor:
-    return features @ w("lm_head").T
+def lm_head(w: DecoderWeights, features: torch.Tensor, name: str = "lm_head") -> torch.Tensor:
+    return features @ w(name).T
 
 
 def draft_forward(w: DecoderWeights, desc, feat_in, emb_in, pos, slots, visible, cache: KVCache):

@@ -240,7 +240,9 @@ class SpecVLAOracle:
                     produced_by[n] = out[t]
             nxt = []
             for n in ranked:
-                logits = D.lm_head(self.w, produced_by[n][None, :])[0]
+                # the draft model scores with its own copy of the LM head when the target's is quantised
+                head = "draft.lm_head" if "draft.lm_head" in self.w.raw else "lm_head"
+                logits = D.lm_head(self.w, produced_by[n][None, :], head)[0]
                 if self.action_only:
                     lp_all = torch.log_softmax(logits[a0:a0 + nb], dim=0)
                     base = a0
