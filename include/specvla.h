@@ -61,6 +61,14 @@ typedef struct {
   int max_episodes;     /* episodes with their own KV caches */
   int max_rows;         /* rows of one forward call summed over its episodes (prefill sets this) */
   int action_only;      /* 1: greedy argmax and draft top-k range over the action ids only */
+  int weight_bits;      /* 0 or 16: the target's matrices are streamed as given (bf16). 8: quantised
+                         * target (Appendix C): at creation the four matrices of every target layer and
+                         * the LM head are quantised to int8, per output row, symmetric: scale =
+                         * max|w| / 127 (1 for a zero row), code = round-half-even(w / scale) in
+                         * [-127, 127], both in float32; the kernels stream the codes (half the bytes),
+                         * expand them to bf16 in shared memory and apply the scale to the accumulator.
+                         * Embedding, norms and the draft model (with the original LM-head rows it
+                         * scores with) are not quantised. The paper does not specify its scheme. */
 } specvla_model_desc;
 
 /* Target (verification) model weights. Per-layer members are HOST arrays of n_layers DEVICE

@@ -23,7 +23,7 @@ class ModelDesc(C.Structure):
     _fields_ = [(n, C.c_int) for n in ("n_layers", "d_model", "n_heads", "head_dim", "d_ffn", "vocab",
                                        "action_base", "n_bins")] + \
                [("rms_eps", C.c_float), ("rope_theta", C.c_float)] + \
-               [(n, C.c_int) for n in ("max_seq", "max_episodes", "max_rows", "action_only")]
+               [(n, C.c_int) for n in ("max_seq", "max_episodes", "max_rows", "action_only", "weight_bits")]
 
 
 class Weights(C.Structure):
@@ -135,11 +135,12 @@ def make_shape(branch, expand, prune: bool = False, keep: int = 0) -> TreeShape:
 class SpecVLA:
     """One library context over weights held in torch CUDA tensors (kept alive here)."""
 
-    def __init__(self, desc, weights: dict, max_seq=512, max_episodes=1, max_rows=512, action_only=True):
+    def __init__(self, desc, weights: dict, max_seq=512, max_episodes=1, max_rows=512, action_only=True,
+                 weight_bits=16):
         self.model = desc
         self.md = ModelDesc(desc.n_layers, desc.d_model, desc.n_heads, desc.head_dim, desc.d_ffn, desc.vocab,
                             desc.action_base, desc.n_bins, desc.rms_eps, desc.rope_theta,
-                            max_seq, max_episodes, max_rows, int(action_only))
+                            max_seq, max_episodes, max_rows, int(action_only), int(weight_bits))
         self.w = weights
         L = desc.n_layers
 

@@ -48,7 +48,7 @@ __device__ __forceinline__ void cluster_sync_all() {
 __host__ __device__ constexpr int ck_tmem_cols(int TN) { return 2 * acc_width(TN) < 32 ? 32 : 2 * acc_width(TN); }
 
 // EpiArgs as in gemm_tc: the mode is a template parameter. KB = K blocks per tile.
-template <int TN, int MODE>
+template <int TN, int MODE, bool Q8>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                const __grid_constant__ CUtensorMap tmXtail, const EpiArgs ea, const int KB,
@@ -63,6 +63,8 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
   const uint32_t tfull_bar = bars + 8u * (2 * STAGES);
   const uint32_t tmem_slot = bars + 8u * (2 * STAGES + 1);
+  // Q8: the stage's weight tile has been expanded from int8 codes to bf16 by the epilogue warps
+  auto conv_bar = [&](int s) { return bars + 8u * (2 * STAGES + 2 + s); };
   __shared__ float s_scale[MAX_T];
   __shared__ int s_pos[MAX_T], s_slot[MAX_T], s_ep[MAX_T];
   // RoPE factors of the CTA's rows (EPI_QKV, up to 32 rows of up to 64 pairs): fetched while the
@@ -91,7 +93,8 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   const bool tail = TN == MAX_T && blockIdx.y == gridDim.y - 1;
   const int tn = tail ? ea.tn_tail : TN;
   const CUtensorMap *xmap = tail ? &tmXtail : &tmX;
-  const uint32_t stage_tx = (uint32_t)(W_STAGE_BYTES + 2 * tn * BK * 2);
+  constexpr int W_LOAD_BYTES = Q8 ? W_STAGE_BYTES / 2 : W_STAGE_BYTES;   // int8 codes: half the bytes from HBM
+  const uint32_t stage_tx = (uint32_t)(W_LOAD_BYTES + 2 * tn * BK * 2);
   const uint32_t idesc = instr_desc(2 * tn);
 
   const int npre = n_units < STAGES ? n_units : STAGES;
@@ -103,7 +106,11 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     const int st = it % STAGES;
     const uint32_t sW = base + st * STAGE;
     mbar_expect_tx(full_bar(st), stage_tx);
-    if (ea.wpacked) {
+    if (Q8) {
+      // the codes of the 256 x 64 tile land in the upper half of the stage's weight area and are
+      // expanded in place (epilogue warps, below)
+      bulk_load(sW + W_STAGE_BYTES / 2, ea.wq8 + (size_t)(u0 + it) * (BM * BK), W_STAGE_BYTES / 2, full_bar(st), pol_w);
+    } else if (ea.wpacked) {
       bulk_load(sW, ea.wpacked + (size_t)(u0 + it) * (BM * BK), W_STAGE_BYTES, full_bar(st), pol_w);
     } else {
       // the two 128-row halves of the tile: consecutive rows, or gate rows + up rows
@@ -119,6 +126,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     for (int s = 0; s < STAGES; s++) {
       mbar_init(full_bar(s), 1);
       mbar_init(empty_bar(s), 1);
+      if (Q8) mbar_init(conv_bar(s), 1);
     }
     mbar_init(tfull_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -166,7 +174,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     if (lane == 0 && n_units > 0) {
       for (int it = 0; it < n_units; it++) {
         const int st = it % STAGES, rnd = it / STAGES;
-        if (!mbar_wait(full_bar(st), rnd & 1, ea.wait_ns)) {
+        if (!mbar_wait(Q8 ? conv_bar(st) : full_bar(st), rnd & 1, ea.wait_ns)) {
           atomicExch(err, SV_ERR_WAIT_FULL);
           break;
         }
@@ -223,6 +231,48 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         s_rope[t * ROPE_HALF + j] = ea.rope_tab[(size_t)s_pos[t] * half + j];
       }
     }
+    if (Q8) {
+      // int8 -> bf16 expansion of every stage as it lands: thread et owns row et of the tile (64
+      // codes = 64 bytes in, one 128-byte swizzled row out). All rows are read before any is
+      // written: the rows of the second half overwrite the code area.
+      for (int it = 0; it < n_units; it++) {
+        const int st = it % STAGES, rnd = it / STAGES;
+        const bool mine = mbar_wait(full_bar(st), rnd & 1, ea.wait_ns);
+        if (lane == 0) s_flag[warp - 2] = mine ? 1 : 0;
+        const uint32_t sW = base + st * STAGE;
+        uint32_t c[16];
+#pragma unroll
+        for (int i = 0; i < 4; i++)
+          asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                       : "=r"(c[4 * i]), "=r"(c[4 * i + 1]), "=r"(c[4 * i + 2]), "=r"(c[4 * i + 3])
+                       : "r"(sW + W_STAGE_BYTES / 2 + et * 64 + i * 16) : "memory");
+        epi_barrier();
+        if (!(s_flag[0] && s_flag[1] && s_flag[2] && s_flag[3] && s_flag[4] && s_flag[5] && s_flag[6] && s_flag[7])) {
+          if (et == 0) atomicExch(err, SV_ERR_WAIT_FULL);
+          epi_barrier();                                   // the flags have been read by everybody
+          break;
+        }
+#pragma unroll
+        for (int ch = 0; ch < 8; ch++) {
+          // codes 8 ch .. 8 ch + 7 of the row: two words -> eight bf16 (exact: |code| <= 127)
+          uint32_t o[4];
+#pragma unroll
+          for (int h = 0; h < 2; h++) {
+            const uint32_t w = c[2 * ch + h];
+            const float f0 = (float)(int)(signed char)(w & 0xff), f1 = (float)(int)(signed char)((w >> 8) & 0xff);
+            const float f2 = (float)(int)(signed char)((w >> 16) & 0xff), f3 = (float)(int)(signed char)(w >> 24);
+            const __nv_bfloat162 lo = __floats2bfloat162_rn(f0, f1), hi = __floats2bfloat162_rn(f2, f3);
+            o[2 * h] = *reinterpret_cast<const uint32_t *>(&lo);
+            o[2 * h + 1] = *reinterpret_cast<const uint32_t *>(&hi);
+          }
+          asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(sW + et * 128 + ((ch ^ (et & 7)) << 4)), "r"(o[0]),
+                       "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> tensor-core reads
+        epi_barrier();
+        if (et == 0) mbar_arrive(conv_bar(st));
+      }
+    }
     bool have = n_units > 0;
     if (have) {
       const bool mine = mbar_wait(tfull_bar, 0, ea.wait_ns);
@@ -273,7 +323,9 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       const int pk0 = r * ea.pf_KB / ea.pf_S;
       int n = (r + 1) * ea.pf_KB / ea.pf_S - pk0;
       if (n > ea.pf_units) n = ea.pf_units;
-      if (n > 0) prefetch_l2(ea.pf_w + ((size_t)ptile * ea.pf_KB + pk0) * (BM * BK), (uint32_t)n * W_STAGE_BYTES);
+      if (n > 0)
+        prefetch_l2(static_cast<const char *>(ea.pf_w) + ((size_t)ptile * ea.pf_KB + pk0) * ea.pf_unit_bytes,
+                    (uint32_t)(n * ea.pf_unit_bytes));
     }
   }
 
@@ -320,6 +372,15 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         }
       return acc;
     };
+    // Q8: the accumulators are sums over integer codes; every output column takes the scale of its
+    // weight row (the rotation partner and the up projection have theirs)
+    float4 ws = make_float4(1.f, 1.f, 1.f, 1.f), ws2 = ws;
+    if (Q8 && col_ok) {
+      ws = *reinterpret_cast<const float4 *>(ea.wscale + n);
+      if (rot) ws2 = *reinterpret_cast<const float4 *>(ea.wscale + n + (lo ? half : -half));
+      if (swiglu) ws2 = *reinterpret_cast<const float4 *>(ea.wscale + ea.up_off + n);
+    }
+    auto scaled = [](float4 v, const float4 &w) { return make_float4(v.x * w.x, v.y * w.y, v.z * w.z, v.w * w.w); };
     int iter = 0;
     for (int t = rank + rg * S; t < T; t += RG * S, iter++) {
       const size_t row = (size_t)(row0 + t);
@@ -337,6 +398,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       }
       const int slot = MODE == EPI_QKV ? s_slot[t] : 0, ep = MODE == EPI_QKV ? s_ep[t] : 0;
       float4 v = partial_sum(t * BM + c4);
+      if (Q8) v = scaled(v, ws);
       if (MODE == EPI_PLAIN) {
         const float4 ov = make_float4(sc * v.x, sc * v.y, sc * v.z, sc * v.w);
         if (ea.out && col_ok) *reinterpret_cast<float4 *>(ea.out + row * ea.ldo + n) = ov;
@@ -418,7 +480,8 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         // the partner columns of the rotation (dh / 2 away) are in the same tile
         float4 o = make_float4(sc * v.x, sc * v.y, sc * v.z, sc * v.w);
         if (rot) {
-          const float4 w = partial_sum(t * BM + c4 + (lo ? half : -half));
+          float4 w = partial_sum(t * BM + c4 + (lo ? half : -half));
+          if (Q8) w = scaled(w, ws2);
           const float sg = lo ? -sc : sc;
           o.x = o.x * cs01.x + sg * w.x * cs01.y;
           o.y = o.y * cs01.z + sg * w.y * cs01.w;
@@ -432,7 +495,8 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           *reinterpret_cast<float4 *>(dst) = o;
         }
       } else if (swiglu) {
-        const float4 u = partial_sum(t * BM + 128 + c4);
+        float4 u = partial_sum(t * BM + 128 + c4);
+        if (Q8) u = scaled(u, ws2);
         if (col_ok) {
           const float gx = sc * v.x, gy = sc * v.y, gz = sc * v.z, gw = sc * v.w;
           store_limbs4(ea.hid, ea.hid_plane, row * ea.N + n,
@@ -484,11 +548,11 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   if (warp == 1) tc_dealloc(tmem_base, ck_tmem_cols(TN));
 }
 
-template <int TN, int MODE>
-inline cudaError_t launch_tm(const CUtensorMap &tmW, const CUtensorMap &tmX, const CUtensorMap &tmXtail,
+template <int TN, int MODE, bool Q8>
+inline cudaError_t launch_tq(const CUtensorMap &tmW, const CUtensorMap &tmX, const CUtensorMap &tmXtail,
                              const EpiArgs &ea, int tiles, int KB, int S, int *err, cudaStream_t st, bool pdl) {
   // per device and cheap: set on every launch, so that every device of the process has it
-  cudaError_t e = cudaFuncSetAttribute(gemm_ck_kernel<TN, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(gemm_ck_kernel<TN, MODE, Q8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        smem_bytes(TN));
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
@@ -505,7 +569,15 @@ inline cudaError_t launch_tm(const CUtensorMap &tmW, const CUtensorMap &tmX, con
   at[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = pdl ? 2 : 1;
-  return cudaLaunchKernelEx(&cfg, gemm_ck_kernel<TN, MODE>, tmW, tmX, tmXtail, ea, KB, err);
+  return cudaLaunchKernelEx(&cfg, gemm_ck_kernel<TN, MODE, Q8>, tmW, tmX, tmXtail, ea, KB, err);
+}
+// int8 weights (ea.wq8) take the instantiation that expands the codes in shared memory; the draft
+// scoring mode never runs on quantised weights.
+template <int TN, int MODE>
+inline cudaError_t launch_tm(const CUtensorMap &tmW, const CUtensorMap &tmX, const CUtensorMap &tmXtail,
+                             const EpiArgs &ea, int tiles, int KB, int S, int *err, cudaStream_t st, bool pdl) {
+  if (ea.wq8 && MODE != EPI_TOPK) return launch_tq<TN, MODE == EPI_TOPK ? EPI_PLAIN : MODE, true>(tmW, tmX, tmXtail, ea, tiles, KB, S, err, st, pdl);
+  return launch_tq<TN, MODE, false>(tmW, tmX, tmXtail, ea, tiles, KB, S, err, st, pdl);
 }
 
 // The epilogue mode is a template parameter: each instantiation carries only its own finishing
@@ -530,7 +602,7 @@ struct ClusterFit {
 // of an SM's shared memory: one CTA per SM).
 inline ClusterFit query_cluster_fit() {
   ClusterFit f = {};
-  cudaFuncSetAttribute(gemm_ck_kernel<32, EPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(32));
+  cudaFuncSetAttribute(gemm_ck_kernel<32, EPI_RESID, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(32));
   for (int S = 1; S <= MAX_S; S++) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(S * 64);
@@ -544,7 +616,7 @@ inline ClusterFit query_cluster_fit() {
     cfg.attrs = at;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, gemm_ck_kernel<32, EPI_RESID>, &cfg) == cudaSuccess) f.max_active[S] = n;
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_ck_kernel<32, EPI_RESID, false>, &cfg) == cudaSuccess) f.max_active[S] = n;
   }
   cudaGetLastError();
   return f;

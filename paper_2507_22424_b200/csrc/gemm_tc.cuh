@@ -201,13 +201,16 @@ struct EpiArgs {
   unsigned long long wait_ns;   // limit of every mbarrier wait
   int withhold_unit;     // test hook (specvla_gemm_fault_test): > 0: the producer of every CTA skips its
                          // (withhold_unit - 1)-th K block, so the waits for it run out; 0: off
+  const signed char *wq8;   // int8 codes of the weights in the same unit order (16 KB per unit, rows of 64
+                            // codes, not swizzled), or NULL; wscale[n] = scale of weight row n
+  const float *wscale;
   const bf16 *wpacked;   // weights repacked by pack_weights_kernel (one contiguous 32 KB block per
                          // (tile, K block), in unit order); NULL: strided boxes through the W map
   // L2 prefetch for the GEMM that follows: once its own loads are issued, every CTA asks for
   // the first pf_units 32 KB blocks of some of the next GEMM's per-CTA ranges, so that HBM keeps
   // working through this kernel's epilogue, the kernel boundary and the next kernel's start.
-  const bf16 *pf_w;      // packed weights of the next GEMM; NULL: no prefetch
-  int pf_tiles, pf_KB, pf_S, pf_units;
+  const void *pf_w;      // packed weights (or int8 codes) of the next GEMM; NULL: no prefetch
+  int pf_tiles, pf_KB, pf_S, pf_units, pf_unit_bytes;
   // row scale of the RMSNorm in front of this GEMM: rsqrt(sum_j ssq_in[row][j] * inv_k + eps)
   const float *ssq_in;   // [rows][nt_in] partial sums of squares; NULL: scale 1
   int nt_in;
@@ -275,6 +278,53 @@ __global__ void pack_weights_kernel(const bf16 *__restrict__ W, int N, int K, in
     *reinterpret_cast<uint4 *>(out + unit * (BM * BK) + (size_t)r * BK + ((c ^ (r & 7)) << 3)) = v;
   }
 }
+// Weight-only int8 quantisation, per output row (symmetric): scale[n] = max_k |W[n][k]| / 127 (1 for
+// an all-zero row), code = round-half-even(W / scale) clipped to [-127, 127]; scale and quotient in
+// IEEE float32, so that any implementation of the same rule derives the same codes. One warp per row.
+__global__ void row_scale_q8_kernel(const bf16 *__restrict__ W, int N, int K, float *__restrict__ scale) {
+  const int n = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (n >= N) return;
+  float m = 0.f;
+  for (int k = lane; k < K; k += 32) m = fmaxf(m, fabsf(__bfloat162float(W[(size_t)n * K + k])));
+  m = warp_max(m);
+  if (lane == 0) scale[n] = m > 0.f ? __fdiv_rn(m, 127.f) : 1.f;
+}
+// The codes in the GEMM's unit order: one 16 KB block per (tile, K block), 256 rows of 64 codes, rows
+// and tiles as in pack_weights_kernel (swiglu: 128 gate rows, then the 128 matching up rows). Rows and
+// columns past the matrix are zero.
+__global__ void pack_weights_q8_kernel(const bf16 *__restrict__ W, int N, int K, int tiles, int KB, int swiglu,
+                                       int F, const float *__restrict__ scale, signed char *__restrict__ out) {
+  const size_t total = (size_t)tiles * KB * BM * 4;                  // 16 codes per thread step
+  for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+       idx += (size_t)gridDim.x * blockDim.x) {
+    const int c = (int)(idx & 3), r = (int)((idx >> 2) & (BM - 1));
+    const size_t unit = idx >> 10;
+    const int kb = (int)(unit % KB), tile = (int)(unit / KB);
+    int n;
+    bool ok;
+    if (swiglu) {
+      n = (r < 128) ? tile * 128 + r : F + tile * 128 + (r - 128);
+      ok = tile * 128 + (r & 127) < F;
+    } else {
+      n = tile * BM + r;
+      ok = n < N;
+    }
+    const float s = ok ? scale[n] : 1.f;
+    uint32_t words[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+    for (int e = 0; e < 16; e++) {
+      const int k = kb * BK + c * 16 + e;
+      int q = 0;
+      if (ok && k < K) {
+        const float t = __fdiv_rn(__bfloat162float(W[(size_t)n * K + k]), s);
+        q = (int)fminf(fmaxf(rintf(t), -127.f), 127.f);
+      }
+      words[e >> 2] |= (uint32_t)(q & 0xff) << (8 * (e & 3));
+    }
+    *reinterpret_cast<uint4 *>(out + unit * (BM * BK) + (size_t)r * BK + c * 16) = make_uint4(words[0], words[1], words[2], words[3]);
+  }
+}
+
 inline size_t packed_elems(int tiles, int K) { return (size_t)tiles * ((K + BK - 1) / BK) * BM * BK; }
 
 // ------------------------------------------------------------------------- host side

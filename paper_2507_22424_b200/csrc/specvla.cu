@@ -29,6 +29,8 @@ struct WMat {
   bool has_map;
   CUtensorMap map;
   const bf16 *packed;     // the library's repacked copy (gemm_tc::pack_weights_kernel), in the workspace
+  const signed char *q8;  // quantised target: int8 codes in the same unit order (then packed is NULL)
+  const float *scale;     // ... and the scale of every weight row
 };
 // A two-limb activation buffer [2][rows][K] and its TMA maps, one per row-tile size 16/32/64/128.
 struct XBuf {
@@ -89,6 +91,10 @@ struct specvla_ctx {
   int cand_nc;
   bf16 *packed;                 // repacked weight matrices, one after the other
   size_t packed_elems;
+  signed char *packed_q8;       // quantised target: int8 codes of its matrices, one after the other
+  size_t packed_q8_bytes;
+  float *wscale;                // ... and their row scales
+  size_t wscale_elems;
   int lgs_rows;                 // rows of the logits buffer
 
   // GEMM operands, two bf16 limbs each: hi plane, then the lo plane `plane` elements later
@@ -162,6 +168,7 @@ bool desc_ok(const specvla_model_desc *d) {
   if (d->head_dim != 64 && d->head_dim != 128) return false;
   if (d->d_model % 8 || d->d_ffn % 8 || (d->n_heads * d->head_dim) % 8 || d->vocab % 4 || d->n_bins % 4) return false;
   if (d->n_bins < 1 || d->action_base < 0 || d->action_base + d->n_bins > d->vocab) return false;
+  if (d->weight_bits != 0 && d->weight_bits != 8 && d->weight_bits != 16) return false;
   if (d->max_seq < 2 || d->max_episodes < 1 || d->max_episodes > SV_MAX_EP || d->max_rows < 1) return false;
   if (!(d->rms_eps > 0.f) || !(d->rope_theta > 1.f)) return false;
   return true;
@@ -246,10 +253,17 @@ size_t carve(specvla_ctx *c, char *base) {
                          gemm_tc::packed_elems(tiles256(d.d_model), hd) +
                          gemm_tc::packed_elems((d.d_ffn + 127) / 128, d.d_model) +
                          gemm_tc::packed_elems(tiles256(d.d_model), d.d_ffn);
-    c->packed_elems = layer * ((size_t)d.n_layers + 1) + gemm_tc::packed_elems(tiles256(d.vocab), d.d_model) +
-                      gemm_tc::packed_elems(tiles256(d.n_bins), d.d_model) +
-                      gemm_tc::packed_elems(tiles256(d.d_model), 2 * d.d_model);
+    const size_t lm = gemm_tc::packed_elems(tiles256(d.vocab), d.d_model);
+    const size_t draft = layer + gemm_tc::packed_elems(tiles256(d.n_bins), d.d_model) +
+                         gemm_tc::packed_elems(tiles256(d.d_model), 2 * d.d_model);
+    const bool q8 = d.weight_bits == 8;
+    // quantised target: its matrices are kept as int8 codes (one byte per element) plus row scales
+    c->packed_elems = draft + (q8 ? 0 : layer * (size_t)d.n_layers + lm);
     c->packed = cv.take<bf16>(c->packed_elems);
+    c->packed_q8_bytes = q8 ? layer * (size_t)d.n_layers + lm : 0;
+    c->packed_q8 = cv.take<signed char>(c->packed_q8_bytes);
+    c->wscale_elems = q8 ? (size_t)d.n_layers * (3 * hd + 2 * d.d_model + 2 * d.d_ffn) + d.vocab : 0;
+    c->wscale = cv.take<float>(c->wscale_elems);
   }
   // full-vocabulary logits are stored only for the draft model's top-k when it ranges over the
   // whole vocabulary (action_only = 0); the greedy argmax works from per-128-column candidates
@@ -279,7 +293,7 @@ size_t carve(specvla_ctx *c, char *base) {
   c->trees = cv.take<DevTree>(E);
   c->err = cv.take<int>(32);
   // persistent forward kernel: packed operands, partial tiles, attention slices, candidates
-  if (pk_shapes_ok(d)) {
+  if (pk_shapes_ok(d) && d.weight_bits != 8) {
     const size_t G = c->pk_G;
     auto kblocks = [](int K) { return (size_t)((K + gemm_tc::BK - 1) / gemm_tc::BK); };
     c->pk_nt = d.d_model / 128;
@@ -351,6 +365,8 @@ int gemm(specvla_ctx *ctx, const XBuf &A, const WMat &W, int R, gemm_tc::EpiArgs
   const int tiles = swiglu ? (ea.N + 127) / 128 : (W.N + SV_TILE_ROWS - 1) / SV_TILE_ROWS;
   const int KB = (W.K + gemm_tc::BK - 1) / gemm_tc::BK;
   ea.wpacked = W.packed;
+  ea.wq8 = W.q8;
+  ea.wscale = W.scale;
   ea.wait_ns = ctx->wait_ns;
   ea.inv_k = 1.f / (float)W.K;
   ea.eps = ctx->desc.rms_eps;
@@ -362,14 +378,15 @@ int gemm(specvla_ctx *ctx, const XBuf &A, const WMat &W, int R, gemm_tc::EpiArgs
   ea.T = R;
   ea.tn_tail = gemm_tc::tn_of(R - (chunks - 1) * gemm_tc::MAX_T);
   ea.pf_w = nullptr;
-  if (next && next->packed && ctx->use_l2_prefetch) {
+  if (next && (next->packed || next->q8) && ctx->use_l2_prefetch) {
     // start pulling the next matrix (up to L2_PREFETCH_BYTES of it)
     ea.pf_tiles = next_swiglu ? (next->N / 2 + 127) / 128 : (next->N + SV_TILE_ROWS - 1) / SV_TILE_ROWS;
     ea.pf_KB = (next->K + gemm_tc::BK - 1) / gemm_tc::BK;
     ea.pf_S = gemm_ck::slices_for(ea.pf_tiles * chunks, ea.pf_KB, ctx->fit);
-    const size_t per_cta = L2_PREFETCH_BYTES / ((size_t)ea.pf_tiles * ea.pf_S) / gemm_tc::W_STAGE_BYTES;
+    ea.pf_unit_bytes = next->q8 ? gemm_tc::W_STAGE_BYTES / 2 : gemm_tc::W_STAGE_BYTES;
+    const size_t per_cta = L2_PREFETCH_BYTES / ((size_t)ea.pf_tiles * ea.pf_S) / ea.pf_unit_bytes;
     ea.pf_units = per_cta < 1 ? 1 : (int)per_cta;
-    ea.pf_w = next->packed;
+    ea.pf_w = next->q8 ? static_cast<const void *>(next->q8) : static_cast<const void *>(next->packed);
   }
   CU(gemm_ck::launch(W.map, A.map[tn_index(gemm_tc::tn_of(R))], A.map[tn_index(ea.tn_tail)], ea, tiles, KB, S,
                      ctx->err, st, ctx->use_pdl));
@@ -377,7 +394,7 @@ int gemm(specvla_ctx *ctx, const XBuf &A, const WMat &W, int R, gemm_tc::EpiArgs
   if (prof) {
     CU(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used + 1], st));
     ctx->prof_cls[ctx->prof_used++] = cls;
-    ctx->prof_bytes[cls] += (double)W.N * W.K * sizeof(bf16);
+    ctx->prof_bytes[cls] += (double)W.N * W.K * (W.q8 ? 1 : sizeof(bf16));
   }
   return SPECVLA_OK;
 }
@@ -795,16 +812,37 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
   ctx->use_pdl = true;
   ctx->use_l2_prefetch = true;
   ctx->fit = gemm_ck::query_cluster_fit();
-  size_t packed_used = 0;
+  size_t packed_used = 0, q8_used = 0, scale_used = 0;
   bool pack_ok = true;
-  // swiglu: the matrix is [gate; up] stacked ([2F, K]) and is packed as tiles of 128 + 128 rows
-  auto wmat = [&](const void *p, int N, int K, bool swiglu = false) {
+  const bool quantise = desc->weight_bits == 8;
+  // swiglu: the matrix is [gate; up] stacked ([2F, K]) and is packed as tiles of 128 + 128 rows.
+  // q8: a matrix of the quantised target: row scales and int8 codes instead of the bf16 copy.
+  auto wmat = [&](const void *p, int N, int K, bool swiglu = false, bool q8 = false) {
     WMat w{};
     w.p = static_cast<const bf16 *>(p);
     w.N = N;
     w.K = K;
     w.has_map = p && gemm_tc::make_w_map(&w.map, w.p, N, K);
     w.packed = nullptr;
+    if (p && q8) {
+      const int F = N / 2;
+      const int tiles = swiglu ? (F + 127) / 128 : (N + SV_TILE_ROWS - 1) / SV_TILE_ROWS;
+      const int KB = (K + gemm_tc::BK - 1) / gemm_tc::BK;
+      const size_t bytes = gemm_tc::packed_elems(tiles, K);
+      if (q8_used + bytes > ctx->packed_q8_bytes || scale_used + (size_t)N > ctx->wscale_elems) {
+        pack_ok = false;
+        return w;
+      }
+      float *sc = ctx->wscale + scale_used;
+      signed char *dst = ctx->packed_q8 + q8_used;
+      scale_used += N;
+      q8_used += bytes;
+      gemm_tc::row_scale_q8_kernel<<<(N + 7) / 8, 256>>>(w.p, N, K, sc);
+      gemm_tc::pack_weights_q8_kernel<<<148 * 8, 256>>>(w.p, N, K, tiles, KB, swiglu ? 1 : 0, F, sc, dst);
+      w.q8 = dst;
+      w.scale = sc;
+      return w;
+    }
     if (p) {
       const int F = N / 2;
       const int tiles = swiglu ? (F + 127) / 128 : (N + SV_TILE_ROWS - 1) / SV_TILE_ROWS;
@@ -833,7 +871,7 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
   xmaps(ctx->hid);
   xmaps(ctx->lm_in);
   ctx->embed = static_cast<const bf16 *>(tw->embed);
-  ctx->lm_head = wmat(tw->lm_head, desc->vocab, D);
+  ctx->lm_head = wmat(tw->lm_head, desc->vocab, D, false, quantise);
   ctx->final_norm = tw->final_norm;
   ctx->layers.resize(desc->n_layers);
   for (int l = 0; l < desc->n_layers; l++) {
@@ -841,8 +879,9 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
       delete ctx;
       return SPECVLA_ERR_INVALID_ARG;
     }
-    ctx->layers[l] = LayerW{wmat(tw->wqkv[l], 3 * hd, D), wmat(tw->wo[l], D, hd), wmat(tw->wgu[l], 2 * F, D, true),
-                            wmat(tw->wd[l], D, F), tw->norm1[l], tw->norm2[l]};
+    ctx->layers[l] = LayerW{wmat(tw->wqkv[l], 3 * hd, D, false, quantise), wmat(tw->wo[l], D, hd, false, quantise),
+                            wmat(tw->wgu[l], 2 * F, D, true, quantise), wmat(tw->wd[l], D, F, false, quantise),
+                            tw->norm1[l], tw->norm2[l]};
   }
   ctx->has_draft = dw && dw->fc && dw->wqkv && dw->wo && dw->wgu && dw->wd && dw->norm1 && dw->norm2;
   if (ctx->has_draft) {
@@ -857,7 +896,7 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
   ctx->last_nt = ctx->nt;
   ctx->pk_ok = false;
   ctx->use_pk = false;            // measured slower than one launch per GEMM on B200: opt-in
-  if (pk_shapes_ok(*desc) && pack_ok) {
+  if (pk_shapes_ok(*desc) && pack_ok && !quantise) {
     pk_build_target_ops(ctx);
     ctx->pk_ok = pk_prepare(ctx);
   }

@@ -30,7 +30,13 @@ def test_binding_declares_every_export():
 
 def test_host_side_validation_without_gpu():
     from paper_2507_22424_b200 import binding as B
-    md = B.ModelDesc(2, 256, 4, 64, 688, 1024, 768, 256, 1e-6, 1e4, 512, 1, 512, 1)
+    md = B.ModelDesc(2, 256, 4, 64, 688, 1024, 768, 256, 1e-6, 1e4, 512, 1, 512, 1, 16)
+    full = B.lib.specvla_workspace_bytes(ctypes.byref(md))
+    md.weight_bits = 8
+    assert 0 < B.lib.specvla_workspace_bytes(ctypes.byref(md)) < full      # int8 codes: smaller weight copy
+    md.weight_bits = 5
+    assert B.lib.specvla_workspace_bytes(ctypes.byref(md)) == 0
+    md.weight_bits = 16
     assert B.lib.specvla_workspace_bytes(ctypes.byref(md)) > 0
     md.head_dim = 48
     assert B.lib.specvla_workspace_bytes(ctypes.byref(md)) == 0

@@ -272,3 +272,24 @@ def test_c1_persistent_forward_kernel_matches_oracle(env):
         assert tally.accepts == tally.caches == 1 and tally.rows_exact >= 18
     finally:
         gpu.set_option(OPT_PERSISTENT_FORWARD, 0)
+
+
+def test_c1_quantised_target_matches_quantised_oracle(env):
+    """Appendix C on the 7B-shaped model: int8 target (this repository's per-row scheme), bf16 draft
+    model. Prefill and one verification of the oracle's draft tree, everything compared."""
+    from oracle import quant as Q
+    from oracle.specvla import SpecVLAOracle
+    wc = env["gpu"].w
+    wh = env["orc"].w.raw
+    orc = SpecVLAOracle(DESC, Q.quantize_target(wh), action_only=True, max_seq=448, max_tree_rows=128)
+    gpu = G.make_gpu(DESC, wc, max_seq=512, max_episodes=1, max_rows=512, action_only=True, weight_bits=8)
+    try:
+        tally = G.Tally()
+        ep, _, _ = G.prefill_both(orc, gpu, env["emb"], env["ids"], 0, tally, DESC)
+        tree = orc.draft_tree(ep, C.TREE_26)
+        gpu.draft_tree([0], env["shape"], want_trees=False)
+        G.verify_both(orc, gpu, ep, tree, 0, tally, DESC, where="q8.g")
+        tally.report("C1 int8 target")
+        assert tally.accepts == tally.caches == 1 and tally.rows_exact >= 18
+    finally:
+        gpu.close()
