@@ -583,7 +583,7 @@ def run_micro(spec: str, steps: int, warmup: int):
     f = spec.split(":")
     if f[0] == "verify":
         return run_micro_verify(int(f[1]), int(f[2]) if len(f) > 2 else 27, steps, warmup,
-                                persistent=(int(f[3]) if len(f) > 3 else 1))
+                                persistent=(int(f[3]) if len(f) > 3 else 0), bits=(int(f[4]) if len(f) > 4 else 16))
     if f[0] == "batch":
         return run_micro_batch(int(f[1]) if len(f) > 1 else 16, steps, warmup)
     assert f[0] == "gemm" and len(f) in (4, 5), spec
@@ -614,8 +614,9 @@ def run_micro(spec: str, steps: int, warmup: int):
                           peak_source=peaks["source"])), flush=True)
 
 
-def run_micro_verify(n_layers: int, rows: int, steps: int, warmup: int, persistent: int = 1):
-    """`--micro verify:L[:T[:P]]` (P = 0: one launch per GEMM instead of the persistent forward kernel): verification steps of a 7B-SHAPED decoder cut down to L layers (a few
+def run_micro_verify(n_layers: int, rows: int, steps: int, warmup: int, persistent: int = 0, bits: int = 16):
+    """`--micro verify:L[:T[:P[:B]]]` (P = 1: the persistent forward kernel instead of one launch per GEMM;
+    B = 8: int8 target): verification steps of a 7B-SHAPED decoder cut down to L layers (a few
     GB on the device instead of 28), random T-row trees, strict acceptance. The small case of the
     real kernels (repacked weights, fused epilogues, PDL) for ncu --set full captures; also prints
     the per-GEMM device times of the verification phase."""
@@ -629,7 +630,7 @@ def run_micro_verify(n_layers: int, rows: int, steps: int, warmup: int, persiste
     weights = data.make_weights(desc, wl.seed, device="cuda", with_draft=False)
     embeds, ids = data.make_prefix(wl, device="cuda")
     ids_host, P = ids.tolist(), len(ids)
-    gpu = SpecVLA(desc, weights, max_seq=1024, max_episodes=1, max_rows=512, action_only=True)
+    gpu = SpecVLA(desc, weights, max_seq=1024, max_episodes=1, max_rows=512, action_only=True, weight_bits=bits)
     from paper_2507_22424_b200.binding import OPT_PERSISTENT_FORWARD
     gpu.set_option(OPT_PERSISTENT_FORWARD, persistent)
     first = gpu.prefill([0], embeds, ids_host, [P])
@@ -650,7 +651,10 @@ def run_micro_verify(n_layers: int, rows: int, steps: int, warmup: int, persiste
     prof = gpu.profile_read()
     ms = a.elapsed_time(b) / steps
     wbytes = n_layers * 404_750_336 + 262_668_288
-    print(json.dumps(dict(micro="verify", layers=n_layers, rows=rows, steps=steps, persistent=persistent, ms_per_step=ms,
+    if bits == 8:
+        wbytes //= 2
+    print(json.dumps(dict(micro="verify", layers=n_layers, rows=rows, steps=steps, persistent=persistent,
+                          weight_bits=bits, ms_per_step=ms,
                           weight_bytes=wbytes, gbs=wbytes / ms / 1e6,
                           note="ms_per_step includes the per-GEMM timing events and the host read-back",
                           per_class={k: dict(us_per_launch=1e3 * v["ms"] / max(1, v["launches"]),

@@ -47,29 +47,55 @@ __device__ __forceinline__ void cluster_sync_all() {
 }
 __host__ __device__ constexpr int ck_tmem_cols(int TN) { return 2 * acc_width(TN) < 32 ? 32 : 2 * acc_width(TN); }
 
+// Quantised weights (Q8): a stage holds the int8 codes of a unit (16 KB from HBM) and its X slice;
+// the bf16 image the tensor cores read is written by the epilogue warps into one of two 32 KB
+// buffers in front of the ring. With half the bytes per unit the ring needs twice the units in
+// flight for the same HBM rate, so it takes all the shared memory there is.
+__host__ __device__ constexpr int q8_stage_bytes(int TN) { return W_STAGE_BYTES / 2 + 2 * TN * BK * 2; }
+// expanded buffers: as many units as can be in expansion at once (the expansion of a unit is a
+// chain of shared-memory latencies, barriers and a proxy fence of about a microsecond)
+__host__ __device__ constexpr int q8_expanded(int TN) { return TN <= 32 ? 3 : 2; }
+__host__ __device__ constexpr int q8_stages(int TN) {
+  return (216 * 1024 - q8_expanded(TN) * W_STAGE_BYTES) / q8_stage_bytes(TN) > 8
+             ? 8
+             : (216 * 1024 - q8_expanded(TN) * W_STAGE_BYTES) / q8_stage_bytes(TN);
+}
+__host__ __device__ constexpr int q8_smem_bytes(int TN) {
+  return q8_expanded(TN) * W_STAGE_BYTES + q8_stages(TN) * q8_stage_bytes(TN) + 1024 + 256;
+}
+// Expansion groups: one per expanded buffer (group g always writes buffer g and takes the units
+// g, g + NE, ...: it waits for the MMAs of its previous unit before anything else, which also tells
+// it that every earlier load has landed, so a mbarrier parity can never be read a phase late).
+__host__ __device__ constexpr int q8_group_threads(int TN) { return q8_expanded(TN) == 3 ? 64 : 128; }
+
 // EpiArgs as in gemm_tc: the mode is a template parameter. KB = K blocks per tile.
 template <int TN, int MODE, bool Q8>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                const __grid_constant__ CUtensorMap tmXtail, const EpiArgs ea, const int KB,
                int *__restrict__ err) {
-  constexpr int STAGES = stages_of(TN);
-  constexpr int STAGE = stage_bytes(TN);
+  constexpr int STAGES = Q8 ? q8_stages(TN) : stages_of(TN);
+  constexpr int STAGE = Q8 ? q8_stage_bytes(TN) : stage_bytes(TN);
+  constexpr int NE = Q8 ? q8_expanded(TN) : 1;
+  constexpr uint32_t RING0 = Q8 ? NE * W_STAGE_BYTES : 0;     // Q8: the expanded weight buffers come first
+  constexpr uint32_t XOFF = Q8 ? W_STAGE_BYTES / 2 : W_STAGE_BYTES;   // X slice within a stage
   constexpr int AW = acc_width(TN);
   extern __shared__ unsigned char smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t bars = base + STAGES * STAGE;
+  const uint32_t bars = base + RING0 + STAGES * STAGE;
   auto full_bar = [&](int s) { return bars + 8u * s; };
   auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
   const uint32_t tfull_bar = bars + 8u * (2 * STAGES);
   const uint32_t tmem_slot = bars + 8u * (2 * STAGES + 1);
-  // Q8: the stage's weight tile has been expanded from int8 codes to bf16 by the epilogue warps
-  auto conv_bar = [&](int s) { return bars + 8u * (2 * STAGES + 2 + s); };
+  // Q8: expanded buffer e holds the bf16 image of a unit (conv) / has been read by its MMAs (efree)
+  auto conv_bar = [&](int e) { return bars + 8u * (2 * STAGES + 2 + e); };
+  auto efree_bar = [&](int e) { return bars + 8u * (2 * STAGES + 2 + NE + e); };
+  __shared__ int s_gflag[4];
   __shared__ float s_scale[MAX_T];
   __shared__ int s_pos[MAX_T], s_slot[MAX_T], s_ep[MAX_T];
   // RoPE factors of the CTA's rows (EPI_QKV, up to 32 rows of up to 64 pairs): fetched while the
   // MMAs run, so that the finishing loop does not wait for them row after row
-  constexpr bool ROPE_SMEM = TN <= 32 && MODE == EPI_QKV;
+  constexpr bool ROPE_SMEM = TN <= 32 && MODE == EPI_QKV && !Q8;   // (Q8: the ring takes that shared memory)
   constexpr int ROPE_ROWS = ROPE_SMEM ? 32 : 1, ROPE_HALF = ROPE_SMEM ? 64 : 1;
   __shared__ __align__(16) float2 s_rope[ROPE_ROWS * ROPE_HALF];
   __shared__ float s_red[8][MAX_T];
@@ -104,12 +130,11 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   auto load_w = [&](int it) {
     if (it == withheld) return;
     const int st = it % STAGES;
-    const uint32_t sW = base + st * STAGE;
+    const uint32_t sW = base + RING0 + st * STAGE;
     mbar_expect_tx(full_bar(st), stage_tx);
     if (Q8) {
-      // the codes of the 256 x 64 tile land in the upper half of the stage's weight area and are
-      // expanded in place (epilogue warps, below)
-      bulk_load(sW + W_STAGE_BYTES / 2, ea.wq8 + (size_t)(u0 + it) * (BM * BK), W_STAGE_BYTES / 2, full_bar(st), pol_w);
+      // the codes of the 256 x 64 tile; the epilogue warps expand them (below)
+      bulk_load(sW, ea.wq8 + (size_t)(u0 + it) * (BM * BK), W_STAGE_BYTES / 2, full_bar(st), pol_w);
     } else if (ea.wpacked) {
       bulk_load(sW, ea.wpacked + (size_t)(u0 + it) * (BM * BK), W_STAGE_BYTES, full_bar(st), pol_w);
     } else {
@@ -125,9 +150,13 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     if (!ea.wpacked) prefetch_tensormap(&tmW);
     for (int s = 0; s < STAGES; s++) {
       mbar_init(full_bar(s), 1);
-      mbar_init(empty_bar(s), 1);
-      if (Q8) mbar_init(conv_bar(s), 1);
+      mbar_init(empty_bar(s), Q8 ? 2 : 1);     // Q8: the codes have been expanded AND the MMAs have read X
     }
+    if (Q8)
+      for (int e = 0; e < NE; e++) {
+        mbar_init(conv_bar(e), 1);
+        mbar_init(efree_bar(e), 1);
+      }
     mbar_init(tfull_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -156,7 +185,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       grid_dep_wait();
       for (int j = 0; j < npre; j++)
         if (j != withheld)
-          tma_load_3d(base + j * STAGE + W_STAGE_BYTES, xmap, (kb0 + j) * BK, row0, 0, full_bar(j), pol_x);
+          tma_load_3d(base + RING0 + j * STAGE + XOFF, xmap, (kb0 + j) * BK, row0, 0, full_bar(j), pol_x);
       for (int it = npre; it < n_units; it++) {
         const int st = it % STAGES, rnd = it / STAGES;
         if (!mbar_wait(empty_bar(st), (rnd - 1) & 1, ea.wait_ns)) {
@@ -165,7 +194,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         }
         load_w(it);
         if (it != withheld)
-          tma_load_3d(base + st * STAGE + W_STAGE_BYTES, xmap, (kb0 + it) * BK, row0, 0, full_bar(st), pol_x);
+          tma_load_3d(base + RING0 + st * STAGE + XOFF, xmap, (kb0 + it) * BK, row0, 0, full_bar(st), pol_x);
       }
     }
     __syncwarp();
@@ -174,12 +203,13 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     if (lane == 0 && n_units > 0) {
       for (int it = 0; it < n_units; it++) {
         const int st = it % STAGES, rnd = it / STAGES;
-        if (!mbar_wait(Q8 ? conv_bar(st) : full_bar(st), rnd & 1, ea.wait_ns)) {
+        if (!mbar_wait(Q8 ? conv_bar(it % NE) : full_bar(st), Q8 ? (it / NE) & 1 : rnd & 1, ea.wait_ns)) {
           atomicExch(err, SV_ERR_WAIT_FULL);
           break;
         }
         tc_fence_after();
-        const uint32_t sW = base + st * STAGE, sX = sW + W_STAGE_BYTES;
+        const uint32_t sW = Q8 ? base + (it % NE) * W_STAGE_BYTES : base + st * STAGE;
+        const uint32_t sX = base + RING0 + st * STAGE + XOFF;
 #pragma unroll
         for (int kk = 0; kk < BK / 16; kk++) {
 #pragma unroll
@@ -190,6 +220,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           }
         }
         tc_commit(empty_bar(st));
+        if (Q8) tc_commit(efree_bar(it % NE));
         if (it == n_units - 1) tc_commit(tfull_bar);
       }
     }
@@ -232,46 +263,65 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       }
     }
     if (Q8) {
-      // int8 -> bf16 expansion of every stage as it lands: thread et owns row et of the tile (64
-      // codes = 64 bytes in, one 128-byte swizzled row out). All rows are read before any is
-      // written: the rows of the second half overwrite the code area.
-      for (int it = 0; it < n_units; it++) {
-        const int st = it % STAGES, rnd = it / STAGES;
-        const bool mine = mbar_wait(full_bar(st), rnd & 1, ea.wait_ns);
-        if (lane == 0) s_flag[warp - 2] = mine ? 1 : 0;
-        const uint32_t sW = base + st * STAGE;
-        uint32_t c[16];
-#pragma unroll
-        for (int i = 0; i < 4; i++)
-          asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
-                       : "=r"(c[4 * i]), "=r"(c[4 * i + 1]), "=r"(c[4 * i + 2]), "=r"(c[4 * i + 3])
-                       : "r"(sW + W_STAGE_BYTES / 2 + et * 64 + i * 16) : "memory");
-        epi_barrier();
-        if (!(s_flag[0] && s_flag[1] && s_flag[2] && s_flag[3] && s_flag[4] && s_flag[5] && s_flag[6] && s_flag[7])) {
-          if (et == 0) atomicExch(err, SV_ERR_WAIT_FULL);
-          epi_barrier();                                   // the flags have been read by everybody
-          break;
-        }
-#pragma unroll
-        for (int ch = 0; ch < 8; ch++) {
-          // codes 8 ch .. 8 ch + 7 of the row: two words -> eight bf16 (exact: |code| <= 127)
-          uint32_t o[4];
-#pragma unroll
-          for (int h = 0; h < 2; h++) {
-            const uint32_t w = c[2 * ch + h];
-            const float f0 = (float)(int)(signed char)(w & 0xff), f1 = (float)(int)(signed char)((w >> 8) & 0xff);
-            const float f2 = (float)(int)(signed char)((w >> 16) & 0xff), f3 = (float)(int)(signed char)(w >> 24);
-            const __nv_bfloat162 lo = __floats2bfloat162_rn(f0, f1), hi = __floats2bfloat162_rn(f2, f3);
-            o[2 * h] = *reinterpret_cast<const uint32_t *>(&lo);
-            o[2 * h + 1] = *reinterpret_cast<const uint32_t *>(&hi);
+      // int8 -> bf16 expansion of every unit as it lands. NE groups of warps take the units in
+      // turn (group g: units g, g + NE, ... into expanded buffer g), so that NE units are in
+      // expansion at once; a thread owns rows gt, gt + GT, ... of the tile (64 codes = 64 bytes in,
+      // one 128-byte swizzled row out).
+      constexpr int GT = q8_group_threads(TN);
+      const int g = et / GT, gt = et - g * GT;
+      auto group_sync = [&]() { asm volatile("bar.sync %0, %1;" ::"r"(2 + g), "n"(GT) : "memory"); };
+      if (g < NE) {
+        for (int it = g; it < n_units; it += NE) {
+          const int st = it % STAGES, rnd = it / STAGES, use = it / NE;
+          if (gt == 0) {
+            bool ok = true;
+            if (use > 0) ok = mbar_wait(efree_bar(g), (use - 1) & 1, ea.wait_ns);   // first: see above
+            if (ok) ok = mbar_wait(full_bar(st), rnd & 1, ea.wait_ns);
+            s_gflag[g] = ok ? 1 : 0;
           }
-          asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(sW + et * 128 + ((ch ^ (et & 7)) << 4)), "r"(o[0]),
-                       "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
+          group_sync();                                    // the buffer is free, the codes are there
+          if (!s_gflag[g]) {
+            if (gt == 0) atomicExch(err, SV_ERR_WAIT_FULL);
+            break;
+          }
+          const uint32_t sC = base + RING0 + st * STAGE, sE = base + g * W_STAGE_BYTES;
+#pragma unroll 1
+          for (int r = gt; r < BM; r += GT) {
+            uint32_t c[16];
+#pragma unroll
+            for (int i = 0; i < 4; i++)
+              asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                           : "=r"(c[4 * i]), "=r"(c[4 * i + 1]), "=r"(c[4 * i + 2]), "=r"(c[4 * i + 3])
+                           : "r"(sC + r * 64 + i * 16) : "memory");
+#pragma unroll
+            for (int ch = 0; ch < 8; ch++) {
+              // codes 8 ch .. 8 ch + 7 of the row: two words -> eight bf16, exact (|code| <= 127), on
+              // the integer and FMA pipes only: code + 128 in the low mantissa byte of 2^23, minus
+              // (2^23 + 128), gives the code as fp32, whose upper half is its bf16 image
+              uint32_t o[4];
+#pragma unroll
+              for (int h = 0; h < 2; h++) {
+                const uint32_t x = c[2 * ch + h] ^ 0x80808080u;
+                const float f0 = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7650)) - 8388736.f;
+                const float f1 = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7651)) - 8388736.f;
+                const float f2 = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7652)) - 8388736.f;
+                const float f3 = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7653)) - 8388736.f;
+                o[2 * h] = __byte_perm(__float_as_uint(f0), __float_as_uint(f1), 0x7632);
+                o[2 * h + 1] = __byte_perm(__float_as_uint(f2), __float_as_uint(f3), 0x7632);
+              }
+              asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(sE + r * 128 + ((ch ^ (r & 7)) << 4)),
+                           "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
+            }
+          }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> tensor-core reads
+          group_sync();                                    // the whole tile is written
+          if (gt == 0) {
+            mbar_arrive(conv_bar(g));
+            mbar_arrive(empty_bar(st));                    // the codes are no longer needed
+          }
         }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> tensor-core reads
-        epi_barrier();
-        if (et == 0) mbar_arrive(conv_bar(st));
       }
+      epi_barrier();                                       // the groups (and the idle warps) meet again
     }
     bool have = n_units > 0;
     if (have) {
@@ -552,13 +602,13 @@ template <int TN, int MODE, bool Q8>
 inline cudaError_t launch_tq(const CUtensorMap &tmW, const CUtensorMap &tmX, const CUtensorMap &tmXtail,
                              const EpiArgs &ea, int tiles, int KB, int S, int *err, cudaStream_t st, bool pdl) {
   // per device and cheap: set on every launch, so that every device of the process has it
-  cudaError_t e = cudaFuncSetAttribute(gemm_ck_kernel<TN, MODE, Q8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       smem_bytes(TN));
+  constexpr int SMEM = Q8 ? q8_smem_bytes(TN) : smem_bytes(TN);
+  cudaError_t e = cudaFuncSetAttribute(gemm_ck_kernel<TN, MODE, Q8>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(tiles * S, (ea.T + MAX_T - 1) / MAX_T);
   cfg.blockDim = dim3(THREADS);
-  cfg.dynamicSmemBytes = smem_bytes(TN);
+  cfg.dynamicSmemBytes = SMEM;
   cfg.stream = st;
   cudaLaunchAttribute at[2];
   at[0].id = cudaLaunchAttributeClusterDimension;
