@@ -315,6 +315,34 @@ def c4_batch(weights, desc, steps=3):
                 note="random trees (nothing planted): acceptance near zero; algorithmic flops, burst bf16 peak")
 
 
+def int8_target(weights, desc, embeds, ids_host, P, shape, r, n_tok, steps=5):
+    """Appendix C's direction on C1: the target's matrices as int8 codes (per output row, symmetric;
+    the draft model stays bf16). Chunks/s through specvla_generate_action and the verification step,
+    next to the bf16 numbers of the same run; strict decoding must equal the quantised model's own
+    autoregressive decoding."""
+    import torch
+    from paper_2507_22424_b200.binding import SpecVLA, make_shape
+    gpu = SpecVLA(desc, weights, max_seq=512, max_episodes=1, max_rows=512, action_only=True, weight_bits=8)
+    toks, _, _ = gpu.generate_action([0], embeds, ids_host, [P], shape, r, n_tok)
+    ar, _, _ = gpu.generate_action([0], embeds, ids_host, [P], make_shape((), ()), 0, n_tok)
+    torch.cuda.synchronize()
+    ms_v = iters = 0
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(steps):
+        toks, _, st = gpu.generate_action([0], embeds, ids_host, [P], shape, r, n_tok)
+        ms_v += st.ms_verify
+        iters += st.iterations
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b)
+    gpu.close()
+    return dict(value=steps / (ms * 1e-3), unit=UNIT, verify_ms_per_step=ms_v / max(1, iters),
+                weight_bytes_per_step=WEIGHT_BYTES_PER_VERIFY // 2, lossless_vs_own_ar=bool(toks == ar), tokens=toks[0],
+                note="int8 codes are streamed at half the bytes but expanded to bf16 inside the SM before the "
+                     "tensor cores read them; that expansion, not HBM, bounds this path")
+
+
 # --------------------------------------------------------------------------- CUDA arm
 def run_ours(args, rank, local_rank, world):
     import torch
@@ -485,19 +513,25 @@ def run_ours(args, rank, local_rank, world):
     all_bytes = sum(v["bytes"] for v in prof.values())
     ipc = max(1, round(iters / args.steps))
     # --- C2: relaxed-acceptance sweep with planted drafts (target's greedy bin + seeded offset) -----
-    c2 = c2_sweep(gpu, wl, desc, embeds, ids_host, P, shape, n_tok)
+    extras = not args.skip_reports
+    c2 = c2_sweep(gpu, wl, desc, embeds, ids_host, P, shape, n_tok) if extras else None
     # --- C3: verification step alone over random trees of each size ------------------------------
-    c3 = c3_sweep(gpu, desc, n_tok)
+    c3 = c3_sweep(gpu, desc, n_tok) if extras else None
     # --- C4: 16 ragged episodes prefilled and verified in one call each (tensor-bound) -------------
-    c4 = c4_batch(weights, desc)
+    c4 = c4_batch(weights, desc) if extras else None
+    # --- Appendix C: the same chunk with an int8 target (this repository's per-row scheme) -------------
+    q8 = int8_target(weights, desc, embeds, ids_host, P, shape, r, n_tok) if extras else None
     # --- the oracle on the host cores: real prefill, draft tree and verification step of C1 --------
-    weights_host = {k: v.cpu() for k, v in weights.items()}
-    t_cpu = time.perf_counter()
-    orc = OracleC1(weights_host)
-    t_ver = orc.verify_step()
-    cpu_val = orc.chunks_per_s(t_ver, ipc)
-    cpu_sec = time.perf_counter() - t_cpu
-    pieces = dict(prefill_s=orc.t_prefill, draft_tree_s=orc.t_draft, verify_step_s=t_ver)
+    if extras:
+        weights_host = {k: v.cpu() for k, v in weights.items()}
+        t_cpu = time.perf_counter()
+        orc = OracleC1(weights_host)
+        t_ver = orc.verify_step()
+        cpu_val, cpu_cores = orc.chunks_per_s(t_ver, ipc), orc.cores
+        cpu_sec = time.perf_counter() - t_cpu
+        pieces = dict(prefill_s=orc.t_prefill, draft_tree_s=orc.t_draft, verify_step_s=t_ver)
+    else:
+        cpu_val, cpu_cores, cpu_sec, pieces = None, None, 0.0, None
     # algorithmic flops of the prefill: target 2 * 6.607e9 per row + causal attention, plus the draft
     # model (fc + one layer) over the shifted pairs
     d_, F_, hd_ = desc.d_model, desc.d_ffn, desc.n_heads * desc.head_dim
@@ -536,7 +570,7 @@ def run_ours(args, rank, local_rank, world):
                               peak_source=peaks["source"] + " bf16 GEMM, sustained",
                               note="algorithmic flops (one bf16 pass) of target + draft prefill over 290 rows; the "
                                    "kernels multiply both activation limbs, i.e. execute twice these"),
-        c2_sweep=c2, c3_sweep=c3, c4_batch=c4,
+        c2_sweep=c2, c3_sweep=c3, c4_batch=c4, int8_target=q8,
         accept_by_position=dict(iterations=pos_it[:n_tok - 1], mean_m=[(pos_sum[k] / pos_it[k]) if pos_it[k] else None
                                                                     for k in range(n_tok - 1)],
                                 note="Table 3's statistic on C1: accepted draft tokens by the position at which "
@@ -557,7 +591,7 @@ def run_ours(args, rank, local_rank, world):
                                  "continuation on its first-child chain: the ceiling acceptance could reach here"),
         dynamic_tree=dict(value=world * ar_steps / (ms_dy / 1000.0), unit=UNIT, same_tokens=bool(dy_toks == toks),
                           note="top-8, depth 5, best 50 of 264 drafted nodes verified (51 rows per step)"),
-        cpu_baseline=dict(value=cpu_val, unit=UNIT, cores=orc.cores, kind="oracle",
+        cpu_baseline=dict(value=cpu_val, unit=UNIT, cores=cpu_cores, kind="oracle",
                           sample=("the oracle (float64) on C1 with the full 7B-shaped weights: one real prefill of "
                                   "the 290-row prefix, one real 26-node draft tree, one real verification step (32 "
                                   "layers + LM head over 27 rows under the tree mask), each run once; chunk = prefill "
@@ -719,6 +753,9 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--skip-reports", action="store_true",
+                    help="leave out the extra reports (C2/C3/C4 sweeps, int8 target, oracle timing): the timed "
+                         "regions only, e.g. for a profiler's launch list")
     ap.add_argument("--micro", default=None, help="gemm:T:N:K[:M], verify:L[:T] or batch[:E] - small cases for kernel timing / ncu (see run_micro)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
