@@ -33,9 +33,10 @@ WEIGHT_BYTES_PER_VERIFY = 13_214_679_040      # 32 layers + LM head, bf16, read 
 
 # DRAM traffic of one gate/up launch at T = 27 from the ncu capture under profiles/ (bytes); to be
 # re-taken (or set to None) whenever gemm_ck.cuh changes.
-GATE_UP_DRAM_BYTES = None
-GATE_UP_DRAM_SOURCE = ("null: the GEMM kernel changed after the last ncu capture "
-                       "(profiles/gemm_ck_verify_T27_ncu_full.md has the previous 208.8 MB)")
+GATE_UP_DRAM_BYTES = 203_322_624 + 3_482_880
+GATE_UP_DRAM_SOURCE = ("ncu dram__bytes_read.sum + dram__bytes_write.sum of this launch at full size "
+                       "(profiles/gemm_ck_verify_T27_ncu_full.md); the ~23 MB above the weights are the operand "
+                       "and the L2 prefetch of the next GEMM's weights")
 
 
 def load_peaks():
