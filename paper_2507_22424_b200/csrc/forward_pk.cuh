@@ -445,8 +445,8 @@ struct RowInfo {
 // one row x 128 output columns (SwiGLU: 128 gate + 128 up columns) are dealt out to the epilogue
 // warps of the whole grid; a warp sums the item's partial tiles in CTA order (deterministic) and
 // applies the phase's epilogue. IB items are handled together, the first NB partial tiles of each
-// loaded in one round before anything is used (loads from L2 take a microsecond: a warp that
-// waited for each in turn would need several). A tile shared by more CTAs takes further rounds.
+// loaded together before anything is used (loads from L2 take a microsecond: a warp that
+// waited for each in turn would need several). A tile shared by more CTAs takes further batches.
 template <int MODE, int IB, int NB>
 __device__ __forceinline__ void finish_phase(const Params &p, const Op &o, const RowInfo &ri, int T, int G,
                                              int gw, int GW, int lane) {
@@ -460,7 +460,7 @@ __device__ __forceinline__ void finish_phase(const Params &p, const Op &o, const
     // operands that do not depend on the partial tiles: residual and gain (EPI_RESID), RoPE factors
     // (EPI_QKV), requested in the same round
     float4 ex0[IB], ex1[IB];
-    // round 1 of every item
+    // first batch of partial tiles of every item
 #pragma unroll
     for (int k = 0; k < IB; k++) {
       const int item = base + k * GW;
@@ -516,7 +516,7 @@ __device__ __forceinline__ void finish_phase(const Params &p, const Op &o, const
         v.x += a[k][i].x; v.y += a[k][i].y; v.z += a[k][i].z; v.w += a[k][i].w;
         if (SW) { v2.x += b[k][i].x; v2.y += b[k][i].y; v2.z += b[k][i].z; v2.w += b[k][i].w; }
       }
-      // further rounds (tiles shared by more than NB CTAs)
+      // further batches (tiles shared by more than NB CTAs)
       for (int c0 = cfs[k] + NB; c0 <= cls[k]; c0 += NB) {
         float4 e[NB], f[SW ? NB : 1];
 #pragma unroll

@@ -1129,7 +1129,7 @@ int specvla_draft_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const sp
   // Per level: the shared LM head over the rows just run (draft layer outputs as they are: no
   // norm, no row scale) with log-softmax + top-k, then one kernel that grows the tree and writes
   // the next level's input rows, then the draft model over those.
-  int scored_rows = R;               // round 0 scores every catch-up row; only each episode's last one is used
+  int scored_rows = R;               // level 0 scores every catch-up row; only each episode's last one is used
   for (int l = 0; l < shape->depth; l++) {
     if (scored_rows > ctx->lgs_rows) return SPECVLA_ERR_CAPACITY;
     if (d.action_only && d.n_bins <= SV_TILE_ROWS) {
