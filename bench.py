@@ -327,16 +327,21 @@ def int8_target(weights, desc, embeds, ids_host, P, shape, r, n_tok, steps=5):
     toks, _, _ = gpu.generate_action([0], embeds, ids_host, [P], shape, r, n_tok)
     ar, _, _ = gpu.generate_action([0], embeds, ids_host, [P], make_shape((), ()), 0, n_tok)
     torch.cuda.synchronize()
-    ms_v = iters = 0
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     a.record()
     for _ in range(steps):
         toks, _, st = gpu.generate_action([0], embeds, ids_host, [P], shape, r, n_tok)
-        ms_v += st.ms_verify
-        iters += st.iterations
     b.record()
     torch.cuda.synchronize()
     ms = a.elapsed_time(b)
+    # the verification step alone: the loop on the host times its phases apart
+    from paper_2507_22424_b200.binding import OPT_DEVICE_LOOP
+    gpu.set_option(OPT_DEVICE_LOOP, 0)
+    ms_v = iters = 0
+    for _ in range(3):
+        _, _, st = gpu.generate_action([0], embeds, ids_host, [P], shape, r, n_tok)
+        ms_v += st.ms_verify
+        iters += st.iterations
     gpu.close()
     return dict(value=steps / (ms * 1e-3), unit=UNIT, verify_ms_per_step=ms_v / max(1, iters),
                 weight_bytes_per_step=WEIGHT_BYTES_PER_VERIFY // 2, lossless_vs_own_ar=bool(toks == ar), tokens=toks[0],
@@ -381,14 +386,14 @@ def run_ours(args, rank, local_rank, world):
     l0 = gpu.kernel_launches()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    ms_verify = ms_draft = ms_prefill = 0.0
-    iters = accept = 0
+    ms_loop = ms_prefill = 0.0
+    iters = accept = device_loop = 0
     pos_it, pos_sum = [0] * 16, [0] * 16
     for _ in range(args.steps):
         toks, _, stats = chunk()
-        ms_verify += stats.ms_verify
-        ms_draft += stats.ms_draft
+        ms_loop += stats.ms_loop
         ms_prefill += stats.ms_prefill
+        device_loop += stats.device_loop
         iters += stats.iterations
         accept += sum(stats.accept_len[i] for i in range(min(16, stats.iterations)))
         for k in range(16):
@@ -411,6 +416,27 @@ def run_ours(args, rank, local_rank, world):
     e3.record()
     barrier()
     ms_e2e = e2.elapsed_time(e3)
+    # --- the same chunks with the loop driven from the host (one read-back per iteration): draft and
+    # verification are timed apart only there
+    from paper_2507_22424_b200.binding import OPT_DEVICE_LOOP
+    gpu.set_option(OPT_DEVICE_LOOP, 0)
+    chunk()
+    barrier()
+    h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    h0.record()
+    host_steps = max(3, args.steps // 2)
+    ms_verify = ms_draft = ms_prefill_h = 0.0
+    iters_h = 0
+    for _ in range(host_steps):
+        toks_h, _, sth = chunk()
+        ms_verify += sth.ms_verify
+        ms_draft += sth.ms_draft
+        ms_prefill_h += sth.ms_prefill
+        iters_h += sth.iterations
+    h1.record()
+    barrier()
+    ms_host = h0.elapsed_time(h1)
+    gpu.set_option(OPT_DEVICE_LOOP, 1)
     # --- AR baseline from the same kernels (depth-0 tree) --------------------------------
     ar_shape = make_shape((), ())
     gpu.generate_action([0], embeds, ids_host, [P], ar_shape, 0, n_tok)
@@ -421,7 +447,7 @@ def run_ours(args, rank, local_rank, world):
     ar_ms_verify = 0.0
     for _ in range(ar_steps):
         ar_toks, _, ar_stats = gpu.generate_action([0], embeds, ids_host, [P], ar_shape, 0, n_tok)
-        ar_ms_verify += ar_stats.ms_verify
+        ar_ms_verify += ar_stats.ms_loop
     e5.record()
     barrier()
     ms_ar = e4.elapsed_time(e5)
@@ -499,7 +525,7 @@ def run_ours(args, rank, local_rank, world):
     value = replica_throughput(world, args.steps, ms)
     e2e_value = replica_throughput(world, args.steps, ms_e2e)
     T = 1 + wl.tree.n_nodes
-    verify_ms = ms_verify / max(1, iters)
+    verify_ms = ms_verify / max(1, iters_h)
     # algorithmic bytes of a step: the weights once, the cache rows read (committed + tree) and the
     # tree rows written, counted at two bytes per element (a bf16 cache is all the method needs; this
     # library keeps it in fp32 for the 2e-2 logit tolerance, which doubles that 1.4 % share)
@@ -550,7 +576,8 @@ def run_ours(args, rank, local_rank, world):
                     n_tokens=n_tok, r=r, action_only=1, replicas=world,
                     l2="inputs larger than L2: every step streams 13.9 GB of weights"),
         e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=embeds.numel() * 2 + 4 * P,
-                 d2h_bytes_per_step=4 * n_tok * 2 + 8 * max(1, round(iters / args.steps)) * 10),
+                 # chunk state (tokens, statistics) + episode state + status word, read back once per chunk
+                 d2h_bytes_per_step=(16 + 64 * 4 + 64 * 64 * 4 + 3 * 16 * 4) + 64 + 4),
         gpu_launches=launches,
         clocks=clocks,
         roofline=dict(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
@@ -576,8 +603,15 @@ def run_ours(args, rank, local_rank, world):
                                                                     for k in range(n_tok - 1)],
                                 note="Table 3's statistic on C1: accepted draft tokens by the position at which "
                                      "an iteration starts (random draft head: zero)"),
-        phases_ms_per_chunk=dict(prefill=ms_prefill / args.steps, draft=ms_draft / args.steps,
-                                 verify=ms_verify / args.steps),
+        chunk_loop=dict(on_device=bool(device_loop == args.steps), ms_prefill=ms_prefill / args.steps,
+                        ms_iterations=ms_loop / args.steps,
+                        note="`value` and `e2e`: Algorithm 1's iterations as one launch of a CUDA graph (while node "
+                             "around draft tree, verification, token append), one read-back per chunk"),
+        host_loop=dict(value=world * host_steps / (ms_host / 1000.0), unit=UNIT, same_tokens=bool(toks_h == toks),
+                       note="same kernels, the loop on the host with a read-back of the accepted length per "
+                            "iteration; the phase times below come from this pass"),
+        phases_ms_per_chunk=dict(prefill=ms_prefill_h / host_steps, draft=ms_draft / host_steps,
+                                 verify=ms_verify / host_steps),
         accept=dict(iterations_per_chunk=iters / args.steps, mean_m=accept / max(1, iters),
                     mean_tokens_per_forward=accept / max(1, iters) + 1.0),
         ar_baseline=dict(value=world * ar_steps / (ms_ar / 1000.0), unit=UNIT,

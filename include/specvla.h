@@ -129,13 +129,16 @@ typedef struct {
   int iterations;                 /* draft+verify iterations run (max over episodes) */
   int tokens_emitted;             /* before clipping, first episode */
   int accept_len[16];             /* accepted draft tokens m of the first 16 iterations, first episode */
-  float ms_prefill, ms_draft, ms_verify;   /* device time, CUDA events */
+  float ms_prefill, ms_draft, ms_verify;   /* device time, CUDA events; draft and verify are measured
+                                            * apart only when the loop runs on the host (0 otherwise) */
   /* Accepted draft tokens by the position at which an iteration starts (Table 3): an iteration
    * that begins when k + 1 tokens of the chunk exist starts at position k (0 .. n_tokens - 2).
    * Iterations counted and accepted lengths m summed per position, first episode; positions past
    * 15 go uncounted. mean = pos_accept_sum[k] / pos_iterations[k]. */
   int pos_iterations[16];
   int pos_accept_sum[16];
+  float ms_loop;                  /* device time of all draft+verify iterations together */
+  int device_loop;                /* 1: the iterations ran as one graph launch (SPECVLA_OPT_DEVICE_LOOP) */
 } specvla_stats;
 
 /* Bytes of device workspace a context of this description needs. 0 on invalid description. */
@@ -160,11 +163,19 @@ int specvla_destroy(specvla_ctx *ctx);
  *   SPECVLA_OPT_L2_PREFETCH         1: a GEMM of the per-GEMM path prefetches the head of the next
  *       matrix into L2.
  *   SPECVLA_OPT_WAIT_LIMIT_NS       limit of every device-side wait of the persistent kernel in
- *       nanoseconds (default 2e9); a wait that runs out makes the call return SPECVLA_ERR_TIMEOUT. */
+ *       nanoseconds (default 2e9); a wait that runs out makes the call return SPECVLA_ERR_TIMEOUT.
+ *   SPECVLA_OPT_DEVICE_LOOP         1 (default): specvla_generate_action runs the iterations of
+ *       Algorithm 1 as ONE launch of a CUDA graph whose while node repeats draft tree, verification
+ *       and the appending of the emitted tokens until the chunk is complete; the host reads tokens,
+ *       statistics and episode state back once. Applies when every iteration launches the same
+ *       kernels (shape.prune = 0, no per-GEMM timing, per-GEMM forward) and the caches hold
+ *       prefix + n_tokens + depth + tree rows; otherwise, and with 0, the host runs the loop and
+ *       reads the accepted length back every iteration. Same tokens either way. */
 #define SPECVLA_OPT_PERSISTENT_FORWARD 1
 #define SPECVLA_OPT_DEPENDENT_LAUNCH   2
 #define SPECVLA_OPT_L2_PREFETCH        3
 #define SPECVLA_OPT_WAIT_LIMIT_NS      4
+#define SPECVLA_OPT_DEVICE_LOOP        5
 int specvla_set_option(specvla_ctx *ctx, int option, long long value);
 
 /* Forgets an episode's state (its caches are simply overwritten by the next prefill). */

@@ -15,7 +15,7 @@ from .build import LIB_PATH
 MAX_DEPTH = 8
 MAX_TREE_ROWS = 128
 
-OPT_PERSISTENT_FORWARD, OPT_DEPENDENT_LAUNCH, OPT_L2_PREFETCH, OPT_WAIT_LIMIT_NS = 1, 2, 3, 4
+OPT_PERSISTENT_FORWARD, OPT_DEPENDENT_LAUNCH, OPT_L2_PREFETCH, OPT_WAIT_LIMIT_NS, OPT_DEVICE_LOOP = 1, 2, 3, 4, 5
 BUF_GREEDY, BUF_MARGIN, BUF_FEATURES, BUF_PATH, BUF_STATE, BUF_TOPK_TOK, BUF_TOPK_LP = 1, 2, 3, 4, 5, 6, 7
 
 
@@ -48,7 +48,8 @@ class Tree(C.Structure):
 class Stats(C.Structure):
     _fields_ = [("iterations", C.c_int), ("tokens_emitted", C.c_int), ("accept_len", C.c_int * 16),
                 ("ms_prefill", C.c_float), ("ms_draft", C.c_float), ("ms_verify", C.c_float),
-                ("pos_iterations", C.c_int * 16), ("pos_accept_sum", C.c_int * 16)]
+                ("pos_iterations", C.c_int * 16), ("pos_accept_sum", C.c_int * 16),
+                ("ms_loop", C.c_float), ("device_loop", C.c_int)]
 
 
 EXPORTS = {

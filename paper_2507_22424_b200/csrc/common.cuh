@@ -60,6 +60,16 @@ struct DevTree {
   uint32_t dmask[SV_MAX_TREE][4]; // ancestors-and-self over draft rows (draft mask), by draft row
 };
 
+// Device-resident state of the chunk being generated (specvla_generate_action with the loop on the
+// device): tokens emitted so far per call slot, and the statistics of specvla_stats.
+#define SV_MAX_CHUNK 64
+struct ChunkState {
+  int n_tokens, iterations, max_iterations, pad;
+  int count[SV_MAX_EP];                 // tokens emitted (not clipped)
+  int tokens[SV_MAX_EP][SV_MAX_CHUNK];  // the first n_tokens of them
+  int accept_len[16], pos_iterations[16], pos_accept_sum[16];   // first episode of the call
+};
+
 #define SV_TILE_ROWS 256         // output columns per GEMM tile
 
 // Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may

@@ -133,6 +133,17 @@ struct specvla_ctx {
   char cuda_err[256];
   cudaEvent_t ev[4];
 
+  // chunk loop on the device (specvla_generate_action): draft + verify + append as the body of a
+  // CUDA-graph while node, captured once per (episodes, tree shape, r) and kept
+  bool use_device_loop;
+  ChunkState *chunk;              // device
+  ChunkState *pin_chunk;          // pinned copy read back after the loop, then max_episodes EpState
+  cudaStream_t cap_stream;        // capture happens on a stream of the context's own
+  cudaGraph_t loop_graph;
+  cudaGraphExec_t loop_exec;
+  std::vector<int> loop_key;      // what the kept graph was captured for
+  long long loop_launches_once, loop_launches_iter;   // kernels per graph launch: outside / inside the loop
+
   // optional per-GEMM timing (specvla_profile): events around every GEMM launch, summed per
   // weight-matrix class when the stream is next synchronised
   int prof_mask;                        // phases timed: 1 prefill, 2 draft, 4 verify
@@ -292,6 +303,7 @@ size_t carve(specvla_ctx *c, char *base) {
   c->st = cv.take<EpState>(E);
   c->trees = cv.take<DevTree>(E);
   c->err = cv.take<int>(32);
+  c->chunk = cv.take<ChunkState>(1);
   // persistent forward kernel: packed operands, partial tiles, attention slices, candidates
   if (pk_shapes_ok(d) && d.weight_bits != 8) {
     const size_t G = c->pk_G;
@@ -905,7 +917,8 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
   ctx->hTreeRows.assign(desc->max_episodes, 0);
   const size_t small_b = 4096 * sizeof(int);
   const size_t trees_b = (sizeof(DevTree) * desc->max_episodes + 255) / 256 * 256;
-  ctx->pinned_bytes = small_b + trees_b + ((size_t)desc->max_rows * 11 + SV_MAX_EP + 256) * sizeof(int);
+  const size_t rows_b = ((size_t)desc->max_rows * 11 + SV_MAX_EP + 256) * sizeof(int);
+  ctx->pinned_bytes = small_b + trees_b + rows_b + sizeof(ChunkState) + sizeof(EpState) * desc->max_episodes;
   ctx->cuda_err[0] = 0;
   if (cudaHostAlloc(&ctx->pinned, ctx->pinned_bytes, cudaHostAllocDefault) != cudaSuccess) {
     delete ctx;
@@ -914,6 +927,12 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
   ctx->pin_small = static_cast<int *>(ctx->pinned);
   ctx->pin_trees = reinterpret_cast<DevTree *>(static_cast<char *>(ctx->pinned) + small_b);
   ctx->pin_rows = reinterpret_cast<int *>(static_cast<char *>(ctx->pinned) + small_b + trees_b);
+  ctx->pin_chunk = reinterpret_cast<ChunkState *>(static_cast<char *>(ctx->pinned) + small_b + trees_b + rows_b);
+  ctx->use_device_loop = true;
+  ctx->cap_stream = nullptr;
+  ctx->loop_graph = nullptr;
+  ctx->loop_exec = nullptr;
+  ctx->loop_launches_once = ctx->loop_launches_iter = 0;
   for (int i = 0; i < 4; i++) cudaEventCreate(&ctx->ev[i]);
   ctx->prof_mask = 0;
   ctx->phase = 0;
@@ -938,9 +957,20 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
   return SPECVLA_OK;
 }
 
+// Forgets the captured chunk loop (its launches were recorded under other settings).
+static void drop_loop_graph(specvla_ctx *ctx) {
+  if (ctx->loop_exec) cudaGraphExecDestroy(ctx->loop_exec);
+  if (ctx->loop_graph) cudaGraphDestroy(ctx->loop_graph);
+  ctx->loop_exec = nullptr;
+  ctx->loop_graph = nullptr;
+  ctx->loop_key.clear();
+}
+
 int specvla_destroy(specvla_ctx *ctx) {
   if (!ctx) return SPECVLA_ERR_INVALID_ARG;
   cudaDeviceSynchronize();
+  drop_loop_graph(ctx);
+  if (ctx->cap_stream) cudaStreamDestroy(ctx->cap_stream);
   for (int i = 0; i < 4; i++) cudaEventDestroy(ctx->ev[i]);
   for (cudaEvent_t e : ctx->prof_ev) cudaEventDestroy(e);
   cudaFreeHost(ctx->pinned);
@@ -950,7 +980,9 @@ int specvla_destroy(specvla_ctx *ctx) {
 
 int specvla_set_option(specvla_ctx *ctx, int option, long long value) {
   if (!ctx) return SPECVLA_ERR_INVALID_ARG;
+  drop_loop_graph(ctx);
   switch (option) {
+    case SPECVLA_OPT_DEVICE_LOOP: ctx->use_device_loop = value != 0; break;
     case SPECVLA_OPT_PERSISTENT_FORWARD: ctx->use_pk = value != 0; break;
     case SPECVLA_OPT_DEPENDENT_LAUNCH: ctx->use_pdl = value != 0; break;
     case SPECVLA_OPT_L2_PREFETCH: ctx->use_l2_prefetch = value != 0; break;
@@ -970,13 +1002,35 @@ int specvla_reset(specvla_ctx *ctx, int episode) {
   return SPECVLA_OK;
 }
 
+static int prefill_enqueue(specvla_ctx *ctx, int n_ep, const int *episodes, const void *embeds,
+                           const int *token_ids, const int *lens, float *logits_out, cudaStream_t st);
+
 int specvla_prefill(specvla_ctx *ctx, int n_ep, const int *episodes, const void *embeds,
                     const int *token_ids, const int *lens, int *first_token_out, float *logits_out,
                     void *stream) {
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  TRY(prefill_enqueue(ctx, n_ep, episodes, embeds, token_ids, lens, logits_out, st));
+  int *h_g = ctx->pin_small;
+  CU(cudaMemcpyAsync(h_g, ctx->greedy, n_ep * sizeof(int), cudaMemcpyDeviceToHost, st));
+  CU(cudaMemcpyAsync(h_g + 4000, ctx->err, sizeof(int), cudaMemcpyDeviceToHost, st));
+  CU(cudaStreamSynchronize(st));
+  prof_collect(ctx);
+  if (h_g[4000] != 0) {
+    for (int i = 0; i < n_ep; i++) ctx->hP[episodes[i]] = -1;
+    return SPECVLA_ERR_TIMEOUT;
+  }
+  for (int i = 0; i < n_ep; i++)
+    if (first_token_out) first_token_out[i] = h_g[i];
+  return SPECVLA_OK;
+}
+
+// Validation, row tables and all device work of a prefill, without waiting for it. The host
+// mirror is updated at once: prefix lengths do not depend on results.
+static int prefill_enqueue(specvla_ctx *ctx, int n_ep, const int *episodes, const void *embeds,
+                           const int *token_ids, const int *lens, float *logits_out, cudaStream_t st) {
   TRY(check_episodes(ctx, n_ep, episodes));
   if (!token_ids || !lens) return SPECVLA_ERR_INVALID_ARG;
   const specvla_model_desc &d = ctx->desc;
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
   EpArgs ea{};
   ea.n_ep = n_ep;
   int R = 0;
@@ -1074,20 +1128,17 @@ int specvla_prefill(specvla_ctx *ctx, int n_ep, const int *episodes, const void 
       TRY(draft_forward(ctx, Rd, ed, st));
     }
   }
-  int *h_g = ctx->pin_small;
-  CU(cudaMemcpyAsync(h_g, ctx->greedy, n_ep * sizeof(int), cudaMemcpyDeviceToHost, st));
-  CU(cudaMemcpyAsync(h_g + 4000, ctx->err, sizeof(int), cudaMemcpyDeviceToHost, st));
-  CU(cudaStreamSynchronize(st));
-  prof_collect(ctx);
-  if (h_g[4000] != 0) return SPECVLA_ERR_TIMEOUT;
   for (int i = 0; i < n_ep; i++) {
     ctx->hP[episodes[i]] = lens[i];
     ctx->hPending[episodes[i]] = 1;
     ctx->hTreeRows[episodes[i]] = 0;
-    if (first_token_out) first_token_out[i] = h_g[i];
   }
   return SPECVLA_OK;
 }
+
+static int draft_enqueue(specvla_ctx *ctx, const EpArgs &ea, int R, const specvla_tree_shape *shape, int n_nodes,
+                         int n_tree_rows, cudaStream_t st);
+static int draft_readback(specvla_ctx *ctx, int n_ep, const int *episodes, specvla_tree *trees_out, cudaStream_t st);
 
 int specvla_draft_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const specvla_tree_shape *shape,
                        specvla_tree *trees_out, void *stream) {
@@ -1107,11 +1158,28 @@ int specvla_draft_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const sp
     // target cache: the rows verified; draft cache: one row per node expanded below the root
     if (ctx->hP[e] + n_tree_rows > d.max_seq || ctx->hP[e] + n_draft_rows > d.max_seq) return SPECVLA_ERR_CAPACITY;
     ea.eps[i] = e;
+    // a fixed number of catch-up rows per episode: the pending pairs, the last one repeated (the
+    // launch shapes then do not depend on the accepted length of the previous iteration)
     ea.row0[i] = R;
-    ea.nrows[i] = ctx->hPending[e];
-    R += ctx->hPending[e];
+    ea.nrows[i] = SV_MAX_PENDING;
+    R += SV_MAX_PENDING;
   }
   if (R > d.max_rows || n_ep * 16 > ctx->max_draft_rows) return SPECVLA_ERR_CAPACITY;
+  TRY(draft_enqueue(ctx, ea, R, shape, n_nodes, n_tree_rows, st));
+  for (int i = 0; i < n_ep; i++) {
+    ctx->hPending[episodes[i]] = 0;
+    ctx->hTreeRows[episodes[i]] = n_tree_rows;
+  }
+  return draft_readback(ctx, n_ep, episodes, trees_out, st);
+}
+
+// The device work of a draft call over the episodes of `ea` (SV_MAX_PENDING catch-up rows each):
+// catch-up forward, then level by level head + tree growth + draft forward, then the re-ranking
+// of a dynamic tree. Launch shapes depend only on the tree shape.
+static int draft_enqueue(specvla_ctx *ctx, const EpArgs &ea, int R, const specvla_tree_shape *shape, int n_nodes,
+                         int n_tree_rows, cudaStream_t st) {
+  const specvla_model_desc &d = ctx->desc;
+  const int n_ep = ea.n_ep;
   int lo, hi;
   argmax_range(ctx, &lo, &hi);
 
@@ -1121,10 +1189,6 @@ int specvla_draft_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const sp
          (const float *)ctx->pend_feat, ctx->embed, d.d_model, ctx->xin.p, ctx->xin.plane);
   TRY(draft_forward(ctx, R, ea, st));
   ctx->feat_valid = false;
-  for (int i = 0; i < n_ep; i++) {
-    ctx->hPending[episodes[i]] = 0;
-    ctx->hTreeRows[episodes[i]] = n_tree_rows;
-  }
 
   // Per level: the shared LM head over the rows just run (draft layer outputs as they are: no
   // norm, no row scale) with log-softmax + top-k, then one kernel that grows the tree and writes
@@ -1169,7 +1233,11 @@ int specvla_draft_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const sp
 
   if (n_tree_rows < 1 + n_nodes)
     LAUNCH(tree::rerank_keep_kernel, dim3(n_ep), dim3(SV_MAX_CAND), ea, ctx->trees, n_tree_rows - 1);
+  return SPECVLA_OK;
+}
 
+// Copies the device-resident trees of the call's episodes to the caller's host structs.
+static int draft_readback(specvla_ctx *ctx, int n_ep, const int *episodes, specvla_tree *trees_out, cudaStream_t st) {
   if (trees_out) {
     DevTree *h = ctx->pin_trees;
     for (int i = 0; i < n_ep; i++)
@@ -1329,22 +1397,205 @@ int specvla_score_tree(specvla_ctx *ctx, int n_ep, const int *episodes, const sp
   return SPECVLA_OK;
 }
 
+// Row layout of a call whose episodes all bring `rows` rows.
+static EpArgs uniform_rows(int n_ep, const int *episodes, int rows) {
+  EpArgs ea{};
+  ea.n_ep = n_ep;
+  for (int i = 0; i < n_ep; i++) {
+    ea.eps[i] = episodes[i];
+    ea.row0[i] = i * rows;
+    ea.nrows[i] = rows;
+  }
+  return ea;
+}
+
+// Captures the chunk loop of Algorithm 1 for these episodes, this tree shape and this r as a graph:
+// a kernel that arms the loop, then a while node whose body drafts the trees, verifies them and
+// appends the emitted tokens; the appending kernel decides whether the body runs again. Launch
+// shapes inside the body depend only on the tree shape, everything else is read from device state.
+static int build_loop_graph(specvla_ctx *ctx, int n_ep, const int *episodes, const specvla_tree_shape *shape,
+                            int n_nodes, int n_tree_rows, int r) {
+  drop_loop_graph(ctx);
+  if (!ctx->cap_stream) CU(cudaStreamCreateWithFlags(&ctx->cap_stream, cudaStreamNonBlocking));
+  cudaStream_t st = ctx->cap_stream;
+  CU(cudaGraphCreate(&ctx->loop_graph, 0));
+  cudaGraphConditionalHandle handle;
+  CU(cudaGraphConditionalHandleCreate(&handle, ctx->loop_graph, 0, cudaGraphCondAssignDefault));
+  cudaGraphNode_t arm_node, loop_node;
+  {
+    const ChunkState *cs = ctx->chunk;
+    void *args[2] = {&cs, &handle};
+    cudaKernelNodeParams kp = {};
+    kp.func = (void *)tree::chunk_arm_kernel;
+    kp.gridDim = dim3(1);
+    kp.blockDim = dim3(1);
+    kp.kernelParams = args;
+    CU(cudaGraphAddKernelNode(&arm_node, ctx->loop_graph, nullptr, 0, &kp));
+  }
+  cudaGraphNodeParams np = {};
+  np.type = cudaGraphNodeTypeConditional;
+  np.conditional.handle = handle;
+  np.conditional.type = cudaGraphCondTypeWhile;
+  np.conditional.size = 1;
+  CU(cudaGraphAddNode(&loop_node, ctx->loop_graph, &arm_node, 1, &np));
+  cudaGraph_t body = np.conditional.phGraph_out[0];
+
+  const long long before = ctx->launches;
+  CU(cudaStreamBeginCaptureToGraph(st, body, nullptr, nullptr, 0, cudaStreamCaptureModeRelaxed));
+  auto record = [&]() -> int {
+    int rows = 1;
+    if (shape->depth > 0) {
+      const EpArgs ea = uniform_rows(n_ep, episodes, SV_MAX_PENDING);
+      TRY(draft_enqueue(ctx, ea, n_ep * SV_MAX_PENDING, shape, n_nodes, n_tree_rows, st));
+      rows = n_tree_rows;
+    } else {
+      const EpArgs ea = uniform_rows(n_ep, episodes, 1);
+      LAUNCH(tree::root_only_tree_kernel, dim3(1), dim3(SV_MAX_EP), ea, ctx->trees);
+    }
+    const EpArgs ev = uniform_rows(n_ep, episodes, rows);
+    TRY(verify_device_trees(ctx, ev, n_ep * rows, r, nullptr, st));
+    LAUNCH(tree::chunk_append_kernel, dim3(1), dim3(SV_MAX_EP), ev, ctx->chunk, (const int *)ctx->out_m,
+           (const int *)ctx->out_tok, (const int *)ctx->err, handle);
+    return SPECVLA_OK;
+  };
+  const int rc = record();
+  cudaGraph_t captured = nullptr;
+  const cudaError_t ce = cudaStreamEndCapture(st, &captured);
+  ctx->loop_launches_iter = ctx->launches - before;
+  ctx->launches = before;
+  ctx->loop_launches_once = 1;
+  if (rc != SPECVLA_OK || ce != cudaSuccess) {
+    cudaGetLastError();
+    drop_loop_graph(ctx);
+    if (rc != SPECVLA_OK) return rc;
+    CU(ce);
+  }
+  const cudaError_t ie = cudaGraphInstantiate(&ctx->loop_exec, ctx->loop_graph, 0);
+  if (ie != cudaSuccess) {
+    ctx->loop_exec = nullptr;
+    cudaGetLastError();
+    drop_loop_graph(ctx);
+    CU(ie);
+  }
+  return SPECVLA_OK;
+}
+
+static std::vector<int> loop_key_of(const specvla_ctx *ctx, int n_ep, const int *episodes,
+                                    const specvla_tree_shape *shape, int r) {
+  std::vector<int> k = {n_ep, r, shape->depth, shape->keep, (int)ctx->use_pdl, (int)ctx->use_l2_prefetch};
+  for (int i = 0; i < n_ep; i++) k.push_back(episodes[i]);
+  for (int l = 0; l < shape->depth; l++) {
+    k.push_back(shape->branch[l]);
+    k.push_back(shape->expand[l]);
+  }
+  return k;
+}
+
+// The chunk with its loop on the device: prefill, then ONE graph launch for all iterations, then
+// one read-back of tokens, statistics and episode state.
+static int generate_on_device(specvla_ctx *ctx, int n_ep, const int *episodes, const void *embeds,
+                              const int *token_ids, const int *lens, const specvla_tree_shape *shape, int n_nodes,
+                              int n_tree_rows, int r, int n_tokens, int *tokens_out, specvla_stats *stats,
+                              cudaStream_t st) {
+  const std::vector<int> key = loop_key_of(ctx, n_ep, episodes, shape, r);
+  if (!ctx->loop_exec || key != ctx->loop_key) {
+    TRY(build_loop_graph(ctx, n_ep, episodes, shape, n_nodes, n_tree_rows, r));
+    ctx->loop_key = key;
+  }
+  float ms = 0.f;
+  CU(cudaEventRecord(ctx->ev[0], st));
+  TRY(prefill_enqueue(ctx, n_ep, episodes, embeds, token_ids, lens, nullptr, st));
+  CU(cudaEventRecord(ctx->ev[1], st));
+  ctx->phase = 4;
+  const EpArgs ea = uniform_rows(n_ep, episodes, 1);
+  LAUNCH(tree::chunk_begin_kernel, dim3(1), dim3(SV_MAX_EP), ea, ctx->chunk, (const int *)ctx->greedy, n_tokens,
+         4 * n_tokens);
+  CU(cudaGraphLaunch(ctx->loop_exec, st));
+  CU(cudaEventRecord(ctx->ev[2], st));
+  ChunkState *h = ctx->pin_chunk;
+  EpState *hs = reinterpret_cast<EpState *>(h + 1);
+  CU(cudaMemcpyAsync(h, ctx->chunk, sizeof(ChunkState), cudaMemcpyDeviceToHost, st));
+  CU(cudaMemcpyAsync(hs, ctx->st, sizeof(EpState) * ctx->desc.max_episodes, cudaMemcpyDeviceToHost, st));
+  CU(cudaMemcpyAsync(ctx->pin_small + 4000, ctx->err, sizeof(int), cudaMemcpyDeviceToHost, st));
+  CU(cudaStreamSynchronize(st));
+  ctx->launches += ctx->loop_launches_once + (long long)h->iterations * ctx->loop_launches_iter;
+  ctx->feat_valid = false;
+  bool complete = true;
+  for (int i = 0; i < n_ep; i++) {
+    const int e = episodes[i];
+    ctx->hP[e] = hs[e].P;
+    ctx->hPending[e] = hs[e].n_pending;
+    ctx->hTreeRows[e] = 0;
+    complete &= h->count[i] >= n_tokens;
+  }
+  if (ctx->pin_small[4000] != 0) {
+    for (int i = 0; i < n_ep; i++) ctx->hP[episodes[i]] = -1;
+    return SPECVLA_ERR_TIMEOUT;
+  }
+  if (!complete) return SPECVLA_ERR_BAD_STATE;
+  for (int i = 0; i < n_ep; i++)
+    for (int k = 0; k < n_tokens; k++) tokens_out[(size_t)i * n_tokens + k] = h->tokens[i][k];
+  if (stats) {
+    CU(cudaEventElapsedTime(&ms, ctx->ev[0], ctx->ev[1]));
+    stats->ms_prefill = ms;
+    CU(cudaEventElapsedTime(&ms, ctx->ev[1], ctx->ev[2]));
+    stats->ms_loop = ms;
+    stats->device_loop = 1;
+    stats->iterations = h->iterations;
+    stats->tokens_emitted = h->count[0];
+    for (int k = 0; k < 16; k++) {
+      stats->accept_len[k] = h->accept_len[k];
+      stats->pos_iterations[k] = h->pos_iterations[k];
+      stats->pos_accept_sum[k] = h->pos_accept_sum[k];
+    }
+  }
+  return SPECVLA_OK;
+}
+
 int specvla_generate_action(specvla_ctx *ctx, int n_ep, const int *episodes, const void *embeds,
                             const int *token_ids, const int *lens, const specvla_tree_shape *shape, int r,
                             int n_tokens, int *tokens_out, float *actions_out, specvla_stats *stats,
                             void *stream) {
   TRY(check_episodes(ctx, n_ep, episodes));
-  int n_nodes = 0;
-  TRY(validate_shape(shape, &n_nodes));
-  if (r < 0 || n_tokens < 1 || n_tokens > 64 || !tokens_out) return SPECVLA_ERR_INVALID_ARG;
+  int n_nodes = 0, n_tree_rows = 0;
+  TRY(validate_shape(shape, &n_nodes, &n_tree_rows));
+  if (r < 0 || n_tokens < 1 || n_tokens > SV_MAX_CHUNK || !tokens_out || !lens) return SPECVLA_ERR_INVALID_ARG;
   if (shape->depth > 0 && !ctx->has_draft) return SPECVLA_ERR_BAD_STATE;
   const specvla_model_desc &d = ctx->desc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int W = SV_MAX_DEPTH + 1;
-  std::vector<int> first(n_ep), count(n_ep, 0), m_out(n_ep), tok_out((size_t)n_ep * W);
   if (stats) memset(stats, 0, sizeof(*stats));
-  float ms = 0.f;
+  auto actions = [&]() {
+    if (actions_out)
+      for (int i = 0; i < n_ep * n_tokens; i++) {
+        const int b = tokens_out[i] - d.action_base;
+        actions_out[i] = (b >= 0 && b < d.n_bins) ? (-1.f + (2.f * b + 1.f) / d.n_bins) : NAN;
+      }
+  };
 
+  // The loop runs on the device when its launches are the same every iteration (no depth pruning,
+  // no per-GEMM timing, the per-GEMM forward) and the caches certainly hold every iteration's rows.
+  bool on_device = ctx->use_device_loop && !shape->prune && ctx->prof_mask == 0 && !(ctx->pk_ok && ctx->use_pk);
+  if (on_device) {
+    const int rows = shape->depth > 0 ? n_tree_rows : 1;
+    int draft_rows = 0;
+    for (int l = 1; l < shape->depth; l++) draft_rows += shape->expand[l];
+    for (int i = 0; i < n_ep; i++) {
+      const int worst = lens[i] + n_tokens + shape->depth;      // committed positions never exceed this
+      on_device &= lens[i] >= 1 && worst + rows <= d.max_seq && worst + draft_rows <= d.max_seq;
+    }
+    on_device &= n_ep * rows <= d.max_rows && n_ep * rows <= ctx->max_lm_rows &&
+                 n_ep * SV_MAX_PENDING <= d.max_rows && n_ep * 16 <= ctx->max_draft_rows;
+  }
+  if (on_device) {
+    TRY(generate_on_device(ctx, n_ep, episodes, embeds, token_ids, lens, shape, n_nodes, n_tree_rows, r, n_tokens,
+                           tokens_out, stats, st));
+    actions();
+    return SPECVLA_OK;
+  }
+
+  std::vector<int> first(n_ep), count(n_ep, 0), m_out(n_ep), tok_out((size_t)n_ep * W);
+  float ms = 0.f;
   CU(cudaEventRecord(ctx->ev[0], st));
   TRY(specvla_prefill(ctx, n_ep, episodes, embeds, token_ids, lens, first.data(), nullptr, stream));
   CU(cudaEventRecord(ctx->ev[1], st));
@@ -1376,15 +1627,9 @@ int specvla_generate_action(specvla_ctx *ctx, int n_ep, const int *episodes, con
       TRY(specvla_draft_tree(ctx, n_ep, episodes, &now, nullptr, stream));
     } else {
       // no drafting: a one-row tree (the root) per episode = one autoregressive step
-      DevTree *h = ctx->pin_trees;
-      for (int i = 0; i < n_ep; i++) {
-        memset(&h[i], 0, sizeof(DevTree));
-        h[i].n_rows = 1;
-        h[i].tok[0] = -1;
-        h[i].parent[0] = -1;
-        CU(cudaMemcpyAsync(&ctx->trees[episodes[i]], &h[i], sizeof(DevTree), cudaMemcpyHostToDevice, st));
-        ctx->hTreeRows[episodes[i]] = 1;
-      }
+      const EpArgs one = uniform_rows(n_ep, episodes, 1);
+      LAUNCH(tree::root_only_tree_kernel, dim3(1), dim3(SV_MAX_EP), one, ctx->trees);
+      for (int i = 0; i < n_ep; i++) ctx->hTreeRows[episodes[i]] = 1;
     }
     CU(cudaEventRecord(ctx->ev[1], st));
     for (int i = 0; i < n_ep; i++) {
@@ -1422,12 +1667,9 @@ int specvla_generate_action(specvla_ctx *ctx, int n_ep, const int *episodes, con
   if (stats) {
     stats->iterations = iterations;
     stats->tokens_emitted = count[0];
+    stats->ms_loop = stats->ms_draft + stats->ms_verify;
   }
-  if (actions_out)
-    for (int i = 0; i < n_ep * n_tokens; i++) {
-      const int b = tokens_out[i] - d.action_base;
-      actions_out[i] = (b >= 0 && b < d.n_bins) ? (-1.f + (2.f * b + 1.f) / d.n_bins) : NAN;
-    }
+  actions();
   return SPECVLA_OK;
 }
 

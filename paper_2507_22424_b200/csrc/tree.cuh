@@ -7,6 +7,81 @@
 namespace tree {
 
 // ---------------------------------------------------------------------------------------
+// The chunk loop of Algorithm 1 on the device: the first token after prefill, then after every
+// iteration the m accepted draft tokens and the target's token are appended per episode; the loop
+// (a CUDA-graph while node) goes on while an episode still misses tokens.
+__global__ void chunk_begin_kernel(EpArgs a, ChunkState *cs, const int *__restrict__ first_tok, int n_tokens,
+                                   int max_iterations) {
+  pdl_launch();
+  pdl_wait();
+  const int i = threadIdx.x;
+  if (i < a.n_ep) {
+    cs->count[i] = 1;
+    cs->tokens[i][0] = first_tok[i];
+  }
+  if (i < 16) {
+    cs->accept_len[i] = 0;
+    cs->pos_iterations[i] = 0;
+    cs->pos_accept_sum[i] = 0;
+  }
+  if (i == 0) {
+    cs->n_tokens = n_tokens;
+    cs->iterations = 0;
+    cs->max_iterations = max_iterations;
+  }
+}
+// Arms the loop (in front of the while node): it runs only if tokens are missing.
+__global__ void chunk_arm_kernel(const ChunkState *cs, cudaGraphConditionalHandle handle) {
+  cudaGraphSetConditional(handle, cs->n_tokens > 1 ? 1u : 0u);
+}
+__global__ void chunk_append_kernel(EpArgs a, ChunkState *cs, const int *__restrict__ out_m,
+                                    const int *__restrict__ out_tok, const int *__restrict__ err,
+                                    cudaGraphConditionalHandle handle) {
+  __shared__ int s_missing;
+  pdl_launch();
+  pdl_wait();
+  const int i = threadIdx.x, n_tokens = cs->n_tokens;
+  if (i == 0) s_missing = 0;
+  __syncthreads();
+  if (i < a.n_ep) {
+    const int m = out_m[i];
+    int c = cs->count[i];
+    if (i == 0) {
+      const int it = cs->iterations, pos = c - 1;
+      if (it < 16) cs->accept_len[it] = m;
+      if (pos >= 0 && pos < 16) {
+        cs->pos_iterations[pos]++;
+        cs->pos_accept_sum[pos] += m;
+      }
+    }
+    for (int k = 0; k <= m; k++, c++)
+      if (c < n_tokens) cs->tokens[i][c] = out_tok[i * (SV_MAX_DEPTH + 1) + k];
+    cs->count[i] = c;
+    if (c < n_tokens) atomicAdd(&s_missing, 1);
+  }
+  __syncthreads();
+  if (i == 0) {
+    const int it = ++cs->iterations;
+    // a device-side wait that gave up (status word set) ends the loop as well
+    cudaGraphSetConditional(handle, (s_missing > 0 && it < cs->max_iterations && err[0] == 0) ? 1u : 0u);
+  }
+}
+// A one-row tree (the root alone) per episode: an iteration without drafting is one autoregressive step.
+__global__ void root_only_tree_kernel(EpArgs a, DevTree *trees) {
+  pdl_launch();
+  pdl_wait();
+  const int i = threadIdx.x;
+  if (i >= a.n_ep) return;
+  DevTree &tr = trees[a.eps[i]];
+  tr.n_rows = 1;
+  tr.tok[0] = -1;
+  tr.parent[0] = -1;
+  tr.depth[0] = 0;
+  tr.score[0] = 0.f;
+}
+
+
+// ---------------------------------------------------------------------------------------
 // Verification rows of each episode's tree: row i sits at position P + depth[i], slot P + i,
 // sees the P committed slots, its ancestors and itself (the mask is computed here from the
 // parents, so trees need only tok / parent / depth). One CTA per episode.
@@ -82,25 +157,28 @@ __device__ __forceinline__ void write_draft_input_row(const float *__restrict__ 
   }
 }
 
-// Start of a draft call, one CTA per episode: the (feature_j, token_j) pairs pending since the
+// Start of a draft call, one CTA per episode: the n (feature_j, token_j) pairs pending since the
 // last commit become draft rows at positions Pd + j, causal among themselves (row table and
-// model input written here); Pd advances; a new tree is opened whose root is the episode's last
-// emitted token, scored by the last of these rows.
+// model input written here); Pd advances by n; a new tree is opened whose root is the episode's
+// last emitted token. The call always runs a.nrows[i] >= n rows per episode, whatever n is (so that
+// its launches do not depend on the accepted length, which only the device knows): the rows past
+// n - 1 repeat row n - 1 exactly (same input, position, cache slot and mask: they compute and write
+// the same values), and the LAST row, which is pair n - 1 either way, scores the root's children.
 __global__ void __launch_bounds__(256)
 catchup_input_kernel(EpArgs a, EpState *st, DevTree *trees, RowTable rt, const float *__restrict__ pend_feat,
                      const bf16 *__restrict__ E, int d, bf16 *__restrict__ xin, size_t plane) {
   __shared__ int s_n, s_tok[SV_MAX_PENDING];
   pdl_launch();
   pdl_wait();
-  const int i = blockIdx.x, e = a.eps[i];
+  const int i = blockIdx.x, e = a.eps[i], rows = a.nrows[i];
   EpState &s = st[e];
   if (threadIdx.x == 0) s_n = s.n_pending;
   if (threadIdx.x < SV_MAX_PENDING) s_tok[threadIdx.x] = s.pending_tok[threadIdx.x];
   __syncthreads();
-  const int n = s_n, Pd = s.Pd;
+  const int n = max(1, min(s_n, rows)), Pd = s.Pd;
   __syncthreads();                                  // everybody has the old Pd
-  if (threadIdx.x < n) {
-    const int j = threadIdx.x, r = a.row0[i] + j;
+  if (threadIdx.x < rows) {
+    const int j = min((int)threadIdx.x, n - 1), r = a.row0[i] + threadIdx.x;
     rt.tok[r] = s_tok[j];
     rt.src[r] = 0;
     rt.ep[r] = e;
@@ -120,16 +198,18 @@ catchup_input_kernel(EpArgs a, EpState *st, DevTree *trees, RowTable rt, const f
     tr.depth[0] = 0;
     tr.score[0] = 0.f;
     tr.drow[0] = 0;
-    tr.xrow[0] = a.row0[i] + n - 1;
+    tr.xrow[0] = a.row0[i] + rows - 1;
     for (int w = 0; w < 4; w++) tr.dmask[0][w] = 0;
     tr.level_begin = 0;
     tr.level_end = 1;
     tr.sel_count = 1;
     tr.sel[0] = 0;
   }
-  for (int j = 0; j < n; j++)
-    write_draft_input_row(pend_feat + (size_t)(e * SV_MAX_PENDING + j) * d, E + (size_t)s_tok[j] * d, d, xin, plane,
+  for (int j = 0; j < rows; j++) {
+    const int jj = min(j, n - 1);
+    write_draft_input_row(pend_feat + (size_t)(e * SV_MAX_PENDING + jj) * d, E + (size_t)s_tok[jj] * d, d, xin, plane,
                           a.row0[i] + j);
+  }
 }
 
 // One level of tree growth and the next level's model input, one CTA per episode. The rows

@@ -105,10 +105,18 @@ def test_c1_generate_action_strict_equals_greedy(env):
                                             env["shape"], 0, 7)
     ar, _, _ = gpu.generate_action([0], env["emb"], env["ids"].tolist(), [len(env["ids"])],
                                    make_shape((), ()), 0, 7)
-    assert toks == ar
+    assert toks == ar and stats.device_loop == 1
+    # the same loop driven from the host (one read-back per iteration): same chunk, same statistics
+    from paper_2507_22424_b200 import binding as B
+    gpu.set_option(B.OPT_DEVICE_LOOP, 0)
+    host, _, sth = gpu.generate_action([0], env["emb"], env["ids"].tolist(), [len(env["ids"])], env["shape"], 0, 7)
+    gpu.set_option(B.OPT_DEVICE_LOOP, 1)
+    assert host == toks and sth.device_loop == 0 and sth.iterations == stats.iterations
+    assert list(sth.accept_len) == list(stats.accept_len) and list(sth.pos_accept_sum) == list(stats.pos_accept_sum)
+    print(f"loop on the device {stats.ms_loop:.2f} ms, on the host {sth.ms_loop:.2f} ms ({stats.iterations} iterations)")
     pruned, _, st3 = gpu.generate_action([0], env["emb"], env["ids"].tolist(), [len(env["ids"])],
                                          make_shape(C.TREE_26.branch, C.TREE_26.expand, prune=True), 0, 7)
-    assert pruned == toks and st3.ms_draft < stats.ms_draft
+    assert pruned == toks and st3.ms_draft < sth.ms_draft
     # the paper's own tree (Section 5.1 / Table 4): top-8, depth 5, the best 50 of 264 drafted nodes
     dyn, _, st4 = gpu.generate_action([0], env["emb"], env["ids"].tolist(), [len(env["ids"])],
                                       make_shape((8,) * 5, (1, 8, 8, 8, 8), keep=50), 0, 7)

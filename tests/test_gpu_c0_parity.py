@@ -282,6 +282,53 @@ def test_generate_action_strict_equals_greedy_decoding(c0, wcuda):
     gpu.close()
 
 
+@pytest.mark.parametrize("branch,expand,keep,r,n_tokens", [
+    ((4, 2, 2, 1, 1), (1, 2, 2, 2, 2), 0, 0, 7), ((4, 2, 2, 1, 1), (1, 2, 2, 2, 2), 0, 4, 7),
+    ((8, 8, 8), (1, 8, 8), 50, 2, 7), ((), (), 0, 0, 7), ((3, 2), (1, 3), 0, 9, 12), ((2,), (1,), 0, 0, 1)])
+def test_chunk_loop_on_the_device_equals_the_loop_on_the_host(c0, wcuda, branch, expand, keep, r, n_tokens):
+    """Algorithm 1's loop as one graph launch (a while node around draft, verification and the
+    appending of the emitted tokens) against the same loop driven from the host with a read-back
+    per iteration: tokens, actions, iteration count, accepted lengths, per-position statistics,
+    episode state, both caches, the launch count, and what a further draft + verification gives."""
+    from paper_2507_22424_b200 import binding as B
+    shape = B.make_shape(branch, expand, keep=keep)
+    emb2 = rng.normal_bf16(5, 1, (40, c0["desc"].d_model), 1.0)
+    ids2 = torch.full((40,), -1, dtype=torch.int32)
+    emb = torch.cat([c0["embeds"], emb2]).cuda()
+    ids = c0["ids"].tolist() + ids2.tolist()
+    out = []
+    for device_loop in (1, 0):
+        gpu = _gpu(c0, wcuda)
+        gpu.set_option(B.OPT_DEVICE_LOOP, device_loop)
+        before = gpu.kernel_launches()
+        toks, acts, st = gpu.generate_action([1, 0], emb, ids, [64, 40], shape, r, n_tokens)
+        launches = gpu.kernel_launches() - before
+        again, _, st_again = gpu.generate_action([1, 0], emb, ids, [64, 40], shape, r, n_tokens)   # kept graph
+        assert again == toks and st_again.iterations == st.iterations
+        assert st.device_loop == device_loop
+        state = gpu.read_buffer(5, 8, torch.int32).tolist()
+        P = [state[4], state[0]]
+        kv = [gpu.read_kv(e, l, w, 0, P[i]) for i, e in enumerate((1, 0)) for l in range(c0["desc"].n_layers)
+              for w in (0, 1)]
+        kvd = [gpu.read_kv(e, 0, w, 0, state[4 * e + 1], draft=True) for e in (1, 0) for w in (0, 1)]
+        follow = None
+        if branch:
+            trees = gpu.draft_tree([1, 0], shape)
+            follow = (trees, gpu.verify_tree([1, 0], None, r))
+        out.append(dict(toks=toks, acts=acts, it=st.iterations, emitted=st.tokens_emitted,
+                        m=list(st.accept_len), pi=list(st.pos_iterations), ps=list(st.pos_accept_sum),
+                        state=state, kv=kv, kvd=kvd, follow=follow, launches=launches))
+        gpu.close()
+    dev, host = out
+    for key in ("toks", "acts", "it", "emitted", "m", "pi", "ps", "state", "follow"):
+        assert dev[key] == host[key], key
+    for a, b in zip(dev["kv"] + dev["kvd"], host["kv"] + host["kvd"]):
+        assert torch.equal(a, b)
+    assert len(dev["toks"][0]) == n_tokens and dev["it"] >= (1 if n_tokens > 1 else 0)
+    # the device loop adds: the kernel that starts the chunk, the one that arms the loop, one append per iteration
+    assert dev["launches"] == host["launches"] + 2 + dev["it"]
+
+
 def test_two_episodes_ragged_prefixes(c0, wcuda):
     """Two episodes with different prefix lengths (one of them with text ids, i.e. rows gathered
     from the embedding) in one prefill call and one verification call equal two separate oracle
