@@ -30,6 +30,7 @@ namespace gemm_ck {
 using namespace gemm_tc;
 
 constexpr int MAX_S = 8;                   // largest cluster = K slices per tile (portable limit)
+constexpr long FIXED_CLOCKS = 12000;       // start, accumulator read-out and exit of a CTA (cost estimate of a launch plan)
 
 __device__ __forceinline__ uint32_t cluster_size() {
   uint32_t r;
@@ -112,13 +113,15 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
   const int n_units = kb1 - kb0;
   const long long u0 = (long long)tile * KB + kb0;
   const int tiles = gridDim.x / S;
-  // rows of this CTA: the blockIdx.y-th 128-row chunk. The last chunk of a multi-chunk launch may
-  // be narrower than TN: it has a tensor map with its own box and MMAs of its own width.
-  const int row0 = ea.row0 + (int)blockIdx.y * MAX_T;
-  const int T = ea.T - (int)blockIdx.y * MAX_T < MAX_T ? ea.T - (int)blockIdx.y * MAX_T : MAX_T;
-  const bool tail = TN == MAX_T && blockIdx.y == gridDim.y - 1;
-  const int tn = tail ? ea.tn_tail : TN;
-  const CUtensorMap *xmap = tail ? &tmXtail : &tmX;
+  // rows of this CTA: the blockIdx.y-th chunk. The 128-row instantiation takes its chunk length
+  // and MMA width from the launch (rows are spread evenly over the chunks of a long launch, so the
+  // width is rarely the full 128); the last chunk has a tensor map with its own box.
+  const int row0 = ea.row0 + (int)blockIdx.y * ea.chunk_rows;
+  const int T = ea.T - (int)blockIdx.y * ea.chunk_rows < ea.chunk_rows ? ea.T - (int)blockIdx.y * ea.chunk_rows
+                                                                         : ea.chunk_rows;
+  const bool tail = blockIdx.y == gridDim.y - 1;
+  const int tn = TN == MAX_T ? (tail ? ea.tn_tail : ea.tn_chunk) : TN;
+  const CUtensorMap *xmap = (TN == MAX_T && tail) ? &tmXtail : &tmX;
   constexpr int W_LOAD_BYTES = Q8 ? W_STAGE_BYTES / 2 : W_STAGE_BYTES;   // int8 codes: half the bytes from HBM
   const uint32_t stage_tx = (uint32_t)(W_LOAD_BYTES + 2 * tn * BK * 2);
   const uint32_t idesc = instr_desc(2 * tn);
@@ -431,23 +434,53 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       if (swiglu) ws2 = *reinterpret_cast<const float4 *>(ea.wscale + ea.up_off + n);
     }
     auto scaled = [](float4 v, const float4 &w) { return make_float4(v.x * w.x, v.y * w.y, v.z * w.z, v.w * w.w); };
-    int iter = 0;
-    for (int t = rank + rg * S; t < T; t += RG * S, iter++) {
+    // The rows are taken U at a time: first every global operand of the U rows, then their partial
+    // sums, then the arithmetic and the stores, so that a long tile (prefill: up to 32 rows per
+    // thread) pays the load latencies once per batch instead of once per row.
+    constexpr int U = TN == MAX_T ? 4 : 1;
+    const int tstep = RG * S;
+    for (int tb = rank + rg * S, iter0 = 0; tb < T; tb += U * tstep, iter0 += U) {
+      float4 xo_[U], cs01_[U], cs23_[U], v_[U], w_[U];
+#pragma unroll
+      for (int u = 0; u < U; u++) {
+        const int t = tb + u * tstep, iter = iter0 + u;
+        xo_[u] = iter == 0 ? xpre0 : xpre1;
+        cs01_[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        cs23_[u] = cs01_[u];
+        if (t < T) {
+          // global operands first (the first two rows' residuals and, up to 32 rows, the RoPE
+          // factors were fetched in part 1)
+          if (MODE == EPI_RESID && ea.accumulate && col_ok && iter >= 2)
+            xo_[u] = *reinterpret_cast<const float4 *>(ea.x + (size_t)(row0 + t) * ea.N + n);
+          if (rot) {
+            const float2 *cs = rope_staged ? s_rope + t * ROPE_HALF + (lo ? jq : jq - half)
+                                           : ea.rope_tab + (size_t)s_pos[t] * half + (lo ? jq : jq - half);
+            cs01_[u] = *reinterpret_cast<const float4 *>(cs);
+            cs23_[u] = *reinterpret_cast<const float4 *>(cs + 2);
+          }
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < U; u++) {
+        const int t = tb + u * tstep;
+        v_[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        w_[u] = v_[u];
+        if (t < T) {
+          v_[u] = partial_sum(t * BM + c4);
+          // the partner columns of the rotation (dh / 2 away) are in the same tile; so is the up projection
+          if (rot) w_[u] = partial_sum(t * BM + c4 + (lo ? half : -half));
+          if (swiglu) w_[u] = partial_sum(t * BM + 128 + c4);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < U; u++) {
+      const int t = tb + u * tstep;
+      if (t >= T) break;
       const size_t row = (size_t)(row0 + t);
       const float sc = s_scale[t];
-      // global operands first (the first two rows' residuals and, up to 32 rows, the RoPE
-      // factors were fetched in part 1)
-      float4 xo = iter == 0 ? xpre0 : xpre1, cs01 = make_float4(0.f, 0.f, 0.f, 0.f), cs23 = cs01;
-      if (MODE == EPI_RESID && ea.accumulate && col_ok && iter >= 2)
-        xo = *reinterpret_cast<const float4 *>(ea.x + row * ea.N + n);
-      if (rot) {
-        const float2 *cs = rope_staged ? s_rope + t * ROPE_HALF + (lo ? jq : jq - half)
-                                       : ea.rope_tab + (size_t)s_pos[t] * half + (lo ? jq : jq - half);
-        cs01 = *reinterpret_cast<const float4 *>(cs);
-        cs23 = *reinterpret_cast<const float4 *>(cs + 2);
-      }
+      const float4 xo = xo_[u], cs01 = cs01_[u], cs23 = cs23_[u];
       const int slot = MODE == EPI_QKV ? s_slot[t] : 0, ep = MODE == EPI_QKV ? s_ep[t] : 0;
-      float4 v = partial_sum(t * BM + c4);
+      float4 v = v_[u];
       if (Q8) v = scaled(v, ws);
       if (MODE == EPI_PLAIN) {
         const float4 ov = make_float4(sc * v.x, sc * v.y, sc * v.z, sc * v.w);
@@ -527,10 +560,9 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           }
         }
       } else if (MODE == EPI_QKV) {
-        // the partner columns of the rotation (dh / 2 away) are in the same tile
         float4 o = make_float4(sc * v.x, sc * v.y, sc * v.z, sc * v.w);
         if (rot) {
-          float4 w = partial_sum(t * BM + c4 + (lo ? half : -half));
+          float4 w = w_[u];
           if (Q8) w = scaled(w, ws2);
           const float sg = lo ? -sc : sc;
           o.x = o.x * cs01.x + sg * w.x * cs01.y;
@@ -545,15 +577,15 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           *reinterpret_cast<float4 *>(dst) = o;
         }
       } else if (swiglu) {
-        float4 u = partial_sum(t * BM + 128 + c4);
-        if (Q8) u = scaled(u, ws2);
+        float4 up = w_[u];
+        if (Q8) up = scaled(up, ws2);
         if (col_ok) {
           const float gx = sc * v.x, gy = sc * v.y, gz = sc * v.z, gw = sc * v.w;
           store_limbs4(ea.hid, ea.hid_plane, row * ea.N + n,
-                       make_float4(__fdividef(gx, 1.f + __expf(-gx)) * (sc * u.x),
-                                   __fdividef(gy, 1.f + __expf(-gy)) * (sc * u.y),
-                                   __fdividef(gz, 1.f + __expf(-gz)) * (sc * u.z),
-                                   __fdividef(gw, 1.f + __expf(-gw)) * (sc * u.w)));
+                       make_float4(__fdividef(gx, 1.f + __expf(-gx)) * (sc * up.x),
+                                   __fdividef(gy, 1.f + __expf(-gy)) * (sc * up.y),
+                                   __fdividef(gz, 1.f + __expf(-gz)) * (sc * up.z),
+                                   __fdividef(gw, 1.f + __expf(-gw)) * (sc * up.w)));
         }
       } else {
         float s2 = 0.f;
@@ -569,6 +601,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         }
         s2 = warp_sum(s2);
         if (lane == 0) s_red[warp - 2][t] = s2;
+      }
       }
     }
   }
@@ -606,7 +639,7 @@ inline cudaError_t launch_tq(const CUtensorMap &tmW, const CUtensorMap &tmX, con
   cudaError_t e = cudaFuncSetAttribute(gemm_ck_kernel<TN, MODE, Q8>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(tiles * S, (ea.T + MAX_T - 1) / MAX_T);
+  cfg.gridDim = dim3(tiles * S, (ea.T + ea.chunk_rows - 1) / ea.chunk_rows);
   cfg.blockDim = dim3(THREADS);
   cfg.dynamicSmemBytes = SMEM;
   cfg.stream = st;
@@ -698,12 +731,55 @@ inline int slices_for(int units, int KB, const ClusterFit &fit) {
   return best;
 }
 
-// One launch over ea.T rows in chunks of 128 (grid y). tmX: the X map with box rows
-// tn_of(min(ea.T, 128)); tmXtail: the map for the last chunk when ea.T > 128 (box rows
-// ea.tn_tail), else unused.
+// How a launch over R rows is cut: up to 128 rows are one chunk of the instantiation tn_of(R)
+// (between 65 and 128 rows: MMAs as wide as the rows need, to the next multiple of 8). Longer
+// launches (prefill, batched verification) are tensor-bound, and what counts is how evenly the
+// work fills the SMs: the rows are spread evenly over `chunks` chunks (grid y) of the 128-row
+// instantiation, and chunk count and K slices are chosen together by a cost estimate in SM
+// clocks: waves x (fixed part of a CTA + its K blocks x clocks per K block), where a K block of tn
+// rows costs 512 + 6 tn clocks (what its 64 KB + 768 tn bytes of shared-memory traffic take at
+// 128 bytes per clock; the MMAs themselves need 8 tn).
+struct RowPlan {
+  int chunks, chunk_rows, tn_chunk, tn_tail, S;
+};
+inline int ceil8(int x) { return (x + 7) / 8 * 8; }
+inline RowPlan plan_rows(int R, int tiles, int KB, const ClusterFit &fit) {
+  RowPlan p = {1, MAX_T, tn_of(R), tn_of(R), 1};
+  if (R <= MAX_T) {
+    if (R > 64) p.tn_chunk = p.tn_tail = ceil8(R);
+    p.S = slices_for(tiles, KB, fit);
+    return p;
+  }
+  const int fit1 = fit.max_active[1] > 0 ? fit.max_active[1] : 148;
+  const int cmin = (R + MAX_T - 1) / MAX_T;
+  long best = -1;
+  for (int c = cmin; c <= cmin + 6 && c <= R; c++) {
+    const int rows = ceil8((R + c - 1) / c);               // chunk starts stay multiples of 8 rows
+    if (rows > MAX_T || (long)rows * (c - 1) >= R) continue;
+    for (int S = 1; S <= MAX_S; S++) {
+      const int fits = S == 1 ? fit1 : fit.max_active[S];
+      if (fits <= 0 || (S > 1 && KB / S < 4)) continue;
+      const long waves = ((long)tiles * c + fits - 1) / fits;
+      const long cost = waves * (FIXED_CLOCKS + 60L * rows / S + (long)((KB + S - 1) / S) * (512 + 6 * rows));
+      if (best < 0 || cost < best) {
+        best = cost;
+        p.chunks = c;
+        p.chunk_rows = rows;
+        p.S = S;
+      }
+    }
+  }
+  p.tn_chunk = p.chunk_rows;
+  p.tn_tail = ceil8(R - (p.chunks - 1) * p.chunk_rows);
+  return p;
+}
+
+// One launch over ea.T rows in chunks of ea.chunk_rows (grid y). tmX: the X map with box rows
+// ea.tn_chunk; tmXtail: the map for the last chunk (box rows ea.tn_tail).
 inline cudaError_t launch(const CUtensorMap &tmW, const CUtensorMap &tmX, const CUtensorMap &tmXtail,
                           const EpiArgs &ea, int tiles, int KB, int S, int *err, cudaStream_t st, bool pdl) {
-  switch (tn_of(ea.T)) {
+  // (launches of several chunks always take the 128-row instantiation: it alone reads the widths from ea)
+  switch (ea.T > MAX_T ? MAX_T : tn_of(ea.T)) {
     case 16: return launch_tn<16>(tmW, tmX, tmX, ea, tiles, KB, S, err, st, pdl);
     case 32: return launch_tn<32>(tmW, tmX, tmX, ea, tiles, KB, S, err, st, pdl);
     case 64: return launch_tn<64>(tmW, tmX, tmX, ea, tiles, KB, S, err, st, pdl);

@@ -194,8 +194,10 @@ enum EpiMode {
 struct EpiArgs {
   int mode;
   int row0;              // first row of this launch within the call's row range
-  int T;                 // rows of this launch; CTAs with blockIdx.y = c take rows [128 c, 128 c + 128)
-  int tn_tail;           // tn_of(rows of the last 128-row chunk): its X box and MMA width
+  int T;                 // rows of this launch; CTAs with blockIdx.y = c take rows [chunk_rows c, chunk_rows (c + 1))
+  int chunk_rows;        // rows per chunk (<= 128); launches of up to 128 rows are one chunk
+  int tn_chunk, tn_tail; // X box rows = half the MMA width (multiples of 8) of the 128-row instantiation: of
+                         // every chunk but the last, and of the last
   int N;                 // output columns (EPI_SWIGLU: F, the width of gate and of up)
   int up_off;            // EPI_SWIGLU: row of W where the up projection starts (F)
   unsigned long long wait_ns;   // limit of every mbarrier wait

@@ -32,15 +32,15 @@ struct WMat {
   const signed char *q8;  // quantised target: int8 codes in the same unit order (then packed is NULL)
   const float *scale;     // ... and the scale of every weight row
 };
-// A two-limb activation buffer [2][rows][K] and its TMA maps, one per row-tile size 16/32/64/128.
+// A two-limb activation buffer [2][rows][K] and its TMA maps, one per box height 8, 16, ..., 128 rows.
 struct XBuf {
   bf16 *p;
   size_t plane;
   int rows, K;
   bool has_map;
-  CUtensorMap map[4];
+  CUtensorMap map[16];
 };
-inline int tn_index(int TN) { return TN == 16 ? 0 : (TN == 32 ? 1 : (TN == 64 ? 2 : 3)); }
+inline int tn_index(int TN) { return TN / 8 - 1; }
 
 struct LayerW {
   WMat wqkv, wo, wgu, wd;
@@ -384,23 +384,25 @@ int gemm(specvla_ctx *ctx, const XBuf &A, const WMat &W, int R, gemm_tc::EpiArgs
   ea.eps = ctx->desc.rms_eps;
   const bool prof = (ctx->prof_mask & ctx->phase) && 2 * (ctx->prof_used + 1) <= (int)ctx->prof_ev.size();
   if (prof) CU(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_used], st));
-  const int chunks = (R + gemm_tc::MAX_T - 1) / gemm_tc::MAX_T;
-  const int S = gemm_ck::slices_for(tiles * chunks, KB, ctx->fit);
+  const gemm_ck::RowPlan plan = gemm_ck::plan_rows(R, tiles, KB, ctx->fit);
+  const int chunks = plan.chunks, S = plan.S;
   ea.row0 = 0;
   ea.T = R;
-  ea.tn_tail = gemm_tc::tn_of(R - (chunks - 1) * gemm_tc::MAX_T);
+  ea.chunk_rows = plan.chunk_rows;
+  ea.tn_chunk = plan.tn_chunk;
+  ea.tn_tail = plan.tn_tail;
   ea.pf_w = nullptr;
   if (next && (next->packed || next->q8) && ctx->use_l2_prefetch) {
     // start pulling the next matrix (up to L2_PREFETCH_BYTES of it)
     ea.pf_tiles = next_swiglu ? (next->N / 2 + 127) / 128 : (next->N + SV_TILE_ROWS - 1) / SV_TILE_ROWS;
     ea.pf_KB = (next->K + gemm_tc::BK - 1) / gemm_tc::BK;
-    ea.pf_S = gemm_ck::slices_for(ea.pf_tiles * chunks, ea.pf_KB, ctx->fit);
+    ea.pf_S = gemm_ck::plan_rows(R, ea.pf_tiles, ea.pf_KB, ctx->fit).S;
     ea.pf_unit_bytes = next->q8 ? gemm_tc::W_STAGE_BYTES / 2 : gemm_tc::W_STAGE_BYTES;
     const size_t per_cta = L2_PREFETCH_BYTES / ((size_t)ea.pf_tiles * ea.pf_S) / ea.pf_unit_bytes;
     ea.pf_units = per_cta < 1 ? 1 : (int)per_cta;
     ea.pf_w = next->q8 ? static_cast<const void *>(next->q8) : static_cast<const void *>(next->packed);
   }
-  CU(gemm_ck::launch(W.map, A.map[tn_index(gemm_tc::tn_of(R))], A.map[tn_index(ea.tn_tail)], ea, tiles, KB, S,
+  CU(gemm_ck::launch(W.map, A.map[tn_index(ea.tn_chunk)], A.map[tn_index(ea.tn_tail)], ea, tiles, KB, S,
                      ctx->err, st, ctx->use_pdl));
   ctx->launches++;
   if (prof) {
@@ -873,9 +875,8 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
   };
   auto xmaps = [&](XBuf &b) {
     b.has_map = true;
-    const int tns[4] = {16, 32, 64, 128};
-    for (int i = 0; i < 4 && b.has_map; i++)
-      b.has_map = gemm_tc::make_x_map(&b.map[i], b.p, b.plane, b.rows, b.K, tns[i]);
+    for (int i = 0; i < 16 && b.has_map; i++)
+      b.has_map = gemm_tc::make_x_map(&b.map[i], b.p, b.plane, b.rows, b.K, 8 * (i + 1));
   };
   xmaps(ctx->xn);
   xmaps(ctx->xin);
@@ -1797,11 +1798,8 @@ static int gemm_entry(const float *X, const void *W, const void *Wp, float *Y, i
   // the status word starts at zero
   if (cudaMemsetAsync(base, 0, GEMM_HDR, st) != cudaSuccess) return SPECVLA_ERR_CUDA;
   epi::split_limbs_kernel<<<(unsigned)((nx + 255) / 256), 256, 0, st>>>(X, nx, limbs);
-  CUtensorMap mw = {}, mx[4];
+  CUtensorMap mw = {}, mx[2];
   if (W && !gemm_tc::make_w_map(&mw, static_cast<const bf16 *>(W), N, K)) return SPECVLA_ERR_CUDA;
-  const int tns[4] = {16, 32, 64, 128};
-  for (int i = 0; i < 4; i++)
-    if (!gemm_tc::make_x_map(&mx[i], limbs, nx, T, K, tns[i])) return SPECVLA_ERR_CUDA;
   const int tiles = (N + SV_TILE_ROWS - 1) / SV_TILE_ROWS;
   const int KB = (K + gemm_tc::BK - 1) / gemm_tc::BK;
   gemm_tc::EpiArgs ea = {};
@@ -1815,13 +1813,16 @@ static int gemm_entry(const float *X, const void *W, const void *Wp, float *Y, i
   g_gemm_wait_ns = gemm_tc::WAIT_LIMIT_NS;           // the test hook holds for one call
   g_gemm_withhold = 0;
   const gemm_ck::ClusterFit fit = cluster_fit_of_current_device();
-  const int chunks = (T + gemm_tc::MAX_T - 1) / gemm_tc::MAX_T;
-  const int S = gemm_ck::slices_for(tiles * chunks, KB, fit);
+  const gemm_ck::RowPlan plan = gemm_ck::plan_rows(T, tiles, KB, fit);
   ea.row0 = 0;
   ea.T = T;
-  ea.tn_tail = gemm_tc::tn_of(T - (chunks - 1) * gemm_tc::MAX_T);
-  if (gemm_ck::launch(mw, mx[tn_index(gemm_tc::tn_of(T))], mx[tn_index(ea.tn_tail)], ea, tiles, KB, S, err, st,
-                      false) != cudaSuccess)
+  ea.chunk_rows = plan.chunk_rows;
+  ea.tn_chunk = plan.tn_chunk;
+  ea.tn_tail = plan.tn_tail;
+  if (!gemm_tc::make_x_map(&mx[0], limbs, nx, T, K, plan.tn_chunk) ||
+      !gemm_tc::make_x_map(&mx[1], limbs, nx, T, K, plan.tn_tail))
+    return SPECVLA_ERR_CUDA;
+  if (gemm_ck::launch(mw, mx[0], mx[1], ea, tiles, KB, plan.S, err, st, false) != cudaSuccess)
     return SPECVLA_ERR_CUDA;
   return cudaGetLastError() == cudaSuccess ? SPECVLA_OK : SPECVLA_ERR_CUDA;
 }
