@@ -113,6 +113,9 @@ tree_attention_kernel(const EpArgs ea, const Args a) {
   const int h = blockIdx.y, hd = a.H * DH;
   int bid = blockIdx.x / a.splits;
   const int sp = blockIdx.x - bid * a.splits;
+  // Unsliced launches (prefill: more row blocks than SMs) take the blocks last to first: causal rows
+  // make the late blocks of an episode the long ones, and those must not be left for the last wave.
+  if (a.splits == 1) bid = (int)gridDim.x - 1 - bid;
   int ei = 0;
   for (; ei < ea.n_ep; ei++) {
     const int nb = (ea.nrows[ei] + RB - 1) / RB;

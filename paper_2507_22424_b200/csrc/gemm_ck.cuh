@@ -179,6 +179,12 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 
   // finishing-loop operands that the epilogue warps fetch while the MMAs run (part 1)
   const bool rope_staged = MODE == EPI_QKV && T <= ROPE_ROWS && (ea.dh >> 1) <= ROPE_HALF;
+  // Long tiles (the 128-row instantiation): the RoPE factors of the CTA's rows are copied into the
+  // idle ring behind the partial tile while the accumulator is read out (asynchronous copies, no
+  // registers), so that the finishing loop has no global loads left.
+  const bool rope_ring = MODE == EPI_QKV && TN == MAX_T && !Q8 && !rope_staged && n_units > 0 && (ea.dh >> 1) <= 64 &&
+                         tn * BM * 4 + T * (ea.dh >> 1) * 8 <= STAGES * STAGE;
+  const uint32_t rope_off = (uint32_t)(tn * BM * 4);
   float4 xpre0 = make_float4(0.f, 0.f, 0.f, 0.f), xpre1 = xpre0;
 
   if (warp == 0) {
@@ -334,6 +340,15 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       have = s_flag[0] && s_flag[1] && s_flag[2] && s_flag[3] && s_flag[4] && s_flag[5] && s_flag[6] && s_flag[7];
       if (!have && et == 0) atomicExch(err, SV_ERR_WAIT_TMEM_FULL);
       tc_fence_after();
+      if (rope_ring) {
+        const int hp = ea.dh >> 2;                         // 16-byte pieces (two pairs) per row
+        for (int i = et; i < T * hp; i += 256) {
+          const int t = i / hp, j2 = i - t * hp;
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(base + rope_off + (uint32_t)(i * 16)),
+                       "l"(ea.rope_tab + (size_t)s_pos[t] * (ea.dh >> 1) + 2 * j2) : "memory");
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+      }
     }
     const uint32_t tadr = tmem_base + ((uint32_t)(q * 32) << 16);
     const int col = q * 32 + lane;                       // column within a 128-column half
@@ -361,6 +376,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
           }
       }
     }
+    if (rope_ring) asm volatile("cp.async.wait_group 0;" ::: "memory");
     tc_fence_before();
   }
 
@@ -405,6 +421,8 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     const int half = ea.dh >> 1, jq = MODE == EPI_QKV ? cq % ea.dh : 0;
     const bool lo = jq < half, rot = MODE == EPI_QKV && which < 2;
     auto partial_sum = [&](int off) {
+      // (the shortcut of the unsplit case only in long tiles: it measured slower in the short ones)
+      if (TN == MAX_T && S == 1) return *reinterpret_cast<const float4 *>(P_own + off);
       float4 p[MAX_S];
 #pragma unroll
       for (int sl = 0; sl < MAX_S; sl++)
@@ -436,29 +454,20 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     auto scaled = [](float4 v, const float4 &w) { return make_float4(v.x * w.x, v.y * w.y, v.z * w.z, v.w * w.w); };
     // The rows are taken U at a time: first every global operand of the U rows, then their partial
     // sums, then the arithmetic and the stores, so that a long tile (prefill: up to 32 rows per
-    // thread) pays the load latencies once per batch instead of once per row.
+    // thread) pays the load latencies once per batch instead of once per row. Short tiles (a
+    // verification step: two or three rows per thread) keep one row at a time: batching them
+    // measured 2 % slower per step, the first stores leaving later.
     constexpr int U = TN == MAX_T ? 4 : 1;
     const int tstep = RG * S;
     for (int tb = rank + rg * S, iter0 = 0; tb < T; tb += U * tstep, iter0 += U) {
-      float4 xo_[U], cs01_[U], cs23_[U], v_[U], w_[U];
+      float4 xo_[U], v_[U], w_[U];
 #pragma unroll
       for (int u = 0; u < U; u++) {
         const int t = tb + u * tstep, iter = iter0 + u;
+        // the residuals of the first two rows were fetched in part 1
         xo_[u] = iter == 0 ? xpre0 : xpre1;
-        cs01_[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-        cs23_[u] = cs01_[u];
-        if (t < T) {
-          // global operands first (the first two rows' residuals and, up to 32 rows, the RoPE
-          // factors were fetched in part 1)
-          if (MODE == EPI_RESID && ea.accumulate && col_ok && iter >= 2)
-            xo_[u] = *reinterpret_cast<const float4 *>(ea.x + (size_t)(row0 + t) * ea.N + n);
-          if (rot) {
-            const float2 *cs = rope_staged ? s_rope + t * ROPE_HALF + (lo ? jq : jq - half)
-                                           : ea.rope_tab + (size_t)s_pos[t] * half + (lo ? jq : jq - half);
-            cs01_[u] = *reinterpret_cast<const float4 *>(cs);
-            cs23_[u] = *reinterpret_cast<const float4 *>(cs + 2);
-          }
-        }
+        if (MODE == EPI_RESID && ea.accumulate && col_ok && iter >= 2 && t < T)
+          xo_[u] = *reinterpret_cast<const float4 *>(ea.x + (size_t)(row0 + t) * ea.N + n);
       }
 #pragma unroll
       for (int u = 0; u < U; u++) {
@@ -474,134 +483,145 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
       }
 #pragma unroll
       for (int u = 0; u < U; u++) {
-      const int t = tb + u * tstep;
-      if (t >= T) break;
-      const size_t row = (size_t)(row0 + t);
-      const float sc = s_scale[t];
-      const float4 xo = xo_[u], cs01 = cs01_[u], cs23 = cs23_[u];
-      const int slot = MODE == EPI_QKV ? s_slot[t] : 0, ep = MODE == EPI_QKV ? s_ep[t] : 0;
-      float4 v = v_[u];
-      if (Q8) v = scaled(v, ws);
-      if (MODE == EPI_PLAIN) {
-        const float4 ov = make_float4(sc * v.x, sc * v.y, sc * v.z, sc * v.w);
-        if (ea.out && col_ok) *reinterpret_cast<float4 *>(ea.out + row * ea.ldo + n) = ov;
-        if (ea.cand) {
-          // greedy argmax, first step: the top-2 of this warp's 128 columns over [lo, hi)
-          sv::Top2 b{-INFINITY, -INFINITY, 0x7fffffff};
-          const float vv[4] = {ov.x, ov.y, ov.z, ov.w};
-#pragma unroll
-          for (int e = 0; e < 4; e++)
-            if (n + e >= ea.lo && n + e < ea.hi && n + e < ea.N) sv::top2_push(b, vv[e], n + e);
-          sv::top2_warp(b);
-          if (lane == 0)
-            ea.cand[row * (size_t)(2 * tiles) + tile * 2 + ((et >> 5) & 1)] = make_float4(b.v1, __int_as_float(b.i1), b.v2, 0.f);
-        }
-      } else if (MODE == EPI_TOPK) {
-        // the row's 256 scores sit in the two warps of this row group, four per thread
-        const int wg = (et >> 5) & 1;
-        const float xv[4] = {sc * v.x, sc * v.y, sc * v.z, sc * v.w};
-        bool in[4];
-#pragma unroll
-        for (int e = 0; e < 4; e++) in[e] = n + e >= ea.lo && n + e < ea.hi && n + e < ea.N;
-        if (ea.out && col_ok) *reinterpret_cast<float4 *>(ea.out + row * ea.ldo + n) = make_float4(xv[0], xv[1], xv[2], xv[3]);
-        auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(2 + rg) : "memory"); };
-        float mx = -INFINITY;
-#pragma unroll
-        for (int e = 0; e < 4; e++)
-          if (in[e]) mx = fmaxf(mx, xv[e]);
-        mx = warp_max(mx);
-        if (lane == 0) s_xv[rg][wg] = mx;
-        pair_sync();
-        mx = fmaxf(s_xv[rg][0], s_xv[rg][1]);
-        pair_sync();
-        float se = 0.f;
-#pragma unroll
-        for (int e = 0; e < 4; e++)
-          if (in[e]) se += expf(xv[e] - mx);
-        se = warp_sum(se);
-        if (lane == 0) s_xv[rg][wg] = se;
-        pair_sync();
-        const float lse = mx + logf(s_xv[rg][0] + s_xv[rg][1]);
-        pair_sync();
-        unsigned taken = 0;
-        for (int k = 0; k < SV_TOPK; k++) {
-          float bv = -INFINITY;
-          int bi = 0x7fffffff;
-#pragma unroll
-          for (int e = 0; e < 4; e++)
-            if (in[e] && !((taken >> e) & 1u) && (xv[e] > bv || (xv[e] == bv && n + e < bi))) {
-              bv = xv[e];
-              bi = n + e;
-            }
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) {
-            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-            if (ov > bv || (ov == bv && oi < bi)) {
-              bv = ov;
-              bi = oi;
-            }
-          }
-          if (lane == 0) {
-            s_xv[rg][wg] = bv;
-            s_xi[rg][wg] = bi;
-          }
-          pair_sync();
-          const float v0 = s_xv[rg][0], v1 = s_xv[rg][1];
-          const int i0 = s_xi[rg][0], i1 = s_xi[rg][1];
-          const bool first = v0 > v1 || (v0 == v1 && i0 < i1);
-          bv = first ? v0 : v1;
-          bi = first ? i0 : i1;
-          pair_sync();
-          if (bi >= n && bi < n + 4) taken |= 1u << (bi - n);
-          if ((et & 63) == 0) {
-            ea.top_tok[row * SV_TOPK + k] = bi + ea.tok_offset;
-            ea.top_lp[row * SV_TOPK + k] = bv - lse;
-          }
-        }
-      } else if (MODE == EPI_QKV) {
-        float4 o = make_float4(sc * v.x, sc * v.y, sc * v.z, sc * v.w);
+        const int t = tb + u * tstep;
+        if (t >= T) break;
+        const size_t row = (size_t)(row0 + t);
+        const float sc = s_scale[t];
+        const float4 xo = xo_[u];
+        float4 cs01 = make_float4(0.f, 0.f, 0.f, 0.f), cs23 = cs01;
         if (rot) {
-          float4 w = w_[u];
-          if (Q8) w = scaled(w, ws2);
-          const float sg = lo ? -sc : sc;
-          o.x = o.x * cs01.x + sg * w.x * cs01.y;
-          o.y = o.y * cs01.z + sg * w.y * cs01.w;
-          o.z = o.z * cs23.x + sg * w.z * cs23.y;
-          o.w = o.w * cs23.z + sg * w.w * cs23.w;
+          // RoPE factors: staged in shared memory (short tiles: part 1; long tiles: the idle ring); the
+          // global table is the fallback of the instantiations that have no room for them
+          const int jh = lo ? jq : jq - half;
+          const float2 *cs = rope_staged ? s_rope + t * ROPE_HALF + jh
+                             : rope_ring ? reinterpret_cast<const float2 *>(P_own + (rope_off >> 2)) + t * half + jh
+                                         : ea.rope_tab + (size_t)s_pos[t] * half + jh;
+          cs01 = *reinterpret_cast<const float4 *>(cs);
+          cs23 = *reinterpret_cast<const float4 *>(cs + 2);
         }
-        if (col_ok) {
-          float *dst = which == 0 ? ea.q + row * ea.hd + cq
-                                  : ea.cache + (size_t)ep * ea.ep_stride +
-                                        ((size_t)(which - 1) * ea.max_seq + slot) * ea.hd + cq;
-          *reinterpret_cast<float4 *>(dst) = o;
+        const int slot = MODE == EPI_QKV ? s_slot[t] : 0, ep = MODE == EPI_QKV ? s_ep[t] : 0;
+        float4 v = v_[u];
+        if (Q8) v = scaled(v, ws);
+        if (MODE == EPI_PLAIN) {
+          const float4 ov = make_float4(sc * v.x, sc * v.y, sc * v.z, sc * v.w);
+          if (ea.out && col_ok) *reinterpret_cast<float4 *>(ea.out + row * ea.ldo + n) = ov;
+          if (ea.cand) {
+            // greedy argmax, first step: the top-2 of this warp's 128 columns over [lo, hi)
+            sv::Top2 b{-INFINITY, -INFINITY, 0x7fffffff};
+            const float vv[4] = {ov.x, ov.y, ov.z, ov.w};
+  #pragma unroll
+            for (int e = 0; e < 4; e++)
+              if (n + e >= ea.lo && n + e < ea.hi && n + e < ea.N) sv::top2_push(b, vv[e], n + e);
+            sv::top2_warp(b);
+            if (lane == 0)
+              ea.cand[row * (size_t)(2 * tiles) + tile * 2 + ((et >> 5) & 1)] = make_float4(b.v1, __int_as_float(b.i1), b.v2, 0.f);
+          }
+        } else if (MODE == EPI_TOPK) {
+          // the row's 256 scores sit in the two warps of this row group, four per thread
+          const int wg = (et >> 5) & 1;
+          const float xv[4] = {sc * v.x, sc * v.y, sc * v.z, sc * v.w};
+          bool in[4];
+  #pragma unroll
+          for (int e = 0; e < 4; e++) in[e] = n + e >= ea.lo && n + e < ea.hi && n + e < ea.N;
+          if (ea.out && col_ok) *reinterpret_cast<float4 *>(ea.out + row * ea.ldo + n) = make_float4(xv[0], xv[1], xv[2], xv[3]);
+          auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(2 + rg) : "memory"); };
+          float mx = -INFINITY;
+  #pragma unroll
+          for (int e = 0; e < 4; e++)
+            if (in[e]) mx = fmaxf(mx, xv[e]);
+          mx = warp_max(mx);
+          if (lane == 0) s_xv[rg][wg] = mx;
+          pair_sync();
+          mx = fmaxf(s_xv[rg][0], s_xv[rg][1]);
+          pair_sync();
+          float se = 0.f;
+  #pragma unroll
+          for (int e = 0; e < 4; e++)
+            if (in[e]) se += expf(xv[e] - mx);
+          se = warp_sum(se);
+          if (lane == 0) s_xv[rg][wg] = se;
+          pair_sync();
+          const float lse = mx + logf(s_xv[rg][0] + s_xv[rg][1]);
+          pair_sync();
+          unsigned taken = 0;
+          for (int k = 0; k < SV_TOPK; k++) {
+            float bv = -INFINITY;
+            int bi = 0x7fffffff;
+  #pragma unroll
+            for (int e = 0; e < 4; e++)
+              if (in[e] && !((taken >> e) & 1u) && (xv[e] > bv || (xv[e] == bv && n + e < bi))) {
+                bv = xv[e];
+                bi = n + e;
+              }
+  #pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+              const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+              const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+              if (ov > bv || (ov == bv && oi < bi)) {
+                bv = ov;
+                bi = oi;
+              }
+            }
+            if (lane == 0) {
+              s_xv[rg][wg] = bv;
+              s_xi[rg][wg] = bi;
+            }
+            pair_sync();
+            const float v0 = s_xv[rg][0], v1 = s_xv[rg][1];
+            const int i0 = s_xi[rg][0], i1 = s_xi[rg][1];
+            const bool first = v0 > v1 || (v0 == v1 && i0 < i1);
+            bv = first ? v0 : v1;
+            bi = first ? i0 : i1;
+            pair_sync();
+            if (bi >= n && bi < n + 4) taken |= 1u << (bi - n);
+            if ((et & 63) == 0) {
+              ea.top_tok[row * SV_TOPK + k] = bi + ea.tok_offset;
+              ea.top_lp[row * SV_TOPK + k] = bv - lse;
+            }
+          }
+        } else if (MODE == EPI_QKV) {
+          float4 o = make_float4(sc * v.x, sc * v.y, sc * v.z, sc * v.w);
+          if (rot) {
+            float4 w = w_[u];
+            if (Q8) w = scaled(w, ws2);
+            const float sg = lo ? -sc : sc;
+            o.x = o.x * cs01.x + sg * w.x * cs01.y;
+            o.y = o.y * cs01.z + sg * w.y * cs01.w;
+            o.z = o.z * cs23.x + sg * w.z * cs23.y;
+            o.w = o.w * cs23.z + sg * w.w * cs23.w;
+          }
+          if (col_ok) {
+            float *dst = which == 0 ? ea.q + row * ea.hd + cq
+                                    : ea.cache + (size_t)ep * ea.ep_stride +
+                                          ((size_t)(which - 1) * ea.max_seq + slot) * ea.hd + cq;
+            *reinterpret_cast<float4 *>(dst) = o;
+          }
+        } else if (swiglu) {
+          float4 up = w_[u];
+          if (Q8) up = scaled(up, ws2);
+          if (col_ok) {
+            const float gx = sc * v.x, gy = sc * v.y, gz = sc * v.z, gw = sc * v.w;
+            store_limbs4(ea.hid, ea.hid_plane, row * ea.N + n,
+                         make_float4(__fdividef(gx, 1.f + __expf(-gx)) * (sc * up.x),
+                                     __fdividef(gy, 1.f + __expf(-gy)) * (sc * up.y),
+                                     __fdividef(gz, 1.f + __expf(-gz)) * (sc * up.z),
+                                     __fdividef(gw, 1.f + __expf(-gw)) * (sc * up.w)));
+          }
+        } else {
+          float s2 = 0.f;
+          if (col_ok) {
+            v.x += xo.x;
+            v.y += xo.y;
+            v.z += xo.z;
+            v.w += xo.w;
+            *reinterpret_cast<float4 *>(ea.x + row * ea.N + n) = v;
+            store_limbs4(ea.xn, ea.xn_plane, row * ea.N + n,
+                         make_float4(v.x * gain.x, v.y * gain.y, v.z * gain.z, v.w * gain.w));
+            s2 = (v.x * v.x + v.y * v.y) + (v.z * v.z + v.w * v.w);
+          }
+          s2 = warp_sum(s2);
+          if (lane == 0) s_red[warp - 2][t] = s2;
         }
-      } else if (swiglu) {
-        float4 up = w_[u];
-        if (Q8) up = scaled(up, ws2);
-        if (col_ok) {
-          const float gx = sc * v.x, gy = sc * v.y, gz = sc * v.z, gw = sc * v.w;
-          store_limbs4(ea.hid, ea.hid_plane, row * ea.N + n,
-                       make_float4(__fdividef(gx, 1.f + __expf(-gx)) * (sc * up.x),
-                                   __fdividef(gy, 1.f + __expf(-gy)) * (sc * up.y),
-                                   __fdividef(gz, 1.f + __expf(-gz)) * (sc * up.z),
-                                   __fdividef(gw, 1.f + __expf(-gw)) * (sc * up.w)));
-        }
-      } else {
-        float s2 = 0.f;
-        if (col_ok) {
-          v.x += xo.x;
-          v.y += xo.y;
-          v.z += xo.z;
-          v.w += xo.w;
-          *reinterpret_cast<float4 *>(ea.x + row * ea.N + n) = v;
-          store_limbs4(ea.xn, ea.xn_plane, row * ea.N + n,
-                       make_float4(v.x * gain.x, v.y * gain.y, v.z * gain.z, v.w * gain.w));
-          s2 = (v.x * v.x + v.y * v.y) + (v.z * v.z + v.w * v.w);
-        }
-        s2 = warp_sum(s2);
-        if (lane == 0) s_red[warp - 2][t] = s2;
-      }
       }
     }
   }
