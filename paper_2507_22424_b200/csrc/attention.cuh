@@ -80,7 +80,12 @@ __device__ __forceinline__ void split4(const float4 v, uint2 &hi, uint2 &lo) {
   lo = make_uint2(*reinterpret_cast<const uint32_t *>(&l01), *reinterpret_cast<const uint32_t *>(&l23));
 }
 
-template <int DH>
+// SLICED: grid (row blocks x key slices, heads), cluster (slices, 1, 1): the few-row launches (a
+// verification step, a draft level). Unsliced (prefill: more CTAs than SMs): grid (heads, row
+// blocks), the blocks taken last to first: causal rows make the late blocks of an episode the long
+// ones, and CTAs are handed out x first, so every head's longest block starts before any short one
+// and the last wave is made of short blocks.
+template <int DH, bool SLICED>
 __global__ void __launch_bounds__(THREADS, 1)
 tree_attention_kernel(const EpArgs ea, const Args a) {
   constexpr int PER = DH / 32;            // head-dim columns per lane in the slice merge
@@ -110,12 +115,10 @@ tree_attention_kernel(const EpArgs ea, const Args a) {
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int mb = warp & 1, wq = warp >> 1;         // 16-row block; key octet (scores) / head-dim quarter (sum)
-  const int h = blockIdx.y, hd = a.H * DH;
-  int bid = blockIdx.x / a.splits;
-  const int sp = blockIdx.x - bid * a.splits;
-  // Unsliced launches (prefill: more row blocks than SMs) take the blocks last to first: causal rows
-  // make the late blocks of an episode the long ones, and those must not be left for the last wave.
-  if (a.splits == 1) bid = (int)gridDim.x - 1 - bid;
+  const int h = SLICED ? blockIdx.y : blockIdx.x, hd = a.H * DH;
+  const int splits = SLICED ? a.splits : 1;
+  int bid = SLICED ? (int)blockIdx.x / splits : (int)gridDim.y - 1 - (int)blockIdx.y;
+  const int sp = SLICED ? (int)blockIdx.x - bid * splits : 0;
   int ei = 0;
   for (; ei < ea.n_ep; ei++) {
     const int nb = (ea.nrows[ei] + RB - 1) / RB;
@@ -164,7 +167,7 @@ tree_attention_kernel(const EpArgs ea, const Args a) {
   __syncthreads();
   const int kmax = s_kmax;
   const int tiles = (kmax + KT - 1) / KT;
-  const int t0 = sp * tiles / a.splits, t1 = (sp + 1) * tiles / a.splits;
+  const int t0 = sp * tiles / splits, t1 = (sp + 1) * tiles / splits;
 
   float4 kreg[NLD], vreg[NLD];
   auto fetch = [&](int t) {
@@ -339,7 +342,7 @@ tree_attention_kernel(const EpArgs ea, const Args a) {
   __syncthreads();
   const int ra = 16 * mb + (lane >> 2), rb = ra + 8;        // this thread's two rows
   const int cbase = (DH / 4) * wq + 2 * (lane & 3);          // + 8 nb: its column pairs
-  if (a.splits == 1) {
+  if (splits == 1) {
     const float ia = 1.f / s_l[ra], ib = 1.f / s_l[rb];
 #pragma unroll
     for (int nb = 0; nb < NB; nb++) {
@@ -375,12 +378,12 @@ tree_attention_kernel(const EpArgs ea, const Args a) {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
   cooperative_groups::cluster_group cluster = cooperative_groups::this_cluster();
-  for (int r = sp + a.splits * warp; r < nrows; r += a.splits * (THREADS / 32)) {
+  for (int r = sp + splits * warp; r < nrows; r += splits * (THREADS / 32)) {
     // every load of the row's slices is issued before any is used: one latency, not one per slice
     float ms[MAX_SPLITS], ls[MAX_SPLITS], os[MAX_SPLITS][PER];
 #pragma unroll
     for (int s2 = 0; s2 < MAX_SPLITS; s2++) {
-      if (s2 < a.splits) {
+      if (s2 < splits) {
         const float *src = cluster.map_shared_rank(sO, (unsigned)s2) + r * LO;
         ms[s2] = src[DH];
         ls[s2] = src[DH + 1];
@@ -396,13 +399,13 @@ tree_attention_kernel(const EpArgs ea, const Args a) {
     float M = -INFINITY;
 #pragma unroll
     for (int s2 = 0; s2 < MAX_SPLITS; s2++)
-      if (s2 < a.splits) M = fmaxf(M, ms[s2]);
+      if (s2 < splits) M = fmaxf(M, ms[s2]);
     float L = 0.f, o[PER];
 #pragma unroll
     for (int k = 0; k < PER; k++) o[k] = 0.f;
 #pragma unroll
     for (int s2 = 0; s2 < MAX_SPLITS; s2++)
-      if (s2 < a.splits) {
+      if (s2 < splits) {
         const float c = (ms[s2] == -INFINITY) ? 0.f : __expf(ms[s2] - M);
         L += ls[s2] * c;
 #pragma unroll

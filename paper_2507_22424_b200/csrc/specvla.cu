@@ -473,7 +473,8 @@ int attention(specvla_ctx *ctx, const EpArgs &rows, const float *cache, size_t e
     if (a.splits < 1) a.splits = 1;
   }
   // the key slices of a row block are one cluster (they merge through distributed shared memory)
-  const dim3 grid(blocks * a.splits, d.n_heads);
+  // (unsliced: heads on x, see the kernel)
+  const dim3 grid = a.splits == 1 ? dim3(d.n_heads, blocks) : dim3(blocks * a.splits, d.n_heads);
   cudaLaunchAttribute at[2];
   cudaLaunchConfig_t cfg = launch_cfg(grid, dim3(attn::THREADS), st, &at[0], ctx->use_pdl);
   at[cfg.numAttrs].id = cudaLaunchAttributeClusterDimension;
@@ -481,12 +482,15 @@ int attention(specvla_ctx *ctx, const EpArgs &rows, const float *cache, size_t e
   at[cfg.numAttrs].val.clusterDim.y = 1;
   at[cfg.numAttrs].val.clusterDim.z = 1;
   cfg.numAttrs++;
+  const bool sliced = a.splits > 1;
   if (d.head_dim == 128) {
     cfg.dynamicSmemBytes = attn::smem_bytes<128>();
-    CU(cudaLaunchKernelEx(&cfg, attn::tree_attention_kernel<128>, rows, a));
+    CU(sliced ? cudaLaunchKernelEx(&cfg, attn::tree_attention_kernel<128, true>, rows, a)
+              : cudaLaunchKernelEx(&cfg, attn::tree_attention_kernel<128, false>, rows, a));
   } else {
     cfg.dynamicSmemBytes = attn::smem_bytes<64>();
-    CU(cudaLaunchKernelEx(&cfg, attn::tree_attention_kernel<64>, rows, a));
+    CU(sliced ? cudaLaunchKernelEx(&cfg, attn::tree_attention_kernel<64, true>, rows, a)
+              : cudaLaunchKernelEx(&cfg, attn::tree_attention_kernel<64, false>, rows, a));
   }
   ctx->launches++;
   return SPECVLA_OK;
@@ -945,9 +949,13 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
   cudaMemsetAsync(ctx->st, 0, sizeof(EpState) * desc->max_episodes);
   cudaMemsetAsync(ctx->trees, 0, sizeof(DevTree) * desc->max_episodes);
   cudaMemsetAsync(ctx->err, 0, 32 * sizeof(int));
-  cudaFuncSetAttribute(attn::tree_attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaFuncSetAttribute(attn::tree_attention_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                        attn::smem_bytes<128>());
-  cudaFuncSetAttribute(attn::tree_attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaFuncSetAttribute(attn::tree_attention_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                       attn::smem_bytes<128>());
+  cudaFuncSetAttribute(attn::tree_attention_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                       attn::smem_bytes<64>());
+  cudaFuncSetAttribute(attn::tree_attention_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                        attn::smem_bytes<64>());
   if (cudaDeviceSynchronize() != cudaSuccess || !pack_ok) {
     cudaFreeHost(ctx->pinned);
