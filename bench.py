@@ -33,7 +33,7 @@ WEIGHT_BYTES_PER_VERIFY = 13_214_679_040      # 32 layers + LM head, bf16, read 
 
 # DRAM traffic of one gate/up launch at T = 27 from the ncu capture under profiles/ (bytes); to be
 # re-taken (or set to None) whenever gemm_ck.cuh changes.
-GATE_UP_DRAM_BYTES = 203_322_624 + 3_482_880
+GATE_UP_DRAM_BYTES = 203_324_416 + 3_255_296
 GATE_UP_DRAM_SOURCE = ("ncu dram__bytes_read.sum + dram__bytes_write.sum of this launch at full size "
                        "(profiles/gemm_ck_verify_T27_ncu_full.md); the ~23 MB above the weights are the operand "
                        "and the L2 prefetch of the next GEMM's weights")
@@ -367,6 +367,9 @@ def run_ours(args, rank, local_rank, world):
     gpu = SpecVLA(desc, weights, max_seq=512, max_episodes=1, max_rows=512, action_only=True)
     shape = make_shape(wl.tree.branch, wl.tree.expand)
     r, n_tok = 0, wl.n_tokens
+    if args.host_loop:
+        from paper_2507_22424_b200.binding import OPT_DEVICE_LOOP as _OPT_LOOP
+        gpu.set_option(_OPT_LOOP, 0)
 
     def chunk():
         return gpu.generate_action([0], embeds, ids_host, [P], shape, r, n_tok)
@@ -436,7 +439,7 @@ def run_ours(args, rank, local_rank, world):
     h1.record()
     barrier()
     ms_host = h0.elapsed_time(h1)
-    gpu.set_option(OPT_DEVICE_LOOP, 1)
+    gpu.set_option(OPT_DEVICE_LOOP, 0 if args.host_loop else 1)
     # --- AR baseline from the same kernels (depth-0 tree) --------------------------------
     ar_shape = make_shape((), ())
     gpu.generate_action([0], embeds, ids_host, [P], ar_shape, 0, n_tok)
@@ -603,7 +606,7 @@ def run_ours(args, rank, local_rank, world):
                                                                     for k in range(n_tok - 1)],
                                 note="Table 3's statistic on C1: accepted draft tokens by the position at which "
                                      "an iteration starts (random draft head: zero)"),
-        chunk_loop=dict(on_device=bool(device_loop == args.steps), ms_prefill=ms_prefill / args.steps,
+        chunk_loop=dict(on_device=bool(device_loop == args.steps), forced_to_host=bool(args.host_loop), ms_prefill=ms_prefill / args.steps,
                         ms_iterations=ms_loop / args.steps,
                         note="`value` and `e2e`: Algorithm 1's iterations as one launch of a CUDA graph (while node "
                              "around draft tree, verification, token append), one read-back per chunk"),
@@ -791,6 +794,9 @@ def main():
     ap.add_argument("--skip-reports", action="store_true",
                     help="leave out the extra reports (C2/C3/C4 sweeps, int8 target, oracle timing): the timed "
                          "regions only, e.g. for a profiler's launch list")
+    ap.add_argument("--host-loop", action="store_true",
+                    help="run Algorithm 1's loop on the host in every timed region (one launch per kernel instead "
+                         "of one graph launch per chunk): for a profiler's launch list")
     ap.add_argument("--micro", default=None, help="gemm:T:N:K[:M], verify:L[:T] or batch[:E] - small cases for kernel timing / ncu (see run_micro)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
