@@ -28,7 +28,9 @@ if ROOT not in sys.path:
 
 METRIC = "action chunks/sec at bs1 (7B)"
 UNIT = "chunks/s"
-WEIGHT_BYTES_PER_VERIFY = 13_214_679_040      # 32 layers + LM head, bf16, read once
+WEIGHT_BYTES_FULL_HEAD = 13_214_679_040       # 32 layers + the whole LM head, bf16, read once
+# greedy decoding over the 256 action ids reads only their rows of the LM head (2 MB instead of 263 MB)
+WEIGHT_BYTES_PER_VERIFY = 32 * 404_750_336 + 256 * 4096 * 2
 
 
 # DRAM traffic of one gate/up launch at T = 27 from the ncu capture under profiles/ (bytes); to be
@@ -344,7 +346,7 @@ def int8_target(weights, desc, embeds, ids_host, P, shape, r, n_tok, steps=5):
         iters += st.iterations
     gpu.close()
     return dict(value=steps / (ms * 1e-3), unit=UNIT, verify_ms_per_step=ms_v / max(1, iters),
-                weight_bytes_per_step=WEIGHT_BYTES_PER_VERIFY // 2, lossless_vs_own_ar=bool(toks == ar), tokens=toks[0],
+                weight_bytes_per_step=WEIGHT_BYTES_FULL_HEAD // 2, lossless_vs_own_ar=bool(toks == ar), tokens=toks[0],
                 note="int8 codes are streamed at half the bytes but expanded to bf16 inside the SM before the "
                      "tensor cores read them; that expansion, not HBM, bounds this path")
 

@@ -126,9 +126,10 @@ using sv::top2_warp;
 
 // Greedy token per row from the candidates a GEMM epilogue left: cand[row][0..nc) holds the top-2
 // of each 128-column group of the row's logits (value, column as int bits, second value). One
-// warp per row; ties go to the lowest id; margin = top-1 minus top-2.
+// warp per row; ties go to the lowest id; margin = top-1 minus top-2. Column c is token tok_offset + c
+// (the GEMM may have covered only a slice of the vocabulary).
 __global__ void __launch_bounds__(128)
-argmax_merge_kernel(const float4 *__restrict__ cand, int nc, int rows, int *__restrict__ greedy,
+argmax_merge_kernel(const float4 *__restrict__ cand, int nc, int rows, int tok_offset, int *__restrict__ greedy,
                     float *__restrict__ margin) {
   pdl_launch();
   pdl_wait();
@@ -142,7 +143,7 @@ argmax_merge_kernel(const float4 *__restrict__ cand, int nc, int rows, int *__re
   }
   top2_warp(best);
   if (lane == 0) {
-    greedy[t] = best.i1;
+    greedy[t] = best.i1 + tok_offset;
     margin[t] = best.v1 - best.v2;
   }
 }

@@ -537,6 +537,10 @@ int run_layer(specvla_ctx *ctx, const LayerW &w, int R, const EpArgs &rows, floa
 // Target model over the R rows described by ctx->rt: embedding, all layers. Leaves the residual
 // in ctx->x, limbs(x * final-norm gain) in ctx->xn and the sums of squares in ctx->ssq: the
 // final RMSNorm itself is applied by whoever consumes them (LM head epilogue, feature readers).
+// The head matrix the greedy decoding after a target forward reads (see lm_head_greedy).
+const WMat *head_after_forward(const specvla_ctx *ctx) {
+  return (ctx->desc.action_only && ctx->has_draft && !ctx->lm_head.q8) ? &ctx->lm_head_act : &ctx->lm_head;
+}
 int target_forward(specvla_ctx *ctx, int R, const EpArgs &rows, const bf16 *embeds, cudaStream_t st) {
   const specvla_model_desc &d = ctx->desc;
   LAUNCH(epi::embed_kernel, dim3(R), dim3(epi::THREADS), ctx->rt, embeds, ctx->embed, ctx->layers[0].norm1,
@@ -545,7 +549,7 @@ int target_forward(specvla_ctx *ctx, int R, const EpArgs &rows, const bf16 *embe
     const bool last = (l + 1 == d.n_layers);
     TRY(run_layer(ctx, ctx->layers[l], R, rows, ctx->kv_t + (size_t)l * ctx->kv_t_layer_stride,
                   ctx->kv_t_ep_stride, last ? ctx->final_norm : ctx->layers[l + 1].norm1,
-                  last ? &ctx->lm_head : &ctx->layers[l + 1].wqkv, st));
+                  last ? head_after_forward(ctx) : &ctx->layers[l + 1].wqkv, st));
   }
   ctx->last_rows = R;
   ctx->last_ssq = ctx->ssq;
@@ -576,12 +580,24 @@ void argmax_range(const specvla_ctx *ctx, int *lo, int *hi);
 // themselves are written only when logits_out is given (parity tests).
 int lm_head_greedy(specvla_ctx *ctx, const XBuf &A, const float *ssq, int rows, float *logits_out, cudaStream_t st) {
   if (rows > ctx->max_lm_rows) return SPECVLA_ERR_CAPACITY;
-  gemm_tc::EpiArgs e = epi_plain(logits_out, ctx->desc.vocab, ctx->desc.vocab, ssq, ctx->nt);
+  const specvla_model_desc &d = ctx->desc;
+  // Greedy decoding over the action ids alone needs only their rows of the LM head (the copy the
+  // draft scoring uses: one or a few tiles instead of the whole vocabulary), unless the caller
+  // wants the logits themselves.
+  const bool act_rows = d.action_only && !logits_out && ctx->has_draft && !ctx->lm_head.q8;
+  const WMat &W = act_rows ? ctx->lm_head_act : ctx->lm_head;
+  gemm_tc::EpiArgs e = epi_plain(logits_out, d.vocab, W.N, ssq, ctx->nt);
   e.cand = ctx->cand;
-  argmax_range(ctx, &e.lo, &e.hi);
-  TRY(gemm(ctx, A, ctx->lm_head, rows, e, st, SPECVLA_PROF_LM_HEAD));
-  LAUNCH(epi::argmax_merge_kernel, dim3((rows + 3) / 4), dim3(128), (const float4 *)ctx->cand, ctx->cand_nc, rows,
-         ctx->greedy, ctx->margin);
+  if (act_rows) {
+    e.lo = 0;
+    e.hi = d.n_bins;
+  } else {
+    argmax_range(ctx, &e.lo, &e.hi);
+  }
+  TRY(gemm(ctx, A, W, rows, e, st, SPECVLA_PROF_LM_HEAD));
+  const int nc = 2 * ((W.N + SV_TILE_ROWS - 1) / SV_TILE_ROWS);
+  LAUNCH(epi::argmax_merge_kernel, dim3((rows + 3) / 4), dim3(128), (const float4 *)ctx->cand, nc, rows,
+         act_rows ? d.action_base : 0, ctx->greedy, ctx->margin);
   return SPECVLA_OK;
 }
 
