@@ -20,6 +20,11 @@
  *    repacked copy of every weight matrix, about the size of the weights themselves) is one
  *    device buffer allocated by the caller, at least specvla_workspace_bytes() long, 1024-byte aligned;
  *    it must outlive the context and must not be touched while a call is in flight.
+ *  - specvla_create reads every weight MATRIX once (wqkv, wo, wgu, wd, lm_head and the draft
+ *    model's fc / wqkv / wo / wgu / wd) and keeps its own repacked copy in the workspace; once it has
+ *    returned, those matrices may be freed or overwritten: two copies of a 7B model need not stay
+ *    resident. The embedding table and the norm gain vectors are read in place by every call and
+ *    must outlive the context.
  *  - Work is enqueued on `stream` (a cudaStream_t passed as void*). Calls that return
  *    values through host pointers synchronise that stream before returning.
  *  - One context per host thread; calls on one context must not overlap.

@@ -329,6 +329,38 @@ def test_chunk_loop_on_the_device_equals_the_loop_on_the_host(c0, wcuda, branch,
     assert dev["launches"] == host["launches"] + 2 + dev["it"]
 
 
+def test_weight_matrices_may_be_released_after_creation(c0, wcuda):
+    """The library keeps its own repacked copy of every weight matrix: once the context exists the
+    caller's matrices can go (here: overwritten with zeros); embedding and norm gains stay. Logits
+    (whole LM head), draft trees and the chunk are unchanged."""
+    from paper_2507_22424_b200.binding import make_shape
+    mine = {k: v.clone() for k, v in wcuda.items()}
+    gpu = _gpu(c0, mine)
+    shape = make_shape(c0["wl"].tree.branch, c0["wl"].tree.expand)
+    args = ([0], c0["embeds"].cuda(), c0["ids"].tolist(), [64])
+
+    def run():
+        first, logits = gpu.prefill(*args, want_logits=True)
+        tree = gpu.draft_tree([0], shape)[0]
+        given = dict(tokens=tree["tokens"], parent=tree["parent"], depth=tree["depth"])
+        m, emitted, vlogits = gpu.verify_tree([0], [given], 2, want_logits=True)
+        toks, _, _ = gpu.generate_action(*args, shape, 2, 7)
+        return first, logits.clone(), tree["tokens"], m, emitted, vlogits.clone(), toks
+
+    before = run()
+    kept = 0
+    for k, v in mine.items():
+        if v.dim() == 2 and "embed" not in k:
+            v.zero_()
+        else:
+            kept += 1
+    torch.cuda.synchronize()
+    after = run()
+    assert kept >= 2 and before[0] == after[0] and before[2:5] == after[2:5] and before[6] == after[6]
+    assert torch.equal(before[1], after[1]) and torch.equal(before[5], after[5])
+    gpu.close()
+
+
 def test_two_episodes_ragged_prefixes(c0, wcuda):
     """Two episodes with different prefix lengths (one of them with text ids, i.e. rows gathered
     from the embedding) in one prefill call and one verification call equal two separate oracle
