@@ -174,8 +174,10 @@ int specvla_destroy(specvla_ctx *ctx);
  *       and the appending of the emitted tokens until the chunk is complete; the host reads tokens,
  *       statistics and episode state back once. Applies when every iteration launches the same
  *       kernels (shape.prune = 0, no per-GEMM timing, per-GEMM forward) and the caches hold
- *       prefix + n_tokens + depth + tree rows; otherwise, and with 0, the host runs the loop and
- *       reads the accepted length back every iteration. Same tokens either way. */
+ *       prefix + n_tokens + depth + tree rows; otherwise, with 0, and when the driver refuses the
+ *       graph (remembered until this option is set again), the host runs the loop and reads the
+ *       accepted length back every iteration. Same tokens either way; specvla_stats.device_loop
+ *       says which loop ran. */
 #define SPECVLA_OPT_PERSISTENT_FORWARD 1
 #define SPECVLA_OPT_DEPENDENT_LAUNCH   2
 #define SPECVLA_OPT_L2_PREFETCH        3

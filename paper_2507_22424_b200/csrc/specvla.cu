@@ -136,6 +136,7 @@ struct specvla_ctx {
   // chunk loop on the device (specvla_generate_action): draft + verify + append as the body of a
   // CUDA-graph while node, captured once per (episodes, tree shape, r) and kept
   bool use_device_loop;
+  bool loop_unavailable;          // capturing or instantiating the loop graph failed once: the host runs the loop
   ChunkState *chunk;              // device
   ChunkState *pin_chunk;          // pinned copy read back after the loop, then max_episodes EpState
   cudaStream_t cap_stream;        // capture happens on a stream of the context's own
@@ -950,6 +951,7 @@ int specvla_create(const specvla_model_desc *desc, const specvla_weights *tw,
   ctx->pin_rows = reinterpret_cast<int *>(static_cast<char *>(ctx->pinned) + small_b + trees_b);
   ctx->pin_chunk = reinterpret_cast<ChunkState *>(static_cast<char *>(ctx->pinned) + small_b + trees_b + rows_b);
   ctx->use_device_loop = true;
+  ctx->loop_unavailable = false;
   ctx->cap_stream = nullptr;
   ctx->loop_graph = nullptr;
   ctx->loop_exec = nullptr;
@@ -1007,7 +1009,10 @@ int specvla_set_option(specvla_ctx *ctx, int option, long long value) {
   if (!ctx) return SPECVLA_ERR_INVALID_ARG;
   drop_loop_graph(ctx);
   switch (option) {
-    case SPECVLA_OPT_DEVICE_LOOP: ctx->use_device_loop = value != 0; break;
+    case SPECVLA_OPT_DEVICE_LOOP:
+      ctx->use_device_loop = value != 0;
+      ctx->loop_unavailable = false;
+      break;
     case SPECVLA_OPT_PERSISTENT_FORWARD: ctx->use_pk = value != 0; break;
     case SPECVLA_OPT_DEPENDENT_LAUNCH: ctx->use_pdl = value != 0; break;
     case SPECVLA_OPT_L2_PREFETCH: ctx->use_l2_prefetch = value != 0; break;
@@ -1522,11 +1527,6 @@ static int generate_on_device(specvla_ctx *ctx, int n_ep, const int *episodes, c
                               const int *token_ids, const int *lens, const specvla_tree_shape *shape, int n_nodes,
                               int n_tree_rows, int r, int n_tokens, int *tokens_out, specvla_stats *stats,
                               cudaStream_t st) {
-  const std::vector<int> key = loop_key_of(ctx, n_ep, episodes, shape, r);
-  if (!ctx->loop_exec || key != ctx->loop_key) {
-    TRY(build_loop_graph(ctx, n_ep, episodes, shape, n_nodes, n_tree_rows, r));
-    ctx->loop_key = key;
-  }
   float ms = 0.f;
   CU(cudaEventRecord(ctx->ev[0], st));
   TRY(prefill_enqueue(ctx, n_ep, episodes, embeds, token_ids, lens, nullptr, st));
@@ -1612,7 +1612,21 @@ int specvla_generate_action(specvla_ctx *ctx, int n_ep, const int *episodes, con
     on_device &= n_ep * rows <= d.max_rows && n_ep * rows <= ctx->max_lm_rows &&
                  n_ep * SV_MAX_PENDING <= d.max_rows && n_ep * 16 <= ctx->max_draft_rows;
   }
-  if (on_device) {
+  if (on_device && !ctx->loop_unavailable) {
+    // the graph of this (episodes, shape, r, options) combination: captured on first use and kept. If the
+    // driver refuses it, the host runs the loop from now on (specvla_stats.device_loop tells which ran).
+    const std::vector<int> key = loop_key_of(ctx, n_ep, episodes, shape, r);
+    if (!ctx->loop_exec || key != ctx->loop_key) {
+      if (build_loop_graph(ctx, n_ep, episodes, shape, n_nodes, n_tree_rows, r) == SPECVLA_OK)
+        ctx->loop_key = key;
+      else {
+        ctx->loop_unavailable = true;
+        drop_loop_graph(ctx);
+        cudaGetLastError();
+      }
+    }
+  }
+  if (on_device && !ctx->loop_unavailable) {
     TRY(generate_on_device(ctx, n_ep, episodes, embeds, token_ids, lens, shape, n_nodes, n_tree_rows, r, n_tokens,
                            tokens_out, stats, st));
     actions();
