@@ -274,8 +274,8 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     if (Q8) {
       // int8 -> bf16 expansion of every unit as it lands. NE groups of warps take the units in
       // turn (group g: units g, g + NE, ... into expanded buffer g), so that NE units are in
-      // expansion at once; a thread owns rows gt, gt + GT, ... of the tile (64 codes = 64 bytes in,
-      // one 128-byte swizzled row out).
+      // expansion at once; a thread owns every GT-th 16-byte piece of the codes (16 codes in, two
+      // 16-byte chunks of a 128-byte swizzled row out).
       constexpr int GT = q8_group_threads(TN);
       const int g = et / GT, gt = et - g * GT;
       auto group_sync = [&]() { asm volatile("bar.sync %0, %1;" ::"r"(2 + g), "n"(GT) : "memory"); };
@@ -294,23 +294,25 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
             break;
           }
           const uint32_t sC = base + RING0 + st * STAGE, sE = base + g * W_STAGE_BYTES;
-#pragma unroll 1
-          for (int r = gt; r < BM; r += GT) {
-            uint32_t c[16];
+          // A thread takes 16-byte pieces gt, gt + GT, ... of the unit's codes (piece p = codes
+          // 16 (p % 4) .. + 15 of row p / 4): consecutive lanes read consecutive shared memory, and
+          // the two 16-byte chunks each piece expands to land in their swizzled places.
+#pragma unroll 4
+          for (int p = gt; p < BM * 4; p += GT) {
+            const int r = p >> 2, q = p & 3;
+            uint32_t c[4];
+            asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(c[0]), "=r"(c[1]), "=r"(c[2]), "=r"(c[3]) : "r"(sC + p * 16) : "memory");
 #pragma unroll
-            for (int i = 0; i < 4; i++)
-              asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
-                           : "=r"(c[4 * i]), "=r"(c[4 * i + 1]), "=r"(c[4 * i + 2]), "=r"(c[4 * i + 3])
-                           : "r"(sC + r * 64 + i * 16) : "memory");
-#pragma unroll
-            for (int ch = 0; ch < 8; ch++) {
-              // codes 8 ch .. 8 ch + 7 of the row: two words -> eight bf16, exact (|code| <= 127), on
-              // the integer and FMA pipes only: code + 128 in the low mantissa byte of 2^23, minus
-              // (2^23 + 128), gives the code as fp32, whose upper half is its bf16 image
+            for (int h2 = 0; h2 < 2; h2++) {
+              // eight codes (two words) -> eight bf16, exact (|code| <= 127), on the integer and FMA
+              // pipes only: code + 128 in the low mantissa byte of 2^23, minus (2^23 + 128), gives the
+              // code as fp32, whose upper half is its bf16 image
+              const int ch = 2 * q + h2;
               uint32_t o[4];
 #pragma unroll
               for (int h = 0; h < 2; h++) {
-                const uint32_t x = c[2 * ch + h] ^ 0x80808080u;
+                const uint32_t x = c[2 * h2 + h] ^ 0x80808080u;
                 const float f0 = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7650)) - 8388736.f;
                 const float f1 = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7651)) - 8388736.f;
                 const float f2 = __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7652)) - 8388736.f;
