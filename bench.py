@@ -306,6 +306,14 @@ def c4_batch(weights, desc, steps=3):
             ms_p.append(tp)
             ms_v.append(tv)
             acc.append(sum(m) / n_ep)
+    # whole chunks for all episodes in one call each: the C1 tree (speculative) and no tree (autoregressive)
+    from paper_2507_22424_b200.binding import make_shape
+    chunk_rates = {}
+    for name, shp in (("speculative", make_shape(C.C1.tree.branch, C.C1.tree.expand)), ("autoregressive", make_shape((), ()))):
+        gpu.generate_action(eps, emb, ids, lens, shp, C.C4.extra["r"], C.C4.n_tokens)
+        (_, _, st), t = _timed(lambda: gpu.generate_action(eps, emb, ids, lens, shp, C.C4.extra["r"], C.C4.n_tokens))
+        chunk_rates[name] = dict(chunks_per_s=n_ep / (t * 1e-3), ms_per_call=t, iterations=st.iterations,
+                                 loop_on_device=bool(st.device_loop))
     gpu.close()
     mp, mv = statistics.median(ms_p), statistics.median(ms_v)
     rows_p, rows_v = sum(lens), 27 * n_ep
@@ -315,6 +323,7 @@ def c4_batch(weights, desc, steps=3):
                 prefill_tflops=2 * 6.607e9 * rows_p / mp / 1e9, verify_tflops=2 * 6.607e9 * rows_v / mv / 1e9,
                 prefill_frac_of_bf16_peak=2 * 6.607e9 * rows_p / mp / 1e9 / peak,
                 verify_frac_of_bf16_peak=2 * 6.607e9 * rows_v / mv / 1e9 / peak, mean_accept_len=statistics.mean(acc),
+                chunks_all_episodes=chunk_rates,
                 note="random trees (nothing planted): acceptance near zero; algorithmic flops, burst bf16 peak")
 
 
